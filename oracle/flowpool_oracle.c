@@ -1,0 +1,842 @@
+/*
+ * flowpool_oracle.c -- TEST INFRASTRUCTURE, not the product.
+ *
+ * A plain, slow, single-threaded CPU statement of what the unified-memory-pool
+ * hot path computes: GVA layout and page tables (paper Sec. 3.2), the page
+ * free ring, the producer write with its optional fp32->bf16 cast, the dynamic
+ * packing rule (Algorithm 1, Eq. 3) and the consumer's packed-microbatch
+ * assembly.  Arrays and loops only: no scans, no bitmaps, no blocking.  It
+ * shares nothing with the CUDA library (no header, no helper, no table); only
+ * tests, the smoke check and the benchmark's CPU-baseline leg may use it.
+ *
+ * Where the paper is silent the fixed rule used here is stated next to the
+ * code that applies it ("reading:").  Parts whose result the paper does not
+ * determine are marked "parity unpinned": GVA base constants, the page
+ * assignment order (free ring), the best-fit tie-break, the bucket rule, the
+ * bucket/tie orders of the zig-zag, and the NaN encoding of the cast.
+ */
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+/* ---- status codes (same numeric values as the library's public header;
+ *      retyped here on purpose, the two sides share no file) ---- */
+enum {
+  OR_OK = 0,
+  OR_ERR_INVALID_ARG = -1,
+  OR_ERR_POOL_EXHAUSTED = -2,
+  OR_ERR_UNKNOWN_SAMPLE = -3,
+  OR_ERR_ALREADY_WRITTEN = -4,
+  OR_ERR_NOT_READY = -5,
+  OR_ERR_TOO_LONG = -6,
+  OR_ERR_BAD_GVA = -7,
+  OR_ERR_PLACEHOLDER_MISMATCH = -8,
+  OR_ERR_BAD_TOKEN_ID = -9,
+  OR_ERR_SLOT_IN_USE = -10,
+  OR_ERR_CAPACITY = -11,
+  OR_ERR_CUDA = -12,
+  OR_ERR_TIMEOUT = -13
+};
+
+enum { OR_RING_SORTED = 0, OR_RING_SHUFFLED = 1 };
+enum { OR_BIND_IDENTITY = 0, OR_BIND_PERMUTED = 1 };
+enum { OR_BF16 = 0, OR_F32 = 1 };
+enum { OR_PLAN_ALLOW_UNWRITTEN = 1 };
+enum { SLOT_FREE = 0, SLOT_REGISTERED = 1, SLOT_READY = 2 };
+
+#define TEXT_PAGE_BYTES 4096u /* reading: token ids live in 4 KiB text pages */
+#define TEXT_PAGE_IDS 1024u
+
+typedef struct {
+  uint64_t page_bytes;
+  uint64_t hbm_pages, host_pages;
+  uint64_t max_text_tokens;
+  uint64_t ring_seed, bind_seed;
+  uint64_t gva_hbm_start, gva_host_start, max_size;
+  uint32_t hidden;
+  uint32_t max_samples, max_spans_per_sample, max_pages_per_span, max_seq_len;
+  int32_t placeholder_id;
+  uint32_t ring_order, bind_order;
+  uint32_t world_size, rank;
+} oracle_pool_config;
+
+typedef struct {
+  uint64_t coef_A, coef_B;
+  uint32_t budget_L, n_buckets_K, n_ranks_N, flags;
+} oracle_plan_config;
+
+typedef struct {
+  uint32_t pos_start, n_tokens;
+  uint32_t n_pages; /* 0 until written */
+  uint64_t* pages;  /* page GVAs, by ordinal */
+} or_span;
+
+typedef struct {
+  int state;
+  uint32_t seq_len, n_spans, spans_written;
+  uint64_t generation;
+  or_span* spans;
+  uint32_t n_text_pages;
+  uint64_t* text_pages; /* text-page GVAs */
+} or_sample;
+
+typedef struct oracle_pool {
+  oracle_pool_config c;
+  uint64_t P;        /* hbm_pages + host_pages */
+  uint8_t* hbm_mem;  /* backing frames, HBM tier */
+  uint8_t* host_mem; /* backing frames, DRAM tier */
+  uint8_t* text_mem; /* backing frames, text pages */
+  uint64_t* bind_hbm;  /* vpn -> frame */
+  uint64_t* bind_host; /* vpn -> frame */
+  /* FIFO ring of global page indices */
+  uint32_t* ring;
+  uint64_t ring_head, ring_count;
+  uint64_t n_text_pages;
+  uint32_t* tring;
+  uint64_t tring_head, tring_count;
+  or_sample* samples;
+  /* first asynchronous ("device-side") error: smallest (call, code, detail) */
+  uint64_t call_seq;
+  uint64_t status_key; /* UINT64_MAX = none */
+} oracle_pool;
+
+typedef struct oracle_plan {
+  oracle_plan_config c;
+  uint32_t n, n_mb;
+  uint32_t* slots;           /* [n] the caller's order */
+  uint64_t* slot_generation; /* [n] */
+  uint32_t* sample_len;      /* [n] */
+  uint64_t* sample_cost;     /* [n] */
+  uint32_t* sample_mb;       /* [n] */
+  uint32_t* mb_sample_off;   /* [n_mb+1] */
+  uint32_t* mb_samples;      /* [n] slots, microbatch-major, append order */
+  uint32_t* mb_tokens;       /* [n_mb] */
+  uint32_t* mb_lmax;         /* [n_mb] */
+  uint32_t* mb_residual;     /* [n_mb] */
+  uint64_t* mb_cost;         /* [n_mb] */
+  uint32_t* mb_bucket;       /* [n_mb] */
+  uint32_t* mb_rank;         /* [n_mb] */
+  uint32_t* rank_mb_off;     /* [N+1] */
+  uint32_t* rank_mbs;        /* [n_mb] dispatch order per rank */
+} oracle_plan;
+
+/* ------------------------------------------------------------------------
+ * Counter-based integer hash used for the seeded ring shuffle and the seeded
+ * vpn->frame permutation (both sides implement the same published mixer).
+ * ---------------------------------------------------------------------- */
+static uint64_t mix64(uint64_t z) {
+  z += 0x9E3779B97F4A7C15ull;
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+static uint64_t hash2(uint64_t seed, uint64_t i) { return mix64(seed ^ mix64(i)); }
+
+/* Fisher-Yates, i = n-1 .. 1, j = hash(seed, i) mod (i+1). */
+static void shuffle_u64(uint64_t* a, uint64_t n, uint64_t seed) {
+  for (uint64_t i = n; i-- > 1;) {
+    uint64_t j = hash2(seed, i) % (i + 1);
+    uint64_t t = a[i]; a[i] = a[j]; a[j] = t;
+  }
+}
+static void shuffle_u32(uint32_t* a, uint64_t n, uint64_t seed) {
+  for (uint64_t i = n; i-- > 1;) {
+    uint64_t j = hash2(seed, i) % (i + 1);
+    uint32_t t = a[i]; a[i] = a[j]; a[j] = t;
+  }
+}
+
+/* ------------------------------------------------------------------------
+ * G. GVA layout and translation (Sec. 3.2).
+ * Region t = [start_t, start_t + world_size*max_size); process i owns
+ * [start_t + i*max_size, start_t + (i+1)*max_size).  reading: half-open
+ * everywhere; defaults start_HBM = 2^44, start_DRAM = 2^45, max_size = 2^40
+ * (constants: parity unpinned, the paper gives none).  Page k of tier t of
+ * process i has GVA start_t + i*max_size + k*page_bytes; reading: the page
+ * table has one entry per pool page.  Text pages follow the embedding pages
+ * inside the HBM segment.
+ * ---------------------------------------------------------------------- */
+uint64_t oracle_segment_base(const oracle_pool* p, uint32_t tier, uint32_t proc) {
+  uint64_t start = tier == 0 ? p->c.gva_hbm_start : p->c.gva_host_start;
+  return start + (uint64_t)proc * p->c.max_size;
+}
+
+uint64_t oracle_page_gva(const oracle_pool* p, uint64_t global_page) {
+  if (global_page < p->c.hbm_pages)
+    return oracle_segment_base(p, 0, p->c.rank) + global_page * p->c.page_bytes;
+  return oracle_segment_base(p, 1, p->c.rank) + (global_page - p->c.hbm_pages) * p->c.page_bytes;
+}
+
+/* inverse of oracle_page_gva for a page-aligned GVA of this process */
+static uint64_t global_page_of_gva(const oracle_pool* p, uint64_t g) {
+  uint64_t host_base = oracle_segment_base(p, 1, p->c.rank);
+  if (g >= host_base && g < host_base + p->c.max_size) return p->c.hbm_pages + (g - host_base) / p->c.page_bytes;
+  return (g - oracle_segment_base(p, 0, p->c.rank)) / p->c.page_bytes;
+}
+
+static uint64_t text_page_gva(const oracle_pool* p, uint64_t k) {
+  return oracle_segment_base(p, 0, p->c.rank) + p->c.hbm_pages * p->c.page_bytes + k * TEXT_PAGE_BYTES;
+}
+
+/* kind: 0 = HBM embedding page, 1 = DRAM embedding page, 2 = text page. */
+int32_t oracle_translate(const oracle_pool* p, uint64_t g, uint32_t* kind, uint64_t* frame,
+                         uint64_t* offset) {
+  const uint64_t W = p->c.world_size, M = p->c.max_size, PS = p->c.page_bytes;
+  for (uint32_t t = 0; t < 2; ++t) {
+    uint64_t start = t == 0 ? p->c.gva_hbm_start : p->c.gva_host_start;
+    if (g < start || g >= start + W * M) continue;
+    uint64_t i = (g - start) / M, o = (g - start) % M;
+    if (i != p->c.rank) return OR_ERR_BAD_GVA; /* only this process's binding exists */
+    uint64_t pages = t == 0 ? p->c.hbm_pages : p->c.host_pages;
+    if (o < pages * PS) {
+      uint64_t vpn = o / PS;
+      *kind = t;
+      *frame = t == 0 ? p->bind_hbm[vpn] : p->bind_host[vpn];
+      *offset = o % PS;
+      return OR_OK;
+    }
+    if (t == 0) {
+      uint64_t ot = o - pages * PS;
+      if (ot < p->n_text_pages * (uint64_t)TEXT_PAGE_BYTES) {
+        *kind = 2; *frame = ot / TEXT_PAGE_BYTES; *offset = ot % TEXT_PAGE_BYTES;
+        return OR_OK;
+      }
+    }
+    return OR_ERR_BAD_GVA;
+  }
+  return OR_ERR_BAD_GVA;
+}
+
+static uint8_t* resolve(oracle_pool* p, uint64_t g) {
+  uint32_t kind; uint64_t frame, off;
+  if (oracle_translate(p, g, &kind, &frame, &off) != OR_OK) return NULL;
+  if (kind == 0) return p->hbm_mem + frame * p->c.page_bytes + off;
+  if (kind == 1) return p->host_mem + frame * p->c.page_bytes + off;
+  return p->text_mem + frame * TEXT_PAGE_BYTES + off;
+}
+
+static void note_async_error(oracle_pool* p, int32_t code, uint32_t detail) {
+  uint64_t key = (p->call_seq << 40) | ((uint64_t)(uint32_t)(-code) << 32) | detail;
+  if (key < p->status_key) p->status_key = key;
+}
+
+static uint64_t pages_for_tokens(const oracle_pool* p, uint64_t n_tokens) {
+  uint64_t bytes = n_tokens * 2ull * p->c.hidden;
+  return (bytes + p->c.page_bytes - 1) / p->c.page_bytes;
+}
+
+/* ------------------------------------------------------------------------
+ * Pool creation: lay out the regions, bind frames, fill the free rings.
+ * ---------------------------------------------------------------------- */
+int32_t oracle_pool_create(const oracle_pool_config* cfg, oracle_pool** out) {
+  if (!cfg || !out) return OR_ERR_INVALID_ARG;
+  oracle_pool_config c = *cfg;
+  if (c.gva_hbm_start == 0) c.gva_hbm_start = 1ull << 44;
+  if (c.gva_host_start == 0) c.gva_host_start = 1ull << 45;
+  if (c.max_size == 0) c.max_size = 1ull << 40;
+  if (c.world_size == 0) c.world_size = 1;
+  uint64_t PS = c.page_bytes;
+  if (PS < 4096 || PS > (2u << 20) || (PS & (PS - 1))) return OR_ERR_INVALID_ARG;
+  if (c.hidden == 0 || c.hidden % 8) return OR_ERR_INVALID_ARG;
+  if (c.hbm_pages + c.host_pages == 0) return OR_ERR_INVALID_ARG;
+  if (c.hbm_pages + c.host_pages > 0xFFFFFFFFull) return OR_ERR_INVALID_ARG;
+  if (c.rank >= c.world_size) return OR_ERR_INVALID_ARG;
+  if (c.max_samples == 0 || c.max_seq_len == 0) return OR_ERR_INVALID_ARG;
+  uint64_t n_text_pages = (c.max_text_tokens + TEXT_PAGE_IDS - 1) / TEXT_PAGE_IDS;
+  if (c.hbm_pages * PS + n_text_pages * TEXT_PAGE_BYTES > c.max_size) return OR_ERR_INVALID_ARG;
+  if (c.host_pages * PS > c.max_size) return OR_ERR_INVALID_ARG;
+  uint64_t span = (uint64_t)c.world_size * c.max_size;
+  if (c.gva_hbm_start + span < c.gva_hbm_start || c.gva_host_start + span < c.gva_host_start)
+    return OR_ERR_INVALID_ARG;
+  if (c.gva_hbm_start < c.gva_host_start + span && c.gva_host_start < c.gva_hbm_start + span)
+    return OR_ERR_INVALID_ARG; /* regions overlap */
+
+  oracle_pool* p = (oracle_pool*)calloc(1, sizeof(*p));
+  p->c = c;
+  p->P = c.hbm_pages + c.host_pages;
+  p->n_text_pages = n_text_pages;
+  p->hbm_mem = (uint8_t*)malloc(c.hbm_pages * PS + 1);
+  p->host_mem = (uint8_t*)malloc(c.host_pages * PS + 1);
+  p->text_mem = (uint8_t*)malloc(n_text_pages * TEXT_PAGE_BYTES + 1);
+  /* poison: an unwritten byte shows up as 0xFF in any comparison */
+  memset(p->hbm_mem, 0xFF, c.hbm_pages * PS);
+  memset(p->host_mem, 0xFF, c.host_pages * PS);
+  memset(p->text_mem, 0xFF, n_text_pages * TEXT_PAGE_BYTES);
+
+  /* binding: physical memory need not be contiguous; identity, or a seeded
+   * permutation per tier (reading; makes the table non-trivial) */
+  p->bind_hbm = (uint64_t*)malloc((c.hbm_pages + 1) * sizeof(uint64_t));
+  p->bind_host = (uint64_t*)malloc((c.host_pages + 1) * sizeof(uint64_t));
+  for (uint64_t k = 0; k < c.hbm_pages; ++k) p->bind_hbm[k] = k;
+  for (uint64_t k = 0; k < c.host_pages; ++k) p->bind_host[k] = k;
+  if (c.bind_order == OR_BIND_PERMUTED) {
+    shuffle_u64(p->bind_hbm, c.hbm_pages, c.bind_seed);
+    shuffle_u64(p->bind_host, c.host_pages, c.bind_seed + 1);
+  }
+
+  /* free ring over global page indices (parity unpinned: any assignment of
+   * free pages would be correct; this one is fixed so results are comparable) */
+  p->ring = (uint32_t*)malloc((p->P + 1) * sizeof(uint32_t));
+  for (uint64_t k = 0; k < p->P; ++k) p->ring[k] = (uint32_t)k;
+  if (c.ring_order == OR_RING_SHUFFLED) shuffle_u32(p->ring, p->P, c.ring_seed);
+  p->ring_head = 0; p->ring_count = p->P;
+
+  p->tring = (uint32_t*)malloc((n_text_pages + 1) * sizeof(uint32_t));
+  for (uint64_t k = 0; k < n_text_pages; ++k) p->tring[k] = (uint32_t)k;
+  p->tring_head = 0; p->tring_count = n_text_pages;
+
+  p->samples = (or_sample*)calloc(c.max_samples, sizeof(or_sample));
+  p->status_key = UINT64_MAX;
+  *out = p;
+  return OR_OK;
+}
+
+static void release_sample_storage(or_sample* s) {
+  if (s->spans) {
+    for (uint32_t i = 0; i < s->n_spans; ++i) free(s->spans[i].pages);
+    free(s->spans);
+  }
+  free(s->text_pages);
+  s->spans = NULL; s->text_pages = NULL;
+}
+
+int32_t oracle_pool_destroy(oracle_pool* p) {
+  if (!p) return OR_ERR_INVALID_ARG;
+  for (uint32_t i = 0; i < p->c.max_samples; ++i) release_sample_storage(&p->samples[i]);
+  free(p->samples); free(p->ring); free(p->tring); free(p->bind_hbm); free(p->bind_host);
+  free(p->hbm_mem); free(p->host_mem); free(p->text_mem); free(p);
+  return OR_OK;
+}
+
+/* ------------------------------------------------------------------------
+ * T. Register samples: text tokens and pairing metadata (Sec. 3.1: text
+ * tokens go into the same pool, lightweight metadata tracks the pairing).
+ * reading: a sample is input_ids[seq_len] in which span i occupies one run of
+ * placeholder ids starting at span_pos[i], n_tokens[i] long; runs sorted and
+ * non-overlapping.  All checks first, then the effect (all-or-nothing).
+ * ---------------------------------------------------------------------- */
+int32_t oracle_pool_register_samples(oracle_pool* p, uint32_t n, const uint32_t* slot,
+                                     const uint32_t* seq_len, const uint32_t* n_spans,
+                                     const uint32_t* span_pos, const uint32_t* span_tokens,
+                                     const int32_t* input_ids) {
+  if (!p) return OR_ERR_INVALID_ARG;
+  p->call_seq++;
+  if (n == 0) return OR_OK;
+  if (!slot || !seq_len || !n_spans || !input_ids) return OR_ERR_INVALID_ARG;
+  uint64_t text_need = 0, sp = 0;
+  for (uint32_t i = 0; i < n; ++i) {
+    if (slot[i] >= p->c.max_samples) return OR_ERR_INVALID_ARG;
+    if (p->samples[slot[i]].state != SLOT_FREE) return OR_ERR_SLOT_IN_USE;
+    for (uint32_t j = 0; j < i; ++j)
+      if (slot[j] == slot[i]) return OR_ERR_SLOT_IN_USE;
+    if (seq_len[i] == 0) return OR_ERR_INVALID_ARG;
+    if (seq_len[i] > p->c.max_seq_len) return OR_ERR_CAPACITY;
+    if (n_spans[i] > p->c.max_spans_per_sample) return OR_ERR_CAPACITY;
+    if (n_spans[i] && (!span_pos || !span_tokens)) return OR_ERR_INVALID_ARG;
+    uint64_t prev_end = 0;
+    for (uint32_t j = 0; j < n_spans[i]; ++j, ++sp) {
+      if (span_tokens[sp] == 0) return OR_ERR_INVALID_ARG;
+      if ((uint64_t)span_pos[sp] + span_tokens[sp] > seq_len[i]) return OR_ERR_INVALID_ARG;
+      if (span_pos[sp] < prev_end) return OR_ERR_INVALID_ARG;
+      prev_end = (uint64_t)span_pos[sp] + span_tokens[sp];
+      if (pages_for_tokens(p, span_tokens[sp]) > p->c.max_pages_per_span) return OR_ERR_CAPACITY;
+    }
+    text_need += (seq_len[i] + TEXT_PAGE_IDS - 1) / TEXT_PAGE_IDS;
+  }
+  if (text_need > p->tring_count) return OR_ERR_CAPACITY;
+
+  sp = 0;
+  uint64_t idoff = 0;
+  for (uint32_t i = 0; i < n; ++i) {
+    or_sample* s = &p->samples[slot[i]];
+    s->state = n_spans[i] == 0 ? SLOT_READY : SLOT_REGISTERED; /* text-only: paired at once */
+    s->seq_len = seq_len[i]; s->n_spans = n_spans[i]; s->spans_written = 0;
+    s->spans = (or_span*)calloc(n_spans[i] + 1, sizeof(or_span));
+    uint64_t placeholders = 0;
+    int bad = 0;
+    for (uint32_t j = 0; j < n_spans[i]; ++j, ++sp) {
+      s->spans[j].pos_start = span_pos[sp];
+      s->spans[j].n_tokens = span_tokens[sp];
+      placeholders += span_tokens[sp];
+      for (uint32_t t = 0; t < span_tokens[sp]; ++t)
+        if (input_ids[idoff + span_pos[sp] + t] != p->c.placeholder_id) bad = 1;
+    }
+    uint64_t seen = 0;
+    for (uint32_t t = 0; t < seq_len[i]; ++t)
+      if (input_ids[idoff + t] == p->c.placeholder_id) ++seen;
+    if (seen != placeholders) bad = 1; /* stray placeholder outside every run */
+    if (bad) note_async_error(p, OR_ERR_PLACEHOLDER_MISMATCH, slot[i]);
+    /* ids into text pages popped from the text ring, page by page */
+    s->n_text_pages = (seq_len[i] + TEXT_PAGE_IDS - 1) / TEXT_PAGE_IDS;
+    s->text_pages = (uint64_t*)malloc(s->n_text_pages * sizeof(uint64_t));
+    for (uint32_t k = 0; k < s->n_text_pages; ++k) {
+      uint32_t tp = p->tring[p->tring_head];
+      p->tring_head = (p->tring_head + 1) % p->n_text_pages; p->tring_count--;
+      s->text_pages[k] = text_page_gva(p, tp);
+    }
+    for (uint32_t t = 0; t < seq_len[i]; ++t) {
+      uint8_t* dst = resolve(p, s->text_pages[t / TEXT_PAGE_IDS] + (uint64_t)(t % TEXT_PAGE_IDS) * 4);
+      memcpy(dst, &input_ids[idoff + t], 4);
+    }
+    idoff += seq_len[i];
+  }
+  return OR_OK;
+}
+
+/* ------------------------------------------------------------------------
+ * W. fp32 -> bf16, IEEE round-to-nearest-even on the bit pattern; denormals
+ * kept; overflow rounds to +-Inf.  reading (parity unpinned): every NaN
+ * becomes the sign-preserving quiet NaN 0x7FC0 / 0xFFC0.
+ * ---------------------------------------------------------------------- */
+uint16_t oracle_f32_to_bf16_rne(uint32_t u) {
+  if ((u & 0x7FFFFFFFu) > 0x7F800000u) return (uint16_t)(((u >> 16) & 0x8000u) | 0x7FC0u);
+  return (uint16_t)((u + 0x7FFFu + ((u >> 16) & 1u)) >> 16);
+}
+
+/* ------------------------------------------------------------------------
+ * F + W. Producer write (Sec. 3.1, 3.2: encoders place embeddings into their
+ * own segment of the pool).  Page allocation: span q of the call takes the
+ * next ceil(n_tokens*2H / page_bytes) entries from the ring head, spans in
+ * argument order; whole pages per span.  Byte b of the span's bf16 row-major
+ * [n_tokens, H] image lives in page b / page_bytes at offset b % page_bytes;
+ * the tail of the last page keeps whatever it held.
+ * ---------------------------------------------------------------------- */
+int32_t oracle_pool_write_embeddings(oracle_pool* p, uint32_t n_spans, const uint32_t* slot,
+                                     const uint32_t* span_idx, const uint32_t* n_tokens,
+                                     const void* const* src, uint32_t src_dtype) {
+  if (!p) return OR_ERR_INVALID_ARG;
+  p->call_seq++;
+  if (src_dtype != OR_BF16 && src_dtype != OR_F32) return OR_ERR_INVALID_ARG;
+  if (n_spans == 0) return OR_OK;
+  if (!slot || !span_idx || !n_tokens || !src) return OR_ERR_INVALID_ARG;
+  uint64_t need = 0;
+  for (uint32_t q = 0; q < n_spans; ++q) {
+    if (slot[q] >= p->c.max_samples) return OR_ERR_INVALID_ARG;
+    or_sample* s = &p->samples[slot[q]];
+    if (s->state == SLOT_FREE) return OR_ERR_UNKNOWN_SAMPLE;
+    if (span_idx[q] >= s->n_spans) return OR_ERR_INVALID_ARG;
+    if (n_tokens[q] != s->spans[span_idx[q]].n_tokens) return OR_ERR_INVALID_ARG;
+    if (!src[q]) return OR_ERR_INVALID_ARG;
+    if (s->spans[span_idx[q]].n_pages != 0) return OR_ERR_ALREADY_WRITTEN;
+    for (uint32_t r = 0; r < q; ++r)
+      if (slot[r] == slot[q] && span_idx[r] == span_idx[q]) return OR_ERR_ALREADY_WRITTEN;
+    need += pages_for_tokens(p, n_tokens[q]);
+  }
+  if (need > p->ring_count) return OR_ERR_POOL_EXHAUSTED;
+
+  const uint64_t PS = p->c.page_bytes, H = p->c.hidden;
+  for (uint32_t q = 0; q < n_spans; ++q) {
+    or_sample* s = &p->samples[slot[q]];
+    or_span* sp = &s->spans[span_idx[q]];
+    uint64_t k = pages_for_tokens(p, n_tokens[q]);
+    sp->n_pages = (uint32_t)k;
+    sp->pages = (uint64_t*)malloc(k * sizeof(uint64_t));
+    for (uint64_t o = 0; o < k; ++o) {
+      uint32_t g = p->ring[p->ring_head];
+      p->ring_head = (p->ring_head + 1) % p->P; p->ring_count--;
+      sp->pages[o] = oracle_page_gva(p, g);
+    }
+    uint64_t n_bytes = (uint64_t)n_tokens[q] * H * 2, b = 0;
+    while (b < n_bytes) { /* maximal run inside one page (page_bytes is even: no element straddles) */
+      uint64_t off = b % PS;
+      uint64_t run = PS - off < n_bytes - b ? PS - off : n_bytes - b;
+      uint8_t* dst = resolve(p, sp->pages[b / PS] + off);
+      if (src_dtype == OR_BF16) {
+        memcpy(dst, (const uint8_t*)src[q] + b, run);
+      } else {
+        for (uint64_t e = 0; e < run / 2; ++e) {
+          uint16_t v = oracle_f32_to_bf16_rne(((const uint32_t*)src[q])[b / 2 + e]);
+          memcpy(dst + 2 * e, &v, 2);
+        }
+      }
+      b += run;
+    }
+    s->spans_written++;
+    if (s->spans_written == s->n_spans) s->state = SLOT_READY; /* "paired" */
+  }
+  return OR_OK;
+}
+
+/* ------------------------------------------------------------------------
+ * F. Free: samples in argument order, spans by index, pages by ordinal, each
+ * pushed to the ring tail; the slot returns to FREE.
+ * ---------------------------------------------------------------------- */
+int32_t oracle_pool_free(oracle_pool* p, const uint32_t* slot, uint32_t n) {
+  if (!p) return OR_ERR_INVALID_ARG;
+  p->call_seq++;
+  if (n == 0) return OR_OK;
+  if (!slot) return OR_ERR_INVALID_ARG;
+  for (uint32_t i = 0; i < n; ++i) {
+    if (slot[i] >= p->c.max_samples) return OR_ERR_INVALID_ARG;
+    if (p->samples[slot[i]].state == SLOT_FREE) return OR_ERR_UNKNOWN_SAMPLE;
+    for (uint32_t j = 0; j < i; ++j)
+      if (slot[j] == slot[i]) return OR_ERR_UNKNOWN_SAMPLE;
+  }
+  for (uint32_t i = 0; i < n; ++i) {
+    or_sample* s = &p->samples[slot[i]];
+    for (uint32_t j = 0; j < s->n_spans; ++j)
+      for (uint32_t o = 0; o < s->spans[j].n_pages; ++o) {
+        uint64_t idx = global_page_of_gva(p, s->spans[j].pages[o]);
+        p->ring[(p->ring_head + p->ring_count) % p->P] = (uint32_t)idx;
+        p->ring_count++;
+      }
+    for (uint32_t k = 0; k < s->n_text_pages; ++k) {
+      uint64_t tp = (s->text_pages[k] - text_page_gva(p, 0)) / TEXT_PAGE_BYTES;
+      p->tring[(p->tring_head + p->tring_count) % p->n_text_pages] = (uint32_t)tp;
+      p->tring_count++;
+    }
+    release_sample_storage(s);
+    s->state = SLOT_FREE; s->n_spans = 0; s->seq_len = 0; s->spans_written = 0; s->n_text_pages = 0;
+    s->generation++;
+  }
+  return OR_OK;
+}
+
+/* ------------------------------------------------------------------------
+ * P. Dynamic packing (Algorithm 1, Eq. 3).
+ * ---------------------------------------------------------------------- */
+
+/* Best-fit packing, Algorithm 1 lines 1-11, as the definition the segment
+ * tree accelerates: the open microbatch with the smallest residual >= l.
+ * reading (tie-break, parity unpinned): among equal residuals, the one whose
+ * residual changed most recently.  reading: l_min = the smallest length of
+ * this call, so the removal step (lines 10-11) never changes the result and
+ * is omitted here; oracle_bestfit_segment_tree below performs it literally. */
+static uint32_t best_fit(uint32_t n, const uint32_t* len, uint32_t L, uint32_t* sample_mb,
+                         uint32_t* P, uint32_t* tokens, uint32_t* lmax, uint32_t* count) {
+  uint32_t n_mb = 0;
+  uint32_t* stamp = (uint32_t*)malloc((n + 1) * sizeof(uint32_t));
+  for (uint32_t t = 0; t < n; ++t) {
+    uint32_t l = len[t];
+    int64_t best = -1;
+    for (uint32_t j = 0; j < n_mb; ++j) {
+      if (P[j] < l) continue;
+      if (best < 0 || P[j] < P[best] || (P[j] == P[best] && stamp[j] > stamp[best])) best = j;
+    }
+    uint32_t j;
+    if (best >= 0) {
+      j = (uint32_t)best;
+      P[j] -= l; tokens[j] += l; if (l > lmax[j]) lmax[j] = l; count[j]++;
+    } else {
+      j = n_mb++;
+      P[j] = L - l; tokens[j] = l; lmax[j] = l; count[j] = 1;
+    }
+    stamp[j] = t;
+    sample_mb[t] = j;
+  }
+  free(stamp);
+  return n_mb;
+}
+
+/* Second, literal statement of Algorithm 1 lines 1-11: a segment tree over
+ * the residual values [0, L]; leaf r holds the open microbatches whose
+ * residual is r (most recently changed on top), an inner node the largest
+ * non-empty residual below it; the query prefers the left (smaller) subtree
+ * whenever its maximum is >= l; a microbatch whose residual drops below l_min
+ * is removed.  Returns n_mb; used by tests to pin best_fit. */
+uint32_t oracle_bestfit_segment_tree(uint32_t n, const uint32_t* len, uint32_t L, uint32_t l_min,
+                                     uint32_t* sample_mb) {
+  uint32_t leaves = 1; while (leaves < L + 1) leaves <<= 1;
+  int64_t* node = (int64_t*)malloc(2ull * leaves * sizeof(int64_t));
+  for (uint32_t i = 0; i < 2 * leaves; ++i) node[i] = -1;
+  int64_t* top = (int64_t*)malloc(((uint64_t)L + 1) * sizeof(int64_t)); /* stack top per residual */
+  for (uint32_t r = 0; r <= L; ++r) top[r] = -1;
+  int64_t* below = (int64_t*)malloc(((uint64_t)n + 1) * sizeof(int64_t));
+  uint32_t* P = (uint32_t*)malloc(((uint64_t)n + 1) * sizeof(uint32_t));
+  uint32_t n_mb = 0;
+  for (uint32_t t = 0; t < n; ++t) {
+    uint32_t l = len[t];
+    int64_t j = -1;
+    if (node[1] >= (int64_t)l) {
+      uint32_t v = 1;
+      while (v < leaves) v = node[2 * v] >= (int64_t)l ? 2 * v : 2 * v + 1;
+      uint32_t r = v - leaves;
+      j = top[r];
+      top[r] = below[j]; /* take it off leaf r */
+      if (top[r] < 0) { node[v] = -1; for (v >>= 1; v >= 1; v >>= 1) node[v] = node[2*v] > node[2*v+1] ? node[2*v] : node[2*v+1]; }
+      P[j] -= l;
+    } else {
+      j = n_mb++;
+      P[j] = L - l;
+    }
+    sample_mb[t] = (uint32_t)j;
+    if (P[j] >= l_min) { /* (re)insert at its new residual unless removed */
+      uint32_t r = P[j];
+      below[j] = top[r]; top[r] = j;
+      uint32_t v = leaves + r; node[v] = r;
+      for (v >>= 1; v >= 1; v >>= 1) node[v] = node[2*v] > node[2*v+1] ? node[2*v] : node[2*v+1];
+    }
+  }
+  free(node); free(top); free(below); free(P);
+  return n_mb;
+}
+
+/* Eq. 3 scaled to integers: A*sum(l) + B*lmax^2; with (A,B) = (L,1) this is
+ * L^2 * Cost(B_j) exactly.  The quadratic term is lmax^2, as printed. */
+uint64_t oracle_cost_int(uint64_t A, uint64_t B, uint64_t sum_len, uint64_t lmax) {
+  return A * sum_len + B * lmax * lmax;
+}
+
+/* Two-dimension load balancing, Algorithm 1 lines 12-27, on given costs.
+ * Outputs: bucket[n_mb], rank[n_mb], rank_mb_off[N+1], rank_mbs[n_mb]. */
+void oracle_balance(uint32_t n_mb, const uint64_t* cost, uint32_t K, uint32_t N, uint32_t* bucket,
+                    uint32_t* rank, uint32_t* rank_mb_off, uint32_t* rank_mbs) {
+  /* lines 12-14: buckets.  reading (parity unpinned): equal-width
+   * quantisation of the observed cost range into K buckets. */
+  uint64_t lo = UINT64_MAX, hi = 0;
+  for (uint32_t j = 0; j < n_mb; ++j) {
+    if (cost[j] < lo) lo = cost[j];
+    if (cost[j] > hi) hi = cost[j];
+  }
+  for (uint32_t j = 0; j < n_mb; ++j) {
+    /* (cost-lo)*K / (hi-lo+1), in 128-bit so nothing overflows */
+    unsigned __int128 num = (unsigned __int128)(cost[j] - lo) * K;
+    bucket[j] = (uint32_t)(num / ((unsigned __int128)(hi - lo) + 1));
+  }
+  /* lines 15-27: per bucket (reading: highest bucket first), sort by cost
+   * descending (reading: ties by microbatch index ascending), then deal
+   * Rank_0..Rank_{N-1}, reverse, and so on; a and Forward restart per bucket;
+   * reading: the deal stops when the list is exhausted. */
+  uint32_t* list = (uint32_t*)calloc((size_t)n_mb + 1, sizeof(uint32_t));
+  uint32_t* order = (uint32_t*)calloc((size_t)n_mb + 1, sizeof(uint32_t)); /* global dispatch order */
+  uint32_t n_order = 0;
+  for (int64_t k = (int64_t)K - 1; k >= 0; --k) {
+    uint32_t m = 0;
+    for (uint32_t j = 0; j < n_mb; ++j)
+      if (bucket[j] == (uint32_t)k) list[m++] = j;
+    for (uint32_t i = 1; i < m; ++i) { /* insertion sort: stable, so index order survives ties */
+      uint32_t x = list[i]; int64_t h = (int64_t)i - 1;
+      while (h >= 0 && cost[list[h]] < cost[x]) { list[h + 1] = list[h]; --h; }
+      list[h + 1] = x;
+    }
+    uint32_t a = 0; int forward = 1;
+    while (a < m) {
+      if (forward) { for (uint32_t r = 0; r < N && a < m; ++r) { rank[list[a]] = r; order[n_order++] = list[a]; ++a; } }
+      else { for (int64_t r = (int64_t)N - 1; r >= 0 && a < m; --r) { rank[list[a]] = (uint32_t)r; order[n_order++] = list[a]; ++a; } }
+      forward = !forward;
+    }
+  }
+  /* per-rank lists, in the order the microbatches were dealt */
+  rank_mb_off[0] = 0;
+  for (uint32_t r = 0; r < N; ++r) {
+    rank_mb_off[r + 1] = rank_mb_off[r];
+    for (uint32_t i = 0; i < n_order; ++i)
+      if (rank[order[i]] == r) rank_mbs[rank_mb_off[r + 1]++] = order[i];
+  }
+  free(list); free(order);
+}
+
+void oracle_plan_destroy_inner(oracle_plan* pl) {
+  free(pl->slots); free(pl->slot_generation); free(pl->sample_len); free(pl->sample_cost);
+  free(pl->sample_mb); free(pl->mb_sample_off); free(pl->mb_samples); free(pl->mb_tokens);
+  free(pl->mb_lmax); free(pl->mb_residual); free(pl->mb_cost); free(pl->mb_bucket);
+  free(pl->mb_rank); free(pl->rank_mb_off); free(pl->rank_mbs);
+}
+int32_t oracle_plan_destroy(oracle_plan* pl) {
+  if (!pl) return OR_ERR_INVALID_ARG;
+  oracle_plan_destroy_inner(pl); free(pl);
+  return OR_OK;
+}
+
+/* Packing + load balancing over explicit lengths (no pool needed): the whole
+ * of Algorithm 1.  slots may be NULL (then sample t is "slot" t). */
+int32_t oracle_plan_from_lengths(const uint32_t* slots, const uint32_t* len, uint32_t n,
+                                 const oracle_plan_config* cfg, oracle_plan** out) {
+  if (!cfg || !out) return OR_ERR_INVALID_ARG;
+  const uint32_t L = cfg->budget_L, K = cfg->n_buckets_K, N = cfg->n_ranks_N;
+  if (L == 0 || K == 0 || N == 0) return OR_ERR_INVALID_ARG;
+  for (uint32_t t = 0; t < n; ++t) {
+    if (len[t] == 0) return OR_ERR_INVALID_ARG;
+    if (len[t] > L) return OR_ERR_TOO_LONG;
+  }
+  oracle_plan* pl = (oracle_plan*)calloc(1, sizeof(*pl));
+  pl->c = *cfg; pl->n = n;
+#define ALLOC(T, cnt) (T*)calloc((size_t)(cnt) + 1, sizeof(T))
+  pl->slots = ALLOC(uint32_t, n); pl->slot_generation = ALLOC(uint64_t, n);
+  pl->sample_len = ALLOC(uint32_t, n); pl->sample_cost = ALLOC(uint64_t, n);
+  pl->sample_mb = ALLOC(uint32_t, n); pl->mb_samples = ALLOC(uint32_t, n);
+  pl->mb_sample_off = ALLOC(uint32_t, n + 1);
+  pl->mb_tokens = ALLOC(uint32_t, n); pl->mb_lmax = ALLOC(uint32_t, n);
+  pl->mb_residual = ALLOC(uint32_t, n); pl->mb_cost = ALLOC(uint64_t, n);
+  pl->mb_bucket = ALLOC(uint32_t, n); pl->mb_rank = ALLOC(uint32_t, n);
+  pl->rank_mb_off = ALLOC(uint32_t, N + 1); pl->rank_mbs = ALLOC(uint32_t, n);
+  uint32_t* count = ALLOC(uint32_t, n);
+  for (uint32_t t = 0; t < n; ++t) {
+    pl->slots[t] = slots ? slots[t] : t;
+    pl->sample_len[t] = len[t];
+    /* per-sample score: Eq. 3 on a singleton microbatch */
+    pl->sample_cost[t] = oracle_cost_int(cfg->coef_A, cfg->coef_B, len[t], len[t]);
+  }
+  /* lines 1-11 */
+  uint32_t n_mb = best_fit(n, len, L, pl->sample_mb, pl->mb_residual, pl->mb_tokens, pl->mb_lmax, count);
+  pl->n_mb = n_mb;
+  /* samples inside a microbatch stay in arrival order (line 5: append) */
+  for (uint32_t j = 0; j < n_mb; ++j) pl->mb_sample_off[j + 1] = pl->mb_sample_off[j] + count[j];
+  for (uint32_t j = 0; j < n_mb; ++j) {
+    uint32_t w = pl->mb_sample_off[j];
+    for (uint32_t t = 0; t < n; ++t)
+      if (pl->sample_mb[t] == j) pl->mb_samples[w++] = pl->slots[t];
+  }
+  /* lines 12-14: Cost(B_j) */
+  for (uint32_t j = 0; j < n_mb; ++j)
+    pl->mb_cost[j] = oracle_cost_int(cfg->coef_A, cfg->coef_B, pl->mb_tokens[j], pl->mb_lmax[j]);
+  /* lines 12-27: buckets and zig-zag dispatch */
+  oracle_balance(n_mb, pl->mb_cost, K, N, pl->mb_bucket, pl->mb_rank, pl->rank_mb_off, pl->rank_mbs);
+  free(count);
+  *out = pl;
+  return OR_OK;
+}
+
+int32_t oracle_pool_plan_microbatches(oracle_pool* p, const uint32_t* slots, uint32_t n,
+                                      const oracle_plan_config* cfg, oracle_plan** out) {
+  if (!p || !cfg || !out) return OR_ERR_INVALID_ARG;
+  p->call_seq++;
+  if (cfg->budget_L == 0 || cfg->n_buckets_K == 0 || cfg->n_ranks_N == 0) return OR_ERR_INVALID_ARG;
+  if (n && !slots) return OR_ERR_INVALID_ARG;
+  uint32_t* len = (uint32_t*)calloc((size_t)n + 1, sizeof(uint32_t));
+  uint8_t* seen = (uint8_t*)calloc(p->c.max_samples, 1);
+  int32_t rc = OR_OK;
+  for (uint32_t t = 0; t < n && rc == OR_OK; ++t) {
+    if (slots[t] >= p->c.max_samples) { rc = OR_ERR_INVALID_ARG; break; }
+    or_sample* s = &p->samples[slots[t]];
+    if (s->state == SLOT_FREE) rc = OR_ERR_UNKNOWN_SAMPLE;
+    else if (seen[slots[t]]) rc = OR_ERR_INVALID_ARG;
+    else if (s->state != SLOT_READY && !(cfg->flags & OR_PLAN_ALLOW_UNWRITTEN)) rc = OR_ERR_NOT_READY;
+    else if (s->seq_len > cfg->budget_L) rc = OR_ERR_TOO_LONG;
+    seen[slots[t]] = 1;
+    len[t] = s->seq_len; /* l(s): the LLM-side length, text + all vision tokens */
+  }
+  if (rc == OR_OK) rc = oracle_plan_from_lengths(slots, len, n, cfg, out);
+  if (rc == OR_OK)
+    for (uint32_t t = 0; t < n; ++t) (*out)->slot_generation[t] = p->samples[slots[t]].generation;
+  free(len); free(seen);
+  return rc;
+}
+
+/* ------------------------------------------------------------------------
+ * A. Packed assembly (Sec. 3.1-3.2: the backbone consumes microbatches by
+ * GVA; Sec. 4.1: image and text subsequences are interleaved).
+ * Output row cu_seqlens[q] + p of a microbatch = row (p - pos_start) of the
+ * span whose placeholder run contains p, read through the span's page list
+ * and the page table; otherwise embed_table[input_ids[p]].  position id = p.
+ * ---------------------------------------------------------------------- */
+int32_t oracle_pool_gather_packed(oracle_pool* p, const oracle_plan* pl, uint32_t mb_begin,
+                                  uint32_t mb_end, const void* embed_table, uint32_t vocab,
+                                  void* out_embeds, int32_t* out_cu_seqlens,
+                                  int32_t* out_position_ids) {
+  if (!p || !pl) return OR_ERR_INVALID_ARG;
+  p->call_seq++;
+  if (mb_begin > mb_end || mb_end > pl->n_mb) return OR_ERR_INVALID_ARG;
+  for (uint32_t t = 0; t < pl->n; ++t) {
+    or_sample* s = &p->samples[pl->slots[t]];
+    if (s->state != SLOT_READY || s->generation != pl->slot_generation[t]) return OR_ERR_NOT_READY;
+  }
+  if (mb_begin == mb_end) return OR_OK;
+  if (!embed_table || !out_embeds || !out_cu_seqlens || !out_position_ids) return OR_ERR_INVALID_ARG;
+  const uint64_t PS = p->c.page_bytes, row_bytes = 2ull * p->c.hidden;
+  uint8_t* out = (uint8_t*)out_embeds;
+  uint64_t row = 0, cu_w = 0;
+  for (uint32_t j = mb_begin; j < mb_end; ++j) {
+    int32_t cu = 0;
+    out_cu_seqlens[cu_w++] = 0;
+    for (uint32_t qi = pl->mb_sample_off[j]; qi < pl->mb_sample_off[j + 1]; ++qi) {
+      or_sample* s = &p->samples[pl->mb_samples[qi]];
+      for (uint32_t pos = 0; pos < s->seq_len; ++pos, ++row) {
+        int32_t id;
+        memcpy(&id, resolve(p, s->text_pages[pos / TEXT_PAGE_IDS] + (uint64_t)(pos % TEXT_PAGE_IDS) * 4), 4);
+        out_position_ids[row] = (int32_t)pos;
+        const or_span* sp = NULL;
+        for (uint32_t i = 0; i < s->n_spans; ++i)
+          if (pos >= s->spans[i].pos_start && pos < s->spans[i].pos_start + s->spans[i].n_tokens) sp = &s->spans[i];
+        uint8_t* dst = out + row * row_bytes;
+        if (sp) {
+          uint64_t b = (uint64_t)(pos - sp->pos_start) * row_bytes;
+          uint64_t done = 0;
+          while (done < row_bytes) { /* maximal run inside one page */
+            uint64_t off = (b + done) % PS;
+            uint64_t run = PS - off < row_bytes - done ? PS - off : row_bytes - done;
+            uint8_t* src = resolve(p, sp->pages[(b + done) / PS] + off);
+            if (!src) { note_async_error(p, OR_ERR_BAD_GVA, (uint32_t)row); break; }
+            memcpy(dst + done, src, run);
+            done += run;
+          }
+        } else if (id < 0 || (uint32_t)id >= vocab) {
+          note_async_error(p, OR_ERR_BAD_TOKEN_ID, (uint32_t)row); /* row left untouched */
+        } else {
+          memcpy(dst, (const uint8_t*)embed_table + (uint64_t)id * row_bytes, row_bytes);
+        }
+      }
+      cu += (int32_t)s->seq_len;
+      out_cu_seqlens[cu_w++] = cu;
+    }
+  }
+  return OR_OK;
+}
+
+/* ---- accessors for the harness ---- */
+int32_t oracle_pool_status(oracle_pool* p, int32_t* code, uint64_t* detail) {
+  if (!p) return OR_ERR_INVALID_ARG;
+  if (p->status_key == UINT64_MAX) { if (code) *code = 0; if (detail) *detail = 0; return OR_OK; }
+  if (code) *code = -(int32_t)((p->status_key >> 32) & 0xFF);
+  if (detail) *detail = p->status_key & 0xFFFFFFFFull;
+  p->status_key = UINT64_MAX;
+  return OR_OK;
+}
+
+int32_t oracle_pool_debug_span_pages(oracle_pool* p, uint32_t slot, uint32_t span, uint64_t* gva_out,
+                                     uint32_t cap, uint32_t* n) {
+  if (!p || slot >= p->c.max_samples) return OR_ERR_INVALID_ARG;
+  or_sample* s = &p->samples[slot];
+  if (s->state == SLOT_FREE) return OR_ERR_UNKNOWN_SAMPLE;
+  if (span >= s->n_spans) return OR_ERR_INVALID_ARG;
+  if (n) *n = s->spans[span].n_pages;
+  for (uint32_t o = 0; o < s->spans[span].n_pages && o < cap; ++o) gva_out[o] = s->spans[span].pages[o];
+  return OR_OK;
+}
+
+int32_t oracle_pool_free_pages(oracle_pool* p, uint64_t* n_free, uint64_t* n_text_free) {
+  if (!p) return OR_ERR_INVALID_ARG;
+  if (n_free) *n_free = p->ring_count;
+  if (n_text_free) *n_text_free = p->tring_count;
+  return OR_OK;
+}
+
+/* the ring's current content, head first */
+int32_t oracle_pool_debug_ring(oracle_pool* p, uint32_t* out, uint64_t cap, uint64_t* n) {
+  if (!p) return OR_ERR_INVALID_ARG;
+  if (n) *n = p->ring_count;
+  for (uint64_t i = 0; i < p->ring_count && i < cap; ++i) out[i] = p->ring[(p->ring_head + i) % p->P];
+  return OR_OK;
+}
+
+/* raw byte of a backing tier, for read-back checks: kind 0 HBM, 1 DRAM */
+const uint8_t* oracle_pool_backing(oracle_pool* p, uint32_t kind) {
+  return kind == 0 ? p->hbm_mem : kind == 1 ? p->host_mem : p->text_mem;
+}
+
+int32_t oracle_plan_summary(const oracle_plan* pl, uint32_t* n_mb, uint64_t* total_tokens, uint32_t* max_mb_tokens) {
+  if (!pl) return OR_ERR_INVALID_ARG;
+  uint64_t tot = 0; uint32_t mx = 0;
+  for (uint32_t j = 0; j < pl->n_mb; ++j) { tot += pl->mb_tokens[j]; if (pl->mb_tokens[j] > mx) mx = pl->mb_tokens[j]; }
+  if (n_mb) *n_mb = pl->n_mb;
+  if (total_tokens) *total_tokens = tot;
+  if (max_mb_tokens) *max_mb_tokens = mx;
+  return OR_OK;
+}
+
+/* copies every plan array out; any pointer may be NULL */
+int32_t oracle_plan_arrays(const oracle_plan* pl, uint32_t* mb_sample_off, uint32_t* mb_samples,
+                           uint32_t* mb_tokens, uint32_t* mb_lmax, uint32_t* mb_residual,
+                           uint64_t* mb_cost, uint32_t* mb_bucket, uint32_t* mb_rank,
+                           uint32_t* rank_mb_off, uint32_t* rank_mbs, uint64_t* sample_cost,
+                           uint32_t* sample_mb) {
+  if (!pl) return OR_ERR_INVALID_ARG;
+  const uint32_t n = pl->n, m = pl->n_mb, N = pl->c.n_ranks_N;
+#define CP(dst, src, cnt) if (dst) memcpy(dst, src, (size_t)(cnt) * sizeof(*(src)))
+  CP(mb_sample_off, pl->mb_sample_off, m + 1); CP(mb_samples, pl->mb_samples, n);
+  CP(mb_tokens, pl->mb_tokens, m); CP(mb_lmax, pl->mb_lmax, m); CP(mb_residual, pl->mb_residual, m);
+  CP(mb_cost, pl->mb_cost, m); CP(mb_bucket, pl->mb_bucket, m); CP(mb_rank, pl->mb_rank, m);
+  CP(rank_mb_off, pl->rank_mb_off, N + 1); CP(rank_mbs, pl->rank_mbs, m);
+  CP(sample_cost, pl->sample_cost, n); CP(sample_mb, pl->sample_mb, n);
+  return OR_OK;
+}

@@ -1,0 +1,563 @@
+"""Pins the CPU oracle to things other than itself: hand-executed fixtures, closed forms, invariants,
+library routines on special cases, and brute force on tiny inputs.  CPU only."""
+import itertools
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import workloads
+from harness import bits16, bits32, pool_config_fields, register_args, run_oracle, write_args, host_span
+from oracle import (OraclePool, PlanConfig, PoolConfig, balance, bestfit_segment_tree, cost_int,
+                    f32_to_bf16_rne, plan_from_lengths)
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def golden(name):
+    d = {}
+    for line in open(os.path.join(GOLD, name)):
+        line = line.split("#")[0].strip()
+        if ":" in line:
+            k, v = line.split(":")
+            d[k.strip()] = [int(x) for x in v.split()]
+    return d
+
+
+def plan_cfg(L, A=None, B=1, K=1, N=1, flags=0):
+    return PlanConfig(coef_A=L if A is None else A, coef_B=B, budget_L=L, n_buckets_K=K, n_ranks_N=N, flags=flags)
+
+
+# ------------------------------------------------------------------ G. GVA layout (Sec. 3.2)
+
+def small_pool(**kw):
+    f = dict(page_bytes=4096, hbm_pages=6, host_pages=5, max_text_tokens=4096, ring_seed=1, bind_seed=2,
+             gva_hbm_start=0, gva_host_start=0, max_size=0, hidden=64, max_samples=8, max_spans_per_sample=4,
+             max_pages_per_span=64, max_seq_len=4096, placeholder_id=99, ring_order=0, bind_order=0,
+             world_size=1, rank=0)
+    f.update(kw)
+    return OraclePool(PoolConfig(**f))
+
+
+def test_segment_formula_matches_hand_values():
+    g = golden("gva_segments.txt")
+    start, M, W = g["start"][0], g["max_size"][0], g["world_size"][0]
+    # page_bytes must be >= 4096, so scale the fixture by 4096 (the formula is linear in its three inputs)
+    s = 4096
+    for i in range(W):
+        p = small_pool(gva_hbm_start=start * s, gva_host_start=10 * start * s, max_size=M * s, world_size=W, rank=i,
+                       hbm_pages=2, host_pages=2, max_text_tokens=1024)
+        assert p.rc == 0
+        for proc in range(W):
+            assert p.segment_base(0, proc) == g["segment_bases"][proc] * s
+            assert p.segment_base(1, proc) == (10 * start + (g["segment_bases"][proc] - start)) * s
+        # this process's page k sits at its own segment base + k * page_bytes
+        assert p.page_gva(0) == g["segment_bases"][i] * s
+        assert p.page_gva(1) == g["segment_bases"][i] * s + 4096
+        assert p.page_gva(2) == (10 * start) * s + (g["segment_bases"][i] - start) * s  # first DRAM page
+        # the region is half-open: its end belongs to nobody
+        assert p.translate(g["region_end"][0] * s)[0] == -7
+        p.destroy()
+
+
+def test_default_layout_and_bad_gvas():
+    p = small_pool()
+    assert p.segment_base(0, 0) == 1 << 44 and p.segment_base(1, 0) == 1 << 45
+    PS = 4096
+    for bad in (0, (1 << 44) - 1, (1 << 45) - 1, (1 << 45) + 5 * PS, (1 << 44) + 6 * PS + 4096 * 4, (1 << 45) + (1 << 40)):
+        assert p.translate(bad)[0] == -7, hex(bad)
+    assert p.translate((1 << 44) + 6 * PS)[:2] == (0, 2)  # first text page follows the embedding pages
+    assert p.translate((1 << 45) + 5 * PS - 1) == (0, 1, 4, PS - 1)
+    p.destroy()
+
+
+def fisher_yates(n, seed):
+    """Independent retyping of the stated shuffle: i = n-1..1, j = hash(seed, i) mod (i+1)."""
+    M = (1 << 64) - 1
+
+    def mix(z):
+        z = (z + 0x9E3779B97F4A7C15) & M
+        z = ((z ^ (z >> 30)) * 0xBF58476D1CE4E5B9) & M
+        z = ((z ^ (z >> 27)) * 0x94D049BB133111EB) & M
+        return z ^ (z >> 31)
+    a = list(range(n))
+    for i in range(n - 1, 0, -1):
+        j = mix(seed ^ mix(i)) % (i + 1)
+        a[i], a[j] = a[j], a[i]
+    return a
+
+
+@pytest.mark.parametrize("bind_order", [0, 1])
+def test_translation_is_a_bijection(bind_order):
+    p = small_pool(hbm_pages=37, host_pages=21, bind_order=bind_order, bind_seed=77)
+    seen = set()
+    exp_h = fisher_yates(37, 77) if bind_order else list(range(37))
+    exp_d = fisher_yates(21, 78) if bind_order else list(range(21))
+    for g in range(58):
+        gva = p.page_gva(g)
+        rc, kind, frame, off = p.translate(gva)
+        assert rc == 0 and off == 0
+        assert kind == (0 if g < 37 else 1)
+        assert frame == (exp_h[g] if g < 37 else exp_d[g - 37])
+        seen.add((kind, frame))
+        assert p.translate(gva + 4095) == (0, kind, frame, 4095)
+    assert len(seen) == 58  # distinct frames: no two pages alias
+    p.destroy()
+
+
+def test_shuffled_ring_is_the_stated_permutation():
+    p = small_pool(hbm_pages=40, host_pages=24, ring_order=1, ring_seed=5)
+    assert list(p.ring()) == fisher_yates(64, 5)
+    p.destroy()
+    p = small_pool(hbm_pages=40, host_pages=24, ring_order=0)
+    assert list(p.ring()) == list(range(64))  # HBM pages first, DRAM is the overflow tier
+    p.destroy()
+
+
+def test_create_rejects_bad_configs():
+    for kw in (dict(page_bytes=2048), dict(page_bytes=4 << 20), dict(page_bytes=12288), dict(hidden=12),
+               dict(hbm_pages=0, host_pages=0), dict(max_size=4096 * 4), dict(gva_hbm_start=1 << 45, gva_host_start=1 << 45),
+               dict(world_size=2, rank=2)):
+        p = small_pool(**kw)
+        assert p.rc == -1, kw
+
+
+# ------------------------------------------------------------------ W. cast
+
+def test_rne_cast_hand_values():
+    for line in open(os.path.join(GOLD, "rne_cast.txt")):
+        line = line.split("#")[0].split()
+        if len(line) == 2:
+            assert f32_to_bf16_rne(int(line[0], 16)) == int(line[1], 16), line
+
+
+def test_rne_cast_equals_library_rounding_on_non_nan():
+    rng = np.random.default_rng(0)
+    bits = rng.integers(0, 1 << 32, size=400000, dtype=np.uint64).astype(np.uint32)
+    bits = np.concatenate([bits, workloads.special_f32_bits(), np.arange(0x3F7F0000, 0x3F810000, 7, dtype=np.uint32)])
+    f = torch.from_numpy(bits.view(np.int32).copy()).view(torch.float32)
+    lib_bits = bits16(f.to(torch.bfloat16))
+    nan = np.isnan(bits.view(np.float32))
+    ours = np.array([f32_to_bf16_rne(int(b)) for b in bits[~nan][:60000]], dtype=np.uint16)
+    assert np.array_equal(ours, lib_bits[~nan][:60000])
+    ours_tail = np.array([f32_to_bf16_rne(int(b)) for b in bits[-20000:]], dtype=np.uint16)
+    keep = ~nan[-20000:]
+    assert np.array_equal(ours_tail[keep], lib_bits[-20000:][keep])
+    # fixed rule for NaNs: sign-preserving quiet NaN
+    for b in bits[nan][:2000]:
+        assert f32_to_bf16_rne(int(b)) == (((int(b) >> 16) & 0x8000) | 0x7FC0)
+
+
+# ------------------------------------------------------------------ P. packing (Algorithm 1)
+
+def test_bestfit_hand_examples():
+    g = golden("bestfit_hand.txt")
+    for case in "ABC":
+        L = g[f"{case}_L"][0]
+        rc, plan = plan_from_lengths(g[f"{case}_lengths"], plan_cfg(L))
+        assert rc == 0
+        a = plan.arrays()
+        assert list(a["sample_mb"]) == g[f"{case}_sample_mb"]
+        assert list(a["mb_residual"]) == g[f"{case}_residual"]
+        if f"{case}_tokens" in g:
+            assert list(a["mb_tokens"]) == g[f"{case}_tokens"] and list(a["mb_lmax"]) == g[f"{case}_lmax"]
+        plan.destroy()
+
+
+def opt_bins(lengths, L):
+    """Brute force: fewest bins of capacity L (n <= 10)."""
+    best = [len(lengths)]
+    items = sorted(lengths, reverse=True)
+
+    def rec(i, bins):
+        if len(bins) >= best[0]:
+            return
+        if i == len(items):
+            best[0] = len(bins)
+            return
+        seen = set()
+        for b in range(len(bins)):
+            if bins[b] + items[i] <= L and bins[b] not in seen:
+                seen.add(bins[b])
+                bins[b] += items[i]
+                rec(i + 1, bins)
+                bins[b] -= items[i]
+        bins.append(items[i])
+        rec(i + 1, bins)
+        bins.pop()
+    rec(0, [])
+    return best[0]
+
+
+def check_packing_invariants(lengths, L, a):
+    lengths = np.asarray(lengths)
+    n_mb = a["n_mb"]
+    smb = a["sample_mb"]
+    assert smb.max() + 1 == n_mb
+    for j in range(n_mb):
+        members = np.nonzero(smb == j)[0]
+        assert len(members) > 0
+        assert lengths[members].sum() == a["mb_tokens"][j] <= L  # token budget respected
+        assert a["mb_residual"][j] == L - a["mb_tokens"][j]
+        assert a["mb_lmax"][j] == lengths[members].max()
+        # append order inside the microbatch = arrival order
+        assert list(a["mb_samples"][a["mb_sample_off"][j]:a["mb_sample_off"][j + 1]]) == list(members)
+    # any-fit: when B_j is opened no earlier microbatch could have taken its first sequence
+    res = {}
+    for t, l in enumerate(lengths):
+        j = smb[t]
+        if j not in res:
+            assert all(r < l for r in res.values()), (t, l)
+            res[j] = L - l
+        else:
+            fitting = [r for r in res.values() if r >= l]
+            assert res[j] == min(fitting)  # best fit: the minimal sufficient residual
+            res[j] -= l
+
+
+def test_bestfit_invariants_and_brute_force_optimum():
+    rng = np.random.default_rng(1)
+    for trial in range(300):
+        n = int(rng.integers(1, 11))
+        L = int(rng.integers(4, 40))
+        lengths = rng.integers(1, L + 1, size=n)
+        rc, plan = plan_from_lengths(lengths, plan_cfg(L))
+        assert rc == 0
+        a = plan.arrays()
+        check_packing_invariants(lengths, L, a)
+        opt = opt_bins([int(x) for x in lengths], L)
+        assert -(-int(lengths.sum()) // L) <= opt <= a["n_mb"] <= (17 * opt) // 10
+        plan.destroy()
+
+
+def test_linear_scan_equals_literal_segment_tree():
+    rng = np.random.default_rng(2)
+    for trial in range(200):
+        n = int(rng.integers(1, 400))
+        L = int(rng.integers(8, 600))
+        lo = int(rng.integers(1, L))
+        lengths = rng.integers(lo, L + 1, size=n) if trial % 2 else rng.integers(1, max(2, L // 4), size=n)
+        rc, plan = plan_from_lengths(lengths, plan_cfg(L))
+        a = plan.arrays()
+        n_mb, smb = bestfit_segment_tree(lengths, L, int(lengths.min()))  # with removal at l_min of this call
+        assert n_mb == a["n_mb"] and np.array_equal(smb, a["sample_mb"])
+        n_mb0, smb0 = bestfit_segment_tree(lengths, L, 0)                 # and without removal
+        assert n_mb0 == n_mb and np.array_equal(smb0, smb)
+        check_packing_invariants(lengths, L, a)
+        plan.destroy()
+
+
+def test_plan_errors():
+    assert plan_from_lengths([5, 11], plan_cfg(10))[0] == -6       # longer than the budget
+    assert plan_from_lengths([5, 0], plan_cfg(10))[0] == -1
+    assert plan_from_lengths([5], plan_cfg(0))[0] == -1
+    assert plan_from_lengths([5], plan_cfg(10, K=0))[0] == -1
+    assert plan_from_lengths([5], plan_cfg(10, N=0))[0] == -1
+    rc, plan = plan_from_lengths([], plan_cfg(10))
+    assert rc == 0 and plan.summary() == (0, 0, 0)
+
+
+def test_cost_closed_form_eq3():
+    g = golden("cost_eq3.txt")
+    L = g["L"][0]
+    ls = g["lengths"]
+    assert cost_int(L, 1, sum(ls), max(ls)) == g["cost_int"][0]
+    assert g["cost_int"][0] * 1000 == g["cost_real_times_1000"][0] * L * L
+    assert cost_int(L, 1, L, L) == g["full_cost_int"][0]
+    rc, plan = plan_from_lengths(ls, plan_cfg(L))
+    a = plan.arrays()
+    assert a["n_mb"] == 1 and int(a["mb_cost"][0]) == g["cost_int"][0]
+    # per-sample score = Eq. 3 on a singleton
+    assert [int(x) for x in a["sample_cost"]] == [L * l + l * l for l in ls]
+    # the quadratic term is lmax^2, not sum of squares; cost never exceeds A*L + B*L^2
+    rng = np.random.default_rng(3)
+    lengths = rng.integers(1, 500, size=300)
+    rc, plan = plan_from_lengths(lengths, plan_cfg(1000, A=777, B=5))
+    a = plan.arrays()
+    for j in range(a["n_mb"]):
+        m = lengths[a["sample_mb"] == j]
+        assert int(a["mb_cost"][j]) == 777 * int(m.sum()) + 5 * int(m.max()) ** 2 <= 777 * 1000 + 5 * 1000 ** 2
+
+
+def test_zigzag_hand_example():
+    g = golden("zigzag_hand.txt")
+    r = balance(g["costs"], 1, g["N"][0])
+    assert list(r["rank"]) == g["K1_rank"] and list(r["bucket"]) == [0] * 7
+    assert list(r["rank_mbs"]) == g["K1_rank_mbs"] and list(r["rank_mb_off"]) == g["K1_rank_mb_off"]
+    loads = [sum(c for c, k in zip(g["costs"], r["rank"]) if k == n) for n in range(3)]
+    assert loads == g["K1_loads"]
+    r = balance(g["costs"], 2, g["N"][0])
+    assert list(r["bucket"]) == g["K2_bucket"] and list(r["rank"]) == g["K2_rank"]
+    # unsorted input, ties broken by index
+    r = balance([5, 9, 5, 7], 1, 2)
+    assert list(r["rank"]) == [1, 0, 0, 1] and list(r["rank_mbs"]) == [1, 2, 3, 0]
+    assert list(balance([4, 4, 4], 3, 1)["bucket"]) == [0, 0, 0]  # hi == lo: one bucket
+    assert list(balance([4, 2, 9], 1, 1)["rank_mbs"]) == [2, 0, 1]
+
+
+def test_zigzag_imbalance_bound_and_bucket_width():
+    rng = np.random.default_rng(4)
+    for trial in range(400):
+        m, K, N = int(rng.integers(1, 60)), int(rng.integers(1, 6)), int(rng.integers(1, 9))
+        costs = rng.integers(1, 1000, size=m).astype(np.uint64)
+        r = balance(costs, K, N)
+        lo, hi = int(costs.min()), int(costs.max())
+        width = -(-(hi - lo + 1) // K)
+        total_bound = 0
+        for k in range(K):
+            idx = np.nonzero(r["bucket"] == k)[0]
+            if len(idx) == 0:
+                continue
+            c = costs[idx].astype(np.int64)
+            assert c.max() - c.min() < width                     # similar cost inside a bucket
+            loads = np.array([c[r["rank"][idx] == n].sum() for n in range(N)])
+            counts = np.array([(r["rank"][idx] == n).sum() for n in range(N)])
+            assert counts.max() - counts.min() <= 1
+            assert loads.max() - loads.min() <= c.max()          # what Algorithm 1 guarantees per bucket
+            if len(idx) % N == 0:
+                assert loads.max() - loads.min() <= c.max() - c.min()
+            total_bound += int(c.max())
+        loads = np.array([costs[r["rank"] == n].astype(np.int64).sum() for n in range(N)])
+        assert loads.max() - loads.min() <= total_bound
+        # every microbatch dealt exactly once, per-rank lists consistent with ranks
+        assert sorted(r["rank_mbs"]) == list(range(m))
+        for n in range(N):
+            assert all(r["rank"][j] == n for j in r["rank_mbs"][r["rank_mb_off"][n]:r["rank_mb_off"][n + 1]])
+
+
+def test_zigzag_against_brute_force_makespan():
+    rng = np.random.default_rng(5)
+    for trial in range(60):
+        m, N = int(rng.integers(1, 8)), int(rng.integers(1, 4))
+        costs = [int(x) for x in rng.integers(1, 50, size=m)]
+        r = balance(costs, 1, N)
+        ours = max(sum(c for c, k in zip(costs, r["rank"]) if k == n) for n in range(N))
+        opt = min(max(sum(c for c, k in zip(costs, assign) if k == n) for n in range(N))
+                  for assign in itertools.product(range(N), repeat=m))
+        assert opt <= ours <= opt + max(costs)
+
+
+# ------------------------------------------------------------------ F. free ring, W. write, A. assembly
+
+def all_pages_partition(pool, live_spans, total_pages):
+    """ring + live span pages = every page exactly once (conservation, no aliasing)."""
+    ring = [pool.page_gva(int(g)) for g in pool.ring()]
+    live = []
+    for s, j in live_spans:
+        live += [int(x) for x in pool.span_pages(s, j)[1]]
+    allp = ring + live
+    assert len(allp) == total_pages and len(set(allp)) == total_pages
+    assert set(allp) == {pool.page_gva(g) for g in range(total_pages)}
+
+
+@pytest.mark.parametrize("ring_order", [0, 1])
+def test_ring_conservation_under_write_and_free(ring_order):
+    w = workloads.make_workload("image_mix_7b", n_samples=24, hidden=64, page_bytes=4096)
+    w.ring_order = ring_order
+    P = w.hbm_pages + w.host_pages
+    pool = OraclePool(PoolConfig(**pool_config_fields(w)))
+    all_pages_partition(pool, [], P)
+    live = []
+    samples = list(range(24))
+    assert pool.register_samples(*register_args(w, samples)) == 0
+    first_ring = list(pool.ring())
+    for s in samples[:12]:
+        call = [(s, j) for j in range(int(w.n_spans[s]))]
+        before = pool.free_pages()[0]
+        assert pool.write_embeddings(*write_args(w, call), [host_span(w, s, j) for s, j in call], 0) == 0
+        need = sum(w.pages_of_span(w.spans_of(s)[1][j]) for s, j in call)
+        assert before - pool.free_pages()[0] == need          # exactly ceil(bytes/page) pages per span
+        live += call
+        all_pages_partition(pool, live, P)
+    # pages are handed out from the ring head, spans in argument order
+    got = [int(x) for s, j in live for x in pool.span_pages(s, j)[1]]
+    assert got == [pool.page_gva(g) for g in first_ring[:len(got)]]
+    # free a few (argument order, spans by index, pages by ordinal go to the tail)
+    gone = [3, 0, 7]
+    tail = [int(x) for s in gone for j in range(int(w.n_spans[s])) for x in pool.span_pages(s, j)[1]]
+    assert pool.free(gone) == 0
+    live = [c for c in live if c[0] not in gone]
+    all_pages_partition(pool, live, P)
+    assert [pool.page_gva(int(g)) for g in pool.ring()][-len(tail):] == tail
+    # free everything: the ring is a permutation of all pages again
+    assert pool.free([s for s in samples if s not in gone]) == 0
+    all_pages_partition(pool, [], P)
+    assert pool.free_pages()[1] == w.total_text_tokens_capacity // 1024
+    pool.destroy()
+
+
+@pytest.mark.parametrize("name,kw", [
+    ("tiny", dict(hidden=64, page_bytes=4096)),
+    ("image_mix_7b", dict(n_samples=12, hidden=56, page_bytes=4096)),      # row 112 B does not divide the page
+    ("host_tier_stress", dict(n_samples=3, hidden=16, page_bytes=4096)),   # fp32 source, shuffled ring, two tiers
+])
+def test_write_read_back_through_the_page_table(name, kw):
+    w = workloads.make_workload(name, **kw)
+    r = run_oracle(w, keep_pool=True)
+    assert all(c == 0 for c in r["rc"]) and r["status"] == (0, 0)
+    pool = r["pool"]
+    touched = 0
+    for call in w.write_calls:
+        for s, j in call:
+            v = workloads.span_values(w, s, j)
+            exp = bits16(v.to(torch.bfloat16)) if w.src_dtype == 0 else None
+            if exp is None:
+                exp = np.array([f32_to_bf16_rne(int(b)) for b in bits32(v).ravel()], dtype=np.uint16)
+            exp = exp.ravel().view(np.uint8)
+            pages = r["span_pages"][(s, j)]
+            assert len(pages) == w.pages_of_span(w.spans_of(s)[1][j])
+            got = []
+            for g in pages:
+                rc, kind, frame, off = pool.translate(int(g))
+                assert rc == 0 and off == 0 and kind in (0, 1)
+                got.append(pool.backing(kind)[frame * w.page_bytes:(frame + 1) * w.page_bytes])
+            got = np.concatenate(got)
+            assert np.array_equal(got[:len(exp)], exp)
+            touched += len(exp)
+    assert touched == w.total_vision_tokens * w.row_bytes
+    if w.host_pages:
+        kinds = {pool.translate(int(g))[1] for pg in r["span_pages"].values() for g in pg}
+        assert kinds == {0, 1}  # both tiers really hold data
+    r["plan_handle"].destroy()
+    pool.destroy()
+
+
+@pytest.mark.parametrize("name,kw", [
+    ("tiny", dict(hidden=64, page_bytes=4096)),
+    ("image_mix_7b", dict(n_samples=20, hidden=56, page_bytes=4096)),
+    ("video_heavy", dict(n_samples=6, hidden=64, page_bytes=32768)),
+    ("host_tier_stress", dict(n_samples=3, hidden=16, page_bytes=4096)),
+])
+def test_assembly_equals_textbook_masked_scatter(name, kw):
+    """x = embedding(ids, table); x[ids == placeholder] = cat(vision spans); cat over the microbatch."""
+    w = workloads.make_workload(name, **kw)
+    r = run_oracle(w)
+    assert all(c == 0 for c in r["rc"]) and r["status"] == (0, 0)
+    table = workloads.embed_table(w)
+    a = r["plan"]
+    rows, cu_all, pos_all = [], [], []
+    for j in range(a["n_mb"]):
+        members = a["mb_samples"][a["mb_sample_off"][j]:a["mb_sample_off"][j + 1]]
+        lens = []
+        for s in members:
+            s = int(s)
+            ids = torch.from_numpy(workloads.input_ids(w, s)).long()
+            x = torch.nn.functional.embedding(ids.clamp(max=w.vocab - 1), table)
+            if int(w.n_spans[s]):
+                vis = torch.cat([workloads.span_values(w, s, jj) for jj in range(int(w.n_spans[s]))])
+                if w.src_dtype == 1:  # library rounding; NaN rows compared separately below
+                    vis = vis.to(torch.bfloat16)
+                x[ids == w.placeholder_id] = vis
+            rows.append(x)
+            lens.append(len(ids))
+            pos_all.append(torch.arange(len(ids), dtype=torch.int32))
+        cu_all.append(torch.cat([torch.zeros(1, dtype=torch.int64), torch.cumsum(torch.tensor(lens), 0)]).to(torch.int32))
+    exp = bits16(torch.cat(rows))
+    got = r["out"]
+    assert got.shape == exp.shape
+    exp_nan = (exp & 0x7FFF) > 0x7F80
+    assert np.array_equal(got[~exp_nan], exp[~exp_nan])
+    assert np.all((got[exp_nan] & 0x7FFF) == 0x7FC0)  # fixed NaN rule
+    assert np.array_equal(r["cu_seqlens"], torch.cat(cu_all).numpy())
+    assert np.array_equal(r["position_ids"], torch.cat(pos_all).numpy())
+    assert not np.any(np.all(got == 0xFFFF, axis=1))  # no output row left at poison
+
+
+def test_gather_ranges_concatenate():
+    w = workloads.make_workload("image_mix_7b", n_samples=16, hidden=56, page_bytes=4096)
+    w.budget_L = 12000
+    r = run_oracle(w, keep_pool=True)
+    pool, plan, a = r["pool"], r["plan_handle"], r["plan"]
+    assert a["n_mb"] >= 3
+    row = 0
+    for j in range(a["n_mb"]):
+        t = int(a["mb_tokens"][j])
+        out = np.zeros((t, w.hidden), np.uint16)
+        nj = int(a["mb_sample_off"][j + 1] - a["mb_sample_off"][j])
+        cu = np.zeros(nj + 1, np.int32)
+        pos = np.zeros(t, np.int32)
+        assert pool.gather_packed(plan, j, j + 1, r["table"], out, cu, pos) == 0
+        assert np.array_equal(out, r["out"][row:row + t]) and cu[0] == 0 and cu[-1] == t
+        row += t
+    assert row == w.total_tokens
+    plan.destroy()
+    pool.destroy()
+
+
+# ------------------------------------------------------------------ status codes
+
+def test_status_codes_and_all_or_nothing():
+    w = workloads.make_workload("image_mix_7b", n_samples=6, hidden=64, page_bytes=4096)
+    f = pool_config_fields(w)
+    f["hbm_pages"], f["host_pages"] = w.pages_of_span(w.spans_of(0)[1][0]) + 1, 0
+    pool = OraclePool(PoolConfig(**f))
+    reg = register_args(w, [0, 1, 2])
+    assert pool.register_samples(*reg) == 0
+    assert pool.register_samples(*register_args(w, [3, 1])) == -10        # slot in use; nothing registered
+    assert pool.write_embeddings([3], [0], [w.spans_of(3)[1][0]], [host_span(w, 3, 0)], 0) == -3
+    s, sp, nt, ids = register_args(w, [4])[0], *register_args(w, [4])[3:5], register_args(w, [4])[5]
+    assert pool.register_samples([9], [10], [0], [], [], np.zeros(10, np.int32)) == -1      # slot out of range
+    assert pool.register_samples([4], [10], [1], [8], [5], np.zeros(10, np.int32)) == -1    # run beyond the sequence
+    assert pool.register_samples([4], [10], [2], [2, 3], [2, 2], np.zeros(10, np.int32)) == -1  # overlapping runs
+    assert pool.register_samples([4], [10], [5], [0] * 5, [1] * 5, np.zeros(10, np.int32)) == -11
+    t0 = int(w.spans_of(0)[1][0])
+    assert pool.write_embeddings([0], [7], [t0], [host_span(w, 0, 0)], 0) == -1
+    assert pool.write_embeddings([0], [0], [t0 + 1], [host_span(w, 0, 0)], 0) == -1
+    assert pool.write_embeddings([0, 0], [0, 0], [t0, t0], [host_span(w, 0, 0)] * 2, 0) == -4
+    before = pool.free_pages()
+    big = [(1, j) for j in range(int(w.n_spans[1]))] + [(2, j) for j in range(int(w.n_spans[2]))] + [(0, 0)]
+    assert pool.write_embeddings(*write_args(w, big), [host_span(w, s, j) for s, j in big], 0) == -2
+    assert pool.free_pages() == before                                     # exhausted call changed nothing
+    assert pool.write_embeddings([0], [0], [t0], [host_span(w, 0, 0)], 0) == 0
+    assert pool.write_embeddings([0], [0], [t0], [host_span(w, 0, 0)], 0) == -4
+    cfg = PlanConfig(coef_A=1, coef_B=1, budget_L=1 << 20, n_buckets_K=1, n_ranks_N=1, flags=0)
+    ready0 = int(w.n_spans[0]) == 1
+    assert pool.plan_microbatches([1], cfg)[0] == -5                       # not every span written
+    assert pool.plan_microbatches([5], cfg)[0] == -3
+    cfg.flags = 1
+    rc, plan = pool.plan_microbatches([1, 2], cfg)
+    assert rc == 0 and plan.summary()[0] == 1
+    assert pool.gather_packed(plan, 0, 1, np.zeros((4, 64), np.uint16), np.zeros((1, 64), np.uint16),
+                              np.zeros(3, np.int32), np.zeros(1, np.int32)) == -5   # unwritten sample in the plan
+    assert pool.plan_microbatches([1, 1], cfg)[0] == -1
+    cfg.budget_L = 10
+    assert pool.plan_microbatches([1], cfg)[0] == -6
+    assert pool.free([5]) == -3 and pool.free([0, 0]) == -3
+    assert pool.free([0, 1, 2]) == 0
+    assert pool.free_pages()[0] == f["hbm_pages"]
+    pool.destroy()
+
+
+def test_placeholder_mismatch_and_bad_token_are_reported_with_smallest_detail():
+    w = workloads.make_workload("tiny", n_samples=4, hidden=64, page_bytes=4096)
+    pool = OraclePool(PoolConfig(**pool_config_fields(w)))
+    slots, seq_len, n_spans, pos, tok, ids = register_args(w, [0, 1, 2, 3])
+    off = [0] + [int(x) for x in np.cumsum(seq_len)]
+    pos, tok = [int(x) for x in pos], [int(x) for x in tok]
+    ids = ids.copy()
+    ids[off[2] + pos[2]] = 5                      # a run position that is not the placeholder (sample 2)
+    text_pos = 0 if pos[1] > 0 else int(pos[1] + tok[1])
+    ids[off[1] + text_pos] = w.placeholder_id     # a stray placeholder (sample 1)
+    assert pool.register_samples(slots, seq_len, n_spans, pos, tok, ids) == 0
+    assert pool.status() == (-8, 1)               # smallest slot wins
+    assert pool.status() == (0, 0)                # drained
+    pool.destroy()
+    # token id outside the table: row skipped, BAD_TOKEN_ID with the smallest row index
+    pool = OraclePool(PoolConfig(**pool_config_fields(w)))
+    slots, seq_len, n_spans, pos, tok, ids = register_args(w, [0, 1])
+    assert pool.register_samples(slots, seq_len, n_spans, pos, tok, ids) == 0
+    call = [(0, 0), (1, 0)]
+    assert pool.write_embeddings(*write_args(w, call), [host_span(w, s, j) for s, j in call], 0) == 0
+    rc, plan = pool.plan_microbatches([0, 1], PlanConfig(coef_A=1, coef_B=1, budget_L=4096, n_buckets_K=1, n_ranks_N=1, flags=0))
+    total = plan.summary()[1]
+    small_vocab = 100
+    table = np.zeros((small_vocab, 64), np.uint16)
+    out = np.full((total, 64), 0xFFFF, np.uint16)
+    assert pool.gather_packed(plan, 0, 1, table, out, np.zeros(3, np.int32), np.zeros(total, np.int32)) == 0
+    ids0 = workloads.input_ids(w, 0)
+    first_bad = int(np.nonzero((ids0 >= small_vocab) & (ids0 != w.placeholder_id))[0][0])
+    assert pool.status() == (-9, first_bad)
+    assert np.all(out[first_bad] == 0xFFFF)
+    plan.destroy()
+    pool.destroy()
