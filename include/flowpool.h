@@ -1,0 +1,267 @@
+/*
+ * flowpool.h -- C ABI of the unified-memory-pool hot path on one B200 (sm_100a).
+ *
+ * The pool is the coordination layer between encoder producers and the LLM
+ * backbone (paper Sec. 3.1-3.2): producers scatter embeddings into fixed-size
+ * pages addressed by 64-bit global virtual addresses (GVAs); a page table maps
+ * GVA -> physical frame in HBM or in pinned host DRAM; the dynamic packing
+ * scheduler (Sec. 3.4, Algorithm 1, Eq. 3) forms balanced microbatches; the
+ * consumer translates GVAs and assembles each packed microbatch.
+ *
+ * Conventions
+ *  - Every call returns an int32 status: FT_OK or a negative FT_ERR_* code.
+ *    Nothing throws, aborts or traps.
+ *  - "host" / "device" in a parameter comment says where the pointer lives.
+ *    Host arrays are read before the call returns.  Device work is enqueued on
+ *    the caller's stream (`stream` = a cudaStream_t passed as void*; NULL = the
+ *    legacy default stream); ordering between calls is stream order.
+ *  - One caller thread per pool.  The caller owns every buffer it passes in
+ *    (backing memory, sources, table, outputs); the library owns its metadata
+ *    and anything it allocated itself.
+ *  - Errors the host can know (argument, state, capacity) are returned at once
+ *    and the failed call has no effect (all-or-nothing; checks run in argument
+ *    order, first failure wins).  Errors only the device can see go to an
+ *    asynchronous status word read by pool_status(); the offending item is
+ *    skipped.
+ *  - The library needs a CUDA device; there is no CPU fallback.
+ */
+#ifndef FLOWPOOL_H_
+#define FLOWPOOL_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  FT_OK = 0,
+  FT_ERR_INVALID_ARG = -1,
+  FT_ERR_POOL_EXHAUSTED = -2,
+  FT_ERR_UNKNOWN_SAMPLE = -3,
+  FT_ERR_ALREADY_WRITTEN = -4,
+  FT_ERR_NOT_READY = -5,
+  FT_ERR_TOO_LONG = -6,
+  FT_ERR_BAD_GVA = -7,
+  FT_ERR_PLACEHOLDER_MISMATCH = -8,
+  FT_ERR_BAD_TOKEN_ID = -9,
+  FT_ERR_SLOT_IN_USE = -10,
+  FT_ERR_CAPACITY = -11,
+  FT_ERR_CUDA = -12,
+  FT_ERR_TIMEOUT = -13
+};
+
+enum { FT_RING_SORTED = 0, FT_RING_SHUFFLED = 1 }; /* initial free-ring order */
+enum { FT_BIND_IDENTITY = 0, FT_BIND_PERMUTED = 1 }; /* virtual page -> frame */
+enum { FT_BF16 = 0, FT_F32 = 1 };                    /* producer source dtype */
+enum { FT_PLAN_ALLOW_UNWRITTEN = 1 };                /* plan flags */
+
+#define FT_TEXT_PAGE_BYTES 4096u /* token ids live in 4 KiB text pages (1024 ids) */
+
+typedef struct ft_pool ft_pool;
+typedef struct ft_plan ft_plan;
+
+/*
+ * Pool geometry (Sec. 3.2).  The GVA space has two disjoint regions, one per
+ * tier; region t is [start_t, start_t + world_size*max_size) and process i
+ * owns [start_t + i*max_size, start_t + (i+1)*max_size).  This process binds
+ * hbm_pages (resp. host_pages) frames of page_bytes at the base of its
+ * segment; page k has GVA start_t + rank*max_size + k*page_bytes.  Text pages
+ * follow the embedding pages inside the HBM segment.
+ */
+typedef struct {
+  uint64_t page_bytes;      /* power of two, 4 KiB .. 2 MiB */
+  uint64_t hbm_pages;       /* frames bound in HBM */
+  uint64_t host_pages;      /* frames bound in pinned, device-mapped host DRAM */
+  uint64_t max_text_tokens; /* text-page budget, in token ids (rounded up to whole text pages) */
+  uint64_t ring_seed;       /* seed of FT_RING_SHUFFLED */
+  uint64_t bind_seed;       /* seed of FT_BIND_PERMUTED (HBM: seed, host: seed+1) */
+  uint64_t gva_hbm_start;   /* 0 => 2^44 */
+  uint64_t gva_host_start;  /* 0 => 2^45 */
+  uint64_t max_size;        /* per-process segment size; 0 => 2^40 */
+  uint32_t hidden;          /* H, a multiple of 8 (a bf16 row is a multiple of 16 bytes) */
+  uint32_t max_samples;     /* number of sample slots */
+  uint32_t max_spans_per_sample;
+  uint32_t max_pages_per_span;
+  uint32_t max_seq_len;     /* longest sequence a slot may hold */
+  int32_t placeholder_id;   /* the image-placeholder token id */
+  uint32_t ring_order;      /* FT_RING_* */
+  uint32_t bind_order;      /* FT_BIND_* */
+  uint32_t world_size;      /* 0 => 1; only this process's binding exists in this build */
+  uint32_t rank;
+} ft_pool_config;
+
+/* Packing parameters (Sec. 3.4): budget L, integer cost A*sum(l) + B*lmax^2
+ * (Eq. 3 times L^2 when A = L, B = 1), K cost buckets, N data-parallel ranks. */
+typedef struct {
+  uint64_t coef_A, coef_B;
+  uint32_t budget_L, n_buckets_K, n_ranks_N, flags;
+} ft_plan_config;
+
+typedef struct {
+  uint64_t pages_total, pages_free, hbm_pages, host_pages;
+  uint64_t text_pages_total, text_pages_free;
+  uint64_t live_samples, live_spans;
+  uint64_t bytes_written, bytes_gathered; /* algorithmic bytes enqueued so far */
+  uint64_t gpu_launches;                  /* kernels of this library launched so far */
+} ft_pool_stats;
+
+/*
+ * pool_create -- pool initialisation and binding (Sec. 3.2: each process
+ * reserves a GVA range in its segment, allocates physical memory and binds it;
+ * every process holds the page table locally).
+ *   cfg      host.  See ft_pool_config.
+ *   hbm_base device, caller-owned, >= hbm_pages*page_bytes, 256-byte aligned;
+ *            NULL => the library allocates (and frees at pool_destroy).
+ *   host_base host, caller-owned PINNED memory mapped into the device address
+ *            space (cudaHostAlloc/cudaHostRegister with the mapped flag),
+ *            >= host_pages*page_bytes; NULL => the library allocates.
+ *   out      host; receives the handle.
+ * Errors: INVALID_ARG (page_bytes not a power of two in range, hidden % 8,
+ * no pages, segment too small, overlapping regions, rank >= world_size),
+ * CUDA (allocation or launch failure).  Synchronises the device once.
+ */
+int32_t pool_create(const ft_pool_config* cfg, void* hbm_base, void* host_base, ft_pool** out);
+
+/*
+ * pool_register_samples -- text tokens and pairing metadata enter the pool
+ * (Sec. 3.1: text tokens are inserted directly into the same pool; lightweight
+ * metadata tracks the cross-modal pairing).  Sample i occupies slot
+ * sample_slot[i]; its input_ids hold, for span j, one run of placeholder_id of
+ * span_tokens[.] ids starting at span_pos[.] (sequence coordinates, sorted,
+ * non-overlapping; spans of all samples concatenated in order).
+ *   sample_slot, seq_len, n_spans  host [n]
+ *   span_pos, span_tokens          host [sum n_spans]
+ *   input_ids                      DEVICE int32 [sum seq_len], concatenated
+ * Slot life cycle: FREE -> REGISTERED -> (all spans written) READY -> FREE.
+ * Errors, per sample in order: slot >= max_samples INVALID_ARG; slot not FREE
+ * or repeated SLOT_IN_USE; seq_len 0 INVALID_ARG; seq_len > max_seq_len or
+ * n_spans > max_spans_per_sample CAPACITY; per span: 0 tokens, run past the
+ * sequence, unsorted/overlapping runs INVALID_ARG, pages > max_pages_per_span
+ * CAPACITY; then text pages exhausted CAPACITY.  Asynchronous: a run position
+ * that is not placeholder_id or a stray placeholder -> PLACEHOLDER_MISMATCH
+ * (detail = slot; the sample stays registered).
+ */
+int32_t pool_register_samples(ft_pool* pool, uint32_t n, const uint32_t* sample_slot,
+                              const uint32_t* seq_len, const uint32_t* n_spans,
+                              const uint32_t* span_pos, const uint32_t* span_tokens,
+                              const int32_t* input_ids, void* stream);
+
+/*
+ * pool_write_embeddings -- the producer scatter (Sec. 3.1-3.2: encoders place
+ * embeddings into their own segment and proceed at once).  Span q takes the
+ * next ceil(n_tokens*2H/page_bytes) pages from the free ring, spans in
+ * argument order; its bf16 row-major [n_tokens, H] image is laid into those
+ * pages in order (rows may straddle pages; the last page's tail is untouched).
+ *   sample_slot, span_idx, n_tokens  host [n_spans]
+ *   src        host array [n_spans] of DEVICE pointers, each [n_tokens, H]
+ *              contiguous, 16-byte aligned, FT_BF16 or FT_F32 elements
+ *   src_dtype  FT_F32 fuses the fp32->bf16 cast: IEEE round-to-nearest-even
+ *              on the bit pattern, denormals kept, every NaN -> sign | 0x7FC0.
+ * Asynchronous: returns after enqueueing.  Errors, per span in order:
+ * slot >= max_samples INVALID_ARG; slot FREE UNKNOWN_SAMPLE; span_idx out of
+ * range, n_tokens != registered, src NULL or misaligned INVALID_ARG; span
+ * written before or named twice ALREADY_WRITTEN; then sum of pages > free
+ * pages POOL_EXHAUSTED.
+ */
+int32_t pool_write_embeddings(ft_pool* pool, uint32_t n_spans, const uint32_t* sample_slot,
+                              const uint32_t* span_idx, const uint32_t* n_tokens,
+                              const void* const* src, uint32_t src_dtype, void* stream);
+
+/*
+ * pool_plan_microbatches -- the dynamic packing rule (Algorithm 1, Eq. 3), on
+ * the device.  Samples are packed online in the order given, by best fit on
+ * l(s) = seq_len (ties between equal residuals: the microbatch changed most
+ * recently); each microbatch is scored A*sum(l) + B*lmax^2, bucketed by
+ * equal-width quantisation of the observed cost range into K buckets, and
+ * dealt zig-zag over N ranks per bucket (highest bucket first, cost
+ * descending, ties by index).
+ *   sample_slot host [n]; cfg host; out host, receives the plan handle.
+ * Synchronises the stream once; the summary is valid on return.
+ * Errors: L, K or N zero INVALID_ARG; per sample in order: slot out of range
+ * INVALID_ARG, FREE UNKNOWN_SAMPLE, listed twice INVALID_ARG, not READY
+ * (without FT_PLAN_ALLOW_UNWRITTEN) NOT_READY, seq_len > L TOO_LONG.
+ * n = 0 gives an empty plan.
+ */
+int32_t pool_plan_microbatches(ft_pool* pool, const uint32_t* sample_slot, uint32_t n,
+                               const ft_plan_config* cfg, ft_plan** out, void* stream);
+
+/* Plan summary: number of microbatches, tokens over all of them, largest microbatch. */
+int32_t plan_summary(const ft_plan* plan, uint32_t* n_mb, uint64_t* total_tokens,
+                     uint32_t* max_mb_tokens);
+
+/*
+ * plan_arrays -- host copies of every plan array (any pointer may be NULL):
+ * mb_sample_off[n_mb+1], mb_samples[n] (slots, microbatch-major, append
+ * order), mb_tokens, mb_lmax, mb_residual, mb_cost (u64), mb_bucket,
+ * mb_rank [n_mb], rank_mb_off[N+1], rank_mbs[n_mb] (dispatch order per rank),
+ * sample_cost[n] (u64, Eq. 3 on a singleton), sample_mb[n].  Synchronises.
+ */
+int32_t plan_arrays(const ft_plan* plan, uint32_t* mb_sample_off, uint32_t* mb_samples,
+                    uint32_t* mb_tokens, uint32_t* mb_lmax, uint32_t* mb_residual,
+                    uint64_t* mb_cost, uint32_t* mb_bucket, uint32_t* mb_rank,
+                    uint32_t* rank_mb_off, uint32_t* rank_mbs, uint64_t* sample_cost,
+                    uint32_t* sample_mb);
+
+int32_t plan_destroy(ft_plan* plan);
+
+/*
+ * pool_gather_packed -- the consumer (Sec. 3.1-3.2: the backbone consumes
+ * microbatches by GVA; the GVA is resolved through the page table).  For
+ * microbatches [mb_begin, mb_end) of the plan, concatenated: output row
+ * cu_seqlens[q] + p of a microbatch is row (p - pos_start) of the span whose
+ * placeholder run contains position p of its q-th sample, read through the
+ * span's page list and the page table (HBM frame, or host frame read in place
+ * over the mapped pointer); any other position is embed_table[input_ids[p]].
+ *   embed_table       device bf16 [vocab, H]
+ *   out_embeds        device bf16 [sum of tokens of the range, H], 16-byte aligned
+ *   out_cu_seqlens    device int32, per microbatch (n_j + 1) entries starting at 0
+ *   out_position_ids  device int32 [sum of tokens]: p, restarting per sample
+ * Padding rows are not materialised.  Asynchronous.  Errors: bad range
+ * INVALID_ARG; a sample of the plan freed or not READY NOT_READY; NULL buffer
+ * INVALID_ARG.  Asynchronous: id outside [0, vocab) BAD_TOKEN_ID, page GVA that
+ * does not translate BAD_GVA (detail = row index in the range; row skipped).
+ */
+int32_t pool_gather_packed(ft_pool* pool, const ft_plan* plan, uint32_t mb_begin, uint32_t mb_end,
+                           const void* embed_table, uint32_t vocab, void* out_embeds,
+                           int32_t* out_cu_seqlens, int32_t* out_position_ids, void* stream);
+
+/*
+ * pool_free -- release samples: their pages go back to the free-ring tail
+ * (samples in argument order, spans by index, pages by ordinal), their text
+ * pages and slots are recycled.  Plans holding a freed sample become invalid.
+ * The paper does not discuss recycling; the ring is this build's fixed rule.
+ *   sample_slot host [n].  Errors: slot out of range INVALID_ARG; FREE or
+ * listed twice UNKNOWN_SAMPLE.  Asynchronous.
+ */
+int32_t pool_free(ft_pool* pool, const uint32_t* sample_slot, uint32_t n, void* stream);
+
+/* First asynchronous error since the last call (smallest call, then smallest
+ * detail), then cleared.  Synchronises the device. */
+int32_t pool_status(ft_pool* pool, int32_t* first_device_error, uint64_t* detail);
+
+int32_t pool_stats(ft_pool* pool, ft_pool_stats* out);
+
+/* Page GVAs of one span, by ordinal (for parity checks).  Synchronises. */
+int32_t pool_debug_span_pages(ft_pool* pool, uint32_t slot, uint32_t span, uint64_t* gva_out,
+                              uint32_t cap, uint32_t* n);
+
+/* Free ring content, head first, as global page indices.  Synchronises. */
+int32_t pool_debug_ring(ft_pool* pool, uint32_t* out, uint64_t cap, uint64_t* n);
+
+/* Device-side GVA translation of a host array of GVAs (for parity checks):
+ * kind 0 HBM / 1 host / 2 text, frame index within its tier, byte offset;
+ * status[i] = FT_OK or FT_ERR_BAD_GVA.  Synchronises. */
+int32_t pool_debug_translate(ft_pool* pool, const uint64_t* gva, uint32_t n, uint32_t* kind,
+                             uint64_t* frame, uint64_t* offset, int32_t* status);
+
+/* Tear down: frees everything the library allocated.  Synchronises. */
+int32_t pool_destroy(ft_pool* pool);
+
+/* Last CUDA error string seen by this library in this process (static storage). */
+const char* flowpool_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FLOWPOOL_H_ */

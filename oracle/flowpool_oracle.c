@@ -626,6 +626,13 @@ void oracle_balance(uint32_t n_mb, const uint64_t* cost, uint32_t K, uint32_t N,
   free(list); free(order);
 }
 
+/* argument check: the largest cost a microbatch can have, A*L + B*L^2, must fit 64 bits */
+static int cost_fits(const oracle_plan_config* cfg) {
+  unsigned __int128 mx = (unsigned __int128)cfg->coef_A * cfg->budget_L +
+                         (unsigned __int128)cfg->coef_B * cfg->budget_L * cfg->budget_L;
+  return (mx >> 64) == 0;
+}
+
 void oracle_plan_destroy_inner(oracle_plan* pl) {
   free(pl->slots); free(pl->slot_generation); free(pl->sample_len); free(pl->sample_cost);
   free(pl->sample_mb); free(pl->mb_sample_off); free(pl->mb_samples); free(pl->mb_tokens);
@@ -645,6 +652,7 @@ int32_t oracle_plan_from_lengths(const uint32_t* slots, const uint32_t* len, uin
   if (!cfg || !out) return OR_ERR_INVALID_ARG;
   const uint32_t L = cfg->budget_L, K = cfg->n_buckets_K, N = cfg->n_ranks_N;
   if (L == 0 || K == 0 || N == 0) return OR_ERR_INVALID_ARG;
+  if (!cost_fits(cfg)) return OR_ERR_INVALID_ARG;
   for (uint32_t t = 0; t < n; ++t) {
     if (len[t] == 0) return OR_ERR_INVALID_ARG;
     if (len[t] > L) return OR_ERR_TOO_LONG;
@@ -692,6 +700,7 @@ int32_t oracle_pool_plan_microbatches(oracle_pool* p, const uint32_t* slots, uin
   if (!p || !cfg || !out) return OR_ERR_INVALID_ARG;
   p->call_seq++;
   if (cfg->budget_L == 0 || cfg->n_buckets_K == 0 || cfg->n_ranks_N == 0) return OR_ERR_INVALID_ARG;
+  if (!cost_fits(cfg)) return OR_ERR_INVALID_ARG;
   if (n && !slots) return OR_ERR_INVALID_ARG;
   uint32_t* len = (uint32_t*)calloc((size_t)n + 1, sizeof(uint32_t));
   uint8_t* seen = (uint8_t*)calloc(p->c.max_samples, 1);

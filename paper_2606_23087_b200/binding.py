@@ -1,0 +1,222 @@
+"""ctypes binding of libflowpool.so: the same calls as include/flowpool.h, argument marshalling only.
+
+Device buffers are passed as integer addresses (torch tensors' data_ptr()); host arrays as numpy.
+There is no fallback: if the shared library is missing or cannot be loaded, importing this module fails.
+"""
+import ctypes as C
+import os
+
+import numpy as np
+
+from .build import SO, build
+
+FT_BF16, FT_F32 = 0, 1
+FT_RING_SORTED, FT_RING_SHUFFLED = 0, 1
+FT_BIND_IDENTITY, FT_BIND_PERMUTED = 0, 1
+FT_PLAN_ALLOW_UNWRITTEN = 1
+
+STATUS = {
+    0: "OK", -1: "INVALID_ARG", -2: "POOL_EXHAUSTED", -3: "UNKNOWN_SAMPLE", -4: "ALREADY_WRITTEN",
+    -5: "NOT_READY", -6: "TOO_LONG", -7: "BAD_GVA", -8: "PLACEHOLDER_MISMATCH", -9: "BAD_TOKEN_ID",
+    -10: "SLOT_IN_USE", -11: "CAPACITY", -12: "CUDA", -13: "TIMEOUT",
+}
+
+EXPORTS = (
+    "pool_create", "pool_register_samples", "pool_write_embeddings", "pool_plan_microbatches", "plan_summary",
+    "plan_arrays", "plan_destroy", "pool_gather_packed", "pool_free", "pool_status", "pool_stats",
+    "pool_debug_span_pages", "pool_debug_ring", "pool_debug_translate", "pool_destroy", "flowpool_last_cuda_error",
+)
+
+
+class FlowpoolError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = code
+        detail = ""
+        if code == -12:
+            detail = ": " + (lib().flowpool_last_cuda_error() or b"").decode()
+        super().__init__(f"{where}: FT_ERR_{STATUS.get(code, code)}{detail}")
+
+
+class PoolConfig(C.Structure):
+    _fields_ = [
+        ("page_bytes", C.c_uint64), ("hbm_pages", C.c_uint64), ("host_pages", C.c_uint64),
+        ("max_text_tokens", C.c_uint64), ("ring_seed", C.c_uint64), ("bind_seed", C.c_uint64),
+        ("gva_hbm_start", C.c_uint64), ("gva_host_start", C.c_uint64), ("max_size", C.c_uint64),
+        ("hidden", C.c_uint32), ("max_samples", C.c_uint32), ("max_spans_per_sample", C.c_uint32),
+        ("max_pages_per_span", C.c_uint32), ("max_seq_len", C.c_uint32),
+        ("placeholder_id", C.c_int32), ("ring_order", C.c_uint32), ("bind_order", C.c_uint32),
+        ("world_size", C.c_uint32), ("rank", C.c_uint32),
+    ]
+
+
+class PlanConfig(C.Structure):
+    _fields_ = [
+        ("coef_A", C.c_uint64), ("coef_B", C.c_uint64), ("budget_L", C.c_uint32),
+        ("n_buckets_K", C.c_uint32), ("n_ranks_N", C.c_uint32), ("flags", C.c_uint32),
+    ]
+
+
+class PoolStats(C.Structure):
+    _fields_ = [(k, C.c_uint64) for k in (
+        "pages_total", "pages_free", "hbm_pages", "host_pages", "text_pages_total", "text_pages_free",
+        "live_samples", "live_spans", "bytes_written", "bytes_gathered", "gpu_launches")]
+
+
+_lib = None
+
+
+def lib():
+    """The loaded shared library (built in-tree on first use when nvcc is available)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(SO):
+            build()
+        _lib = C.CDLL(SO)
+        P, u32, u64, i32 = C.c_void_p, C.c_uint32, C.c_uint64, C.c_int32
+        sig = {
+            "pool_create": [P, P, P, P],
+            "pool_register_samples": [P, u32, P, P, P, P, P, P, P],
+            "pool_write_embeddings": [P, u32, P, P, P, P, u32, P],
+            "pool_plan_microbatches": [P, P, u32, P, P, P],
+            "plan_summary": [P, P, P, P],
+            "plan_arrays": [P] * 13,
+            "plan_destroy": [P],
+            "pool_gather_packed": [P, P, u32, u32, P, u32, P, P, P, P],
+            "pool_free": [P, P, u32, P],
+            "pool_status": [P, P, P],
+            "pool_stats": [P, P],
+            "pool_debug_span_pages": [P, u32, u32, P, u32, P],
+            "pool_debug_ring": [P, P, u64, P],
+            "pool_debug_translate": [P, P, u32, P, P, P, P],
+            "pool_destroy": [P],
+        }
+        for name, argtypes in sig.items():
+            fn = getattr(_lib, name)
+            fn.argtypes, fn.restype = argtypes, i32
+        _lib.flowpool_last_cuda_error.restype = C.c_char_p
+        _lib.flowpool_last_cuda_error.argtypes = []
+    return _lib
+
+
+def _u32(a):
+    return np.ascontiguousarray(a, dtype=np.uint32)
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+class Plan:
+    def __init__(self, handle, n, n_ranks):
+        self.h, self.n, self.n_ranks = handle, n, n_ranks
+
+    def summary(self):
+        n_mb, tot, mx = C.c_uint32(), C.c_uint64(), C.c_uint32()
+        rc = lib().plan_summary(self.h, C.byref(n_mb), C.byref(tot), C.byref(mx))
+        if rc:
+            raise FlowpoolError(rc, "plan_summary")
+        return n_mb.value, tot.value, mx.value
+
+    def arrays(self):
+        n_mb = self.summary()[0]
+        n, N = self.n, self.n_ranks
+        a = {
+            "mb_sample_off": np.zeros(n_mb + 1, np.uint32), "mb_samples": np.zeros(n, np.uint32),
+            "mb_tokens": np.zeros(n_mb, np.uint32), "mb_lmax": np.zeros(n_mb, np.uint32),
+            "mb_residual": np.zeros(n_mb, np.uint32), "mb_cost": np.zeros(n_mb, np.uint64),
+            "mb_bucket": np.zeros(n_mb, np.uint32), "mb_rank": np.zeros(n_mb, np.uint32),
+            "rank_mb_off": np.zeros(N + 1, np.uint32), "rank_mbs": np.zeros(n_mb, np.uint32),
+            "sample_cost": np.zeros(n, np.uint64), "sample_mb": np.zeros(n, np.uint32),
+        }
+        rc = lib().plan_arrays(self.h, *[_p(v) for v in a.values()])
+        if rc:
+            raise FlowpoolError(rc, "plan_arrays")
+        a["n_mb"] = n_mb
+        return a
+
+    def destroy(self):
+        if self.h:
+            lib().plan_destroy(self.h)
+            self.h = None
+
+
+class Pool:
+    """Thin handle around ft_pool.  Every method returns the library's int32 status unchanged
+    (0 = OK); nothing is computed on the Python side."""
+
+    def __init__(self, cfg: PoolConfig, hbm_base: int = 0, host_base: int = 0):
+        self.cfg = cfg
+        self.h = C.c_void_p()
+        self.rc = lib().pool_create(C.byref(cfg), hbm_base or None, host_base or None, C.byref(self.h))
+        if self.rc != 0:
+            self.h = None
+
+    def destroy(self):
+        if self.h:
+            lib().pool_destroy(self.h)
+            self.h = None
+
+    def register_samples(self, slots, seq_len, n_spans, span_pos, span_tokens, input_ids_ptr: int, stream: int = 0):
+        slots, seq_len, n_spans = _u32(slots), _u32(seq_len), _u32(n_spans)
+        span_pos, span_tokens = _u32(span_pos), _u32(span_tokens)
+        return lib().pool_register_samples(self.h, len(slots), _p(slots), _p(seq_len), _p(n_spans), _p(span_pos),
+                                           _p(span_tokens), input_ids_ptr or None, stream or None)
+
+    def write_embeddings(self, slots, span_idx, n_tokens, src_ptrs, dtype, stream: int = 0):
+        slots, span_idx, n_tokens = _u32(slots), _u32(span_idx), _u32(n_tokens)
+        src = np.ascontiguousarray(src_ptrs, dtype=np.uint64)
+        return lib().pool_write_embeddings(self.h, len(slots), _p(slots), _p(span_idx), _p(n_tokens), _p(src),
+                                           dtype, stream or None)
+
+    def plan_microbatches(self, slots, cfg: PlanConfig, stream: int = 0):
+        slots = _u32(slots)
+        h = C.c_void_p()
+        rc = lib().pool_plan_microbatches(self.h, _p(slots), len(slots), C.byref(cfg), C.byref(h), stream or None)
+        return rc, (Plan(h, len(slots), cfg.n_ranks_N) if rc == 0 else None)
+
+    def gather_packed(self, plan: Plan, mb_begin, mb_end, table_ptr: int, vocab: int, out_ptr: int, cu_ptr: int,
+                      pos_ptr: int, stream: int = 0):
+        return lib().pool_gather_packed(self.h, plan.h, mb_begin, mb_end, table_ptr or None, vocab, out_ptr or None,
+                                        cu_ptr or None, pos_ptr or None, stream or None)
+
+    def free(self, slots, stream: int = 0):
+        slots = _u32(slots)
+        return lib().pool_free(self.h, _p(slots), len(slots), stream or None)
+
+    def status(self):
+        code, detail = C.c_int32(), C.c_uint64()
+        rc = lib().pool_status(self.h, C.byref(code), C.byref(detail))
+        if rc:
+            raise FlowpoolError(rc, "pool_status")
+        return code.value, detail.value
+
+    def stats(self):
+        s = PoolStats()
+        rc = lib().pool_stats(self.h, C.byref(s))
+        if rc:
+            raise FlowpoolError(rc, "pool_stats")
+        return {k: getattr(s, k) for k, _ in PoolStats._fields_}
+
+    def span_pages(self, slot, span, cap=1 << 16):
+        out = np.zeros(cap, np.uint64)
+        n = C.c_uint32()
+        rc = lib().pool_debug_span_pages(self.h, slot, span, _p(out), cap, C.byref(n))
+        return rc, out[: n.value].copy()
+
+    def ring(self):
+        total = self.cfg.hbm_pages + self.cfg.host_pages
+        out = np.zeros(total, np.uint32)
+        n = C.c_uint64()
+        rc = lib().pool_debug_ring(self.h, _p(out), total, C.byref(n))
+        if rc:
+            raise FlowpoolError(rc, "pool_debug_ring")
+        return out[: n.value].copy()
+
+    def translate(self, gvas):
+        g = np.ascontiguousarray(gvas, dtype=np.uint64)
+        kind, frame = np.zeros(len(g), np.uint32), np.zeros(len(g), np.uint64)
+        off, st = np.zeros(len(g), np.uint64), np.zeros(len(g), np.int32)
+        rc = lib().pool_debug_translate(self.h, _p(g), len(g), _p(kind), _p(frame), _p(off), _p(st))
+        if rc:
+            raise FlowpoolError(rc, "pool_debug_translate")
+        return st, kind, frame, off

@@ -1,0 +1,230 @@
+// Internal declarations of the flowpool CUDA library (sm_100a).  Not part of the ABI.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "../../include/flowpool.h"
+
+namespace ft {
+
+constexpr uint32_t kTextPageIds = 1024;       // ids per 4 KiB text page
+constexpr uint32_t kListBlock = 64;           // page GVAs per list block (two-level span page lists)
+constexpr uint32_t kNone = 0xFFFFFFFFu;
+constexpr uint64_t kPteValid = 1, kPteHost = 2, kPteText = 4, kPteFlagMask = 0xFF;
+
+struct RingState {
+  uint32_t head;   // index of the oldest free entry
+  uint32_t count;  // free entries
+};
+
+// Everything a kernel needs to know about a pool; passed by value.
+struct PoolView {
+  // GVA layout (Sec. 3.2): two regions, per-process segments
+  uint64_t region_start[2];  // start_HBM, start_DRAM
+  uint64_t region_bytes;     // world_size * max_size
+  uint64_t max_size;
+  uint64_t seg_base[2];      // this process's segment bases
+  uint64_t text_gva_base;    // first text page: seg_base[0] + hbm_pages * page_bytes
+  uint32_t rank, page_shift;
+  uint64_t page_bytes, hbm_pages, host_pages, text_pages;
+  uint32_t hidden, row_bytes;
+  int32_t placeholder_id;
+  uint32_t max_samples, spans_per_sample, text_pages_per_sample, blocks_per_span;
+  // page tables: entry = device-visible frame address | flags
+  const uint64_t* pte_hbm;
+  const uint64_t* pte_host;
+  const uint64_t* pte_text;
+  // FIFO free rings
+  uint32_t* ring;   RingState* ring_state;   uint32_t ring_cap;    // embedding pages (global page index)
+  uint32_t* tring;  RingState* tring_state;  uint32_t tring_cap;   // text pages
+  uint32_t* bring;  RingState* bring_state;  uint32_t bring_cap;   // list blocks
+  // sample table (by slot)
+  uint32_t* s_seq_len;
+  uint32_t* s_n_spans;
+  uint32_t* s_text_pages;  // [max_samples][text_pages_per_sample] text page index
+  // span table (span id = slot * spans_per_sample + j)
+  uint32_t* sp_pos;
+  uint32_t* sp_tokens;
+  uint32_t* sp_npages;     // 0 until written
+  uint32_t* sp_blocks;     // [span id][blocks_per_span] list block index
+  uint64_t* list_blocks;   // [bring_cap][kListBlock] page GVAs
+  unsigned long long* status;  // first asynchronous error key; ~0 = none
+};
+
+// key = call_seq << 40 | (-code) << 32 | detail ; the smallest key is reported
+__device__ __forceinline__ void note_error(const PoolView& v, uint64_t call_seq, int32_t code, uint32_t detail) {
+  unsigned long long key = (call_seq << 40) | ((unsigned long long)(uint32_t)(-code) << 32) | detail;
+  atomicMin(v.status, key);
+}
+
+__device__ __forceinline__ uint64_t page_gva(const PoolView& v, uint32_t global_page) {
+  return global_page < v.hbm_pages ? v.seg_base[0] + (uint64_t)global_page * v.page_bytes
+                                   : v.seg_base[1] + ((uint64_t)global_page - v.hbm_pages) * v.page_bytes;
+}
+
+// inverse of page_gva for a page GVA produced by it
+__device__ __forceinline__ uint32_t global_page_of(const PoolView& v, uint64_t gva) {
+  uint64_t d = gva - v.seg_base[1];
+  if (d < v.max_size) return (uint32_t)(v.hbm_pages + (d >> v.page_shift));
+  return (uint32_t)((gva - v.seg_base[0]) >> v.page_shift);
+}
+
+// GVA -> page-table entry (+ byte offset inside the frame).  Purely local: region by
+// interval test, process by division, virtual page number by shift (Sec. 3.2).
+// Returns 0 (no valid bit) when the GVA does not translate.
+__device__ __forceinline__ uint64_t translate(const PoolView& v, uint64_t gva, uint64_t* offset) {
+#pragma unroll
+  for (int t = 0; t < 2; ++t) {
+    uint64_t d = gva - v.region_start[t];
+    if (d >= v.region_bytes) continue;
+    uint64_t proc = d / v.max_size, o = d - proc * v.max_size;
+    if (proc != v.rank) return 0;
+    uint64_t pages = t == 0 ? v.hbm_pages : v.host_pages;
+    uint64_t vpn = o >> v.page_shift;
+    if (vpn < pages) {
+      *offset = o & (v.page_bytes - 1);
+      return t == 0 ? v.pte_hbm[vpn] : v.pte_host[vpn];
+    }
+    if (t == 0) {
+      uint64_t ot = o - (pages << v.page_shift);
+      uint64_t tp = ot / FT_TEXT_PAGE_BYTES;
+      if (tp < v.text_pages) {
+        *offset = ot % FT_TEXT_PAGE_BYTES;
+        return v.pte_text[tp];
+      }
+    }
+    return 0;
+  }
+  return 0;
+}
+
+// page GVA of ordinal o of a span, through the two-level list
+__device__ __forceinline__ uint64_t span_page_gva(const PoolView& v, uint32_t span_id, uint32_t o) {
+  uint32_t blk = v.sp_blocks[(uint64_t)span_id * v.blocks_per_span + o / kListBlock];
+  return v.list_blocks[(uint64_t)blk * kListBlock + o % kListBlock];
+}
+
+// block-wide exclusive scan of one value per thread (blockDim.x a multiple of 32, <= 1024);
+// returns the exclusive prefix, *total = block sum.  All threads must call.
+__device__ __forceinline__ uint64_t block_exclusive_scan(uint64_t x, uint64_t* total) {
+  __shared__ uint64_t warp_sums[32];
+  __shared__ uint64_t block_total;
+  const unsigned lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  uint64_t incl = x;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    uint64_t y = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+    if (lane >= (unsigned)d) incl += y;
+  }
+  __syncthreads();  // protect warp_sums from a previous call
+  if (lane == 31) warp_sums[wid] = incl;
+  __syncthreads();
+  if (wid == 0) {
+    uint64_t s = lane < nw ? warp_sums[lane] : 0, si = s;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      uint64_t y = __shfl_up_sync(0xFFFFFFFFu, si, d);
+      if (lane >= (unsigned)d) si += y;
+    }
+    if (lane < nw) warp_sums[lane] = si - s;
+    if (lane == 31) block_total = si;
+  }
+  __syncthreads();
+  *total = block_total;
+  return warp_sums[wid] + incl - x;
+}
+
+// ---- plan: device arrays and host summary -------------------------------------------------
+struct PlanView {
+  uint32_t n, n_mb, n_ranks;
+  const uint32_t* mb_samples;        // [n] slots, plan order
+  const uint32_t* plan_sample_mb;    // [n] microbatch of the sample at plan position q
+  const uint64_t* sample_row_off;    // [n+1] first output row of the sample at plan position q
+  const uint32_t* mb_sample_off;     // [n_mb+1]
+  const uint64_t* mb_row_off;        // [n_mb+1]
+  const uint32_t* tile_first_sample; // [ceil(rows/32)] plan position of the sample holding row 32*T
+};
+
+}  // namespace ft
+
+// ---- host-side objects -------------------------------------------------------------------
+struct ft_plan {
+  ft_pool* pool;
+  ft_plan_config cfg;
+  uint32_t n = 0, n_mb = 0;
+  uint64_t total_tokens = 0;
+  uint32_t max_mb_tokens = 0;
+  uint64_t free_epoch = 0;
+  std::vector<uint32_t> slots;            // caller's order
+  std::vector<uint64_t> slot_generation;
+  std::vector<uint32_t> h_mb_sample_off;  // host copies used to size gathers
+  std::vector<uint64_t> h_mb_row_off;
+  void* d_block = nullptr;                // one allocation holding every array below
+  uint32_t *d_slots, *d_len, *d_sample_mb, *d_sample_rank, *d_mb_sample_off, *d_mb_samples, *d_plan_sample_mb;
+  uint32_t *d_mb_tokens, *d_mb_lmax, *d_mb_residual, *d_mb_count, *d_mb_bucket, *d_mb_rank, *d_mb_pos;
+  uint32_t *d_rank_mb_off, *d_rank_mbs, *d_rank_cnt, *d_tile_first_sample, *d_scalars;
+  uint64_t *d_sample_cost, *d_mb_cost, *d_sample_row_off, *d_mb_row_off, *d_plan_len;
+};
+
+namespace ft {
+int32_t cuda_fail(cudaError_t e, const char* what);
+#define FT_CUDA(call)                                          \
+  do {                                                         \
+    cudaError_t e__ = (call);                                  \
+    if (e__ != cudaSuccess) return ft::cuda_fail(e__, #call);  \
+  } while (0)
+}  // namespace ft
+
+// ---- the pool's host object ----------------------------------------------------------------
+enum { FT_SLOT_FREE = 0, FT_SLOT_REGISTERED = 1, FT_SLOT_READY = 2 };
+
+struct ft_slot_mirror {
+  uint8_t state = FT_SLOT_FREE;
+  uint32_t seq_len = 0, n_spans = 0, spans_written = 0, n_text_pages = 0;
+  uint64_t generation = 0;
+};
+struct ft_span_mirror {
+  uint32_t pos = 0, tokens = 0, npages = 0;
+  bool written = false;
+};
+
+// Pinned staging for per-call descriptor uploads: a small ring of buffers, each guarded by an
+// event, so a call never rewrites host memory that an earlier asynchronous copy may still read.
+struct ft_staging {
+  static constexpr int kBufs = 8;
+  void* h[kBufs] = {};
+  size_t cap[kBufs] = {};
+  cudaEvent_t ev[kBufs] = {};
+  bool busy[kBufs] = {};
+  int next = 0;
+};
+
+struct ft_pool {
+  ft_pool_config cfg;
+  ft::PoolView view;
+  int device = 0;
+  std::vector<ft_slot_mirror> slots;
+  std::vector<ft_span_mirror> spans;  // [max_samples * spans_per_sample]
+  uint64_t free_pages = 0, free_text_pages = 0, free_blocks = 0;
+  uint64_t call_seq = 0, free_epoch = 0, live_samples = 0, live_spans = 0;
+  uint64_t bytes_written = 0, bytes_gathered = 0, gpu_launches = 0;
+  // allocations
+  void* d_meta = nullptr;      // page tables, rings, tables, list blocks, status
+  void* d_text = nullptr;      // text page frames
+  void* hbm_base = nullptr;    bool own_hbm = false;
+  void* host_base = nullptr;   bool own_host = false;  // host pointer
+  void* host_dev = nullptr;                            // the same memory as the device sees it
+  void* d_scratch = nullptr;   size_t scratch_cap = 0; // per-call descriptors and scan outputs
+  ft_staging staging;
+  cudaStream_t side_stream = nullptr;                  // host-tier traffic runs beside the HBM kernels
+  cudaEvent_t fork_ev = nullptr, join_ev = nullptr;
+  int sm_count = 148;
+};
+
+namespace ft {
+// uploads `bytes` from `src` (pageable) to the front of the pool's device scratch, asynchronously,
+// through the staging ring; afterwards at least `total_bytes` of scratch exist.  Returns the device pointer.
+int32_t stage_upload(ft_pool* p, const void* src, size_t bytes, size_t total_bytes, cudaStream_t st, void** d_out);
+}  // namespace ft

@@ -1,0 +1,202 @@
+// The consumer: GVA translation and packed-microbatch assembly (Sec. 3.1-3.2).
+//
+// k_gather: output rows are cut into tiles of 32 consecutive rows.  For each tile one warp resolves the
+// 32 row sources, one lane per row (plan position -> slot -> token id from the text page; a placeholder
+// position -> span -> page ordinal -> page GVA from the span's two-level list -> page-table entry), and
+// leaves the frame addresses in shared memory; then every warp of the CTA streams rows with 16-byte
+// vectors.  Rows that straddle pages carry one address per page touched.  With a two-tier pool the
+// kernel is launched twice, once per tier, so host-link reads never stall HBM reads.
+#include "flowpool_internal.cuh"
+
+namespace ft {
+
+constexpr int kTileRows = 32;
+constexpr int kMaxSeg = 10;  // pages one row can touch: row_bytes <= 32 KiB over 4 KiB pages, plus a straddle
+constexpr int kGatherThreads = 256;
+
+enum { kTierAll = 0, kTierDeviceOnly = 1, kTierHostOnly = 2 };
+
+struct RowDesc {
+  uint64_t seg[kMaxSeg];  // page-table entries (frame address | flags) of the pages the row touches
+  uint32_t off0;          // byte offset of the row inside its first page (0 for a text row)
+  uint32_t shift;         // log2(page bytes); 31 for a text row (one segment)
+  uint32_t nseg;          // 0 = nothing to copy
+  uint32_t pad;
+};
+
+struct GatherArgs {
+  uint32_t q_lo, q_hi, mb_begin;  // plan positions and first microbatch of the range
+  uint64_t row_lo, row_hi;        // plan-global output rows of the range
+  const uint8_t* table;
+  uint32_t vocab;
+  uint8_t* out;
+  int32_t* cu;
+  int32_t* pos_ids;
+  uint64_t call_seq;
+  uint32_t write_index;  // this launch writes cu_seqlens / position ids
+};
+
+template <int MODE>
+__global__ void __launch_bounds__(kGatherThreads) k_gather(PoolView v, PlanView pl, GatherArgs a) {
+  __shared__ RowDesc desc[kTileRows];
+  const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const uint64_t tile_lo = a.row_lo / kTileRows, tile_hi = (a.row_hi + kTileRows - 1) / kTileRows;
+  const uint32_t row_vecs = v.row_bytes >> 4;
+
+  for (uint64_t tile = tile_lo + blockIdx.x; tile < tile_hi; tile += gridDim.x) {
+    if (warp == 0) {
+      const uint64_t row = tile * kTileRows + lane;
+      RowDesc d;
+      d.nseg = 0; d.off0 = 0; d.shift = 31; d.pad = 0;
+      if (row >= a.row_lo && row < a.row_hi) {
+        // plan position of the sample holding this row: the tile's first sample, then a short walk
+        uint32_t q = pl.tile_first_sample[tile];
+        if (q < a.q_lo) q = a.q_lo;
+        while (row >= pl.sample_row_off[q + 1]) ++q;
+        const uint32_t p = (uint32_t)(row - pl.sample_row_off[q]);
+        const uint32_t slot = pl.mb_samples[q];
+        const uint64_t out_row = row - a.row_lo;
+        if (a.write_index) {
+          a.pos_ids[out_row] = (int32_t)p;
+          if (p == 0) {  // cu_seqlens: every sample writes its start; the last of a microbatch also the end
+            const uint32_t j = pl.plan_sample_mb[q];
+            const uint64_t e = (uint64_t)(q - a.q_lo) + (j - a.mb_begin);
+            a.cu[e] = (int32_t)(pl.sample_row_off[q] - pl.mb_row_off[j]);
+            if (q + 1 == pl.mb_sample_off[j + 1]) a.cu[e + 1] = (int32_t)(pl.sample_row_off[q + 1] - pl.mb_row_off[j]);
+          }
+        }
+        // token id, through the text page
+        const uint32_t tp = v.s_text_pages[(uint64_t)slot * v.text_pages_per_sample + p / kTextPageIds];
+        uint64_t off;
+        const uint64_t tpte = translate(v, v.text_gva_base + (uint64_t)tp * FT_TEXT_PAGE_BYTES, &off);
+        const int32_t id = reinterpret_cast<const int32_t*>(tpte & ~kPteFlagMask)[p % kTextPageIds];
+        if (id != v.placeholder_id) {
+          if (id < 0 || (uint32_t)id >= a.vocab) {
+            note_error(v, a.call_seq, FT_ERR_BAD_TOKEN_ID, (uint32_t)out_row);
+          } else {
+            // a table row is one segment in device memory: the low address bits ride in off0
+            const uint64_t addr = reinterpret_cast<uint64_t>(a.table + (uint64_t)id * v.row_bytes);
+            d.seg[0] = addr & ~kPteFlagMask;
+            d.off0 = (uint32_t)(addr & kPteFlagMask);
+            d.nseg = 1;
+          }
+        } else {
+          // the span whose run contains p: last span with pos_start <= p
+          const uint32_t sbase = slot * v.spans_per_sample, ns = v.s_n_spans[slot];
+          uint32_t lo = 0, hi = ns;
+          while (lo < hi) {
+            const uint32_t mid = (lo + hi) >> 1;
+            if (v.sp_pos[sbase + mid] <= p) lo = mid + 1; else hi = mid;
+          }
+          const uint32_t sid = sbase + lo - 1;
+          const uint64_t b = (uint64_t)(p - v.sp_pos[sid]) * v.row_bytes;  // byte offset inside the span image
+          const uint32_t o0 = (uint32_t)(b >> v.page_shift);
+          d.off0 = (uint32_t)(b & (v.page_bytes - 1));
+          d.shift = v.page_shift;
+          const uint32_t nseg = ((d.off0 + v.row_bytes - 1) >> v.page_shift) + 1;
+          bool ok = lo > 0 && nseg <= kMaxSeg;
+          for (uint32_t s = 0; ok && s < nseg; ++s) {
+            uint64_t poff;
+            const uint64_t pte = translate(v, span_page_gva(v, sid, o0 + s), &poff);
+            ok = (pte & kPteValid) && !(pte & kPteText);
+            d.seg[s] = pte;
+          }
+          if (ok) d.nseg = nseg; else note_error(v, a.call_seq, FT_ERR_BAD_GVA, (uint32_t)out_row);
+        }
+      }
+      desc[lane] = d;
+    }
+    __syncthreads();
+    for (uint32_t r = warp; r < kTileRows; r += kGatherThreads / 32) {
+      const uint32_t nseg = desc[r].nseg;
+      if (nseg == 0) continue;
+      const uint32_t off0 = desc[r].off0, shift = desc[r].shift, mask = (1u << shift) - 1;
+      uint4* dst = reinterpret_cast<uint4*>(a.out + (tile * kTileRows + r - a.row_lo) * v.row_bytes);
+      auto src_of = [&](uint32_t x, bool* take) -> const uint4* {
+        const uint32_t ab = off0 + (x << 4);
+        const uint64_t pte = desc[r].seg[ab >> shift];
+        const bool host = (pte & kPteHost) != 0;
+        *take = MODE == kTierAll || (MODE == kTierHostOnly) == host;
+        return reinterpret_cast<const uint4*>((pte & ~kPteFlagMask) + (ab & mask));
+      };
+      uint32_t x = lane;
+      for (; x + 96 < row_vecs; x += 128) {
+        bool t0, t1, t2, t3;
+        const uint4* s0 = src_of(x, &t0);
+        const uint4* s1 = src_of(x + 32, &t1);
+        const uint4* s2 = src_of(x + 64, &t2);
+        const uint4* s3 = src_of(x + 96, &t3);
+        uint4 a0, a1, a2, a3;
+        if (t0) a0 = __ldcs(s0);
+        if (t1) a1 = __ldcs(s1);
+        if (t2) a2 = __ldcs(s2);
+        if (t3) a3 = __ldcs(s3);
+        if (t0) __stcs(dst + x, a0);
+        if (t1) __stcs(dst + x + 32, a1);
+        if (t2) __stcs(dst + x + 64, a2);
+        if (t3) __stcs(dst + x + 96, a3);
+      }
+      for (; x < row_vecs; x += 32) {
+        bool t0;
+        const uint4* s0 = src_of(x, &t0);
+        if (t0) __stcs(dst + x, __ldcs(s0));
+      }
+    }
+    __syncthreads();
+  }
+}
+
+}  // namespace ft
+
+using namespace ft;
+
+extern "C" __attribute__((visibility("default"))) int32_t pool_gather_packed(ft_pool* p, const ft_plan* pl, uint32_t mb_begin, uint32_t mb_end,
+                                      const void* embed_table, uint32_t vocab, void* out_embeds, int32_t* out_cu,
+                                      int32_t* out_pos, void* stream) {
+  if (!p || !pl || pl->pool != p) return FT_ERR_INVALID_ARG;
+  p->call_seq++;
+  if (mb_begin > mb_end || mb_end > pl->n_mb) return FT_ERR_INVALID_ARG;
+  // a plan dies with any of its samples (freed, or never completed under ALLOW_UNWRITTEN)
+  if (pl->free_epoch != p->free_epoch || (pl->cfg.flags & FT_PLAN_ALLOW_UNWRITTEN)) {
+    for (uint32_t t = 0; t < pl->n; ++t) {
+      const ft_slot_mirror& s = p->slots[pl->slots[t]];
+      if (s.state != FT_SLOT_READY || s.generation != pl->slot_generation[t]) return FT_ERR_NOT_READY;
+    }
+  }
+  if (mb_begin == mb_end) return FT_OK;
+  if (!embed_table || !out_embeds || !out_cu || !out_pos) return FT_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(out_embeds) & 15 || reinterpret_cast<uintptr_t>(embed_table) & 15) return FT_ERR_INVALID_ARG;
+  if (p->view.row_bytes > (kMaxSeg - 1) * 4096) return FT_ERR_CAPACITY;
+
+  PlanView pv;
+  pv.n = pl->n; pv.n_mb = pl->n_mb; pv.n_ranks = pl->cfg.n_ranks_N;
+  pv.mb_samples = pl->d_mb_samples; pv.plan_sample_mb = pl->d_plan_sample_mb;
+  pv.sample_row_off = pl->d_sample_row_off; pv.mb_sample_off = pl->d_mb_sample_off;
+  pv.mb_row_off = pl->d_mb_row_off; pv.tile_first_sample = pl->d_tile_first_sample;
+  GatherArgs a;
+  a.q_lo = pl->h_mb_sample_off[mb_begin]; a.q_hi = pl->h_mb_sample_off[mb_end]; a.mb_begin = mb_begin;
+  a.row_lo = pl->h_mb_row_off[mb_begin]; a.row_hi = pl->h_mb_row_off[mb_end];
+  a.table = static_cast<const uint8_t*>(embed_table); a.vocab = vocab;
+  a.out = static_cast<uint8_t*>(out_embeds); a.cu = out_cu; a.pos_ids = out_pos;
+  a.call_seq = p->call_seq; a.write_index = 1;
+  const uint64_t n_tiles = (a.row_hi + kTileRows - 1) / kTileRows - a.row_lo / kTileRows;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  auto grid_for = [&](uint32_t per_sm) { return (unsigned)std::min<uint64_t>(n_tiles, (uint64_t)p->sm_count * per_sm); };
+  if (p->cfg.host_pages == 0 || p->cfg.hbm_pages == 0) {
+    k_gather<kTierAll><<<grid_for(8), kGatherThreads, 0, st>>>(p->view, pv, a);
+    p->gpu_launches += 1;
+  } else {
+    FT_CUDA(cudaEventRecord(p->fork_ev, st));
+    FT_CUDA(cudaStreamWaitEvent(p->side_stream, p->fork_ev, 0));
+    GatherArgs ah = a;
+    ah.write_index = 0;
+    k_gather<kTierHostOnly><<<grid_for(2), kGatherThreads, 0, p->side_stream>>>(p->view, pv, ah);
+    FT_CUDA(cudaEventRecord(p->join_ev, p->side_stream));
+    k_gather<kTierDeviceOnly><<<grid_for(8), kGatherThreads, 0, st>>>(p->view, pv, a);
+    FT_CUDA(cudaStreamWaitEvent(st, p->join_ev, 0));
+    p->gpu_launches += 2;
+  }
+  FT_CUDA(cudaGetLastError());
+  p->bytes_gathered += (a.row_hi - a.row_lo) * 2ull * p->view.row_bytes;
+  return FT_OK;
+}

@@ -1,0 +1,459 @@
+// The dynamic packing rule on the device (Sec. 3.4, Algorithm 1, Eq. 3).
+//
+// Kernels in this file
+//   k_plan_prepare   l(s) from the pool's sample table, per-sample score (Eq. 3 on a singleton)
+//   k_bestfit        Algorithm 1 lines 1-11: online best fit.  The paper's segment tree over [0, L]
+//                    becomes a 32-ary bitmap hierarchy in shared memory (find-next-set = best-fit query,
+//                    same answer, O(log_32 L)); per-residual LIFO stacks give the tie rule.
+//   k_mb_finalize    Cost(B_j), min/max cost, exclusive scans -> mb_sample_off, mb_row_off
+//   k_plan_scatter   samples into microbatch-major, append order
+//   k_row_offsets    exclusive scan of lengths in plan order
+//   k_tiles          plan position of the sample holding each 32-row output tile
+//   k_bucket         lines 12-14: equal-width cost buckets
+//   k_sort_deal      lines 15-27: rank-by-counting sort (bucket desc, cost desc, index asc), zig-zag deal
+//   k_rank_index/_scan/_lists  per-rank lists in dispatch order
+#include <algorithm>
+#include <cstring>
+
+#include "flowpool_internal.cuh"
+
+namespace ft {
+
+struct MbRec { uint32_t residual, lmax, count, next; };
+
+constexpr uint32_t kFitChunk = 2048;  // samples staged through shared memory per round
+enum { SC_NMB = 0, SC_MAXTOK = 1, SC_TOTAL_LO = 2, SC_TOTAL_HI = 3, SC_LO = 4, SC_HI = 6, SC_COUNT = 8 };
+
+__global__ void k_plan_prepare(PoolView v, const uint32_t* slots, uint32_t n, uint64_t A, uint64_t B, uint32_t* len,
+                               uint64_t* sample_cost) {
+  const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= n) return;
+  const uint64_t l = v.s_seq_len[slots[t]];  // l(s): the LLM-side length, text + all vision tokens
+  len[t] = (uint32_t)l;
+  sample_cost[t] = A * l + B * l * l;
+}
+
+struct FitLevels {
+  uint32_t* bits[4];
+  uint32_t words[4];
+};
+
+__device__ __forceinline__ uint32_t fit_find(const FitLevels& f, uint32_t l) {
+  // smallest set index >= l, or kNone
+  uint32_t idx = l;
+#pragma unroll
+  for (int lvl = 0; lvl < 4; ++lvl) {
+    const uint32_t w = idx >> 5, b = idx & 31;
+    if (w < f.words[lvl]) {
+      const uint32_t m = f.bits[lvl][w] & (0xFFFFFFFFu << b);
+      if (m) {
+        uint32_t pos = (w << 5) + __ffs(m) - 1;
+        for (int d = lvl - 1; d >= 0; --d) pos = (pos << 5) + __ffs(f.bits[d][pos]) - 1;
+        return pos;
+      }
+    }
+    idx = w + 1;
+  }
+  return kNone;
+}
+__device__ __forceinline__ void fit_set(const FitLevels& f, uint32_t r) {
+#pragma unroll
+  for (int lvl = 0; lvl < 4; ++lvl) {
+    const uint32_t old = f.bits[lvl][r >> 5];
+    f.bits[lvl][r >> 5] = old | (1u << (r & 31));
+    if (old) return;
+    r >>= 5;
+  }
+}
+__device__ __forceinline__ void fit_clear(const FitLevels& f, uint32_t r) {
+#pragma unroll
+  for (int lvl = 0; lvl < 4; ++lvl) {
+    const uint32_t nw = f.bits[lvl][r >> 5] & ~(1u << (r & 31));
+    f.bits[lvl][r >> 5] = nw;
+    if (nw) return;
+    r >>= 5;
+  }
+}
+
+// One block.  Thread 0 walks the samples in order (the dependency chain of online best fit); the other
+// threads stage lengths in and results out, coalesced, and initialise / flush the tables.
+__global__ void __launch_bounds__(1024) k_bestfit(const uint32_t* __restrict__ len, uint32_t n, uint32_t L,
+                                                  uint32_t* head_g, MbRec* recs_g, uint32_t head_in_smem,
+                                                  uint32_t rec_smem_cap, uint32_t* sample_mb, uint32_t* sample_rank,
+                                                  uint32_t* mb_residual, uint32_t* mb_tokens, uint32_t* mb_lmax,
+                                                  uint32_t* mb_count, uint32_t* scalars) {
+  extern __shared__ uint32_t sm[];
+  FitLevels f;
+  uint32_t* p = sm;
+  uint32_t w = (L + 1 + 31) / 32;
+  uint32_t total_words = 0;
+  for (int lvl = 0; lvl < 4; ++lvl) {
+    f.bits[lvl] = p; f.words[lvl] = w; p += w; total_words += w;
+    w = (w + 31) / 32;
+  }
+  uint32_t* c_len = p; p += kFitChunk;
+  uint32_t* c_mb = p; p += kFitChunk;
+  uint32_t* c_rank = p; p += kFitChunk;
+  uint32_t* head = head_g;
+  if (head_in_smem) { head = p; p += L + 1; }
+  p += (4 - ((p - sm) & 3)) & 3;  // 16-byte align the records
+  MbRec* recs_s = reinterpret_cast<MbRec*>(p);
+
+  for (uint32_t i = threadIdx.x; i < total_words; i += blockDim.x) sm[i] = 0;
+  for (uint32_t i = threadIdx.x; i <= L; i += blockDim.x) head[i] = kNone;
+  __shared__ uint32_t s_nmb;
+  if (threadIdx.x == 0) s_nmb = 0;
+  __syncthreads();
+
+  for (uint32_t base = 0; base < n; base += kFitChunk) {
+    const uint32_t cnt = min(kFitChunk, n - base);
+    for (uint32_t i = threadIdx.x; i < cnt; i += blockDim.x) c_len[i] = len[base + i];
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      uint32_t n_mb = s_nmb;
+      for (uint32_t i = 0; i < cnt; ++i) {
+        const uint32_t l = c_len[i];
+        const uint32_t r = fit_find(f, l);  // the smallest residual >= l among open microbatches
+        uint32_t j;
+        MbRec rec;
+        if (r != kNone) {
+          j = head[r];  // most recently changed microbatch with that residual
+          rec = j < rec_smem_cap ? recs_s[j] : recs_g[j];
+          head[r] = rec.next;
+          if (rec.next == kNone) fit_clear(f, r);
+          rec.residual = r - l;
+          rec.lmax = max(rec.lmax, l);
+          rec.count++;
+        } else {
+          j = n_mb++;
+          rec.residual = L - l; rec.lmax = l; rec.count = 1;
+        }
+        // a residual of 0 can never be chosen again (l >= 1): it needs no stack entry
+        if (rec.residual) {
+          rec.next = head[rec.residual];
+          head[rec.residual] = j;
+          if (rec.next == kNone) fit_set(f, rec.residual);
+        } else {
+          rec.next = kNone;
+        }
+        if (j < rec_smem_cap) recs_s[j] = rec; else recs_g[j] = rec;
+        c_mb[i] = j;
+        c_rank[i] = rec.count - 1;
+      }
+      s_nmb = n_mb;
+    }
+    __syncthreads();
+    for (uint32_t i = threadIdx.x; i < cnt; i += blockDim.x) { sample_mb[base + i] = c_mb[i]; sample_rank[base + i] = c_rank[i]; }
+    __syncthreads();
+  }
+  const uint32_t n_mb = s_nmb;
+  for (uint32_t j = threadIdx.x; j < n_mb; j += blockDim.x) {
+    const MbRec rec = j < rec_smem_cap ? recs_s[j] : recs_g[j];
+    mb_residual[j] = rec.residual; mb_tokens[j] = L - rec.residual; mb_lmax[j] = rec.lmax; mb_count[j] = rec.count;
+  }
+  if (threadIdx.x == 0) scalars[SC_NMB] = n_mb;
+}
+
+__global__ void __launch_bounds__(1024) k_mb_finalize(uint64_t A, uint64_t B, const uint32_t* mb_tokens,
+                                                      const uint32_t* mb_lmax, const uint32_t* mb_count, uint64_t* mb_cost,
+                                                      uint32_t* mb_sample_off, uint64_t* mb_row_off, uint32_t* scalars) {
+  __shared__ unsigned long long s_lo, s_hi;
+  __shared__ uint32_t s_max;
+  const uint32_t n_mb = scalars[SC_NMB];
+  if (threadIdx.x == 0) { s_lo = ~0ull; s_hi = 0; s_max = 0; }
+  __syncthreads();
+  uint64_t cs = 0, cr = 0;
+  for (uint32_t base = 0; base < n_mb; base += blockDim.x) {
+    const uint32_t j = base + threadIdx.x;
+    uint64_t cnt = 0, tok = 0;
+    if (j < n_mb) {
+      cnt = mb_count[j]; tok = mb_tokens[j];
+      const uint64_t lm = mb_lmax[j];
+      const uint64_t cost = A * tok + B * lm * lm;  // Eq. 3 times L^2 when (A, B) = (L, 1)
+      mb_cost[j] = cost;
+      atomicMin(&s_lo, (unsigned long long)cost);
+      atomicMax(&s_hi, (unsigned long long)cost);
+      atomicMax(&s_max, (uint32_t)tok);
+    }
+    uint64_t ts, tr;
+    const uint64_t es = block_exclusive_scan(cnt, &ts);
+    const uint64_t er = block_exclusive_scan(tok, &tr);
+    if (j < n_mb) { mb_sample_off[j] = (uint32_t)(cs + es); mb_row_off[j] = cr + er; }
+    cs += ts; cr += tr;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    mb_sample_off[n_mb] = (uint32_t)cs; mb_row_off[n_mb] = cr;
+    scalars[SC_MAXTOK] = s_max;
+    scalars[SC_TOTAL_LO] = (uint32_t)cr; scalars[SC_TOTAL_HI] = (uint32_t)(cr >> 32);
+    *reinterpret_cast<unsigned long long*>(scalars + SC_LO) = s_lo;
+    *reinterpret_cast<unsigned long long*>(scalars + SC_HI) = s_hi;
+  }
+}
+
+__global__ void k_plan_scatter(const uint32_t* slots, const uint32_t* len, const uint32_t* sample_mb,
+                               const uint32_t* sample_rank, const uint32_t* mb_sample_off, uint32_t n,
+                               uint32_t* mb_samples, uint64_t* plan_len, uint32_t* plan_sample_mb) {
+  const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= n) return;
+  const uint32_t j = sample_mb[t], q = mb_sample_off[j] + sample_rank[t];  // append order = arrival order
+  mb_samples[q] = slots[t];
+  plan_len[q] = len[t];
+  plan_sample_mb[q] = j;
+}
+
+__global__ void __launch_bounds__(1024) k_row_offsets(const uint64_t* plan_len, uint32_t n, uint64_t* sample_row_off) {
+  uint64_t carry = 0;
+  for (uint32_t base = 0; base < n; base += blockDim.x) {
+    const uint32_t q = base + threadIdx.x;
+    uint64_t total;
+    const uint64_t ex = block_exclusive_scan(q < n ? plan_len[q] : 0, &total);
+    if (q < n) sample_row_off[q] = carry + ex;
+    carry += total;
+  }
+  if (threadIdx.x == 0) sample_row_off[n] = carry;
+}
+
+__global__ void k_tiles(const uint64_t* sample_row_off, uint32_t n, uint32_t* tile_first_sample) {
+  const uint32_t q = blockIdx.x * blockDim.x + threadIdx.x;
+  if (q >= n) return;
+  const uint64_t t0 = (sample_row_off[q] + 31) / 32, t1 = (sample_row_off[q + 1] + 31) / 32;
+  for (uint64_t t = t0; t < t1; ++t) tile_first_sample[t] = q;  // rows 32t lies inside sample q
+}
+
+__global__ void k_bucket(const uint64_t* mb_cost, uint32_t K, const uint32_t* scalars, uint32_t* mb_bucket) {
+  const uint32_t j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= scalars[SC_NMB]) return;
+  const uint64_t lo = *reinterpret_cast<const unsigned long long*>(scalars + SC_LO);
+  const uint64_t hi = *reinterpret_cast<const unsigned long long*>(scalars + SC_HI);
+  const unsigned __int128 num = (unsigned __int128)(mb_cost[j] - lo) * K;
+  mb_bucket[j] = (uint32_t)(num / ((unsigned __int128)(hi - lo) + 1));
+}
+
+// Sorted position by counting: i comes before j when its bucket is higher, or equal bucket and cost higher,
+// or both equal and i < j.  Position inside the bucket -> zig-zag rank: round a/N forward when even.
+__global__ void k_sort_deal(const uint64_t* mb_cost, const uint32_t* mb_bucket, uint32_t N, const uint32_t* scalars,
+                            uint32_t* mb_pos, uint32_t* mb_rank) {
+  const uint32_t j = blockIdx.x * blockDim.x + threadIdx.x;
+  const uint32_t n_mb = scalars[SC_NMB];
+  if (j >= n_mb) return;
+  const uint64_t cj = mb_cost[j];
+  const uint32_t bj = mb_bucket[j];
+  uint32_t before = 0, higher = 0;
+  for (uint32_t i = 0; i < n_mb; ++i) {
+    const uint32_t bi = mb_bucket[i];
+    const uint64_t ci = mb_cost[i];
+    higher += bi > bj;
+    before += (bi > bj) || (bi == bj && (ci > cj || (ci == cj && i < j)));
+  }
+  const uint32_t a = before - higher;  // index in the bucket's descending list
+  const uint32_t rnd = a / N, i = a % N;
+  mb_pos[j] = before;
+  mb_rank[j] = (rnd & 1) ? N - 1 - i : i;
+}
+
+__global__ void k_rank_index(const uint32_t* mb_pos, const uint32_t* mb_rank, const uint32_t* scalars, uint32_t* mb_idx,
+                             uint32_t* rank_cnt) {
+  const uint32_t j = blockIdx.x * blockDim.x + threadIdx.x;
+  const uint32_t n_mb = scalars[SC_NMB];
+  if (j >= n_mb) return;
+  const uint32_t rj = mb_rank[j], pj = mb_pos[j];
+  uint32_t idx = 0;
+  for (uint32_t i = 0; i < n_mb; ++i) idx += (mb_rank[i] == rj) && (mb_pos[i] < pj);
+  mb_idx[j] = idx;
+  atomicAdd(&rank_cnt[rj], 1u);
+}
+
+__global__ void __launch_bounds__(1024) k_rank_scan(const uint32_t* rank_cnt, uint32_t N, uint32_t* rank_mb_off) {
+  uint64_t carry = 0;
+  for (uint32_t base = 0; base < N; base += blockDim.x) {
+    const uint32_t r = base + threadIdx.x;
+    uint64_t total;
+    const uint64_t ex = block_exclusive_scan(r < N ? rank_cnt[r] : 0, &total);
+    if (r < N) rank_mb_off[r] = (uint32_t)(carry + ex);
+    carry += total;
+  }
+  if (threadIdx.x == 0) rank_mb_off[N] = (uint32_t)carry;
+}
+
+__global__ void k_rank_lists(const uint32_t* mb_rank, const uint32_t* mb_idx, const uint32_t* rank_mb_off,
+                             const uint32_t* scalars, uint32_t* rank_mbs) {
+  const uint32_t j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= scalars[SC_NMB]) return;
+  rank_mbs[rank_mb_off[mb_rank[j]] + mb_idx[j]] = j;
+}
+
+static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace ft
+
+using namespace ft;
+
+extern "C" __attribute__((visibility("default"))) int32_t plan_destroy(ft_plan* pl) {
+  if (!pl) return FT_ERR_INVALID_ARG;
+  if (pl->d_block) { cudaDeviceSynchronize(); cudaFree(pl->d_block); }
+  delete pl;
+  return FT_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int32_t pool_plan_microbatches(ft_pool* p, const uint32_t* slot, uint32_t n, const ft_plan_config* cfg,
+                                          ft_plan** out, void* stream) {
+  if (!p || !cfg || !out) return FT_ERR_INVALID_ARG;
+  p->call_seq++;
+  const uint32_t L = cfg->budget_L, K = cfg->n_buckets_K, N = cfg->n_ranks_N;
+  if (L == 0 || K == 0 || N == 0) return FT_ERR_INVALID_ARG;
+  if (L >= (1u << 20)) return FT_ERR_CAPACITY;  // the bitmap hierarchy covers residuals below 2^20
+  {  // the largest possible cost A*L + B*L^2 must fit 64 bits
+    const unsigned __int128 mx = (unsigned __int128)cfg->coef_A * L + (unsigned __int128)cfg->coef_B * L * L;
+    if (mx >> 64) return FT_ERR_INVALID_ARG;
+  }
+  if (n && !slot) return FT_ERR_INVALID_ARG;
+  const ft_pool_config& c = p->cfg;
+  {
+    std::vector<uint8_t> seen(c.max_samples, 0);
+    for (uint32_t t = 0; t < n; ++t) {
+      if (slot[t] >= c.max_samples) return FT_ERR_INVALID_ARG;
+      const ft_slot_mirror& s = p->slots[slot[t]];
+      if (s.state == FT_SLOT_FREE) return FT_ERR_UNKNOWN_SAMPLE;
+      if (seen[slot[t]]) return FT_ERR_INVALID_ARG;
+      if (s.state != FT_SLOT_READY && !(cfg->flags & FT_PLAN_ALLOW_UNWRITTEN)) return FT_ERR_NOT_READY;
+      if (s.seq_len > L) return FT_ERR_TOO_LONG;
+      seen[slot[t]] = 1;
+    }
+  }
+  ft_plan* pl = new ft_plan();
+  pl->pool = p; pl->cfg = *cfg; pl->n = n; pl->free_epoch = p->free_epoch;
+  pl->slots.assign(slot, slot + n);
+  pl->slot_generation.resize(n);
+  uint64_t total_tokens = 0;
+  for (uint32_t t = 0; t < n; ++t) { pl->slot_generation[t] = p->slots[slot[t]].generation; total_tokens += p->slots[slot[t]].seq_len; }
+  if (n == 0) {
+    pl->h_mb_sample_off.assign(1, 0); pl->h_mb_row_off.assign(1, 0);
+    *out = pl;
+    return FT_OK;
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const uint64_t n_tiles = (total_tokens + 31) / 32 + 1;
+
+  // one device block for every plan array
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  const size_t n1 = (size_t)n + 1;
+  const size_t o_cost = take(n * 8), o_mbcost = take(n * 8), o_srow = take(n1 * 8), o_mbrow = take(n1 * 8), o_plen = take(n * 8);
+  const size_t o_recs = take(n * sizeof(MbRec)), o_head = take(((size_t)L + 1) * 4);
+  const size_t o_slots = take(n * 4), o_len = take(n * 4), o_smb = take(n * 4), o_srank = take(n * 4);
+  const size_t o_mboff = take(n1 * 4), o_mbs = take(n * 4), o_psmb = take(n * 4);
+  const size_t o_tok = take(n * 4), o_lmax = take(n * 4), o_res = take(n * 4), o_cnt = take(n * 4);
+  const size_t o_bkt = take(n * 4), o_rank = take(n * 4), o_pos = take(n * 4), o_idx = take(n * 4);
+  const size_t o_roff = take(((size_t)N + 1) * 4), o_rmbs = take(n * 4), o_rcnt = take((size_t)N * 4);
+  const size_t o_tiles = take(n_tiles * 4), o_scal = take(SC_COUNT * 4);
+  cudaError_t e = cudaMalloc(&pl->d_block, off);
+  if (e != cudaSuccess) { delete pl; return ft::cuda_fail(e, "cudaMalloc(plan)"); }
+  uint8_t* b = static_cast<uint8_t*>(pl->d_block);
+#define U32(o) reinterpret_cast<uint32_t*>(b + (o))
+#define U64(o) reinterpret_cast<uint64_t*>(b + (o))
+  pl->d_sample_cost = U64(o_cost); pl->d_mb_cost = U64(o_mbcost); pl->d_sample_row_off = U64(o_srow);
+  pl->d_mb_row_off = U64(o_mbrow); pl->d_plan_len = U64(o_plen);
+  pl->d_slots = U32(o_slots); pl->d_len = U32(o_len); pl->d_sample_mb = U32(o_smb); pl->d_sample_rank = U32(o_srank);
+  pl->d_mb_sample_off = U32(o_mboff); pl->d_mb_samples = U32(o_mbs); pl->d_plan_sample_mb = U32(o_psmb);
+  pl->d_mb_tokens = U32(o_tok); pl->d_mb_lmax = U32(o_lmax); pl->d_mb_residual = U32(o_res); pl->d_mb_count = U32(o_cnt);
+  pl->d_mb_bucket = U32(o_bkt); pl->d_mb_rank = U32(o_rank); pl->d_mb_pos = U32(o_pos);
+  pl->d_rank_mb_off = U32(o_roff); pl->d_rank_mbs = U32(o_rmbs); pl->d_rank_cnt = U32(o_rcnt);
+  pl->d_tile_first_sample = U32(o_tiles); pl->d_scalars = U32(o_scal);
+  uint32_t* d_mb_idx = U32(o_idx);
+  MbRec* d_recs = reinterpret_cast<MbRec*>(b + o_recs);
+  uint32_t* d_head = U32(o_head);
+
+  int32_t rc = FT_OK;
+#define CK(call)                                                                            \
+  do {                                                                                      \
+    cudaError_t e__ = (call);                                                               \
+    if (e__ != cudaSuccess) { rc = ft::cuda_fail(e__, #call); plan_destroy(pl); return rc; } \
+  } while (0)
+  // the slot list goes up through the pool's staging ring (scratch front), then into the plan
+  void* d_up = nullptr;
+  rc = stage_upload(p, slot, (size_t)n * 4, (size_t)n * 4, st, &d_up);
+  if (rc != FT_OK) { plan_destroy(pl); return rc; }
+  CK(cudaMemcpyAsync(pl->d_slots, d_up, (size_t)n * 4, cudaMemcpyDeviceToDevice, st));
+  CK(cudaMemsetAsync(pl->d_rank_cnt, 0, (size_t)N * 4, st));
+
+  const unsigned gb = (n + 255) / 256;
+  k_plan_prepare<<<gb, 256, 0, st>>>(p->view, pl->d_slots, n, cfg->coef_A, cfg->coef_B, pl->d_len, pl->d_sample_cost);
+
+  // shared memory plan of k_bestfit: bitmaps, staging chunk, then the stack heads and records if they fit
+  size_t words = 0;
+  { uint32_t w = (L + 1 + 31) / 32; for (int l = 0; l < 4; ++l) { words += w; w = (w + 31) / 32; } }
+  const size_t fixed = (words + 3 * (size_t)kFitChunk) * 4 + 16;
+  const size_t limit = 227 * 1024 - 64;
+  const size_t head_bytes = ((size_t)L + 1) * 4;
+  const uint32_t head_in_smem = fixed + head_bytes + 1024 * sizeof(MbRec) <= limit;
+  size_t used = fixed + (head_in_smem ? head_bytes : 0);
+  const uint32_t rec_cap = (uint32_t)std::min<size_t>(n, (limit - used) / sizeof(MbRec));
+  used += (size_t)rec_cap * sizeof(MbRec);
+  static bool attr_set = false;
+  if (!attr_set) {
+    CK(cudaFuncSetAttribute(k_bestfit, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)limit));
+    attr_set = true;
+  }
+  k_bestfit<<<1, 1024, used, st>>>(pl->d_len, n, L, d_head, d_recs, head_in_smem, rec_cap, pl->d_sample_mb,
+                                   pl->d_sample_rank, pl->d_mb_residual, pl->d_mb_tokens, pl->d_mb_lmax, pl->d_mb_count,
+                                   pl->d_scalars);
+  k_mb_finalize<<<1, 1024, 0, st>>>(cfg->coef_A, cfg->coef_B, pl->d_mb_tokens, pl->d_mb_lmax, pl->d_mb_count, pl->d_mb_cost,
+                                    pl->d_mb_sample_off, pl->d_mb_row_off, pl->d_scalars);
+  k_plan_scatter<<<gb, 256, 0, st>>>(pl->d_slots, pl->d_len, pl->d_sample_mb, pl->d_sample_rank, pl->d_mb_sample_off, n,
+                                     pl->d_mb_samples, pl->d_plan_len, pl->d_plan_sample_mb);
+  k_row_offsets<<<1, 1024, 0, st>>>(pl->d_plan_len, n, pl->d_sample_row_off);
+  k_tiles<<<gb, 256, 0, st>>>(pl->d_sample_row_off, n, pl->d_tile_first_sample);
+  k_bucket<<<gb, 256, 0, st>>>(pl->d_mb_cost, K, pl->d_scalars, pl->d_mb_bucket);
+  k_sort_deal<<<gb, 256, 0, st>>>(pl->d_mb_cost, pl->d_mb_bucket, N, pl->d_scalars, pl->d_mb_pos, pl->d_mb_rank);
+  k_rank_index<<<gb, 256, 0, st>>>(pl->d_mb_pos, pl->d_mb_rank, pl->d_scalars, d_mb_idx, pl->d_rank_cnt);
+  k_rank_scan<<<1, 1024, 0, st>>>(pl->d_rank_cnt, N, pl->d_rank_mb_off);
+  k_rank_lists<<<gb, 256, 0, st>>>(pl->d_mb_rank, d_mb_idx, pl->d_rank_mb_off, pl->d_scalars, pl->d_rank_mbs);
+  CK(cudaGetLastError());
+  p->gpu_launches += 11;
+
+  uint32_t sc[SC_COUNT];
+  CK(cudaMemcpyAsync(sc, pl->d_scalars, sizeof(sc), cudaMemcpyDeviceToHost, st));
+  CK(cudaStreamSynchronize(st));
+  pl->n_mb = sc[SC_NMB];
+  pl->max_mb_tokens = sc[SC_MAXTOK];
+  pl->total_tokens = (uint64_t)sc[SC_TOTAL_LO] | ((uint64_t)sc[SC_TOTAL_HI] << 32);
+  pl->h_mb_sample_off.resize((size_t)pl->n_mb + 1);
+  pl->h_mb_row_off.resize((size_t)pl->n_mb + 1);
+  CK(cudaMemcpy(pl->h_mb_sample_off.data(), pl->d_mb_sample_off, ((size_t)pl->n_mb + 1) * 4, cudaMemcpyDeviceToHost));
+  CK(cudaMemcpy(pl->h_mb_row_off.data(), pl->d_mb_row_off, ((size_t)pl->n_mb + 1) * 8, cudaMemcpyDeviceToHost));
+#undef CK
+  *out = pl;
+  return FT_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int32_t plan_summary(const ft_plan* pl, uint32_t* n_mb, uint64_t* total_tokens, uint32_t* max_mb_tokens) {
+  if (!pl) return FT_ERR_INVALID_ARG;
+  if (n_mb) *n_mb = pl->n_mb;
+  if (total_tokens) *total_tokens = pl->total_tokens;
+  if (max_mb_tokens) *max_mb_tokens = pl->max_mb_tokens;
+  return FT_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int32_t plan_arrays(const ft_plan* pl, uint32_t* mb_sample_off, uint32_t* mb_samples, uint32_t* mb_tokens,
+                               uint32_t* mb_lmax, uint32_t* mb_residual, uint64_t* mb_cost, uint32_t* mb_bucket,
+                               uint32_t* mb_rank, uint32_t* rank_mb_off, uint32_t* rank_mbs, uint64_t* sample_cost,
+                               uint32_t* sample_mb) {
+  if (!pl) return FT_ERR_INVALID_ARG;
+  const size_t n = pl->n, m = pl->n_mb, N = pl->cfg.n_ranks_N;
+  if (n == 0) {
+    if (mb_sample_off) mb_sample_off[0] = 0;
+    if (rank_mb_off) memset(rank_mb_off, 0, (N + 1) * 4);
+    return FT_OK;
+  }
+  FT_CUDA(cudaDeviceSynchronize());
+#define CP(dst, src, cnt, sz) \
+  if (dst) FT_CUDA(cudaMemcpy(dst, src, (size_t)(cnt) * (sz), cudaMemcpyDeviceToHost))
+  CP(mb_sample_off, pl->d_mb_sample_off, m + 1, 4); CP(mb_samples, pl->d_mb_samples, n, 4);
+  CP(mb_tokens, pl->d_mb_tokens, m, 4); CP(mb_lmax, pl->d_mb_lmax, m, 4); CP(mb_residual, pl->d_mb_residual, m, 4);
+  CP(mb_cost, pl->d_mb_cost, m, 8); CP(mb_bucket, pl->d_mb_bucket, m, 4); CP(mb_rank, pl->d_mb_rank, m, 4);
+  CP(rank_mb_off, pl->d_rank_mb_off, N + 1, 4); CP(rank_mbs, pl->d_rank_mbs, m, 4);
+  CP(sample_cost, pl->d_sample_cost, n, 8); CP(sample_mb, pl->d_sample_mb, n, 4);
+#undef CP
+  return FT_OK;
+}

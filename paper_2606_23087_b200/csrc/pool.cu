@@ -1,0 +1,924 @@
+// Pool life cycle, registration, page allocation, producer scatter and free (sm_100a).
+//
+// Kernels in this file
+//   k_page_table_init  PTEs from the vpn->frame binding (Sec. 3.2: page tables map GVA -> physical)
+//   k_register_scan    per-sample text-page counts -> exclusive scan, sample + span tables
+//   k_register_ids     token ids into text pages, placeholder-run validation
+//   k_alloc_scan       pages/list blocks/chunks per span -> exclusive scans, ring pops
+//   k_alloc_fill       span page lists (two-level) from consecutive ring entries
+//   k_scatter          the producer byte copy into pages, optional fused fp32->bf16 RNE cast
+//   k_free_scan/_fill  pages, list blocks and text pages back to the ring tails
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <unordered_set>
+
+#include "flowpool_internal.cuh"
+
+namespace ft {
+
+static char g_last_error[512] = "";
+
+int32_t cuda_fail(cudaError_t e, const char* what) {
+  snprintf(g_last_error, sizeof(g_last_error), "%s: %s", what, cudaGetErrorString(e));
+  cudaGetLastError();
+  return FT_ERR_CUDA;
+}
+
+// Counter-based hash of the seeded shuffles: the published SplitMix64 finaliser,
+// hash(seed, i) = mix(seed ^ mix(i)); Fisher-Yates runs i = n-1..1 with j = hash mod (i+1).
+static inline uint64_t mix64(uint64_t z) {
+  z += 0x9E3779B97F4A7C15ull;
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+static void seeded_shuffle(std::vector<uint32_t>& a, uint64_t seed) {
+  for (uint64_t i = a.size(); i-- > 1;) {
+    uint64_t j = mix64(seed ^ mix64(i)) % (i + 1);
+    std::swap(a[i], a[j]);
+  }
+}
+
+int32_t stage_upload(ft_pool* p, const void* src, size_t bytes, size_t total_bytes, cudaStream_t st, void** d_out) {
+  ft_staging& s = p->staging;
+  const int i = s.next;
+  s.next = (i + 1) % ft_staging::kBufs;
+  if (s.busy[i]) { FT_CUDA(cudaEventSynchronize(s.ev[i])); s.busy[i] = false; }
+  if (!s.ev[i]) FT_CUDA(cudaEventCreateWithFlags(&s.ev[i], cudaEventDisableTiming));
+  if (s.cap[i] < bytes) {
+    if (s.h[i]) FT_CUDA(cudaFreeHost(s.h[i]));
+    size_t cap = 1 << 16;
+    while (cap < bytes) cap <<= 1;
+    s.h[i] = nullptr; s.cap[i] = 0;
+    FT_CUDA(cudaHostAlloc(&s.h[i], cap, cudaHostAllocDefault));
+    s.cap[i] = cap;
+  }
+  memcpy(s.h[i], src, bytes);
+  if (p->scratch_cap < total_bytes) {
+    if (p->d_scratch) FT_CUDA(cudaFree(p->d_scratch));  // synchronises: no kernel still reads the old scratch
+    size_t cap = 1 << 20;
+    while (cap < total_bytes) cap <<= 1;
+    p->d_scratch = nullptr; p->scratch_cap = 0;
+    FT_CUDA(cudaMalloc(&p->d_scratch, cap));
+    p->scratch_cap = cap;
+  }
+  FT_CUDA(cudaMemcpyAsync(p->d_scratch, s.h[i], bytes, cudaMemcpyHostToDevice, st));
+  FT_CUDA(cudaEventRecord(s.ev[i], st));
+  s.busy[i] = true;
+  *d_out = p->d_scratch;
+  return FT_OK;
+}
+
+static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// ------------------------------------------------------------------------------------------
+// K1: page tables
+// ------------------------------------------------------------------------------------------
+__global__ void k_page_table_init(uint64_t* pte, const uint32_t* bind, uint64_t n, uint64_t base, uint64_t frame_bytes,
+                                  uint64_t flags) {
+  uint64_t v = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (v < n) pte[v] = (base + (bind ? (uint64_t)bind[v] : v) * frame_bytes) | flags;
+}
+
+__global__ void k_iota(uint32_t* a, uint64_t n) {
+  uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) a[i] = (uint32_t)i;
+}
+
+// ------------------------------------------------------------------------------------------
+// K2: registration
+// ------------------------------------------------------------------------------------------
+struct RegisterCall {
+  uint32_t n;
+  const uint32_t *slot, *seq_len, *n_spans, *span_begin;  // [n], [n], [n], [n+1]
+  const uint64_t* ids_off;                                // [n+1]
+  const uint32_t *span_pos, *span_tok;                    // concatenated
+  const int32_t* ids;                                     // device, concatenated
+  uint32_t* tp_off;                                       // [n+1] out: exclusive scan of text pages
+  uint32_t* head;                                         // [1]   out: text ring head before the pops
+  uint64_t call_seq;
+};
+
+__global__ void __launch_bounds__(1024) k_register_scan(PoolView v, RegisterCall c) {
+  uint64_t carry = 0;
+  for (uint32_t base = 0; base < c.n; base += blockDim.x) {
+    uint32_t i = base + threadIdx.x;
+    uint64_t ntp = 0;
+    if (i < c.n) {
+      ntp = (c.seq_len[i] + kTextPageIds - 1) / kTextPageIds;
+      const uint32_t slot = c.slot[i];
+      v.s_seq_len[slot] = c.seq_len[i];
+      v.s_n_spans[slot] = c.n_spans[i];
+      for (uint32_t j = 0; j < c.n_spans[i]; ++j) {
+        const uint32_t sid = slot * v.spans_per_sample + j;
+        v.sp_pos[sid] = c.span_pos[c.span_begin[i] + j];
+        v.sp_tokens[sid] = c.span_tok[c.span_begin[i] + j];
+        v.sp_npages[sid] = 0;
+      }
+    }
+    uint64_t total, ex = block_exclusive_scan(ntp, &total);
+    if (i < c.n) c.tp_off[i] = (uint32_t)(carry + ex);
+    carry += total;
+  }
+  if (threadIdx.x == 0) {
+    c.tp_off[c.n] = (uint32_t)carry;
+    RingState s = *v.tring_state;
+    c.head[0] = s.head;
+    s.head = (uint32_t)((s.head + carry) % v.tring_cap);
+    s.count -= (uint32_t)carry;
+    *v.tring_state = s;
+  }
+}
+
+// one block per (sample, text page): pops the page, stores up to 1024 ids, validates the runs
+__global__ void __launch_bounds__(256) k_register_ids(PoolView v, RegisterCall c) {
+  __shared__ uint32_t sh_i;
+  const uint32_t b = blockIdx.x;
+  if (threadIdx.x == 0) {
+    uint32_t lo = 0, hi = c.n;  // largest i with tp_off[i] <= b
+    while (hi - lo > 1) {
+      uint32_t mid = (lo + hi) >> 1;
+      if (c.tp_off[mid] <= b) lo = mid; else hi = mid;
+    }
+    sh_i = lo;
+  }
+  __syncthreads();
+  const uint32_t i = sh_i, k = b - c.tp_off[i], slot = c.slot[i];
+  const uint32_t tp = v.tring[(c.head[0] + b) % v.tring_cap];
+  if (threadIdx.x == 0) v.s_text_pages[(uint64_t)slot * v.text_pages_per_sample + k] = tp;
+  uint64_t off;
+  const uint64_t pte = translate(v, v.text_gva_base + (uint64_t)tp * FT_TEXT_PAGE_BYTES, &off);
+  int32_t* dst = reinterpret_cast<int32_t*>(pte & ~kPteFlagMask);
+  const uint32_t len = c.seq_len[i], p0 = k * kTextPageIds;
+  const uint32_t cnt = min(kTextPageIds, len - p0);
+  const uint32_t sb = c.span_begin[i], ns = c.n_spans[i];
+  bool bad = false;
+  for (uint32_t t = threadIdx.x; t < cnt; t += blockDim.x) {
+    const uint32_t p = p0 + t;
+    const int32_t id = c.ids[c.ids_off[i] + p];
+    dst[t] = id;
+    // is p inside a placeholder run?  last span with pos <= p
+    uint32_t lo = 0, hi = ns;
+    while (lo < hi) {
+      uint32_t mid = (lo + hi) >> 1;
+      if (c.span_pos[sb + mid] <= p) lo = mid + 1; else hi = mid;
+    }
+    const bool in_run = lo > 0 && p < c.span_pos[sb + lo - 1] + c.span_tok[sb + lo - 1];
+    bad |= (id == v.placeholder_id) != in_run;
+  }
+  if (bad) note_error(v, c.call_seq, FT_ERR_PLACEHOLDER_MISMATCH, slot);
+}
+
+// ------------------------------------------------------------------------------------------
+// K3: page allocation
+// ------------------------------------------------------------------------------------------
+struct WriteCall {
+  uint32_t n;
+  const uint64_t* src;       // [n] device pointers
+  const uint32_t* span_id;   // [n]
+  const uint32_t* n_tokens;  // [n]
+  uint32_t* page_off;        // [n+1] out
+  uint32_t* blk_off;         // [n+1] out
+  uint64_t* chunk_off;       // [n+1] out
+  uint32_t* heads;           // [2]   out: page ring head, block ring head before the pops
+  uint32_t chunk_shift;      // scatter work unit = 2^chunk_shift destination bytes, never straddles a page
+};
+
+__global__ void __launch_bounds__(1024) k_alloc_scan(PoolView v, WriteCall c) {
+  uint64_t cp = 0, cb = 0, cc = 0;
+  for (uint32_t base = 0; base < c.n; base += blockDim.x) {
+    uint32_t q = base + threadIdx.x;
+    uint64_t k = 0, nb = 0, nc = 0;
+    if (q < c.n) {
+      const uint64_t bytes = (uint64_t)c.n_tokens[q] * v.row_bytes;
+      k = (bytes + v.page_bytes - 1) >> v.page_shift;
+      nb = (k + kListBlock - 1) / kListBlock;
+      nc = (bytes + (1ull << c.chunk_shift) - 1) >> c.chunk_shift;
+      v.sp_npages[c.span_id[q]] = (uint32_t)k;
+    }
+    uint64_t tp, tb, tc;
+    uint64_t ep = block_exclusive_scan(k, &tp);
+    uint64_t eb = block_exclusive_scan(nb, &tb);
+    uint64_t ec = block_exclusive_scan(nc, &tc);
+    if (q < c.n) { c.page_off[q] = (uint32_t)(cp + ep); c.blk_off[q] = (uint32_t)(cb + eb); c.chunk_off[q] = cc + ec; }
+    cp += tp; cb += tb; cc += tc;
+  }
+  if (threadIdx.x == 0) {
+    c.page_off[c.n] = (uint32_t)cp; c.blk_off[c.n] = (uint32_t)cb; c.chunk_off[c.n] = cc;
+    RingState s = *v.ring_state;
+    c.heads[0] = s.head;
+    s.head = (uint32_t)((s.head + cp) % v.ring_cap); s.count -= (uint32_t)cp;
+    *v.ring_state = s;
+    s = *v.bring_state;
+    c.heads[1] = s.head;
+    s.head = (uint32_t)((s.head + cb) % v.bring_cap); s.count -= (uint32_t)cb;
+    *v.bring_state = s;
+  }
+}
+
+// one thread per allocated page: span q takes ring entries [page_off[q], page_off[q+1]) after the head
+__global__ void __launch_bounds__(256) k_alloc_fill(PoolView v, WriteCall c, uint32_t total_pages) {
+  const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= total_pages) return;
+  uint32_t lo = 0, hi = c.n;  // largest q with page_off[q] <= t
+  while (hi - lo > 1) {
+    uint32_t mid = (lo + hi) >> 1;
+    if (c.page_off[mid] <= t) lo = mid; else hi = mid;
+  }
+  const uint32_t q = lo, o = t - c.page_off[q], sid = c.span_id[q];
+  const uint32_t g = v.ring[(c.heads[0] + t) % v.ring_cap];
+  const uint32_t blk = v.bring[(c.heads[1] + c.blk_off[q] + o / kListBlock) % v.bring_cap];
+  if (o % kListBlock == 0) v.sp_blocks[(uint64_t)sid * v.blocks_per_span + o / kListBlock] = blk;
+  v.list_blocks[(uint64_t)blk * kListBlock + o % kListBlock] = page_gva(v, g);
+}
+
+// ------------------------------------------------------------------------------------------
+// K4: producer scatter.  Work unit = one chunk of destination bytes inside one page; each CTA owns a
+// contiguous chunk range (one search at its start, then a walk), resolves the destination frame through
+// the span's page list and the page table once per page, and moves 16-byte vectors.
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t rne_bf16(uint32_t u) {
+  // IEEE round-to-nearest-even on the bit pattern; NaN -> sign | 0x7FC0; denormals kept
+  if ((u & 0x7FFFFFFFu) > 0x7F800000u) return ((u >> 16) & 0x8000u) | 0x7FC0u;
+  return (u + 0x7FFFu + ((u >> 16) & 1u)) >> 16;
+}
+__device__ __forceinline__ uint32_t pack2(uint32_t a, uint32_t b) { return rne_bf16(a) | (rne_bf16(b) << 16); }
+
+enum { kTierAll = 0, kTierDeviceOnly = 1, kTierHostOnly = 2 };
+
+template <int MODE, bool F32>
+__global__ void __launch_bounds__(256) k_scatter(PoolView v, WriteCall c, uint64_t total_chunks, uint64_t per_cta) {
+  const uint64_t c0 = (uint64_t)blockIdx.x * per_cta;
+  const uint64_t c1 = min(total_chunks, c0 + per_cta);
+  if (c0 >= c1) return;
+  uint32_t lo = 0, hi = c.n;  // largest q with chunk_off[q] <= c0
+  while (hi - lo > 1) {
+    uint32_t mid = (lo + hi) >> 1;
+    if (c.chunk_off[mid] <= c0) lo = mid; else hi = mid;
+  }
+  uint32_t q = lo;
+  uint64_t q_end = c.chunk_off[q + 1], q_begin = c.chunk_off[q];
+  uint64_t bytes_q = (uint64_t)c.n_tokens[q] * v.row_bytes;
+  const uint8_t* src_q = reinterpret_cast<const uint8_t*>(c.src[q]);
+  uint32_t sid = c.span_id[q];
+  uint32_t cached_o = kNone;
+  uint64_t pte = 0;
+  const uint64_t CH = 1ull << c.chunk_shift;
+  for (uint64_t ch = c0; ch < c1; ++ch) {
+    while (ch >= q_end) {
+      ++q;
+      q_begin = q_end; q_end = c.chunk_off[q + 1];
+      bytes_q = (uint64_t)c.n_tokens[q] * v.row_bytes;
+      src_q = reinterpret_cast<const uint8_t*>(c.src[q]);
+      sid = c.span_id[q];
+      cached_o = kNone;
+    }
+    const uint64_t b0 = (ch - q_begin) << c.chunk_shift;  // byte offset inside the span image
+    const uint32_t o = (uint32_t)(b0 >> v.page_shift);
+    if (o != cached_o) {
+      uint64_t off;
+      pte = translate(v, span_page_gva(v, sid, o), &off);
+      cached_o = o;
+    }
+    const bool host = (pte & kPteHost) != 0;
+    if ((MODE == kTierDeviceOnly && host) || (MODE == kTierHostOnly && !host)) continue;
+    uint8_t* dst = reinterpret_cast<uint8_t*>(pte & ~kPteFlagMask) + (b0 & (v.page_bytes - 1));
+    const uint32_t len = (uint32_t)min(CH, bytes_q - b0);
+    if (!F32) {
+      const uint4* s = reinterpret_cast<const uint4*>(src_q + b0);
+      uint4* d = reinterpret_cast<uint4*>(dst);
+      const uint32_t nv = len >> 4;
+      uint32_t x = threadIdx.x;
+      for (; x + 3 * 256 < nv; x += 4 * 256) {
+        uint4 a0 = __ldcs(s + x), a1 = __ldcs(s + x + 256), a2 = __ldcs(s + x + 512), a3 = __ldcs(s + x + 768);
+        __stcs(d + x, a0); __stcs(d + x + 256, a1); __stcs(d + x + 512, a2); __stcs(d + x + 768, a3);
+      }
+      for (; x < nv; x += 256) __stcs(d + x, __ldcs(s + x));
+    } else {
+      const uint4* s = reinterpret_cast<const uint4*>(src_q + 2 * b0);  // 2 source vectors per destination vector
+      uint4* d = reinterpret_cast<uint4*>(dst);
+      const uint32_t nv = len >> 4;
+      uint32_t x = threadIdx.x;
+      for (; x + 256 < nv; x += 2 * 256) {
+        uint4 a0 = __ldcs(s + 2 * x), a1 = __ldcs(s + 2 * x + 1);
+        uint4 b0v = __ldcs(s + 2 * (x + 256)), b1v = __ldcs(s + 2 * (x + 256) + 1);
+        __stcs(d + x, make_uint4(pack2(a0.x, a0.y), pack2(a0.z, a0.w), pack2(a1.x, a1.y), pack2(a1.z, a1.w)));
+        __stcs(d + x + 256, make_uint4(pack2(b0v.x, b0v.y), pack2(b0v.z, b0v.w), pack2(b1v.x, b1v.y), pack2(b1v.z, b1v.w)));
+      }
+      for (; x < nv; x += 256) {
+        uint4 a0 = __ldcs(s + 2 * x), a1 = __ldcs(s + 2 * x + 1);
+        __stcs(d + x, make_uint4(pack2(a0.x, a0.y), pack2(a0.z, a0.w), pack2(a1.x, a1.y), pack2(a1.z, a1.w)));
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// K9: free
+// ------------------------------------------------------------------------------------------
+struct FreeCall {
+  uint32_t n_spans, n_samples;
+  const uint32_t* span_id;  // [n_spans] written spans, canonical order
+  const uint32_t* slot;     // [n_samples]
+  uint32_t* page_off;       // [n_spans+1]
+  uint32_t* blk_off;        // [n_spans+1]
+  uint32_t* tp_off;         // [n_samples+1]
+  uint32_t* tails;          // [3] page ring, block ring, text ring tails before the pushes
+};
+
+__global__ void __launch_bounds__(1024) k_free_scan(PoolView v, FreeCall c) {
+  uint64_t cp = 0, cb = 0, ct = 0;
+  const uint32_t m = max(c.n_spans, c.n_samples);
+  for (uint32_t base = 0; base < m; base += blockDim.x) {
+    uint32_t i = base + threadIdx.x;
+    uint64_t k = 0, nb = 0, nt = 0;
+    if (i < c.n_spans) { k = v.sp_npages[c.span_id[i]]; nb = (k + kListBlock - 1) / kListBlock; }
+    if (i < c.n_samples) nt = (v.s_seq_len[c.slot[i]] + kTextPageIds - 1) / kTextPageIds;
+    uint64_t tp, tb, tt;
+    uint64_t ep = block_exclusive_scan(k, &tp);
+    uint64_t eb = block_exclusive_scan(nb, &tb);
+    uint64_t et = block_exclusive_scan(nt, &tt);
+    if (i < c.n_spans) { c.page_off[i] = (uint32_t)(cp + ep); c.blk_off[i] = (uint32_t)(cb + eb); }
+    if (i < c.n_samples) c.tp_off[i] = (uint32_t)(ct + et);
+    cp += tp; cb += tb; ct += tt;
+  }
+  if (threadIdx.x == 0) {
+    c.page_off[c.n_spans] = (uint32_t)cp; c.blk_off[c.n_spans] = (uint32_t)cb; c.tp_off[c.n_samples] = (uint32_t)ct;
+    RingState s = *v.ring_state;
+    c.tails[0] = (uint32_t)(((uint64_t)s.head + s.count) % v.ring_cap); s.count += (uint32_t)cp; *v.ring_state = s;
+    s = *v.bring_state;
+    c.tails[1] = (uint32_t)(((uint64_t)s.head + s.count) % v.bring_cap); s.count += (uint32_t)cb; *v.bring_state = s;
+    s = *v.tring_state;
+    c.tails[2] = (uint32_t)(((uint64_t)s.head + s.count) % v.tring_cap); s.count += (uint32_t)ct; *v.tring_state = s;
+  }
+}
+
+// threads [0, total_pages): one page each, pushed at the tail in canonical order;
+// threads [total_pages, total_pages + total_text): one text page each
+__global__ void __launch_bounds__(256) k_free_fill(PoolView v, FreeCall c, uint32_t total_pages, uint32_t total_text) {
+  const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t < total_pages) {
+    uint32_t lo = 0, hi = c.n_spans;
+    while (hi - lo > 1) {
+      uint32_t mid = (lo + hi) >> 1;
+      if (c.page_off[mid] <= t) lo = mid; else hi = mid;
+    }
+    const uint32_t q = lo, o = t - c.page_off[q], sid = c.span_id[q];
+    const uint32_t blk = v.sp_blocks[(uint64_t)sid * v.blocks_per_span + o / kListBlock];
+    const uint64_t gva = v.list_blocks[(uint64_t)blk * kListBlock + o % kListBlock];
+    v.ring[(c.tails[0] + t) % v.ring_cap] = global_page_of(v, gva);
+    if (o % kListBlock == 0) v.bring[(c.tails[1] + c.blk_off[q] + o / kListBlock) % v.bring_cap] = blk;
+    if (o == 0) v.sp_npages[sid] = 0;
+  } else if (t < total_pages + total_text) {
+    const uint32_t u = t - total_pages;
+    uint32_t lo = 0, hi = c.n_samples;
+    while (hi - lo > 1) {
+      uint32_t mid = (lo + hi) >> 1;
+      if (c.tp_off[mid] <= u) lo = mid; else hi = mid;
+    }
+    const uint32_t i = lo, k = u - c.tp_off[i], slot = c.slot[i];
+    v.tring[(c.tails[2] + u) % v.tring_cap] = v.s_text_pages[(uint64_t)slot * v.text_pages_per_sample + k];
+  }
+}
+
+__global__ void k_free_clear(PoolView v, FreeCall c) {
+  const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < c.n_samples) { v.s_seq_len[c.slot[i]] = 0; v.s_n_spans[c.slot[i]] = 0; }
+}
+
+__global__ void k_debug_translate(PoolView v, const uint64_t* gva, uint32_t n, uint32_t* kind, uint64_t* frame,
+                                  uint64_t* offset, int32_t* status, uint64_t hbm_base, uint64_t host_base,
+                                  uint64_t text_base) {
+  const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  uint64_t off = 0;
+  const uint64_t pte = translate(v, gva[i], &off);
+  if (!(pte & kPteValid)) { status[i] = FT_ERR_BAD_GVA; kind[i] = 0; frame[i] = 0; offset[i] = 0; return; }
+  const uint64_t addr = pte & ~kPteFlagMask;
+  status[i] = FT_OK;
+  offset[i] = off;
+  if (pte & kPteText) { kind[i] = 2; frame[i] = (addr - text_base) / FT_TEXT_PAGE_BYTES; }
+  else if (pte & kPteHost) { kind[i] = 1; frame[i] = (addr - host_base) >> v.page_shift; }
+  else { kind[i] = 0; frame[i] = (addr - hbm_base) >> v.page_shift; }
+}
+
+static inline uint64_t pages_for_tokens(const ft_pool* p, uint64_t n_tokens) {
+  const uint64_t bytes = n_tokens * 2ull * p->cfg.hidden;
+  return (bytes + p->cfg.page_bytes - 1) / p->cfg.page_bytes;
+}
+
+}  // namespace ft
+
+using namespace ft;
+
+// ==========================================================================================
+// C ABI
+// ==========================================================================================
+extern "C" __attribute__((visibility("default"))) const char* flowpool_last_cuda_error(void) { return ft::g_last_error; }
+
+extern "C" __attribute__((visibility("default"))) int32_t pool_destroy(ft_pool* p) {
+  if (!p) return FT_ERR_INVALID_ARG;
+  cudaSetDevice(p->device);
+  cudaDeviceSynchronize();
+  for (int i = 0; i < ft_staging::kBufs; ++i) {
+    if (p->staging.h[i]) cudaFreeHost(p->staging.h[i]);
+    if (p->staging.ev[i]) cudaEventDestroy(p->staging.ev[i]);
+  }
+  if (p->d_scratch) cudaFree(p->d_scratch);
+  if (p->d_meta) cudaFree(p->d_meta);
+  if (p->d_text) cudaFree(p->d_text);
+  if (p->own_hbm && p->hbm_base) cudaFree(p->hbm_base);
+  if (p->own_host && p->host_base) cudaFreeHost(p->host_base);
+  if (p->side_stream) cudaStreamDestroy(p->side_stream);
+  if (p->fork_ev) cudaEventDestroy(p->fork_ev);
+  if (p->join_ev) cudaEventDestroy(p->join_ev);
+  delete p;
+  cudaGetLastError();
+  return FT_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int32_t pool_create(const ft_pool_config* cfg_in, void* hbm_base, void* host_base, ft_pool** out) {
+  if (!cfg_in || !out) return FT_ERR_INVALID_ARG;
+  ft_pool_config c = *cfg_in;
+  if (c.gva_hbm_start == 0) c.gva_hbm_start = 1ull << 44;
+  if (c.gva_host_start == 0) c.gva_host_start = 1ull << 45;
+  if (c.max_size == 0) c.max_size = 1ull << 40;
+  if (c.world_size == 0) c.world_size = 1;
+  const uint64_t PS = c.page_bytes;
+  if (PS < 4096 || PS > (2u << 20) || (PS & (PS - 1))) return FT_ERR_INVALID_ARG;
+  if (c.hidden == 0 || c.hidden % 8) return FT_ERR_INVALID_ARG;
+  if (c.hbm_pages + c.host_pages == 0) return FT_ERR_INVALID_ARG;
+  if (c.hbm_pages + c.host_pages > 0xFFFFFFFFull) return FT_ERR_INVALID_ARG;
+  if (c.rank >= c.world_size) return FT_ERR_INVALID_ARG;
+  if (c.max_samples == 0 || c.max_seq_len == 0) return FT_ERR_INVALID_ARG;
+  if (c.max_spans_per_sample == 0) c.max_spans_per_sample = 1;
+  if (c.max_pages_per_span == 0) c.max_pages_per_span = 1;
+  const uint64_t n_text = (c.max_text_tokens + kTextPageIds - 1) / kTextPageIds;
+  if (c.hbm_pages * PS + n_text * FT_TEXT_PAGE_BYTES > c.max_size) return FT_ERR_INVALID_ARG;
+  if (c.host_pages * PS > c.max_size) return FT_ERR_INVALID_ARG;
+  const uint64_t region = (uint64_t)c.world_size * c.max_size;
+  if (c.gva_hbm_start + region < c.gva_hbm_start || c.gva_host_start + region < c.gva_host_start) return FT_ERR_INVALID_ARG;
+  if (c.gva_hbm_start < c.gva_host_start + region && c.gva_host_start < c.gva_hbm_start + region) return FT_ERR_INVALID_ARG;
+  if (hbm_base && (reinterpret_cast<uintptr_t>(hbm_base) & 255)) return FT_ERR_INVALID_ARG;
+  if (host_base && (reinterpret_cast<uintptr_t>(host_base) & 255)) return FT_ERR_INVALID_ARG;
+
+  ft_pool* p = new ft_pool();
+  p->cfg = c;
+  int32_t rc = FT_OK;
+#define CK(call)                                                                          \
+  do {                                                                                    \
+    cudaError_t e__ = (call);                                                             \
+    if (e__ != cudaSuccess) { rc = ft::cuda_fail(e__, #call); pool_destroy(p); return rc; } \
+  } while (0)
+  CK(cudaGetDevice(&p->device));
+  CK(cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, p->device));
+  CK(cudaStreamCreateWithFlags(&p->side_stream, cudaStreamNonBlocking));
+  CK(cudaEventCreateWithFlags(&p->fork_ev, cudaEventDisableTiming));
+  CK(cudaEventCreateWithFlags(&p->join_ev, cudaEventDisableTiming));
+
+  const uint64_t P = c.hbm_pages + c.host_pages;
+  const uint32_t S = c.max_spans_per_sample;
+  const uint32_t TPS = (c.max_seq_len + kTextPageIds - 1) / kTextPageIds;
+  const uint32_t MB = (c.max_pages_per_span + kListBlock - 1) / kListBlock;
+  const uint64_t span_ids = (uint64_t)c.max_samples * S;
+  const uint64_t NB = (P + kListBlock - 1) / kListBlock + std::min<uint64_t>(span_ids, P) + 1;
+  if (NB > 0xFFFFFFFFull || span_ids > 0xFFFFFFFFull) { pool_destroy(p); return FT_ERR_INVALID_ARG; }
+
+  // backing memory
+  if (c.hbm_pages) {
+    if (hbm_base) p->hbm_base = hbm_base;
+    else { CK(cudaMalloc(&p->hbm_base, c.hbm_pages * PS)); p->own_hbm = true; }
+  }
+  if (c.host_pages) {
+    if (host_base) p->host_base = host_base;
+    else { CK(cudaHostAlloc(&p->host_base, c.host_pages * PS, cudaHostAllocMapped | cudaHostAllocPortable)); p->own_host = true; }
+    cudaError_t e = cudaHostGetDevicePointer(&p->host_dev, p->host_base, 0);
+    if (e != cudaSuccess) { ft::cuda_fail(e, "cudaHostGetDevicePointer(host_base)"); pool_destroy(p); return host_base ? FT_ERR_INVALID_ARG : FT_ERR_CUDA; }
+  }
+  CK(cudaMalloc(&p->d_text, std::max<uint64_t>(n_text, 1) * FT_TEXT_PAGE_BYTES));
+
+  // metadata block
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  const size_t o_pte_hbm = take(c.hbm_pages * 8), o_pte_host = take(c.host_pages * 8), o_pte_text = take(n_text * 8);
+  const size_t o_ring = take(P * 4), o_tring = take(n_text * 4), o_bring = take(NB * 4);
+  const size_t o_states = take(3 * sizeof(RingState)), o_status = take(8);
+  const size_t o_seq = take((size_t)c.max_samples * 4), o_nsp = take((size_t)c.max_samples * 4);
+  const size_t o_stp = take((size_t)c.max_samples * TPS * 4);
+  const size_t o_pos = take(span_ids * 4), o_tok = take(span_ids * 4), o_npg = take(span_ids * 4);
+  const size_t o_blk = take(span_ids * MB * 4), o_lst = take(NB * kListBlock * 8);
+  CK(cudaMalloc(&p->d_meta, off));
+  CK(cudaMemset(p->d_meta, 0, off));
+  uint8_t* m = static_cast<uint8_t*>(p->d_meta);
+
+  PoolView& v = p->view;
+  v.region_start[0] = c.gva_hbm_start; v.region_start[1] = c.gva_host_start;
+  v.region_bytes = region; v.max_size = c.max_size;
+  v.seg_base[0] = c.gva_hbm_start + (uint64_t)c.rank * c.max_size;
+  v.seg_base[1] = c.gva_host_start + (uint64_t)c.rank * c.max_size;
+  v.text_gva_base = v.seg_base[0] + c.hbm_pages * PS;
+  v.rank = c.rank;
+  v.page_shift = 0; while ((1ull << v.page_shift) < PS) ++v.page_shift;
+  v.page_bytes = PS; v.hbm_pages = c.hbm_pages; v.host_pages = c.host_pages; v.text_pages = n_text;
+  v.hidden = c.hidden; v.row_bytes = 2 * c.hidden; v.placeholder_id = c.placeholder_id;
+  v.max_samples = c.max_samples; v.spans_per_sample = S; v.text_pages_per_sample = TPS; v.blocks_per_span = MB;
+  v.pte_hbm = reinterpret_cast<uint64_t*>(m + o_pte_hbm);
+  v.pte_host = reinterpret_cast<uint64_t*>(m + o_pte_host);
+  v.pte_text = reinterpret_cast<uint64_t*>(m + o_pte_text);
+  v.ring = reinterpret_cast<uint32_t*>(m + o_ring); v.ring_cap = (uint32_t)P;
+  v.tring = reinterpret_cast<uint32_t*>(m + o_tring); v.tring_cap = (uint32_t)std::max<uint64_t>(n_text, 1);
+  v.bring = reinterpret_cast<uint32_t*>(m + o_bring); v.bring_cap = (uint32_t)NB;
+  RingState* st = reinterpret_cast<RingState*>(m + o_states);
+  v.ring_state = st; v.tring_state = st + 1; v.bring_state = st + 2;
+  v.status = reinterpret_cast<unsigned long long*>(m + o_status);
+  v.s_seq_len = reinterpret_cast<uint32_t*>(m + o_seq); v.s_n_spans = reinterpret_cast<uint32_t*>(m + o_nsp);
+  v.s_text_pages = reinterpret_cast<uint32_t*>(m + o_stp);
+  v.sp_pos = reinterpret_cast<uint32_t*>(m + o_pos); v.sp_tokens = reinterpret_cast<uint32_t*>(m + o_tok);
+  v.sp_npages = reinterpret_cast<uint32_t*>(m + o_npg); v.sp_blocks = reinterpret_cast<uint32_t*>(m + o_blk);
+  v.list_blocks = reinterpret_cast<uint64_t*>(m + o_lst);
+
+  // binding (identity or seeded permutation per tier) and the initial ring order are made on the host, once
+  std::vector<uint32_t> bind_h(c.hbm_pages), bind_d(c.host_pages), ring(P);
+  for (uint64_t k = 0; k < c.hbm_pages; ++k) bind_h[k] = (uint32_t)k;
+  for (uint64_t k = 0; k < c.host_pages; ++k) bind_d[k] = (uint32_t)k;
+  for (uint64_t k = 0; k < P; ++k) ring[k] = (uint32_t)k;
+  if (c.bind_order == FT_BIND_PERMUTED) { seeded_shuffle(bind_h, c.bind_seed); seeded_shuffle(bind_d, c.bind_seed + 1); }
+  if (c.ring_order == FT_RING_SHUFFLED) seeded_shuffle(ring, c.ring_seed);
+  uint32_t* d_tmp = nullptr;
+  CK(cudaMalloc(&d_tmp, std::max<uint64_t>(P, 1) * 4));
+  auto blocks = [](uint64_t n) { return (unsigned)((n + 255) / 256); };
+  if (c.hbm_pages) {
+    CK(cudaMemcpy(d_tmp, bind_h.data(), c.hbm_pages * 4, cudaMemcpyHostToDevice));
+    k_page_table_init<<<blocks(c.hbm_pages), 256>>>(const_cast<uint64_t*>(v.pte_hbm), d_tmp, c.hbm_pages,
+                                                   reinterpret_cast<uint64_t>(p->hbm_base), PS, kPteValid);
+    CK(cudaDeviceSynchronize());
+  }
+  if (c.host_pages) {
+    CK(cudaMemcpy(d_tmp, bind_d.data(), c.host_pages * 4, cudaMemcpyHostToDevice));
+    k_page_table_init<<<blocks(c.host_pages), 256>>>(const_cast<uint64_t*>(v.pte_host), d_tmp, c.host_pages,
+                                                    reinterpret_cast<uint64_t>(p->host_dev), PS, kPteValid | kPteHost);
+    CK(cudaDeviceSynchronize());
+  }
+  if (n_text) {
+    k_page_table_init<<<blocks(n_text), 256>>>(const_cast<uint64_t*>(v.pte_text), nullptr, n_text,
+                                              reinterpret_cast<uint64_t>(p->d_text), FT_TEXT_PAGE_BYTES, kPteValid | kPteText);
+    k_iota<<<blocks(n_text), 256>>>(v.tring, n_text);
+  }
+  k_iota<<<blocks(NB), 256>>>(v.bring, NB);
+  CK(cudaMemcpy(v.ring, ring.data(), P * 4, cudaMemcpyHostToDevice));
+  RingState init[3] = {{0, (uint32_t)P}, {0, (uint32_t)n_text}, {0, (uint32_t)NB}};
+  CK(cudaMemcpy(st, init, sizeof(init), cudaMemcpyHostToDevice));
+  CK(cudaMemset(v.status, 0xFF, 8));
+  CK(cudaDeviceSynchronize());
+  CK(cudaFree(d_tmp));
+  p->gpu_launches += 5;
+#undef CK
+  p->slots.resize(c.max_samples);
+  p->spans.resize(span_ids);
+  p->free_pages = P; p->free_text_pages = n_text; p->free_blocks = NB;
+  *out = p;
+  return FT_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int32_t pool_register_samples(ft_pool* p, uint32_t n, const uint32_t* slot, const uint32_t* seq_len,
+                                         const uint32_t* n_spans, const uint32_t* span_pos,
+                                         const uint32_t* span_tokens, const int32_t* input_ids, void* stream) {
+  if (!p) return FT_ERR_INVALID_ARG;
+  p->call_seq++;
+  if (n == 0) return FT_OK;
+  if (!slot || !seq_len || !n_spans || !input_ids) return FT_ERR_INVALID_ARG;
+  const ft_pool_config& c = p->cfg;
+  uint64_t text_need = 0, sp = 0;
+  std::vector<uint8_t> seen(c.max_samples, 0);
+  for (uint32_t i = 0; i < n; ++i) {
+    if (slot[i] >= c.max_samples) return FT_ERR_INVALID_ARG;
+    if (p->slots[slot[i]].state != FT_SLOT_FREE || seen[slot[i]]) return FT_ERR_SLOT_IN_USE;
+    seen[slot[i]] = 1;
+    if (seq_len[i] == 0) return FT_ERR_INVALID_ARG;
+    if (seq_len[i] > c.max_seq_len) return FT_ERR_CAPACITY;
+    if (n_spans[i] > c.max_spans_per_sample) return FT_ERR_CAPACITY;
+    if (n_spans[i] && (!span_pos || !span_tokens)) return FT_ERR_INVALID_ARG;
+    uint64_t prev_end = 0;
+    for (uint32_t j = 0; j < n_spans[i]; ++j, ++sp) {
+      if (span_tokens[sp] == 0) return FT_ERR_INVALID_ARG;
+      if ((uint64_t)span_pos[sp] + span_tokens[sp] > seq_len[i]) return FT_ERR_INVALID_ARG;
+      if (span_pos[sp] < prev_end) return FT_ERR_INVALID_ARG;
+      prev_end = (uint64_t)span_pos[sp] + span_tokens[sp];
+      if (pages_for_tokens(p, span_tokens[sp]) > c.max_pages_per_span) return FT_ERR_CAPACITY;
+    }
+    text_need += (seq_len[i] + kTextPageIds - 1) / kTextPageIds;
+  }
+  if (text_need > p->free_text_pages) return FT_ERR_CAPACITY;
+  const uint64_t total_spans = sp;
+
+  // descriptor blob: [ids_off u64 (n+1)] [slot][seq_len][n_spans][span_begin (n+1)][span_pos][span_tok]
+  const size_t o_idsoff = 0, o_slot = align_up((size_t)(n + 1) * 8, 16);
+  const size_t o_len = o_slot + (size_t)n * 4, o_nsp = o_len + (size_t)n * 4, o_sb = o_nsp + (size_t)n * 4;
+  const size_t o_pos = o_sb + (size_t)(n + 1) * 4, o_tok = o_pos + total_spans * 4;
+  const size_t blob_bytes = align_up(o_tok + total_spans * 4, 256);
+  const size_t o_tpoff = blob_bytes, o_head = align_up(o_tpoff + (size_t)(n + 1) * 4, 16);
+  const size_t total_bytes = o_head + 16;
+  std::vector<uint8_t> blob(blob_bytes, 0);
+  uint64_t* ids_off = reinterpret_cast<uint64_t*>(blob.data() + o_idsoff);
+  uint32_t* sb = reinterpret_cast<uint32_t*>(blob.data() + o_sb);
+  ids_off[0] = 0; sb[0] = 0;
+  for (uint32_t i = 0; i < n; ++i) { ids_off[i + 1] = ids_off[i] + seq_len[i]; sb[i + 1] = sb[i] + n_spans[i]; }
+  memcpy(blob.data() + o_slot, slot, (size_t)n * 4);
+  memcpy(blob.data() + o_len, seq_len, (size_t)n * 4);
+  memcpy(blob.data() + o_nsp, n_spans, (size_t)n * 4);
+  if (total_spans) {
+    memcpy(blob.data() + o_pos, span_pos, total_spans * 4);
+    memcpy(blob.data() + o_tok, span_tokens, total_spans * 4);
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  void* d = nullptr;
+  int32_t rc = stage_upload(p, blob.data(), blob_bytes, total_bytes, st, &d);
+  if (rc != FT_OK) return rc;
+  uint8_t* db = static_cast<uint8_t*>(d);
+  RegisterCall rcall;
+  rcall.n = n;
+  rcall.ids_off = reinterpret_cast<uint64_t*>(db + o_idsoff);
+  rcall.slot = reinterpret_cast<uint32_t*>(db + o_slot);
+  rcall.seq_len = reinterpret_cast<uint32_t*>(db + o_len);
+  rcall.n_spans = reinterpret_cast<uint32_t*>(db + o_nsp);
+  rcall.span_begin = reinterpret_cast<uint32_t*>(db + o_sb);
+  rcall.span_pos = reinterpret_cast<uint32_t*>(db + o_pos);
+  rcall.span_tok = reinterpret_cast<uint32_t*>(db + o_tok);
+  rcall.ids = input_ids;
+  rcall.tp_off = reinterpret_cast<uint32_t*>(db + o_tpoff);
+  rcall.head = reinterpret_cast<uint32_t*>(db + o_head);
+  rcall.call_seq = p->call_seq;
+  k_register_scan<<<1, 1024, 0, st>>>(p->view, rcall);
+  k_register_ids<<<(unsigned)text_need, 256, 0, st>>>(p->view, rcall);
+  FT_CUDA(cudaGetLastError());
+  p->gpu_launches += 2;
+
+  // host mirror
+  sp = 0;
+  for (uint32_t i = 0; i < n; ++i) {
+    ft_slot_mirror& s = p->slots[slot[i]];
+    s.state = n_spans[i] == 0 ? FT_SLOT_READY : FT_SLOT_REGISTERED;
+    s.seq_len = seq_len[i]; s.n_spans = n_spans[i]; s.spans_written = 0;
+    s.n_text_pages = (seq_len[i] + kTextPageIds - 1) / kTextPageIds;
+    for (uint32_t j = 0; j < n_spans[i]; ++j, ++sp) {
+      ft_span_mirror& m = p->spans[(uint64_t)slot[i] * c.max_spans_per_sample + j];
+      m.pos = span_pos[sp]; m.tokens = span_tokens[sp]; m.npages = 0; m.written = false;
+    }
+    p->live_samples++; p->live_spans += n_spans[i];
+  }
+  p->free_text_pages -= text_need;
+  return FT_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings(ft_pool* p, uint32_t n, const uint32_t* slot, const uint32_t* span_idx,
+                                         const uint32_t* n_tokens, const void* const* src, uint32_t src_dtype,
+                                         void* stream) {
+  if (!p) return FT_ERR_INVALID_ARG;
+  p->call_seq++;
+  if (src_dtype != FT_BF16 && src_dtype != FT_F32) return FT_ERR_INVALID_ARG;
+  if (n == 0) return FT_OK;
+  if (!slot || !span_idx || !n_tokens || !src) return FT_ERR_INVALID_ARG;
+  const ft_pool_config& c = p->cfg;
+  const uint32_t S = c.max_spans_per_sample;
+  uint64_t need = 0, need_blocks = 0, total_chunks = 0, bytes_total = 0;
+  const uint32_t chunk_shift = std::min<uint32_t>(p->view.page_shift, 14);
+  std::vector<uint32_t> span_id(n);
+  {
+    std::unordered_set<uint32_t> named;
+    named.reserve(n * 2);
+    for (uint32_t q = 0; q < n; ++q) {
+      if (slot[q] >= c.max_samples) return FT_ERR_INVALID_ARG;
+      const ft_slot_mirror& s = p->slots[slot[q]];
+      if (s.state == FT_SLOT_FREE) return FT_ERR_UNKNOWN_SAMPLE;
+      if (span_idx[q] >= s.n_spans) return FT_ERR_INVALID_ARG;
+      const ft_span_mirror& m = p->spans[(uint64_t)slot[q] * S + span_idx[q]];
+      if (n_tokens[q] != m.tokens) return FT_ERR_INVALID_ARG;
+      if (!src[q] || (reinterpret_cast<uintptr_t>(src[q]) & 15)) return FT_ERR_INVALID_ARG;
+      span_id[q] = slot[q] * S + span_idx[q];
+      if (m.written || !named.insert(span_id[q]).second) return FT_ERR_ALREADY_WRITTEN;
+      const uint64_t k = pages_for_tokens(p, n_tokens[q]);
+      need += k; need_blocks += (k + kListBlock - 1) / kListBlock;
+      const uint64_t bytes = (uint64_t)n_tokens[q] * p->view.row_bytes;
+      total_chunks += (bytes + (1ull << chunk_shift) - 1) >> chunk_shift;
+      bytes_total += bytes;
+    }
+  }
+  if (need > p->free_pages) return FT_ERR_POOL_EXHAUSTED;
+  if (need_blocks > p->free_blocks) return FT_ERR_CAPACITY;
+  if (need > 0xFFFFFFFFull) return FT_ERR_INVALID_ARG;
+
+  // blob: [src u64 n][span_id n][n_tokens n] ; outputs: page_off, blk_off (n+1), chunk_off u64 (n+1), heads
+  const size_t o_src = 0, o_sid = (size_t)n * 8, o_ntk = o_sid + (size_t)n * 4;
+  const size_t blob_bytes = align_up(o_ntk + (size_t)n * 4, 256);
+  const size_t o_choff = blob_bytes, o_poff = align_up(o_choff + (size_t)(n + 1) * 8, 16);
+  const size_t o_boff = o_poff + (size_t)(n + 1) * 4, o_heads = align_up(o_boff + (size_t)(n + 1) * 4, 16);
+  const size_t total_bytes = o_heads + 16;
+  std::vector<uint8_t> blob(blob_bytes, 0);
+  for (uint32_t q = 0; q < n; ++q) reinterpret_cast<uint64_t*>(blob.data())[q] = reinterpret_cast<uint64_t>(src[q]);
+  memcpy(blob.data() + o_sid, span_id.data(), (size_t)n * 4);
+  memcpy(blob.data() + o_ntk, n_tokens, (size_t)n * 4);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  void* d = nullptr;
+  int32_t rc = stage_upload(p, blob.data(), blob_bytes, total_bytes, st, &d);
+  if (rc != FT_OK) return rc;
+  uint8_t* db = static_cast<uint8_t*>(d);
+  WriteCall w;
+  w.n = n;
+  w.src = reinterpret_cast<uint64_t*>(db + o_src);
+  w.span_id = reinterpret_cast<uint32_t*>(db + o_sid);
+  w.n_tokens = reinterpret_cast<uint32_t*>(db + o_ntk);
+  w.chunk_off = reinterpret_cast<uint64_t*>(db + o_choff);
+  w.page_off = reinterpret_cast<uint32_t*>(db + o_poff);
+  w.blk_off = reinterpret_cast<uint32_t*>(db + o_boff);
+  w.heads = reinterpret_cast<uint32_t*>(db + o_heads);
+  w.chunk_shift = chunk_shift;
+  k_alloc_scan<<<1, 1024, 0, st>>>(p->view, w);
+  k_alloc_fill<<<(unsigned)((need + 255) / 256), 256, 0, st>>>(p->view, w, (uint32_t)need);
+  p->gpu_launches += 2;
+
+  // the byte copy: HBM-bound chunks on the caller's stream, host-bound chunks beside them
+  const bool f32 = src_dtype == FT_F32;
+  auto launch = [&](int mode, cudaStream_t s, uint32_t ctas_per_sm) {
+    uint64_t grid = std::min<uint64_t>(total_chunks, (uint64_t)p->sm_count * ctas_per_sm);
+    uint64_t per = (total_chunks + grid - 1) / grid;
+    grid = (total_chunks + per - 1) / per;
+    if (mode == kTierAll) { if (f32) k_scatter<kTierAll, true><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); else k_scatter<kTierAll, false><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); }
+    else if (mode == kTierDeviceOnly) { if (f32) k_scatter<kTierDeviceOnly, true><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); else k_scatter<kTierDeviceOnly, false><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); }
+    else { if (f32) k_scatter<kTierHostOnly, true><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); else k_scatter<kTierHostOnly, false><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); }
+    p->gpu_launches++;
+  };
+  if (c.host_pages == 0) {
+    launch(kTierAll, st, 8);
+  } else if (c.hbm_pages == 0) {
+    launch(kTierAll, st, 2);
+  } else {
+    FT_CUDA(cudaEventRecord(p->fork_ev, st));
+    FT_CUDA(cudaStreamWaitEvent(p->side_stream, p->fork_ev, 0));
+    launch(kTierHostOnly, p->side_stream, 2);
+    FT_CUDA(cudaEventRecord(p->join_ev, p->side_stream));
+    launch(kTierDeviceOnly, st, 8);
+    FT_CUDA(cudaStreamWaitEvent(st, p->join_ev, 0));
+  }
+  FT_CUDA(cudaGetLastError());
+
+  for (uint32_t q = 0; q < n; ++q) {
+    ft_slot_mirror& s = p->slots[slot[q]];
+    ft_span_mirror& m = p->spans[span_id[q]];
+    m.written = true; m.npages = (uint32_t)pages_for_tokens(p, n_tokens[q]);
+    if (++s.spans_written == s.n_spans) s.state = FT_SLOT_READY;
+  }
+  p->free_pages -= need; p->free_blocks -= need_blocks;
+  p->bytes_written += bytes_total * (f32 ? 3 : 2);
+  return FT_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int32_t pool_free(ft_pool* p, const uint32_t* slot, uint32_t n, void* stream) {
+  if (!p) return FT_ERR_INVALID_ARG;
+  p->call_seq++;
+  if (n == 0) return FT_OK;
+  if (!slot) return FT_ERR_INVALID_ARG;
+  const ft_pool_config& c = p->cfg;
+  const uint32_t S = c.max_spans_per_sample;
+  std::vector<uint8_t> seen(c.max_samples, 0);
+  for (uint32_t i = 0; i < n; ++i) {
+    if (slot[i] >= c.max_samples) return FT_ERR_INVALID_ARG;
+    if (p->slots[slot[i]].state == FT_SLOT_FREE || seen[slot[i]]) return FT_ERR_UNKNOWN_SAMPLE;
+    seen[slot[i]] = 1;
+  }
+  std::vector<uint32_t> span_ids;
+  uint64_t pages = 0, blocks = 0, text = 0;
+  for (uint32_t i = 0; i < n; ++i) {
+    const ft_slot_mirror& s = p->slots[slot[i]];
+    for (uint32_t j = 0; j < s.n_spans; ++j) {
+      const ft_span_mirror& m = p->spans[(uint64_t)slot[i] * S + j];
+      if (!m.written) continue;
+      span_ids.push_back(slot[i] * S + j);
+      pages += m.npages; blocks += (m.npages + kListBlock - 1) / kListBlock;
+    }
+    text += s.n_text_pages;
+  }
+  const uint32_t ns = (uint32_t)span_ids.size();
+  const size_t o_sid = 0, o_slot = (size_t)ns * 4;
+  const size_t blob_bytes = align_up(o_slot + (size_t)n * 4, 256);
+  const size_t o_poff = blob_bytes, o_boff = o_poff + (size_t)(ns + 1) * 4, o_toff = o_boff + (size_t)(ns + 1) * 4;
+  const size_t o_tails = align_up(o_toff + (size_t)(n + 1) * 4, 16);
+  const size_t total_bytes = o_tails + 16;
+  std::vector<uint8_t> blob(blob_bytes, 0);
+  if (ns) memcpy(blob.data() + o_sid, span_ids.data(), (size_t)ns * 4);
+  memcpy(blob.data() + o_slot, slot, (size_t)n * 4);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  void* d = nullptr;
+  int32_t rc = stage_upload(p, blob.data(), blob_bytes, total_bytes, st, &d);
+  if (rc != FT_OK) return rc;
+  uint8_t* db = static_cast<uint8_t*>(d);
+  FreeCall f;
+  f.n_spans = ns; f.n_samples = n;
+  f.span_id = reinterpret_cast<uint32_t*>(db + o_sid);
+  f.slot = reinterpret_cast<uint32_t*>(db + o_slot);
+  f.page_off = reinterpret_cast<uint32_t*>(db + o_poff);
+  f.blk_off = reinterpret_cast<uint32_t*>(db + o_boff);
+  f.tp_off = reinterpret_cast<uint32_t*>(db + o_toff);
+  f.tails = reinterpret_cast<uint32_t*>(db + o_tails);
+  k_free_scan<<<1, 1024, 0, st>>>(p->view, f);
+  const uint64_t items = pages + text;
+  if (items) k_free_fill<<<(unsigned)((items + 255) / 256), 256, 0, st>>>(p->view, f, (uint32_t)pages, (uint32_t)text);
+  k_free_clear<<<(n + 255) / 256, 256, 0, st>>>(p->view, f);
+  FT_CUDA(cudaGetLastError());
+  p->gpu_launches += items ? 3 : 2;
+
+  for (uint32_t i = 0; i < n; ++i) {
+    ft_slot_mirror& s = p->slots[slot[i]];
+    for (uint32_t j = 0; j < s.n_spans; ++j) p->spans[(uint64_t)slot[i] * S + j] = ft_span_mirror();
+    p->live_samples--; p->live_spans -= s.n_spans;
+    const uint64_t gen = s.generation + 1;
+    s = ft_slot_mirror();
+    s.generation = gen;
+  }
+  p->free_pages += pages; p->free_blocks += blocks; p->free_text_pages += text;
+  p->free_epoch++;
+  return FT_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int32_t pool_status(ft_pool* p, int32_t* code, uint64_t* detail) {
+  if (!p) return FT_ERR_INVALID_ARG;
+  FT_CUDA(cudaDeviceSynchronize());
+  unsigned long long key = 0;
+  FT_CUDA(cudaMemcpy(&key, p->view.status, 8, cudaMemcpyDeviceToHost));
+  if (key == ~0ull) { if (code) *code = 0; if (detail) *detail = 0; return FT_OK; }
+  if (code) *code = -(int32_t)((key >> 32) & 0xFF);
+  if (detail) *detail = key & 0xFFFFFFFFull;
+  FT_CUDA(cudaMemset(p->view.status, 0xFF, 8));
+  return FT_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int32_t pool_stats(ft_pool* p, ft_pool_stats* out) {
+  if (!p || !out) return FT_ERR_INVALID_ARG;
+  out->pages_total = p->cfg.hbm_pages + p->cfg.host_pages;
+  out->pages_free = p->free_pages;
+  out->hbm_pages = p->cfg.hbm_pages; out->host_pages = p->cfg.host_pages;
+  out->text_pages_total = p->view.text_pages; out->text_pages_free = p->free_text_pages;
+  out->live_samples = p->live_samples; out->live_spans = p->live_spans;
+  out->bytes_written = p->bytes_written; out->bytes_gathered = p->bytes_gathered;
+  out->gpu_launches = p->gpu_launches;
+  return FT_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int32_t pool_debug_span_pages(ft_pool* p, uint32_t slot, uint32_t span, uint64_t* gva_out, uint32_t cap,
+                                         uint32_t* n) {
+  if (!p || slot >= p->cfg.max_samples) return FT_ERR_INVALID_ARG;
+  const ft_slot_mirror& s = p->slots[slot];
+  if (s.state == FT_SLOT_FREE) return FT_ERR_UNKNOWN_SAMPLE;
+  if (span >= s.n_spans) return FT_ERR_INVALID_ARG;
+  const uint32_t sid = slot * p->cfg.max_spans_per_sample + span;
+  const uint32_t k = p->spans[sid].npages;
+  if (n) *n = k;
+  FT_CUDA(cudaDeviceSynchronize());
+  const uint32_t want = std::min(k, cap);
+  const uint32_t nb = (want + kListBlock - 1) / kListBlock;
+  std::vector<uint32_t> blks(nb);
+  if (nb) FT_CUDA(cudaMemcpy(blks.data(), p->view.sp_blocks + (uint64_t)sid * p->view.blocks_per_span, (size_t)nb * 4, cudaMemcpyDeviceToHost));
+  for (uint32_t b = 0; b < nb; ++b) {
+    const uint32_t cnt = std::min(kListBlock, want - b * kListBlock);
+    FT_CUDA(cudaMemcpy(gva_out + (size_t)b * kListBlock, p->view.list_blocks + (uint64_t)blks[b] * kListBlock, (size_t)cnt * 8, cudaMemcpyDeviceToHost));
+  }
+  return FT_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int32_t pool_debug_ring(ft_pool* p, uint32_t* out, uint64_t cap, uint64_t* n) {
+  if (!p) return FT_ERR_INVALID_ARG;
+  FT_CUDA(cudaDeviceSynchronize());
+  RingState s;
+  FT_CUDA(cudaMemcpy(&s, p->view.ring_state, sizeof(s), cudaMemcpyDeviceToHost));
+  if (n) *n = s.count;
+  std::vector<uint32_t> all(p->view.ring_cap);
+  FT_CUDA(cudaMemcpy(all.data(), p->view.ring, (size_t)p->view.ring_cap * 4, cudaMemcpyDeviceToHost));
+  for (uint64_t i = 0; i < s.count && i < cap; ++i) out[i] = all[(s.head + i) % p->view.ring_cap];
+  return FT_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int32_t pool_debug_translate(ft_pool* p, const uint64_t* gva, uint32_t n, uint32_t* kind, uint64_t* frame,
+                                        uint64_t* offset, int32_t* status) {
+  if (!p || (n && (!gva || !kind || !frame || !offset || !status))) return FT_ERR_INVALID_ARG;
+  if (n == 0) return FT_OK;
+  uint8_t* d = nullptr;
+  const size_t bytes = (size_t)n * (8 + 4 + 8 + 8 + 4);
+  FT_CUDA(cudaMalloc(&d, bytes));
+  uint64_t* d_gva = reinterpret_cast<uint64_t*>(d);
+  uint64_t* d_frame = d_gva + n;
+  uint64_t* d_off = d_frame + n;
+  uint32_t* d_kind = reinterpret_cast<uint32_t*>(d_off + n);
+  int32_t* d_status = reinterpret_cast<int32_t*>(d_kind + n);
+  FT_CUDA(cudaMemcpy(d_gva, gva, (size_t)n * 8, cudaMemcpyHostToDevice));
+  k_debug_translate<<<(n + 255) / 256, 256>>>(p->view, d_gva, n, d_kind, d_frame, d_off, d_status,
+                                              reinterpret_cast<uint64_t>(p->hbm_base), reinterpret_cast<uint64_t>(p->host_dev),
+                                              reinterpret_cast<uint64_t>(p->d_text));
+  p->gpu_launches++;
+  FT_CUDA(cudaDeviceSynchronize());
+  FT_CUDA(cudaMemcpy(kind, d_kind, (size_t)n * 4, cudaMemcpyDeviceToHost));
+  FT_CUDA(cudaMemcpy(frame, d_frame, (size_t)n * 8, cudaMemcpyDeviceToHost));
+  FT_CUDA(cudaMemcpy(offset, d_off, (size_t)n * 8, cudaMemcpyDeviceToHost));
+  FT_CUDA(cudaMemcpy(status, d_status, (size_t)n * 4, cudaMemcpyDeviceToHost));
+  FT_CUDA(cudaFree(d));
+  return FT_OK;
+}
