@@ -242,6 +242,20 @@ int32_t pool_status(ft_pool* pool, int32_t* first_device_error, uint64_t* detail
 
 int32_t pool_stats(ft_pool* pool, ft_pool_stats* out);
 
+/*
+ * Kernel timing for benchmarks.  While enabled, the library brackets each of its copy kernels with CUDA
+ * events on the stream that kernel is launched on (the host-tier kernels run on the pool's side stream).
+ * pool_profile_read synchronises the device, adds up the elapsed time and launch count per kernel class
+ * since the last read, and clears them.  Classes: a single-tier pool's kernels count under its tier.
+ */
+enum { FT_K_GATHER_DEVICE = 0, FT_K_GATHER_HOST = 1, FT_K_SCATTER_DEVICE = 2, FT_K_SCATTER_HOST = 3, FT_K_COUNT = 4 };
+typedef struct {
+  double ms;
+  uint64_t launches;
+} ft_kernel_time;
+int32_t pool_profile_enable(ft_pool* pool, int32_t on);
+int32_t pool_profile_read(ft_pool* pool, ft_kernel_time* out /* host [FT_K_COUNT] */);
+
 /* Page GVAs of one span, by ordinal (for parity checks).  Synchronises. */
 int32_t pool_debug_span_pages(ft_pool* pool, uint32_t slot, uint32_t span, uint64_t* gva_out,
                               uint32_t cap, uint32_t* n);

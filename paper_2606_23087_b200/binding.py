@@ -24,7 +24,7 @@ STATUS = {
 EXPORTS = (
     "pool_create", "pool_register_samples", "pool_write_embeddings", "pool_plan_microbatches", "plan_summary",
     "plan_arrays", "plan_destroy", "pool_gather_packed", "pool_free", "pool_status", "pool_stats",
-    "pool_debug_span_pages", "pool_debug_ring", "pool_debug_translate", "pool_destroy", "flowpool_last_cuda_error",
+    "pool_profile_enable", "pool_profile_read", "pool_debug_span_pages", "pool_debug_ring", "pool_debug_translate", "pool_destroy", "flowpool_last_cuda_error",
 )
 
 
@@ -62,6 +62,12 @@ class PoolStats(C.Structure):
         "live_samples", "live_spans", "bytes_written", "bytes_gathered", "gpu_launches")]
 
 
+class KernelTime(C.Structure):
+    _fields_ = [("ms", C.c_double), ("launches", C.c_uint64)]
+
+
+KERNEL_CLASSES = ("gather_device", "gather_host", "scatter_device", "scatter_host")
+
 _lib = None
 
 
@@ -85,6 +91,8 @@ def lib():
             "pool_free": [P, P, u32, P],
             "pool_status": [P, P, P],
             "pool_stats": [P, P],
+            "pool_profile_enable": [P, i32],
+            "pool_profile_read": [P, P],
             "pool_debug_span_pages": [P, u32, u32, P, u32, P],
             "pool_debug_ring": [P, P, u64, P],
             "pool_debug_translate": [P, P, u32, P, P, P, P],
@@ -196,6 +204,16 @@ class Pool:
         if rc:
             raise FlowpoolError(rc, "pool_stats")
         return {k: getattr(s, k) for k, _ in PoolStats._fields_}
+
+    def profile_enable(self, on=True):
+        return lib().pool_profile_enable(self.h, 1 if on else 0)
+
+    def profile_read(self):
+        out = (KernelTime * len(KERNEL_CLASSES))()
+        rc = lib().pool_profile_read(self.h, out)
+        if rc:
+            raise FlowpoolError(rc, "pool_profile_read")
+        return {k: {"ms": out[i].ms, "launches": out[i].launches} for i, k in enumerate(KERNEL_CLASSES)}
 
     def span_pages(self, slot, span, cap=1 << 16):
         out = np.zeros(cap, np.uint64)

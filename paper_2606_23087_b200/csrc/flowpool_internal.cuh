@@ -221,10 +221,26 @@ struct ft_pool {
   cudaStream_t side_stream = nullptr;                  // host-tier traffic runs beside the HBM kernels
   cudaEvent_t fork_ev = nullptr, join_ev = nullptr;
   int sm_count = 148;
+  // optional kernel timing (pool_profile_*)
+  bool profiling = false;
+  struct prof_rec { int kind; cudaEvent_t e0, e1; };
+  std::vector<prof_rec> prof;
 };
 
 namespace ft {
 // uploads `bytes` from `src` (pageable) to the front of the pool's device scratch, asynchronously,
 // through the staging ring; afterwards at least `total_bytes` of scratch exist.  Returns the device pointer.
+// timing brackets around one kernel launch on `st` (no-ops unless profiling is on)
+inline void prof_begin(ft_pool* p, int kind, cudaStream_t st) {
+  if (!p->profiling) return;
+  ft_pool::prof_rec r{kind, nullptr, nullptr};
+  cudaEventCreate(&r.e0); cudaEventCreate(&r.e1);
+  cudaEventRecord(r.e0, st);
+  p->prof.push_back(r);
+}
+inline void prof_end(ft_pool* p, cudaStream_t st) {
+  if (!p->profiling) return;
+  cudaEventRecord(p->prof.back().e1, st);
+}
 int32_t stage_upload(ft_pool* p, const void* src, size_t bytes, size_t total_bytes, cudaStream_t st, void** d_out);
 }  // namespace ft

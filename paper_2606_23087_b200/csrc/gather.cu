@@ -183,16 +183,22 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_gather_packed(ft_
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   auto grid_for = [&](uint32_t per_sm) { return (unsigned)std::min<uint64_t>(n_tiles, (uint64_t)p->sm_count * per_sm); };
   if (p->cfg.host_pages == 0 || p->cfg.hbm_pages == 0) {
+    prof_begin(p, p->cfg.hbm_pages == 0 ? FT_K_GATHER_HOST : FT_K_GATHER_DEVICE, st);
     k_gather<kTierAll><<<grid_for(8), kGatherThreads, 0, st>>>(p->view, pv, a);
+    prof_end(p, st);
     p->gpu_launches += 1;
   } else {
     FT_CUDA(cudaEventRecord(p->fork_ev, st));
     FT_CUDA(cudaStreamWaitEvent(p->side_stream, p->fork_ev, 0));
     GatherArgs ah = a;
     ah.write_index = 0;
+    prof_begin(p, FT_K_GATHER_HOST, p->side_stream);
     k_gather<kTierHostOnly><<<grid_for(2), kGatherThreads, 0, p->side_stream>>>(p->view, pv, ah);
+    prof_end(p, p->side_stream);
     FT_CUDA(cudaEventRecord(p->join_ev, p->side_stream));
+    prof_begin(p, FT_K_GATHER_DEVICE, st);
     k_gather<kTierDeviceOnly><<<grid_for(8), kGatherThreads, 0, st>>>(p->view, pv, a);
+    prof_end(p, st);
     FT_CUDA(cudaStreamWaitEvent(st, p->join_ev, 0));
     p->gpu_launches += 2;
   }

@@ -740,12 +740,15 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings(
   // the byte copy: HBM-bound chunks on the caller's stream, host-bound chunks beside them
   const bool f32 = src_dtype == FT_F32;
   auto launch = [&](int mode, cudaStream_t s, uint32_t ctas_per_sm) {
+    const bool host_class = mode == kTierHostOnly || (mode == kTierAll && c.hbm_pages == 0);
+    prof_begin(p, host_class ? FT_K_SCATTER_HOST : FT_K_SCATTER_DEVICE, s);
     uint64_t grid = std::min<uint64_t>(total_chunks, (uint64_t)p->sm_count * ctas_per_sm);
     uint64_t per = (total_chunks + grid - 1) / grid;
     grid = (total_chunks + per - 1) / per;
     if (mode == kTierAll) { if (f32) k_scatter<kTierAll, true><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); else k_scatter<kTierAll, false><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); }
     else if (mode == kTierDeviceOnly) { if (f32) k_scatter<kTierDeviceOnly, true><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); else k_scatter<kTierDeviceOnly, false><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); }
     else { if (f32) k_scatter<kTierHostOnly, true><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); else k_scatter<kTierHostOnly, false><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); }
+    prof_end(p, s);
     p->gpu_launches++;
   };
   if (c.host_pages == 0) {
@@ -861,6 +864,26 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_stats(ft_pool* p,
   out->live_samples = p->live_samples; out->live_spans = p->live_spans;
   out->bytes_written = p->bytes_written; out->bytes_gathered = p->bytes_gathered;
   out->gpu_launches = p->gpu_launches;
+  return FT_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int32_t pool_profile_enable(ft_pool* p, int32_t on) {
+  if (!p) return FT_ERR_INVALID_ARG;
+  p->profiling = on != 0;
+  return FT_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int32_t pool_profile_read(ft_pool* p, ft_kernel_time* out) {
+  if (!p || !out) return FT_ERR_INVALID_ARG;
+  FT_CUDA(cudaDeviceSynchronize());
+  for (int k = 0; k < FT_K_COUNT; ++k) { out[k].ms = 0; out[k].launches = 0; }
+  for (auto& r : p->prof) {
+    float ms = 0;
+    if (cudaEventElapsedTime(&ms, r.e0, r.e1) == cudaSuccess) { out[r.kind].ms += ms; out[r.kind].launches++; }
+    cudaEventDestroy(r.e0); cudaEventDestroy(r.e1);
+  }
+  p->prof.clear();
+  cudaGetLastError();
   return FT_OK;
 }
 
