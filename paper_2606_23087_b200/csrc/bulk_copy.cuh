@@ -1,0 +1,139 @@
+// Bulk asynchronous copies (the TMA unit's non-tensor form, cp.async.bulk) driven by one warp through a ring
+// of shared-memory stages: global -> shared (completion on an mbarrier), then shared -> global (bulk groups).
+// One thread keeps `kDepth` loads in flight, so a handful of single-warp CTAs saturate a long-latency link
+// (mapped pinned host memory) without tying up the load/store pipelines of the SMs that stream HBM.
+// No cluster multicast anywhere.  Every wait is bounded.
+#pragma once
+#include <stdint.h>
+
+namespace ft {
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* b, uint32_t n) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(b)), "r"(n));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* b, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(b)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* b, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok) : "r"(smem_u32(b)), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ void bulk_g2s(void* dst_s, const void* src_g, uint32_t bytes, uint64_t* b) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_u32(dst_s)), "l"(src_g), "r"(bytes), "r"(smem_u32(b)) : "memory");
+}
+__device__ __forceinline__ void bulk_s2g(void* dst_g, const void* src_s, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+               ::"l"(dst_g), "r"(smem_u32(src_s)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+constexpr int kBulkStages = 12;            // ring size
+constexpr int kBulkDepth = 8;              // loads in flight
+constexpr uint32_t kBulkStageBytes = 16384;
+constexpr uint32_t kBulkSpinLimit = 20000000;  // mbarrier polls before a copy is declared lost
+
+// fp32 -> bf16 on bit patterns: IEEE round-to-nearest-even, denormals kept, NaN -> sign | 0x7FC0
+__device__ __forceinline__ uint32_t bulk_rne_bf16(uint32_t u) {
+  if ((u & 0x7FFFFFFFu) > 0x7F800000u) return ((u >> 16) & 0x8000u) | 0x7FC0u;
+  return (u + 0x7FFFu + ((u >> 16) & 1u)) >> 16;
+}
+
+// Warp-wide copy pipeline: every lane of a one-warp CTA calls push()/drain() with the same arguments; lane 0
+// issues the asynchronous operations.  Copy number i goes into stage i % kBulkStages; before that, copy
+// i - kBulkDepth is retired (wait for its load, optionally cast it in place, start its store).  A stage is
+// reused only after the store that last read it has finished reading shared memory.
+// CAST: the staged bytes are fp32 and the stored bytes their bf16 image (half as many).
+template <bool CAST>
+struct BulkRing {
+  uint8_t* stage;    // kBulkStages * kBulkStageBytes of shared memory, 128-byte aligned
+  uint64_t* bar;     // kBulkStages mbarriers
+  uint64_t* dst_q;   // kBulkStages pending destinations (shared memory)
+  uint32_t* len_q;   // kBulkStages pending staged lengths
+  uint64_t issued, retired;
+  bool lost;
+
+  __device__ void init(uint8_t* stage_, uint64_t* bar_, uint64_t* dst_q_, uint32_t* len_q_) {
+    stage = stage_; bar = bar_; dst_q = dst_q_; len_q = len_q_;
+    issued = retired = 0; lost = false;
+    if ((threadIdx.x & 31) == 0) {
+      for (int i = 0; i < kBulkStages; ++i) mbar_init(&bar[i], 1);
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+      fence_async_smem();
+    }
+    __syncwarp();
+  }
+  __device__ void retire_one() {
+    const uint32_t lane = threadIdx.x & 31;
+    const uint64_t k = retired++;
+    const int st = (int)(k % kBulkStages);
+    const uint32_t parity = (uint32_t)((k / kBulkStages) & 1);
+    uint32_t bad = 0;
+    if (lane == 0) {
+      uint32_t spins = 0;
+      while (!mbar_try_wait(&bar[st], parity)) {
+        if (++spins > kBulkSpinLimit) { bad = 1; break; }
+      }
+    }
+    bad = __shfl_sync(0xFFFFFFFFu, bad, 0);
+    if (bad) { lost = true; return; }
+    uint8_t* sp = stage + (size_t)st * kBulkStageBytes;
+    uint32_t len = len_q[st];
+    if (CAST) {
+      // in place: lane t of round r reads floats [4t, 4t+4) and writes bf16 [4t, 4t+4); a round's writes land
+      // below every later round's reads, and inside a round all reads come before all writes
+      const uint32_t nvec = len >> 4;
+      for (uint32_t t0 = 0; t0 < nvec; t0 += 32) {
+        const uint32_t t = t0 + lane;
+        uint4 f = make_uint4(0, 0, 0, 0);
+        if (t < nvec) f = reinterpret_cast<const uint4*>(sp)[t];
+        __syncwarp();
+        if (t < nvec)
+          reinterpret_cast<uint2*>(sp)[t] = make_uint2(bulk_rne_bf16(f.x) | (bulk_rne_bf16(f.y) << 16),
+                                                       bulk_rne_bf16(f.z) | (bulk_rne_bf16(f.w) << 16));
+        __syncwarp();
+      }
+      len >>= 1;
+      fence_async_smem();  // the cast's generic-proxy writes must be visible to the bulk store
+      __syncwarp();
+    }
+    if (lane == 0) {
+      bulk_s2g(reinterpret_cast<void*>(dst_q[st]), sp, len);
+      bulk_commit();
+    }
+  }
+  // bytes staged: multiple of 16 (32 with CAST), <= kBulkStageBytes; src and dst 16-byte aligned
+  __device__ void push(const void* src, void* dst, uint32_t bytes) {
+    if (lost) return;
+    if (issued - retired >= (uint64_t)kBulkDepth) retire_one();
+    if (lost) return;
+    const int st = (int)(issued % kBulkStages);
+    if ((threadIdx.x & 31) == 0) {
+      bulk_wait_read<kBulkStages - kBulkDepth>();
+      dst_q[st] = reinterpret_cast<uint64_t>(dst);
+      len_q[st] = bytes;
+      mbar_expect_tx(&bar[st], bytes);
+      bulk_g2s(stage + (size_t)st * kBulkStageBytes, src, bytes, &bar[st]);
+    }
+    __syncwarp();
+    ++issued;
+  }
+  __device__ void drain() {
+    while (!lost && retired < issued) retire_one();
+    if ((threadIdx.x & 31) == 0) bulk_wait_all<0>();
+    __syncwarp();
+  }
+};
+
+constexpr size_t kBulkSmemBytes = (size_t)kBulkStages * kBulkStageBytes;
+
+}  // namespace ft

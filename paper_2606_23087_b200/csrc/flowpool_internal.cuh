@@ -221,6 +221,10 @@ struct ft_pool {
   cudaStream_t side_stream = nullptr;                  // host-tier traffic runs beside the HBM kernels
   cudaEvent_t fork_ev = nullptr, join_ev = nullptr;
   int sm_count = 148;
+  int host_ctas = 8;            // grid of the host-tier copy kernels: few SMs, so that long-latency host-link
+                                // accesses do not clog the memory pipelines of the SMs that stream HBM
+                                // (FLOWPOOL_HOST_CTAS overrides)
+  int dev_ctas_per_sm = 8;      // resident CTAs per SM of the device-tier copy kernels
   // optional kernel timing (pool_profile_*)
   bool profiling = false;
   struct prof_rec { int kind; cudaEvent_t e0, e1; };

@@ -6,6 +6,9 @@
 // leaves the frame addresses in shared memory; then every warp of the CTA streams rows with 16-byte
 // vectors.  Rows that straddle pages carry one address per page touched.  With a two-tier pool the
 // kernel is launched twice, once per tier, so host-link reads never stall HBM reads.
+#include <algorithm>
+
+#include "bulk_copy.cuh"
 #include "flowpool_internal.cuh"
 
 namespace ft {
@@ -65,12 +68,21 @@ __global__ void __launch_bounds__(kGatherThreads) k_gather(PoolView v, PlanView 
             if (q + 1 == pl.mb_sample_off[j + 1]) a.cu[e + 1] = (int32_t)(pl.sample_row_off[q + 1] - pl.mb_row_off[j]);
           }
         }
-        // token id, through the text page
-        const uint32_t tp = v.s_text_pages[(uint64_t)slot * v.text_pages_per_sample + p / kTextPageIds];
-        uint64_t off;
-        const uint64_t tpte = translate(v, v.text_gva_base + (uint64_t)tp * FT_TEXT_PAGE_BYTES, &off);
-        const int32_t id = reinterpret_cast<const int32_t*>(tpte & ~kPteFlagMask)[p % kTextPageIds];
-        if (id != v.placeholder_id) {
+        // Is position p inside a placeholder run?  The span table decides (last span with pos_start <= p).
+        const uint32_t sbase = slot * v.spans_per_sample, ns = v.s_n_spans[slot];
+        uint32_t lo = 0, hi = ns;
+        while (lo < hi) {
+          const uint32_t mid = (lo + hi) >> 1;
+          if (v.sp_pos[sbase + mid] <= p) lo = mid + 1; else hi = mid;
+        }
+        const uint32_t sid = sbase + lo - 1;
+        const bool in_run = lo > 0 && p < v.sp_pos[sid] + v.sp_tokens[sid];
+        if (!in_run) {
+          // token id, through the text page, then the embedding-table row
+          const uint32_t tp = v.s_text_pages[(uint64_t)slot * v.text_pages_per_sample + p / kTextPageIds];
+          uint64_t off;
+          const uint64_t tpte = translate(v, v.text_gva_base + (uint64_t)tp * FT_TEXT_PAGE_BYTES, &off);
+          const int32_t id = reinterpret_cast<const int32_t*>(tpte & ~kPteFlagMask)[p % kTextPageIds];
           if (id < 0 || (uint32_t)id >= a.vocab) {
             note_error(v, a.call_seq, FT_ERR_BAD_TOKEN_ID, (uint32_t)out_row);
           } else {
@@ -81,20 +93,12 @@ __global__ void __launch_bounds__(kGatherThreads) k_gather(PoolView v, PlanView 
             d.nseg = 1;
           }
         } else {
-          // the span whose run contains p: last span with pos_start <= p
-          const uint32_t sbase = slot * v.spans_per_sample, ns = v.s_n_spans[slot];
-          uint32_t lo = 0, hi = ns;
-          while (lo < hi) {
-            const uint32_t mid = (lo + hi) >> 1;
-            if (v.sp_pos[sbase + mid] <= p) lo = mid + 1; else hi = mid;
-          }
-          const uint32_t sid = sbase + lo - 1;
           const uint64_t b = (uint64_t)(p - v.sp_pos[sid]) * v.row_bytes;  // byte offset inside the span image
           const uint32_t o0 = (uint32_t)(b >> v.page_shift);
           d.off0 = (uint32_t)(b & (v.page_bytes - 1));
           d.shift = v.page_shift;
           const uint32_t nseg = ((d.off0 + v.row_bytes - 1) >> v.page_shift) + 1;
-          bool ok = lo > 0 && nseg <= kMaxSeg;
+          bool ok = nseg <= kMaxSeg;
           for (uint32_t s = 0; ok && s < nseg; ++s) {
             uint64_t poff;
             const uint64_t pte = translate(v, span_page_gva(v, sid, o0 + s), &poff);
@@ -119,31 +123,72 @@ __global__ void __launch_bounds__(kGatherThreads) k_gather(PoolView v, PlanView 
         *take = MODE == kTierAll || (MODE == kTierHostOnly) == host;
         return reinterpret_cast<const uint4*>((pte & ~kPteFlagMask) + (ab & mask));
       };
-      uint32_t x = lane;
-      for (; x + 96 < row_vecs; x += 128) {
-        bool t0, t1, t2, t3;
-        const uint4* s0 = src_of(x, &t0);
-        const uint4* s1 = src_of(x + 32, &t1);
-        const uint4* s2 = src_of(x + 64, &t2);
-        const uint4* s3 = src_of(x + 96, &t3);
-        uint4 a0, a1, a2, a3;
-        if (t0) a0 = __ldcs(s0);
-        if (t1) a1 = __ldcs(s1);
-        if (t2) a2 = __ldcs(s2);
-        if (t3) a3 = __ldcs(s3);
-        if (t0) __stcs(dst + x, a0);
-        if (t1) __stcs(dst + x + 32, a1);
-        if (t2) __stcs(dst + x + 64, a2);
-        if (t3) __stcs(dst + x + 96, a3);
-      }
-      for (; x < row_vecs; x += 32) {
-        bool t0;
-        const uint4* s0 = src_of(x, &t0);
-        if (t0) __stcs(dst + x, __ldcs(s0));
+      // U vectors per lane in flight before the first store: 4 for HBM frames; 16 for host frames, whose
+      // reads cross the host link with microseconds of latency and need far more bytes outstanding
+      constexpr int U = MODE == kTierHostOnly ? 16 : 4;
+      for (uint32_t x0 = lane; x0 < row_vecs; x0 += 32 * U) {
+        uint4 val[U];
+        bool take[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          const uint32_t x = x0 + 32 * u;
+          take[u] = false;
+          if (x < row_vecs) {
+            const uint4* s = src_of(x, &take[u]);
+            if (take[u]) val[u] = __ldcs(s);
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+          if (take[u]) __stcs(dst + x0 + 32 * u, val[u]);
       }
     }
     __syncthreads();
   }
+}
+
+// Host-tier vision data, page by page.  A span's rows are consecutive output rows, so a page of the span is one
+// contiguous byte range of the output: each host-tier page becomes a few bulk copies host frame -> shared ->
+// output, read in place over the mapped pointer.  One warp per CTA: the lanes translate 32 page ordinals at a
+// time (page list -> GVA -> page-table entry), lane 0 drives the copy ring.  A handful of CTAs saturate the link.
+__global__ void __launch_bounds__(32) k_gather_host_bulk(PoolView v, PlanView pl, GatherArgs a) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  __shared__ uint64_t bars[kBulkStages];
+  __shared__ uint64_t dst_q[kBulkStages];
+  __shared__ uint32_t len_q[kBulkStages];
+  const uint32_t lane = threadIdx.x;
+  BulkRing<false> ring;
+  ring.init(smem, bars, dst_q, len_q);
+  uint64_t item = 0;
+  for (uint32_t q = a.q_lo; q < a.q_hi; ++q) {
+    const uint32_t slot = pl.mb_samples[q], ns = v.s_n_spans[slot];
+    const uint64_t row0 = pl.sample_row_off[q] - a.row_lo;
+    for (uint32_t j = 0; j < ns; ++j) {
+      const uint32_t sid = slot * v.spans_per_sample + j;
+      const uint32_t npages = v.sp_npages[sid];
+      const uint64_t nbytes = (uint64_t)v.sp_tokens[sid] * v.row_bytes;
+      uint8_t* dst_base = a.out + (row0 + v.sp_pos[sid]) * v.row_bytes;
+      for (uint32_t g = 0; g < npages; g += 32, ++item) {
+        if (item % gridDim.x != blockIdx.x) continue;
+        const uint32_t o = g + lane;
+        uint64_t pte = 0, off;
+        if (o < npages) pte = translate(v, span_page_gva(v, sid, o), &off);
+        const bool host = (pte & kPteValid) && (pte & kPteHost);
+        const uint32_t mask = __ballot_sync(0xFFFFFFFFu, host);
+        for (uint32_t m = mask; m; m &= m - 1) {
+          const int l = __ffs(m) - 1;
+          const uint64_t p_l = __shfl_sync(0xFFFFFFFFu, pte, l);
+          const uint64_t b0 = (uint64_t)(g + l) << v.page_shift;
+          const uint64_t len = min(v.page_bytes, nbytes - b0);
+          const uint8_t* src = reinterpret_cast<const uint8_t*>(p_l & ~kPteFlagMask);
+          for (uint64_t x = 0; x < len; x += kBulkStageBytes)
+            ring.push(src + x, dst_base + b0 + x, (uint32_t)min((uint64_t)kBulkStageBytes, len - x));
+        }
+      }
+    }
+  }
+  ring.drain();
+  if (ring.lost && lane == 0) note_error(v, a.call_seq, FT_ERR_TIMEOUT, blockIdx.x);
 }
 
 }  // namespace ft
@@ -181,10 +226,11 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_gather_packed(ft_
   a.call_seq = p->call_seq; a.write_index = 1;
   const uint64_t n_tiles = (a.row_hi + kTileRows - 1) / kTileRows - a.row_lo / kTileRows;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  auto grid_for = [&](uint32_t per_sm) { return (unsigned)std::min<uint64_t>(n_tiles, (uint64_t)p->sm_count * per_sm); };
+  auto grid_for = [&](uint64_t ctas) { return (unsigned)std::min<uint64_t>(n_tiles, ctas); };
+  const uint64_t dev_ctas = (uint64_t)p->sm_count * p->dev_ctas_per_sm, host_ctas = p->host_ctas;
   if (p->cfg.host_pages == 0 || p->cfg.hbm_pages == 0) {
     prof_begin(p, p->cfg.hbm_pages == 0 ? FT_K_GATHER_HOST : FT_K_GATHER_DEVICE, st);
-    k_gather<kTierAll><<<grid_for(8), kGatherThreads, 0, st>>>(p->view, pv, a);
+    k_gather<kTierAll><<<grid_for(p->cfg.hbm_pages == 0 ? host_ctas : dev_ctas), kGatherThreads, 0, st>>>(p->view, pv, a);
     prof_end(p, st);
     p->gpu_launches += 1;
   } else {
@@ -193,11 +239,16 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_gather_packed(ft_
     GatherArgs ah = a;
     ah.write_index = 0;
     prof_begin(p, FT_K_GATHER_HOST, p->side_stream);
-    k_gather<kTierHostOnly><<<grid_for(2), kGatherThreads, 0, p->side_stream>>>(p->view, pv, ah);
+    static bool attr_set = false;
+    if (!attr_set) {
+      FT_CUDA(cudaFuncSetAttribute(k_gather_host_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBulkSmemBytes));
+      attr_set = true;
+    }
+    k_gather_host_bulk<<<(unsigned)host_ctas, 32, kBulkSmemBytes, p->side_stream>>>(p->view, pv, ah);
     prof_end(p, p->side_stream);
     FT_CUDA(cudaEventRecord(p->join_ev, p->side_stream));
     prof_begin(p, FT_K_GATHER_DEVICE, st);
-    k_gather<kTierDeviceOnly><<<grid_for(8), kGatherThreads, 0, st>>>(p->view, pv, a);
+    k_gather<kTierDeviceOnly><<<grid_for(dev_ctas), kGatherThreads, 0, st>>>(p->view, pv, a);
     prof_end(p, st);
     FT_CUDA(cudaStreamWaitEvent(st, p->join_ev, 0));
     p->gpu_launches += 2;

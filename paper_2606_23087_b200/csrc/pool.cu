@@ -10,9 +10,11 @@
 //   k_free_scan/_fill  pages, list blocks and text pages back to the ring tails
 #include <algorithm>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <unordered_set>
 
+#include "bulk_copy.cuh"
 #include "flowpool_internal.cuh"
 
 namespace ft {
@@ -248,7 +250,7 @@ __device__ __forceinline__ uint32_t pack2(uint32_t a, uint32_t b) { return rne_b
 enum { kTierAll = 0, kTierDeviceOnly = 1, kTierHostOnly = 2 };
 
 template <int MODE, bool F32>
-__global__ void __launch_bounds__(256) k_scatter(PoolView v, WriteCall c, uint64_t total_chunks, uint64_t per_cta) {
+__global__ void __launch_bounds__(256, 8) k_scatter(PoolView v, WriteCall c, uint64_t total_chunks, uint64_t per_cta) {
   const uint64_t c0 = (uint64_t)blockIdx.x * per_cta;
   const uint64_t c1 = min(total_chunks, c0 + per_cta);
   if (c0 >= c1) return;
@@ -312,6 +314,50 @@ __global__ void __launch_bounds__(256) k_scatter(PoolView v, WriteCall c, uint64
       }
     }
   }
+}
+
+
+// Host-tier pages of a producer call, page by page: source bytes -> shared -> host frame with bulk copies (the
+// fp32 source is cast in shared memory on the way).  One warp per CTA; lanes translate 32 page ordinals at a
+// time, lane 0 drives the ring; a handful of CTAs saturate the host link.
+template <bool F32>
+__global__ void __launch_bounds__(32) k_scatter_host_bulk(PoolView v, WriteCall c, uint64_t call_seq) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  __shared__ uint64_t bars[kBulkStages];
+  __shared__ uint64_t dst_q[kBulkStages];
+  __shared__ uint32_t len_q[kBulkStages];
+  const uint32_t lane = threadIdx.x;
+  BulkRing<F32> ring;
+  ring.init(smem, bars, dst_q, len_q);
+  constexpr uint32_t kOutPiece = F32 ? kBulkStageBytes / 2 : kBulkStageBytes;  // destination bytes per staged copy
+  uint64_t item = 0;
+  for (uint32_t q = 0; q < c.n; ++q) {
+    const uint32_t sid = c.span_id[q];
+    const uint64_t nbytes = (uint64_t)c.n_tokens[q] * v.row_bytes;
+    const uint32_t npages = (uint32_t)((nbytes + v.page_bytes - 1) >> v.page_shift);
+    const uint8_t* src_q = reinterpret_cast<const uint8_t*>(c.src[q]);
+    for (uint32_t g = 0; g < npages; g += 32, ++item) {
+      if (item % gridDim.x != blockIdx.x) continue;
+      const uint32_t o = g + lane;
+      uint64_t pte = 0, off;
+      if (o < npages) pte = translate(v, span_page_gva(v, sid, o), &off);
+      const bool host = (pte & kPteValid) && (pte & kPteHost);
+      const uint32_t mask = __ballot_sync(0xFFFFFFFFu, host);
+      for (uint32_t m = mask; m; m &= m - 1) {
+        const int l = __ffs(m) - 1;
+        const uint64_t p_l = __shfl_sync(0xFFFFFFFFu, pte, l);
+        const uint64_t b0 = (uint64_t)(g + l) << v.page_shift;  // destination byte offset inside the span image
+        const uint64_t len = min(v.page_bytes, nbytes - b0);
+        uint8_t* dst = reinterpret_cast<uint8_t*>(p_l & ~kPteFlagMask);
+        for (uint64_t x = 0; x < len; x += kOutPiece) {
+          const uint32_t out_bytes = (uint32_t)min((uint64_t)kOutPiece, len - x);
+          ring.push(src_q + (F32 ? 2 : 1) * (b0 + x), dst + x, F32 ? 2 * out_bytes : out_bytes);
+        }
+      }
+    }
+  }
+  ring.drain();
+  if (ring.lost && lane == 0) note_error(v, call_seq, FT_ERR_TIMEOUT, blockIdx.x);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -473,6 +519,9 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_create(const ft_p
   } while (0)
   CK(cudaGetDevice(&p->device));
   CK(cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, p->device));
+  p->host_ctas = 8;
+  if (const char* e = getenv("FLOWPOOL_HOST_CTAS")) { int v = atoi(e); if (v > 0) p->host_ctas = v; }
+  if (const char* e = getenv("FLOWPOOL_DEV_CTAS_PER_SM")) { int v = atoi(e); if (v > 0) p->dev_ctas_per_sm = v; }
   CK(cudaStreamCreateWithFlags(&p->side_stream, cudaStreamNonBlocking));
   CK(cudaEventCreateWithFlags(&p->fork_ev, cudaEventDisableTiming));
   CK(cudaEventCreateWithFlags(&p->join_ev, cudaEventDisableTiming));
@@ -739,10 +788,10 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings(
 
   // the byte copy: HBM-bound chunks on the caller's stream, host-bound chunks beside them
   const bool f32 = src_dtype == FT_F32;
-  auto launch = [&](int mode, cudaStream_t s, uint32_t ctas_per_sm) {
+  auto launch = [&](int mode, cudaStream_t s) {
     const bool host_class = mode == kTierHostOnly || (mode == kTierAll && c.hbm_pages == 0);
     prof_begin(p, host_class ? FT_K_SCATTER_HOST : FT_K_SCATTER_DEVICE, s);
-    uint64_t grid = std::min<uint64_t>(total_chunks, (uint64_t)p->sm_count * ctas_per_sm);
+    uint64_t grid = std::min<uint64_t>(total_chunks, host_class ? (uint64_t)p->host_ctas : (uint64_t)p->sm_count * p->dev_ctas_per_sm);
     uint64_t per = (total_chunks + grid - 1) / grid;
     grid = (total_chunks + per - 1) / per;
     if (mode == kTierAll) { if (f32) k_scatter<kTierAll, true><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); else k_scatter<kTierAll, false><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); }
@@ -752,15 +801,25 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings(
     p->gpu_launches++;
   };
   if (c.host_pages == 0) {
-    launch(kTierAll, st, 8);
+    launch(kTierAll, st);
   } else if (c.hbm_pages == 0) {
-    launch(kTierAll, st, 2);
+    launch(kTierAll, st);
   } else {
     FT_CUDA(cudaEventRecord(p->fork_ev, st));
     FT_CUDA(cudaStreamWaitEvent(p->side_stream, p->fork_ev, 0));
-    launch(kTierHostOnly, p->side_stream, 2);
+    static bool attr_set = false;
+    if (!attr_set) {
+      FT_CUDA(cudaFuncSetAttribute(k_scatter_host_bulk<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBulkSmemBytes));
+      FT_CUDA(cudaFuncSetAttribute(k_scatter_host_bulk<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBulkSmemBytes));
+      attr_set = true;
+    }
+    prof_begin(p, FT_K_SCATTER_HOST, p->side_stream);
+    if (f32) k_scatter_host_bulk<true><<<(unsigned)p->host_ctas, 32, kBulkSmemBytes, p->side_stream>>>(p->view, w, p->call_seq);
+    else k_scatter_host_bulk<false><<<(unsigned)p->host_ctas, 32, kBulkSmemBytes, p->side_stream>>>(p->view, w, p->call_seq);
+    prof_end(p, p->side_stream);
+    p->gpu_launches++;
     FT_CUDA(cudaEventRecord(p->join_ev, p->side_stream));
-    launch(kTierDeviceOnly, st, 8);
+    launch(kTierDeviceOnly, st);
     FT_CUDA(cudaStreamWaitEvent(st, p->join_ev, 0));
   }
   FT_CUDA(cudaGetLastError());
