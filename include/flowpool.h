@@ -169,6 +169,36 @@ int32_t pool_write_embeddings(ft_pool* pool, uint32_t n_spans, const uint32_t* s
                               const void* const* src, uint32_t src_dtype, void* stream);
 
 /*
+ * pool_write_embeddings_noalloc -- the same producer scatter for callers that must not allocate.
+ * (The paper has no counterpart: this entry point exists for integration reasons only.)
+ *
+ * Who needs it: code that runs where a CUDA allocation is forbidden or would stall -- a producer thread
+ * inside a region where the framework has frozen its allocator, a caller holding a memory budget it may
+ * not exceed, a real-time loop that cannot afford the implicit device synchronisation of cudaMalloc/
+ * cudaFree.  pool_write_embeddings may grow the pool's device scratch and its pinned staging buffers; this
+ * variant never does.  It calls no cudaMalloc/cudaFree/cudaHostAlloc nor any other allocating routine:
+ * the per-call descriptors and scan outputs (the only scratch memory the write path needs beyond its
+ * inputs and the pool) live in one fixed array in the library's device image, FT_NOALLOC_SCRATCH_BYTES
+ * long, which every GPU that loads the library holds until the process exits.
+ *
+ * Same arguments, result, status codes and check order as pool_write_embeddings, plus:
+ *   - n_spans > FT_NOALLOC_MAX_SPANS -> FT_ERR_CAPACITY ("call too large for the fixed scratch"; split it);
+ *   - the device current at the call must be the pool's device, else FT_ERR_INVALID_ARG.
+ * The first call on each device looks up the array's device address once (cudaGetSymbolAddress); make
+ * that first call before any stream capture begins.  All calls, from every pool on the device, share
+ * the one array: it still holds the previous call's descriptors when the next call starts, nothing in
+ * it needs to start at zero (each call overwrites all it reads), and two calls whose kernels may overlap
+ * on the GPU (different streams without an ordering between them) race on it -- keep no-alloc writes on
+ * one stream, or order them with events.  The descriptors are copied from pageable host memory with
+ * cudaMemcpyAsync, which returns only after the host data has been taken.
+ */
+#define FT_NOALLOC_MAX_SPANS 4096u
+#define FT_NOALLOC_SCRATCH_BYTES (256u + 32u * (FT_NOALLOC_MAX_SPANS + 8u))
+int32_t pool_write_embeddings_noalloc(ft_pool* pool, uint32_t n_spans, const uint32_t* sample_slot,
+                                      const uint32_t* span_idx, const uint32_t* n_tokens,
+                                      const void* const* src, uint32_t src_dtype, void* stream);
+
+/*
  * pool_plan_microbatches -- the dynamic packing rule (Algorithm 1, Eq. 3), on
  * the device.  Samples are packed online in the order given, by best fit on
  * l(s) = seq_len (ties between equal residuals: the microbatch changed most

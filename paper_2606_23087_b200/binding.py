@@ -14,6 +14,7 @@ FT_BF16, FT_F32 = 0, 1
 FT_RING_SORTED, FT_RING_SHUFFLED = 0, 1
 FT_BIND_IDENTITY, FT_BIND_PERMUTED = 0, 1
 FT_PLAN_ALLOW_UNWRITTEN = 1
+FT_NOALLOC_MAX_SPANS = 4096
 
 STATUS = {
     0: "OK", -1: "INVALID_ARG", -2: "POOL_EXHAUSTED", -3: "UNKNOWN_SAMPLE", -4: "ALREADY_WRITTEN",
@@ -22,7 +23,8 @@ STATUS = {
 }
 
 EXPORTS = (
-    "pool_create", "pool_register_samples", "pool_write_embeddings", "pool_plan_microbatches", "plan_summary",
+    "pool_create", "pool_register_samples", "pool_write_embeddings", "pool_write_embeddings_noalloc",
+    "pool_plan_microbatches", "plan_summary",
     "plan_arrays", "plan_destroy", "pool_gather_packed", "pool_free", "pool_status", "pool_stats",
     "pool_profile_enable", "pool_profile_read", "pool_debug_span_pages", "pool_debug_ring", "pool_debug_translate", "pool_destroy", "flowpool_last_cuda_error",
 )
@@ -83,6 +85,7 @@ def lib():
             "pool_create": [P, P, P, P],
             "pool_register_samples": [P, u32, P, P, P, P, P, P, P],
             "pool_write_embeddings": [P, u32, P, P, P, P, u32, P],
+            "pool_write_embeddings_noalloc": [P, u32, P, P, P, P, u32, P],
             "pool_plan_microbatches": [P, P, u32, P, P, P],
             "plan_summary": [P, P, P, P],
             "plan_arrays": [P] * 13,
@@ -175,6 +178,14 @@ class Pool:
         src = np.ascontiguousarray(src_ptrs, dtype=np.uint64)
         return lib().pool_write_embeddings(self.h, len(slots), _p(slots), _p(span_idx), _p(n_tokens), _p(src),
                                            dtype, stream or None)
+
+    def write_embeddings_noalloc(self, slots, span_idx, n_tokens, src_ptrs, dtype, stream: int = 0):
+        """pool_write_embeddings_noalloc: same scatter, per-call scratch in the library's fixed device array
+        (for callers that may not allocate); at most FT_NOALLOC_MAX_SPANS spans per call."""
+        slots, span_idx, n_tokens = _u32(slots), _u32(span_idx), _u32(n_tokens)
+        src = np.ascontiguousarray(src_ptrs, dtype=np.uint64)
+        return lib().pool_write_embeddings_noalloc(self.h, len(slots), _p(slots), _p(span_idx), _p(n_tokens), _p(src),
+                                                   dtype, stream or None)
 
     def plan_microbatches(self, slots, cfg: PlanConfig, stream: int = 0):
         slots = _u32(slots)

@@ -1004,3 +1004,144 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_debug_translate(f
   FT_CUDA(cudaFree(d));
   return FT_OK;
 }
+
+// ------------------------------------------------------------------------------------------
+// No-allocation variant of the producer write.  Its per-call scratch (descriptors in, scan outputs out) is a
+// fixed array in the device image instead of the pool's growable cudaMalloc'd scratch, and the descriptors go
+// up from a stack buffer instead of the pinned staging ring.  The kernels are the ones pool_write_embeddings
+// launches.
+// ------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_noalloc_scratch[FT_NOALLOC_SCRATCH_BYTES];
+
+namespace ft {
+constexpr int kMaxDevices = 64;
+// g_noalloc_scratch is a host-side stand-in here, not a device address: kernels get the address that
+// cudaGetSymbolAddress returns for the device that is current (looked up once per device).
+static void* g_noalloc_dev_ptr[kMaxDevices] = {};
+
+static int32_t noalloc_scratch(int device, uint8_t** out) {
+  if (device < 0 || device >= kMaxDevices) return FT_ERR_INVALID_ARG;
+  if (!g_noalloc_dev_ptr[device]) {
+    void* ptr = nullptr;
+    FT_CUDA(cudaGetSymbolAddress(&ptr, g_noalloc_scratch));
+    g_noalloc_dev_ptr[device] = ptr;
+  }
+  *out = static_cast<uint8_t*>(g_noalloc_dev_ptr[device]);
+  return FT_OK;
+}
+}  // namespace ft
+
+extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings_noalloc(
+    ft_pool* p, uint32_t n, const uint32_t* slot, const uint32_t* span_idx, const uint32_t* n_tokens,
+    const void* const* src, uint32_t src_dtype, void* stream) {
+  if (!p) return FT_ERR_INVALID_ARG;
+  p->call_seq++;
+  if (src_dtype != FT_BF16 && src_dtype != FT_F32) return FT_ERR_INVALID_ARG;
+  if (n == 0) return FT_OK;
+  if (n > FT_NOALLOC_MAX_SPANS) return FT_ERR_CAPACITY;  // call too large for the fixed scratch: split it
+  if (!slot || !span_idx || !n_tokens || !src) return FT_ERR_INVALID_ARG;
+  int cur = -1;
+  FT_CUDA(cudaGetDevice(&cur));
+  if (cur != p->device) return FT_ERR_INVALID_ARG;
+  const ft_pool_config& c = p->cfg;
+  const uint32_t S = c.max_spans_per_sample;
+  const uint32_t chunk_shift = std::min<uint32_t>(p->view.page_shift, 14);
+  uint64_t need = 0, need_blocks = 0, total_chunks = 0, bytes_total = 0;
+
+  // descriptor blob on the stack: [src u64 n][span_id n][n_tokens n]; duplicate check in a fixed hash table
+  constexpr size_t kBlobMax = 16 * (size_t)FT_NOALLOC_MAX_SPANS + 256;
+  alignas(16) uint8_t blob[kBlobMax];
+  constexpr uint32_t kTab = 4 * FT_NOALLOC_MAX_SPANS;  // open addressing, load <= 1/4
+  uint32_t table[kTab];
+  memset(table, 0xFF, sizeof(table));
+  const size_t o_src = 0, o_sid = (size_t)n * 8, o_ntk = o_sid + (size_t)n * 4;
+  const size_t blob_bytes = align_up(o_ntk + (size_t)n * 4, 256);
+  uint64_t* b_src = reinterpret_cast<uint64_t*>(blob + o_src);
+  uint32_t* b_sid = reinterpret_cast<uint32_t*>(blob + o_sid);
+  uint32_t* b_ntk = reinterpret_cast<uint32_t*>(blob + o_ntk);
+  for (uint32_t q = 0; q < n; ++q) {
+    if (slot[q] >= c.max_samples) return FT_ERR_INVALID_ARG;
+    const ft_slot_mirror& s = p->slots[slot[q]];
+    if (s.state == FT_SLOT_FREE) return FT_ERR_UNKNOWN_SAMPLE;
+    if (span_idx[q] >= s.n_spans) return FT_ERR_INVALID_ARG;
+    const ft_span_mirror& m = p->spans[(uint64_t)slot[q] * S + span_idx[q]];
+    if (n_tokens[q] != m.tokens) return FT_ERR_INVALID_ARG;
+    if (!src[q] || (reinterpret_cast<uintptr_t>(src[q]) & 15)) return FT_ERR_INVALID_ARG;
+    const uint32_t sid = slot[q] * S + span_idx[q];
+    if (m.written) return FT_ERR_ALREADY_WRITTEN;
+    uint32_t h = (sid * 2654435761u) % kTab;
+    while (table[h] != 0xFFFFFFFFu) {
+      if (table[h] == sid) return FT_ERR_ALREADY_WRITTEN;  // named twice in this call
+      h = (h + 1) % kTab;
+    }
+    table[h] = sid;
+    b_src[q] = reinterpret_cast<uint64_t>(src[q]); b_sid[q] = sid; b_ntk[q] = n_tokens[q];
+    const uint64_t k = pages_for_tokens(p, n_tokens[q]);
+    need += k; need_blocks += (k + kListBlock - 1) / kListBlock;
+    const uint64_t bytes = (uint64_t)n_tokens[q] * p->view.row_bytes;
+    total_chunks += (bytes + (1ull << chunk_shift) - 1) >> chunk_shift;
+    bytes_total += bytes;
+  }
+  if (need > p->free_pages) return FT_ERR_POOL_EXHAUSTED;
+  if (need_blocks > p->free_blocks) return FT_ERR_CAPACITY;
+  if (need > 0xFFFFFFFFull) return FT_ERR_INVALID_ARG;
+
+  const size_t o_choff = blob_bytes, o_poff = align_up(o_choff + (size_t)(n + 1) * 8, 16);
+  const size_t o_boff = o_poff + (size_t)(n + 1) * 4, o_heads = align_up(o_boff + (size_t)(n + 1) * 4, 16);
+  if (o_heads + 16 > FT_NOALLOC_SCRATCH_BYTES) return FT_ERR_CAPACITY;
+  uint8_t* db = nullptr;
+  int32_t rc = noalloc_scratch(p->device, &db);
+  if (rc != FT_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // pageable source: the call returns once the bytes have been taken, so the stack buffer may die after it
+  FT_CUDA(cudaMemcpyAsync(db, blob, blob_bytes, cudaMemcpyHostToDevice, st));
+  WriteCall w;
+  w.n = n;
+  w.src = reinterpret_cast<uint64_t*>(db + o_src);
+  w.span_id = reinterpret_cast<uint32_t*>(db + o_sid);
+  w.n_tokens = reinterpret_cast<uint32_t*>(db + o_ntk);
+  w.chunk_off = reinterpret_cast<uint64_t*>(db + o_choff);
+  w.page_off = reinterpret_cast<uint32_t*>(db + o_poff);
+  w.blk_off = reinterpret_cast<uint32_t*>(db + o_boff);
+  w.heads = reinterpret_cast<uint32_t*>(db + o_heads);
+  w.chunk_shift = chunk_shift;
+  k_alloc_scan<<<1, 1024, 0, st>>>(p->view, w);
+  k_alloc_fill<<<(unsigned)((need + 255) / 256), 256, 0, st>>>(p->view, w, (uint32_t)need);
+  p->gpu_launches += 2;
+
+  const bool f32 = src_dtype == FT_F32;
+  auto launch = [&](int mode, cudaStream_t s) {
+    const bool host_class = mode == kTierAll && c.hbm_pages == 0;
+    uint64_t grid = std::min<uint64_t>(total_chunks, host_class ? (uint64_t)p->host_ctas : (uint64_t)p->sm_count * p->dev_ctas_per_sm);
+    uint64_t per = (total_chunks + grid - 1) / grid;
+    grid = (total_chunks + per - 1) / per;
+    if (mode == kTierAll) { if (f32) k_scatter<kTierAll, true><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); else k_scatter<kTierAll, false><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); }
+    else { if (f32) k_scatter<kTierDeviceOnly, true><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); else k_scatter<kTierDeviceOnly, false><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); }
+    p->gpu_launches++;
+  };
+  if (c.host_pages == 0 || c.hbm_pages == 0) {
+    launch(kTierAll, st);
+  } else {
+    FT_CUDA(cudaFuncSetAttribute(k_scatter_host_bulk<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBulkSmemBytes));
+    FT_CUDA(cudaFuncSetAttribute(k_scatter_host_bulk<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBulkSmemBytes));
+    FT_CUDA(cudaEventRecord(p->fork_ev, st));
+    FT_CUDA(cudaStreamWaitEvent(p->side_stream, p->fork_ev, 0));
+    if (f32) k_scatter_host_bulk<true><<<(unsigned)p->host_ctas, 32, kBulkSmemBytes, p->side_stream>>>(p->view, w, p->call_seq);
+    else k_scatter_host_bulk<false><<<(unsigned)p->host_ctas, 32, kBulkSmemBytes, p->side_stream>>>(p->view, w, p->call_seq);
+    p->gpu_launches++;
+    FT_CUDA(cudaEventRecord(p->join_ev, p->side_stream));
+    launch(kTierDeviceOnly, st);
+    FT_CUDA(cudaStreamWaitEvent(st, p->join_ev, 0));
+  }
+  FT_CUDA(cudaGetLastError());
+
+  for (uint32_t q = 0; q < n; ++q) {
+    ft_slot_mirror& s = p->slots[slot[q]];
+    ft_span_mirror& m = p->spans[b_sid[q]];
+    m.written = true; m.npages = (uint32_t)pages_for_tokens(p, n_tokens[q]);
+    if (++s.spans_written == s.n_spans) s.state = FT_SLOT_READY;
+  }
+  p->free_pages -= need; p->free_blocks -= need_blocks;
+  p->bytes_written += bytes_total * (f32 ? 3 : 2);
+  return FT_OK;
+}
