@@ -30,8 +30,10 @@ for p in (ROOT, os.path.join(ROOT, "tests")):
 METRIC = "packed-microbatch assembly throughput (producer scatter + plan + packed gather + free)"
 UNIT = "GB/s"
 CPU_SAMPLE = 256         # samples of the workload the oracle is timed on (about 10-30 s of CPU work)
-# dram bytes / algorithmic bytes of k_gather from the committed ncu summary (profiles/); None = not captured yet
-NCU_TRAFFIC_RATIO_GATHER = None
+# dram__bytes_read.sum + dram__bytes_write.sum over algorithmic bytes for one k_gather launch, from the ncu capture
+# summarised in profiles/k_gather_image_mix_7b_64samples_all_hbm.md (4.599 GB / 4.698 GB on the first 64 samples);
+# traffic grows in proportion to the tokens assembled, so a full launch is this ratio times its algorithmic bytes
+NCU_TRAFFIC_RATIO_GATHER = 0.979
 
 
 def algorithmic_bytes(w):
@@ -251,6 +253,21 @@ class DeviceJob:
         self.pool.destroy()
 
 
+def max_over_ranks(ms, dist, device="cuda"):
+    """A multi-rank time is the slowest rank's."""
+    if dist is None:
+        return ms
+    import torch
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_value(bytes_per_rank, world, ms):
+    """Whole-job GB/s: every rank moved bytes_per_rank in the (max-over-ranks) step time."""
+    return world * bytes_per_rank / ms / 1e6
+
+
 def timed_steps(job, steps, warmup, dist):
     torch = job.torch
     for _ in range(warmup):
@@ -275,10 +292,8 @@ def timed_steps(job, steps, warmup, dist):
     job.pool.profile_enable(False)
     launches = job.pool.stats()["gpu_launches"] - launches0
     if dist:
-        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = max_over_ranks(ms, dist)
         dist.barrier()
-        ms = float(t.item())
     torch.cuda.synchronize()
     return ms, prof, launches, n_mb
 
@@ -369,7 +384,7 @@ def run_ours(args):
     ms, prof, launches, n_mb = timed_steps(job, args.steps, args.warmup, dist)
     clocks = sampler.stop()
     wb, gb = algorithmic_bytes(w)
-    value = world * (wb + gb) / ms / 1e6
+    value = aggregate_value(wb + gb, world, ms)
     kern, host_b = kernel_breakdown(job, prof, args.steps)
     plan_ms = float(np.median(job.plan_ms)) if job.plan_ms else None
 

@@ -1,0 +1,86 @@
+"""Parity at the benchmark's full size (the 7B image-mix batch, 80 % HBM / 20 % pinned host, as bench.py
+launches it).  The oracle cannot hold this pool in seconds, so: the plan is compared array by array with the
+oracle's Algorithm 1 on the same lengths; cu_seqlens and position ids are compared in full with what the plan
+arrays determine; and sampled output rows are compared with rows the oracle side computes one by one from the
+generator (vision rows: the span's source row, through the oracle's cast when the source is fp32; text rows:
+the table row of the generated id)."""
+import numpy as np
+import pytest
+import torch
+
+import workloads
+from harness import bits16, bits32, plan_config_fields
+from oracle import PlanConfig, f32_to_bf16_rne, plan_from_lengths
+
+pytestmark = pytest.mark.gpu
+
+PLAN_KEYS = ("mb_sample_off", "mb_samples", "mb_tokens", "mb_lmax", "mb_residual", "mb_cost", "mb_bucket", "mb_rank",
+             "rank_mb_off", "rank_mbs", "sample_cost", "sample_mb")
+
+
+def expected_row(w, s, p):
+    """Row of position p of sample s, from the generator (oracle side; no CUDA library involved)."""
+    pos, tok = w.spans_of(s)
+    for j in range(len(pos)):
+        if int(pos[j]) <= p < int(pos[j]) + int(tok[j]):
+            r = p - int(pos[j])
+            v = workloads.span_values(w, s, j, device="cpu", rows=(r, r + 1))
+            if w.src_dtype == 0:
+                return bits16(v).ravel()
+            return np.array([f32_to_bf16_rne(int(b)) for b in bits32(v).ravel()], dtype=np.uint16)
+    i = int(workloads.input_ids(w, s)[p])
+    return bits16(workloads.embed_table(w, "cpu", rows=(i, i + 1))).ravel()
+
+
+@pytest.mark.parametrize("name,kw", [("image_mix_7b", {}), ("video_heavy", {})])
+def test_full_size_plan_and_sampled_rows(name, kw):
+    if not torch.cuda.is_available():
+        pytest.fail("a CUDA device is required for -m gpu tests")
+    from gpu_harness import CudaRun
+    w = workloads.make_workload(name, **kw)
+    run = CudaRun(w)
+    for call in w.write_calls:
+        samples = sorted({s for s, _ in call}, key=[s for s, _ in call].index)
+        assert run.register(samples) == 0
+        assert run.write(call, keep_src=False) == 0
+    rc, plan = run.plan()
+    assert rc == 0
+    got = plan.arrays()
+    rc, oplan = plan_from_lengths(w.seq_len[w.plan_order], PlanConfig(**plan_config_fields(w)), slots=w.plan_order)
+    assert rc == 0
+    exp = oplan.arrays()
+    for k in PLAN_KEYS:
+        assert np.array_equal(got[k], exp[k]), k
+    assert plan.summary() == oplan.summary()
+    rc, out, cu, pos = run.gather_all()
+    assert rc == 0 and run.pool.status() == (0, 0)
+    # what the plan arrays determine about cu_seqlens / position ids (numpy only)
+    lens = w.seq_len[exp["mb_samples"]].astype(np.int64)
+    exp_pos = np.concatenate([np.arange(l, dtype=np.int32) for l in lens])
+    assert np.array_equal(pos.cpu().numpy(), exp_pos)
+    exp_cu = []
+    for j in range(exp["n_mb"]):
+        a, b = int(exp["mb_sample_off"][j]), int(exp["mb_sample_off"][j + 1])
+        exp_cu.append(np.concatenate([[0], np.cumsum(lens[a:b])]))
+    assert np.array_equal(cu.cpu().numpy(), np.concatenate(exp_cu).astype(np.int32))
+    # sampled rows, including each sample's first/last rows and span boundaries
+    row_off = np.concatenate([[0], np.cumsum(lens)])
+    rng = np.random.default_rng(11)
+    picks = []
+    for q in rng.choice(len(lens), size=24, replace=False):
+        s = int(exp["mb_samples"][q])
+        sp, st = w.spans_of(s)
+        cand = {0, int(lens[q]) - 1, int(rng.integers(0, lens[q]))}
+        j = int(rng.integers(0, len(sp)))
+        cand |= {int(sp[j]), int(sp[j]) + int(st[j]) - 1, min(int(lens[q]) - 1, int(sp[j]) + int(st[j]))}
+        if int(sp[j]) > 0:
+            cand.add(int(sp[j]) - 1)
+        picks += [(q, s, p) for p in sorted(cand)]
+    rows = torch.tensor([int(row_off[q]) + p for q, s, p in picks], device="cuda")
+    got_rows = out[rows].cpu().numpy().view(np.uint16)
+    for i, (q, s, p) in enumerate(picks):
+        assert np.array_equal(got_rows[i], expected_row(w, s, p)), (q, s, p)
+    # no row left at poison anywhere (checked on the device)
+    assert not bool((out == -1).all(dim=1).any().item())
+    oplan.destroy()
+    run.close()
