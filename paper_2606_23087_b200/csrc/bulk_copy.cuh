@@ -42,18 +42,10 @@ constexpr int kBulkDepth = 8;              // loads in flight
 constexpr uint32_t kBulkStageBytes = 16384;
 constexpr uint32_t kBulkSpinLimit = 20000000;  // mbarrier polls before a copy is declared lost
 
-// fp32 -> bf16 on bit patterns: IEEE round-to-nearest-even, denormals kept, NaN -> sign | 0x7FC0
-__device__ __forceinline__ uint32_t bulk_rne_bf16(uint32_t u) {
-  if ((u & 0x7FFFFFFFu) > 0x7F800000u) return ((u >> 16) & 0x8000u) | 0x7FC0u;
-  return (u + 0x7FFFu + ((u >> 16) & 1u)) >> 16;
-}
-
 // Warp-wide copy pipeline: every lane of a one-warp CTA calls push()/drain() with the same arguments; lane 0
 // issues the asynchronous operations.  Copy number i goes into stage i % kBulkStages; before that, copy
-// i - kBulkDepth is retired (wait for its load, optionally cast it in place, start its store).  A stage is
-// reused only after the store that last read it has finished reading shared memory.
-// CAST: the staged bytes are fp32 and the stored bytes their bf16 image (half as many).
-template <bool CAST>
+// i - kBulkDepth is retired (wait for its load, start its store).  A stage is reused only after the store
+// that last read it has finished reading shared memory.
 struct BulkRing {
   uint8_t* stage;    // kBulkStages * kBulkStageBytes of shared memory, 128-byte aligned
   uint64_t* bar;     // kBulkStages mbarriers
@@ -87,31 +79,13 @@ struct BulkRing {
     bad = __shfl_sync(0xFFFFFFFFu, bad, 0);
     if (bad) { lost = true; return; }
     uint8_t* sp = stage + (size_t)st * kBulkStageBytes;
-    uint32_t len = len_q[st];
-    if (CAST) {
-      // in place: lane t of round r reads floats [4t, 4t+4) and writes bf16 [4t, 4t+4); a round's writes land
-      // below every later round's reads, and inside a round all reads come before all writes
-      const uint32_t nvec = len >> 4;
-      for (uint32_t t0 = 0; t0 < nvec; t0 += 32) {
-        const uint32_t t = t0 + lane;
-        uint4 f = make_uint4(0, 0, 0, 0);
-        if (t < nvec) f = reinterpret_cast<const uint4*>(sp)[t];
-        __syncwarp();
-        if (t < nvec)
-          reinterpret_cast<uint2*>(sp)[t] = make_uint2(bulk_rne_bf16(f.x) | (bulk_rne_bf16(f.y) << 16),
-                                                       bulk_rne_bf16(f.z) | (bulk_rne_bf16(f.w) << 16));
-        __syncwarp();
-      }
-      len >>= 1;
-      fence_async_smem();  // the cast's generic-proxy writes must be visible to the bulk store
-      __syncwarp();
-    }
+    const uint32_t len = len_q[st];
     if (lane == 0) {
       bulk_s2g(reinterpret_cast<void*>(dst_q[st]), sp, len);
       bulk_commit();
     }
   }
-  // bytes staged: multiple of 16 (32 with CAST), <= kBulkStageBytes; src and dst 16-byte aligned
+  // bytes: multiple of 16, <= kBulkStageBytes; src and dst 16-byte aligned
   __device__ void push(const void* src, void* dst, uint32_t bytes) {
     if (lost) return;
     if (issued - retired >= (uint64_t)kBulkDepth) retire_one();

@@ -157,7 +157,7 @@ __global__ void __launch_bounds__(32) k_gather_host_bulk(PoolView v, PlanView pl
   __shared__ uint64_t dst_q[kBulkStages];
   __shared__ uint32_t len_q[kBulkStages];
   const uint32_t lane = threadIdx.x;
-  BulkRing<false> ring;
+  BulkRing ring;
   ring.init(smem, bars, dst_q, len_q);
   uint64_t item = 0;
   for (uint32_t q = a.q_lo; q < a.q_hi; ++q) {

@@ -7,6 +7,7 @@
 //   k_alloc_scan       pages/list blocks/chunks per span -> exclusive scans, ring pops
 //   k_alloc_fill       span page lists (two-level) from consecutive ring entries
 //   k_scatter          the producer byte copy into pages, optional fused fp32->bf16 RNE cast
+//   k_scatter_host_bulk  bf16 sources into host-tier pages by bulk-async copies
 //   k_free_scan/_fill  pages, list blocks and text pages back to the ring tails
 #include <algorithm>
 #include <cstdio>
@@ -251,9 +252,11 @@ enum { kTierAll = 0, kTierDeviceOnly = 1, kTierHostOnly = 2 };
 
 template <int MODE, bool F32>
 __global__ void __launch_bounds__(256, 8) k_scatter(PoolView v, WriteCall c, uint64_t total_chunks, uint64_t per_cta) {
-  const uint64_t c0 = (uint64_t)blockIdx.x * per_cta;
+  // groups of per_cta consecutive chunks are dealt round-robin over the CTAs: at any moment the grid streams
+  // one contiguous window of the call's bytes
+  const uint64_t CH = 1ull << c.chunk_shift;
+  for (uint64_t c0 = (uint64_t)blockIdx.x * per_cta; c0 < total_chunks; c0 += (uint64_t)gridDim.x * per_cta) {
   const uint64_t c1 = min(total_chunks, c0 + per_cta);
-  if (c0 >= c1) return;
   uint32_t lo = 0, hi = c.n;  // largest q with chunk_off[q] <= c0
   while (hi - lo > 1) {
     uint32_t mid = (lo + hi) >> 1;
@@ -266,7 +269,6 @@ __global__ void __launch_bounds__(256, 8) k_scatter(PoolView v, WriteCall c, uin
   uint32_t sid = c.span_id[q];
   uint32_t cached_o = kNone;
   uint64_t pte = 0;
-  const uint64_t CH = 1ull << c.chunk_shift;
   for (uint64_t ch = c0; ch < c1; ++ch) {
     while (ch >= q_end) {
       ++q;
@@ -291,12 +293,22 @@ __global__ void __launch_bounds__(256, 8) k_scatter(PoolView v, WriteCall c, uin
       const uint4* s = reinterpret_cast<const uint4*>(src_q + b0);
       uint4* d = reinterpret_cast<uint4*>(dst);
       const uint32_t nv = len >> 4;
-      uint32_t x = threadIdx.x;
-      for (; x + 3 * 256 < nv; x += 4 * 256) {
-        uint4 a0 = __ldcs(s + x), a1 = __ldcs(s + x + 256), a2 = __ldcs(s + x + 512), a3 = __ldcs(s + x + 768);
-        __stcs(d + x, a0); __stcs(d + x + 256, a1); __stcs(d + x + 512, a2); __stcs(d + x + 768, a3);
+      // warp w streams its own contiguous eighth of the chunk, 2 KiB (four 512-byte lines) in flight at a time
+      const uint32_t wv = (uint32_t)(CH >> 7);  // vectors per warp region
+      const uint32_t xw = (threadIdx.x >> 5) * wv + (threadIdx.x & 31);
+      for (uint32_t b = 0; b < wv; b += 128) {
+        const uint32_t x = xw + b;
+        uint4 a0, a1, a2, a3;
+        const bool t0 = b < wv && x < nv, t1 = b + 32 < wv && x + 32 < nv, t2 = b + 64 < wv && x + 64 < nv, t3 = b + 96 < wv && x + 96 < nv;
+        if (t0) a0 = __ldcs(s + x);
+        if (t1) a1 = __ldcs(s + x + 32);
+        if (t2) a2 = __ldcs(s + x + 64);
+        if (t3) a3 = __ldcs(s + x + 96);
+        if (t0) __stcs(d + x, a0);
+        if (t1) __stcs(d + x + 32, a1);
+        if (t2) __stcs(d + x + 64, a2);
+        if (t3) __stcs(d + x + 96, a3);
       }
-      for (; x < nv; x += 256) __stcs(d + x, __ldcs(s + x));
     } else {
       const uint4* s = reinterpret_cast<const uint4*>(src_q + 2 * b0);  // 2 source vectors per destination vector
       uint4* d = reinterpret_cast<uint4*>(dst);
@@ -314,22 +326,21 @@ __global__ void __launch_bounds__(256, 8) k_scatter(PoolView v, WriteCall c, uin
       }
     }
   }
+  }
 }
 
 
-// Host-tier pages of a producer call, page by page: source bytes -> shared -> host frame with bulk copies (the
-// fp32 source is cast in shared memory on the way).  One warp per CTA; lanes translate 32 page ordinals at a
-// time, lane 0 drives the ring; a handful of CTAs saturate the host link.
-template <bool F32>
+// Host-tier pages of a producer call (bf16 source), page by page: source bytes -> shared -> host frame with
+// bulk copies.  One warp per CTA; lanes translate 32 page ordinals at a time, lane 0 drives the ring; a
+// handful of CTAs saturate the host link.
 __global__ void __launch_bounds__(32) k_scatter_host_bulk(PoolView v, WriteCall c, uint64_t call_seq) {
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ uint64_t bars[kBulkStages];
   __shared__ uint64_t dst_q[kBulkStages];
   __shared__ uint32_t len_q[kBulkStages];
   const uint32_t lane = threadIdx.x;
-  BulkRing<F32> ring;
+  BulkRing ring;
   ring.init(smem, bars, dst_q, len_q);
-  constexpr uint32_t kOutPiece = F32 ? kBulkStageBytes / 2 : kBulkStageBytes;  // destination bytes per staged copy
   uint64_t item = 0;
   for (uint32_t q = 0; q < c.n; ++q) {
     const uint32_t sid = c.span_id[q];
@@ -349,10 +360,8 @@ __global__ void __launch_bounds__(32) k_scatter_host_bulk(PoolView v, WriteCall 
         const uint64_t b0 = (uint64_t)(g + l) << v.page_shift;  // destination byte offset inside the span image
         const uint64_t len = min(v.page_bytes, nbytes - b0);
         uint8_t* dst = reinterpret_cast<uint8_t*>(p_l & ~kPteFlagMask);
-        for (uint64_t x = 0; x < len; x += kOutPiece) {
-          const uint32_t out_bytes = (uint32_t)min((uint64_t)kOutPiece, len - x);
-          ring.push(src_q + (F32 ? 2 : 1) * (b0 + x), dst + x, F32 ? 2 * out_bytes : out_bytes);
-        }
+        for (uint64_t x = 0; x < len; x += kBulkStageBytes)
+          ring.push(src_q + b0 + x, dst + x, (uint32_t)min((uint64_t)kBulkStageBytes, len - x));
       }
     }
   }
@@ -521,6 +530,8 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_create(const ft_p
   CK(cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, p->device));
   p->host_ctas = 8;
   if (const char* e = getenv("FLOWPOOL_HOST_CTAS")) { int v = atoi(e); if (v > 0) p->host_ctas = v; }
+  if (const char* e = getenv("FLOWPOOL_CHUNK_SHIFT")) { int v = atoi(e); if (v >= 12 && v <= 21) p->chunk_shift = v; }
+  if (const char* e = getenv("FLOWPOOL_SCATTER_GROUP")) { int v = atoi(e); if (v >= 0) p->scatter_group = v; }
   if (const char* e = getenv("FLOWPOOL_DEV_CTAS_PER_SM")) { int v = atoi(e); if (v > 0) p->dev_ctas_per_sm = v; }
   CK(cudaStreamCreateWithFlags(&p->side_stream, cudaStreamNonBlocking));
   CK(cudaEventCreateWithFlags(&p->fork_ev, cudaEventDisableTiming));
@@ -731,7 +742,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings(
   const ft_pool_config& c = p->cfg;
   const uint32_t S = c.max_spans_per_sample;
   uint64_t need = 0, need_blocks = 0, total_chunks = 0, bytes_total = 0;
-  const uint32_t chunk_shift = std::min<uint32_t>(p->view.page_shift, 14);
+  const uint32_t chunk_shift = std::min<uint32_t>(p->view.page_shift, p->chunk_shift);
   std::vector<uint32_t> span_id(n);
   {
     std::unordered_set<uint32_t> named;
@@ -792,8 +803,8 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings(
     const bool host_class = mode == kTierHostOnly || (mode == kTierAll && c.hbm_pages == 0);
     prof_begin(p, host_class ? FT_K_SCATTER_HOST : FT_K_SCATTER_DEVICE, s);
     uint64_t grid = std::min<uint64_t>(total_chunks, host_class ? (uint64_t)p->host_ctas : (uint64_t)p->sm_count * p->dev_ctas_per_sm);
-    uint64_t per = (total_chunks + grid - 1) / grid;
-    grid = (total_chunks + per - 1) / per;
+    uint64_t per = p->scatter_group ? (uint64_t)p->scatter_group : (total_chunks + grid - 1) / grid;
+    grid = std::min<uint64_t>(grid, (total_chunks + per - 1) / per);
     if (mode == kTierAll) { if (f32) k_scatter<kTierAll, true><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); else k_scatter<kTierAll, false><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); }
     else if (mode == kTierDeviceOnly) { if (f32) k_scatter<kTierDeviceOnly, true><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); else k_scatter<kTierDeviceOnly, false><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); }
     else { if (f32) k_scatter<kTierHostOnly, true><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); else k_scatter<kTierHostOnly, false><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); }
@@ -809,13 +820,19 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings(
     FT_CUDA(cudaStreamWaitEvent(p->side_stream, p->fork_ev, 0));
     static bool attr_set = false;
     if (!attr_set) {
-      FT_CUDA(cudaFuncSetAttribute(k_scatter_host_bulk<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBulkSmemBytes));
-      FT_CUDA(cudaFuncSetAttribute(k_scatter_host_bulk<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBulkSmemBytes));
+      FT_CUDA(cudaFuncSetAttribute(k_scatter_host_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBulkSmemBytes));
       attr_set = true;
     }
     prof_begin(p, FT_K_SCATTER_HOST, p->side_stream);
-    if (f32) k_scatter_host_bulk<true><<<(unsigned)p->host_ctas, 32, kBulkSmemBytes, p->side_stream>>>(p->view, w, p->call_seq);
-    else k_scatter_host_bulk<false><<<(unsigned)p->host_ctas, 32, kBulkSmemBytes, p->side_stream>>>(p->view, w, p->call_seq);
+    // bf16 source: bulk-async copies through shared memory.  fp32 source: the cast needs the values in
+    // registers, and stores to host memory are posted (no latency to hide), so a few vector-store CTAs do it
+    if (f32) {
+      uint64_t grid = std::min<uint64_t>(total_chunks, (uint64_t)p->host_ctas);
+      uint64_t per = p->scatter_group ? (uint64_t)p->scatter_group : (total_chunks + grid - 1) / grid;
+      k_scatter<kTierHostOnly, true><<<(unsigned)grid, 256, 0, p->side_stream>>>(p->view, w, total_chunks, per);
+    } else {
+      k_scatter_host_bulk<<<(unsigned)p->host_ctas, 32, kBulkSmemBytes, p->side_stream>>>(p->view, w, p->call_seq);
+    }
     prof_end(p, p->side_stream);
     p->gpu_launches++;
     FT_CUDA(cudaEventRecord(p->join_ev, p->side_stream));
@@ -1045,7 +1062,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings_
   if (cur != p->device) return FT_ERR_INVALID_ARG;
   const ft_pool_config& c = p->cfg;
   const uint32_t S = c.max_spans_per_sample;
-  const uint32_t chunk_shift = std::min<uint32_t>(p->view.page_shift, 14);
+  const uint32_t chunk_shift = std::min<uint32_t>(p->view.page_shift, p->chunk_shift);
   uint64_t need = 0, need_blocks = 0, total_chunks = 0, bytes_total = 0;
 
   // descriptor blob on the stack: [src u64 n][span_id n][n_tokens n]; duplicate check in a fixed hash table
@@ -1113,8 +1130,8 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings_
   auto launch = [&](int mode, cudaStream_t s) {
     const bool host_class = mode == kTierAll && c.hbm_pages == 0;
     uint64_t grid = std::min<uint64_t>(total_chunks, host_class ? (uint64_t)p->host_ctas : (uint64_t)p->sm_count * p->dev_ctas_per_sm);
-    uint64_t per = (total_chunks + grid - 1) / grid;
-    grid = (total_chunks + per - 1) / per;
+    uint64_t per = p->scatter_group ? (uint64_t)p->scatter_group : (total_chunks + grid - 1) / grid;
+    grid = std::min<uint64_t>(grid, (total_chunks + per - 1) / per);
     if (mode == kTierAll) { if (f32) k_scatter<kTierAll, true><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); else k_scatter<kTierAll, false><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); }
     else { if (f32) k_scatter<kTierDeviceOnly, true><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); else k_scatter<kTierDeviceOnly, false><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); }
     p->gpu_launches++;
@@ -1122,12 +1139,16 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings_
   if (c.host_pages == 0 || c.hbm_pages == 0) {
     launch(kTierAll, st);
   } else {
-    FT_CUDA(cudaFuncSetAttribute(k_scatter_host_bulk<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBulkSmemBytes));
-    FT_CUDA(cudaFuncSetAttribute(k_scatter_host_bulk<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBulkSmemBytes));
+    FT_CUDA(cudaFuncSetAttribute(k_scatter_host_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBulkSmemBytes));
     FT_CUDA(cudaEventRecord(p->fork_ev, st));
     FT_CUDA(cudaStreamWaitEvent(p->side_stream, p->fork_ev, 0));
-    if (f32) k_scatter_host_bulk<true><<<(unsigned)p->host_ctas, 32, kBulkSmemBytes, p->side_stream>>>(p->view, w, p->call_seq);
-    else k_scatter_host_bulk<false><<<(unsigned)p->host_ctas, 32, kBulkSmemBytes, p->side_stream>>>(p->view, w, p->call_seq);
+    if (f32) {
+      uint64_t grid = std::min<uint64_t>(total_chunks, (uint64_t)p->host_ctas);
+      uint64_t per = p->scatter_group ? (uint64_t)p->scatter_group : (total_chunks + grid - 1) / grid;
+      k_scatter<kTierHostOnly, true><<<(unsigned)grid, 256, 0, p->side_stream>>>(p->view, w, total_chunks, per);
+    } else {
+      k_scatter_host_bulk<<<(unsigned)p->host_ctas, 32, kBulkSmemBytes, p->side_stream>>>(p->view, w, p->call_seq);
+    }
     p->gpu_launches++;
     FT_CUDA(cudaEventRecord(p->join_ev, p->side_stream));
     launch(kTierDeviceOnly, st);
