@@ -253,6 +253,27 @@ class DeviceJob:
         self.pool.destroy()
 
 
+def measure_host_link(torch, nbytes=1 << 30, reps=5):
+    """Host-link reference rates: plain cudaMemcpyAsync between pinned host memory and the device, best of reps."""
+    try:
+        h = torch.empty(nbytes, dtype=torch.uint8, pin_memory=True)
+        d = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    except RuntimeError:
+        return None
+    res = {}
+    for name, (dst, src) in (("h2d_gbs", (d, h)), ("d2h_gbs", (h, d))):
+        best = 0.0
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            dst.copy_(src, non_blocking=True)
+            e1.record()
+            torch.cuda.synchronize()
+            best = max(best, nbytes / e0.elapsed_time(e1) / 1e6)
+        res[name] = best
+    return res
+
+
 def max_over_ranks(ms, dist, device="cuda"):
     """A multi-rank time is the slowest rank's."""
     if dist is None:
@@ -425,6 +446,14 @@ def run_ours(args):
     value = aggregate_value(wb + gb, world, ms)
     kern, host_b = kernel_breakdown(job, prof, args.steps)
     phases = phase_breakdown(job)
+    link = measure_host_link(torch) if (w.host_pages and rank == 0) else None
+    if link:
+        # bytes that cross the link per step: host-tier vision bytes, once per direction
+        for k, ref in (("gather_host", "h2d_gbs"), ("scatter_host", "d2h_gbs")):
+            ms_k = kern[k]["ms_per_step"]
+            if ms_k > 0:
+                kern[k]["link_gbs"] = host_b / ms_k / 1e6
+                kern[k]["link_frac_of_memcpy"] = kern[k]["link_gbs"] / link[ref]
 
     line = None
     if rank == 0:
@@ -448,7 +477,7 @@ def run_ours(args):
                        "host_pages": w.host_pages, "host_tier_bytes": host_b,
                        "l2": "inputs larger than L2 (no flush needed)", "parallelism": f"dp{world} (independent batches)"},
             "tokens_per_s": world * w.total_tokens / ms * 1e3,
-            "gpu_launches": launches, "kernels": kern, "phase_ms": phases, "roofline": roofline, "clocks": clocks,
+            "gpu_launches": launches, "kernels": kern, "phase_ms": phases, "host_link_memcpy": link, "roofline": roofline, "clocks": clocks,
         }
     # all-HBM variant of the same batch (the benchmark spec's target is stated for HBM-resident pools)
     if not args.all_hbm and not args.skip_variants:
@@ -481,6 +510,122 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+# ---------------------------------------------------------------------------------------------
+# scale + fragmentation sweep (one page size per invocation)
+# ---------------------------------------------------------------------------------------------
+def run_sweep(args):
+    """Config 5: a stream of samples flows through a fixed-capacity pool (10 x {admit while it fits, free a
+    seeded half}, final admit), then the residents are planned and gathered.  Prints one JSON line with the
+    gather/write bandwidth, plan time, fragmentation and packing figures for the given page size."""
+    import torch
+    import workloads
+    from harness import pool_config_fields, plan_config_fields, register_args, write_args
+    from paper_2606_23087_b200 import binding as fp
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    st = torch.cuda.current_stream().cuda_stream
+    PS = args.page_bytes
+    w = workloads.make_workload("frag_sweep", n_samples=args.samples or 65536, page_bytes=PS,
+                                pool_bytes=int(args.pool_gib * (1 << 30)))
+    ops, residents = workloads.admit_free_schedule(w, cycles=args.cycles)
+    pool = fp.Pool(fp.PoolConfig(**pool_config_fields(w)))
+    if pool.rc != 0:
+        raise fp.FlowpoolError(pool.rc, "pool_create")
+    pool.profile_enable(True)
+    written_vis = 0
+    consumed = 0
+    for kind, samples in ops:
+        if kind == "free":
+            rc = pool.free(samples, st)
+            assert rc == 0, rc
+            continue
+        consumed += len(samples)
+        for i in range(0, len(samples), 256):
+            part = samples[i:i + 256]
+            reg = register_args(w, part)
+            ids = torch.from_numpy(reg[5]).cuda()
+            srcs = [workloads.span_values(w, s, 0, device="cuda") for s in part]
+            assert pool.register_samples(*reg[:5], ids.data_ptr(), st) == 0
+            rc = pool.write_embeddings(*write_args(w, [(s, 0) for s in part]), [t.data_ptr() for t in srcs], 0, st)
+            assert rc == 0, rc
+            torch.cuda.synchronize()
+            written_vis += int(sum(int(w.spans_of(s)[1][0]) for s in part))
+    prof_w = pool.profile_read()
+    write_ms = prof_w["scatter_device"]["ms"]
+    stats = pool.stats()
+    # plan the residents (admission order)
+    order = np.asarray(residents, dtype=np.uint32)
+    pcfg = fp.PlanConfig(**plan_config_fields(w))
+    plan_ms = []
+    plan = None
+    for _ in range(3):
+        if plan:
+            plan.destroy()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        rc, plan = pool.plan_microbatches(order, pcfg, st)
+        plan_ms.append((time.perf_counter() - t0) * 1e3)
+        assert rc == 0, rc
+    a = plan.arrays()
+    n_mb, total_tokens, _ = plan.summary()
+    # gather everything, in ranges that fit a reusable output buffer
+    table = workloads.embed_table(w, device="cuda")
+    buf_rows = min(total_tokens, 1 << 20)
+    out = torch.empty((buf_rows, w.hidden), dtype=torch.bfloat16, device="cuda")
+    cu = torch.empty((len(residents) + n_mb + 8,), dtype=torch.int32, device="cuda")
+    pos = torch.empty((buf_rows,), dtype=torch.int32, device="cuda")
+    ranges, b, rows = [], 0, 0
+    for j in range(n_mb):
+        t = int(a["mb_tokens"][j])
+        if rows + t > buf_rows:
+            ranges.append((b, j)); b, rows = j, 0
+        rows += t
+    ranges.append((b, n_mb))
+    gather_ms = None
+    for rep in range(3):
+        pool.profile_read()
+        for lo, hi in ranges:
+            rc = pool.gather_packed(plan, lo, hi, table.data_ptr(), w.vocab, out.data_ptr(), cu.data_ptr(), pos.data_ptr(), st)
+            assert rc == 0, rc
+        g = pool.profile_read()["gather_device"]
+        gather_ms = g["ms"] if gather_ms is None else min(gather_ms, g["ms"])
+    assert pool.status() == (0, 0)
+    # planner scale: every descriptor of the stream, metadata only (needs free slots: use a second pool)
+    plan.destroy()
+    # fragmentation figures
+    need_bytes = sum(int(w.spans_of(s)[1][0]) * w.row_bytes for s in residents)
+    used_pages = stats["pages_total"] - stats["pages_free"]
+    runs = []
+    for s in residents[:: max(1, len(residents) // 200)]:
+        pg = pool.span_pages(s, 0, cap=1 << 16)[1].astype(np.int64)
+        if len(pg) > 1:
+            brk = int((np.diff(pg) != PS).sum())
+            runs.append(len(pg) / (brk + 1))
+        elif len(pg) == 1:
+            runs.append(1.0)
+    loads = np.array([a["mb_cost"][a["mb_rank"] == r].astype(np.float64).sum() for r in range(w.n_ranks_N)])
+    row_b = w.row_bytes
+    peak, peak_src = measured_peak()
+    gbs = 2 * total_tokens * row_b / gather_ms / 1e6
+    line = {
+        "metric": "packed-microbatch assembly GB/s after churn (fragmentation sweep)", "value": gbs, "unit": "GB/s",
+        "n_gpus": 1, "higher_is_better": True, "dtype": "u8", "data": "synthetic",
+        "config": {"workload": f"frag_sweep: stream of {w.n_samples} samples, hidden {w.hidden}, page {PS} B, pool "
+                               f"{args.pool_gib} GiB all HBM, {args.cycles} write/free cycles, budget {w.budget_L}",
+                   "page_bytes": PS},
+        "residents": len(residents), "stream_consumed": consumed, "packed_tokens": int(total_tokens), "microbatches": n_mb,
+        "gather_ms": gather_ms, "gather_launches": len(ranges), "frac_of_measured_peak": gbs / peak,
+        "write_gbs": 2 * written_vis * row_b / write_ms / 1e6, "write_ms_total": write_ms,
+        "plan_ms_host_wall_median": float(np.median(plan_ms)),
+        "internal_fragmentation": 1.0 - need_bytes / (used_pages * PS),
+        "mean_contiguous_run_pages": float(np.mean(runs)) if runs else None,
+        "padding_waste": 1.0 - total_tokens / (n_mb * w.budget_L),
+        "rank_imbalance": float((loads.max() - loads.min()) / loads.mean()),
+        "gpu_launches": pool.stats()["gpu_launches"],
+    }
+    pool.destroy()
+    print(json.dumps(line))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -493,10 +638,15 @@ def main():
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-cpu", action="store_true")
     ap.add_argument("--skip-variants", action="store_true")
+    ap.add_argument("--page-bytes", type=int, default=2 << 20, help="frag_sweep: page size")
+    ap.add_argument("--pool-gib", type=float, default=64.0, help="frag_sweep: pool capacity")
+    ap.add_argument("--cycles", type=int, default=10, help="frag_sweep: write/free cycles")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload == "frag_sweep":
+        run_sweep(args)
     else:
         run_ours(args)
 

@@ -224,9 +224,9 @@ struct ft_pool {
   int host_ctas = 8;            // grid of the host-tier copy kernels: few SMs, so that long-latency host-link
                                 // accesses do not clog the memory pipelines of the SMs that stream HBM
                                 // (FLOWPOOL_HOST_CTAS overrides)
-  int chunk_shift = 16;         // log2 of k_scatter's work unit in destination bytes (capped by the page size)
+  int chunk_shift = 16;         // log2 of k_scatter's work unit in bytes of a span's image
   int scatter_group = 4;        // chunks per round-robin group of k_scatter (0 = one static range per CTA)
-  int dev_ctas_per_sm = 8;      // resident CTAs per SM of the device-tier copy kernels
+  int dev_ctas_per_sm = 8;      // resident CTAs per SM of the device-tier gather kernel
   // optional kernel timing (pool_profile_*)
   bool profiling = false;
   struct prof_rec { int kind; cudaEvent_t e0, e1; };

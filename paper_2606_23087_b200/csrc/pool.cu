@@ -185,7 +185,7 @@ struct WriteCall {
   uint32_t* blk_off;         // [n+1] out
   uint64_t* chunk_off;       // [n+1] out
   uint32_t* heads;           // [2]   out: page ring head, block ring head before the pops
-  uint32_t chunk_shift;      // scatter work unit = 2^chunk_shift destination bytes, never straddles a page
+  uint32_t chunk_shift;      // scatter work unit = 2^chunk_shift bytes of a span's image
 };
 
 __global__ void __launch_bounds__(1024) k_alloc_scan(PoolView v, WriteCall c) {
@@ -251,84 +251,103 @@ __device__ __forceinline__ uint32_t pack2(uint32_t a, uint32_t b) { return rne_b
 enum { kTierAll = 0, kTierDeviceOnly = 1, kTierHostOnly = 2 };
 
 template <int MODE, bool F32>
-__global__ void __launch_bounds__(256, 8) k_scatter(PoolView v, WriteCall c, uint64_t total_chunks, uint64_t per_cta) {
-  // groups of per_cta consecutive chunks are dealt round-robin over the CTAs: at any moment the grid streams
-  // one contiguous window of the call's bytes
+__global__ void __launch_bounds__(256, F32 ? 4 : 6) k_scatter(PoolView v, WriteCall c, uint64_t total_chunks, uint64_t per_cta) {
+  // Work unit = a chunk of 2^chunk_shift bytes of one span's image (the page size does not cap it).  Groups of
+  // per_cta consecutive chunks are dealt round-robin over the CTAs, so at any moment the grid streams one
+  // contiguous window of the call's bytes.  Inside a chunk warp w owns the w-th eighth and walks it in 2 KiB
+  // batches (four 512-byte lines per lane in flight); a batch never straddles a page (pages are >= 4 KiB and
+  // batches 2 KiB-aligned), and each warp resolves its batch's frame through the span's page list and the
+  // page table, once per page.
+  const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const uint64_t CH = 1ull << c.chunk_shift;
+  const uint32_t region = (uint32_t)(CH >> 3);  // bytes per warp and chunk
   for (uint64_t c0 = (uint64_t)blockIdx.x * per_cta; c0 < total_chunks; c0 += (uint64_t)gridDim.x * per_cta) {
-  const uint64_t c1 = min(total_chunks, c0 + per_cta);
-  uint32_t lo = 0, hi = c.n;  // largest q with chunk_off[q] <= c0
-  while (hi - lo > 1) {
-    uint32_t mid = (lo + hi) >> 1;
-    if (c.chunk_off[mid] <= c0) lo = mid; else hi = mid;
-  }
-  uint32_t q = lo;
-  uint64_t q_end = c.chunk_off[q + 1], q_begin = c.chunk_off[q];
-  uint64_t bytes_q = (uint64_t)c.n_tokens[q] * v.row_bytes;
-  const uint8_t* src_q = reinterpret_cast<const uint8_t*>(c.src[q]);
-  uint32_t sid = c.span_id[q];
-  uint32_t cached_o = kNone;
-  uint64_t pte = 0;
-  for (uint64_t ch = c0; ch < c1; ++ch) {
-    while (ch >= q_end) {
-      ++q;
-      q_begin = q_end; q_end = c.chunk_off[q + 1];
-      bytes_q = (uint64_t)c.n_tokens[q] * v.row_bytes;
-      src_q = reinterpret_cast<const uint8_t*>(c.src[q]);
-      sid = c.span_id[q];
-      cached_o = kNone;
+    const uint64_t c1 = min(total_chunks, c0 + per_cta);
+    uint32_t lo = 0, hi = c.n;  // largest q with chunk_off[q] <= c0
+    while (hi - lo > 1) {
+      uint32_t mid = (lo + hi) >> 1;
+      if (c.chunk_off[mid] <= c0) lo = mid; else hi = mid;
     }
-    const uint64_t b0 = (ch - q_begin) << c.chunk_shift;  // byte offset inside the span image
-    const uint32_t o = (uint32_t)(b0 >> v.page_shift);
-    if (o != cached_o) {
-      uint64_t off;
-      pte = translate(v, span_page_gva(v, sid, o), &off);
-      cached_o = o;
-    }
-    const bool host = (pte & kPteHost) != 0;
-    if ((MODE == kTierDeviceOnly && host) || (MODE == kTierHostOnly && !host)) continue;
-    uint8_t* dst = reinterpret_cast<uint8_t*>(pte & ~kPteFlagMask) + (b0 & (v.page_bytes - 1));
-    const uint32_t len = (uint32_t)min(CH, bytes_q - b0);
-    if (!F32) {
-      const uint4* s = reinterpret_cast<const uint4*>(src_q + b0);
-      uint4* d = reinterpret_cast<uint4*>(dst);
-      const uint32_t nv = len >> 4;
-      // warp w streams its own contiguous eighth of the chunk, 2 KiB (four 512-byte lines) in flight at a time
-      const uint32_t wv = (uint32_t)(CH >> 7);  // vectors per warp region
-      const uint32_t xw = (threadIdx.x >> 5) * wv + (threadIdx.x & 31);
-      for (uint32_t b = 0; b < wv; b += 128) {
-        const uint32_t x = xw + b;
-        uint4 a0, a1, a2, a3;
-        const bool t0 = b < wv && x < nv, t1 = b + 32 < wv && x + 32 < nv, t2 = b + 64 < wv && x + 64 < nv, t3 = b + 96 < wv && x + 96 < nv;
-        if (t0) a0 = __ldcs(s + x);
-        if (t1) a1 = __ldcs(s + x + 32);
-        if (t2) a2 = __ldcs(s + x + 64);
-        if (t3) a3 = __ldcs(s + x + 96);
-        if (t0) __stcs(d + x, a0);
-        if (t1) __stcs(d + x + 32, a1);
-        if (t2) __stcs(d + x + 64, a2);
-        if (t3) __stcs(d + x + 96, a3);
+    uint32_t q = lo;
+    uint64_t q_end = c.chunk_off[q + 1], q_begin = c.chunk_off[q];
+    uint64_t bytes_q = (uint64_t)c.n_tokens[q] * v.row_bytes;
+    const uint8_t* src_q = reinterpret_cast<const uint8_t*>(c.src[q]);
+    uint32_t sid = c.span_id[q];
+    uint32_t cached_o = kNone;
+    uint64_t pte = 0;
+    for (uint64_t ch = c0; ch < c1; ++ch) {
+      while (ch >= q_end) {
+        ++q;
+        q_begin = q_end; q_end = c.chunk_off[q + 1];
+        bytes_q = (uint64_t)c.n_tokens[q] * v.row_bytes;
+        src_q = reinterpret_cast<const uint8_t*>(c.src[q]);
+        sid = c.span_id[q];
+        cached_o = kNone;
       }
-    } else {
-      const uint4* s = reinterpret_cast<const uint4*>(src_q + 2 * b0);  // 2 source vectors per destination vector
-      uint4* d = reinterpret_cast<uint4*>(dst);
-      const uint32_t nv = len >> 4;
-      uint32_t x = threadIdx.x;
-      for (; x + 256 < nv; x += 2 * 256) {
-        uint4 a0 = __ldcs(s + 2 * x), a1 = __ldcs(s + 2 * x + 1);
-        uint4 b0v = __ldcs(s + 2 * (x + 256)), b1v = __ldcs(s + 2 * (x + 256) + 1);
-        __stcs(d + x, make_uint4(pack2(a0.x, a0.y), pack2(a0.z, a0.w), pack2(a1.x, a1.y), pack2(a1.z, a1.w)));
-        __stcs(d + x + 256, make_uint4(pack2(b0v.x, b0v.y), pack2(b0v.z, b0v.w), pack2(b1v.x, b1v.y), pack2(b1v.z, b1v.w)));
-      }
-      for (; x < nv; x += 256) {
-        uint4 a0 = __ldcs(s + 2 * x), a1 = __ldcs(s + 2 * x + 1);
-        __stcs(d + x, make_uint4(pack2(a0.x, a0.y), pack2(a0.z, a0.w), pack2(a1.x, a1.y), pack2(a1.z, a1.w)));
+      const uint64_t b0 = ((ch - q_begin) << c.chunk_shift) + (uint64_t)warp * region;  // this warp's span offset
+      for (uint32_t b = 0; b < region; b += 2048) {
+        const uint64_t B = b0 + b;
+        if (B >= bytes_q) break;
+        const uint32_t o = (uint32_t)(B >> v.page_shift);
+        if (o != cached_o) {
+          uint64_t off;
+          pte = translate(v, span_page_gva(v, sid, o), &off);
+          cached_o = o;
+        }
+        const bool host = (pte & kPteHost) != 0;
+        if ((MODE == kTierDeviceOnly && host) || (MODE == kTierHostOnly && !host)) continue;
+        uint4* d = reinterpret_cast<uint4*>((pte & ~kPteFlagMask) + (B & (v.page_bytes - 1)));
+        const uint32_t nv = (uint32_t)(min((uint64_t)2048, bytes_q - B) >> 4);  // vectors in this batch (<= 128)
+        const bool t0 = lane < nv, t1 = lane + 32 < nv, t2 = lane + 64 < nv, t3 = lane + 96 < nv;
+        if (!F32) {
+          const uint4* s = reinterpret_cast<const uint4*>(src_q + B);
+          uint4 a0, a1, a2, a3;
+          if (t0) a0 = __ldcs(s + lane);
+          if (t1) a1 = __ldcs(s + lane + 32);
+          if (t2) a2 = __ldcs(s + lane + 64);
+          if (t3) a3 = __ldcs(s + lane + 96);
+          if (t0) __stcs(d + lane, a0);
+          if (t1) __stcs(d + lane + 32, a1);
+          if (t2) __stcs(d + lane + 64, a2);
+          if (t3) __stcs(d + lane + 96, a3);
+        } else {
+          const uint4* s = reinterpret_cast<const uint4*>(src_q + 2 * B);  // two fp32 vectors per bf16 vector
+          uint4 a0, a1, a2, a3, e0, e1, e2, e3;
+          if (t0) { a0 = __ldcs(s + 2 * lane); e0 = __ldcs(s + 2 * lane + 1); }
+          if (t1) { a1 = __ldcs(s + 2 * (lane + 32)); e1 = __ldcs(s + 2 * (lane + 32) + 1); }
+          if (t2) { a2 = __ldcs(s + 2 * (lane + 64)); e2 = __ldcs(s + 2 * (lane + 64) + 1); }
+          if (t3) { a3 = __ldcs(s + 2 * (lane + 96)); e3 = __ldcs(s + 2 * (lane + 96) + 1); }
+          if (t0) __stcs(d + lane, make_uint4(pack2(a0.x, a0.y), pack2(a0.z, a0.w), pack2(e0.x, e0.y), pack2(e0.z, e0.w)));
+          if (t1) __stcs(d + lane + 32, make_uint4(pack2(a1.x, a1.y), pack2(a1.z, a1.w), pack2(e1.x, e1.y), pack2(e1.z, e1.w)));
+          if (t2) __stcs(d + lane + 64, make_uint4(pack2(a2.x, a2.y), pack2(a2.z, a2.w), pack2(e2.x, e2.y), pack2(e2.z, e2.w)));
+          if (t3) __stcs(d + lane + 96, make_uint4(pack2(a3.x, a3.y), pack2(a3.z, a3.w), pack2(e3.x, e3.y), pack2(e3.z, e3.w)));
+        }
       }
     }
-  }
   }
 }
 
+
+// launches k_scatter<MODE, F32> on a grid of at most `max_ctas` CTAs, never more than fit on the GPU at once
+// (the round-robin deal assumes every CTA runs from the start)
+template <int MODE, bool F32>
+static void launch_scatter(ft_pool* p, const WriteCall& w, uint64_t total_chunks, uint64_t max_ctas, cudaStream_t s) {
+  static int per_sm = 0;
+  if (per_sm == 0) {
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_scatter<MODE, F32>, 256, 0) != cudaSuccess || per_sm < 1) per_sm = 1;
+  }
+  uint64_t grid = std::min<uint64_t>(max_ctas, (uint64_t)p->sm_count * per_sm);
+  const uint64_t per = p->scatter_group > 0 ? (uint64_t)p->scatter_group : 1;
+  grid = std::max<uint64_t>(1, std::min<uint64_t>(grid, (total_chunks + per - 1) / per));
+  k_scatter<MODE, F32><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per);
+}
+
+static void launch_scatter_any(ft_pool* p, int mode, bool f32, const WriteCall& w, uint64_t total_chunks, uint64_t max_ctas,
+                               cudaStream_t s) {
+  if (mode == kTierAll) { if (f32) launch_scatter<kTierAll, true>(p, w, total_chunks, max_ctas, s); else launch_scatter<kTierAll, false>(p, w, total_chunks, max_ctas, s); }
+  else if (mode == kTierDeviceOnly) { if (f32) launch_scatter<kTierDeviceOnly, true>(p, w, total_chunks, max_ctas, s); else launch_scatter<kTierDeviceOnly, false>(p, w, total_chunks, max_ctas, s); }
+  else { if (f32) launch_scatter<kTierHostOnly, true>(p, w, total_chunks, max_ctas, s); else launch_scatter<kTierHostOnly, false>(p, w, total_chunks, max_ctas, s); }
+}
 
 // Host-tier pages of a producer call (bf16 source), page by page: source bytes -> shared -> host frame with
 // bulk copies.  One warp per CTA; lanes translate 32 page ordinals at a time, lane 0 drives the ring; a
@@ -742,7 +761,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings(
   const ft_pool_config& c = p->cfg;
   const uint32_t S = c.max_spans_per_sample;
   uint64_t need = 0, need_blocks = 0, total_chunks = 0, bytes_total = 0;
-  const uint32_t chunk_shift = std::min<uint32_t>(p->view.page_shift, p->chunk_shift);
+  const uint32_t chunk_shift = (uint32_t)p->chunk_shift;
   std::vector<uint32_t> span_id(n);
   {
     std::unordered_set<uint32_t> named;
@@ -802,12 +821,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings(
   auto launch = [&](int mode, cudaStream_t s) {
     const bool host_class = mode == kTierHostOnly || (mode == kTierAll && c.hbm_pages == 0);
     prof_begin(p, host_class ? FT_K_SCATTER_HOST : FT_K_SCATTER_DEVICE, s);
-    uint64_t grid = std::min<uint64_t>(total_chunks, host_class ? (uint64_t)p->host_ctas : (uint64_t)p->sm_count * p->dev_ctas_per_sm);
-    uint64_t per = p->scatter_group ? (uint64_t)p->scatter_group : (total_chunks + grid - 1) / grid;
-    grid = std::min<uint64_t>(grid, (total_chunks + per - 1) / per);
-    if (mode == kTierAll) { if (f32) k_scatter<kTierAll, true><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); else k_scatter<kTierAll, false><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); }
-    else if (mode == kTierDeviceOnly) { if (f32) k_scatter<kTierDeviceOnly, true><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); else k_scatter<kTierDeviceOnly, false><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); }
-    else { if (f32) k_scatter<kTierHostOnly, true><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); else k_scatter<kTierHostOnly, false><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); }
+    launch_scatter_any(p, mode, f32, w, total_chunks, host_class ? (uint64_t)p->host_ctas : ~0ull, s);
     prof_end(p, s);
     p->gpu_launches++;
   };
@@ -827,9 +841,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings(
     // bf16 source: bulk-async copies through shared memory.  fp32 source: the cast needs the values in
     // registers, and stores to host memory are posted (no latency to hide), so a few vector-store CTAs do it
     if (f32) {
-      uint64_t grid = std::min<uint64_t>(total_chunks, (uint64_t)p->host_ctas);
-      uint64_t per = p->scatter_group ? (uint64_t)p->scatter_group : (total_chunks + grid - 1) / grid;
-      k_scatter<kTierHostOnly, true><<<(unsigned)grid, 256, 0, p->side_stream>>>(p->view, w, total_chunks, per);
+      launch_scatter<kTierHostOnly, true>(p, w, total_chunks, (uint64_t)p->host_ctas, p->side_stream);
     } else {
       k_scatter_host_bulk<<<(unsigned)p->host_ctas, 32, kBulkSmemBytes, p->side_stream>>>(p->view, w, p->call_seq);
     }
@@ -1062,7 +1074,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings_
   if (cur != p->device) return FT_ERR_INVALID_ARG;
   const ft_pool_config& c = p->cfg;
   const uint32_t S = c.max_spans_per_sample;
-  const uint32_t chunk_shift = std::min<uint32_t>(p->view.page_shift, p->chunk_shift);
+  const uint32_t chunk_shift = (uint32_t)p->chunk_shift;
   uint64_t need = 0, need_blocks = 0, total_chunks = 0, bytes_total = 0;
 
   // descriptor blob on the stack: [src u64 n][span_id n][n_tokens n]; duplicate check in a fixed hash table
@@ -1129,11 +1141,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings_
   const bool f32 = src_dtype == FT_F32;
   auto launch = [&](int mode, cudaStream_t s) {
     const bool host_class = mode == kTierAll && c.hbm_pages == 0;
-    uint64_t grid = std::min<uint64_t>(total_chunks, host_class ? (uint64_t)p->host_ctas : (uint64_t)p->sm_count * p->dev_ctas_per_sm);
-    uint64_t per = p->scatter_group ? (uint64_t)p->scatter_group : (total_chunks + grid - 1) / grid;
-    grid = std::min<uint64_t>(grid, (total_chunks + per - 1) / per);
-    if (mode == kTierAll) { if (f32) k_scatter<kTierAll, true><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); else k_scatter<kTierAll, false><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); }
-    else { if (f32) k_scatter<kTierDeviceOnly, true><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); else k_scatter<kTierDeviceOnly, false><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per); }
+    launch_scatter_any(p, mode, f32, w, total_chunks, host_class ? (uint64_t)p->host_ctas : ~0ull, s);
     p->gpu_launches++;
   };
   if (c.host_pages == 0 || c.hbm_pages == 0) {
@@ -1143,9 +1151,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings_
     FT_CUDA(cudaEventRecord(p->fork_ev, st));
     FT_CUDA(cudaStreamWaitEvent(p->side_stream, p->fork_ev, 0));
     if (f32) {
-      uint64_t grid = std::min<uint64_t>(total_chunks, (uint64_t)p->host_ctas);
-      uint64_t per = p->scatter_group ? (uint64_t)p->scatter_group : (total_chunks + grid - 1) / grid;
-      k_scatter<kTierHostOnly, true><<<(unsigned)grid, 256, 0, p->side_stream>>>(p->view, w, total_chunks, per);
+      launch_scatter<kTierHostOnly, true>(p, w, total_chunks, (uint64_t)p->host_ctas, p->side_stream);
     } else {
       k_scatter_host_bulk<<<(unsigned)p->host_ctas, 32, kBulkSmemBytes, p->side_stream>>>(p->view, w, p->call_seq);
     }
