@@ -225,8 +225,10 @@ struct ft_pool {
                                 // accesses do not clog the memory pipelines of the SMs that stream HBM
                                 // (FLOWPOOL_HOST_CTAS overrides)
   int chunk_shift = 16;         // log2 of k_scatter's work unit in bytes of a span's image
-  int scatter_group = 4;        // chunks per round-robin group of k_scatter (0 = one static range per CTA)
-  int dev_ctas_per_sm = 8;      // resident CTAs per SM of the device-tier gather kernel
+  int scatter_group = 0;        // chunks per round-robin group of k_scatter; 0 = the measured default
+  int scatter_ctas_per_sm = 0;  // resident CTAs per SM of the device-tier scatter kernel; 0 = the measured default
+  int gather_unroll = 4;        // 16-byte vectors per lane in flight in k_gather (4 or 8)
+  int dev_ctas_per_sm = 4;      // resident CTAs per SM of the device-tier gather kernel (measured optimum 3-5)
   // optional kernel timing (pool_profile_*)
   bool profiling = false;
   struct prof_rec { int kind; cudaEvent_t e0, e1; };

@@ -7,6 +7,7 @@
 // vectors.  Rows that straddle pages carry one address per page touched.  With a two-tier pool the
 // kernel is launched twice, once per tier, so host-link reads never stall HBM reads.
 #include <algorithm>
+#include <cstdlib>
 
 #include "bulk_copy.cuh"
 #include "flowpool_internal.cuh"
@@ -37,16 +38,24 @@ struct GatherArgs {
   int32_t* pos_ids;
   uint64_t call_seq;
   uint32_t write_index;  // this launch writes cu_seqlens / position ids
+  unsigned long long* tile_counter;  // device, zero at launch
 };
 
-template <int MODE>
+template <int MODE, int U>
 __global__ void __launch_bounds__(kGatherThreads) k_gather(PoolView v, PlanView pl, GatherArgs a) {
   __shared__ RowDesc desc[kTileRows];
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const uint64_t tile_lo = a.row_lo / kTileRows, tile_hi = (a.row_hi + kTileRows - 1) / kTileRows;
   const uint32_t row_vecs = v.row_bytes >> 4;
 
-  for (uint64_t tile = tile_lo + blockIdx.x; tile < tile_hi; tile += gridDim.x) {
+  __shared__ uint64_t next_tile;
+  for (;;) {
+    // tiles are claimed in order from a device counter (zeroed by the host before the launch): the CTAs in
+    // flight always cover one compact window of the output, and uneven tiles balance themselves
+    if (threadIdx.x == 0) next_tile = tile_lo + atomicAdd(a.tile_counter, 1ull);
+    __syncthreads();
+    const uint64_t tile = next_tile;
+    if (tile >= tile_hi) break;
     if (warp == 0) {
       const uint64_t row = tile * kTileRows + lane;
       RowDesc d;
@@ -123,9 +132,7 @@ __global__ void __launch_bounds__(kGatherThreads) k_gather(PoolView v, PlanView 
         *take = MODE == kTierAll || (MODE == kTierHostOnly) == host;
         return reinterpret_cast<const uint4*>((pte & ~kPteFlagMask) + (ab & mask));
       };
-      // U vectors per lane in flight before the first store: 4 for HBM frames; 16 for host frames, whose
-      // reads cross the host link with microseconds of latency and need far more bytes outstanding
-      constexpr int U = MODE == kTierHostOnly ? 16 : 4;
+      // U vectors per lane in flight before the first store
       for (uint32_t x0 = lane; x0 < row_vecs; x0 += 32 * U) {
         uint4 val[U];
         bool take[U];
@@ -224,13 +231,22 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_gather_packed(ft_
   a.table = static_cast<const uint8_t*>(embed_table); a.vocab = vocab;
   a.out = static_cast<uint8_t*>(out_embeds); a.cu = out_cu; a.pos_ids = out_pos;
   a.call_seq = p->call_seq; a.write_index = 1;
+  a.tile_counter = p->view.status + 1;  // scratch word next to the status word
+  FT_CUDA(cudaMemsetAsync(a.tile_counter, 0, 8, static_cast<cudaStream_t>(stream)));
   const uint64_t n_tiles = (a.row_hi + kTileRows - 1) / kTileRows - a.row_lo / kTileRows;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  auto grid_for = [&](uint64_t ctas) { return (unsigned)std::min<uint64_t>(n_tiles, ctas); };
-  const uint64_t dev_ctas = (uint64_t)p->sm_count * p->dev_ctas_per_sm, host_ctas = p->host_ctas;
+  // the grid-stride tile loop assumes every CTA runs from the start: never launch more than fit at once
+  auto launch = [&](auto kernel, uint64_t want_per_sm, const GatherArgs& args, cudaStream_t s) {
+    int resident = 1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, kernel, kGatherThreads, 0) != cudaSuccess || resident < 1) resident = 1;
+    const uint64_t ctas = (uint64_t)p->sm_count * std::min<uint64_t>(want_per_sm, (uint64_t)resident);
+    kernel<<<(unsigned)std::min<uint64_t>(n_tiles, ctas), kGatherThreads, 0, s>>>(p->view, pv, args);
+  };
+  const uint64_t per_sm = p->cfg.hbm_pages == 0 ? 1 : (uint64_t)p->dev_ctas_per_sm;
+  const bool u8 = p->gather_unroll == 8;
   if (p->cfg.host_pages == 0 || p->cfg.hbm_pages == 0) {
     prof_begin(p, p->cfg.hbm_pages == 0 ? FT_K_GATHER_HOST : FT_K_GATHER_DEVICE, st);
-    k_gather<kTierAll><<<grid_for(p->cfg.hbm_pages == 0 ? host_ctas : dev_ctas), kGatherThreads, 0, st>>>(p->view, pv, a);
+    if (u8) launch(k_gather<kTierAll, 8>, per_sm, a, st); else launch(k_gather<kTierAll, 4>, per_sm, a, st);
     prof_end(p, st);
     p->gpu_launches += 1;
   } else {
@@ -238,17 +254,17 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_gather_packed(ft_
     FT_CUDA(cudaStreamWaitEvent(p->side_stream, p->fork_ev, 0));
     GatherArgs ah = a;
     ah.write_index = 0;
-    prof_begin(p, FT_K_GATHER_HOST, p->side_stream);
     static bool attr_set = false;
     if (!attr_set) {
       FT_CUDA(cudaFuncSetAttribute(k_gather_host_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBulkSmemBytes));
       attr_set = true;
     }
-    k_gather_host_bulk<<<(unsigned)host_ctas, 32, kBulkSmemBytes, p->side_stream>>>(p->view, pv, ah);
+    prof_begin(p, FT_K_GATHER_HOST, p->side_stream);
+    k_gather_host_bulk<<<(unsigned)p->host_ctas, 32, kBulkSmemBytes, p->side_stream>>>(p->view, pv, ah);
     prof_end(p, p->side_stream);
     FT_CUDA(cudaEventRecord(p->join_ev, p->side_stream));
     prof_begin(p, FT_K_GATHER_DEVICE, st);
-    k_gather<kTierDeviceOnly><<<grid_for(dev_ctas), kGatherThreads, 0, st>>>(p->view, pv, a);
+    if (u8) launch(k_gather<kTierDeviceOnly, 8>, per_sm, a, st); else launch(k_gather<kTierDeviceOnly, 4>, per_sm, a, st);
     prof_end(p, st);
     FT_CUDA(cudaStreamWaitEvent(st, p->join_ev, 0));
     p->gpu_launches += 2;

@@ -184,6 +184,7 @@ struct WriteCall {
   uint32_t* page_off;        // [n+1] out
   uint32_t* blk_off;         // [n+1] out
   uint64_t* chunk_off;       // [n+1] out
+  uint32_t* chunk_span;      // [total chunks] out: call-local span index of each chunk; NULL = search chunk_off
   uint32_t* heads;           // [2]   out: page ring head, block ring head before the pops
   uint32_t chunk_shift;      // scatter work unit = 2^chunk_shift bytes of a span's image
 };
@@ -209,6 +210,7 @@ __global__ void __launch_bounds__(1024) k_alloc_scan(PoolView v, WriteCall c) {
   }
   if (threadIdx.x == 0) {
     c.page_off[c.n] = (uint32_t)cp; c.blk_off[c.n] = (uint32_t)cb; c.chunk_off[c.n] = cc;
+    v.status[2] = 0; v.status[3] = 0;  // k_scatter's claim counters (main and side stream) start at zero
     RingState s = *v.ring_state;
     c.heads[0] = s.head;
     s.head = (uint32_t)((s.head + cp) % v.ring_cap); s.count -= (uint32_t)cp;
@@ -221,9 +223,18 @@ __global__ void __launch_bounds__(1024) k_alloc_scan(PoolView v, WriteCall c) {
 }
 
 // one thread per allocated page: span q takes ring entries [page_off[q], page_off[q+1]) after the head
-__global__ void __launch_bounds__(256) k_alloc_fill(PoolView v, WriteCall c, uint32_t total_pages) {
-  const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
-  if (t >= total_pages) return;
+__global__ void __launch_bounds__(256) k_alloc_fill(PoolView v, WriteCall c, uint32_t total_pages, uint64_t total_chunks) {
+  const uint64_t tc = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (c.chunk_span && tc < total_chunks) {  // which span of the call does chunk tc belong to
+    uint32_t lo = 0, hi = c.n;
+    while (hi - lo > 1) {
+      uint32_t mid = (lo + hi) >> 1;
+      if (c.chunk_off[mid] <= tc) lo = mid; else hi = mid;
+    }
+    c.chunk_span[tc] = lo;
+  }
+  if (tc >= total_pages) return;
+  const uint32_t t = (uint32_t)tc;
   uint32_t lo = 0, hi = c.n;  // largest q with page_off[q] <= t
   while (hi - lo > 1) {
     uint32_t mid = (lo + hi) >> 1;
@@ -251,24 +262,36 @@ __device__ __forceinline__ uint32_t pack2(uint32_t a, uint32_t b) { return rne_b
 enum { kTierAll = 0, kTierDeviceOnly = 1, kTierHostOnly = 2 };
 
 template <int MODE, bool F32>
-__global__ void __launch_bounds__(256, F32 ? 4 : 6) k_scatter(PoolView v, WriteCall c, uint64_t total_chunks, uint64_t per_cta) {
+__global__ void __launch_bounds__(256, F32 ? 4 : 6) k_scatter(PoolView v, WriteCall c, uint64_t total_chunks, uint64_t per_cta,
+                                                              unsigned long long* group_counter) {
   // Work unit = a chunk of 2^chunk_shift bytes of one span's image (the page size does not cap it).  Groups of
-  // per_cta consecutive chunks are dealt round-robin over the CTAs, so at any moment the grid streams one
-  // contiguous window of the call's bytes.  Inside a chunk warp w owns the w-th eighth and walks it in 2 KiB
+  // per_cta consecutive chunks are claimed in order from a device counter (zeroed before the launch), so at
+  // any moment the grid streams one compact window of the call's bytes.  Inside a chunk warp w owns the w-th eighth and walks it in 2 KiB
   // batches (four 512-byte lines per lane in flight); a batch never straddles a page (pages are >= 4 KiB and
   // batches 2 KiB-aligned), and each warp resolves its batch's frame through the span's page list and the
   // page table, once per page.
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const uint64_t CH = 1ull << c.chunk_shift;
   const uint32_t region = (uint32_t)(CH >> 3);  // bytes per warp and chunk
-  for (uint64_t c0 = (uint64_t)blockIdx.x * per_cta; c0 < total_chunks; c0 += (uint64_t)gridDim.x * per_cta) {
+  __shared__ uint64_t next_group;
+  for (;;) {
+    __syncthreads();  // everyone has read the previous claim
+    if (threadIdx.x == 0) next_group = atomicAdd(group_counter, 1ull);
+    __syncthreads();
+    const uint64_t c0 = next_group * per_cta;
+    if (c0 >= total_chunks) break;
     const uint64_t c1 = min(total_chunks, c0 + per_cta);
-    uint32_t lo = 0, hi = c.n;  // largest q with chunk_off[q] <= c0
-    while (hi - lo > 1) {
-      uint32_t mid = (lo + hi) >> 1;
-      if (c.chunk_off[mid] <= c0) lo = mid; else hi = mid;
+    uint32_t q;
+    if (c.chunk_span) {
+      q = c.chunk_span[c0];
+    } else {
+      uint32_t lo = 0, hi = c.n;  // largest q with chunk_off[q] <= c0
+      while (hi - lo > 1) {
+        uint32_t mid = (lo + hi) >> 1;
+        if (c.chunk_off[mid] <= c0) lo = mid; else hi = mid;
+      }
+      q = lo;
     }
-    uint32_t q = lo;
     uint64_t q_end = c.chunk_off[q + 1], q_begin = c.chunk_off[q];
     uint64_t bytes_q = (uint64_t)c.n_tokens[q] * v.row_bytes;
     const uint8_t* src_q = reinterpret_cast<const uint8_t*>(c.src[q]);
@@ -332,14 +355,20 @@ __global__ void __launch_bounds__(256, F32 ? 4 : 6) k_scatter(PoolView v, WriteC
 // (the round-robin deal assumes every CTA runs from the start)
 template <int MODE, bool F32>
 static void launch_scatter(ft_pool* p, const WriteCall& w, uint64_t total_chunks, uint64_t max_ctas, cudaStream_t s) {
+  // one claim counter per stream the library launches on: main (word 2) and side (word 3) of the status block
+  // (k_alloc_scan, which precedes every scatter launch of the call, zeroes them)
+  unsigned long long* counter = p->view.status + (s == p->side_stream ? 3 : 2);
   static int per_sm = 0;
   if (per_sm == 0) {
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_scatter<MODE, F32>, 256, 0) != cudaSuccess || per_sm < 1) per_sm = 1;
   }
-  uint64_t grid = std::min<uint64_t>(max_ctas, (uint64_t)p->sm_count * per_sm);
+  // HBM streams best with a bounded amount of loads in flight per SM; more resident warps only deepen the DRAM
+  // queues (measured optimum: 4 CTAs/SM, one chunk per claim)
+  const int want = p->scatter_ctas_per_sm > 0 ? p->scatter_ctas_per_sm : 4;
+  uint64_t grid = std::min<uint64_t>(max_ctas, (uint64_t)p->sm_count * std::min(per_sm, want));
   const uint64_t per = p->scatter_group > 0 ? (uint64_t)p->scatter_group : 1;
   grid = std::max<uint64_t>(1, std::min<uint64_t>(grid, (total_chunks + per - 1) / per));
-  k_scatter<MODE, F32><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per);
+  k_scatter<MODE, F32><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per, counter);
 }
 
 static void launch_scatter_any(ft_pool* p, int mode, bool f32, const WriteCall& w, uint64_t total_chunks, uint64_t max_ctas,
@@ -550,7 +579,9 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_create(const ft_p
   p->host_ctas = 8;
   if (const char* e = getenv("FLOWPOOL_HOST_CTAS")) { int v = atoi(e); if (v > 0) p->host_ctas = v; }
   if (const char* e = getenv("FLOWPOOL_CHUNK_SHIFT")) { int v = atoi(e); if (v >= 12 && v <= 21) p->chunk_shift = v; }
-  if (const char* e = getenv("FLOWPOOL_SCATTER_GROUP")) { int v = atoi(e); if (v >= 0) p->scatter_group = v; }
+  if (const char* e = getenv("FLOWPOOL_SCATTER_GROUP")) { int v = atoi(e); if (v > 0) p->scatter_group = v; }
+  if (const char* e = getenv("FLOWPOOL_SCATTER_CTAS_PER_SM")) { int v = atoi(e); if (v > 0) p->scatter_ctas_per_sm = v; }
+  if (const char* e = getenv("FLOWPOOL_GATHER_U")) { int v = atoi(e); if (v == 4 || v == 8) p->gather_unroll = v; }
   if (const char* e = getenv("FLOWPOOL_DEV_CTAS_PER_SM")) { int v = atoi(e); if (v > 0) p->dev_ctas_per_sm = v; }
   CK(cudaStreamCreateWithFlags(&p->side_stream, cudaStreamNonBlocking));
   CK(cudaEventCreateWithFlags(&p->fork_ev, cudaEventDisableTiming));
@@ -582,7 +613,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_create(const ft_p
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
   const size_t o_pte_hbm = take(c.hbm_pages * 8), o_pte_host = take(c.host_pages * 8), o_pte_text = take(n_text * 8);
   const size_t o_ring = take(P * 4), o_tring = take(n_text * 4), o_bring = take(NB * 4);
-  const size_t o_states = take(3 * sizeof(RingState)), o_status = take(8);
+  const size_t o_states = take(3 * sizeof(RingState)), o_status = take(32);  // status word, the gather's tile counter, the scatter's claim counters
   const size_t o_seq = take((size_t)c.max_samples * 4), o_nsp = take((size_t)c.max_samples * 4);
   const size_t o_stp = take((size_t)c.max_samples * TPS * 4);
   const size_t o_pos = take(span_ids * 4), o_tok = take(span_ids * 4), o_npg = take(span_ids * 4);
@@ -792,7 +823,8 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings(
   const size_t blob_bytes = align_up(o_ntk + (size_t)n * 4, 256);
   const size_t o_choff = blob_bytes, o_poff = align_up(o_choff + (size_t)(n + 1) * 8, 16);
   const size_t o_boff = o_poff + (size_t)(n + 1) * 4, o_heads = align_up(o_boff + (size_t)(n + 1) * 4, 16);
-  const size_t total_bytes = o_heads + 16;
+  const size_t o_cspan = o_heads + 16;
+  const size_t total_bytes = o_cspan + total_chunks * 4;
   std::vector<uint8_t> blob(blob_bytes, 0);
   for (uint32_t q = 0; q < n; ++q) reinterpret_cast<uint64_t*>(blob.data())[q] = reinterpret_cast<uint64_t>(src[q]);
   memcpy(blob.data() + o_sid, span_id.data(), (size_t)n * 4);
@@ -811,9 +843,10 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings(
   w.page_off = reinterpret_cast<uint32_t*>(db + o_poff);
   w.blk_off = reinterpret_cast<uint32_t*>(db + o_boff);
   w.heads = reinterpret_cast<uint32_t*>(db + o_heads);
+  w.chunk_span = reinterpret_cast<uint32_t*>(db + o_cspan);
   w.chunk_shift = chunk_shift;
   k_alloc_scan<<<1, 1024, 0, st>>>(p->view, w);
-  k_alloc_fill<<<(unsigned)((need + 255) / 256), 256, 0, st>>>(p->view, w, (uint32_t)need);
+  k_alloc_fill<<<(unsigned)((std::max<uint64_t>(need, total_chunks) + 255) / 256), 256, 0, st>>>(p->view, w, (uint32_t)need, total_chunks);
   p->gpu_launches += 2;
 
   // the byte copy: HBM-bound chunks on the caller's stream, host-bound chunks beside them
@@ -1133,9 +1166,10 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings_
   w.page_off = reinterpret_cast<uint32_t*>(db + o_poff);
   w.blk_off = reinterpret_cast<uint32_t*>(db + o_boff);
   w.heads = reinterpret_cast<uint32_t*>(db + o_heads);
+  w.chunk_span = nullptr;  // the fixed scratch has no room for a per-chunk table: k_scatter searches chunk_off
   w.chunk_shift = chunk_shift;
   k_alloc_scan<<<1, 1024, 0, st>>>(p->view, w);
-  k_alloc_fill<<<(unsigned)((need + 255) / 256), 256, 0, st>>>(p->view, w, (uint32_t)need);
+  k_alloc_fill<<<(unsigned)((need + 255) / 256), 256, 0, st>>>(p->view, w, (uint32_t)need, 0);
   p->gpu_launches += 2;
 
   const bool f32 = src_dtype == FT_F32;
