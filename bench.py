@@ -31,9 +31,9 @@ METRIC = "packed-microbatch assembly throughput (producer scatter + plan + packe
 UNIT = "GB/s"
 CPU_SAMPLE = 256         # samples of the workload the oracle is timed on (about 10-30 s of CPU work)
 # dram__bytes_read.sum + dram__bytes_write.sum over algorithmic bytes for one k_gather launch, from the ncu capture
-# summarised in profiles/k_gather_image_mix_7b_64samples_all_hbm.md (4.599 GB / 4.698 GB on the first 64 samples);
+# summarised in profiles/k_gather_image_mix_7b_64samples_all_hbm.md (4.592 GB / 4.698 GB on the first 64 samples);
 # traffic grows in proportion to the tokens assembled, so a full launch is this ratio times its algorithmic bytes
-NCU_TRAFFIC_RATIO_GATHER = 0.979
+NCU_TRAFFIC_RATIO_GATHER = 0.977
 
 
 def algorithmic_bytes(w):
