@@ -233,6 +233,8 @@ int32_t plan_arrays(const ft_plan* plan, uint32_t* mb_sample_off, uint32_t* mb_s
                     uint32_t* rank_mb_off, uint32_t* rank_mbs, uint64_t* sample_cost,
                     uint32_t* sample_mb);
 
+/* Releases the plan.  Its device block is freed in stream order after the plan's latest work (no device-wide
+ * synchronisation); the handle is invalid on return. */
 int32_t plan_destroy(ft_plan* plan);
 
 /*

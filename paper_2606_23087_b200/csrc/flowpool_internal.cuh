@@ -161,7 +161,8 @@ struct ft_plan {
   std::vector<uint64_t> slot_generation;
   std::vector<uint32_t> h_mb_sample_off;  // host copies used to size gathers
   std::vector<uint64_t> h_mb_row_off;
-  void* d_block = nullptr;                // one allocation holding every array below
+  void* d_block = nullptr;                // one stream-ordered allocation holding every array below
+  cudaStream_t last_stream = nullptr;     // stream of the plan's latest device work (creation, then gathers)
   uint32_t *d_slots, *d_len, *d_sample_mb, *d_sample_rank, *d_mb_sample_off, *d_mb_samples, *d_plan_sample_mb;
   uint32_t *d_mb_tokens, *d_mb_lmax, *d_mb_residual, *d_mb_count, *d_mb_bucket, *d_mb_rank, *d_mb_pos;
   uint32_t *d_rank_mb_off, *d_rank_mbs, *d_rank_cnt, *d_tile_first_sample, *d_scalars;

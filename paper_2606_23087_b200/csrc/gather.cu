@@ -269,6 +269,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_gather_packed(ft_
     FT_CUDA(cudaStreamWaitEvent(st, p->join_ev, 0));
     p->gpu_launches += 2;
   }
+  const_cast<ft_plan*>(pl)->last_stream = st;
   FT_CUDA(cudaGetLastError());
   p->bytes_gathered += (a.row_hi - a.row_lo) * 2ull * p->view.row_bytes;
   return FT_OK;

@@ -291,7 +291,8 @@ using namespace ft;
 
 extern "C" __attribute__((visibility("default"))) int32_t plan_destroy(ft_plan* pl) {
   if (!pl) return FT_ERR_INVALID_ARG;
-  if (pl->d_block) { cudaDeviceSynchronize(); cudaFree(pl->d_block); }
+  // stream-ordered free: the block is released after the plan's last kernel, with no device-wide synchronisation
+  if (pl->d_block && cudaFreeAsync(pl->d_block, pl->last_stream) != cudaSuccess) { cudaGetLastError(); cudaDeviceSynchronize(); cudaFree(pl->d_block); }
   delete pl;
   return FT_OK;
 }
@@ -347,7 +348,16 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_plan_microbatches
   const size_t o_bkt = take(n * 4), o_rank = take(n * 4), o_pos = take(n * 4), o_idx = take(n * 4);
   const size_t o_roff = take(((size_t)N + 1) * 4), o_rmbs = take(n * 4), o_rcnt = take((size_t)N * 4);
   const size_t o_tiles = take(n_tiles * 4), o_scal = take(SC_COUNT * 4);
-  cudaError_t e = cudaMalloc(&pl->d_block, off);
+  static bool pool_tuned = false;
+  if (!pool_tuned) {  // keep freed plan blocks cached in the device's default memory pool instead of returning them
+    cudaMemPool_t mp;
+    uint64_t keep = ~0ull;
+    if (cudaDeviceGetDefaultMemPool(&mp, p->device) == cudaSuccess) cudaMemPoolSetAttribute(mp, cudaMemPoolAttrReleaseThreshold, &keep);
+    cudaGetLastError();
+    pool_tuned = true;
+  }
+  pl->last_stream = st;
+  cudaError_t e = cudaMallocAsync(&pl->d_block, off, st);
   if (e != cudaSuccess) { delete pl; return ft::cuda_fail(e, "cudaMalloc(plan)"); }
   uint8_t* b = static_cast<uint8_t*>(pl->d_block);
 #define U32(o) reinterpret_cast<uint32_t*>(b + (o))
