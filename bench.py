@@ -615,6 +615,20 @@ def run_sweep(args):
         assert rc == 0, rc
     a = plan.arrays()
     n_mb, total_tokens, _ = plan.summary()
+    # scheduler variants on the same residents: what each buys in padding waste and rank balance
+    variants = {}
+    for name, fl in (("as_printed", 0), ("longest_first", 2), ("sum_of_squares", 4), ("carried_zigzag", 8), ("all_three", 14)):
+        vc = plan_config_fields(w, flags=fl)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        rc, vp = pool.plan_microbatches(order, fp.PlanConfig(**vc), st)
+        dt = (time.perf_counter() - t0) * 1e3
+        assert rc == 0, rc
+        va = vp.arrays()
+        vl = np.array([va["mb_cost"][va["mb_rank"] == r].astype(np.float64).sum() for r in range(w.n_ranks_N)])
+        variants[name] = {"microbatches": int(va["n_mb"]), "padding_waste": 1.0 - total_tokens / (int(va["n_mb"]) * w.budget_L),
+                          "rank_imbalance": float((vl.max() - vl.min()) / vl.mean()), "plan_ms_host_wall": dt}
+        vp.destroy()
     # gather everything, in ranges that fit a reusable output buffer
     table = workloads.embed_table(w, device="cuda")
     buf_rows = min(total_tokens, 1 << 20)
@@ -668,6 +682,7 @@ def run_sweep(args):
         "mean_contiguous_run_pages": float(np.mean(runs)) if runs else None,
         "padding_waste": 1.0 - total_tokens / (n_mb * w.budget_L),
         "rank_imbalance": float((loads.max() - loads.min()) / loads.mean()),
+        "plan_variants": variants,
         "gpu_launches": pool.stats()["gpu_launches"],
     }
     pool.destroy()

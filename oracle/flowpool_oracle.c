@@ -41,7 +41,8 @@ enum {
 enum { OR_RING_SORTED = 0, OR_RING_SHUFFLED = 1 };
 enum { OR_BIND_IDENTITY = 0, OR_BIND_PERMUTED = 1 };
 enum { OR_BF16 = 0, OR_F32 = 1 };
-enum { OR_PLAN_ALLOW_UNWRITTEN = 1 };
+/* plan flags; the last three are variants at points where the paper is silent or could be read otherwise */
+enum { OR_PLAN_ALLOW_UNWRITTEN = 1, OR_PLAN_SORT_DECREASING = 2, OR_PLAN_COST_SUMSQ = 4, OR_PLAN_ZIGZAG_CARRY = 8 };
 enum { SLOT_FREE = 0, SLOT_REGISTERED = 1, SLOT_READY = 2 };
 
 #define TEXT_PAGE_BYTES 4096u /* reading: token ids live in 4 KiB text pages */
@@ -579,7 +580,7 @@ uint64_t oracle_cost_int(uint64_t A, uint64_t B, uint64_t sum_len, uint64_t lmax
 
 /* Two-dimension load balancing, Algorithm 1 lines 12-27, on given costs.
  * Outputs: bucket[n_mb], rank[n_mb], rank_mb_off[N+1], rank_mbs[n_mb]. */
-void oracle_balance(uint32_t n_mb, const uint64_t* cost, uint32_t K, uint32_t N, uint32_t* bucket,
+void oracle_balance(uint32_t n_mb, const uint64_t* cost, uint32_t K, uint32_t N, int carry, uint32_t* bucket,
                     uint32_t* rank, uint32_t* rank_mb_off, uint32_t* rank_mbs) {
   /* lines 12-14: buckets.  reading (parity unpinned): equal-width
    * quantisation of the observed cost range into K buckets. */
@@ -595,11 +596,14 @@ void oracle_balance(uint32_t n_mb, const uint64_t* cost, uint32_t K, uint32_t N,
   }
   /* lines 15-27: per bucket (reading: highest bucket first), sort by cost
    * descending (reading: ties by microbatch index ascending), then deal
-   * Rank_0..Rank_{N-1}, reverse, and so on; a and Forward restart per bucket;
-   * reading: the deal stops when the list is exhausted. */
+   * Rank_0..Rank_{N-1}, reverse, and so on; a and Forward restart per bucket
+   * (as printed); reading: the deal stops when the list is exhausted.
+   * Variant `carry`: one continuous zig-zag over the buckets' lists in turn: the
+   * position inside the current round and the direction carry over. */
   uint32_t* list = (uint32_t*)calloc((size_t)n_mb + 1, sizeof(uint32_t));
   uint32_t* order = (uint32_t*)calloc((size_t)n_mb + 1, sizeof(uint32_t)); /* global dispatch order */
   uint32_t n_order = 0;
+  uint32_t r_next = 0; int forward_c = 1; /* carried state: next rank to serve and the direction */
   for (int64_t k = (int64_t)K - 1; k >= 0; --k) {
     uint32_t m = 0;
     for (uint32_t j = 0; j < n_mb; ++j)
@@ -608,6 +612,14 @@ void oracle_balance(uint32_t n_mb, const uint64_t* cost, uint32_t K, uint32_t N,
       uint32_t x = list[i]; int64_t h = (int64_t)i - 1;
       while (h >= 0 && cost[list[h]] < cost[x]) { list[h + 1] = list[h]; --h; }
       list[h + 1] = x;
+    }
+    if (carry) {
+      for (uint32_t a = 0; a < m; ++a) {
+        rank[list[a]] = r_next; order[n_order++] = list[a];
+        if (forward_c) { if (r_next + 1 == N) forward_c = 0; else ++r_next; }   /* R0..R(N-1), then R(N-1)..R0 */
+        else           { if (r_next == 0) forward_c = 1; else --r_next; }
+      }
+      continue;
     }
     uint32_t a = 0; int forward = 1;
     while (a < m) {
@@ -675,21 +687,45 @@ int32_t oracle_plan_from_lengths(const uint32_t* slots, const uint32_t* len, uin
     /* per-sample score: Eq. 3 on a singleton microbatch */
     pl->sample_cost[t] = oracle_cost_int(cfg->coef_A, cfg->coef_B, len[t], len[t]);
   }
+  /* packing order: the caller's order (reading), or, as a variant, longest first (best-fit decreasing;
+   * equal lengths keep the caller's order) */
+  uint32_t* ord = ALLOC(uint32_t, n);
+  uint32_t* olen = ALLOC(uint32_t, n);
+  uint32_t* omb = ALLOC(uint32_t, n);
+  for (uint32_t t = 0; t < n; ++t) ord[t] = t;
+  if (cfg->flags & OR_PLAN_SORT_DECREASING)
+    for (uint32_t i = 1; i < n; ++i) { /* stable insertion sort by length, descending */
+      uint32_t x = ord[i]; int64_t h = (int64_t)i - 1;
+      while (h >= 0 && len[ord[h]] < len[x]) { ord[h + 1] = ord[h]; --h; }
+      ord[h + 1] = x;
+    }
+  for (uint32_t r = 0; r < n; ++r) olen[r] = len[ord[r]];
   /* lines 1-11 */
-  uint32_t n_mb = best_fit(n, len, L, pl->sample_mb, pl->mb_residual, pl->mb_tokens, pl->mb_lmax, count);
+  uint32_t n_mb = best_fit(n, olen, L, omb, pl->mb_residual, pl->mb_tokens, pl->mb_lmax, count);
   pl->n_mb = n_mb;
-  /* samples inside a microbatch stay in arrival order (line 5: append) */
+  for (uint32_t r = 0; r < n; ++r) pl->sample_mb[ord[r]] = omb[r];
+  /* samples inside a microbatch stay in packing order (line 5: append) */
   for (uint32_t j = 0; j < n_mb; ++j) pl->mb_sample_off[j + 1] = pl->mb_sample_off[j] + count[j];
   for (uint32_t j = 0; j < n_mb; ++j) {
     uint32_t w = pl->mb_sample_off[j];
-    for (uint32_t t = 0; t < n; ++t)
-      if (pl->sample_mb[t] == j) pl->mb_samples[w++] = pl->slots[t];
+    for (uint32_t r = 0; r < n; ++r)
+      if (omb[r] == j) pl->mb_samples[w++] = pl->slots[ord[r]];
   }
-  /* lines 12-14: Cost(B_j) */
-  for (uint32_t j = 0; j < n_mb; ++j)
-    pl->mb_cost[j] = oracle_cost_int(cfg->coef_A, cfg->coef_B, pl->mb_tokens[j], pl->mb_lmax[j]);
+  /* lines 12-14: Cost(B_j).  As printed the quadratic term is lmax^2; variant: the sum of squares */
+  for (uint32_t j = 0; j < n_mb; ++j) {
+    if (cfg->flags & OR_PLAN_COST_SUMSQ) {
+      uint64_t sq = 0;
+      for (uint32_t r = 0; r < n; ++r)
+        if (omb[r] == j) sq += (uint64_t)olen[r] * olen[r];
+      pl->mb_cost[j] = cfg->coef_A * pl->mb_tokens[j] + cfg->coef_B * sq;
+    } else {
+      pl->mb_cost[j] = oracle_cost_int(cfg->coef_A, cfg->coef_B, pl->mb_tokens[j], pl->mb_lmax[j]);
+    }
+  }
   /* lines 12-27: buckets and zig-zag dispatch */
-  oracle_balance(n_mb, pl->mb_cost, K, N, pl->mb_bucket, pl->mb_rank, pl->rank_mb_off, pl->rank_mbs);
+  oracle_balance(n_mb, pl->mb_cost, K, N, (cfg->flags & OR_PLAN_ZIGZAG_CARRY) != 0, pl->mb_bucket, pl->mb_rank,
+                 pl->rank_mb_off, pl->rank_mbs);
+  free(ord); free(olen); free(omb);
   free(count);
   *out = pl;
   return OR_OK;

@@ -92,13 +92,14 @@ def bestfit_segment_tree(lengths, L, l_min):
     return int(n_mb), out
 
 
-def balance(costs, K, N):
-    """Algorithm 1 lines 12-27 on explicit costs -> dict(bucket, rank, rank_mb_off, rank_mbs)."""
+def balance(costs, K, N, carry=0):
+    """Algorithm 1 lines 12-27 on explicit costs -> dict(bucket, rank, rank_mb_off, rank_mbs).
+    carry=1: the zig-zag position and direction carry over from bucket to bucket (variant)."""
     costs = np.ascontiguousarray(costs, dtype=np.uint64)
     m = len(costs)
     out = {"bucket": np.zeros(m, np.uint32), "rank": np.zeros(m, np.uint32),
            "rank_mb_off": np.zeros(N + 1, np.uint32), "rank_mbs": np.zeros(m, np.uint32)}
-    lib().oracle_balance(C.c_uint32(m), _p(costs), C.c_uint32(K), C.c_uint32(N), *[_p(v) for v in out.values()])
+    lib().oracle_balance(C.c_uint32(m), _p(costs), C.c_uint32(K), C.c_uint32(N), C.c_int(carry), *[_p(v) for v in out.values()])
     return out
 
 

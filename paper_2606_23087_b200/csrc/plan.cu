@@ -5,8 +5,10 @@
 //   k_bestfit        Algorithm 1 lines 1-11: online best fit.  The paper's segment tree over [0, L]
 //                    becomes a 32-ary bitmap hierarchy in shared memory (find-next-set = best-fit query,
 //                    same answer, O(log_32 L)); per-residual LIFO stacks give the tie rule.
-//   k_mb_finalize    Cost(B_j), min/max cost, exclusive scans -> mb_sample_off, mb_row_off
+//   k_pack_order     packing order: the caller's, or longest first (variant), by counting
+//   k_mb_finalize    exclusive scans -> mb_sample_off, mb_row_off
 //   k_plan_scatter   samples into microbatch-major, append order
+//   k_mb_cost        Cost(B_j) (lmax^2 as printed, or the sum-of-squares variant), min/max cost
 //   k_row_offsets    exclusive scan of lengths in plan order
 //   k_tiles          plan position of the sample holding each 32-row output tile
 //   k_bucket         lines 12-14: equal-width cost buckets
@@ -31,6 +33,28 @@ __global__ void k_plan_prepare(PoolView v, const uint32_t* slots, uint32_t n, ui
   const uint64_t l = v.s_seq_len[slots[t]];  // l(s): the LLM-side length, text + all vision tokens
   len[t] = (uint32_t)l;
   sample_cost[t] = A * l + B * l * l;
+}
+
+// Packing order.  Default: the caller's order.  Variant (longest first): position of sample t = number of
+// samples that are longer, or equally long and earlier -- rank by counting, tiles of lengths through shared memory.
+__global__ void __launch_bounds__(256) k_pack_order(const uint32_t* __restrict__ len, uint32_t n, uint32_t sort_desc,
+                                                    uint32_t* pk_t, uint32_t* pk_len) {
+  __shared__ uint32_t tile[1024];
+  const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
+  const uint32_t lt = t < n ? len[t] : 0;
+  uint32_t r = t;
+  if (sort_desc) {
+    r = 0;
+    for (uint32_t base = 0; base < n; base += 1024) {
+      const uint32_t cnt = min(1024u, n - base);
+      __syncthreads();
+      for (uint32_t i = threadIdx.x; i < cnt; i += blockDim.x) tile[i] = len[base + i];
+      __syncthreads();
+      if (t < n)
+        for (uint32_t i = 0; i < cnt; ++i) r += (tile[i] > lt) || (tile[i] == lt && base + i < t);
+    }
+  }
+  if (t < n) { pk_t[r] = t; pk_len[r] = lt; }
 }
 
 struct FitLevels {
@@ -154,13 +178,11 @@ __global__ void __launch_bounds__(1024) k_bestfit(const uint32_t* __restrict__ l
   if (threadIdx.x == 0) scalars[SC_NMB] = n_mb;
 }
 
-__global__ void __launch_bounds__(1024) k_mb_finalize(uint64_t A, uint64_t B, const uint32_t* mb_tokens,
-                                                      const uint32_t* mb_lmax, const uint32_t* mb_count, uint64_t* mb_cost,
+__global__ void __launch_bounds__(1024) k_mb_finalize(const uint32_t* mb_tokens, const uint32_t* mb_count,
                                                       uint32_t* mb_sample_off, uint64_t* mb_row_off, uint32_t* scalars) {
-  __shared__ unsigned long long s_lo, s_hi;
   __shared__ uint32_t s_max;
   const uint32_t n_mb = scalars[SC_NMB];
-  if (threadIdx.x == 0) { s_lo = ~0ull; s_hi = 0; s_max = 0; }
+  if (threadIdx.x == 0) s_max = 0;
   __syncthreads();
   uint64_t cs = 0, cr = 0;
   for (uint32_t base = 0; base < n_mb; base += blockDim.x) {
@@ -168,11 +190,6 @@ __global__ void __launch_bounds__(1024) k_mb_finalize(uint64_t A, uint64_t B, co
     uint64_t cnt = 0, tok = 0;
     if (j < n_mb) {
       cnt = mb_count[j]; tok = mb_tokens[j];
-      const uint64_t lm = mb_lmax[j];
-      const uint64_t cost = A * tok + B * lm * lm;  // Eq. 3 times L^2 when (A, B) = (L, 1)
-      mb_cost[j] = cost;
-      atomicMin(&s_lo, (unsigned long long)cost);
-      atomicMax(&s_hi, (unsigned long long)cost);
       atomicMax(&s_max, (uint32_t)tok);
     }
     uint64_t ts, tr;
@@ -186,20 +203,41 @@ __global__ void __launch_bounds__(1024) k_mb_finalize(uint64_t A, uint64_t B, co
     mb_sample_off[n_mb] = (uint32_t)cs; mb_row_off[n_mb] = cr;
     scalars[SC_MAXTOK] = s_max;
     scalars[SC_TOTAL_LO] = (uint32_t)cr; scalars[SC_TOTAL_HI] = (uint32_t)(cr >> 32);
-    *reinterpret_cast<unsigned long long*>(scalars + SC_LO) = s_lo;
-    *reinterpret_cast<unsigned long long*>(scalars + SC_HI) = s_hi;
+    *reinterpret_cast<unsigned long long*>(scalars + SC_LO) = ~0ull;  // cost range, filled by k_mb_cost
+    *reinterpret_cast<unsigned long long*>(scalars + SC_HI) = 0;
   }
 }
 
-__global__ void k_plan_scatter(const uint32_t* slots, const uint32_t* len, const uint32_t* sample_mb,
-                               const uint32_t* sample_rank, const uint32_t* mb_sample_off, uint32_t n,
-                               uint32_t* mb_samples, uint64_t* plan_len, uint32_t* plan_sample_mb) {
-  const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
-  if (t >= n) return;
-  const uint32_t j = sample_mb[t], q = mb_sample_off[j] + sample_rank[t];  // append order = arrival order
+// Cost(B_j), lines 12-14: A * sum(l) + B * lmax^2 (Eq. 3 times L^2 when (A, B) = (L, 1)); variant: B * sum(l^2).
+__global__ void k_mb_cost(uint64_t A, uint64_t B, uint32_t sumsq, const uint32_t* mb_tokens, const uint32_t* mb_lmax,
+                          const uint32_t* mb_sample_off, const uint64_t* plan_len, uint64_t* mb_cost, uint32_t* scalars) {
+  const uint32_t j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= scalars[SC_NMB]) return;
+  uint64_t quad;
+  if (sumsq) {
+    quad = 0;
+    for (uint32_t q = mb_sample_off[j]; q < mb_sample_off[j + 1]; ++q) quad += plan_len[q] * plan_len[q];
+  } else {
+    const uint64_t lm = mb_lmax[j];
+    quad = lm * lm;
+  }
+  const uint64_t cost = A * mb_tokens[j] + B * quad;
+  mb_cost[j] = cost;
+  atomicMin(reinterpret_cast<unsigned long long*>(scalars + SC_LO), (unsigned long long)cost);
+  atomicMax(reinterpret_cast<unsigned long long*>(scalars + SC_HI), (unsigned long long)cost);
+}
+
+__global__ void k_plan_scatter(const uint32_t* slots, const uint32_t* pk_t, const uint32_t* pk_len, const uint32_t* pk_mb,
+                               const uint32_t* pk_rank, const uint32_t* mb_sample_off, uint32_t n, uint32_t* mb_samples,
+                               uint64_t* plan_len, uint32_t* plan_sample_mb, uint32_t* sample_mb) {
+  const uint32_t r = blockIdx.x * blockDim.x + threadIdx.x;  // packing position
+  if (r >= n) return;
+  const uint32_t j = pk_mb[r], q = mb_sample_off[j] + pk_rank[r];  // append order = packing order
+  const uint32_t t = pk_t[r];
   mb_samples[q] = slots[t];
-  plan_len[q] = len[t];
+  plan_len[q] = pk_len[r];
   plan_sample_mb[q] = j;
+  sample_mb[t] = j;
 }
 
 __global__ void __launch_bounds__(1024) k_row_offsets(const uint64_t* plan_len, uint32_t n, uint64_t* sample_row_off) {
@@ -232,8 +270,8 @@ __global__ void k_bucket(const uint64_t* mb_cost, uint32_t K, const uint32_t* sc
 
 // Sorted position by counting: i comes before j when its bucket is higher, or equal bucket and cost higher,
 // or both equal and i < j.  Position inside the bucket -> zig-zag rank: round a/N forward when even.
-__global__ void k_sort_deal(const uint64_t* mb_cost, const uint32_t* mb_bucket, uint32_t N, const uint32_t* scalars,
-                            uint32_t* mb_pos, uint32_t* mb_rank) {
+__global__ void k_sort_deal(const uint64_t* mb_cost, const uint32_t* mb_bucket, uint32_t N, uint32_t carry,
+                            const uint32_t* scalars, uint32_t* mb_pos, uint32_t* mb_rank) {
   const uint32_t j = blockIdx.x * blockDim.x + threadIdx.x;
   const uint32_t n_mb = scalars[SC_NMB];
   if (j >= n_mb) return;
@@ -246,7 +284,8 @@ __global__ void k_sort_deal(const uint64_t* mb_cost, const uint32_t* mb_bucket, 
     higher += bi > bj;
     before += (bi > bj) || (bi == bj && (ci > cj || (ci == cj && i < j)));
   }
-  const uint32_t a = before - higher;  // index in the bucket's descending list
+  // index in the bucket's descending list; variant: in the concatenation of all lists (the zig-zag carries on)
+  const uint32_t a = carry ? before : before - higher;
   const uint32_t rnd = a / N, i = a % N;
   mb_pos[j] = before;
   mb_rank[j] = (rnd & 1) ? N - 1 - i : i;
@@ -343,6 +382,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_plan_microbatches
   const size_t o_cost = take(n * 8), o_mbcost = take(n * 8), o_srow = take(n1 * 8), o_mbrow = take(n1 * 8), o_plen = take(n * 8);
   const size_t o_recs = take(n * sizeof(MbRec)), o_head = take(((size_t)L + 1) * 4);
   const size_t o_slots = take(n * 4), o_len = take(n * 4), o_smb = take(n * 4), o_srank = take(n * 4);
+  const size_t o_pkt = take(n * 4), o_pklen = take(n * 4), o_pkmb = take(n * 4);
   const size_t o_mboff = take(n1 * 4), o_mbs = take(n * 4), o_psmb = take(n * 4);
   const size_t o_tok = take(n * 4), o_lmax = take(n * 4), o_res = take(n * 4), o_cnt = take(n * 4);
   const size_t o_bkt = take(n * 4), o_rank = take(n * 4), o_pos = take(n * 4), o_idx = take(n * 4);
@@ -371,6 +411,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_plan_microbatches
   pl->d_rank_mb_off = U32(o_roff); pl->d_rank_mbs = U32(o_rmbs); pl->d_rank_cnt = U32(o_rcnt);
   pl->d_tile_first_sample = U32(o_tiles); pl->d_scalars = U32(o_scal);
   uint32_t* d_mb_idx = U32(o_idx);
+  uint32_t *d_pk_t = U32(o_pkt), *d_pk_len = U32(o_pklen), *d_pk_mb = U32(o_pkmb);
   MbRec* d_recs = reinterpret_cast<MbRec*>(b + o_recs);
   uint32_t* d_head = U32(o_head);
 
@@ -405,22 +446,26 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_plan_microbatches
     CK(cudaFuncSetAttribute(k_bestfit, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)limit));
     attr_set = true;
   }
-  k_bestfit<<<1, 1024, used, st>>>(pl->d_len, n, L, d_head, d_recs, head_in_smem, rec_cap, pl->d_sample_mb,
+  const uint32_t f_sort = (cfg->flags & FT_PLAN_SORT_DECREASING) != 0, f_sumsq = (cfg->flags & FT_PLAN_COST_SUMSQ) != 0;
+  const uint32_t f_carry = (cfg->flags & FT_PLAN_ZIGZAG_CARRY) != 0;
+  k_pack_order<<<gb, 256, 0, st>>>(pl->d_len, n, f_sort, d_pk_t, d_pk_len);
+  k_bestfit<<<1, 1024, used, st>>>(d_pk_len, n, L, d_head, d_recs, head_in_smem, rec_cap, d_pk_mb,
                                    pl->d_sample_rank, pl->d_mb_residual, pl->d_mb_tokens, pl->d_mb_lmax, pl->d_mb_count,
                                    pl->d_scalars);
-  k_mb_finalize<<<1, 1024, 0, st>>>(cfg->coef_A, cfg->coef_B, pl->d_mb_tokens, pl->d_mb_lmax, pl->d_mb_count, pl->d_mb_cost,
-                                    pl->d_mb_sample_off, pl->d_mb_row_off, pl->d_scalars);
-  k_plan_scatter<<<gb, 256, 0, st>>>(pl->d_slots, pl->d_len, pl->d_sample_mb, pl->d_sample_rank, pl->d_mb_sample_off, n,
-                                     pl->d_mb_samples, pl->d_plan_len, pl->d_plan_sample_mb);
+  k_mb_finalize<<<1, 1024, 0, st>>>(pl->d_mb_tokens, pl->d_mb_count, pl->d_mb_sample_off, pl->d_mb_row_off, pl->d_scalars);
+  k_plan_scatter<<<gb, 256, 0, st>>>(pl->d_slots, d_pk_t, d_pk_len, d_pk_mb, pl->d_sample_rank, pl->d_mb_sample_off, n,
+                                     pl->d_mb_samples, pl->d_plan_len, pl->d_plan_sample_mb, pl->d_sample_mb);
+  k_mb_cost<<<gb, 256, 0, st>>>(cfg->coef_A, cfg->coef_B, f_sumsq, pl->d_mb_tokens, pl->d_mb_lmax, pl->d_mb_sample_off,
+                                pl->d_plan_len, pl->d_mb_cost, pl->d_scalars);
   k_row_offsets<<<1, 1024, 0, st>>>(pl->d_plan_len, n, pl->d_sample_row_off);
   k_tiles<<<gb, 256, 0, st>>>(pl->d_sample_row_off, n, pl->d_tile_first_sample);
   k_bucket<<<gb, 256, 0, st>>>(pl->d_mb_cost, K, pl->d_scalars, pl->d_mb_bucket);
-  k_sort_deal<<<gb, 256, 0, st>>>(pl->d_mb_cost, pl->d_mb_bucket, N, pl->d_scalars, pl->d_mb_pos, pl->d_mb_rank);
+  k_sort_deal<<<gb, 256, 0, st>>>(pl->d_mb_cost, pl->d_mb_bucket, N, f_carry, pl->d_scalars, pl->d_mb_pos, pl->d_mb_rank);
   k_rank_index<<<gb, 256, 0, st>>>(pl->d_mb_pos, pl->d_mb_rank, pl->d_scalars, d_mb_idx, pl->d_rank_cnt);
   k_rank_scan<<<1, 1024, 0, st>>>(pl->d_rank_cnt, N, pl->d_rank_mb_off);
   k_rank_lists<<<gb, 256, 0, st>>>(pl->d_mb_rank, d_mb_idx, pl->d_rank_mb_off, pl->d_scalars, pl->d_rank_mbs);
   CK(cudaGetLastError());
-  p->gpu_launches += 11;
+  p->gpu_launches += 13;
 
   uint32_t sc[SC_COUNT];
   CK(cudaMemcpyAsync(sc, pl->d_scalars, sizeof(sc), cudaMemcpyDeviceToHost, st));

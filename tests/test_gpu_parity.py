@@ -389,3 +389,64 @@ def test_planner_scale_matches_oracle():
     gp.destroy()
     op.destroy()
     pool.destroy()
+
+
+@pytest.mark.parametrize("flags", [2, 4, 8, 2 | 4 | 8])
+def test_plan_variants_match_oracle(flags):
+    """Scheduler variants (longest-first packing, sum-of-squares cost, carried zig-zag): every plan array equals
+    the oracle's, on 6000 descriptors (metadata only) and on a written batch whose gather follows the new order."""
+    gh = _gpu()
+    from paper_2606_23087_b200 import binding as fp
+    w = workloads.make_workload("frag_sweep", n_samples=6000, hidden=64, page_bytes=4096, pool_bytes=4096 * 16)
+    pool = fp.Pool(fp.PoolConfig(**pool_config_fields(w)))
+    assert pool.rc == 0
+    seq_len, n_spans = w.seq_len.astype(np.uint32), w.n_spans.astype(np.uint32)
+    off = np.concatenate([[0], np.cumsum(seq_len.astype(np.int64))])
+    ids = np.zeros(int(off[-1]), np.int32)
+    for s in range(w.n_samples):
+        p0 = int(off[s]) + int(w.span_pos[s])
+        ids[p0:p0 + int(w.span_tokens[s])] = w.placeholder_id
+    d_ids = torch.from_numpy(ids).cuda()
+    assert pool.register_samples(list(range(w.n_samples)), seq_len, n_spans, w.span_pos, w.span_tokens, d_ids.data_ptr(), gh.cuda_stream()) == 0
+    order = [int(x) for x in np.random.default_rng(flags).permutation(w.n_samples)]
+    for K, N, L in ((4, 8, 32768), (1, 3, 18000), (7, 5, 131072)):
+        cfg = dict(coef_A=L, coef_B=1, budget_L=L, n_buckets_K=K, n_ranks_N=N, flags=flags | 1)
+        rc, gp = pool.plan_microbatches(order, fp.PlanConfig(**cfg), gh.cuda_stream())
+        rc2, op = plan_from_lengths(seq_len[order], PlanConfig(**cfg), slots=order)
+        assert rc == rc2 == 0
+        ga, oa = gp.arrays(), op.arrays()
+        assert ga["n_mb"] == oa["n_mb"]
+        for k in PLAN_KEYS:
+            assert np.array_equal(ga[k], oa[k]), (k, K, N, L)
+        gp.destroy(); op.destroy()
+    pool.destroy()
+    # end to end with the variant: the gather must follow the variant's append order
+    w = workloads.make_workload("image_mix_7b", n_samples=24, hidden=128, page_bytes=16384)
+    w.budget_L = 20000
+    opool, pool = OraclePool(PoolConfig(**pool_config_fields(w))), fp.Pool(fp.PoolConfig(**pool_config_fields(w)))
+    keep = []
+    for call in w.write_calls:
+        samples = sorted({s for s, _ in call}, key=[s for s, _ in call].index)
+        a = register_args(w, samples)
+        d = torch.from_numpy(a[5]).cuda(); keep.append(d)
+        assert pool.register_samples(*a[:5], d.data_ptr(), gh.cuda_stream()) == opool.register_samples(*a) == 0
+        srcs = [workloads.span_values(w, s, j, device="cuda") for s, j in call]; keep.append(srcs)
+        assert pool.write_embeddings(*write_args(w, call), [t.data_ptr() for t in srcs], 0, gh.cuda_stream()) == 0
+        assert opool.write_embeddings(*write_args(w, call), [bits16(t) for t in srcs], 0) == 0
+    cfg = plan_config_fields(w, flags=flags)
+    rc, gp = pool.plan_microbatches(w.plan_order, fp.PlanConfig(**cfg), gh.cuda_stream())
+    rc2, op = opool.plan_microbatches(w.plan_order, PlanConfig(**cfg))
+    assert rc == rc2 == 0
+    n_mb, total, _ = gp.summary()
+    assert (n_mb, total) == op.summary()[:2]
+    table = workloads.embed_table(w, device="cuda")
+    out = torch.full((total, w.hidden), -1, dtype=torch.int16, device="cuda")
+    cu = torch.full((w.n_samples + n_mb,), -1, dtype=torch.int32, device="cuda")
+    pos = torch.full((total,), -1, dtype=torch.int32, device="cuda")
+    assert pool.gather_packed(gp, 0, n_mb, table.data_ptr(), w.vocab, out.data_ptr(), cu.data_ptr(), pos.data_ptr(), gh.cuda_stream()) == 0
+    oout = np.full((total, w.hidden), 0xFFFF, np.uint16); ocu = np.full(w.n_samples + n_mb, -1, np.int32); opos = np.full(total, -1, np.int32)
+    assert opool.gather_packed(op, 0, n_mb, bits16(table), oout, ocu, opos) == 0
+    torch.cuda.synchronize()
+    assert np.array_equal(out.cpu().numpy().view(np.uint16), oout)
+    assert np.array_equal(cu.cpu().numpy(), ocu) and np.array_equal(pos.cpu().numpy(), opos)
+    pool.destroy(); opool.destroy()
