@@ -280,6 +280,40 @@ int32_t pool_status(ft_pool* pool, int32_t* first_device_error, uint64_t* detail
 int32_t pool_stats(ft_pool* pool, ft_pool_stats* out);
 
 /*
+ * More than one process in the GVA space (Sec. 3.2: "each process exports its memory mapping information to all
+ * other processes, which update their page table accordingly"; afterwards address translation is local).
+ * Pools created with the same world_size, page_bytes, GVA starts and max_size and distinct ranks form one space.
+ *
+ * pool_backing        the addresses of this pool's slabs as THIS process sees them (device pointers; the host
+ *                     slab as the device sees it).  A peer in another process needs its own view of them (an IPC
+ *                     or fabric mapping); in one process, with peer access enabled, these are usable as they are.
+ * pool_export_mapping this process's binding (geometry + vpn->frame of both tiers) into a host buffer.
+ *                     buf = NULL queries the size.  CAPACITY if cap is too small.
+ * pool_import_mapping installs a peer's binding: builds that process's page-table arrays from the blob and the
+ *                     three base addresses at which this device reaches the peer's HBM slab, host slab and text
+ *                     frames.  INVALID_ARG: malformed blob, another GVA space, own rank, missing or misaligned
+ *                     base; SLOT_IN_USE: that rank was imported before.  Init-time: allocates, synchronises.
+ * pool_export_samples descriptors of READY samples (lengths, spans, page GVAs, text-page GVAs) into a host buffer
+ *                     -- the "lightweight metadata" a consumer needs; no embedding bytes.  Synchronises `stream`.
+ *                     UNKNOWN_SAMPLE / NOT_READY / INVALID_ARG (repeated slot) per sample in order; buf = NULL
+ *                     queries the size.
+ * pool_import_samples registers the described samples in local FREE slots as READY, imported samples: their page
+ *                     lists point into the peer's segment and are read in place by pool_gather_packed; they take
+ *                     list blocks but no pages here, and pool_free returns nothing to the page rings for them.
+ *                     The producer must keep the samples alive until the consumer has freed its imports.
+ *                     INVALID_ARG: malformed blob or the source rank's mapping not imported; SLOT_IN_USE;
+ *                     CAPACITY: a sample exceeds this pool's limits or the list blocks run out.  Asynchronous.
+ */
+int32_t pool_backing(ft_pool* pool, void** hbm_base, void** host_base_device, void** text_base);
+int32_t pool_export_mapping(ft_pool* pool, void* buf /* host */, uint64_t cap, uint64_t* bytes);
+int32_t pool_import_mapping(ft_pool* pool, const void* buf /* host */, uint64_t bytes, void* peer_hbm_base,
+                            void* peer_host_base, void* peer_text_base);
+int32_t pool_export_samples(ft_pool* pool, const uint32_t* sample_slot, uint32_t n, void* buf /* host */, uint64_t cap,
+                            uint64_t* bytes, void* stream);
+int32_t pool_import_samples(ft_pool* pool, const uint32_t* local_slot, uint32_t n, const void* buf /* host */,
+                            uint64_t bytes, void* stream);
+
+/*
  * Kernel timing for benchmarks.  While enabled, the library brackets each of its copy kernels with CUDA
  * events on the stream that kernel is launched on (the host-tier kernels run on the pool's side stream).
  * pool_profile_read synchronises the device, adds up the elapsed time and launch count per kernel class

@@ -74,6 +74,7 @@ typedef struct {
 
 typedef struct {
   int state;
+  int remote; /* imported from another process: its pages and text pages are not ours to recycle */
   uint32_t seq_len, n_spans, spans_written;
   uint64_t generation;
   or_span* spans;
@@ -81,8 +82,18 @@ typedef struct {
   uint64_t* text_pages; /* text-page GVAs */
 } or_sample;
 
+/* one process's binding as this process holds it (Sec. 3.2: the collected page tables) */
+typedef struct {
+  int present;
+  uint64_t hbm_pages, host_pages, text_pages;
+  uint64_t* bind_hbm;  /* vpn -> frame */
+  uint64_t* bind_host;
+  uint8_t *hbm_mem, *host_mem, *text_mem; /* where this process reaches that process's frames */
+} or_peer;
+
 typedef struct oracle_pool {
   oracle_pool_config c;
+  or_peer* peers; /* [world_size]; entry c.rank is this process's own binding */
   uint64_t P;        /* hbm_pages + host_pages */
   uint8_t* hbm_mem;  /* backing frames, HBM tier */
   uint8_t* host_mem; /* backing frames, DRAM tier */
@@ -179,26 +190,30 @@ static uint64_t text_page_gva(const oracle_pool* p, uint64_t k) {
   return oracle_segment_base(p, 0, p->c.rank) + p->c.hbm_pages * p->c.page_bytes + k * TEXT_PAGE_BYTES;
 }
 
-/* kind: 0 = HBM embedding page, 1 = DRAM embedding page, 2 = text page. */
-int32_t oracle_translate(const oracle_pool* p, uint64_t g, uint32_t* kind, uint64_t* frame,
-                         uint64_t* offset) {
+/* kind: 0 = HBM embedding page, 1 = DRAM embedding page, 2 = text page; proc = owning process.
+ * Translation is local: the region by interval test, the process by division, then that process's table
+ * (its own, or one installed by oracle_pool_import_mapping; unknown processes do not translate). */
+int32_t oracle_translate_ex(const oracle_pool* p, uint64_t g, uint32_t* proc, uint32_t* kind, uint64_t* frame,
+                            uint64_t* offset) {
   const uint64_t W = p->c.world_size, M = p->c.max_size, PS = p->c.page_bytes;
   for (uint32_t t = 0; t < 2; ++t) {
     uint64_t start = t == 0 ? p->c.gva_hbm_start : p->c.gva_host_start;
     if (g < start || g >= start + W * M) continue;
     uint64_t i = (g - start) / M, o = (g - start) % M;
-    if (i != p->c.rank) return OR_ERR_BAD_GVA; /* only this process's binding exists */
-    uint64_t pages = t == 0 ? p->c.hbm_pages : p->c.host_pages;
+    const or_peer* pr = &p->peers[i];
+    if (!pr->present) return OR_ERR_BAD_GVA;
+    uint64_t pages = t == 0 ? pr->hbm_pages : pr->host_pages;
+    *proc = (uint32_t)i;
     if (o < pages * PS) {
       uint64_t vpn = o / PS;
       *kind = t;
-      *frame = t == 0 ? p->bind_hbm[vpn] : p->bind_host[vpn];
+      *frame = t == 0 ? pr->bind_hbm[vpn] : pr->bind_host[vpn];
       *offset = o % PS;
       return OR_OK;
     }
     if (t == 0) {
       uint64_t ot = o - pages * PS;
-      if (ot < p->n_text_pages * (uint64_t)TEXT_PAGE_BYTES) {
+      if (ot < pr->text_pages * (uint64_t)TEXT_PAGE_BYTES) {
         *kind = 2; *frame = ot / TEXT_PAGE_BYTES; *offset = ot % TEXT_PAGE_BYTES;
         return OR_OK;
       }
@@ -208,12 +223,18 @@ int32_t oracle_translate(const oracle_pool* p, uint64_t g, uint32_t* kind, uint6
   return OR_ERR_BAD_GVA;
 }
 
+int32_t oracle_translate(const oracle_pool* p, uint64_t g, uint32_t* kind, uint64_t* frame, uint64_t* offset) {
+  uint32_t proc;
+  return oracle_translate_ex(p, g, &proc, kind, frame, offset);
+}
+
 static uint8_t* resolve(oracle_pool* p, uint64_t g) {
-  uint32_t kind; uint64_t frame, off;
-  if (oracle_translate(p, g, &kind, &frame, &off) != OR_OK) return NULL;
-  if (kind == 0) return p->hbm_mem + frame * p->c.page_bytes + off;
-  if (kind == 1) return p->host_mem + frame * p->c.page_bytes + off;
-  return p->text_mem + frame * TEXT_PAGE_BYTES + off;
+  uint32_t proc, kind; uint64_t frame, off;
+  if (oracle_translate_ex(p, g, &proc, &kind, &frame, &off) != OR_OK) return NULL;
+  const or_peer* pr = &p->peers[proc];
+  if (kind == 0) return pr->hbm_mem + frame * p->c.page_bytes + off;
+  if (kind == 1) return pr->host_mem + frame * p->c.page_bytes + off;
+  return pr->text_mem + frame * TEXT_PAGE_BYTES + off;
 }
 
 static void note_async_error(oracle_pool* p, int32_t code, uint32_t detail) {
@@ -288,6 +309,12 @@ int32_t oracle_pool_create(const oracle_pool_config* cfg, oracle_pool** out) {
 
   p->samples = (or_sample*)calloc(c.max_samples, sizeof(or_sample));
   p->status_key = UINT64_MAX;
+  p->peers = (or_peer*)calloc(c.world_size, sizeof(or_peer));
+  or_peer* self = &p->peers[c.rank];
+  self->present = 1;
+  self->hbm_pages = c.hbm_pages; self->host_pages = c.host_pages; self->text_pages = n_text_pages;
+  self->bind_hbm = p->bind_hbm; self->bind_host = p->bind_host;
+  self->hbm_mem = p->hbm_mem; self->host_mem = p->host_mem; self->text_mem = p->text_mem;
   *out = p;
   return OR_OK;
 }
@@ -304,6 +331,9 @@ static void release_sample_storage(or_sample* s) {
 int32_t oracle_pool_destroy(oracle_pool* p) {
   if (!p) return OR_ERR_INVALID_ARG;
   for (uint32_t i = 0; i < p->c.max_samples; ++i) release_sample_storage(&p->samples[i]);
+  for (uint32_t i = 0; i < p->c.world_size; ++i)
+    if (i != p->c.rank && p->peers[i].present) { free(p->peers[i].bind_hbm); free(p->peers[i].bind_host); }
+  free(p->peers);
   free(p->samples); free(p->ring); free(p->tring); free(p->bind_hbm); free(p->bind_host);
   free(p->hbm_mem); free(p->host_mem); free(p->text_mem); free(p);
   return OR_OK;
@@ -351,7 +381,7 @@ int32_t oracle_pool_register_samples(oracle_pool* p, uint32_t n, const uint32_t*
   for (uint32_t i = 0; i < n; ++i) {
     or_sample* s = &p->samples[slot[i]];
     s->state = n_spans[i] == 0 ? SLOT_READY : SLOT_REGISTERED; /* text-only: paired at once */
-    s->seq_len = seq_len[i]; s->n_spans = n_spans[i]; s->spans_written = 0;
+    s->seq_len = seq_len[i]; s->n_spans = n_spans[i]; s->spans_written = 0; s->remote = 0;
     s->spans = (or_span*)calloc(n_spans[i] + 1, sizeof(or_span));
     uint64_t placeholders = 0;
     int bad = 0;
@@ -475,19 +505,21 @@ int32_t oracle_pool_free(oracle_pool* p, const uint32_t* slot, uint32_t n) {
   }
   for (uint32_t i = 0; i < n; ++i) {
     or_sample* s = &p->samples[slot[i]];
-    for (uint32_t j = 0; j < s->n_spans; ++j)
-      for (uint32_t o = 0; o < s->spans[j].n_pages; ++o) {
-        uint64_t idx = global_page_of_gva(p, s->spans[j].pages[o]);
-        p->ring[(p->ring_head + p->ring_count) % p->P] = (uint32_t)idx;
-        p->ring_count++;
+    if (!s->remote) { /* an imported sample's pages and text pages belong to the process that wrote them */
+      for (uint32_t j = 0; j < s->n_spans; ++j)
+        for (uint32_t o = 0; o < s->spans[j].n_pages; ++o) {
+          uint64_t idx = global_page_of_gva(p, s->spans[j].pages[o]);
+          p->ring[(p->ring_head + p->ring_count) % p->P] = (uint32_t)idx;
+          p->ring_count++;
+        }
+      for (uint32_t k = 0; k < s->n_text_pages; ++k) {
+        uint64_t tp = (s->text_pages[k] - text_page_gva(p, 0)) / TEXT_PAGE_BYTES;
+        p->tring[(p->tring_head + p->tring_count) % p->n_text_pages] = (uint32_t)tp;
+        p->tring_count++;
       }
-    for (uint32_t k = 0; k < s->n_text_pages; ++k) {
-      uint64_t tp = (s->text_pages[k] - text_page_gva(p, 0)) / TEXT_PAGE_BYTES;
-      p->tring[(p->tring_head + p->tring_count) % p->n_text_pages] = (uint32_t)tp;
-      p->tring_count++;
     }
     release_sample_storage(s);
-    s->state = SLOT_FREE; s->n_spans = 0; s->seq_len = 0; s->spans_written = 0; s->n_text_pages = 0;
+    s->state = SLOT_FREE; s->n_spans = 0; s->seq_len = 0; s->spans_written = 0; s->n_text_pages = 0; s->remote = 0;
     s->generation++;
   }
   return OR_OK;
@@ -814,6 +846,144 @@ int32_t oracle_pool_gather_packed(oracle_pool* p, const oracle_plan* pl, uint32_
       cu += (int32_t)s->seq_len;
       out_cu_seqlens[cu_w++] = cu;
     }
+  }
+  return OR_OK;
+}
+
+/* ------------------------------------------------------------------------
+ * More than one process (Sec. 3.2): each process exports its memory mapping,
+ * the others update their page tables; samples cross processes as descriptors
+ * (lengths, spans, page GVAs, text-page GVAs) and are read in place.
+ * Blob formats are this file's own.
+ * ---------------------------------------------------------------------- */
+typedef struct {
+  uint64_t magic, page_bytes, hbm_pages, host_pages, text_pages, gva_hbm_start, gva_host_start, max_size;
+  uint32_t rank, world_size;
+} or_map_header;
+#define OR_MAP_MAGIC 0x4F5241434C454D50ull
+#define OR_SMP_MAGIC 0x4F5241434C455350ull
+
+int32_t oracle_pool_export_mapping(oracle_pool* p, void* buf, uint64_t cap, uint64_t* bytes) {
+  if (!p) return OR_ERR_INVALID_ARG;
+  uint64_t need = sizeof(or_map_header) + 8 * (p->c.hbm_pages + p->c.host_pages);
+  if (bytes) *bytes = need;
+  if (!buf) return OR_OK;
+  if (cap < need) return OR_ERR_CAPACITY;
+  or_map_header h;
+  memset(&h, 0, sizeof(h));
+  h.magic = OR_MAP_MAGIC; h.page_bytes = p->c.page_bytes; h.hbm_pages = p->c.hbm_pages; h.host_pages = p->c.host_pages;
+  h.text_pages = p->n_text_pages; h.gva_hbm_start = p->c.gva_hbm_start; h.gva_host_start = p->c.gva_host_start;
+  h.max_size = p->c.max_size; h.rank = p->c.rank; h.world_size = p->c.world_size;
+  memcpy(buf, &h, sizeof(h));
+  memcpy((uint8_t*)buf + sizeof(h), p->bind_hbm, 8 * p->c.hbm_pages);
+  memcpy((uint8_t*)buf + sizeof(h) + 8 * p->c.hbm_pages, p->bind_host, 8 * p->c.host_pages);
+  return OR_OK;
+}
+
+/* peer_*: where this process reaches the peer's frames (host pointers here) */
+int32_t oracle_pool_import_mapping(oracle_pool* p, const void* buf, uint64_t bytes, void* peer_hbm, void* peer_host,
+                                   void* peer_text) {
+  if (!p || !buf || bytes < sizeof(or_map_header)) return OR_ERR_INVALID_ARG;
+  or_map_header h;
+  memcpy(&h, buf, sizeof(h));
+  if (h.magic != OR_MAP_MAGIC || bytes != sizeof(h) + 8 * (h.hbm_pages + h.host_pages)) return OR_ERR_INVALID_ARG;
+  if (h.world_size != p->c.world_size || h.rank >= p->c.world_size || h.rank == p->c.rank) return OR_ERR_INVALID_ARG;
+  if (h.page_bytes != p->c.page_bytes || h.gva_hbm_start != p->c.gva_hbm_start || h.gva_host_start != p->c.gva_host_start ||
+      h.max_size != p->c.max_size)
+    return OR_ERR_INVALID_ARG;
+  or_peer* pr = &p->peers[h.rank];
+  if (pr->present) return OR_ERR_SLOT_IN_USE;
+  if ((h.hbm_pages && !peer_hbm) || (h.host_pages && !peer_host) || (h.text_pages && !peer_text)) return OR_ERR_INVALID_ARG;
+  pr->hbm_pages = h.hbm_pages; pr->host_pages = h.host_pages; pr->text_pages = h.text_pages;
+  pr->bind_hbm = (uint64_t*)malloc(8 * (h.hbm_pages + 1));
+  pr->bind_host = (uint64_t*)malloc(8 * (h.host_pages + 1));
+  memcpy(pr->bind_hbm, (const uint8_t*)buf + sizeof(h), 8 * h.hbm_pages);
+  memcpy(pr->bind_host, (const uint8_t*)buf + sizeof(h) + 8 * h.hbm_pages, 8 * h.host_pages);
+  pr->hbm_mem = (uint8_t*)peer_hbm; pr->host_mem = (uint8_t*)peer_host; pr->text_mem = (uint8_t*)peer_text;
+  pr->present = 1;
+  return OR_OK;
+}
+
+/* blob: header {magic, n, src_rank}, then per sample: seq_len, n_spans, n_text_pages, its spans (pos, tokens,
+ * n_pages, page GVAs...), its text-page GVAs -- all as u64 words */
+int32_t oracle_pool_export_samples(oracle_pool* p, const uint32_t* slot, uint32_t n, void* buf, uint64_t cap,
+                                   uint64_t* bytes) {
+  if (!p || (n && !slot)) return OR_ERR_INVALID_ARG;
+  uint64_t words = 3;
+  for (uint32_t i = 0; i < n; ++i) {
+    if (slot[i] >= p->c.max_samples) return OR_ERR_INVALID_ARG;
+    const or_sample* s = &p->samples[slot[i]];
+    if (s->state == SLOT_FREE) return OR_ERR_UNKNOWN_SAMPLE;
+    for (uint32_t j = 0; j < i; ++j)
+      if (slot[j] == slot[i]) return OR_ERR_INVALID_ARG;
+    if (s->state != SLOT_READY) return OR_ERR_NOT_READY;
+    words += 3 + s->n_text_pages;
+    for (uint32_t j = 0; j < s->n_spans; ++j) words += 3 + s->spans[j].n_pages;
+  }
+  if (bytes) *bytes = 8 * words;
+  if (!buf) return OR_OK;
+  if (cap < 8 * words) return OR_ERR_CAPACITY;
+  uint64_t* w = (uint64_t*)buf;
+  *w++ = OR_SMP_MAGIC; *w++ = n; *w++ = p->c.rank;
+  for (uint32_t i = 0; i < n; ++i) {
+    const or_sample* s = &p->samples[slot[i]];
+    *w++ = s->seq_len; *w++ = s->n_spans; *w++ = s->n_text_pages;
+    for (uint32_t j = 0; j < s->n_spans; ++j) {
+      *w++ = s->spans[j].pos_start; *w++ = s->spans[j].n_tokens; *w++ = s->spans[j].n_pages;
+      for (uint32_t o = 0; o < s->spans[j].n_pages; ++o) *w++ = s->spans[j].pages[o];
+    }
+    for (uint32_t k = 0; k < s->n_text_pages; ++k) *w++ = s->text_pages[k];
+  }
+  return OR_OK;
+}
+
+int32_t oracle_pool_import_samples(oracle_pool* p, const uint32_t* local_slot, uint32_t n, const void* buf,
+                                   uint64_t bytes) {
+  if (!p || !buf || bytes < 24 || (n && !local_slot)) return OR_ERR_INVALID_ARG;
+  p->call_seq++;
+  const uint64_t* w = (const uint64_t*)buf;
+  const uint64_t* end = w + bytes / 8;
+  if (w[0] != OR_SMP_MAGIC || w[1] != n) return OR_ERR_INVALID_ARG;
+  if (w[2] >= p->c.world_size || !p->peers[w[2]].present) return OR_ERR_INVALID_ARG; /* mapping first */
+  if (n == 0) return OR_OK;
+  /* checks, in argument order */
+  const uint64_t* r = w + 3;
+  for (uint32_t i = 0; i < n; ++i) {
+    if (local_slot[i] >= p->c.max_samples) return OR_ERR_INVALID_ARG;
+    if (p->samples[local_slot[i]].state != SLOT_FREE) return OR_ERR_SLOT_IN_USE;
+    for (uint32_t j = 0; j < i; ++j)
+      if (local_slot[j] == local_slot[i]) return OR_ERR_SLOT_IN_USE;
+    if (r + 3 > end) return OR_ERR_INVALID_ARG;
+    uint64_t seq_len = r[0], n_spans = r[1], ntp = r[2];
+    r += 3;
+    if (seq_len == 0 || ntp != (seq_len + TEXT_PAGE_IDS - 1) / TEXT_PAGE_IDS) return OR_ERR_INVALID_ARG;
+    if (seq_len > p->c.max_seq_len || n_spans > p->c.max_spans_per_sample) return OR_ERR_CAPACITY;
+    for (uint64_t j = 0; j < n_spans; ++j) {
+      if (r + 3 > end) return OR_ERR_INVALID_ARG;
+      uint64_t np = r[2];
+      if (np > (uint64_t)((p->c.max_pages_per_span + 63) / 64) * 64) return OR_ERR_CAPACITY;
+      r += 3 + np;
+    }
+    r += ntp;
+    if (r > end) return OR_ERR_INVALID_ARG;
+  }
+  if (r != end) return OR_ERR_INVALID_ARG;
+  r = w + 3;
+  for (uint32_t i = 0; i < n; ++i) {
+    or_sample* s = &p->samples[local_slot[i]];
+    s->state = SLOT_READY; s->remote = 1;
+    s->seq_len = (uint32_t)r[0]; s->n_spans = (uint32_t)r[1]; s->n_text_pages = (uint32_t)r[2];
+    s->spans_written = s->n_spans;
+    r += 3;
+    s->spans = (or_span*)calloc(s->n_spans + 1, sizeof(or_span));
+    for (uint32_t j = 0; j < s->n_spans; ++j) {
+      s->spans[j].pos_start = (uint32_t)r[0]; s->spans[j].n_tokens = (uint32_t)r[1]; s->spans[j].n_pages = (uint32_t)r[2];
+      r += 3;
+      s->spans[j].pages = (uint64_t*)malloc(8 * (s->spans[j].n_pages + 1));
+      for (uint32_t o = 0; o < s->spans[j].n_pages; ++o) s->spans[j].pages[o] = *r++;
+    }
+    s->text_pages = (uint64_t*)malloc(8 * (s->n_text_pages + 1));
+    for (uint32_t k = 0; k < s->n_text_pages; ++k) s->text_pages[k] = *r++;
   }
   return OR_OK;
 }

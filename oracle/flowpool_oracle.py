@@ -225,6 +225,39 @@ class OraclePool:
     def segment_base(self, tier, proc):
         return int(lib().oracle_segment_base(self.h, C.c_uint32(tier), C.c_uint32(proc)))
 
+    def translate_ex(self, gva):
+        proc, kind, frame, off = C.c_uint32(), C.c_uint32(), C.c_uint64(), C.c_uint64()
+        rc = lib().oracle_translate_ex(self.h, C.c_uint64(gva), C.byref(proc), C.byref(kind), C.byref(frame), C.byref(off))
+        return rc, proc.value, kind.value, frame.value, off.value
+
+    def export_mapping(self):
+        n = C.c_uint64()
+        lib().oracle_pool_export_mapping(self.h, None, C.c_uint64(0), C.byref(n))
+        buf = np.zeros(n.value, np.uint8)
+        rc = lib().oracle_pool_export_mapping(self.h, _p(buf), C.c_uint64(n.value), C.byref(n))
+        return rc, buf
+
+    def import_mapping(self, blob, peer):
+        """peer: the OraclePool whose mapping this is (its backing arrays are reached directly: one process)."""
+        blob = np.ascontiguousarray(blob, dtype=np.uint8)
+        ptrs = [C.c_void_p(lib().oracle_pool_backing(peer.h, C.c_uint32(k))) for k in range(3)] if peer is not None else [None] * 3
+        return lib().oracle_pool_import_mapping(self.h, _p(blob), C.c_uint64(len(blob)), *ptrs)
+
+    def export_samples(self, slots):
+        slots = _u32(slots)
+        n = C.c_uint64()
+        rc = lib().oracle_pool_export_samples(self.h, _p(slots), C.c_uint32(len(slots)), None, C.c_uint64(0), C.byref(n))
+        if rc:
+            return rc, None
+        buf = np.zeros(n.value, np.uint8)
+        rc = lib().oracle_pool_export_samples(self.h, _p(slots), C.c_uint32(len(slots)), _p(buf), C.c_uint64(n.value), C.byref(n))
+        return rc, buf
+
+    def import_samples(self, local_slots, blob):
+        local_slots = _u32(local_slots)
+        blob = np.ascontiguousarray(blob, dtype=np.uint8)
+        return lib().oracle_pool_import_samples(self.h, _p(local_slots), C.c_uint32(len(local_slots)), _p(blob), C.c_uint64(len(blob)))
+
     def backing(self, kind):
         """numpy view (uint8) of a tier's backing frames: 0 HBM, 1 DRAM."""
         pages = self.cfg.hbm_pages if kind == 0 else self.cfg.host_pages

@@ -26,6 +26,7 @@ EXPORTS = (
     "pool_create", "pool_register_samples", "pool_write_embeddings", "pool_write_embeddings_noalloc",
     "pool_plan_microbatches", "plan_summary",
     "plan_arrays", "plan_destroy", "pool_gather_packed", "pool_free", "pool_status", "pool_stats",
+    "pool_backing", "pool_export_mapping", "pool_import_mapping", "pool_export_samples", "pool_import_samples",
     "pool_profile_enable", "pool_profile_read", "pool_debug_span_pages", "pool_debug_ring", "pool_debug_translate", "pool_destroy", "flowpool_last_cuda_error",
 )
 
@@ -94,6 +95,11 @@ def lib():
             "pool_free": [P, P, u32, P],
             "pool_status": [P, P, P],
             "pool_stats": [P, P],
+            "pool_backing": [P, P, P, P],
+            "pool_export_mapping": [P, P, u64, P],
+            "pool_import_mapping": [P, P, u64, P, P, P],
+            "pool_export_samples": [P, P, u32, P, u64, P, P],
+            "pool_import_samples": [P, P, u32, P, u64, P],
             "pool_profile_enable": [P, i32],
             "pool_profile_read": [P, P],
             "pool_debug_span_pages": [P, u32, u32, P, u32, P],
@@ -215,6 +221,43 @@ class Pool:
         if rc:
             raise FlowpoolError(rc, "pool_stats")
         return {k: getattr(s, k) for k, _ in PoolStats._fields_}
+
+    def backing(self):
+        """(hbm_base, host_base as the device sees it, text_base) of this pool's slabs."""
+        a, b, c = C.c_void_p(), C.c_void_p(), C.c_void_p()
+        rc = lib().pool_backing(self.h, C.byref(a), C.byref(b), C.byref(c))
+        if rc:
+            raise FlowpoolError(rc, "pool_backing")
+        return a.value or 0, b.value or 0, c.value or 0
+
+    def export_mapping(self):
+        n = C.c_uint64()
+        rc = lib().pool_export_mapping(self.h, None, 0, C.byref(n))
+        if rc:
+            return rc, None
+        buf = np.zeros(n.value, np.uint8)
+        rc = lib().pool_export_mapping(self.h, _p(buf), n.value, C.byref(n))
+        return rc, buf
+
+    def import_mapping(self, blob, peer_hbm_base, peer_host_base, peer_text_base):
+        blob = np.ascontiguousarray(blob, dtype=np.uint8)
+        return lib().pool_import_mapping(self.h, _p(blob), len(blob), peer_hbm_base or None, peer_host_base or None,
+                                         peer_text_base or None)
+
+    def export_samples(self, slots, stream: int = 0):
+        slots = _u32(slots)
+        n = C.c_uint64()
+        rc = lib().pool_export_samples(self.h, _p(slots), len(slots), None, 0, C.byref(n), stream or None)
+        if rc:
+            return rc, None
+        buf = np.zeros(n.value, np.uint8)
+        rc = lib().pool_export_samples(self.h, _p(slots), len(slots), _p(buf), n.value, C.byref(n), stream or None)
+        return rc, buf
+
+    def import_samples(self, local_slots, blob, stream: int = 0):
+        local_slots = _u32(local_slots)
+        blob = np.ascontiguousarray(blob, dtype=np.uint8)
+        return lib().pool_import_samples(self.h, _p(local_slots), len(local_slots), _p(blob), len(blob), stream or None)
 
     def profile_enable(self, on=True):
         return lib().pool_profile_enable(self.h, 1 if on else 0)

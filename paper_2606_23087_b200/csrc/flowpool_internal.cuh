@@ -3,6 +3,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <array>
 #include <vector>
 
 #include "../../include/flowpool.h"
@@ -17,6 +18,16 @@ constexpr uint64_t kPteValid = 1, kPteHost = 2, kPteText = 4, kPteFlagMask = 0xF
 struct RingState {
   uint32_t head;   // index of the oldest free entry
   uint32_t count;  // free entries
+};
+
+// Page tables of one process of the GVA space, as this process holds them (Sec. 3.2: every process keeps the
+// collected page tables locally).  Entry 'rank' is this process's own binding; the others are filled by
+// pool_import_mapping and stay empty (no pages) until then.
+struct PeerTables {
+  const uint64_t* pte_hbm;
+  const uint64_t* pte_host;
+  const uint64_t* pte_text;
+  uint64_t hbm_pages, host_pages, text_pages;
 };
 
 // Everything a kernel needs to know about a pool; passed by value.
@@ -36,6 +47,8 @@ struct PoolView {
   const uint64_t* pte_hbm;
   const uint64_t* pte_host;
   const uint64_t* pte_text;
+  const PeerTables* peers;   // [world_size] device array: every process's tables (own entry included)
+  uint32_t world_size;
   // FIFO free rings
   uint32_t* ring;   RingState* ring_state;   uint32_t ring_cap;    // embedding pages (global page index)
   uint32_t* tring;  RingState* tring_state;  uint32_t tring_cap;   // text pages
@@ -43,7 +56,8 @@ struct PoolView {
   // sample table (by slot)
   uint32_t* s_seq_len;
   uint32_t* s_n_spans;
-  uint32_t* s_text_pages;  // [max_samples][text_pages_per_sample] text page index
+  uint64_t* s_text_pages;  // [max_samples][text_pages_per_sample] text page GVA (own or a peer's)
+  uint32_t* s_flags;       // bit 0: the sample was imported (its pages and text pages belong to a peer)
   // span table (span id = slot * spans_per_sample + j)
   uint32_t* sp_pos;
   uint32_t* sp_tokens;
@@ -79,20 +93,26 @@ __device__ __forceinline__ uint64_t translate(const PoolView& v, uint64_t gva, u
   for (int t = 0; t < 2; ++t) {
     uint64_t d = gva - v.region_start[t];
     if (d >= v.region_bytes) continue;
-    uint64_t proc = d / v.max_size, o = d - proc * v.max_size;
-    if (proc != v.rank) return 0;
-    uint64_t pages = t == 0 ? v.hbm_pages : v.host_pages;
-    uint64_t vpn = o >> v.page_shift;
+    const uint64_t proc = d / v.max_size, o = d - proc * v.max_size;
+    uint64_t hbm_pages = v.hbm_pages, host_pages = v.host_pages, text_pages = v.text_pages;
+    const uint64_t *pte_hbm = v.pte_hbm, *pte_host = v.pte_host, *pte_text = v.pte_text;
+    if (proc != v.rank) {  // another process's segment: its imported tables (no pages if never imported)
+      const PeerTables pt = v.peers[proc];
+      hbm_pages = pt.hbm_pages; host_pages = pt.host_pages; text_pages = pt.text_pages;
+      pte_hbm = pt.pte_hbm; pte_host = pt.pte_host; pte_text = pt.pte_text;
+    }
+    const uint64_t pages = t == 0 ? hbm_pages : host_pages;
+    const uint64_t vpn = o >> v.page_shift;
     if (vpn < pages) {
       *offset = o & (v.page_bytes - 1);
-      return t == 0 ? v.pte_hbm[vpn] : v.pte_host[vpn];
+      return t == 0 ? pte_hbm[vpn] : pte_host[vpn];
     }
     if (t == 0) {
-      uint64_t ot = o - (pages << v.page_shift);
-      uint64_t tp = ot / FT_TEXT_PAGE_BYTES;
-      if (tp < v.text_pages) {
+      const uint64_t ot = o - (pages << v.page_shift);
+      const uint64_t tp = ot / FT_TEXT_PAGE_BYTES;
+      if (tp < text_pages) {
         *offset = ot % FT_TEXT_PAGE_BYTES;
-        return v.pte_text[tp];
+        return pte_text[tp];
       }
     }
     return 0;
@@ -183,6 +203,7 @@ enum { FT_SLOT_FREE = 0, FT_SLOT_REGISTERED = 1, FT_SLOT_READY = 2 };
 
 struct ft_slot_mirror {
   uint8_t state = FT_SLOT_FREE;
+  bool remote = false;  // imported from a peer: pages and text pages are not ours to recycle
   uint32_t seq_len = 0, n_spans = 0, spans_written = 0, n_text_pages = 0;
   uint64_t generation = 0;
 };
@@ -218,6 +239,11 @@ struct ft_pool {
   void* host_base = nullptr;   bool own_host = false;  // host pointer
   void* host_dev = nullptr;                            // the same memory as the device sees it
   void* d_scratch = nullptr;   size_t scratch_cap = 0; // per-call descriptors and scan outputs
+  std::vector<uint32_t> bind_hbm, bind_host;           // vpn -> frame of this process's binding (exported to peers)
+  void* d_text_base() const { return d_text; }
+  std::vector<void*> peer_allocs;                      // imported peers' page-table arrays
+  std::vector<uint8_t> peer_imported;                  // [world_size]
+  std::vector<std::array<uint64_t, 3>> peer_bases;     // [world_size] slab addresses (HBM, host, text) as seen here
   ft_staging staging;
   cudaStream_t side_stream = nullptr;                  // host-tier traffic runs beside the HBM kernels
   cudaEvent_t fork_ev = nullptr, join_ev = nullptr;
@@ -237,6 +263,8 @@ struct ft_pool {
 };
 
 namespace ft {
+__global__ void k_page_table_init(uint64_t* pte, const uint32_t* bind, uint64_t n, uint64_t base, uint64_t frame_bytes,
+                                  uint64_t flags);
 // uploads `bytes` from `src` (pageable) to the front of the pool's device scratch, asynchronously,
 // through the staging ring; afterwards at least `total_bytes` of scratch exist.  Returns the device pointer.
 // timing brackets around one kernel launch on `st` (no-ops unless profiling is on)
@@ -251,5 +279,6 @@ inline void prof_end(ft_pool* p, cudaStream_t st) {
   if (!p->profiling) return;
   cudaEventRecord(p->prof.back().e1, st);
 }
+size_t align_up_sz(size_t x, size_t a);
 int32_t stage_upload(ft_pool* p, const void* src, size_t bytes, size_t total_bytes, cudaStream_t st, void** d_out);
 }  // namespace ft

@@ -88,11 +88,15 @@ __global__ void __launch_bounds__(kGatherThreads) k_gather(PoolView v, PlanView 
         const bool in_run = lo > 0 && p < v.sp_pos[sid] + v.sp_tokens[sid];
         if (!in_run) {
           // token id, through the text page, then the embedding-table row
-          const uint32_t tp = v.s_text_pages[(uint64_t)slot * v.text_pages_per_sample + p / kTextPageIds];
+          const uint64_t tp_gva = v.s_text_pages[(uint64_t)slot * v.text_pages_per_sample + p / kTextPageIds];
           uint64_t off;
-          const uint64_t tpte = translate(v, v.text_gva_base + (uint64_t)tp * FT_TEXT_PAGE_BYTES, &off);
-          const int32_t id = reinterpret_cast<const int32_t*>(tpte & ~kPteFlagMask)[p % kTextPageIds];
-          if (id < 0 || (uint32_t)id >= a.vocab) {
+          const uint64_t tpte = translate(v, tp_gva, &off);
+          int32_t id = -1;
+          const bool text_ok = (tpte & kPteValid) && (tpte & kPteText);  // e.g. a peer's page whose mapping was never imported
+          if (text_ok) id = reinterpret_cast<const int32_t*>(tpte & ~kPteFlagMask)[p % kTextPageIds];
+          if (!text_ok) {
+            note_error(v, a.call_seq, FT_ERR_BAD_GVA, (uint32_t)out_row);
+          } else if (id < 0 || (uint32_t)id >= a.vocab) {
             note_error(v, a.call_seq, FT_ERR_BAD_TOKEN_ID, (uint32_t)out_row);
           } else {
             // a table row is one segment in device memory: the low address bits ride in off0

@@ -74,6 +74,7 @@ int32_t stage_upload(ft_pool* p, const void* src, size_t bytes, size_t total_byt
 }
 
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+size_t align_up_sz(size_t x, size_t a) { return align_up(x, a); }
 
 // ------------------------------------------------------------------------------------------
 // K1: page tables
@@ -113,6 +114,7 @@ __global__ void __launch_bounds__(1024) k_register_scan(PoolView v, RegisterCall
       const uint32_t slot = c.slot[i];
       v.s_seq_len[slot] = c.seq_len[i];
       v.s_n_spans[slot] = c.n_spans[i];
+      v.s_flags[slot] = 0;
       for (uint32_t j = 0; j < c.n_spans[i]; ++j) {
         const uint32_t sid = slot * v.spans_per_sample + j;
         v.sp_pos[sid] = c.span_pos[c.span_begin[i] + j];
@@ -149,9 +151,10 @@ __global__ void __launch_bounds__(256) k_register_ids(PoolView v, RegisterCall c
   __syncthreads();
   const uint32_t i = sh_i, k = b - c.tp_off[i], slot = c.slot[i];
   const uint32_t tp = v.tring[(c.head[0] + b) % v.tring_cap];
-  if (threadIdx.x == 0) v.s_text_pages[(uint64_t)slot * v.text_pages_per_sample + k] = tp;
+  const uint64_t tp_gva = v.text_gva_base + (uint64_t)tp * FT_TEXT_PAGE_BYTES;
+  if (threadIdx.x == 0) v.s_text_pages[(uint64_t)slot * v.text_pages_per_sample + k] = tp_gva;
   uint64_t off;
-  const uint64_t pte = translate(v, v.text_gva_base + (uint64_t)tp * FT_TEXT_PAGE_BYTES, &off);
+  const uint64_t pte = translate(v, tp_gva, &off);
   int32_t* dst = reinterpret_cast<int32_t*>(pte & ~kPteFlagMask);
   const uint32_t len = c.seq_len[i], p0 = k * kTextPageIds;
   const uint32_t cnt = min(kTextPageIds, len - p0);
@@ -431,13 +434,20 @@ struct FreeCall {
 };
 
 __global__ void __launch_bounds__(1024) k_free_scan(PoolView v, FreeCall c) {
+  // per span: list blocks to return, and pages to return unless the sample was imported (a peer owns them);
+  // per sample: text pages to return, likewise
   uint64_t cp = 0, cb = 0, ct = 0;
   const uint32_t m = max(c.n_spans, c.n_samples);
   for (uint32_t base = 0; base < m; base += blockDim.x) {
     uint32_t i = base + threadIdx.x;
     uint64_t k = 0, nb = 0, nt = 0;
-    if (i < c.n_spans) { k = v.sp_npages[c.span_id[i]]; nb = (k + kListBlock - 1) / kListBlock; }
-    if (i < c.n_samples) nt = (v.s_seq_len[c.slot[i]] + kTextPageIds - 1) / kTextPageIds;
+    if (i < c.n_spans) {
+      const uint32_t sid = c.span_id[i];
+      const uint32_t np = v.sp_npages[sid];
+      nb = (np + kListBlock - 1) / kListBlock;
+      k = (v.s_flags[sid / v.spans_per_sample] & 1) ? 0 : np;
+    }
+    if (i < c.n_samples && !(v.s_flags[c.slot[i]] & 1)) nt = (v.s_seq_len[c.slot[i]] + kTextPageIds - 1) / kTextPageIds;
     uint64_t tp, tb, tt;
     uint64_t ep = block_exclusive_scan(k, &tp);
     uint64_t eb = block_exclusive_scan(nb, &tb);
@@ -457,53 +467,66 @@ __global__ void __launch_bounds__(1024) k_free_scan(PoolView v, FreeCall c) {
   }
 }
 
-// threads [0, total_pages): one page each, pushed at the tail in canonical order;
-// threads [total_pages, total_pages + total_text): one text page each
-__global__ void __launch_bounds__(256) k_free_fill(PoolView v, FreeCall c, uint32_t total_pages, uint32_t total_text) {
-  const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
+__device__ __forceinline__ uint32_t last_le(const uint32_t* off, uint32_t n, uint32_t x) {
+  uint32_t lo = 0, hi = n;  // largest i with off[i] <= x (off[0] = 0)
+  while (hi - lo > 1) {
+    uint32_t mid = (lo + hi) >> 1;
+    if (off[mid] <= x) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+// threads [0, P): one page each, pushed at the tail in canonical order; [P, P+B): one list block each;
+// [P+B, P+B+T): one text page each
+__global__ void __launch_bounds__(256) k_free_fill(PoolView v, FreeCall c, uint32_t total_pages, uint32_t total_blocks,
+                                                  uint32_t total_text) {
+  uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
   if (t < total_pages) {
-    uint32_t lo = 0, hi = c.n_spans;
-    while (hi - lo > 1) {
-      uint32_t mid = (lo + hi) >> 1;
-      if (c.page_off[mid] <= t) lo = mid; else hi = mid;
-    }
-    const uint32_t q = lo, o = t - c.page_off[q], sid = c.span_id[q];
-    const uint32_t blk = v.sp_blocks[(uint64_t)sid * v.blocks_per_span + o / kListBlock];
-    const uint64_t gva = v.list_blocks[(uint64_t)blk * kListBlock + o % kListBlock];
-    v.ring[(c.tails[0] + t) % v.ring_cap] = global_page_of(v, gva);
-    if (o % kListBlock == 0) v.bring[(c.tails[1] + c.blk_off[q] + o / kListBlock) % v.bring_cap] = blk;
-    if (o == 0) v.sp_npages[sid] = 0;
-  } else if (t < total_pages + total_text) {
-    const uint32_t u = t - total_pages;
-    uint32_t lo = 0, hi = c.n_samples;
-    while (hi - lo > 1) {
-      uint32_t mid = (lo + hi) >> 1;
-      if (c.tp_off[mid] <= u) lo = mid; else hi = mid;
-    }
-    const uint32_t i = lo, k = u - c.tp_off[i], slot = c.slot[i];
-    v.tring[(c.tails[2] + u) % v.tring_cap] = v.s_text_pages[(uint64_t)slot * v.text_pages_per_sample + k];
+    // spans with no pages to return (imported) have equal consecutive offsets: last_le lands on the last of
+    // a run of equal offsets, which is the span that owns entry t
+    const uint32_t q = last_le(c.page_off, c.n_spans, t), o = t - c.page_off[q], sid = c.span_id[q];
+    v.ring[(c.tails[0] + t) % v.ring_cap] = global_page_of(v, span_page_gva(v, sid, o));
+    return;
+  }
+  t -= total_pages;
+  if (t < total_blocks) {
+    const uint32_t q = last_le(c.blk_off, c.n_spans, t), b = t - c.blk_off[q], sid = c.span_id[q];
+    v.bring[(c.tails[1] + t) % v.bring_cap] = v.sp_blocks[(uint64_t)sid * v.blocks_per_span + b];
+    return;
+  }
+  t -= total_blocks;
+  if (t < total_text) {
+    const uint32_t i = last_le(c.tp_off, c.n_samples, t), k = t - c.tp_off[i], slot = c.slot[i];
+    const uint64_t g = v.s_text_pages[(uint64_t)slot * v.text_pages_per_sample + k];
+    v.tring[(c.tails[2] + t) % v.tring_cap] = (uint32_t)((g - v.text_gva_base) / FT_TEXT_PAGE_BYTES);
   }
 }
 
 __global__ void k_free_clear(PoolView v, FreeCall c) {
   const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < c.n_samples) { v.s_seq_len[c.slot[i]] = 0; v.s_n_spans[c.slot[i]] = 0; }
+  if (i < c.n_spans) v.sp_npages[c.span_id[i]] = 0;
+  if (i < c.n_samples) { v.s_seq_len[c.slot[i]] = 0; v.s_n_spans[c.slot[i]] = 0; v.s_flags[c.slot[i]] = 0; }
 }
 
 __global__ void k_debug_translate(PoolView v, const uint64_t* gva, uint32_t n, uint32_t* kind, uint64_t* frame,
-                                  uint64_t* offset, int32_t* status, uint64_t hbm_base, uint64_t host_base,
-                                  uint64_t text_base) {
+                                  uint64_t* offset, int32_t* status, const uint64_t* bases /* [world][3] */) {
   const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n) return;
   uint64_t off = 0;
   const uint64_t pte = translate(v, gva[i], &off);
   if (!(pte & kPteValid)) { status[i] = FT_ERR_BAD_GVA; kind[i] = 0; frame[i] = 0; offset[i] = 0; return; }
+  // the owning process, to express the frame as an index into that process's slab
+  uint64_t proc = 0;
+  for (int t = 0; t < 2; ++t) {
+    const uint64_t d = gva[i] - v.region_start[t];
+    if (d < v.region_bytes) proc = d / v.max_size;
+  }
   const uint64_t addr = pte & ~kPteFlagMask;
   status[i] = FT_OK;
   offset[i] = off;
-  if (pte & kPteText) { kind[i] = 2; frame[i] = (addr - text_base) / FT_TEXT_PAGE_BYTES; }
-  else if (pte & kPteHost) { kind[i] = 1; frame[i] = (addr - host_base) >> v.page_shift; }
-  else { kind[i] = 0; frame[i] = (addr - hbm_base) >> v.page_shift; }
+  if (pte & kPteText) { kind[i] = 2; frame[i] = (addr - bases[3 * proc + 2]) / FT_TEXT_PAGE_BYTES; }
+  else if (pte & kPteHost) { kind[i] = 1; frame[i] = (addr - bases[3 * proc + 1]) >> v.page_shift; }
+  else { kind[i] = 0; frame[i] = (addr - bases[3 * proc]) >> v.page_shift; }
 }
 
 static inline uint64_t pages_for_tokens(const ft_pool* p, uint64_t n_tokens) {
@@ -529,6 +552,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_destroy(ft_pool* 
     if (p->staging.ev[i]) cudaEventDestroy(p->staging.ev[i]);
   }
   if (p->d_scratch) cudaFree(p->d_scratch);
+  for (void* a : p->peer_allocs) cudaFree(a);
   if (p->d_meta) cudaFree(p->d_meta);
   if (p->d_text) cudaFree(p->d_text);
   if (p->own_hbm && p->hbm_base) cudaFree(p->hbm_base);
@@ -615,7 +639,8 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_create(const ft_p
   const size_t o_ring = take(P * 4), o_tring = take(n_text * 4), o_bring = take(NB * 4);
   const size_t o_states = take(3 * sizeof(RingState)), o_status = take(32);  // status word, the gather's tile counter, the scatter's claim counters
   const size_t o_seq = take((size_t)c.max_samples * 4), o_nsp = take((size_t)c.max_samples * 4);
-  const size_t o_stp = take((size_t)c.max_samples * TPS * 4);
+  const size_t o_stp = take((size_t)c.max_samples * TPS * 8), o_sfl = take((size_t)c.max_samples * 4);
+  const size_t o_peers = take((size_t)c.world_size * sizeof(PeerTables));
   const size_t o_pos = take(span_ids * 4), o_tok = take(span_ids * 4), o_npg = take(span_ids * 4);
   const size_t o_blk = take(span_ids * MB * 4), o_lst = take(NB * kListBlock * 8);
   CK(cudaMalloc(&p->d_meta, off));
@@ -643,7 +668,10 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_create(const ft_p
   v.ring_state = st; v.tring_state = st + 1; v.bring_state = st + 2;
   v.status = reinterpret_cast<unsigned long long*>(m + o_status);
   v.s_seq_len = reinterpret_cast<uint32_t*>(m + o_seq); v.s_n_spans = reinterpret_cast<uint32_t*>(m + o_nsp);
-  v.s_text_pages = reinterpret_cast<uint32_t*>(m + o_stp);
+  v.s_text_pages = reinterpret_cast<uint64_t*>(m + o_stp);
+  v.s_flags = reinterpret_cast<uint32_t*>(m + o_sfl);
+  v.peers = reinterpret_cast<PeerTables*>(m + o_peers);
+  v.world_size = c.world_size;
   v.sp_pos = reinterpret_cast<uint32_t*>(m + o_pos); v.sp_tokens = reinterpret_cast<uint32_t*>(m + o_tok);
   v.sp_npages = reinterpret_cast<uint32_t*>(m + o_npg); v.sp_blocks = reinterpret_cast<uint32_t*>(m + o_blk);
   v.list_blocks = reinterpret_cast<uint64_t*>(m + o_lst);
@@ -680,8 +708,17 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_create(const ft_p
   RingState init[3] = {{0, (uint32_t)P}, {0, (uint32_t)n_text}, {0, (uint32_t)NB}};
   CK(cudaMemcpy(st, init, sizeof(init), cudaMemcpyHostToDevice));
   CK(cudaMemset(v.status, 0xFF, 8));
+  {  // this process's own entry of the collected page tables
+    PeerTables self{v.pte_hbm, v.pte_host, v.pte_text, v.hbm_pages, v.host_pages, v.text_pages};
+    CK(cudaMemcpy(const_cast<PeerTables*>(v.peers) + c.rank, &self, sizeof(self), cudaMemcpyHostToDevice));
+  }
+  p->peer_imported.assign(c.world_size, 0);
+  p->peer_imported[c.rank] = 1;
+  p->peer_bases.assign(c.world_size, {0, 0, 0});
+  p->peer_bases[c.rank] = {reinterpret_cast<uint64_t>(p->hbm_base), reinterpret_cast<uint64_t>(p->host_dev), reinterpret_cast<uint64_t>(p->d_text)};
   CK(cudaDeviceSynchronize());
   CK(cudaFree(d_tmp));
+  p->bind_hbm = bind_h; p->bind_host = bind_d;
   p->gpu_launches += 5;
 #undef CK
   p->slots.resize(c.max_samples);
@@ -918,9 +955,10 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_free(ft_pool* p, 
       const ft_span_mirror& m = p->spans[(uint64_t)slot[i] * S + j];
       if (!m.written) continue;
       span_ids.push_back(slot[i] * S + j);
-      pages += m.npages; blocks += (m.npages + kListBlock - 1) / kListBlock;
+      blocks += (m.npages + kListBlock - 1) / kListBlock;
+      if (!s.remote) pages += m.npages;  // an imported sample's pages belong to the peer that wrote them
     }
-    text += s.n_text_pages;
+    if (!s.remote) text += s.n_text_pages;
   }
   const uint32_t ns = (uint32_t)span_ids.size();
   const size_t o_sid = 0, o_slot = (size_t)ns * 4;
@@ -945,9 +983,9 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_free(ft_pool* p, 
   f.tp_off = reinterpret_cast<uint32_t*>(db + o_toff);
   f.tails = reinterpret_cast<uint32_t*>(db + o_tails);
   k_free_scan<<<1, 1024, 0, st>>>(p->view, f);
-  const uint64_t items = pages + text;
-  if (items) k_free_fill<<<(unsigned)((items + 255) / 256), 256, 0, st>>>(p->view, f, (uint32_t)pages, (uint32_t)text);
-  k_free_clear<<<(n + 255) / 256, 256, 0, st>>>(p->view, f);
+  const uint64_t items = pages + blocks + text;
+  if (items) k_free_fill<<<(unsigned)((items + 255) / 256), 256, 0, st>>>(p->view, f, (uint32_t)pages, (uint32_t)blocks, (uint32_t)text);
+  k_free_clear<<<(std::max(n, ns) + 255) / 256, 256, 0, st>>>(p->view, f);
   FT_CUDA(cudaGetLastError());
   p->gpu_launches += items ? 3 : 2;
 
@@ -1046,17 +1084,21 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_debug_translate(f
   if (!p || (n && (!gva || !kind || !frame || !offset || !status))) return FT_ERR_INVALID_ARG;
   if (n == 0) return FT_OK;
   uint8_t* d = nullptr;
-  const size_t bytes = (size_t)n * (8 + 4 + 8 + 8 + 4);
+  const size_t W = p->cfg.world_size;
+  const size_t bytes = (size_t)n * (8 + 4 + 8 + 8 + 4) + W * 24;
   FT_CUDA(cudaMalloc(&d, bytes));
   uint64_t* d_gva = reinterpret_cast<uint64_t*>(d);
   uint64_t* d_frame = d_gva + n;
   uint64_t* d_off = d_frame + n;
-  uint32_t* d_kind = reinterpret_cast<uint32_t*>(d_off + n);
+  uint64_t* d_bases = d_off + n;
+  uint32_t* d_kind = reinterpret_cast<uint32_t*>(d_bases + 3 * W);
   int32_t* d_status = reinterpret_cast<int32_t*>(d_kind + n);
+  std::vector<uint64_t> bases(3 * W, 0);
+  for (size_t r = 0; r < W; ++r)
+    if (r < p->peer_bases.size()) { bases[3 * r] = p->peer_bases[r][0]; bases[3 * r + 1] = p->peer_bases[r][1]; bases[3 * r + 2] = p->peer_bases[r][2]; }
+  FT_CUDA(cudaMemcpy(d_bases, bases.data(), 24 * W, cudaMemcpyHostToDevice));
   FT_CUDA(cudaMemcpy(d_gva, gva, (size_t)n * 8, cudaMemcpyHostToDevice));
-  k_debug_translate<<<(n + 255) / 256, 256>>>(p->view, d_gva, n, d_kind, d_frame, d_off, d_status,
-                                              reinterpret_cast<uint64_t>(p->hbm_base), reinterpret_cast<uint64_t>(p->host_dev),
-                                              reinterpret_cast<uint64_t>(p->d_text));
+  k_debug_translate<<<(n + 255) / 256, 256>>>(p->view, d_gva, n, d_kind, d_frame, d_off, d_status, d_bases);
   p->gpu_launches++;
   FT_CUDA(cudaDeviceSynchronize());
   FT_CUDA(cudaMemcpy(kind, d_kind, (size_t)n * 4, cudaMemcpyDeviceToHost));
