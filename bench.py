@@ -689,6 +689,85 @@ def run_sweep(args):
     print(json.dumps(line))
 
 
+# ---------------------------------------------------------------------------------------------
+# two processes of one GVA space, emulated on one GPU: producer pool (rank 1) -> consumer pool (rank 0)
+# ---------------------------------------------------------------------------------------------
+def run_peer(args):
+    """The producer writes the batch into its own segment; the consumer imports its mapping (once) and, per step,
+    the samples' descriptors, plans, and assembles every microbatch by reading the producer's pages in place.
+    With one GPU both segments live in the same HBM, so this measures the path's own overheads (descriptor
+    exchange, translation through imported tables), not a link."""
+    import torch
+    import workloads
+    from harness import pool_config_fields, plan_config_fields, register_args, write_args
+    from paper_2606_23087_b200 import binding as fp
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    st = torch.cuda.current_stream().cuda_stream
+    w = workloads.make_workload(args.workload, n_samples=args.samples, all_hbm=args.all_hbm)
+    n = w.n_samples
+
+    def cfg(rank):
+        f = pool_config_fields(w, max_samples=n)
+        f.update(world_size=2, rank=rank)
+        if rank == 0:  # the consumer holds no embeddings of its own here
+            f.update(hbm_pages=64, host_pages=0, max_imported_pages=w.hbm_pages + w.host_pages)
+        return f
+    prod, cons = fp.Pool(fp.PoolConfig(**cfg(1))), fp.Pool(fp.PoolConfig(**cfg(0)))
+    assert prod.rc == 0 and cons.rc == 0
+    rc, mblob = prod.export_mapping()
+    assert rc == 0 and cons.import_mapping(mblob, *prod.backing()) == 0
+    calls = []
+    for call in w.write_calls:
+        samples = sorted({s for s, _ in call}, key=[s for s, _ in call].index)
+        reg = register_args(w, samples)
+        calls.append((reg[:5], torch.from_numpy(reg[5]).cuda(), write_args(w, call),
+                      [workloads.span_values(w, s, j, device="cuda") for s, j in call]))
+    table = workloads.embed_table(w, device="cuda")
+    out = torch.empty((w.total_tokens, w.hidden), dtype=torch.bfloat16, device="cuda")
+    cu = torch.empty((2 * n + 8,), dtype=torch.int32, device="cuda")
+    pos = torch.empty((w.total_tokens,), dtype=torch.int32, device="cuda")
+    order = np.asarray(w.plan_order, dtype=np.uint32)
+    pcfg = fp.PlanConfig(**plan_config_fields(w))
+    cons.profile_enable(True)
+    xfer_ms, step_ms, blob_bytes = [], [], 0
+    for it in range(args.warmup + args.steps):
+        torch.cuda.synchronize()
+        t_step = time.perf_counter()
+        for reg, ids, wr, srcs in calls:
+            assert prod.register_samples(*reg, ids.data_ptr(), st) == 0
+            assert prod.write_embeddings(*wr, [t.data_ptr() for t in srcs], w.src_dtype, st) == 0
+        t0 = time.perf_counter()
+        rc, sblob = prod.export_samples(order, st)
+        assert rc == 0 and cons.import_samples(order, sblob, st) == 0
+        torch.cuda.synchronize()
+        dt = (time.perf_counter() - t0) * 1e3
+        rc, plan = cons.plan_microbatches(order, pcfg, st)
+        assert rc == 0
+        n_mb = plan.summary()[0]
+        if it == args.warmup:
+            cons.profile_read()
+        assert cons.gather_packed(plan, 0, n_mb, table.data_ptr(), w.vocab, out.data_ptr(), cu.data_ptr(), pos.data_ptr(), st) == 0
+        assert cons.free(order, st) == 0 and prod.free(order, st) == 0
+        plan.destroy()
+        torch.cuda.synchronize()
+        if it >= args.warmup:
+            xfer_ms.append(dt); step_ms.append((time.perf_counter() - t_step) * 1e3); blob_bytes = len(sblob)
+    prof = cons.profile_read()
+    assert cons.status() == (0, 0)
+    g_ms = (prof["gather_device"]["ms"] + 0.0) / args.steps
+    gh_ms = prof["gather_host"]["ms"] / args.steps
+    peak, _ = measured_peak()
+    gbs = 2 * w.total_tokens * w.row_bytes / max(g_ms, gh_ms) / 1e6
+    line = {"metric": "packed-microbatch assembly GB/s, consumer reading a peer process's pages (one GPU, emulated)",
+            "value": gbs, "unit": "GB/s", "n_gpus": 1, "higher_is_better": True, "dtype": "u8", "data": "synthetic",
+            "config": {"workload": workload_label(args), "ranks": 2, "note": "both segments in the same HBM"},
+            "gather_device_ms": g_ms, "gather_host_ms": gh_ms, "frac_of_measured_peak": gbs / peak,
+            "descriptor_export_import_ms": float(np.median(xfer_ms)), "descriptor_blob_bytes": blob_bytes,
+            "step_ms_host_wall": float(np.median(step_ms)), "microbatches": n_mb}
+    prod.destroy(); cons.destroy()
+    print(json.dumps(line))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -704,12 +783,15 @@ def main():
     ap.add_argument("--page-bytes", type=int, default=2 << 20, help="frag_sweep: page size")
     ap.add_argument("--pool-gib", type=float, default=64.0, help="frag_sweep: pool capacity")
     ap.add_argument("--cycles", type=int, default=10, help="frag_sweep: write/free cycles")
+    ap.add_argument("--via-peer", action="store_true", help="producer and consumer are two processes' pools of one GVA space")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         run_reference(args)
     elif args.workload == "frag_sweep":
         run_sweep(args)
+    elif args.via_peer:
+        run_peer(args)
     else:
         run_ours(args)
 

@@ -92,8 +92,9 @@ typedef struct {
   int32_t placeholder_id;   /* the image-placeholder token id */
   uint32_t ring_order;      /* FT_RING_* */
   uint32_t bind_order;      /* FT_BIND_* */
-  uint32_t world_size;      /* 0 => 1; only this process's binding exists in this build */
+  uint32_t world_size;      /* 0 => 1; processes of the GVA space (peers' bindings arrive by pool_import_mapping) */
   uint32_t rank;
+  uint64_t max_imported_pages; /* list-block budget for samples imported from peers (their pages are not local) */
 } ft_pool_config;
 
 /* Packing parameters (Sec. 3.4): budget L, integer cost A*sum(l) + B*lmax^2

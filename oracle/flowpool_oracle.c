@@ -59,6 +59,7 @@ typedef struct {
   int32_t placeholder_id;
   uint32_t ring_order, bind_order;
   uint32_t world_size, rank;
+  uint64_t max_imported_pages; /* a capacity knob of the device library; unused here */
 } oracle_pool_config;
 
 typedef struct {

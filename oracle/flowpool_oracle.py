@@ -28,7 +28,7 @@ class PoolConfig(C.Structure):
         ("hidden", C.c_uint32), ("max_samples", C.c_uint32), ("max_spans_per_sample", C.c_uint32),
         ("max_pages_per_span", C.c_uint32), ("max_seq_len", C.c_uint32),
         ("placeholder_id", C.c_int32), ("ring_order", C.c_uint32), ("bind_order", C.c_uint32),
-        ("world_size", C.c_uint32), ("rank", C.c_uint32),
+        ("world_size", C.c_uint32), ("rank", C.c_uint32), ("max_imported_pages", C.c_uint64),
     ]
 
 

@@ -243,6 +243,7 @@ struct ft_pool {
   void* d_text_base() const { return d_text; }
   std::vector<void*> peer_allocs;                      // imported peers' page-table arrays
   std::vector<uint8_t> peer_imported;                  // [world_size]
+  bool peer_host_frames = false;                       // some imported peer binds host-tier pages
   std::vector<std::array<uint64_t, 3>> peer_bases;     // [world_size] slab addresses (HBM, host, text) as seen here
   ft_staging staging;
   cudaStream_t side_stream = nullptr;                  // host-tier traffic runs beside the HBM kernels

@@ -246,10 +246,13 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_gather_packed(ft_
     const uint64_t ctas = (uint64_t)p->sm_count * std::min<uint64_t>(want_per_sm, (uint64_t)resident);
     kernel<<<(unsigned)std::min<uint64_t>(n_tiles, ctas), kGatherThreads, 0, s>>>(p->view, pv, args);
   };
-  const uint64_t per_sm = p->cfg.hbm_pages == 0 ? 1 : (uint64_t)p->dev_ctas_per_sm;
+  const uint64_t per_sm = (p->cfg.hbm_pages == 0 && p->cfg.world_size == 1) ? 1 : (uint64_t)p->dev_ctas_per_sm;
   const bool u8 = p->gather_unroll == 8;
-  if (p->cfg.host_pages == 0 || p->cfg.hbm_pages == 0) {
-    prof_begin(p, p->cfg.hbm_pages == 0 ? FT_K_GATHER_HOST : FT_K_GATHER_DEVICE, st);
+  // one launch when only one tier can be a source (own and imported bindings); otherwise one launch per tier
+  const bool host_sources = p->cfg.host_pages != 0 || p->peer_host_frames;
+  const bool only_host = p->cfg.hbm_pages == 0 && !(p->cfg.world_size > 1);
+  if (!host_sources || only_host) {
+    prof_begin(p, only_host ? FT_K_GATHER_HOST : FT_K_GATHER_DEVICE, st);
     if (u8) launch(k_gather<kTierAll, 8>, per_sm, a, st); else launch(k_gather<kTierAll, 4>, per_sm, a, st);
     prof_end(p, st);
     p->gpu_launches += 1;

@@ -184,6 +184,7 @@ FT_API int32_t pool_import_mapping(ft_pool* p, const void* buf, uint64_t bytes, 
   cudaFree(d_bind);
   p->peer_allocs.push_back(d_pte);
   p->peer_imported[h.rank] = 1;
+  if (h.host_pages) p->peer_host_frames = true;
   p->peer_bases[h.rank] = {reinterpret_cast<uint64_t>(peer_hbm_base), reinterpret_cast<uint64_t>(peer_host_base), reinterpret_cast<uint64_t>(peer_text_base)};
   return FT_OK;
 }

@@ -616,7 +616,10 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_create(const ft_p
   const uint32_t TPS = (c.max_seq_len + kTextPageIds - 1) / kTextPageIds;
   const uint32_t MB = (c.max_pages_per_span + kListBlock - 1) / kListBlock;
   const uint64_t span_ids = (uint64_t)c.max_samples * S;
-  const uint64_t NB = (P + kListBlock - 1) / kListBlock + std::min<uint64_t>(span_ids, P) + 1;
+  // list blocks: one per 64 pages plus at most one partial block per live span; imported samples bring pages that
+  // are not local, budgeted by max_imported_pages
+  const uint64_t imp = c.max_imported_pages;
+  const uint64_t NB = (P + imp + kListBlock - 1) / kListBlock + std::min<uint64_t>(span_ids, P + imp) + 1;
   if (NB > 0xFFFFFFFFull || span_ids > 0xFFFFFFFFull) { pool_destroy(p); return FT_ERR_INVALID_ARG; }
 
   // backing memory

@@ -28,7 +28,7 @@ def pool_config_fields(w, max_samples=None, ring_seed=11, bind_seed=12):
         max_samples=max_samples or w.n_samples, max_spans_per_sample=w.max_spans_per_sample,
         max_pages_per_span=w.max_pages_per_span, max_seq_len=w.max_seq_len,
         placeholder_id=w.placeholder_id, ring_order=w.ring_order, bind_order=w.bind_order,
-        world_size=1, rank=0,
+        world_size=1, rank=0, max_imported_pages=0,
     )
 
 

@@ -32,7 +32,7 @@ def test_binding_struct_layouts_match_the_header_order():
     fields = [f.strip() for decl in body.split(";") for f in decl.split(",") if f.strip()]
     names = [re.split(r"\s+", f)[-1] for f in fields]
     assert names == [n for n, _ in binding.PoolConfig._fields_]
-    assert ctypes.sizeof(binding.PoolConfig) == 9 * 8 + 10 * 4 + 0
+    assert ctypes.sizeof(binding.PoolConfig) == 9 * 8 + 10 * 4 + 8
     assert ctypes.sizeof(binding.PlanConfig) == 32
 
 

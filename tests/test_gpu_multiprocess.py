@@ -31,7 +31,7 @@ def test_consumer_reads_producer_pages_in_place(name, kw):
 
     def cfg(rank):
         f = pool_config_fields(w, max_samples=2 * n)
-        f.update(world_size=2, rank=rank, bind_seed=100 + rank, ring_seed=200 + rank)
+        f.update(world_size=2, rank=rank, bind_seed=100 + rank, ring_seed=200 + rank, max_imported_pages=w.hbm_pages + w.host_pages)
         return f
     g = {r: fp.Pool(fp.PoolConfig(**cfg(r))) for r in (0, 1)}
     o = {r: OraclePool(PoolConfig(**cfg(r))) for r in (0, 1)}
