@@ -249,6 +249,8 @@ struct ft_pool {
   cudaStream_t side_stream = nullptr;                  // host-tier traffic runs beside the HBM kernels
   cudaEvent_t fork_ev = nullptr, join_ev = nullptr;
   int sm_count = 148;
+  int occ_scatter[3][2] = {};   // resident CTAs/SM of k_scatter<tier mode, f32>, from the occupancy API
+  int occ_gather[3][2] = {};    // resident CTAs/SM of k_gather<tier mode, U = 4 | 8>
   int host_ctas = 8;            // grid of the host-tier copy kernels: few SMs, so that long-latency host-link
                                 // accesses do not clog the memory pipelines of the SMs that stream HBM
                                 // (FLOWPOOL_HOST_CTAS overrides)
@@ -264,6 +266,10 @@ struct ft_pool {
 };
 
 namespace ft {
+// per-device set-up of each translation unit's kernels (shared-memory opt-ins, occupancy), run by pool_create
+// with the pool's device current
+int32_t gather_device_setup(ft_pool* p);
+int32_t plan_device_setup(ft_pool* p);
 __global__ void k_page_table_init(uint64_t* pte, const uint32_t* bind, uint64_t n, uint64_t base, uint64_t frame_bytes,
                                   uint64_t flags);
 // uploads `bytes` from `src` (pageable) to the front of the pool's device scratch, asynchronously,

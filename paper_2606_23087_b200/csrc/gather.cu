@@ -204,6 +204,16 @@ __global__ void __launch_bounds__(32) k_gather_host_bulk(PoolView v, PlanView pl
 
 }  // namespace ft
 
+namespace ft {
+int32_t gather_device_setup(ft_pool* p) {
+  FT_CUDA(cudaFuncSetAttribute(k_gather_host_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBulkSmemBytes));
+  auto occ = [](auto kernel) { int v = 0; return cudaOccupancyMaxActiveBlocksPerMultiprocessor(&v, kernel, kGatherThreads, 0) == cudaSuccess && v > 0 ? v : 1; };
+  p->occ_gather[kTierAll][0] = occ(k_gather<kTierAll, 4>); p->occ_gather[kTierAll][1] = occ(k_gather<kTierAll, 8>);
+  p->occ_gather[kTierDeviceOnly][0] = occ(k_gather<kTierDeviceOnly, 4>); p->occ_gather[kTierDeviceOnly][1] = occ(k_gather<kTierDeviceOnly, 8>);
+  return FT_OK;
+}
+}  // namespace ft
+
 using namespace ft;
 
 extern "C" __attribute__((visibility("default"))) int32_t pool_gather_packed(ft_pool* p, const ft_plan* pl, uint32_t mb_begin, uint32_t mb_end,
@@ -240,10 +250,9 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_gather_packed(ft_
   const uint64_t n_tiles = (a.row_hi + kTileRows - 1) / kTileRows - a.row_lo / kTileRows;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   // the grid-stride tile loop assumes every CTA runs from the start: never launch more than fit at once
-  auto launch = [&](auto kernel, uint64_t want_per_sm, const GatherArgs& args, cudaStream_t s) {
-    int resident = 1;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, kernel, kGatherThreads, 0) != cudaSuccess || resident < 1) resident = 1;
-    const uint64_t ctas = (uint64_t)p->sm_count * std::min<uint64_t>(want_per_sm, (uint64_t)resident);
+  auto launch = [&](auto kernel, int mode, uint64_t want_per_sm, const GatherArgs& args, cudaStream_t s) {
+    const uint64_t resident = (uint64_t)std::max(1, p->occ_gather[mode][p->gather_unroll == 8 ? 1 : 0]);
+    const uint64_t ctas = (uint64_t)p->sm_count * std::min<uint64_t>(want_per_sm, resident);
     kernel<<<(unsigned)std::min<uint64_t>(n_tiles, ctas), kGatherThreads, 0, s>>>(p->view, pv, args);
   };
   const uint64_t per_sm = (p->cfg.hbm_pages == 0 && p->cfg.world_size == 1) ? 1 : (uint64_t)p->dev_ctas_per_sm;
@@ -253,7 +262,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_gather_packed(ft_
   const bool only_host = p->cfg.hbm_pages == 0 && !(p->cfg.world_size > 1);
   if (!host_sources || only_host) {
     prof_begin(p, only_host ? FT_K_GATHER_HOST : FT_K_GATHER_DEVICE, st);
-    if (u8) launch(k_gather<kTierAll, 8>, per_sm, a, st); else launch(k_gather<kTierAll, 4>, per_sm, a, st);
+    if (u8) launch(k_gather<kTierAll, 8>, kTierAll, per_sm, a, st); else launch(k_gather<kTierAll, 4>, kTierAll, per_sm, a, st);
     prof_end(p, st);
     p->gpu_launches += 1;
   } else {
@@ -261,17 +270,12 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_gather_packed(ft_
     FT_CUDA(cudaStreamWaitEvent(p->side_stream, p->fork_ev, 0));
     GatherArgs ah = a;
     ah.write_index = 0;
-    static bool attr_set = false;
-    if (!attr_set) {
-      FT_CUDA(cudaFuncSetAttribute(k_gather_host_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBulkSmemBytes));
-      attr_set = true;
-    }
     prof_begin(p, FT_K_GATHER_HOST, p->side_stream);
     k_gather_host_bulk<<<(unsigned)p->host_ctas, 32, kBulkSmemBytes, p->side_stream>>>(p->view, pv, ah);
     prof_end(p, p->side_stream);
     FT_CUDA(cudaEventRecord(p->join_ev, p->side_stream));
     prof_begin(p, FT_K_GATHER_DEVICE, st);
-    if (u8) launch(k_gather<kTierDeviceOnly, 8>, per_sm, a, st); else launch(k_gather<kTierDeviceOnly, 4>, per_sm, a, st);
+    if (u8) launch(k_gather<kTierDeviceOnly, 8>, kTierDeviceOnly, per_sm, a, st); else launch(k_gather<kTierDeviceOnly, 4>, kTierDeviceOnly, per_sm, a, st);
     prof_end(p, st);
     FT_CUDA(cudaStreamWaitEvent(st, p->join_ev, 0));
     p->gpu_launches += 2;

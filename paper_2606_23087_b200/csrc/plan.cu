@@ -326,6 +326,19 @@ static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; 
 
 }  // namespace ft
 
+namespace ft {
+constexpr size_t kBestfitSmemLimit = 227 * 1024 - 64;
+int32_t plan_device_setup(ft_pool* p) {
+  FT_CUDA(cudaFuncSetAttribute(k_bestfit, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBestfitSmemLimit));
+  // keep freed plan blocks cached in the device's default memory pool instead of returning them to the driver
+  cudaMemPool_t mp;
+  uint64_t keep = ~0ull;
+  if (cudaDeviceGetDefaultMemPool(&mp, p->device) == cudaSuccess) cudaMemPoolSetAttribute(mp, cudaMemPoolAttrReleaseThreshold, &keep);
+  cudaGetLastError();
+  return FT_OK;
+}
+}  // namespace ft
+
 using namespace ft;
 
 extern "C" __attribute__((visibility("default"))) int32_t plan_destroy(ft_plan* pl) {
@@ -388,14 +401,6 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_plan_microbatches
   const size_t o_bkt = take(n * 4), o_rank = take(n * 4), o_pos = take(n * 4), o_idx = take(n * 4);
   const size_t o_roff = take(((size_t)N + 1) * 4), o_rmbs = take(n * 4), o_rcnt = take((size_t)N * 4);
   const size_t o_tiles = take(n_tiles * 4), o_scal = take(SC_COUNT * 4);
-  static bool pool_tuned = false;
-  if (!pool_tuned) {  // keep freed plan blocks cached in the device's default memory pool instead of returning them
-    cudaMemPool_t mp;
-    uint64_t keep = ~0ull;
-    if (cudaDeviceGetDefaultMemPool(&mp, p->device) == cudaSuccess) cudaMemPoolSetAttribute(mp, cudaMemPoolAttrReleaseThreshold, &keep);
-    cudaGetLastError();
-    pool_tuned = true;
-  }
   pl->last_stream = st;
   cudaError_t e = cudaMallocAsync(&pl->d_block, off, st);
   if (e != cudaSuccess) { delete pl; return ft::cuda_fail(e, "cudaMalloc(plan)"); }
@@ -435,17 +440,12 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_plan_microbatches
   size_t words = 0;
   { uint32_t w = (L + 1 + 31) / 32; for (int l = 0; l < 4; ++l) { words += w; w = (w + 31) / 32; } }
   const size_t fixed = (words + 3 * (size_t)kFitChunk) * 4 + 16;
-  const size_t limit = 227 * 1024 - 64;
+  const size_t limit = kBestfitSmemLimit;
   const size_t head_bytes = ((size_t)L + 1) * 4;
   const uint32_t head_in_smem = fixed + head_bytes + 1024 * sizeof(MbRec) <= limit;
   size_t used = fixed + (head_in_smem ? head_bytes : 0);
   const uint32_t rec_cap = (uint32_t)std::min<size_t>(n, (limit - used) / sizeof(MbRec));
   used += (size_t)rec_cap * sizeof(MbRec);
-  static bool attr_set = false;
-  if (!attr_set) {
-    CK(cudaFuncSetAttribute(k_bestfit, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)limit));
-    attr_set = true;
-  }
   const uint32_t f_sort = (cfg->flags & FT_PLAN_SORT_DECREASING) != 0, f_sumsq = (cfg->flags & FT_PLAN_COST_SUMSQ) != 0;
   const uint32_t f_carry = (cfg->flags & FT_PLAN_ZIGZAG_CARRY) != 0;
   k_pack_order<<<gb, 256, 0, st>>>(pl->d_len, n, f_sort, d_pk_t, d_pk_len);

@@ -361,10 +361,7 @@ static void launch_scatter(ft_pool* p, const WriteCall& w, uint64_t total_chunks
   // one claim counter per stream the library launches on: main (word 2) and side (word 3) of the status block
   // (k_alloc_scan, which precedes every scatter launch of the call, zeroes them)
   unsigned long long* counter = p->view.status + (s == p->side_stream ? 3 : 2);
-  static int per_sm = 0;
-  if (per_sm == 0) {
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_scatter<MODE, F32>, 256, 0) != cudaSuccess || per_sm < 1) per_sm = 1;
-  }
+  const int per_sm = std::max(1, p->occ_scatter[MODE][F32 ? 1 : 0]);
   // HBM streams best with a bounded amount of loads in flight per SM; more resident warps only deepen the DRAM
   // queues (measured optimum: 4 CTAs/SM, one chunk per claim)
   const int want = p->scatter_ctas_per_sm > 0 ? p->scatter_ctas_per_sm : 4;
@@ -608,6 +605,15 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_create(const ft_p
   if (const char* e = getenv("FLOWPOOL_GATHER_U")) { int v = atoi(e); if (v == 4 || v == 8) p->gather_unroll = v; }
   if (const char* e = getenv("FLOWPOOL_DEV_CTAS_PER_SM")) { int v = atoi(e); if (v > 0) p->dev_ctas_per_sm = v; }
   CK(cudaStreamCreateWithFlags(&p->side_stream, cudaStreamNonBlocking));
+  // per-device kernel set-up: shared-memory opt-ins and occupancy of the data kernels
+  CK(cudaFuncSetAttribute(k_scatter_host_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBulkSmemBytes));
+  {
+    auto occ = [](auto kernel) { int v = 0; return cudaOccupancyMaxActiveBlocksPerMultiprocessor(&v, kernel, 256, 0) == cudaSuccess && v > 0 ? v : 1; };
+    p->occ_scatter[kTierAll][0] = occ(k_scatter<kTierAll, false>); p->occ_scatter[kTierAll][1] = occ(k_scatter<kTierAll, true>);
+    p->occ_scatter[kTierDeviceOnly][0] = occ(k_scatter<kTierDeviceOnly, false>); p->occ_scatter[kTierDeviceOnly][1] = occ(k_scatter<kTierDeviceOnly, true>);
+    p->occ_scatter[kTierHostOnly][0] = occ(k_scatter<kTierHostOnly, false>); p->occ_scatter[kTierHostOnly][1] = occ(k_scatter<kTierHostOnly, true>);
+  }
+  if ((rc = gather_device_setup(p)) != FT_OK || (rc = plan_device_setup(p)) != FT_OK) { pool_destroy(p); return rc; }
   CK(cudaEventCreateWithFlags(&p->fork_ev, cudaEventDisableTiming));
   CK(cudaEventCreateWithFlags(&p->join_ev, cudaEventDisableTiming));
 
@@ -905,11 +911,6 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings(
   } else {
     FT_CUDA(cudaEventRecord(p->fork_ev, st));
     FT_CUDA(cudaStreamWaitEvent(p->side_stream, p->fork_ev, 0));
-    static bool attr_set = false;
-    if (!attr_set) {
-      FT_CUDA(cudaFuncSetAttribute(k_scatter_host_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBulkSmemBytes));
-      attr_set = true;
-    }
     prof_begin(p, FT_K_SCATTER_HOST, p->side_stream);
     // bf16 source: bulk-async copies through shared memory.  fp32 source: the cast needs the values in
     // registers, and stores to host memory are posted (no latency to hide), so a few vector-store CTAs do it
@@ -1226,7 +1227,6 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings_
   if (c.host_pages == 0 || c.hbm_pages == 0) {
     launch(kTierAll, st);
   } else {
-    FT_CUDA(cudaFuncSetAttribute(k_scatter_host_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBulkSmemBytes));
     FT_CUDA(cudaEventRecord(p->fork_ev, st));
     FT_CUDA(cudaStreamWaitEvent(p->side_stream, p->fork_ev, 0));
     if (f32) {
