@@ -57,77 +57,99 @@ __global__ void __launch_bounds__(256) k_pack_order(const uint32_t* __restrict__
   if (t < n) { pk_t[r] = t; pk_len[r] = lt; }
 }
 
+// Residual bitmap: bit r of level 0 is set when some open microbatch has residual r; bit i of level k+1 is set
+// when word i of level k is non-zero.  Four levels of 32-ary words cover residuals below 2^20.
 struct FitLevels {
-  uint32_t* bits[4];
-  uint32_t words[4];
+  uint32_t *b0, *b1, *b2, *b3;
+  uint32_t w0, w1, w2, w3;
 };
 
+// smallest set index >= l, or kNone: the best-fit query (the segment-tree descent of Algorithm 1, 32-ary)
 __device__ __forceinline__ uint32_t fit_find(const FitLevels& f, uint32_t l) {
-  // smallest set index >= l, or kNone
-  uint32_t idx = l;
-#pragma unroll
-  for (int lvl = 0; lvl < 4; ++lvl) {
-    const uint32_t w = idx >> 5, b = idx & 31;
-    if (w < f.words[lvl]) {
-      const uint32_t m = f.bits[lvl][w] & (0xFFFFFFFFu << b);
-      if (m) {
-        uint32_t pos = (w << 5) + __ffs(m) - 1;
-        for (int d = lvl - 1; d >= 0; --d) pos = (pos << 5) + __ffs(f.bits[d][pos]) - 1;
-        return pos;
-      }
-    }
-    idx = w + 1;
+  uint32_t w = l >> 5;
+  uint32_t m = w < f.w0 ? f.b0[w] & (0xFFFFFFFFu << (l & 31)) : 0;
+  if (m) return (w << 5) + __ffs(m) - 1;
+  uint32_t i1 = w + 1;
+  w = i1 >> 5;
+  m = w < f.w1 ? f.b1[w] & (0xFFFFFFFFu << (i1 & 31)) : 0;
+  if (m) {
+    const uint32_t p0 = (w << 5) + __ffs(m) - 1;
+    return (p0 << 5) + __ffs(f.b0[p0]) - 1;
+  }
+  uint32_t i2 = w + 1;
+  w = i2 >> 5;
+  m = w < f.w2 ? f.b2[w] & (0xFFFFFFFFu << (i2 & 31)) : 0;
+  if (m) {
+    const uint32_t p1 = (w << 5) + __ffs(m) - 1;
+    const uint32_t p0 = (p1 << 5) + __ffs(f.b1[p1]) - 1;
+    return (p0 << 5) + __ffs(f.b0[p0]) - 1;
+  }
+  uint32_t i3 = w + 1;
+  w = i3 >> 5;
+  m = w < f.w3 ? f.b3[w] & (0xFFFFFFFFu << (i3 & 31)) : 0;
+  if (m) {
+    const uint32_t p2 = (w << 5) + __ffs(m) - 1;
+    const uint32_t p1 = (p2 << 5) + __ffs(f.b2[p2]) - 1;
+    const uint32_t p0 = (p1 << 5) + __ffs(f.b1[p1]) - 1;
+    return (p0 << 5) + __ffs(f.b0[p0]) - 1;
   }
   return kNone;
 }
 __device__ __forceinline__ void fit_set(const FitLevels& f, uint32_t r) {
-#pragma unroll
-  for (int lvl = 0; lvl < 4; ++lvl) {
-    const uint32_t old = f.bits[lvl][r >> 5];
-    f.bits[lvl][r >> 5] = old | (1u << (r & 31));
-    if (old) return;
-    r >>= 5;
-  }
+  uint32_t old = f.b0[r >> 5];
+  f.b0[r >> 5] = old | (1u << (r & 31));
+  if (old) return;
+  r >>= 5; old = f.b1[r >> 5]; f.b1[r >> 5] = old | (1u << (r & 31));
+  if (old) return;
+  r >>= 5; old = f.b2[r >> 5]; f.b2[r >> 5] = old | (1u << (r & 31));
+  if (old) return;
+  r >>= 5; f.b3[r >> 5] |= 1u << (r & 31);
 }
 __device__ __forceinline__ void fit_clear(const FitLevels& f, uint32_t r) {
-#pragma unroll
-  for (int lvl = 0; lvl < 4; ++lvl) {
-    const uint32_t nw = f.bits[lvl][r >> 5] & ~(1u << (r & 31));
-    f.bits[lvl][r >> 5] = nw;
-    if (nw) return;
-    r >>= 5;
-  }
+  uint32_t nw = f.b0[r >> 5] & ~(1u << (r & 31));
+  f.b0[r >> 5] = nw;
+  if (nw) return;
+  r >>= 5; nw = f.b1[r >> 5] & ~(1u << (r & 31)); f.b1[r >> 5] = nw;
+  if (nw) return;
+  r >>= 5; nw = f.b2[r >> 5] & ~(1u << (r & 31)); f.b2[r >> 5] = nw;
+  if (nw) return;
+  r >>= 5; f.b3[r >> 5] &= ~(1u << (r & 31));
 }
 
 // One block.  Thread 0 walks the samples in order (the dependency chain of online best fit); the other
 // threads stage lengths in and results out, coalesced, and initialise / flush the tables.
+// HEAD_SMEM: the per-residual stack heads live in shared memory (budgets up to about 32 K), else in global.
+template <bool HEAD_SMEM>
 __global__ void __launch_bounds__(1024) k_bestfit(const uint32_t* __restrict__ len, uint32_t n, uint32_t L,
-                                                  uint32_t* head_g, MbRec* recs_g, uint32_t head_in_smem,
+                                                  uint32_t* __restrict__ head_g, MbRec* __restrict__ recs_g,
                                                   uint32_t rec_smem_cap, uint32_t* sample_mb, uint32_t* sample_rank,
                                                   uint32_t* mb_residual, uint32_t* mb_tokens, uint32_t* mb_lmax,
                                                   uint32_t* mb_count, uint32_t* scalars) {
   extern __shared__ uint32_t sm[];
   FitLevels f;
   uint32_t* p = sm;
-  uint32_t w = (L + 1 + 31) / 32;
-  uint32_t total_words = 0;
-  for (int lvl = 0; lvl < 4; ++lvl) {
-    f.bits[lvl] = p; f.words[lvl] = w; p += w; total_words += w;
-    w = (w + 31) / 32;
-  }
+  f.w0 = (L + 1 + 31) / 32; f.b0 = p; p += f.w0;
+  f.w1 = (f.w0 + 31) / 32;  f.b1 = p; p += f.w1;
+  f.w2 = (f.w1 + 31) / 32;  f.b2 = p; p += f.w2;
+  f.w3 = (f.w2 + 31) / 32;  f.b3 = p; p += f.w3;
+  const uint32_t total_words = (uint32_t)(p - sm);
   uint32_t* c_len = p; p += kFitChunk;
   uint32_t* c_mb = p; p += kFitChunk;
   uint32_t* c_rank = p; p += kFitChunk;
-  uint32_t* head = head_g;
-  if (head_in_smem) { head = p; p += L + 1; }
+  uint32_t* head_s = p;
+  if (HEAD_SMEM) p += L + 1;
   p += (4 - ((p - sm) & 3)) & 3;  // 16-byte align the records
   MbRec* recs_s = reinterpret_cast<MbRec*>(p);
 
   for (uint32_t i = threadIdx.x; i < total_words; i += blockDim.x) sm[i] = 0;
-  for (uint32_t i = threadIdx.x; i <= L; i += blockDim.x) head[i] = kNone;
+  if (HEAD_SMEM) { for (uint32_t i = threadIdx.x; i <= L; i += blockDim.x) head_s[i] = kNone; }
+  else { for (uint32_t i = threadIdx.x; i <= L; i += blockDim.x) head_g[i] = kNone; }
   __shared__ uint32_t s_nmb;
   if (threadIdx.x == 0) s_nmb = 0;
   __syncthreads();
+
+  auto head_ld = [&](uint32_t r) -> uint32_t { return HEAD_SMEM ? head_s[r] : head_g[r]; };
+  auto head_st = [&](uint32_t r, uint32_t v) { if (HEAD_SMEM) head_s[r] = v; else head_g[r] = v; };
 
   for (uint32_t base = 0; base < n; base += kFitChunk) {
     const uint32_t cnt = min(kFitChunk, n - base);
@@ -141,9 +163,9 @@ __global__ void __launch_bounds__(1024) k_bestfit(const uint32_t* __restrict__ l
         uint32_t j;
         MbRec rec;
         if (r != kNone) {
-          j = head[r];  // most recently changed microbatch with that residual
-          rec = j < rec_smem_cap ? recs_s[j] : recs_g[j];
-          head[r] = rec.next;
+          j = head_ld(r);  // most recently changed microbatch with that residual
+          if (j < rec_smem_cap) rec = recs_s[j]; else rec = recs_g[j];
+          head_st(r, rec.next);
           if (rec.next == kNone) fit_clear(f, r);
           rec.residual = r - l;
           rec.lmax = max(rec.lmax, l);
@@ -154,8 +176,8 @@ __global__ void __launch_bounds__(1024) k_bestfit(const uint32_t* __restrict__ l
         }
         // a residual of 0 can never be chosen again (l >= 1): it needs no stack entry
         if (rec.residual) {
-          rec.next = head[rec.residual];
-          head[rec.residual] = j;
+          rec.next = head_ld(rec.residual);
+          head_st(rec.residual, j);
           if (rec.next == kNone) fit_set(f, rec.residual);
         } else {
           rec.next = kNone;
@@ -329,7 +351,8 @@ static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; 
 namespace ft {
 constexpr size_t kBestfitSmemLimit = 227 * 1024 - 64;
 int32_t plan_device_setup(ft_pool* p) {
-  FT_CUDA(cudaFuncSetAttribute(k_bestfit, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBestfitSmemLimit));
+  FT_CUDA(cudaFuncSetAttribute(k_bestfit<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBestfitSmemLimit));
+  FT_CUDA(cudaFuncSetAttribute(k_bestfit<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBestfitSmemLimit));
   // keep freed plan blocks cached in the device's default memory pool instead of returning them to the driver
   cudaMemPool_t mp;
   uint64_t keep = ~0ull;
@@ -449,9 +472,12 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_plan_microbatches
   const uint32_t f_sort = (cfg->flags & FT_PLAN_SORT_DECREASING) != 0, f_sumsq = (cfg->flags & FT_PLAN_COST_SUMSQ) != 0;
   const uint32_t f_carry = (cfg->flags & FT_PLAN_ZIGZAG_CARRY) != 0;
   k_pack_order<<<gb, 256, 0, st>>>(pl->d_len, n, f_sort, d_pk_t, d_pk_len);
-  k_bestfit<<<1, 1024, used, st>>>(d_pk_len, n, L, d_head, d_recs, head_in_smem, rec_cap, d_pk_mb,
-                                   pl->d_sample_rank, pl->d_mb_residual, pl->d_mb_tokens, pl->d_mb_lmax, pl->d_mb_count,
-                                   pl->d_scalars);
+  if (head_in_smem)
+    k_bestfit<true><<<1, 1024, used, st>>>(d_pk_len, n, L, d_head, d_recs, rec_cap, d_pk_mb, pl->d_sample_rank,
+                                           pl->d_mb_residual, pl->d_mb_tokens, pl->d_mb_lmax, pl->d_mb_count, pl->d_scalars);
+  else
+    k_bestfit<false><<<1, 1024, used, st>>>(d_pk_len, n, L, d_head, d_recs, rec_cap, d_pk_mb, pl->d_sample_rank,
+                                            pl->d_mb_residual, pl->d_mb_tokens, pl->d_mb_lmax, pl->d_mb_count, pl->d_scalars);
   k_mb_finalize<<<1, 1024, 0, st>>>(pl->d_mb_tokens, pl->d_mb_count, pl->d_mb_sample_off, pl->d_mb_row_off, pl->d_scalars);
   k_plan_scatter<<<gb, 256, 0, st>>>(pl->d_slots, d_pk_t, d_pk_len, d_pk_mb, pl->d_sample_rank, pl->d_mb_sample_off, n,
                                      pl->d_mb_samples, pl->d_plan_len, pl->d_plan_sample_mb, pl->d_sample_mb);
