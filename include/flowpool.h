@@ -15,6 +15,12 @@
  *    Host arrays are read before the call returns.  Device work is enqueued on
  *    the caller's stream (`stream` = a cudaStream_t passed as void*; NULL = the
  *    legacy default stream); ordering between calls is stream order.
+ *  - Two streams per pool are supported: a producer side (register, write, import, free) and a consumer side
+ *    (plan, export, gather) may be issued, from one host thread, on two different streams so that the encoder's
+ *    scatter of the next batch overlaps the backbone's assembly of the current one (the decoupled
+ *    producer-consumer flow of Sec. 3.1).  The library orders the sides itself: a consumer-side call waits for
+ *    the producer-side calls issued before it, and pool_free waits for the consumer-side calls issued before it;
+ *    the sides use separate scratch and separate side streams for host-tier traffic.
  *  - One caller thread per pool.  The caller owns every buffer it passes in
  *    (backing memory, sources, table, outputs); the library owns its metadata
  *    and anything it allocated itself.
@@ -279,6 +285,17 @@ int32_t pool_free(ft_pool* pool, const uint32_t* sample_slot, uint32_t n, void* 
 int32_t pool_status(ft_pool* pool, int32_t* first_device_error, uint64_t* detail);
 
 int32_t pool_stats(ft_pool* pool, ft_pool_stats* out);
+
+/*
+ * Ready queue (Sec. 3.1: "after sufficient paired embeddings accumulate in the pool, the scheduler ... constructs
+ * microbatches").  Samples enter a FIFO in the order in which they became READY (last span written, text-only
+ * registration, import).  pool_ready_count reports the live entries and their tokens.  pool_take_ready pops up
+ * to max_samples slots in that order, but only once at least min_tokens tokens are ready (the watermark):
+ * otherwise NOT_READY and nothing is taken.  Entries of samples freed in the meantime are skipped.  Host only.
+ */
+int32_t pool_ready_count(ft_pool* pool, uint32_t* n_samples, uint64_t* n_tokens);
+int32_t pool_take_ready(ft_pool* pool, uint64_t min_tokens, uint32_t max_samples, uint32_t* slots_out /* host */,
+                        uint32_t* n_out, uint64_t* tokens_out);
 
 /*
  * More than one process in the GVA space (Sec. 3.2: "each process exports its memory mapping information to all

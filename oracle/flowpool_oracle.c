@@ -108,6 +108,8 @@ typedef struct oracle_pool {
   uint32_t* tring;
   uint64_t tring_head, tring_count;
   or_sample* samples;
+  /* samples in the order in which they became ready (slot, generation) */
+  uint32_t* rq_slot; uint64_t* rq_gen; uint64_t rq_head, rq_tail, rq_cap;
   /* first asynchronous ("device-side") error: smallest (call, code, detail) */
   uint64_t call_seq;
   uint64_t status_key; /* UINT64_MAX = none */
@@ -238,6 +240,17 @@ static uint8_t* resolve(oracle_pool* p, uint64_t g) {
   return pr->text_mem + frame * TEXT_PAGE_BYTES + off;
 }
 
+/* Sec. 3.1: the scheduler acts once "sufficient paired embeddings accumulate": a FIFO of samples in the order in
+ * which they became ready (reading: completion order; the watermark is a token count chosen by the caller). */
+static void ready_push(oracle_pool* p, uint32_t slot) {
+  if (p->rq_tail == p->rq_cap) {
+    p->rq_cap = p->rq_cap ? 2 * p->rq_cap : 64;
+    p->rq_slot = (uint32_t*)realloc(p->rq_slot, p->rq_cap * sizeof(uint32_t));
+    p->rq_gen = (uint64_t*)realloc(p->rq_gen, p->rq_cap * sizeof(uint64_t));
+  }
+  p->rq_slot[p->rq_tail] = slot; p->rq_gen[p->rq_tail] = p->samples[slot].generation; p->rq_tail++;
+}
+
 static void note_async_error(oracle_pool* p, int32_t code, uint32_t detail) {
   uint64_t key = (p->call_seq << 40) | ((uint64_t)(uint32_t)(-code) << 32) | detail;
   if (key < p->status_key) p->status_key = key;
@@ -334,7 +347,7 @@ int32_t oracle_pool_destroy(oracle_pool* p) {
   for (uint32_t i = 0; i < p->c.max_samples; ++i) release_sample_storage(&p->samples[i]);
   for (uint32_t i = 0; i < p->c.world_size; ++i)
     if (i != p->c.rank && p->peers[i].present) { free(p->peers[i].bind_hbm); free(p->peers[i].bind_host); }
-  free(p->peers);
+  free(p->peers); free(p->rq_slot); free(p->rq_gen);
   free(p->samples); free(p->ring); free(p->tring); free(p->bind_hbm); free(p->bind_host);
   free(p->hbm_mem); free(p->host_mem); free(p->text_mem); free(p);
   return OR_OK;
@@ -382,6 +395,7 @@ int32_t oracle_pool_register_samples(oracle_pool* p, uint32_t n, const uint32_t*
   for (uint32_t i = 0; i < n; ++i) {
     or_sample* s = &p->samples[slot[i]];
     s->state = n_spans[i] == 0 ? SLOT_READY : SLOT_REGISTERED; /* text-only: paired at once */
+    if (s->state == SLOT_READY) ready_push(p, slot[i]);
     s->seq_len = seq_len[i]; s->n_spans = n_spans[i]; s->spans_written = 0; s->remote = 0;
     s->spans = (or_span*)calloc(n_spans[i] + 1, sizeof(or_span));
     uint64_t placeholders = 0;
@@ -484,7 +498,7 @@ int32_t oracle_pool_write_embeddings(oracle_pool* p, uint32_t n_spans, const uin
       b += run;
     }
     s->spans_written++;
-    if (s->spans_written == s->n_spans) s->state = SLOT_READY; /* "paired" */
+    if (s->spans_written == s->n_spans) { s->state = SLOT_READY; ready_push(p, slot[q]); } /* "paired" */
   }
   return OR_OK;
 }
@@ -973,6 +987,7 @@ int32_t oracle_pool_import_samples(oracle_pool* p, const uint32_t* local_slot, u
   for (uint32_t i = 0; i < n; ++i) {
     or_sample* s = &p->samples[local_slot[i]];
     s->state = SLOT_READY; s->remote = 1;
+    ready_push(p, local_slot[i]);
     s->seq_len = (uint32_t)r[0]; s->n_spans = (uint32_t)r[1]; s->n_text_pages = (uint32_t)r[2];
     s->spans_written = s->n_spans;
     r += 3;
@@ -986,6 +1001,44 @@ int32_t oracle_pool_import_samples(oracle_pool* p, const uint32_t* local_slot, u
     s->text_pages = (uint64_t*)malloc(8 * (s->n_text_pages + 1));
     for (uint32_t k = 0; k < s->n_text_pages; ++k) s->text_pages[k] = *r++;
   }
+  return OR_OK;
+}
+
+static int ready_live(const oracle_pool* p, uint64_t i) {
+  const or_sample* s = &p->samples[p->rq_slot[i]];
+  return s->state == SLOT_READY && s->generation == p->rq_gen[i];
+}
+
+int32_t oracle_pool_ready_count(oracle_pool* p, uint32_t* n_samples, uint64_t* n_tokens) {
+  if (!p) return OR_ERR_INVALID_ARG;
+  uint32_t n = 0; uint64_t tok = 0;
+  for (uint64_t i = p->rq_head; i < p->rq_tail; ++i)
+    if (ready_live(p, i)) { ++n; tok += p->samples[p->rq_slot[i]].seq_len; }
+  if (n_samples) *n_samples = n;
+  if (n_tokens) *n_tokens = tok;
+  return OR_OK;
+}
+
+/* pops up to max_samples ready samples in completion order once min_tokens tokens are ready; entries of samples
+ * freed since are skipped */
+int32_t oracle_pool_take_ready(oracle_pool* p, uint64_t min_tokens, uint32_t max_samples, uint32_t* slots_out,
+                               uint32_t* n_out, uint64_t* tokens_out) {
+  if (!p || !n_out || (max_samples && !slots_out)) return OR_ERR_INVALID_ARG;
+  *n_out = 0;
+  if (tokens_out) *tokens_out = 0;
+  uint64_t avail = 0;
+  for (uint64_t i = p->rq_head; i < p->rq_tail; ++i)
+    if (ready_live(p, i)) avail += p->samples[p->rq_slot[i]].seq_len;
+  if (avail < min_tokens || avail == 0) return OR_ERR_NOT_READY;
+  uint32_t n = 0; uint64_t tok = 0;
+  while (p->rq_head < p->rq_tail && n < max_samples) {
+    uint64_t i = p->rq_head++;
+    if (!ready_live(p, i)) continue;
+    slots_out[n++] = p->rq_slot[i];
+    tok += p->samples[p->rq_slot[i]].seq_len;
+  }
+  *n_out = n;
+  if (tokens_out) *tokens_out = tok;
   return OR_OK;
 }
 

@@ -258,6 +258,17 @@ class OraclePool:
         blob = np.ascontiguousarray(blob, dtype=np.uint8)
         return lib().oracle_pool_import_samples(self.h, _p(local_slots), C.c_uint32(len(local_slots)), _p(blob), C.c_uint64(len(blob)))
 
+    def ready_count(self):
+        n, t = C.c_uint32(), C.c_uint64()
+        lib().oracle_pool_ready_count(self.h, C.byref(n), C.byref(t))
+        return n.value, t.value
+
+    def take_ready(self, min_tokens, max_samples):
+        out = np.zeros(max(1, max_samples), np.uint32)
+        n, t = C.c_uint32(), C.c_uint64()
+        rc = lib().oracle_pool_take_ready(self.h, C.c_uint64(min_tokens), C.c_uint32(max_samples), _p(out), C.byref(n), C.byref(t))
+        return rc, out[: n.value].copy(), t.value
+
     def backing(self, kind):
         """numpy view (uint8) of a tier's backing frames: 0 HBM, 1 DRAM."""
         pages = self.cfg.hbm_pages if kind == 0 else self.cfg.host_pages

@@ -26,7 +26,7 @@ EXPORTS = (
     "pool_create", "pool_register_samples", "pool_write_embeddings", "pool_write_embeddings_noalloc",
     "pool_plan_microbatches", "plan_summary",
     "plan_arrays", "plan_destroy", "pool_gather_packed", "pool_free", "pool_status", "pool_stats",
-    "pool_backing", "pool_export_mapping", "pool_import_mapping", "pool_export_samples", "pool_import_samples",
+    "pool_ready_count", "pool_take_ready", "pool_backing", "pool_export_mapping", "pool_import_mapping", "pool_export_samples", "pool_import_samples",
     "pool_profile_enable", "pool_profile_read", "pool_debug_span_pages", "pool_debug_ring", "pool_debug_translate", "pool_destroy", "flowpool_last_cuda_error",
 )
 
@@ -95,6 +95,8 @@ def lib():
             "pool_free": [P, P, u32, P],
             "pool_status": [P, P, P],
             "pool_stats": [P, P],
+            "pool_ready_count": [P, P, P],
+            "pool_take_ready": [P, u64, u32, P, P, P],
             "pool_backing": [P, P, P, P],
             "pool_export_mapping": [P, P, u64, P],
             "pool_import_mapping": [P, P, u64, P, P, P],
@@ -221,6 +223,19 @@ class Pool:
         if rc:
             raise FlowpoolError(rc, "pool_stats")
         return {k: getattr(s, k) for k, _ in PoolStats._fields_}
+
+    def ready_count(self):
+        n, t = C.c_uint32(), C.c_uint64()
+        rc = lib().pool_ready_count(self.h, C.byref(n), C.byref(t))
+        if rc:
+            raise FlowpoolError(rc, "pool_ready_count")
+        return n.value, t.value
+
+    def take_ready(self, min_tokens, max_samples):
+        out = np.zeros(max(1, max_samples), np.uint32)
+        n, t = C.c_uint32(), C.c_uint64()
+        rc = lib().pool_take_ready(self.h, min_tokens, max_samples, _p(out), C.byref(n), C.byref(t))
+        return rc, out[: n.value].copy(), t.value
 
     def backing(self):
         """(hbm_base, host_base as the device sees it, text_base) of this pool's slabs."""

@@ -4,6 +4,8 @@
 #include <stdint.h>
 
 #include <array>
+#include <deque>
+#include <utility>
 #include <vector>
 
 #include "../../include/flowpool.h"
@@ -238,7 +240,9 @@ struct ft_pool {
   void* hbm_base = nullptr;    bool own_hbm = false;
   void* host_base = nullptr;   bool own_host = false;  // host pointer
   void* host_dev = nullptr;                            // the same memory as the device sees it
-  void* d_scratch = nullptr;   size_t scratch_cap = 0; // per-call descriptors and scan outputs
+  // per-call descriptors and scan outputs: one arena per side, so that a producer call and a consumer call issued on
+  // different streams never share scratch (0 = register/write/import/free, 1 = plan/export)
+  void* d_scratch[2] = {nullptr, nullptr};   size_t scratch_cap[2] = {0, 0};
   std::vector<uint32_t> bind_hbm, bind_host;           // vpn -> frame of this process's binding (exported to peers)
   void* d_text_base() const { return d_text; }
   std::vector<void*> peer_allocs;                      // imported peers' page-table arrays
@@ -246,8 +250,16 @@ struct ft_pool {
   bool peer_host_frames = false;                       // some imported peer binds host-tier pages
   std::vector<std::array<uint64_t, 3>> peer_bases;     // [world_size] slab addresses (HBM, host, text) as seen here
   ft_staging staging;
-  cudaStream_t side_stream = nullptr;                  // host-tier traffic runs beside the HBM kernels
-  cudaEvent_t fork_ev = nullptr, join_ev = nullptr;
+  // host-tier traffic runs beside the HBM kernels on a side stream: one per side (0 producer, 1 consumer), so that
+  // host-tier writes and host-tier reads of concurrent calls can use both directions of the link at once
+  cudaStream_t side_stream[2] = {nullptr, nullptr};
+  cudaEvent_t fork_ev[2] = {nullptr, nullptr}, join_ev[2] = {nullptr, nullptr};
+  // cross-stream ordering when the producer side and the consumer side are driven from different streams
+  cudaEvent_t ev_producer = nullptr, ev_consumer = nullptr;  // end of the latest producer-side / consumer-side call
+  cudaStream_t last_producer_stream = nullptr, last_consumer_stream = nullptr;
+  bool have_producer_ev = false, have_consumer_ev = false;
+  // samples in the order in which they became READY (slot, generation), for pool_take_ready
+  std::deque<std::pair<uint32_t, uint64_t>> ready_fifo;
   int sm_count = 148;
   int occ_scatter[3][2] = {};   // resident CTAs/SM of k_scatter<tier mode, f32>, from the occupancy API
   int occ_gather[3][2] = {};    // resident CTAs/SM of k_gather<tier mode, U = 4 | 8>
@@ -287,5 +299,28 @@ inline void prof_end(ft_pool* p, cudaStream_t st) {
   cudaEventRecord(p->prof.back().e1, st);
 }
 size_t align_up_sz(size_t x, size_t a);
-int32_t stage_upload(ft_pool* p, const void* src, size_t bytes, size_t total_bytes, cudaStream_t st, void** d_out);
+// (arena: 0 = producer-side calls, 1 = consumer-side calls)
+int32_t stage_upload(ft_pool* p, int arena, const void* src, size_t bytes, size_t total_bytes, cudaStream_t st, void** d_out);
+
+// Cross-stream ordering (the producer side and the consumer side of a pool may be driven from two streams):
+// a consumer-side call waits for the producer-side calls issued before it; pool_free waits for the consumer-side
+// calls issued before it.  Same-stream use costs one event record per call and no wait.
+inline int32_t begin_consumer(ft_pool* p, cudaStream_t st) {
+  if (p->have_producer_ev && p->last_producer_stream != st) FT_CUDA(cudaStreamWaitEvent(st, p->ev_producer, 0));
+  return FT_OK;
+}
+inline int32_t end_consumer(ft_pool* p, cudaStream_t st) {
+  FT_CUDA(cudaEventRecord(p->ev_consumer, st));
+  p->have_consumer_ev = true; p->last_consumer_stream = st;
+  return FT_OK;
+}
+inline int32_t begin_free(ft_pool* p, cudaStream_t st) {
+  if (p->have_consumer_ev && p->last_consumer_stream != st) FT_CUDA(cudaStreamWaitEvent(st, p->ev_consumer, 0));
+  return FT_OK;
+}
+inline int32_t end_producer(ft_pool* p, cudaStream_t st) {
+  FT_CUDA(cudaEventRecord(p->ev_producer, st));
+  p->have_producer_ev = true; p->last_producer_stream = st;
+  return FT_OK;
+}
 }  // namespace ft

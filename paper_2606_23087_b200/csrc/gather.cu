@@ -245,6 +245,10 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_gather_packed(ft_
   a.table = static_cast<const uint8_t*>(embed_table); a.vocab = vocab;
   a.out = static_cast<uint8_t*>(out_embeds); a.cu = out_cu; a.pos_ids = out_pos;
   a.call_seq = p->call_seq; a.write_index = 1;
+  {
+    const int32_t rc0 = begin_consumer(p, static_cast<cudaStream_t>(stream));  // writes issued on another stream come first
+    if (rc0 != FT_OK) return rc0;
+  }
   a.tile_counter = p->view.status + 1;  // scratch word next to the status word
   FT_CUDA(cudaMemsetAsync(a.tile_counter, 0, 8, static_cast<cudaStream_t>(stream)));
   const uint64_t n_tiles = (a.row_hi + kTileRows - 1) / kTileRows - a.row_lo / kTileRows;
@@ -266,22 +270,22 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_gather_packed(ft_
     prof_end(p, st);
     p->gpu_launches += 1;
   } else {
-    FT_CUDA(cudaEventRecord(p->fork_ev, st));
-    FT_CUDA(cudaStreamWaitEvent(p->side_stream, p->fork_ev, 0));
+    FT_CUDA(cudaEventRecord(p->fork_ev[1], st));
+    FT_CUDA(cudaStreamWaitEvent(p->side_stream[1], p->fork_ev[1], 0));
     GatherArgs ah = a;
     ah.write_index = 0;
-    prof_begin(p, FT_K_GATHER_HOST, p->side_stream);
-    k_gather_host_bulk<<<(unsigned)p->host_ctas, 32, kBulkSmemBytes, p->side_stream>>>(p->view, pv, ah);
-    prof_end(p, p->side_stream);
-    FT_CUDA(cudaEventRecord(p->join_ev, p->side_stream));
+    prof_begin(p, FT_K_GATHER_HOST, p->side_stream[1]);
+    k_gather_host_bulk<<<(unsigned)p->host_ctas, 32, kBulkSmemBytes, p->side_stream[1]>>>(p->view, pv, ah);
+    prof_end(p, p->side_stream[1]);
+    FT_CUDA(cudaEventRecord(p->join_ev[1], p->side_stream[1]));
     prof_begin(p, FT_K_GATHER_DEVICE, st);
     if (u8) launch(k_gather<kTierDeviceOnly, 8>, kTierDeviceOnly, per_sm, a, st); else launch(k_gather<kTierDeviceOnly, 4>, kTierDeviceOnly, per_sm, a, st);
     prof_end(p, st);
-    FT_CUDA(cudaStreamWaitEvent(st, p->join_ev, 0));
+    FT_CUDA(cudaStreamWaitEvent(st, p->join_ev[1], 0));
     p->gpu_launches += 2;
   }
   const_cast<ft_plan*>(pl)->last_stream = st;
   FT_CUDA(cudaGetLastError());
   p->bytes_gathered += (a.row_hi - a.row_lo) * 2ull * p->view.row_bytes;
-  return FT_OK;
+  return end_consumer(p, st);
 }

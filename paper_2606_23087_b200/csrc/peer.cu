@@ -245,7 +245,9 @@ FT_API int32_t pool_export_samples(ft_pool* p, const uint32_t* slot, uint32_t n,
   memcpy(blob.data() + o_tpoff, tp_off.data(), (size_t)(n + 1) * 4);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   void* d = nullptr;
-  int32_t rc = stage_upload(p, blob.data(), blob_bytes, total_bytes, st, &d);
+  int32_t rc = begin_consumer(p, st);  // the lists may still be being written on another stream
+  if (rc != FT_OK) return rc;
+  rc = stage_upload(p, 1, blob.data(), blob_bytes, total_bytes, st, &d);
   if (rc != FT_OK) return rc;
   uint8_t* db = static_cast<uint8_t*>(d);
   ListCall lc{ns, n, reinterpret_cast<uint32_t*>(db + o_sid), reinterpret_cast<uint32_t*>(db + o_poff),
@@ -256,7 +258,7 @@ FT_API int32_t pool_export_samples(ft_pool* p, const uint32_t* slot, uint32_t n,
   p->gpu_launches++;
   FT_CUDA(cudaMemcpyAsync(pg, db + o_out, 8 * items, cudaMemcpyDeviceToHost, st));
   FT_CUDA(cudaStreamSynchronize(st));
-  return FT_OK;
+  return end_consumer(p, st);
 }
 
 FT_API int32_t pool_import_samples(ft_pool* p, const uint32_t* local_slot, uint32_t n, const void* buf, uint64_t bytes,
@@ -328,7 +330,7 @@ FT_API int32_t pool_import_samples(ft_pool* p, const uint32_t* local_slot, uint3
   memcpy(blob.data() + o_tpoff, tpoff.data(), 4ull * (n + 1));
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   void* d = nullptr;
-  int32_t rc = stage_upload(p, blob.data(), blob_bytes, total_bytes, st, &d);
+  int32_t rc = stage_upload(p, 0, blob.data(), blob_bytes, total_bytes, st, &d);
   if (rc != FT_OK) return rc;
   uint8_t* db = static_cast<uint8_t*>(d);
   auto U = [&](size_t o) { return reinterpret_cast<uint32_t*>(db + o); };
@@ -343,6 +345,7 @@ FT_API int32_t pool_import_samples(ft_pool* p, const uint32_t* local_slot, uint3
   for (uint32_t i = 0, g = 0; i < n; ++i) {
     ft_slot_mirror& s = p->slots[local_slot[i]];
     s.state = FT_SLOT_READY; s.remote = true;
+    p->ready_fifo.emplace_back(local_slot[i], s.generation);
     s.seq_len = seq[i]; s.n_spans = nsp[i]; s.spans_written = nsp[i]; s.n_text_pages = ps[3 * i + 2];
     for (uint32_t j = 0; j < nsp[i]; ++j, ++g) {
       ft_span_mirror& m = p->spans[(uint64_t)local_slot[i] * S + j];
@@ -351,5 +354,5 @@ FT_API int32_t pool_import_samples(ft_pool* p, const uint32_t* local_slot, uint3
     p->live_samples++; p->live_spans += nsp[i];
   }
   p->free_blocks -= blocks;
-  return FT_OK;
+  return end_producer(p, st);
 }

@@ -449,9 +449,12 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_plan_microbatches
     cudaError_t e__ = (call);                                                               \
     if (e__ != cudaSuccess) { rc = ft::cuda_fail(e__, #call); plan_destroy(pl); return rc; } \
   } while (0)
+  // the sample table may still be being written on another stream
+  rc = begin_consumer(p, st);
+  if (rc != FT_OK) { plan_destroy(pl); return rc; }
   // the slot list goes up through the pool's staging ring (scratch front), then into the plan
   void* d_up = nullptr;
-  rc = stage_upload(p, slot, (size_t)n * 4, (size_t)n * 4, st, &d_up);
+  rc = stage_upload(p, 1, slot, (size_t)n * 4, (size_t)n * 4, st, &d_up);
   if (rc != FT_OK) { plan_destroy(pl); return rc; }
   CK(cudaMemcpyAsync(pl->d_slots, d_up, (size_t)n * 4, cudaMemcpyDeviceToDevice, st));
   CK(cudaMemsetAsync(pl->d_rank_cnt, 0, (size_t)N * 4, st));
@@ -504,6 +507,8 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_plan_microbatches
   CK(cudaMemcpy(pl->h_mb_sample_off.data(), pl->d_mb_sample_off, ((size_t)pl->n_mb + 1) * 4, cudaMemcpyDeviceToHost));
   CK(cudaMemcpy(pl->h_mb_row_off.data(), pl->d_mb_row_off, ((size_t)pl->n_mb + 1) * 8, cudaMemcpyDeviceToHost));
 #undef CK
+  rc = end_consumer(p, st);
+  if (rc != FT_OK) { plan_destroy(pl); return rc; }
   *out = pl;
   return FT_OK;
 }

@@ -43,7 +43,7 @@ static void seeded_shuffle(std::vector<uint32_t>& a, uint64_t seed) {
   }
 }
 
-int32_t stage_upload(ft_pool* p, const void* src, size_t bytes, size_t total_bytes, cudaStream_t st, void** d_out) {
+int32_t stage_upload(ft_pool* p, int arena, const void* src, size_t bytes, size_t total_bytes, cudaStream_t st, void** d_out) {
   ft_staging& s = p->staging;
   const int i = s.next;
   s.next = (i + 1) % ft_staging::kBufs;
@@ -58,18 +58,18 @@ int32_t stage_upload(ft_pool* p, const void* src, size_t bytes, size_t total_byt
     s.cap[i] = cap;
   }
   memcpy(s.h[i], src, bytes);
-  if (p->scratch_cap < total_bytes) {
-    if (p->d_scratch) FT_CUDA(cudaFree(p->d_scratch));  // synchronises: no kernel still reads the old scratch
+  if (p->scratch_cap[arena] < total_bytes) {
+    if (p->d_scratch[arena]) FT_CUDA(cudaFree(p->d_scratch[arena]));  // synchronises: no kernel still reads the old scratch
     size_t cap = 1 << 20;
     while (cap < total_bytes) cap <<= 1;
-    p->d_scratch = nullptr; p->scratch_cap = 0;
-    FT_CUDA(cudaMalloc(&p->d_scratch, cap));
-    p->scratch_cap = cap;
+    p->d_scratch[arena] = nullptr; p->scratch_cap[arena] = 0;
+    FT_CUDA(cudaMalloc(&p->d_scratch[arena], cap));
+    p->scratch_cap[arena] = cap;
   }
-  FT_CUDA(cudaMemcpyAsync(p->d_scratch, s.h[i], bytes, cudaMemcpyHostToDevice, st));
+  FT_CUDA(cudaMemcpyAsync(p->d_scratch[arena], s.h[i], bytes, cudaMemcpyHostToDevice, st));
   FT_CUDA(cudaEventRecord(s.ev[i], st));
   s.busy[i] = true;
-  *d_out = p->d_scratch;
+  *d_out = p->d_scratch[arena];
   return FT_OK;
 }
 
@@ -360,7 +360,7 @@ template <int MODE, bool F32>
 static void launch_scatter(ft_pool* p, const WriteCall& w, uint64_t total_chunks, uint64_t max_ctas, cudaStream_t s) {
   // one claim counter per stream the library launches on: main (word 2) and side (word 3) of the status block
   // (k_alloc_scan, which precedes every scatter launch of the call, zeroes them)
-  unsigned long long* counter = p->view.status + (s == p->side_stream ? 3 : 2);
+  unsigned long long* counter = p->view.status + (s == p->side_stream[0] ? 3 : 2);
   const int per_sm = std::max(1, p->occ_scatter[MODE][F32 ? 1 : 0]);
   // HBM streams best with a bounded amount of loads in flight per SM; more resident warps only deepen the DRAM
   // queues (measured optimum: 4 CTAs/SM, one chunk per claim)
@@ -548,15 +548,19 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_destroy(ft_pool* 
     if (p->staging.h[i]) cudaFreeHost(p->staging.h[i]);
     if (p->staging.ev[i]) cudaEventDestroy(p->staging.ev[i]);
   }
-  if (p->d_scratch) cudaFree(p->d_scratch);
+  for (int a = 0; a < 2; ++a) if (p->d_scratch[a]) cudaFree(p->d_scratch[a]);
   for (void* a : p->peer_allocs) cudaFree(a);
   if (p->d_meta) cudaFree(p->d_meta);
   if (p->d_text) cudaFree(p->d_text);
   if (p->own_hbm && p->hbm_base) cudaFree(p->hbm_base);
   if (p->own_host && p->host_base) cudaFreeHost(p->host_base);
-  if (p->side_stream) cudaStreamDestroy(p->side_stream);
-  if (p->fork_ev) cudaEventDestroy(p->fork_ev);
-  if (p->join_ev) cudaEventDestroy(p->join_ev);
+  for (int a = 0; a < 2; ++a) {
+    if (p->side_stream[a]) cudaStreamDestroy(p->side_stream[a]);
+    if (p->fork_ev[a]) cudaEventDestroy(p->fork_ev[a]);
+    if (p->join_ev[a]) cudaEventDestroy(p->join_ev[a]);
+  }
+  if (p->ev_producer) cudaEventDestroy(p->ev_producer);
+  if (p->ev_consumer) cudaEventDestroy(p->ev_consumer);
   delete p;
   cudaGetLastError();
   return FT_OK;
@@ -604,7 +608,13 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_create(const ft_p
   if (const char* e = getenv("FLOWPOOL_SCATTER_CTAS_PER_SM")) { int v = atoi(e); if (v > 0) p->scatter_ctas_per_sm = v; }
   if (const char* e = getenv("FLOWPOOL_GATHER_U")) { int v = atoi(e); if (v == 4 || v == 8) p->gather_unroll = v; }
   if (const char* e = getenv("FLOWPOOL_DEV_CTAS_PER_SM")) { int v = atoi(e); if (v > 0) p->dev_ctas_per_sm = v; }
-  CK(cudaStreamCreateWithFlags(&p->side_stream, cudaStreamNonBlocking));
+  for (int a = 0; a < 2; ++a) {
+    CK(cudaStreamCreateWithFlags(&p->side_stream[a], cudaStreamNonBlocking));
+    CK(cudaEventCreateWithFlags(&p->fork_ev[a], cudaEventDisableTiming));
+    CK(cudaEventCreateWithFlags(&p->join_ev[a], cudaEventDisableTiming));
+  }
+  CK(cudaEventCreateWithFlags(&p->ev_producer, cudaEventDisableTiming));
+  CK(cudaEventCreateWithFlags(&p->ev_consumer, cudaEventDisableTiming));
   // per-device kernel set-up: shared-memory opt-ins and occupancy of the data kernels
   CK(cudaFuncSetAttribute(k_scatter_host_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBulkSmemBytes));
   {
@@ -614,8 +624,6 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_create(const ft_p
     p->occ_scatter[kTierHostOnly][0] = occ(k_scatter<kTierHostOnly, false>); p->occ_scatter[kTierHostOnly][1] = occ(k_scatter<kTierHostOnly, true>);
   }
   if ((rc = gather_device_setup(p)) != FT_OK || (rc = plan_device_setup(p)) != FT_OK) { pool_destroy(p); return rc; }
-  CK(cudaEventCreateWithFlags(&p->fork_ev, cudaEventDisableTiming));
-  CK(cudaEventCreateWithFlags(&p->join_ev, cudaEventDisableTiming));
 
   const uint64_t P = c.hbm_pages + c.host_pages;
   const uint32_t S = c.max_spans_per_sample;
@@ -789,7 +797,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_register_samples(
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   void* d = nullptr;
-  int32_t rc = stage_upload(p, blob.data(), blob_bytes, total_bytes, st, &d);
+  int32_t rc = stage_upload(p, 0, blob.data(), blob_bytes, total_bytes, st, &d);
   if (rc != FT_OK) return rc;
   uint8_t* db = static_cast<uint8_t*>(d);
   RegisterCall rcall;
@@ -815,6 +823,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_register_samples(
   for (uint32_t i = 0; i < n; ++i) {
     ft_slot_mirror& s = p->slots[slot[i]];
     s.state = n_spans[i] == 0 ? FT_SLOT_READY : FT_SLOT_REGISTERED;
+    if (s.state == FT_SLOT_READY) p->ready_fifo.emplace_back(slot[i], s.generation);  // text only: paired at once
     s.seq_len = seq_len[i]; s.n_spans = n_spans[i]; s.spans_written = 0;
     s.n_text_pages = (seq_len[i] + kTextPageIds - 1) / kTextPageIds;
     for (uint32_t j = 0; j < n_spans[i]; ++j, ++sp) {
@@ -824,7 +833,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_register_samples(
     p->live_samples++; p->live_spans += n_spans[i];
   }
   p->free_text_pages -= text_need;
-  return FT_OK;
+  return end_producer(p, st);
 }
 
 extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings(ft_pool* p, uint32_t n, const uint32_t* slot, const uint32_t* span_idx,
@@ -877,7 +886,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings(
   memcpy(blob.data() + o_ntk, n_tokens, (size_t)n * 4);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   void* d = nullptr;
-  int32_t rc = stage_upload(p, blob.data(), blob_bytes, total_bytes, st, &d);
+  int32_t rc = stage_upload(p, 0, blob.data(), blob_bytes, total_bytes, st, &d);
   if (rc != FT_OK) return rc;
   uint8_t* db = static_cast<uint8_t*>(d);
   WriteCall w;
@@ -909,21 +918,21 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings(
   } else if (c.hbm_pages == 0) {
     launch(kTierAll, st);
   } else {
-    FT_CUDA(cudaEventRecord(p->fork_ev, st));
-    FT_CUDA(cudaStreamWaitEvent(p->side_stream, p->fork_ev, 0));
-    prof_begin(p, FT_K_SCATTER_HOST, p->side_stream);
+    FT_CUDA(cudaEventRecord(p->fork_ev[0], st));
+    FT_CUDA(cudaStreamWaitEvent(p->side_stream[0], p->fork_ev[0], 0));
+    prof_begin(p, FT_K_SCATTER_HOST, p->side_stream[0]);
     // bf16 source: bulk-async copies through shared memory.  fp32 source: the cast needs the values in
     // registers, and stores to host memory are posted (no latency to hide), so a few vector-store CTAs do it
     if (f32) {
-      launch_scatter<kTierHostOnly, true>(p, w, total_chunks, (uint64_t)p->host_ctas, p->side_stream);
+      launch_scatter<kTierHostOnly, true>(p, w, total_chunks, (uint64_t)p->host_ctas, p->side_stream[0]);
     } else {
-      k_scatter_host_bulk<<<(unsigned)p->host_ctas, 32, kBulkSmemBytes, p->side_stream>>>(p->view, w, p->call_seq);
+      k_scatter_host_bulk<<<(unsigned)p->host_ctas, 32, kBulkSmemBytes, p->side_stream[0]>>>(p->view, w, p->call_seq);
     }
-    prof_end(p, p->side_stream);
+    prof_end(p, p->side_stream[0]);
     p->gpu_launches++;
-    FT_CUDA(cudaEventRecord(p->join_ev, p->side_stream));
+    FT_CUDA(cudaEventRecord(p->join_ev[0], p->side_stream[0]));
     launch(kTierDeviceOnly, st);
-    FT_CUDA(cudaStreamWaitEvent(st, p->join_ev, 0));
+    FT_CUDA(cudaStreamWaitEvent(st, p->join_ev[0], 0));
   }
   FT_CUDA(cudaGetLastError());
 
@@ -931,11 +940,11 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings(
     ft_slot_mirror& s = p->slots[slot[q]];
     ft_span_mirror& m = p->spans[span_id[q]];
     m.written = true; m.npages = (uint32_t)pages_for_tokens(p, n_tokens[q]);
-    if (++s.spans_written == s.n_spans) s.state = FT_SLOT_READY;
+    if (++s.spans_written == s.n_spans) { s.state = FT_SLOT_READY; p->ready_fifo.emplace_back(slot[q], s.generation); }
   }
   p->free_pages -= need; p->free_blocks -= need_blocks;
   p->bytes_written += bytes_total * (f32 ? 3 : 2);
-  return FT_OK;
+  return end_producer(p, st);
 }
 
 extern "C" __attribute__((visibility("default"))) int32_t pool_free(ft_pool* p, const uint32_t* slot, uint32_t n, void* stream) {
@@ -975,7 +984,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_free(ft_pool* p, 
   memcpy(blob.data() + o_slot, slot, (size_t)n * 4);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   void* d = nullptr;
-  int32_t rc = stage_upload(p, blob.data(), blob_bytes, total_bytes, st, &d);
+  int32_t rc = stage_upload(p, 0, blob.data(), blob_bytes, total_bytes, st, &d);
   if (rc != FT_OK) return rc;
   uint8_t* db = static_cast<uint8_t*>(d);
   FreeCall f;
@@ -986,6 +995,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_free(ft_pool* p, 
   f.blk_off = reinterpret_cast<uint32_t*>(db + o_boff);
   f.tp_off = reinterpret_cast<uint32_t*>(db + o_toff);
   f.tails = reinterpret_cast<uint32_t*>(db + o_tails);
+  if ((rc = begin_free(p, st)) != FT_OK) return rc;  // a gather issued earlier on another stream may still read these pages
   k_free_scan<<<1, 1024, 0, st>>>(p->view, f);
   const uint64_t items = pages + blocks + text;
   if (items) k_free_fill<<<(unsigned)((items + 255) / 256), 256, 0, st>>>(p->view, f, (uint32_t)pages, (uint32_t)blocks, (uint32_t)text);
@@ -1003,6 +1013,46 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_free(ft_pool* p, 
   }
   p->free_pages += pages; p->free_blocks += blocks; p->free_text_pages += text;
   p->free_epoch++;
+  return end_producer(p, st);
+}
+
+extern "C" __attribute__((visibility("default"))) int32_t pool_ready_count(ft_pool* p, uint32_t* n_samples, uint64_t* n_tokens) {
+  if (!p) return FT_ERR_INVALID_ARG;
+  uint32_t n = 0;
+  uint64_t tok = 0;
+  for (const auto& e : p->ready_fifo) {
+    const ft_slot_mirror& s = p->slots[e.first];
+    if (s.state == FT_SLOT_READY && s.generation == e.second) { ++n; tok += s.seq_len; }
+  }
+  if (n_samples) *n_samples = n;
+  if (n_tokens) *n_tokens = tok;
+  return FT_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int32_t pool_take_ready(ft_pool* p, uint64_t min_tokens, uint32_t max_samples,
+                                                                         uint32_t* slots_out, uint32_t* n_out, uint64_t* tokens_out) {
+  if (!p || !n_out || (max_samples && !slots_out)) return FT_ERR_INVALID_ARG;
+  *n_out = 0;
+  if (tokens_out) *tokens_out = 0;
+  // drop entries whose sample was freed (or freed and re-registered) since it became ready
+  auto live = [&](const std::pair<uint32_t, uint64_t>& e) {
+    const ft_slot_mirror& s = p->slots[e.first];
+    return s.state == FT_SLOT_READY && s.generation == e.second;
+  };
+  uint64_t avail = 0;
+  for (const auto& e : p->ready_fifo) if (live(e)) avail += p->slots[e.first].seq_len;
+  if (avail < min_tokens || avail == 0) return FT_ERR_NOT_READY;  // not enough paired embeddings have accumulated
+  uint32_t n = 0;
+  uint64_t tok = 0;
+  while (!p->ready_fifo.empty() && n < max_samples) {
+    const auto e = p->ready_fifo.front();
+    p->ready_fifo.pop_front();
+    if (!live(e)) continue;
+    slots_out[n++] = e.first;
+    tok += p->slots[e.first].seq_len;
+  }
+  *n_out = n;
+  if (tokens_out) *tokens_out = tok;
   return FT_OK;
 }
 
@@ -1227,17 +1277,17 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings_
   if (c.host_pages == 0 || c.hbm_pages == 0) {
     launch(kTierAll, st);
   } else {
-    FT_CUDA(cudaEventRecord(p->fork_ev, st));
-    FT_CUDA(cudaStreamWaitEvent(p->side_stream, p->fork_ev, 0));
+    FT_CUDA(cudaEventRecord(p->fork_ev[0], st));
+    FT_CUDA(cudaStreamWaitEvent(p->side_stream[0], p->fork_ev[0], 0));
     if (f32) {
-      launch_scatter<kTierHostOnly, true>(p, w, total_chunks, (uint64_t)p->host_ctas, p->side_stream);
+      launch_scatter<kTierHostOnly, true>(p, w, total_chunks, (uint64_t)p->host_ctas, p->side_stream[0]);
     } else {
-      k_scatter_host_bulk<<<(unsigned)p->host_ctas, 32, kBulkSmemBytes, p->side_stream>>>(p->view, w, p->call_seq);
+      k_scatter_host_bulk<<<(unsigned)p->host_ctas, 32, kBulkSmemBytes, p->side_stream[0]>>>(p->view, w, p->call_seq);
     }
     p->gpu_launches++;
-    FT_CUDA(cudaEventRecord(p->join_ev, p->side_stream));
+    FT_CUDA(cudaEventRecord(p->join_ev[0], p->side_stream[0]));
     launch(kTierDeviceOnly, st);
-    FT_CUDA(cudaStreamWaitEvent(st, p->join_ev, 0));
+    FT_CUDA(cudaStreamWaitEvent(st, p->join_ev[0], 0));
   }
   FT_CUDA(cudaGetLastError());
 
@@ -1245,9 +1295,9 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings_
     ft_slot_mirror& s = p->slots[slot[q]];
     ft_span_mirror& m = p->spans[b_sid[q]];
     m.written = true; m.npages = (uint32_t)pages_for_tokens(p, n_tokens[q]);
-    if (++s.spans_written == s.n_spans) s.state = FT_SLOT_READY;
+    if (++s.spans_written == s.n_spans) { s.state = FT_SLOT_READY; p->ready_fifo.emplace_back(slot[q], s.generation); }
   }
   p->free_pages -= need; p->free_blocks -= need_blocks;
   p->bytes_written += bytes_total * (f32 ? 3 : 2);
-  return FT_OK;
+  return end_producer(p, st);
 }

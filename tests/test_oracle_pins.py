@@ -633,3 +633,35 @@ def test_sumsq_cost_closed_form():
     for j in range(a["n_mb"]):
         m = lengths[a["sample_mb"] == j].astype(np.int64)
         assert int(a["mb_cost"][j]) == 31 * int(m.sum()) + 7 * int((m * m).sum())
+
+
+# ------------------------------------------------------------------ ready queue (Sec. 3.1: "after sufficient paired embeddings accumulate")
+
+def test_ready_queue_is_completion_order_with_a_watermark():
+    w = workloads.make_workload("image_mix_7b", n_samples=8, hidden=64, page_bytes=4096)
+    pool = OraclePool(PoolConfig(**pool_config_fields(w)))
+    assert pool.register_samples(*register_args(w, list(range(8)))) == 0
+    assert pool.ready_count() == (0, 0) and pool.take_ready(1, 8)[0] == -5
+    # spans complete in an order of our choosing: 5, 2, 7 (sample 3 is left one span short if it has more than one)
+    done = []
+    for s in (5, 2, 7):
+        call = [(s, j) for j in range(int(w.n_spans[s]))]
+        assert pool.write_embeddings(*write_args(w, call), [host_span(w, s, j) for s, j in call], 0) == 0
+        done.append(s)
+    tok = [int(w.seq_len[s]) for s in done]
+    assert pool.ready_count() == (3, sum(tok))
+    assert pool.take_ready(sum(tok) + 1, 8)[0] == -5                     # below the watermark: nothing is taken
+    assert pool.ready_count() == (3, sum(tok))
+    rc, slots, t = pool.take_ready(sum(tok), 2)                          # at the watermark: completion order, capped
+    assert rc == 0 and list(slots) == [5, 2] and t == tok[0] + tok[1]
+    assert pool.ready_count() == (1, tok[2])
+    # a sample freed while queued is skipped; one freed and re-registered is a new sample (not ready yet)
+    assert pool.free([7]) == 0
+    assert pool.ready_count() == (0, 0) and pool.take_ready(0, 8)[0] == -5
+    assert pool.register_samples(*register_args(w, [7])) == 0
+    assert pool.ready_count() == (0, 0)
+    call = [(7, j) for j in range(int(w.n_spans[7]))] + [(0, j) for j in range(int(w.n_spans[0]))]
+    assert pool.write_embeddings(*write_args(w, call), [host_span(w, s, j) for s, j in call], 0) == 0
+    rc, slots, t = pool.take_ready(1, 8)
+    assert rc == 0 and list(slots) == [7, 0]                             # order inside one call = argument order
+    pool.destroy()
