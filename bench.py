@@ -547,6 +547,11 @@ def run_ours(args):
                                        "phase_ms": phases2,
                                        "gather_frac_of_measured_peak": g2["gbs"] / measured_peak()[0] if g2["gbs"] else None}
     job.close()
+    if rank == 0 and world == 1 and not args.skip_variants:
+        # the decoupled producer/consumer flow on the headline pool's tier split (and all-HBM beside it)
+        line["streaming"] = run_streaming(args, args.all_hbm)
+        if not args.all_hbm:
+            line["all_hbm_variant"]["streaming"] = run_streaming(args, True)
     if rank == 0:
         if world == 1 and not args.skip_cpu:
             n = min(CPU_SAMPLE, w.n_samples)
@@ -687,6 +692,90 @@ def run_sweep(args):
     }
     pool.destroy()
     print(json.dumps(line))
+
+
+# ---------------------------------------------------------------------------------------------
+# streaming: producer stream and consumer stream overlap successive batches
+# ---------------------------------------------------------------------------------------------
+def run_streaming(args, all_hbm, batches=6, warm=2):
+    """The decoupled flow (Sec. 3.1): while the consumer stream plans and assembles batch k, the producer stream
+    registers and writes batch k+1 into a pool that holds two batches; pool_free recycles batch k on the producer
+    stream as soon as it is assembled.  Returns steady-state ms per batch and the whole-path GB/s."""
+    import torch
+    import workloads
+    from harness import pool_config_fields, plan_config_fields, register_args, write_args
+    from paper_2606_23087_b200 import binding as fp
+    w = workloads.make_workload(args.workload, n_samples=args.samples, all_hbm=all_hbm)
+    n = w.n_samples
+    f = pool_config_fields(w, max_samples=2 * n)
+    f["hbm_pages"], f["host_pages"] = 2 * w.hbm_pages, 2 * w.host_pages
+    f["max_text_tokens"] = 2 * w.total_text_tokens_capacity
+    # pages of both tiers interleaved in the free ring: every batch then carries its share of host-tier pages, and
+    # the host-tier writes of batch k+1 (device -> host) can overlap the host-tier reads of batch k (host -> device)
+    f["ring_order"] = 1
+    pool = fp.Pool(fp.PoolConfig(**f))
+    if pool.rc != 0:
+        raise fp.FlowpoolError(pool.rc, "pool_create")
+    prod, cons = torch.cuda.Stream(), torch.cuda.Stream()
+    table = workloads.embed_table(w, device="cuda")
+    calls = []
+    for call in w.write_calls:
+        samples = sorted({s for s, _ in call}, key=[s for s, _ in call].index)
+        reg = register_args(w, samples)
+        wr = write_args(w, call)
+        srcs = [workloads.span_values(w, s, j, device="cuda") for s, j in call]
+        calls.append((reg, torch.from_numpy(reg[5]).cuda(), wr, [t.data_ptr() for t in srcs], srcs))
+    outs = [torch.empty((w.total_tokens, w.hidden), dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+    cu = torch.empty((2 * n + 8,), dtype=torch.int32, device="cuda")
+    pos = torch.empty((w.total_tokens,), dtype=torch.int32, device="cuda")
+    pcfg = fp.PlanConfig(**plan_config_fields(w))
+
+    def produce(k):
+        off = (k % 2) * n
+        for reg, ids, wr, ptrs, _ in calls:
+            rc = pool.register_samples(reg[0] + off, *reg[1:5], ids.data_ptr(), prod.cuda_stream)
+            assert rc == 0, rc
+            rc = pool.write_embeddings(wr[0] + off, wr[1], wr[2], ptrs, w.src_dtype, prod.cuda_stream)
+            assert rc == 0, rc
+
+    def assemble(k):
+        rc, slots, _ = pool.take_ready(w.total_tokens, n)      # watermark: one whole batch is ready
+        assert rc == 0 and len(slots) == n, (rc, len(slots))
+        rc, plan = pool.plan_microbatches(slots, pcfg, cons.cuda_stream)
+        assert rc == 0, rc
+        n_mb = plan.summary()[0]
+        rc = pool.gather_packed(plan, 0, n_mb, table.data_ptr(), w.vocab, outs[k % 2].data_ptr(), cu.data_ptr(), pos.data_ptr(),
+                                cons.cuda_stream)
+        assert rc == 0, rc
+        return slots, plan
+
+    # Issue order per round: assemble batch k (consumer stream), then write batch k+1 (producer stream), then free
+    # batch k (producer stream; the library makes it wait for the gather).  The consumer waits only for producer
+    # calls issued before it, so the write of k+1 and the assembly of k run side by side.
+    torch.cuda.synchronize()
+    produce(0)
+    t0 = None
+    total = warm + batches
+    for k in range(total):
+        if k == warm:
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+        slots, plan = assemble(k)
+        produce(k + 1)
+        assert pool.free(slots, prod.cuda_stream) == 0
+        plan.destroy()
+    torch.cuda.synchronize()
+    ms = (time.perf_counter() - t0) * 1e3 / batches
+    # drain the batch that was produced but never consumed
+    rc, slots, _ = pool.take_ready(1, n)
+    if rc == 0 and len(slots):
+        pool.free(slots, prod.cuda_stream)
+    assert pool.status() == (0, 0)
+    wb, gb = algorithmic_bytes(w)
+    pool.destroy()
+    return {"ms_per_batch": ms, "value": (wb + gb) / ms / 1e6, "unit": UNIT, "tokens_per_s": w.total_tokens / ms * 1e3,
+            "batches": batches, "pool": "two batches resident, same tier split, tiers interleaved in the free ring",
+            "note": "host wall clock over steady-state batches; producer and consumer on two streams"}
 
 
 # ---------------------------------------------------------------------------------------------
