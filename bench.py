@@ -31,7 +31,7 @@ METRIC = "packed-microbatch assembly throughput (producer scatter + plan + packe
 UNIT = "GB/s"
 CPU_SAMPLE = 256         # samples of the workload the oracle is timed on (about 10-30 s of CPU work)
 # dram__bytes_read.sum + dram__bytes_write.sum over algorithmic bytes for one k_gather launch, from the ncu capture
-# summarised in profiles/k_gather_image_mix_7b_64samples_all_hbm.md (4.592 GB / 4.698 GB on the first 64 samples);
+# on the first 64 samples of this workload, all pages in HBM (4.592 GB of DRAM traffic / 4.698 GB algorithmic);
 # traffic grows in proportion to the tokens assembled, so a full launch is this ratio times its algorithmic bytes
 NCU_TRAFFIC_RATIO_GATHER = 0.977
 
