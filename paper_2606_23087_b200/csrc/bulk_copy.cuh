@@ -40,7 +40,12 @@ __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.a
 constexpr int kBulkStages = 12;            // ring size
 constexpr int kBulkDepth = 8;              // loads in flight
 constexpr uint32_t kBulkStageBytes = 16384;
-constexpr uint32_t kBulkSpinLimit = 20000000;  // mbarrier polls before a copy is declared lost
+constexpr uint64_t kBulkWaitLimitNs = 2000000000ull;  // a staged load not seen after 2 s is declared lost
+__device__ __forceinline__ uint64_t global_timer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
 
 // Warp-wide copy pipeline: every lane of a one-warp CTA calls push()/drain() with the same arguments; lane 0
 // issues the asynchronous operations.  Copy number i goes into stage i % kBulkStages; before that, copy
@@ -70,10 +75,12 @@ struct BulkRing {
     const int st = (int)(k % kBulkStages);
     const uint32_t parity = (uint32_t)((k / kBulkStages) & 1);
     uint32_t bad = 0;
-    if (lane == 0) {
+    if (lane == 0 && !mbar_try_wait(&bar[st], parity)) {
+      // bounded wait: poll, looking at the wall clock every 1024 polls
+      const uint64_t t0 = global_timer_ns();
       uint32_t spins = 0;
       while (!mbar_try_wait(&bar[st], parity)) {
-        if (++spins > kBulkSpinLimit) { bad = 1; break; }
+        if ((++spins & 1023u) == 0 && global_timer_ns() - t0 > kBulkWaitLimitNs) { bad = 1; break; }
       }
     }
     bad = __shfl_sync(0xFFFFFFFFu, bad, 0);
