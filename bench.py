@@ -547,6 +547,10 @@ def run_ours(args):
                                        "phase_ms": phases2,
                                        "gather_frac_of_measured_peak": g2["gbs"] / measured_peak()[0] if g2["gbs"] else None}
     job.close()
+    del job          # its resident inputs and outputs go before the streaming measurement builds its own
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()
     if rank == 0 and world == 1 and not args.skip_variants:
         # the decoupled producer/consumer flow on the headline pool's tier split (and all-HBM beside it)
         line["streaming"] = run_streaming(args, args.all_hbm)
@@ -773,6 +777,8 @@ def run_streaming(args, all_hbm, batches=6, warm=2):
     assert pool.status() == (0, 0)
     wb, gb = algorithmic_bytes(w)
     pool.destroy()
+    del calls, outs, table
+    torch.cuda.empty_cache()
     return {"ms_per_batch": ms, "value": (wb + gb) / ms / 1e6, "unit": UNIT, "tokens_per_s": w.total_tokens / ms * 1e3,
             "batches": batches, "pool": "two batches resident, same tier split, tiers interleaved in the free ring",
             "note": "host wall clock over steady-state batches; producer and consumer on two streams"}
