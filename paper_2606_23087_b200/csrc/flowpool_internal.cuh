@@ -302,6 +302,18 @@ size_t align_up_sz(size_t x, size_t a);
 // (arena: 0 = producer-side calls, 1 = consumer-side calls)
 int32_t stage_upload(ft_pool* p, int arena, const void* src, size_t bytes, size_t total_bytes, cudaStream_t st, void** d_out);
 
+// appends a sample that just became READY; entries of samples freed since are dropped whenever the queue has grown
+// past four entries per slot, so a caller that never takes from it cannot make it grow without bound
+inline void ready_push(ft_pool* p, uint32_t slot) {
+  if (p->ready_fifo.size() > 4 * p->slots.size() + 64) {
+    std::deque<std::pair<uint32_t, uint64_t>> live;
+    for (const auto& e : p->ready_fifo)
+      if (p->slots[e.first].state == FT_SLOT_READY && p->slots[e.first].generation == e.second) live.push_back(e);
+    p->ready_fifo.swap(live);
+  }
+  p->ready_fifo.emplace_back(slot, p->slots[slot].generation);
+}
+
 // Cross-stream ordering (the producer side and the consumer side of a pool may be driven from two streams):
 // a consumer-side call waits for the producer-side calls issued before it; pool_free waits for the consumer-side
 // calls issued before it.  Same-stream use costs one event record per call and no wait.

@@ -345,7 +345,7 @@ FT_API int32_t pool_import_samples(ft_pool* p, const uint32_t* local_slot, uint3
   for (uint32_t i = 0, g = 0; i < n; ++i) {
     ft_slot_mirror& s = p->slots[local_slot[i]];
     s.state = FT_SLOT_READY; s.remote = true;
-    p->ready_fifo.emplace_back(local_slot[i], s.generation);
+    ready_push(p, local_slot[i]);
     s.seq_len = seq[i]; s.n_spans = nsp[i]; s.spans_written = nsp[i]; s.n_text_pages = ps[3 * i + 2];
     for (uint32_t j = 0; j < nsp[i]; ++j, ++g) {
       ft_span_mirror& m = p->spans[(uint64_t)local_slot[i] * S + j];

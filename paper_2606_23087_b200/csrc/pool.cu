@@ -823,7 +823,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_register_samples(
   for (uint32_t i = 0; i < n; ++i) {
     ft_slot_mirror& s = p->slots[slot[i]];
     s.state = n_spans[i] == 0 ? FT_SLOT_READY : FT_SLOT_REGISTERED;
-    if (s.state == FT_SLOT_READY) p->ready_fifo.emplace_back(slot[i], s.generation);  // text only: paired at once
+    if (s.state == FT_SLOT_READY) ready_push(p, slot[i]);  // text only: paired at once
     s.seq_len = seq_len[i]; s.n_spans = n_spans[i]; s.spans_written = 0;
     s.n_text_pages = (seq_len[i] + kTextPageIds - 1) / kTextPageIds;
     for (uint32_t j = 0; j < n_spans[i]; ++j, ++sp) {
@@ -940,7 +940,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings(
     ft_slot_mirror& s = p->slots[slot[q]];
     ft_span_mirror& m = p->spans[span_id[q]];
     m.written = true; m.npages = (uint32_t)pages_for_tokens(p, n_tokens[q]);
-    if (++s.spans_written == s.n_spans) { s.state = FT_SLOT_READY; p->ready_fifo.emplace_back(slot[q], s.generation); }
+    if (++s.spans_written == s.n_spans) { s.state = FT_SLOT_READY; ready_push(p, slot[q]); }
   }
   p->free_pages -= need; p->free_blocks -= need_blocks;
   p->bytes_written += bytes_total * (f32 ? 3 : 2);
@@ -1295,7 +1295,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings_
     ft_slot_mirror& s = p->slots[slot[q]];
     ft_span_mirror& m = p->spans[b_sid[q]];
     m.written = true; m.npages = (uint32_t)pages_for_tokens(p, n_tokens[q]);
-    if (++s.spans_written == s.n_spans) { s.state = FT_SLOT_READY; p->ready_fifo.emplace_back(slot[q], s.generation); }
+    if (++s.spans_written == s.n_spans) { s.state = FT_SLOT_READY; ready_push(p, slot[q]); }
   }
   p->free_pages -= need; p->free_blocks -= need_blocks;
   p->bytes_written += bytes_total * (f32 ? 3 : 2);

@@ -32,7 +32,7 @@ def expected_row(w, s, p):
     return bits16(workloads.embed_table(w, "cpu", rows=(i, i + 1))).ravel()
 
 
-@pytest.mark.parametrize("name,kw", [("image_mix_7b", {}), ("video_heavy", {})])
+@pytest.mark.parametrize("name,kw", [("image_mix_7b", {}), ("video_heavy", {}), ("host_tier_stress", {})])
 def test_full_size_plan_and_sampled_rows(name, kw):
     if not torch.cuda.is_available():
         pytest.fail("a CUDA device is required for -m gpu tests")
@@ -79,7 +79,10 @@ def test_full_size_plan_and_sampled_rows(name, kw):
     rows = torch.tensor([int(row_off[q]) + p for q, s, p in picks], device="cuda")
     got_rows = out[rows].cpu().numpy().view(np.uint16)
     for i, (q, s, p) in enumerate(picks):
-        assert np.array_equal(got_rows[i], expected_row(w, s, p)), (q, s, p)
+        exp_row = expected_row(w, s, p)
+        assert np.array_equal(got_rows[i], exp_row), (q, s, p)
+        if w.src_dtype == 1:   # the special bit patterns (every 4099th element) reach some sampled rows
+            pass
     # no row left at poison anywhere (checked on the device)
     assert not bool((out == -1).all(dim=1).any().item())
     oplan.destroy()
