@@ -220,9 +220,12 @@ int32_t pool_write_embeddings_noalloc(ft_pool* pool, uint32_t n_spans, const uin
  * descending, ties by index).
  *   sample_slot host [n]; cfg host; out host, receives the plan handle.
  * Synchronises the stream once; the summary is valid on return.
- * Errors: L, K or N zero INVALID_ARG; per sample in order: slot out of range
- * INVALID_ARG, FREE UNKNOWN_SAMPLE, listed twice INVALID_ARG, not READY
- * (without FT_PLAN_ALLOW_UNWRITTEN) NOT_READY, seq_len > L TOO_LONG.
+ * cfg->flags may select the variants listed at FT_PLAN_*.
+ * Errors: L, K or N zero INVALID_ARG; L >= 2^20 CAPACITY (the residual bitmap
+ * covers budgets below 2^20); A*L + B*L^2 not representable in 64 bits
+ * INVALID_ARG; per sample in order: slot out of range INVALID_ARG, FREE
+ * UNKNOWN_SAMPLE, listed twice INVALID_ARG, not READY (without
+ * FT_PLAN_ALLOW_UNWRITTEN) NOT_READY, seq_len > L TOO_LONG.
  * n = 0 gives an empty plan.
  */
 int32_t pool_plan_microbatches(ft_pool* pool, const uint32_t* sample_slot, uint32_t n,
@@ -263,8 +266,10 @@ int32_t plan_destroy(ft_plan* plan);
  *   out_position_ids  device int32 [sum of tokens]: p, restarting per sample
  * Padding rows are not materialised.  Asynchronous.  Errors: bad range
  * INVALID_ARG; a sample of the plan freed or not READY NOT_READY; NULL buffer
- * INVALID_ARG.  Asynchronous: id outside [0, vocab) BAD_TOKEN_ID, page GVA that
- * does not translate BAD_GVA (detail = row index in the range; row skipped).
+ * INVALID_ARG; hidden > 18432 CAPACITY (a row may touch at most 10 pages).
+ * Asynchronous: id outside [0, vocab) BAD_TOKEN_ID, page GVA that does not
+ * translate BAD_GVA (detail = row index in the range; row skipped).  Whether a
+ * position is a vision row is decided by the sample's span table, not by its id.
  */
 int32_t pool_gather_packed(ft_pool* pool, const ft_plan* plan, uint32_t mb_begin, uint32_t mb_end,
                            const void* embed_table, uint32_t vocab, void* out_embeds,
@@ -274,7 +279,7 @@ int32_t pool_gather_packed(ft_pool* pool, const ft_plan* plan, uint32_t mb_begin
  * pool_free -- release samples: their pages go back to the free-ring tail
  * (samples in argument order, spans by index, pages by ordinal), their text
  * pages and slots are recycled.  Plans holding a freed sample become invalid.
- * The paper does not discuss recycling; the ring is this build's fixed rule.
+ * The paper does not discuss recycling; the FIFO ring is this library's fixed rule.
  *   sample_slot host [n].  Errors: slot out of range INVALID_ARG; FREE or
  * listed twice UNKNOWN_SAMPLE.  Asynchronous.
  */
