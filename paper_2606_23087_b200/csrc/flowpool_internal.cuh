@@ -266,7 +266,7 @@ struct ft_pool {
   int host_ctas = 8;            // grid of the host-tier copy kernels: few SMs, so that long-latency host-link
                                 // accesses do not clog the memory pipelines of the SMs that stream HBM
                                 // (FLOWPOOL_HOST_CTAS overrides)
-  int chunk_shift = 16;         // log2 of k_scatter's work unit in bytes of a span's image
+  int chunk_shift = 16;         // log2 of k_scatter's work unit in bytes of a span's image (14..21)
   int scatter_group = 0;        // chunks per round-robin group of k_scatter; 0 = the measured default
   int scatter_ctas_per_sm = 0;  // resident CTAs per SM of the device-tier scatter kernel; 0 = the measured default
   int gather_unroll = 4;        // 16-byte vectors per lane in flight in k_gather (4 or 8)
