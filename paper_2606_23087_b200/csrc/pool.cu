@@ -603,7 +603,8 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_create(const ft_p
   CK(cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, p->device));
   p->host_ctas = 8;
   if (const char* e = getenv("FLOWPOOL_HOST_CTAS")) { int v = atoi(e); if (v > 0) p->host_ctas = v; }
-  if (const char* e = getenv("FLOWPOOL_CHUNK_SHIFT")) { int v = atoi(e); if (v >= 14 && v <= 21) p->chunk_shift = v;  // a warp region (1/8 chunk) is at least one 2 KiB batch }
+  // A warp's region is 1/8 of a chunk and must hold at least one 2 KiB batch.
+  if (const char* e = getenv("FLOWPOOL_CHUNK_SHIFT")) { int v = atoi(e); if (v >= 14 && v <= 21) p->chunk_shift = v; }
   if (const char* e = getenv("FLOWPOOL_SCATTER_GROUP")) { int v = atoi(e); if (v > 0) p->scatter_group = v; }
   if (const char* e = getenv("FLOWPOOL_SCATTER_CTAS_PER_SM")) { int v = atoi(e); if (v > 0) p->scatter_ctas_per_sm = v; }
   if (const char* e = getenv("FLOWPOOL_GATHER_U")) { int v = atoi(e); if (v == 4 || v == 8) p->gather_unroll = v; }
