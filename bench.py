@@ -626,8 +626,11 @@ def run_sweep(args):
     n_mb, total_tokens, _ = plan.summary()
     # scheduler variants on the same residents: what each buys in padding waste and rank balance
     variants = {}
-    for name, fl in (("as_printed", 0), ("longest_first", 2), ("sum_of_squares", 4), ("carried_zigzag", 8), ("all_three", 14)):
+    for name, fl, k_limit in (("as_printed", 0, 0), ("longest_first", 2, 0), ("sum_of_squares", 4, 0), ("carried_zigzag", 8, 0),
+                              ("all_three", 14, 0), ("auto_k_limit_64", 16, 64), ("fixed_k_64", 0, 64)):
         vc = plan_config_fields(w, flags=fl)
+        if k_limit:
+            vc["n_buckets_K"] = k_limit
         torch.cuda.synchronize()
         t0 = time.perf_counter()
         rc, vp = pool.plan_microbatches(order, fp.PlanConfig(**vc), st)
@@ -636,7 +639,8 @@ def run_sweep(args):
         va = vp.arrays()
         vl = np.array([va["mb_cost"][va["mb_rank"] == r].astype(np.float64).sum() for r in range(w.n_ranks_N)])
         variants[name] = {"microbatches": int(va["n_mb"]), "padding_waste": 1.0 - total_tokens / (int(va["n_mb"]) * w.budget_L),
-                          "rank_imbalance": float((vl.max() - vl.min()) / vl.mean()), "plan_ms_host_wall": dt}
+                          "rank_imbalance": float((vl.max() - vl.min()) / vl.mean()), "plan_ms_host_wall": dt,
+                          "buckets_used": int(len(np.unique(va["mb_bucket"])))}
         vp.destroy()
     # gather everything, in ranges that fit a reusable output buffer
     table = workloads.embed_table(w, device="cuda")

@@ -60,12 +60,14 @@ enum {
 enum { FT_RING_SORTED = 0, FT_RING_SHUFFLED = 1 }; /* initial free-ring order */
 enum { FT_BIND_IDENTITY = 0, FT_BIND_PERMUTED = 1 }; /* virtual page -> frame */
 enum { FT_BF16 = 0, FT_F32 = 1 };                    /* producer source dtype */
-/* plan flags.  ALLOW_UNWRITTEN plans metadata only.  The other three select variants at points where the paper
+/* plan flags.  ALLOW_UNWRITTEN plans metadata only.  The others select variants at points where the paper
  * is silent or could be read otherwise (defaults follow the text): SORT_DECREASING packs longest first (equal
  * lengths keep the caller's order) instead of in the caller's order; COST_SUMSQ uses sum(l^2) instead of lmax^2
  * as the quadratic term of Eq. 3; ZIGZAG_CARRY lets the zig-zag position and direction carry over from bucket to
- * bucket instead of restarting in each. */
-enum { FT_PLAN_ALLOW_UNWRITTEN = 1, FT_PLAN_SORT_DECREASING = 2, FT_PLAN_COST_SUMSQ = 4, FT_PLAN_ZIGZAG_CARRY = 8 };
+ * bucket instead of restarting in each; AUTO_K takes the number of buckets from the data, min(K, max(1,
+ * ceil(n_mb / 2N))): one bucket per full zig-zag round trip over the N ranks, K being the upper limit. */
+enum { FT_PLAN_ALLOW_UNWRITTEN = 1, FT_PLAN_SORT_DECREASING = 2, FT_PLAN_COST_SUMSQ = 4, FT_PLAN_ZIGZAG_CARRY = 8,
+       FT_PLAN_AUTO_K = 16 };
 
 #define FT_TEXT_PAGE_BYTES 4096u /* token ids live in 4 KiB text pages (1024 ids) */
 

@@ -42,7 +42,8 @@ enum { OR_RING_SORTED = 0, OR_RING_SHUFFLED = 1 };
 enum { OR_BIND_IDENTITY = 0, OR_BIND_PERMUTED = 1 };
 enum { OR_BF16 = 0, OR_F32 = 1 };
 /* plan flags; the last three are variants at points where the paper is silent or could be read otherwise */
-enum { OR_PLAN_ALLOW_UNWRITTEN = 1, OR_PLAN_SORT_DECREASING = 2, OR_PLAN_COST_SUMSQ = 4, OR_PLAN_ZIGZAG_CARRY = 8 };
+enum { OR_PLAN_ALLOW_UNWRITTEN = 1, OR_PLAN_SORT_DECREASING = 2, OR_PLAN_COST_SUMSQ = 4, OR_PLAN_ZIGZAG_CARRY = 8,
+       OR_PLAN_AUTO_K = 16 };
 enum { SLOT_FREE = 0, SLOT_REGISTERED = 1, SLOT_READY = 2 };
 
 #define TEXT_PAGE_BYTES 4096u /* reading: token ids live in 4 KiB text pages */
@@ -769,8 +770,17 @@ int32_t oracle_plan_from_lengths(const uint32_t* slots, const uint32_t* len, uin
       pl->mb_cost[j] = oracle_cost_int(cfg->coef_A, cfg->coef_B, pl->mb_tokens[j], pl->mb_lmax[j]);
     }
   }
-  /* lines 12-27: buckets and zig-zag dispatch */
-  oracle_balance(n_mb, pl->mb_cost, K, N, (cfg->flags & OR_PLAN_ZIGZAG_CARRY) != 0, pl->mb_bucket, pl->mb_rank,
+  /* lines 12-27: buckets and zig-zag dispatch.  The paper does not say how many clusters there are.
+   * Default: the caller's K.  Variant AUTO_K: as many buckets as there are full zig-zag round trips
+   * (one forward and one backward pass over the N ranks = 2N microbatches), at least 1, at most the caller's K,
+   * so that every bucket can pair high and low costs on each rank. */
+  uint32_t K_used = K;
+  if (cfg->flags & OR_PLAN_AUTO_K) {
+    uint64_t trips = ((uint64_t)n_mb + 2ull * N - 1) / (2ull * N);
+    if (trips < 1) trips = 1;
+    if (trips < K_used) K_used = (uint32_t)trips;
+  }
+  oracle_balance(n_mb, pl->mb_cost, K_used, N, (cfg->flags & OR_PLAN_ZIGZAG_CARRY) != 0, pl->mb_bucket, pl->mb_rank,
                  pl->rank_mb_off, pl->rank_mbs);
   free(ord); free(olen); free(omb);
   free(count);

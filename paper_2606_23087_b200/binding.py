@@ -13,7 +13,7 @@ from .build import SO, build
 FT_BF16, FT_F32 = 0, 1
 FT_RING_SORTED, FT_RING_SHUFFLED = 0, 1
 FT_BIND_IDENTITY, FT_BIND_PERMUTED = 0, 1
-FT_PLAN_ALLOW_UNWRITTEN, FT_PLAN_SORT_DECREASING, FT_PLAN_COST_SUMSQ, FT_PLAN_ZIGZAG_CARRY = 1, 2, 4, 8
+FT_PLAN_ALLOW_UNWRITTEN, FT_PLAN_SORT_DECREASING, FT_PLAN_COST_SUMSQ, FT_PLAN_ZIGZAG_CARRY, FT_PLAN_AUTO_K = 1, 2, 4, 8, 16
 FT_NOALLOC_MAX_SPANS = 4096
 
 STATUS = {

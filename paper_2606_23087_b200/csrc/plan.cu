@@ -281,9 +281,15 @@ __global__ void k_tiles(const uint64_t* sample_row_off, uint32_t n, uint32_t* ti
   for (uint64_t t = t0; t < t1; ++t) tile_first_sample[t] = q;  // rows 32t lies inside sample q
 }
 
-__global__ void k_bucket(const uint64_t* mb_cost, uint32_t K, const uint32_t* scalars, uint32_t* mb_bucket) {
+// auto_N != 0 (variant): K is only the upper limit; one bucket per full zig-zag round trip of 2N microbatches.
+__global__ void k_bucket(const uint64_t* mb_cost, uint32_t K, uint32_t auto_N, const uint32_t* scalars, uint32_t* mb_bucket) {
   const uint32_t j = blockIdx.x * blockDim.x + threadIdx.x;
-  if (j >= scalars[SC_NMB]) return;
+  const uint32_t n_mb = scalars[SC_NMB];
+  if (j >= n_mb) return;
+  if (auto_N) {
+    const unsigned long long trips = max(1ull, ((unsigned long long)n_mb + 2ull * auto_N - 1) / (2ull * auto_N));
+    if (trips < K) K = (uint32_t)trips;
+  }
   const uint64_t lo = *reinterpret_cast<const unsigned long long*>(scalars + SC_LO);
   const uint64_t hi = *reinterpret_cast<const unsigned long long*>(scalars + SC_HI);
   const unsigned __int128 num = (unsigned __int128)(mb_cost[j] - lo) * K;
@@ -488,7 +494,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_plan_microbatches
                                 pl->d_plan_len, pl->d_mb_cost, pl->d_scalars);
   k_row_offsets<<<1, 1024, 0, st>>>(pl->d_plan_len, n, pl->d_sample_row_off);
   k_tiles<<<gb, 256, 0, st>>>(pl->d_sample_row_off, n, pl->d_tile_first_sample);
-  k_bucket<<<gb, 256, 0, st>>>(pl->d_mb_cost, K, pl->d_scalars, pl->d_mb_bucket);
+  k_bucket<<<gb, 256, 0, st>>>(pl->d_mb_cost, K, (cfg->flags & FT_PLAN_AUTO_K) ? N : 0u, pl->d_scalars, pl->d_mb_bucket);
   k_sort_deal<<<gb, 256, 0, st>>>(pl->d_mb_cost, pl->d_mb_bucket, N, f_carry, pl->d_scalars, pl->d_mb_pos, pl->d_mb_rank);
   k_rank_index<<<gb, 256, 0, st>>>(pl->d_mb_pos, pl->d_mb_rank, pl->d_scalars, d_mb_idx, pl->d_rank_cnt);
   k_rank_scan<<<1, 1024, 0, st>>>(pl->d_rank_cnt, N, pl->d_rank_mb_off);

@@ -102,12 +102,12 @@ def test_random_call_sequences_agree_with_oracle(seed, ring_order, page_bytes, h
                 slots = rng.choice(w.n_samples, size=int(rng.integers(0, 20)), replace=bool(rng.random() < 0.2))
                 cfg = dict(coef_A=int(rng.integers(0, 50000)), coef_B=int(rng.integers(0, 3)),
                            budget_L=int(rng.choice([0, 6000, 20000, 40000, 1 << 19])), n_buckets_K=int(rng.integers(0, 5)),
-                           n_ranks_N=int(rng.integers(0, 9)), flags=int(rng.random() < 0.5) + 2 * int(rng.integers(0, 8)))
+                           n_ranks_N=int(rng.integers(0, 9)), flags=int(rng.random() < 0.5) + 2 * int(rng.integers(0, 16)))
             else:
                 slots = rng.permutation(rdy)[:int(rng.integers(1, len(rdy) + 1))]
                 cfg = dict(coef_A=int(rng.integers(0, 50000)), coef_B=int(rng.integers(0, 3)),
                            budget_L=int(rng.choice([w.max_seq_len, 20000, 40000, 1 << 19])), n_buckets_K=int(rng.integers(1, 5)),
-                           n_ranks_N=int(rng.integers(1, 9)), flags=2 * int(rng.integers(0, 8)))
+                           n_ranks_N=int(rng.integers(1, 9)), flags=2 * int(rng.integers(0, 16)))
             g, gp = pool.plan_microbatches(slots, fp.PlanConfig(**cfg), cuda_stream())
             o, op_ = opool.plan_microbatches(slots, PlanConfig(**cfg))
             if g == 0 and o == 0:

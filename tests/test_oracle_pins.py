@@ -580,6 +580,30 @@ def test_variant_hand_examples():
     r = balance(g["Z_costs"], g["Z_K"][0], g["Z_N"][0], carry=1)
     assert list(r["rank"]) == g["Z_rank"]
     assert list(balance(g["Z_costs"], g["Z_K"][0], g["Z_N"][0], carry=0)["rank"]) == [0, 1, 2, 0, 1, 2, 2]
+    for flags, kb, kr in ((16, "K_bucket", "K_rank"), (0, "K_fixed_bucket", "K_fixed_rank")):
+        rc, plan = plan_from_lengths(g["K_lengths"], plan_cfg(g["K_L"][0], A=1, B=0, K=g["K_K"][0], N=g["K_N"][0], flags=flags))
+        a = plan.arrays()
+        assert list(a["mb_bucket"]) == g[kb] and list(a["mb_rank"]) == g[kr]
+
+
+def test_auto_k_limits():
+    # at most 2N microbatches: one round trip, one bucket, whatever the limit; a limit of 1 switches the variant off;
+    # many microbatches: the limit K is reached and the plan equals the fixed-K plan
+    rng = np.random.default_rng(12)
+    for trial in range(60):
+        N, K, L = int(rng.integers(1, 6)), int(rng.integers(1, 6)), 64
+        n = int(rng.integers(1, 200))
+        lengths = rng.integers(33, L + 1, size=n)   # longer than L/2: every sequence is its own microbatch
+        auto = plan_from_lengths(lengths, plan_cfg(L, A=3, B=1, K=K, N=N, flags=16))[1].arrays()
+        assert auto["n_mb"] == n
+        if n <= 2 * N:
+            same = plan_from_lengths(lengths, plan_cfg(L, A=3, B=1, K=1, N=N))[1].arrays()
+        elif n > 2 * N * (K - 1):
+            same = plan_from_lengths(lengths, plan_cfg(L, A=3, B=1, K=K, N=N))[1].arrays()
+        else:
+            assert auto["mb_bucket"].max() < K and auto["mb_bucket"].max() <= (n - 1) // (2 * N)
+            continue
+        assert list(auto["mb_bucket"]) == list(same["mb_bucket"]) and list(auto["mb_rank"]) == list(same["mb_rank"])
 
 
 def test_variant_invariants():
@@ -587,7 +611,7 @@ def test_variant_invariants():
     for trial in range(150):
         n, L = int(rng.integers(1, 120)), int(rng.integers(8, 300))
         lengths = rng.integers(1, L + 1, size=n)
-        flags = int(rng.integers(0, 8)) * 2
+        flags = int(rng.integers(0, 16)) * 2
         K, N = int(rng.integers(1, 5)), int(rng.integers(1, 7))
         rc, plan = plan_from_lengths(lengths, plan_cfg(L, A=int(rng.integers(0, 100)), B=int(rng.integers(0, 4)), K=K, N=N, flags=flags))
         assert rc == 0
