@@ -72,6 +72,7 @@ typedef struct {
   uint32_t pos_start, n_tokens;
   uint32_t n_pages; /* 0 until written */
   uint64_t* pages;  /* page GVAs, by ordinal */
+  uint32_t grid[3]; /* (T, H, W) of the span's token grid; all zero = none given */
 } or_span;
 
 typedef struct {
@@ -1117,5 +1118,200 @@ int32_t oracle_plan_arrays(const oracle_plan* pl, uint32_t* mb_sample_off, uint3
   CP(mb_cost, pl->mb_cost, m); CP(mb_bucket, pl->mb_bucket, m); CP(mb_rank, pl->mb_rank, m);
   CP(rank_mb_off, pl->rank_mb_off, N + 1); CP(rank_mbs, pl->rank_mbs, m);
   CP(sample_cost, pl->sample_cost, n); CP(sample_mb, pl->sample_mb, n);
+  return OR_OK;
+}
+
+/* ------------------------------------------------------------------------
+ * Backbone-side outputs next to assembly.  The paper stops at "the backbone
+ * consumes microbatches"; nothing below has a passage of its own.  What the
+ * paper does fix: image and text subsequences are interleaved (Sec. 4.1),
+ * a microbatch holds at most L tokens (Sec. 3.4), and the encoders are frozen
+ * (Sec. 4.3), so the only gradient that flows back through the assembled
+ * input is the embedding table's.  Each function states its own definition;
+ * the pins are hand-worked examples and reductions to the packed assembly
+ * and to library routines.
+ * ---------------------------------------------------------------------- */
+
+/* Token grid of a span: (T, H, W) with T*H*W = n_tokens, row-major (t, h, w).
+ * All-or-nothing: the first bad item stops the call and nothing is stored. */
+int32_t oracle_pool_set_span_grids(oracle_pool* p, uint32_t n, const uint32_t* slot, const uint32_t* span_idx,
+                                   const uint32_t* grid_thw) {
+  if (!p) return OR_ERR_INVALID_ARG;
+  p->call_seq++;
+  if (n && (!slot || !span_idx || !grid_thw)) return OR_ERR_INVALID_ARG;
+  for (uint32_t i = 0; i < n; ++i) {
+    if (slot[i] >= p->c.max_samples) return OR_ERR_INVALID_ARG;
+    or_sample* s = &p->samples[slot[i]];
+    if (s->state == SLOT_FREE) return OR_ERR_UNKNOWN_SAMPLE;
+    if (span_idx[i] >= s->n_spans) return OR_ERR_INVALID_ARG;
+    const uint32_t* g = grid_thw + 3ull * i;
+    if (g[0] == 0 || g[1] == 0 || g[2] == 0) return OR_ERR_INVALID_ARG;
+    if ((uint64_t)g[0] * g[1] * g[2] != s->spans[span_idx[i]].n_tokens) return OR_ERR_INVALID_ARG;
+  }
+  for (uint32_t i = 0; i < n; ++i)
+    memcpy(p->samples[slot[i]].spans[span_idx[i]].grid, grid_thw + 3ull * i, 12);
+  return OR_OK;
+}
+
+/* Three-component position of every token of one sample (the multimodal rotary scheme of current
+ * vision-language backbones): a counter st starts at 0; a text token gets (st, st, st) and st += 1; a span
+ * with grid (T, H, W) starting at counter st gives its token (t, h, w) the position (st + t, st + h, st + w)
+ * and then st += max(T, H, W); a span without a grid counts as text. */
+static void sample_positions3(const or_sample* s, int32_t* out /* [seq_len][3] */) {
+  int64_t st = 0;
+  uint32_t pos = 0;
+  while (pos < s->seq_len) {
+    const or_span* sp = NULL;
+    for (uint32_t i = 0; i < s->n_spans; ++i)
+      if (pos >= s->spans[i].pos_start && pos < s->spans[i].pos_start + s->spans[i].n_tokens) sp = &s->spans[i];
+    if (sp && sp->grid[0] && pos == sp->pos_start) {
+      const uint32_t T = sp->grid[0], H = sp->grid[1], W = sp->grid[2];
+      for (uint32_t t = 0; t < T; ++t)
+        for (uint32_t h = 0; h < H; ++h)
+          for (uint32_t w = 0; w < W; ++w, ++pos) {
+            out[3ull * pos + 0] = (int32_t)(st + t); out[3ull * pos + 1] = (int32_t)(st + h); out[3ull * pos + 2] = (int32_t)(st + w);
+          }
+      uint32_t m = T; if (H > m) m = H; if (W > m) m = W;
+      st += m;
+    } else {
+      out[3ull * pos + 0] = out[3ull * pos + 1] = out[3ull * pos + 2] = (int32_t)st;
+      ++st; ++pos;
+    }
+  }
+}
+
+#define OR_IGNORE_LABEL (-100)
+
+/* Padded assembly: every microbatch of [mb_begin, mb_end) occupies exactly L rows.
+ *   out_embeds [(mb_end-mb_begin)*L][H] bf16: the packed rows of the microbatch, then zero rows;
+ *   out_cu_seqlens: per microbatch n_j + 2 entries: 0, the sample ends, then L (the padding as one last sequence,
+ *     of length 0 when the microbatch is full);
+ *   out_pos3 [3][rows]: component-major three-component positions (0 on padding rows);
+ *   out_ids [rows]: the token id of the position (the id stored at a placeholder position included), pad_id on padding;
+ *   out_labels [rows]: next-token target: the id at the following position of the same sample when that
+ *     position is a text position (not inside a span), else -100; -100 on the last position and on padding;
+ *   out_mask [rows] bytes: 1 where the label is not -100.
+ * Errors as oracle_pool_gather_packed; detail of an asynchronous error = padded row index. */
+int32_t oracle_pool_gather_padded(oracle_pool* p, const oracle_plan* pl, uint32_t mb_begin, uint32_t mb_end,
+                                  const void* embed_table, uint32_t vocab, int32_t pad_id, void* out_embeds,
+                                  int32_t* out_cu_seqlens, int32_t* out_pos3, int32_t* out_ids, int32_t* out_labels,
+                                  uint8_t* out_mask) {
+  if (!p || !pl) return OR_ERR_INVALID_ARG;
+  p->call_seq++;
+  if (mb_begin > mb_end || mb_end > pl->n_mb) return OR_ERR_INVALID_ARG;
+  for (uint32_t t = 0; t < pl->n; ++t) {
+    or_sample* s = &p->samples[pl->slots[t]];
+    if (s->state != SLOT_READY || s->generation != pl->slot_generation[t]) return OR_ERR_NOT_READY;
+  }
+  if (mb_begin == mb_end) return OR_OK;
+  if (!embed_table || !out_embeds || !out_cu_seqlens || !out_pos3 || !out_ids || !out_labels || !out_mask)
+    return OR_ERR_INVALID_ARG;
+  const uint64_t PS = p->c.page_bytes, row_bytes = 2ull * p->c.hidden, L = pl->c.budget_L;
+  const uint64_t rows = (uint64_t)(mb_end - mb_begin) * L;
+  uint8_t* out = (uint8_t*)out_embeds;
+  uint64_t cu_w = 0;
+  for (uint32_t j = mb_begin; j < mb_end; ++j) {
+    uint64_t row = (uint64_t)(j - mb_begin) * L;
+    const uint64_t row_end = row + L;
+    int32_t cu = 0;
+    out_cu_seqlens[cu_w++] = 0;
+    for (uint32_t qi = pl->mb_sample_off[j]; qi < pl->mb_sample_off[j + 1]; ++qi) {
+      or_sample* s = &p->samples[pl->mb_samples[qi]];
+      int32_t* p3 = (int32_t*)calloc(3ull * s->seq_len + 3, sizeof(int32_t));
+      int32_t* ids = (int32_t*)calloc((size_t)s->seq_len + 1, sizeof(int32_t));
+      uint8_t* vis = (uint8_t*)calloc((size_t)s->seq_len + 1, 1);
+      sample_positions3(s, p3);
+      for (uint32_t pos = 0; pos < s->seq_len; ++pos) {
+        memcpy(&ids[pos], resolve(p, s->text_pages[pos / TEXT_PAGE_IDS] + (uint64_t)(pos % TEXT_PAGE_IDS) * 4), 4);
+        for (uint32_t i = 0; i < s->n_spans; ++i)
+          if (pos >= s->spans[i].pos_start && pos < s->spans[i].pos_start + s->spans[i].n_tokens) vis[pos] = 1;
+      }
+      for (uint32_t pos = 0; pos < s->seq_len; ++pos, ++row) {
+        for (int c = 0; c < 3; ++c) out_pos3[(uint64_t)c * rows + row] = p3[3ull * pos + c];
+        out_ids[row] = ids[pos];
+        const int has_label = pos + 1 < s->seq_len && !vis[pos + 1];
+        out_labels[row] = has_label ? ids[pos + 1] : OR_IGNORE_LABEL;
+        out_mask[row] = (uint8_t)has_label;
+        uint8_t* dst = out + row * row_bytes;
+        if (vis[pos]) {
+          const or_span* sp = NULL;
+          for (uint32_t i = 0; i < s->n_spans; ++i)
+            if (pos >= s->spans[i].pos_start && pos < s->spans[i].pos_start + s->spans[i].n_tokens) sp = &s->spans[i];
+          uint64_t b = (uint64_t)(pos - sp->pos_start) * row_bytes, done = 0;
+          while (done < row_bytes) {
+            uint64_t off = (b + done) % PS;
+            uint64_t run = PS - off < row_bytes - done ? PS - off : row_bytes - done;
+            uint8_t* src = resolve(p, sp->pages[(b + done) / PS] + off);
+            if (!src) { note_async_error(p, OR_ERR_BAD_GVA, (uint32_t)row); break; }
+            memcpy(dst + done, src, run);
+            done += run;
+          }
+        } else if (ids[pos] < 0 || (uint32_t)ids[pos] >= vocab) {
+          note_async_error(p, OR_ERR_BAD_TOKEN_ID, (uint32_t)row); /* row left untouched */
+        } else {
+          memcpy(dst, (const uint8_t*)embed_table + (uint64_t)ids[pos] * row_bytes, row_bytes);
+        }
+      }
+      free(p3); free(ids); free(vis);
+      cu += (int32_t)s->seq_len;
+      out_cu_seqlens[cu_w++] = cu;
+    }
+    out_cu_seqlens[cu_w++] = (int32_t)L;
+    for (; row < row_end; ++row) { /* padding */
+      memset(out + row * row_bytes, 0, row_bytes);
+      for (int c = 0; c < 3; ++c) out_pos3[(uint64_t)c * rows + row] = 0;
+      out_ids[row] = pad_id; out_labels[row] = OR_IGNORE_LABEL; out_mask[row] = 0;
+    }
+  }
+  return OR_OK;
+}
+
+static float bf16_bits_to_f32(uint16_t h) {
+  uint32_t u = (uint32_t)h << 16;
+  float f;
+  memcpy(&f, &u, 4);
+  return f;
+}
+
+/* Gradient of the embedding table through the assembled input.  grad_out holds one bf16 row per output row of
+ * the range, in the packed layout (padded = 0) or the L-rows-per-microbatch layout (padded != 0).  For the rows in
+ * ascending order: a row at a text position with id v adds its values, widened exactly to fp32, to row v of
+ * grad_table with one fp32 addition per element; rows at span positions (frozen encoders) and padding rows add
+ * nothing.  The order of the additions is part of the definition: fp32 addition is not associative. */
+int32_t oracle_pool_embed_grad(oracle_pool* p, const oracle_plan* pl, uint32_t mb_begin, uint32_t mb_end,
+                               int padded, const void* grad_out, float* grad_table, uint32_t vocab) {
+  if (!p || !pl) return OR_ERR_INVALID_ARG;
+  p->call_seq++;
+  if (mb_begin > mb_end || mb_end > pl->n_mb) return OR_ERR_INVALID_ARG;
+  for (uint32_t t = 0; t < pl->n; ++t) {
+    or_sample* s = &p->samples[pl->slots[t]];
+    if (s->state != SLOT_READY || s->generation != pl->slot_generation[t]) return OR_ERR_NOT_READY;
+  }
+  if (mb_begin == mb_end) return OR_OK;
+  if (!grad_out || !grad_table) return OR_ERR_INVALID_ARG;
+  const uint64_t H = p->c.hidden, L = pl->c.budget_L;
+  const uint16_t* g = (const uint16_t*)grad_out;
+  uint64_t row = 0;
+  for (uint32_t j = mb_begin; j < mb_end; ++j) {
+    if (padded) row = (uint64_t)(j - mb_begin) * L;
+    for (uint32_t qi = pl->mb_sample_off[j]; qi < pl->mb_sample_off[j + 1]; ++qi) {
+      or_sample* s = &p->samples[pl->mb_samples[qi]];
+      for (uint32_t pos = 0; pos < s->seq_len; ++pos, ++row) {
+        int vis = 0;
+        for (uint32_t i = 0; i < s->n_spans; ++i)
+          if (pos >= s->spans[i].pos_start && pos < s->spans[i].pos_start + s->spans[i].n_tokens) vis = 1;
+        if (vis) continue;
+        int32_t id;
+        memcpy(&id, resolve(p, s->text_pages[pos / TEXT_PAGE_IDS] + (uint64_t)(pos % TEXT_PAGE_IDS) * 4), 4);
+        if (id < 0 || (uint32_t)id >= vocab) { note_async_error(p, OR_ERR_BAD_TOKEN_ID, (uint32_t)row); continue; }
+        float* dst = grad_table + (uint64_t)id * H;
+        const uint16_t* src = g + row * H;
+        for (uint64_t c = 0; c < H; ++c) {
+          volatile float sum = dst[c] + bf16_bits_to_f32(src[c]); /* one rounded fp32 addition */
+          dst[c] = sum;
+        }
+      }
+    }
+  }
   return OR_OK;
 }

@@ -187,6 +187,23 @@ class OraclePool:
         return lib().oracle_pool_gather_packed(self.h, plan.h, C.c_uint32(mb_begin), C.c_uint32(mb_end), _p(table),
                                                C.c_uint32(table.shape[0]), _p(out), _p(cu), _p(pos))
 
+    def set_span_grids(self, slots, span_idx, grids):
+        """grids: [n, 3] (T, H, W) per named span."""
+        slots, span_idx = _u32(slots), _u32(span_idx)
+        grids = np.ascontiguousarray(np.asarray(grids, dtype=np.uint32).reshape(-1, 3))
+        return lib().oracle_pool_set_span_grids(self.h, C.c_uint32(len(slots)), _p(slots), _p(span_idx), _p(grids))
+
+    def gather_padded(self, plan, mb_begin, mb_end, table, pad_id, out, cu, pos3, ids, labels, mask):
+        """out: uint16 [n_mb*L, H]; cu: int32; pos3: int32 [3, rows]; ids, labels: int32 [rows]; mask: uint8 [rows]."""
+        return lib().oracle_pool_gather_padded(self.h, plan.h, C.c_uint32(mb_begin), C.c_uint32(mb_end), _p(table),
+                                               C.c_uint32(table.shape[0]), C.c_int32(pad_id), _p(out), _p(cu), _p(pos3),
+                                               _p(ids), _p(labels), _p(mask))
+
+    def embed_grad(self, plan, mb_begin, mb_end, padded, grad_out, grad_table):
+        """grad_out: uint16 (bf16 bits) [rows, H]; grad_table: float32 [vocab, H], accumulated in place."""
+        return lib().oracle_pool_embed_grad(self.h, plan.h, C.c_uint32(mb_begin), C.c_uint32(mb_end), C.c_int(int(padded)),
+                                            _p(grad_out), _p(grad_table), C.c_uint32(grad_table.shape[0]))
+
     def free(self, slots):
         slots = _u32(slots)
         return lib().oracle_pool_free(self.h, _p(slots), C.c_uint32(len(slots)))

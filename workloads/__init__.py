@@ -6,5 +6,5 @@ casting or assembly) and imports neither side.
 """
 from .gen import (  # noqa: F401
     Workload, make_workload, CONFIG_NAMES, input_ids, span_values, embed_table, special_f32_bits,
-    admit_free_schedule,
+    admit_free_schedule, span_grid, grad_values,
 )

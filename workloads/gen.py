@@ -26,7 +26,7 @@ _C1 = 0xBF58476D1CE4E5B9
 _C2 = 0x94D049BB133111EB
 
 # stream ids
-S_NTOK, S_TEXT, S_NSPAN, S_POS, S_IDS, S_EMB, S_TABLE, S_PERM, S_FRAMES, S_FREE = range(1, 11)
+S_NTOK, S_TEXT, S_NSPAN, S_POS, S_IDS, S_EMB, S_TABLE, S_PERM, S_FRAMES, S_FREE, S_GRID, S_GRAD = range(1, 13)
 
 # fp32 reciprocal of the standard deviation of a sum of four uniform 16-bit integers
 _IH_SCALE_BITS = 0x37DDB3D7
@@ -312,6 +312,24 @@ def input_ids(w: Workload, s: int) -> np.ndarray:
     for p, t in zip(pos, tok):
         ids[int(p):int(p) + int(t)] = w.placeholder_id
     return ids
+
+
+def span_grid(w: Workload, s: int, j: int):
+    """Token grid (T, H, W) of span j of sample s, or None (one span in four has none).  W is the largest divisor
+    of the tokens of one frame that is at most its square root, T is 2 for every other even-sized span, else 1."""
+    n = int(w.spans_of(s)[1][j])
+    h = int(hash_np(stream_key(w.seed, S_GRID, s), np.array([j]))[0])
+    if h % 4 == 0:
+        return None
+    T = 2 if (n % 2 == 0 and (h >> 8) % 2 == 0) else 1
+    frame = n // T
+    W = max(d for d in range(1, int(frame ** 0.5) + 1) if frame % d == 0)
+    return T, frame // W, W
+
+
+def grad_values(w: Workload, row0: int, row1: int, device="cpu") -> torch.Tensor:
+    """bf16 [row1-row0, H] stand-in for the gradient w.r.t. the assembled rows row0..row1 of a layout."""
+    return _irwin_hall_f32(stream_key(w.seed, S_GRAD), row0 * w.hidden, row1 * w.hidden, device).to(torch.bfloat16).view(row1 - row0, w.hidden)
 
 
 def _irwin_hall_f32(key: int, e0: int, e1: int, device) -> torch.Tensor:
