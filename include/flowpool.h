@@ -339,12 +339,67 @@ int32_t pool_import_samples(ft_pool* pool, const uint32_t* local_slot, uint32_t 
                             uint64_t bytes, void* stream);
 
 /*
+ * Backbone-side outputs next to assembly.  The paper stops where the backbone consumes a microbatch (Sec. 3.1);
+ * no passage defines what follows, so the definitions are stated here.  They lean on three facts the paper does
+ * fix: image and text subsequences are interleaved (Sec. 4.1), a microbatch holds at most L tokens (Sec. 3.4),
+ * and the encoders are frozen, so the only gradient that flows back through the assembled input is the
+ * embedding table's.
+ *
+ * pool_set_span_grids -- token grid (T, H, W) of named spans, T*H*W = the span's tokens, tokens in row-major
+ * (t, h, w) order.  A span keeps its grid until its sample is freed; a span without one counts as text below.
+ *   slot, span_idx host [n]; grid_thw host [n][3].  All-or-nothing, first bad item in order: slot out of range
+ *   INVALID_ARG, FREE slot UNKNOWN_SAMPLE, no such span INVALID_ARG, a zero extent or a product that is not the
+ *   span's token count INVALID_ARG.  Asynchronous; ordered before later calls on any stream like a producer call.
+ */
+int32_t pool_set_span_grids(ft_pool* pool, uint32_t n, const uint32_t* slot, const uint32_t* span_idx,
+                            const uint32_t* grid_thw, void* stream);
+
+/*
+ * pool_gather_padded -- pool_gather_packed in the padded layout: microbatch j of [mb_begin, mb_end) occupies rows
+ * [(j - mb_begin) * L, (j - mb_begin + 1) * L) of every output, L the plan's budget; rows = (mb_end - mb_begin) * L.
+ *   out_embeds   device bf16 [rows, H], 16-byte aligned: the packed rows of the microbatch, then zero rows
+ *   out_cu       device int32, per microbatch n_j + 2 entries: 0, the sample ends, then L (the padding as one
+ *                last sequence, of length 0 when the microbatch is full)
+ *   out_pos3     device int32 [3, rows], component-major.  A counter st runs over each sample from 0: a text token
+ *                (or a token of a span without a grid) gets (st, st, st) and st += 1; a span with grid (T, H, W)
+ *                starting at counter st gives its token (t, h, w) the position (st + t, st + h, st + w), then
+ *                st += max(T, H, W).  0 on padding rows.  Without any grid all three equal the packed position ids.
+ *   out_ids      device int32 [rows]: the stored token id of the position (the placeholder id inside a span);
+ *                pad_id on padding rows
+ *   out_labels   device int32 [rows]: next-token target: the id at the next position of the same sample when
+ *                that position is a text position, else -100; -100 on a sample's last position and on padding
+ *   out_mask     device uint8 [rows]: 1 where the label is not -100
+ * Errors as pool_gather_packed (detail = padded row index); more than 2^32 - 1 padded rows CAPACITY.  Asynchronous.
+ */
+int32_t pool_gather_padded(ft_pool* pool, const ft_plan* plan, uint32_t mb_begin, uint32_t mb_end,
+                           const void* embed_table, uint32_t vocab, int32_t pad_id, void* out_embeds,
+                           int32_t* out_cu, int32_t* out_pos3, int32_t* out_ids, int32_t* out_labels,
+                           uint8_t* out_mask, void* stream);
+
+/*
+ * pool_embed_grad -- gradient of the embedding table through the assembled input.  grad_out holds one bf16 row
+ * per output row of the range, in the packed layout (padded = 0) or the padded layout (padded != 0).  For the
+ * rows in ascending order: a row at a text position with id v adds its values, widened exactly to fp32, to row v
+ * of grad_table, one rounded fp32 addition per element; rows at span positions and padding rows add nothing.
+ * The order of the additions is part of the definition (fp32 addition is not associative): results are
+ * bit-reproducible and independent of the launch geometry.
+ *   grad_out    device bf16 [rows, H], 16-byte aligned
+ *   grad_table  device fp32 [vocab, H], 16-byte aligned, accumulated in place
+ * Errors: as pool_gather_packed; asynchronous: id outside [0, vocab) BAD_TOKEN_ID (row skipped).  Allocates
+ * 4 bytes per row of stream-ordered scratch for the call.  One CTA owns each table row, so a batch whose text is
+ * dominated by a single id serialises on that CTA.
+ */
+int32_t pool_embed_grad(ft_pool* pool, const ft_plan* plan, uint32_t mb_begin, uint32_t mb_end, uint32_t padded,
+                        const void* grad_out, float* grad_table, uint32_t vocab, void* stream);
+
+/*
  * Kernel timing for benchmarks.  While enabled, the library brackets each of its copy kernels with CUDA
  * events on the stream that kernel is launched on (the host-tier kernels run on the pool's side stream).
  * pool_profile_read synchronises the device, adds up the elapsed time and launch count per kernel class
  * since the last read, and clears them.  Classes: a single-tier pool's kernels count under its tier.
  */
-enum { FT_K_GATHER_DEVICE = 0, FT_K_GATHER_HOST = 1, FT_K_SCATTER_DEVICE = 2, FT_K_SCATTER_HOST = 3, FT_K_COUNT = 4 };
+enum { FT_K_GATHER_DEVICE = 0, FT_K_GATHER_HOST = 1, FT_K_SCATTER_DEVICE = 2, FT_K_SCATTER_HOST = 3, FT_K_EMBED_GRAD = 4,
+       FT_K_COUNT = 5 };
 typedef struct {
   double ms;
   uint64_t launches;

@@ -25,7 +25,7 @@ STATUS = {
 EXPORTS = (
     "pool_create", "pool_register_samples", "pool_write_embeddings", "pool_write_embeddings_noalloc",
     "pool_plan_microbatches", "plan_summary",
-    "plan_arrays", "plan_destroy", "pool_gather_packed", "pool_free", "pool_status", "pool_stats",
+    "plan_arrays", "plan_destroy", "pool_gather_packed", "pool_set_span_grids", "pool_gather_padded", "pool_embed_grad", "pool_free", "pool_status", "pool_stats",
     "pool_ready_count", "pool_take_ready", "pool_backing", "pool_export_mapping", "pool_import_mapping", "pool_export_samples", "pool_import_samples",
     "pool_profile_enable", "pool_profile_read", "pool_debug_span_pages", "pool_debug_ring", "pool_debug_translate", "pool_destroy", "flowpool_last_cuda_error",
 )
@@ -69,7 +69,7 @@ class KernelTime(C.Structure):
     _fields_ = [("ms", C.c_double), ("launches", C.c_uint64)]
 
 
-KERNEL_CLASSES = ("gather_device", "gather_host", "scatter_device", "scatter_host")
+KERNEL_CLASSES = ("gather_device", "gather_host", "scatter_device", "scatter_host", "embed_grad")
 
 _lib = None
 
@@ -92,6 +92,9 @@ def lib():
             "plan_arrays": [P] * 13,
             "plan_destroy": [P],
             "pool_gather_packed": [P, P, u32, u32, P, u32, P, P, P, P],
+            "pool_set_span_grids": [P, u32, P, P, P, P],
+            "pool_gather_padded": [P, P, u32, u32, P, u32, i32, P, P, P, P, P, P, P],
+            "pool_embed_grad": [P, P, u32, u32, u32, P, P, u32, P],
             "pool_free": [P, P, u32, P],
             "pool_status": [P, P, P],
             "pool_stats": [P, P],
@@ -205,6 +208,22 @@ class Pool:
                       pos_ptr: int, stream: int = 0):
         return lib().pool_gather_packed(self.h, plan.h, mb_begin, mb_end, table_ptr or None, vocab, out_ptr or None,
                                         cu_ptr or None, pos_ptr or None, stream or None)
+
+    def set_span_grids(self, slots, span_idx, grids, stream: int = 0):
+        slots, span_idx = _u32(slots), _u32(span_idx)
+        grids = np.ascontiguousarray(np.asarray(grids, dtype=np.uint32).reshape(-1, 3))
+        return lib().pool_set_span_grids(self.h, len(slots), _p(slots), _p(span_idx), _p(grids), stream or None)
+
+    def gather_padded(self, plan: Plan, mb_begin, mb_end, table_ptr: int, vocab: int, pad_id: int, out_ptr: int,
+                      cu_ptr: int, pos3_ptr: int, ids_ptr: int, labels_ptr: int, mask_ptr: int, stream: int = 0):
+        return lib().pool_gather_padded(self.h, plan.h, mb_begin, mb_end, table_ptr or None, vocab, pad_id, out_ptr or None,
+                                        cu_ptr or None, pos3_ptr or None, ids_ptr or None, labels_ptr or None,
+                                        mask_ptr or None, stream or None)
+
+    def embed_grad(self, plan: Plan, mb_begin, mb_end, padded, grad_out_ptr: int, grad_table_ptr: int, vocab: int,
+                   stream: int = 0):
+        return lib().pool_embed_grad(self.h, plan.h, mb_begin, mb_end, 1 if padded else 0, grad_out_ptr or None,
+                                     grad_table_ptr or None, vocab, stream or None)
 
     def free(self, slots, stream: int = 0):
         slots = _u32(slots)

@@ -6,7 +6,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 SO = os.path.join(HERE, "libflowpool.so")
-SOURCES = ["pool.cu", "plan.cu", "gather.cu", "peer.cu"]
+SOURCES = ["pool.cu", "plan.cu", "gather.cu", "peer.cu", "backbone.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC,-fvisibility=hidden"]
 

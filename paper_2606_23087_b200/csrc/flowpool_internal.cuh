@@ -66,6 +66,7 @@ struct PoolView {
   uint32_t* sp_npages;     // 0 until written
   uint32_t* sp_blocks;     // [span id][blocks_per_span] list block index
   uint64_t* list_blocks;   // [bring_cap][kListBlock] page GVAs
+  uint4* sp_grid;          // token grid (T, H, W, 0) of a span; all zero = none given
   unsigned long long* status;  // first asynchronous error key; ~0 = none
 };
 
@@ -192,6 +193,14 @@ struct ft_plan {
 };
 
 namespace ft {
+inline PlanView make_plan_view(const ft_plan* pl) {
+  PlanView pv;
+  pv.n = pl->n; pv.n_mb = pl->n_mb; pv.n_ranks = pl->cfg.n_ranks_N;
+  pv.mb_samples = pl->d_mb_samples; pv.plan_sample_mb = pl->d_plan_sample_mb;
+  pv.sample_row_off = pl->d_sample_row_off; pv.mb_sample_off = pl->d_mb_sample_off;
+  pv.mb_row_off = pl->d_mb_row_off; pv.tile_first_sample = pl->d_tile_first_sample;
+  return pv;
+}
 int32_t cuda_fail(cudaError_t e, const char* what);
 #define FT_CUDA(call)                                          \
   do {                                                         \
@@ -269,6 +278,7 @@ struct ft_pool {
   int chunk_shift = 16;         // log2 of k_scatter's work unit in bytes of a span's image (14..21)
   int scatter_group = 0;        // chunks per round-robin group of k_scatter; 0 = the measured default
   int scatter_ctas_per_sm = 0;  // resident CTAs per SM of the device-tier scatter kernel; 0 = the measured default
+  int grad_ctas_per_sm = 4;     // CTAs per SM of k_embed_grad (each owns the table rows v with v % grid == its index)
   int gather_unroll = 4;        // 16-byte vectors per lane in flight in k_gather (4 or 8)
   int dev_ctas_per_sm = 4;      // resident CTAs per SM of the device-tier gather kernel (measured optimum 3-5)
   // optional kernel timing (pool_profile_*)
@@ -282,6 +292,8 @@ namespace ft {
 // with the pool's device current
 int32_t gather_device_setup(ft_pool* p);
 int32_t plan_device_setup(ft_pool* p);
+int32_t gather_launch(ft_pool* p, const ft_plan* pl, uint32_t mb_begin, uint32_t mb_end, const void* embed_table,
+                      uint32_t vocab, void* out_embeds, int32_t* out_cu, int32_t* out_pos, uint32_t pad_L, cudaStream_t st);
 __global__ void k_page_table_init(uint64_t* pte, const uint32_t* bind, uint64_t n, uint64_t base, uint64_t frame_bytes,
                                   uint64_t flags);
 // uploads `bytes` from `src` (pageable) to the front of the pool's device scratch, asynchronously,

@@ -25,7 +25,7 @@ struct RowDesc {
   uint32_t off0;          // byte offset of the row inside its first page (0 for a text row)
   uint32_t shift;         // log2(page bytes); 31 for a text row (one segment)
   uint32_t nseg;          // 0 = nothing to copy
-  uint32_t pad;
+  uint32_t dst_shift;     // rows to add to the packed output row (padded layout), else 0
 };
 
 struct GatherArgs {
@@ -38,6 +38,7 @@ struct GatherArgs {
   int32_t* pos_ids;
   uint64_t call_seq;
   uint32_t write_index;  // this launch writes cu_seqlens / position ids
+  uint32_t pad_L;        // 0: packed rows; else every microbatch starts at a multiple of pad_L rows (padded layout)
   unsigned long long* tile_counter;  // device, zero at launch
 };
 
@@ -59,7 +60,7 @@ __global__ void __launch_bounds__(kGatherThreads) k_gather(PoolView v, PlanView 
     if (warp == 0) {
       const uint64_t row = tile * kTileRows + lane;
       RowDesc d;
-      d.nseg = 0; d.off0 = 0; d.shift = 31; d.pad = 0;
+      d.nseg = 0; d.off0 = 0; d.shift = 31; d.dst_shift = 0;
       if (row >= a.row_lo && row < a.row_hi) {
         // plan position of the sample holding this row: the tile's first sample, then a short walk
         uint32_t q = pl.tile_first_sample[tile];
@@ -67,7 +68,12 @@ __global__ void __launch_bounds__(kGatherThreads) k_gather(PoolView v, PlanView 
         while (row >= pl.sample_row_off[q + 1]) ++q;
         const uint32_t p = (uint32_t)(row - pl.sample_row_off[q]);
         const uint32_t slot = pl.mb_samples[q];
-        const uint64_t out_row = row - a.row_lo;
+        uint64_t out_row = row - a.row_lo;
+        if (a.pad_L) {  // padded layout: microbatch j of the range starts at row (j - mb_begin) * L
+          const uint32_t j = pl.plan_sample_mb[q];
+          d.dst_shift = (uint32_t)((uint64_t)(j - a.mb_begin) * a.pad_L - (pl.mb_row_off[j] - a.row_lo));
+          out_row += d.dst_shift;
+        }
         if (a.write_index) {
           a.pos_ids[out_row] = (int32_t)p;
           if (p == 0) {  // cu_seqlens: every sample writes its start; the last of a microbatch also the end
@@ -128,7 +134,7 @@ __global__ void __launch_bounds__(kGatherThreads) k_gather(PoolView v, PlanView 
       const uint32_t nseg = desc[r].nseg;
       if (nseg == 0) continue;
       const uint32_t off0 = desc[r].off0, shift = desc[r].shift, mask = (1u << shift) - 1;
-      uint4* dst = reinterpret_cast<uint4*>(a.out + (tile * kTileRows + r - a.row_lo) * v.row_bytes);
+      uint4* dst = reinterpret_cast<uint4*>(a.out + (tile * kTileRows + r - a.row_lo + desc[r].dst_shift) * v.row_bytes);
       auto src_of = [&](uint32_t x, bool* take) -> const uint4* {
         const uint32_t ab = off0 + (x << 4);
         const uint64_t pte = desc[r].seg[ab >> shift];
@@ -173,7 +179,11 @@ __global__ void __launch_bounds__(32) k_gather_host_bulk(PoolView v, PlanView pl
   uint64_t item = 0;
   for (uint32_t q = a.q_lo; q < a.q_hi; ++q) {
     const uint32_t slot = pl.mb_samples[q], ns = v.s_n_spans[slot];
-    const uint64_t row0 = pl.sample_row_off[q] - a.row_lo;
+    uint64_t row0 = pl.sample_row_off[q] - a.row_lo;
+    if (a.pad_L) {
+      const uint32_t mb = pl.plan_sample_mb[q];
+      row0 += (uint64_t)(mb - a.mb_begin) * a.pad_L - (pl.mb_row_off[mb] - a.row_lo);
+    }
     for (uint32_t j = 0; j < ns; ++j) {
       const uint32_t sid = slot * v.spans_per_sample + j;
       const uint32_t npages = v.sp_npages[sid];
@@ -214,45 +224,22 @@ int32_t gather_device_setup(ft_pool* p) {
 }
 }  // namespace ft
 
-using namespace ft;
-
-extern "C" __attribute__((visibility("default"))) int32_t pool_gather_packed(ft_pool* p, const ft_plan* pl, uint32_t mb_begin, uint32_t mb_end,
-                                      const void* embed_table, uint32_t vocab, void* out_embeds, int32_t* out_cu,
-                                      int32_t* out_pos, void* stream) {
-  if (!p || !pl || pl->pool != p) return FT_ERR_INVALID_ARG;
-  p->call_seq++;
-  if (mb_begin > mb_end || mb_end > pl->n_mb) return FT_ERR_INVALID_ARG;
-  // a plan dies with any of its samples (freed, or never completed under ALLOW_UNWRITTEN)
-  if (pl->free_epoch != p->free_epoch || (pl->cfg.flags & FT_PLAN_ALLOW_UNWRITTEN)) {
-    for (uint32_t t = 0; t < pl->n; ++t) {
-      const ft_slot_mirror& s = p->slots[pl->slots[t]];
-      if (s.state != FT_SLOT_READY || s.generation != pl->slot_generation[t]) return FT_ERR_NOT_READY;
-    }
-  }
-  if (mb_begin == mb_end) return FT_OK;
-  if (!embed_table || !out_embeds || !out_cu || !out_pos) return FT_ERR_INVALID_ARG;
-  if (reinterpret_cast<uintptr_t>(out_embeds) & 15 || reinterpret_cast<uintptr_t>(embed_table) & 15) return FT_ERR_INVALID_ARG;
-  if (p->view.row_bytes > (kMaxSeg - 1) * 4096) return FT_ERR_CAPACITY;
-
-  PlanView pv;
-  pv.n = pl->n; pv.n_mb = pl->n_mb; pv.n_ranks = pl->cfg.n_ranks_N;
-  pv.mb_samples = pl->d_mb_samples; pv.plan_sample_mb = pl->d_plan_sample_mb;
-  pv.sample_row_off = pl->d_sample_row_off; pv.mb_sample_off = pl->d_mb_sample_off;
-  pv.mb_row_off = pl->d_mb_row_off; pv.tile_first_sample = pl->d_tile_first_sample;
+namespace ft {
+// The launches of one assembly call over microbatches [mb_begin, mb_end): one k_gather, or one per tier.
+// pad_L = 0: packed rows, cu_seqlens and position ids written; pad_L = L: rows land in the padded layout and
+// the index outputs are left to the caller.  Arguments are validated by the caller.
+int32_t gather_launch(ft_pool* p, const ft_plan* pl, uint32_t mb_begin, uint32_t mb_end, const void* embed_table,
+                      uint32_t vocab, void* out_embeds, int32_t* out_cu, int32_t* out_pos, uint32_t pad_L, cudaStream_t st) {
+  const PlanView pv = make_plan_view(pl);
   GatherArgs a;
   a.q_lo = pl->h_mb_sample_off[mb_begin]; a.q_hi = pl->h_mb_sample_off[mb_end]; a.mb_begin = mb_begin;
   a.row_lo = pl->h_mb_row_off[mb_begin]; a.row_hi = pl->h_mb_row_off[mb_end];
   a.table = static_cast<const uint8_t*>(embed_table); a.vocab = vocab;
   a.out = static_cast<uint8_t*>(out_embeds); a.cu = out_cu; a.pos_ids = out_pos;
-  a.call_seq = p->call_seq; a.write_index = 1;
-  {
-    const int32_t rc0 = begin_consumer(p, static_cast<cudaStream_t>(stream));  // writes issued on another stream come first
-    if (rc0 != FT_OK) return rc0;
-  }
+  a.call_seq = p->call_seq; a.write_index = pad_L == 0; a.pad_L = pad_L;
   a.tile_counter = p->view.status + 1;  // scratch word next to the status word
-  FT_CUDA(cudaMemsetAsync(a.tile_counter, 0, 8, static_cast<cudaStream_t>(stream)));
+  FT_CUDA(cudaMemsetAsync(a.tile_counter, 0, 8, st));
   const uint64_t n_tiles = (a.row_hi + kTileRows - 1) / kTileRows - a.row_lo / kTileRows;
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
   // the grid-stride tile loop assumes every CTA runs from the start: never launch more than fit at once
   auto launch = [&](auto kernel, int mode, uint64_t want_per_sm, const GatherArgs& args, cudaStream_t s) {
     const uint64_t resident = (uint64_t)std::max(1, p->occ_gather[mode][p->gather_unroll == 8 ? 1 : 0]);
@@ -284,8 +271,41 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_gather_packed(ft_
     FT_CUDA(cudaStreamWaitEvent(st, p->join_ev[1], 0));
     p->gpu_launches += 2;
   }
-  const_cast<ft_plan*>(pl)->last_stream = st;
   FT_CUDA(cudaGetLastError());
   p->bytes_gathered += (a.row_hi - a.row_lo) * 2ull * p->view.row_bytes;
+  return FT_OK;
+}
+}  // namespace ft
+
+using namespace ft;
+
+extern "C" __attribute__((visibility("default"))) int32_t pool_gather_packed(ft_pool* p, const ft_plan* pl, uint32_t mb_begin, uint32_t mb_end,
+                                      const void* embed_table, uint32_t vocab, void* out_embeds, int32_t* out_cu,
+                                      int32_t* out_pos, void* stream) {
+  if (!p || !pl || pl->pool != p) return FT_ERR_INVALID_ARG;
+  p->call_seq++;
+  if (mb_begin > mb_end || mb_end > pl->n_mb) return FT_ERR_INVALID_ARG;
+  // a plan dies with any of its samples (freed, or never completed under ALLOW_UNWRITTEN)
+  if (pl->free_epoch != p->free_epoch || (pl->cfg.flags & FT_PLAN_ALLOW_UNWRITTEN)) {
+    for (uint32_t t = 0; t < pl->n; ++t) {
+      const ft_slot_mirror& s = p->slots[pl->slots[t]];
+      if (s.state != FT_SLOT_READY || s.generation != pl->slot_generation[t]) return FT_ERR_NOT_READY;
+    }
+  }
+  if (mb_begin == mb_end) return FT_OK;
+  if (!embed_table || !out_embeds || !out_cu || !out_pos) return FT_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(out_embeds) & 15 || reinterpret_cast<uintptr_t>(embed_table) & 15) return FT_ERR_INVALID_ARG;
+  if (p->view.row_bytes > (kMaxSeg - 1) * 4096) return FT_ERR_CAPACITY;
+
+  {
+    const int32_t rc0 = begin_consumer(p, static_cast<cudaStream_t>(stream));  // writes issued on another stream come first
+    if (rc0 != FT_OK) return rc0;
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  {
+    const int32_t rc1 = gather_launch(p, pl, mb_begin, mb_end, embed_table, vocab, out_embeds, out_cu, out_pos, 0, st);
+    if (rc1 != FT_OK) return rc1;
+  }
+  const_cast<ft_plan*>(pl)->last_stream = st;
   return end_consumer(p, st);
 }

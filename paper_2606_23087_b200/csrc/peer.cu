@@ -89,6 +89,7 @@ __global__ void __launch_bounds__(256) k_import_fill(PoolView v, ImportCall c, u
     for (uint32_t j = 0; j < c.n_spans_of[t]; ++j) {
       const uint32_t sid = slot * v.spans_per_sample + j, g = c.span_begin[t] + j;
       v.sp_pos[sid] = c.span_pos[g]; v.sp_tokens[sid] = c.span_tok[g]; v.sp_npages[sid] = c.span_npages[g];
+      v.sp_grid[sid] = make_uint4(0, 0, 0, 0);
     }
   }
   if (t < total_pages) {

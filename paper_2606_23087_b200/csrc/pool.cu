@@ -120,6 +120,7 @@ __global__ void __launch_bounds__(1024) k_register_scan(PoolView v, RegisterCall
         v.sp_pos[sid] = c.span_pos[c.span_begin[i] + j];
         v.sp_tokens[sid] = c.span_tok[c.span_begin[i] + j];
         v.sp_npages[sid] = 0;
+        v.sp_grid[sid] = make_uint4(0, 0, 0, 0);
       }
     }
     uint64_t total, ex = block_exclusive_scan(ntp, &total);
@@ -607,6 +608,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_create(const ft_p
   if (const char* e = getenv("FLOWPOOL_CHUNK_SHIFT")) { int v = atoi(e); if (v >= 14 && v <= 21) p->chunk_shift = v; }
   if (const char* e = getenv("FLOWPOOL_SCATTER_GROUP")) { int v = atoi(e); if (v > 0) p->scatter_group = v; }
   if (const char* e = getenv("FLOWPOOL_SCATTER_CTAS_PER_SM")) { int v = atoi(e); if (v > 0) p->scatter_ctas_per_sm = v; }
+  if (const char* e = getenv("FLOWPOOL_GRAD_CTAS_PER_SM")) { int v = atoi(e); if (v > 0 && v <= 8) p->grad_ctas_per_sm = v; }
   if (const char* e = getenv("FLOWPOOL_GATHER_U")) { int v = atoi(e); if (v == 4 || v == 8) p->gather_unroll = v; }
   if (const char* e = getenv("FLOWPOOL_DEV_CTAS_PER_SM")) { int v = atoi(e); if (v > 0) p->dev_ctas_per_sm = v; }
   for (int a = 0; a < 2; ++a) {
@@ -661,6 +663,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_create(const ft_p
   const size_t o_peers = take((size_t)c.world_size * sizeof(PeerTables));
   const size_t o_pos = take(span_ids * 4), o_tok = take(span_ids * 4), o_npg = take(span_ids * 4);
   const size_t o_blk = take(span_ids * MB * 4), o_lst = take(NB * kListBlock * 8);
+  const size_t o_grid = take(span_ids * sizeof(uint4));
   CK(cudaMalloc(&p->d_meta, off));
   CK(cudaMemset(p->d_meta, 0, off));
   uint8_t* m = static_cast<uint8_t*>(p->d_meta);
@@ -693,6 +696,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_create(const ft_p
   v.sp_pos = reinterpret_cast<uint32_t*>(m + o_pos); v.sp_tokens = reinterpret_cast<uint32_t*>(m + o_tok);
   v.sp_npages = reinterpret_cast<uint32_t*>(m + o_npg); v.sp_blocks = reinterpret_cast<uint32_t*>(m + o_blk);
   v.list_blocks = reinterpret_cast<uint64_t*>(m + o_lst);
+  v.sp_grid = reinterpret_cast<uint4*>(m + o_grid);
 
   // binding (identity or seeded permutation per tier) and the initial ring order are made on the host, once
   std::vector<uint32_t> bind_h(c.hbm_pages), bind_d(c.host_pages), ring(P);
