@@ -377,6 +377,8 @@ def kernel_breakdown(job, prof, steps):
     }
     out = {}
     for k, v in prof.items():
+        if k not in moved:
+            continue
         ms = v["ms"] / steps
         out[k] = {"ms_per_step": ms, "launches_per_step": v["launches"] / steps, "bytes_per_step": moved[k],
                   "gbs": (moved[k] / ms / 1e6) if ms > 0 else None}
@@ -471,6 +473,83 @@ def run_e2e(job, steps):
             "note": "value = steady state with the result copy-out of step k overlapping the inputs of step k+1"}
 
 
+def backbone_side(job, reps=3):
+    """Backbone-side outputs on the job's batch (device-resident, timed with CUDA events on the launching stream):
+    the padded assembly with positions, ids, labels and mask, and the ordered table gradient."""
+    import workloads
+    torch, pool, w = job.torch, job.pool, job.w
+    st = torch.cuda.current_stream().cuda_stream
+    for c in job.calls:
+        job.check(pool.register_samples(*c["reg"], c["ids"].data_ptr(), st), "register")
+        job.check(pool.write_embeddings(*c["wr"], c["ptrs"], w.src_dtype, st), "write")
+    items = [(s, j, workloads.span_grid(w, s, j)) for s in range(w.n_samples) for j in range(int(w.n_spans[s]))]
+    items = [it for it in items if it[2] is not None]
+    job.check(pool.set_span_grids([s for s, _, _ in items], [j for _, j, _ in items], [g for _, _, g in items], st), "pool_set_span_grids")
+    rc, plan = pool.plan_microbatches(job.order, job.pcfg, st)
+    job.check(rc, "plan")
+    a = plan.arrays()
+    n_mb, L, H = int(a["n_mb"]), w.budget_L, w.hidden
+    per_call = max(1, job.out.shape[0] // L)       # microbatches whose padded rows fit the job's output buffer
+    rows_cap = per_call * L
+    out = job.out if job.out.shape[0] >= rows_cap else torch.empty((rows_cap, H), dtype=torch.bfloat16, device="cuda")
+    cu = torch.empty((w.n_samples + 2 * n_mb + 8,), dtype=torch.int32, device="cuda")
+    pos3 = torch.empty((3 * rows_cap,), dtype=torch.int32, device="cuda")
+    ids = torch.empty((rows_cap,), dtype=torch.int32, device="cuda")
+    labels = torch.empty((rows_cap,), dtype=torch.int32, device="cuda")
+    mask = torch.empty((rows_cap,), dtype=torch.uint8, device="cuda")
+
+    def timed(fn):
+        best = []
+        for _ in range(reps + 1):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            best.append(e0.elapsed_time(e1))
+        return float(np.median(best[1:]))
+
+    def padded_all():
+        for b in range(0, n_mb, per_call):
+            e = min(n_mb, b + per_call)
+            job.check(pool.gather_padded(plan, b, e, job.table.data_ptr(), w.vocab, 0, out.data_ptr(), cu.data_ptr(),
+                                         pos3.data_ptr(), ids.data_ptr(), labels.data_ptr(), mask.data_ptr(), st), "pool_gather_padded")
+
+    def packed_all():
+        job.check(pool.gather_packed(plan, 0, n_mb, job.table.data_ptr(), w.vocab, job.out.data_ptr(), job.cu.data_ptr(),
+                                     job.pos.data_ptr(), st), "pool_gather_packed")
+
+    ms_packed = timed(packed_all)
+    ms_padded = timed(padded_all)
+    pad_rows = n_mb * L - w.total_tokens
+    padded_bytes = w.total_tokens * 4 * H + pad_rows * 2 * H + n_mb * L * 21   # rows read+written, zero rows, 21 index bytes per row
+    # table gradient: the assembled rows stand in for the gradient (bf16 values of unit scale), packed layout
+    packed_all()
+    grad_table = torch.zeros((w.vocab, H), dtype=torch.float32, device="cuda")
+    pool.profile_read()
+    pool.profile_enable(True)
+    ms_grad_call = timed(lambda: job.check(pool.embed_grad(plan, 0, n_mb, False, job.out.data_ptr(), grad_table.data_ptr(),
+                                                           w.vocab, st), "pool_embed_grad"))
+    prof = pool.profile_read()["embed_grad"]
+    pool.profile_enable(False)
+    ms_grad_kernel = prof["ms"] / max(1, prof["launches"])
+    text_rows = w.total_tokens - w.total_vision_tokens
+    grad_bytes = text_rows * 10 * H + w.total_tokens * 8       # bf16 row in, fp32 row read and written; row ids written and read
+    peak = measured_peak()[0]
+    job.check(pool.free(job.order, st), "free")
+    plan.destroy()
+    torch.cuda.synchronize()
+    return {
+        "gather_packed_ms": ms_packed,
+        "gather_padded": {"ms": ms_padded, "calls": -(-n_mb // per_call), "padding_rows": int(pad_rows), "algorithmic_bytes": int(padded_bytes),
+                          "gbs": padded_bytes / ms_padded / 1e6, "frac_of_measured_peak": padded_bytes / ms_padded / 1e6 / peak,
+                          "outputs": "embeds, cu_seqlens, 3-component positions, ids, labels, loss mask"},
+        "embed_grad": {"ms_call": ms_grad_call, "ms_kernel": ms_grad_kernel, "text_rows": int(text_rows), "algorithmic_bytes": int(grad_bytes),
+                       "gbs": grad_bytes / ms_grad_kernel / 1e6, "frac_of_measured_peak": grad_bytes / ms_grad_kernel / 1e6 / peak,
+                       "bound": "hbm", "note": "10H bytes per text row (bf16 gradient row in, fp32 table row read and written); ids uniform over the vocabulary"},
+    }
+
+
 def run_ours(args):
     import torch
     if not torch.cuda.is_available():
@@ -533,6 +612,8 @@ def run_ours(args):
         else:
             line["e2e"] = {"value": None, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
                            "note": "measured at --gpus 1"}
+    if rank == 0 and world == 1 and args.all_hbm and not args.skip_variants:
+        line["backbone_side"] = backbone_side(job)
     # all-HBM variant of the same batch (the benchmark spec's target is stated for HBM-resident pools)
     if not args.all_hbm and not args.skip_variants:
         job.close()
@@ -546,6 +627,8 @@ def run_ours(args):
                                        "tokens_per_s": world * w.total_tokens / ms2 * 1e3, "kernels": kern2,
                                        "phase_ms": phases2,
                                        "gather_frac_of_measured_peak": g2["gbs"] / measured_peak()[0] if g2["gbs"] else None}
+            if world == 1:
+                line["all_hbm_variant"]["backbone_side"] = backbone_side(job)
     job.close()
     del job          # its resident inputs and outputs go before the streaming measurement builds its own
     import gc

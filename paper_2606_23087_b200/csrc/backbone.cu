@@ -160,15 +160,26 @@ __global__ void __launch_bounds__(256) k_backbone_index(PoolView v, PlanView pl,
   a.pos3[R] = c0; a.pos3[a.lay.rows + R] = c1; a.pos3[2 * a.lay.rows + R] = c2;
 }
 
-// Zero rows behind the last token of each microbatch of the range.  8 CTAs per microbatch.
-constexpr uint32_t kPadCtasPerMb = 8;
+// Zero rows behind the last token of each microbatch of the range.  The padding of all microbatches, cut into
+// 64 KiB chunks, is dealt round-robin over the CTAs of a grid that fills the device once, so one nearly empty
+// microbatch (the last of a plan) is zeroed by the whole grid, not by a few CTAs.
+constexpr uint32_t kPadChunkVecs = 4096;  // 16-byte vectors per chunk
 __global__ void __launch_bounds__(256) k_pad_zero(PlanView pl, LayoutArgs a, uint32_t row_bytes, uint8_t* out) {
-  const uint32_t j = a.mb_begin + blockIdx.x / kPadCtasPerMb, part = blockIdx.x % kPadCtasPerMb;
-  const uint64_t tokens = pl.mb_row_off[j + 1] - pl.mb_row_off[j];
-  uint4* dst = reinterpret_cast<uint4*>(out + ((uint64_t)(j - a.mb_begin) * a.L + tokens) * row_bytes);
-  const uint64_t vecs = (a.L - tokens) * (uint64_t)(row_bytes >> 4);
   const uint4 z = make_uint4(0, 0, 0, 0);
-  for (uint64_t x = (uint64_t)part * blockDim.x + threadIdx.x; x < vecs; x += (uint64_t)kPadCtasPerMb * blockDim.x) __stcs(dst + x, z);
+  uint64_t base = 0;  // chunks of the microbatches before j
+  for (uint32_t j = a.mb_begin; j < a.mb_end; ++j) {
+    const uint64_t tokens = pl.mb_row_off[j + 1] - pl.mb_row_off[j];
+    const uint64_t vecs = (a.L - tokens) * (uint64_t)(row_bytes >> 4);
+    const uint64_t chunks = (vecs + kPadChunkVecs - 1) / kPadChunkVecs;
+    uint4* dst = reinterpret_cast<uint4*>(out + ((uint64_t)(j - a.mb_begin) * a.L + tokens) * row_bytes);
+    // this CTA's chunks of microbatch j: global chunk index base + k congruent to blockIdx.x modulo the grid
+    uint64_t k = (blockIdx.x + gridDim.x - base % gridDim.x) % gridDim.x;
+    for (; k < chunks; k += gridDim.x) {
+      const uint64_t x0 = k * kPadChunkVecs, x1 = min(vecs, x0 + kPadChunkVecs);
+      for (uint64_t x = x0 + threadIdx.x; x < x1; x += blockDim.x) __stcs(dst + x, z);
+    }
+    base += chunks;
+  }
 }
 
 }  // namespace ft
@@ -362,7 +373,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_gather_padded(ft_
     if (rc1 != FT_OK) return rc1;
   }
   const PlanView pv = make_plan_view(pl);
-  k_pad_zero<<<(mb_end - mb_begin) * kPadCtasPerMb, 256, 0, st>>>(pv, lay, p->view.row_bytes, static_cast<uint8_t*>(out_embeds));
+  k_pad_zero<<<(unsigned)p->sm_count * 8, 256, 0, st>>>(pv, lay, p->view.row_bytes, static_cast<uint8_t*>(out_embeds));
   IndexArgs ia;
   ia.lay = lay; ia.pad_id = pad_id; ia.cu = out_cu; ia.pos3 = out_pos3; ia.ids = out_ids; ia.labels = out_labels;
   ia.mask = out_mask; ia.call_seq = p->call_seq;

@@ -87,3 +87,152 @@ def test_full_size_plan_and_sampled_rows(name, kw):
     assert not bool((out == -1).all(dim=1).any().item())
     oplan.destroy()
     run.close()
+
+
+def _oracle_samples(w, samples):
+    """Oracle pool holding only the given samples (slot k = k-th of them), written, gridded, planned together;
+    returns per-sample (positions [3, n], ids, labels, mask) read from its padded assembly."""
+    from harness import host_span, pool_config_fields
+    from oracle import OraclePool, PoolConfig
+    f = pool_config_fields(w, max_samples=len(samples))
+    need = sum(w.pages_of_span(int(t)) for s in samples for t in w.spans_of(s)[1])
+    f.update(hbm_pages=need + 2, host_pages=0, max_text_tokens=int(sum(int(w.seq_len[s]) for s in samples)) + 1024 * len(samples))
+    pool = OraclePool(PoolConfig(**f))
+    assert pool.rc == 0
+    for k, s in enumerate(samples):
+        pos, tok = w.spans_of(s)
+        assert pool.register_samples([k], [int(w.seq_len[s])], [len(pos)], pos, tok, workloads.input_ids(w, s)) == 0
+        if len(pos):
+            assert pool.write_embeddings([k] * len(pos), list(range(len(pos))), tok, [host_span(w, s, j) for j in range(len(pos))], w.src_dtype) == 0
+        items = [(j, workloads.span_grid(w, s, j)) for j in range(len(pos))]
+        items = [it for it in items if it[1] is not None]
+        assert pool.set_span_grids([k] * len(items), [j for j, _ in items], [g for _, g in items]) == 0
+    cfg = plan_config_fields(w)
+    rc, plan = pool.plan_microbatches(list(range(len(samples))), PlanConfig(**cfg))
+    assert rc == 0
+    a = plan.arrays()
+    n_mb, L = int(a["n_mb"]), w.budget_L
+    rows = n_mb * L
+    o = dict(out=np.zeros((rows, w.hidden), np.uint16), cu=np.zeros(len(samples) + 2 * n_mb, np.int32), pos3=np.zeros((3, rows), np.int32),
+             ids=np.zeros(rows, np.int32), labels=np.zeros(rows, np.int32), mask=np.zeros(rows, np.uint8))
+    table = np.zeros((w.vocab, w.hidden), np.uint16)
+    assert pool.gather_padded(plan, 0, n_mb, table, 0, o["out"], o["cu"], o["pos3"], o["ids"], o["labels"], o["mask"]) == 0
+    res = {}
+    for j in range(n_mb):
+        row = j * L
+        for k in a["mb_samples"][a["mb_sample_off"][j]:a["mb_sample_off"][j + 1]]:
+            n = int(w.seq_len[samples[int(k)]])
+            res[samples[int(k)]] = (o["pos3"][:, row:row + n].copy(), o["ids"][row:row + n].copy(),
+                                   o["labels"][row:row + n].copy(), o["mask"][row:row + n].copy())
+            row += n
+    plan.destroy()
+    pool.destroy()
+    return res
+
+
+@pytest.mark.parametrize("name", ["image_mix_7b", "video_heavy"])
+def test_full_size_backbone_side(name):
+    """Padded assembly and table gradient at the benchmark's size.  Rows: equal to the packed assembly (itself
+    checked above), zero padding.  Ids, labels, mask: in full against the generator's ids.  Positions: sampled
+    samples against the oracle.  Gradient: small-integer gradients against an exact scatter-add by a library
+    routine, and sampled table rows of a real-valued run against sequential fp32 addition in row order."""
+    if not torch.cuda.is_available():
+        pytest.fail("a CUDA device is required for -m gpu tests")
+    from gpu_harness import CudaRun, cuda_stream
+    w = workloads.make_workload(name)
+    run = CudaRun(w)
+    for call in w.write_calls:
+        samples = sorted({s for s, _ in call}, key=[s for s, _ in call].index)
+        assert run.register(samples) == 0
+        assert run.write(call, keep_src=False) == 0
+    items = [(s, j, workloads.span_grid(w, s, j)) for s in range(w.n_samples) for j in range(int(w.n_spans[s]))]
+    items = [it for it in items if it[2] is not None]
+    assert run.pool.set_span_grids([s for s, _, _ in items], [j for _, j, _ in items], [g for _, _, g in items], cuda_stream()) == 0
+    rc, plan = run.plan()
+    assert rc == 0
+    a = plan.arrays()
+    n_mb, L, H = int(a["n_mb"]), w.budget_L, w.hidden
+    rc, packed, _, packed_pos = run.gather_all()
+    assert rc == 0
+    lens = w.seq_len[a["mb_samples"]].astype(np.int64)
+    all_ids = np.concatenate([workloads.input_ids(w, int(s)) for s in a["mb_samples"]])
+    nxt_text = np.concatenate([np.append(workloads.input_ids(w, int(s))[1:] != w.placeholder_id, False) for s in a["mb_samples"]])
+    nxt_id = np.concatenate([np.append(workloads.input_ids(w, int(s))[1:], 0) for s in a["mb_samples"]])
+    picked = [int(s) for s in np.random.default_rng(3).choice(a["mb_samples"], size=5, replace=False)]
+    exp_s = _oracle_samples(w, picked)
+    per_call = max(1, min(n_mb, (1 << 20) // L))
+    rows_cap = per_call * L
+    out = torch.empty((rows_cap, H), dtype=torch.int16, device="cuda")
+    cu = torch.empty((w.n_samples + 2 * n_mb,), dtype=torch.int32, device="cuda")
+    pos3 = torch.empty((3 * rows_cap,), dtype=torch.int32, device="cuda")
+    ids, labels = (torch.empty((rows_cap,), dtype=torch.int32, device="cuda") for _ in range(2))
+    mask = torch.empty((rows_cap,), dtype=torch.uint8, device="cuda")
+    row_off = np.concatenate([[0], np.cumsum(lens)])
+    seen = 0
+    for b in range(0, n_mb, per_call):
+        e = min(n_mb, b + per_call)
+        rows = (e - b) * L
+        out.fill_(-1); pos3.fill_(-7); ids.fill_(-7); labels.fill_(-7); mask.fill_(7); cu.fill_(-7)
+        assert run.pool.gather_padded(plan, b, e, run.table.data_ptr(), w.vocab, -2, out.data_ptr(), cu.data_ptr(), pos3.data_ptr(),
+                                      ids.data_ptr(), labels.data_ptr(), mask.data_ptr(), cuda_stream()) == 0
+        torch.cuda.synchronize()
+        h_ids, h_lab, h_mask = ids[:rows].cpu().numpy(), labels[:rows].cpu().numpy(), mask[:rows].cpu().numpy()
+        h_pos = pos3[:3 * rows].cpu().numpy().reshape(3, rows)
+        h_cu = cu.cpu().numpy()
+        cu_w = 0
+        for j in range(b, e):
+            q0, q1 = int(a["mb_sample_off"][j]), int(a["mb_sample_off"][j + 1])
+            t = int(a["mb_tokens"][j])
+            r0, R0 = int(row_off[q0]), (j - b) * L
+            assert torch.equal(out[R0:R0 + t], packed[r0:r0 + t])
+            assert not bool(out[R0 + t:R0 + L].any().item())
+            assert np.array_equal(h_ids[R0:R0 + t], all_ids[r0:r0 + t]) and np.all(h_ids[R0 + t:R0 + L] == -2)
+            assert np.array_equal(h_mask[R0:R0 + t], nxt_text[r0:r0 + t].astype(np.uint8)) and not h_mask[R0 + t:R0 + L].any()
+            assert np.array_equal(h_lab[R0:R0 + t], np.where(nxt_text[r0:r0 + t], nxt_id[r0:r0 + t], -100)) and np.all(h_lab[R0 + t:R0 + L] == -100)
+            assert not h_pos[:, R0 + t:R0 + L].any()
+            exp_cu = np.concatenate([[0], np.cumsum(lens[q0:q1]), [L]]).astype(np.int32)
+            assert np.array_equal(h_cu[cu_w:cu_w + len(exp_cu)], exp_cu)
+            cu_w += len(exp_cu)
+            for q in range(q0, q1):
+                s = int(a["mb_samples"][q])
+                if s in exp_s:
+                    R = R0 + int(row_off[q]) - r0
+                    n = int(lens[q])
+                    assert np.array_equal(h_pos[:, R:R + n], exp_s[s][0]) and np.array_equal(h_lab[R:R + n], exp_s[s][2])
+                    seen += 1
+    assert seen == len(picked)
+    del out
+    # gradient, packed layout over the whole plan
+    total = int(lens.sum())
+    text_rows = torch.from_numpy(np.nonzero(all_ids != w.placeholder_id)[0]).cuda()
+    text_ids = torch.from_numpy(all_ids[all_ids != w.placeholder_id].astype(np.int64)).cuda()
+    grad = packed   # reuse the buffer: small integers first
+    torch.manual_seed(5)
+    step = 1 << 18
+    for r in range(0, total, step):
+        grad[r:r + step] = torch.randint(-8, 9, (min(step, total - r), H), device="cuda", dtype=torch.int16).to(torch.bfloat16).view(torch.int16)
+    gt = torch.zeros((w.vocab, H), dtype=torch.float32, device="cuda")
+    assert run.pool.embed_grad(plan, 0, n_mb, False, grad.data_ptr(), gt.data_ptr(), w.vocab, cuda_stream()) == 0
+    ref = torch.zeros((w.vocab, H), dtype=torch.float32, device="cuda")
+    for r in range(0, len(text_rows), step):
+        ref.index_add_(0, text_ids[r:r + step], grad[text_rows[r:r + step]].view(torch.bfloat16).float())   # small integers: exact in any order
+    torch.cuda.synchronize()
+    assert torch.equal(gt, ref)
+    del ref
+    # real values: sampled table rows against sequential fp32 addition in ascending row order
+    for r in range(0, total, step):
+        grad[r:r + step] = workloads.grad_values(w, r, min(total, r + step), device="cuda").view(torch.int16)
+    gt.zero_()
+    assert run.pool.embed_grad(plan, 0, n_mb, False, grad.data_ptr(), gt.data_ptr(), w.vocab, cuda_stream()) == 0
+    torch.cuda.synchronize()
+    ids_np = all_ids
+    counts = np.bincount(ids_np[ids_np != w.placeholder_id], minlength=w.vocab)
+    for v in [int(np.argmax(counts)), int(np.argmin(np.where(counts > 0, counts, 1 << 30))), 17, w.vocab - 2]:
+        rows_v = np.nonzero(ids_np == v)[0]
+        acc = np.zeros(H, np.float32)
+        g_rows = grad[torch.from_numpy(rows_v).cuda()].view(torch.bfloat16).float().cpu().numpy() if len(rows_v) else np.zeros((0, H), np.float32)
+        for k in range(len(rows_v)):
+            acc = acc + g_rows[k]          # float32 + float32, one rounding per element, in row order
+        assert np.array_equal(gt[v].cpu().numpy().view(np.uint32), acc.view(np.uint32)), v
+    assert run.pool.status() == (0, 0)
+    run.close()
