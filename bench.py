@@ -550,6 +550,18 @@ def backbone_side(job, reps=3):
     }
 
 
+def run_backbone_only(args):
+    """One JSON line with the backbone-side measurements alone (small cases for profiler captures)."""
+    import torch
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback for the product path)")
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    job = DeviceJob(args, True)
+    res = backbone_side(job, reps=max(1, args.steps))
+    job.close()
+    print(json.dumps({"workload": workload_label(args) + " (all HBM)", "samples": job.w.n_samples, "backbone_side": res}))
+
+
 def run_ours(args):
     import torch
     if not torch.cuda.is_available():
@@ -965,6 +977,7 @@ def main():
     ap.add_argument("--page-bytes", type=int, default=2 << 20, help="frag_sweep: page size")
     ap.add_argument("--pool-gib", type=float, default=64.0, help="frag_sweep: pool capacity")
     ap.add_argument("--cycles", type=int, default=10, help="frag_sweep: write/free cycles")
+    ap.add_argument("--backbone-only", action="store_true", help="only the backbone-side outputs (padded assembly, table gradient) on an all-HBM pool")
     ap.add_argument("--via-peer", action="store_true", help="producer and consumer are two processes' pools of one GVA space")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -972,6 +985,8 @@ def main():
         run_reference(args)
     elif args.workload == "frag_sweep":
         run_sweep(args)
+    elif args.backbone_only:
+        run_backbone_only(args)
     elif args.via_peer:
         run_peer(args)
     else:
