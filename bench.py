@@ -186,7 +186,7 @@ class DeviceJob:
         from harness import pool_config_fields, plan_config_fields, register_args, write_args
         from paper_2606_23087_b200 import binding as fp
         self.torch, self.fp = torch, fp
-        w = workloads.make_workload(args.workload, n_samples=args.samples, all_hbm=all_hbm)
+        w = workloads.make_workload(args.workload, n_samples=args.samples, all_hbm=all_hbm, id_skew=getattr(args, "id_skew", "uniform"))
         self.w = w
         self.pool = fp.Pool(fp.PoolConfig(**pool_config_fields(w)))
         if self.pool.rc != 0:
@@ -546,7 +546,7 @@ def backbone_side(job, reps=3):
                           "outputs": "embeds, cu_seqlens, 3-component positions, ids, labels, loss mask"},
         "embed_grad": {"ms_call": ms_grad_call, "ms_kernel": ms_grad_kernel, "text_rows": int(text_rows), "algorithmic_bytes": int(grad_bytes),
                        "gbs": grad_bytes / ms_grad_kernel / 1e6, "frac_of_measured_peak": grad_bytes / ms_grad_kernel / 1e6 / peak,
-                       "bound": "hbm", "note": "10H bytes per text row (bf16 gradient row in, fp32 table row read and written); ids uniform over the vocabulary"},
+                       "bound": "hbm", "ids": w.id_skew, "note": "10H bytes per text row (bf16 gradient row in, fp32 table row read and written)"},
     }
 
 
@@ -808,7 +808,7 @@ def run_streaming(args, all_hbm, batches=6, warm=2):
     import workloads
     from harness import pool_config_fields, plan_config_fields, register_args, write_args
     from paper_2606_23087_b200 import binding as fp
-    w = workloads.make_workload(args.workload, n_samples=args.samples, all_hbm=all_hbm)
+    w = workloads.make_workload(args.workload, n_samples=args.samples, all_hbm=all_hbm, id_skew=getattr(args, "id_skew", "uniform"))
     n = w.n_samples
     f = pool_config_fields(w, max_samples=2 * n)
     f["hbm_pages"], f["host_pages"] = 2 * w.hbm_pages, 2 * w.host_pages
@@ -977,6 +977,7 @@ def main():
     ap.add_argument("--page-bytes", type=int, default=2 << 20, help="frag_sweep: page size")
     ap.add_argument("--pool-gib", type=float, default=64.0, help="frag_sweep: pool capacity")
     ap.add_argument("--cycles", type=int, default=10, help="frag_sweep: write/free cycles")
+    ap.add_argument("--id-skew", default="uniform", choices=["uniform", "zipf"], help="distribution of the text-token ids")
     ap.add_argument("--backbone-only", action="store_true", help="only the backbone-side outputs (padded assembly, table gradient) on an all-HBM pool")
     ap.add_argument("--via-peer", action="store_true", help="producer and consumer are two processes' pools of one GVA space")
     args = ap.parse_args()

@@ -278,6 +278,8 @@ struct ft_pool {
   int chunk_shift = 16;         // log2 of k_scatter's work unit in bytes of a span's image (14..21)
   int scatter_group = 0;        // chunks per round-robin group of k_scatter; 0 = the measured default
   int scatter_ctas_per_sm = 0;  // resident CTAs per SM of the device-tier scatter kernel; 0 = the measured default
+  bool grad_attr_set = false;   // k_embed_grad_hot's shared-memory opt-in done
+  int grad_hot_threshold = 0;   // rows from which an id takes k_embed_grad_hot; 0 = rows / (8 x grid), at least 64
   int grad_ctas_per_sm = 6;     // CTAs per SM of k_embed_grad (each owns the table rows v with v % grid == its index)
   int gather_unroll = 4;        // 16-byte vectors per lane in flight in k_gather (4 or 8)
   int dev_ctas_per_sm = 4;      // resident CTAs per SM of the device-tier gather kernel (measured optimum 3-5)

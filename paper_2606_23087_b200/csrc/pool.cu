@@ -608,6 +608,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_create(const ft_p
   if (const char* e = getenv("FLOWPOOL_CHUNK_SHIFT")) { int v = atoi(e); if (v >= 14 && v <= 21) p->chunk_shift = v; }
   if (const char* e = getenv("FLOWPOOL_SCATTER_GROUP")) { int v = atoi(e); if (v > 0) p->scatter_group = v; }
   if (const char* e = getenv("FLOWPOOL_SCATTER_CTAS_PER_SM")) { int v = atoi(e); if (v > 0) p->scatter_ctas_per_sm = v; }
+  if (const char* e = getenv("FLOWPOOL_GRAD_HOT_THRESHOLD")) { int v = atoi(e); if (v > 0) p->grad_hot_threshold = v; }
   if (const char* e = getenv("FLOWPOOL_GRAD_CTAS_PER_SM")) { int v = atoi(e); if (v > 0 && v <= 8) p->grad_ctas_per_sm = v; }
   if (const char* e = getenv("FLOWPOOL_GATHER_U")) { int v = atoi(e); if (v == 4 || v == 8) p->gather_unroll = v; }
   if (const char* e = getenv("FLOWPOOL_DEV_CTAS_PER_SM")) { int v = atoi(e); if (v > 0) p->dev_ctas_per_sm = v; }

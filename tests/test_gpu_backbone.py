@@ -68,6 +68,7 @@ CASES = [
     ("image_mix_7b", dict(n_samples=40, hidden=56, page_bytes=4096)),   # narrow rows: one 16-byte vector chunk per 8 columns
     ("video_heavy", dict(n_samples=6)),                                 # up to 64 gridded spans per sample
     ("host_tier_stress", dict(n_samples=3)),                            # H = 8192, fp32 source
+    ("image_mix_7b", dict(n_samples=24, hidden=64, page_bytes=4096, id_skew="zipf")),   # frequent ids: long runs on one table row
 ]
 
 

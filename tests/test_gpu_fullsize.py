@@ -130,8 +130,8 @@ def _oracle_samples(w, samples):
     return res
 
 
-@pytest.mark.parametrize("name", ["image_mix_7b", "video_heavy"])
-def test_full_size_backbone_side(name):
+@pytest.mark.parametrize("name,id_skew", [("image_mix_7b", "uniform"), ("video_heavy", "uniform"), ("image_mix_7b", "zipf")])
+def test_full_size_backbone_side(name, id_skew):
     """Padded assembly and table gradient at the benchmark's size.  Rows: equal to the packed assembly (itself
     checked above), zero padding.  Ids, labels, mask: in full against the generator's ids.  Positions: sampled
     samples against the oracle.  Gradient: small-integer gradients against an exact scatter-add by a library
@@ -139,7 +139,7 @@ def test_full_size_backbone_side(name):
     if not torch.cuda.is_available():
         pytest.fail("a CUDA device is required for -m gpu tests")
     from gpu_harness import CudaRun, cuda_stream
-    w = workloads.make_workload(name)
+    w = workloads.make_workload(name, id_skew=id_skew)   # zipf: a few ids own most text rows (the frequent-id path)
     run = CudaRun(w)
     for call in w.write_calls:
         samples = sorted({s for s, _ in call}, key=[s for s, _ in call].index)

@@ -126,6 +126,7 @@ class Workload:
     max_spans_per_sample: int = 1
     max_pages_per_span: int = 1
     max_seq_len: int = 1
+    id_skew: str = "uniform"          # text-token ids: "uniform", or "zipf" (P(id = k) roughly proportional to 1 / (k + 1))
 
     @property
     def n_samples(self) -> int:
@@ -201,7 +202,7 @@ def _calls_by_sample(order, per_call, w):
 
 
 def make_workload(name: str, n_samples: int = None, page_bytes: int = None, hidden: int = None,
-                  all_hbm: bool = False, pool_bytes: int = None) -> Workload:
+                  all_hbm: bool = False, pool_bytes: int = None, id_skew: str = "uniform") -> Workload:
     """The five configurations; n_samples / hidden / page_bytes shrink them for parity tests."""
     if name == "tiny":  # seed 0
         seed, n = 0, n_samples or 16
@@ -267,6 +268,8 @@ def make_workload(name: str, n_samples: int = None, page_bytes: int = None, hidd
         raise ValueError(name)
     if all_hbm:
         w.hbm_pages, w.host_pages = w.hbm_pages + w.host_pages, 0
+    assert id_skew in ("uniform", "zipf")
+    w.id_skew = id_skew
     return w
 
 
@@ -305,9 +308,14 @@ def admit_free_schedule(w: Workload, cycles: int = 10):
 # ---------------------------------------------------------------------------------------------
 
 def input_ids(w: Workload, s: int) -> np.ndarray:
-    """int32[seq_len]: uniform ids in [0, vocab-2]; the placeholder id on every span's run."""
+    """int32[seq_len]: ids in [0, vocab-2], uniform or log-uniform (a Zipf-like head: id 0 is the most frequent);
+    the placeholder id on every span's run."""
     n = int(w.seq_len[s])
-    ids = randint(stream_key(w.seed, S_IDS, s), np.arange(n), 0, w.vocab - 2).astype(np.int32)
+    if w.id_skew == "zipf":
+        u = u01(stream_key(w.seed, S_IDS, s), np.arange(n))
+        ids = np.clip(np.floor(np.exp(u * np.log(w.vocab - 1.0))).astype(np.int64) - 1, 0, w.vocab - 2).astype(np.int32)
+    else:
+        ids = randint(stream_key(w.seed, S_IDS, s), np.arange(n), 0, w.vocab - 2).astype(np.int32)
     pos, tok = w.spans_of(s)
     for p, t in zip(pos, tok):
         ids[int(p):int(p) + int(t)] = w.placeholder_id
