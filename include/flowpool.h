@@ -386,8 +386,9 @@ int32_t pool_gather_padded(ft_pool* pool, const ft_plan* plan, uint32_t mb_begin
  *   grad_out    device bf16 [rows, H], 16-byte aligned
  *   grad_table  device fp32 [vocab, H], 16-byte aligned, accumulated in place
  * Errors: as pool_gather_packed; asynchronous: id outside [0, vocab) BAD_TOKEN_ID (row skipped).  Allocates
- * 4 bytes per row of stream-ordered scratch for the call.  One CTA owns each table row, so a batch whose text is
- * dominated by a single id serialises on that CTA.
+ * stream-ordered scratch for the call (about 16 bytes per row plus 8 bytes per table row).  Ids that own many
+ * rows are added by a separate kernel on the pool's second consumer-side stream; the call returns with `stream`
+ * ordered after both.
  */
 int32_t pool_embed_grad(ft_pool* pool, const ft_plan* plan, uint32_t mb_begin, uint32_t mb_end, uint32_t padded,
                         const void* grad_out, float* grad_table, uint32_t vocab, void* stream);
