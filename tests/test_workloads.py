@@ -86,3 +86,29 @@ def test_churn_schedule_respects_capacity():
     assert live == residents and sorted(live) == live        # admission order
     nxt = max(live) + 1
     assert nxt >= w.n_samples or w.pages_of_span(int(w.spans_of(nxt)[1][0])) > free   # the pool is full
+
+
+def test_zipf_like_ids_and_span_grids():
+    w = workloads.make_workload("image_mix_7b", n_samples=24, id_skew="zipf")
+    u = workloads.make_workload("image_mix_7b", n_samples=24)
+    ids = np.concatenate([workloads.input_ids(w, s) for s in range(w.n_samples)])
+    text = ids[ids != w.placeholder_id]
+    assert text.min() >= 0 and text.max() <= w.vocab - 2
+    # log-uniform: id 0 holds ln 2 / ln(vocab - 1) of the text tokens, and the layout is the uniform workload's
+    share0 = float((text == 0).mean())
+    assert abs(share0 - np.log(2.0) / np.log(w.vocab - 1.0)) < 0.01
+    assert np.array_equal(w.seq_len, u.seq_len) and np.array_equal(w.span_pos, u.span_pos)
+    assert np.array_equal(workloads.input_ids(w, 3), workloads.input_ids(w, 3))
+    for s in range(w.n_samples):
+        pos, tok = w.spans_of(s)
+        row = workloads.input_ids(w, s)
+        for j in range(len(pos)):
+            assert np.all(row[int(pos[j]):int(pos[j]) + int(tok[j])] == w.placeholder_id)
+            g = workloads.span_grid(w, s, j)
+            if g is not None:
+                assert g[0] * g[1] * g[2] == int(tok[j]) and min(g) >= 1 and g[0] in (1, 2) and g[2] <= g[1]
+    grids = [workloads.span_grid(w, s, j) for s in range(w.n_samples) for j in range(int(w.n_spans[s]))]
+    assert any(g is None for g in grids) and any(g is not None and g[0] == 2 for g in grids)
+    g0 = workloads.grad_values(w, 5, 9)
+    assert g0.dtype == torch.bfloat16 and g0.shape == (4, w.hidden) and torch.equal(g0, workloads.grad_values(w, 5, 9))
+    assert torch.equal(g0[1:], workloads.grad_values(w, 6, 9))   # a pure function of the row index
