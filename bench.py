@@ -535,6 +535,9 @@ def backbone_side(job, reps=3):
     ms_grad_kernel = prof["ms"] / max(1, prof["launches"])
     text_rows = w.total_tokens - w.total_vision_tokens
     grad_bytes = text_rows * 10 * H + w.total_tokens * 8       # bf16 row in, fp32 row read and written; row ids written and read
+    all_ids = np.concatenate([workloads.input_ids(w, s) for s in range(w.n_samples)])
+    distinct = int(len(np.unique(all_ids[all_ids != w.placeholder_id])))
+    floor_bytes = text_rows * 2 * H + distinct * 8 * H         # every gradient row once, every touched table row once
     peak = measured_peak()[0]
     job.check(pool.free(job.order, st), "free")
     plan.destroy()
