@@ -346,7 +346,8 @@ int32_t pool_import_samples(ft_pool* pool, const uint32_t* local_slot, uint32_t 
  * embedding table's.
  *
  * pool_set_span_grids -- token grid (T, H, W) of named spans, T*H*W = the span's tokens, tokens in row-major
- * (t, h, w) order.  A span keeps its grid until its sample is freed; a span without one counts as text below.
+ * (t, h, w) order.  A span keeps its grid until its sample is freed; a span without one counts as text below; of
+ * several items naming the same span the last one stays.
  *   slot, span_idx host [n]; grid_thw host [n][3].  All-or-nothing, first bad item in order: slot out of range
  *   INVALID_ARG, FREE slot UNKNOWN_SAMPLE, no such span INVALID_ARG, a zero extent or a product that is not the
  *   span's token count INVALID_ARG.  Asynchronous; ordered before later calls on any stream like a producer call.

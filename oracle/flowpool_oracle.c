@@ -1133,7 +1133,8 @@ int32_t oracle_plan_arrays(const oracle_plan* pl, uint32_t* mb_sample_off, uint3
  * ---------------------------------------------------------------------- */
 
 /* Token grid of a span: (T, H, W) with T*H*W = n_tokens, row-major (t, h, w).
- * All-or-nothing: the first bad item stops the call and nothing is stored. */
+ * All-or-nothing: the first bad item stops the call and nothing is stored.  Items are stored in order, so of
+ * several items naming the same span the last one stays. */
 int32_t oracle_pool_set_span_grids(oracle_pool* p, uint32_t n, const uint32_t* slot, const uint32_t* span_idx,
                                    const uint32_t* grid_thw) {
   if (!p) return OR_ERR_INVALID_ARG;

@@ -16,6 +16,7 @@
 //                    one list (row, id) for the rest
 //   k_embed_grad_hot one CTA per (frequent id, 256-column slice): streams the listed rows, adds in list order
 #include <algorithm>
+#include <unordered_set>
 #include <vector>
 
 #include "flowpool_internal.cuh"
@@ -561,13 +562,22 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_set_span_grids(ft
     const uint64_t th = (uint64_t)g[0] * g[1];
     if (th > tokens || th * g[2] != tokens) return FT_ERR_INVALID_ARG;
   }
+  // a span named more than once keeps its last grid: only that item is uploaded (the kernel writes in parallel)
+  std::vector<uint32_t> keep;
+  {
+    std::unordered_set<uint32_t> seen;
+    for (uint32_t i = n; i-- > 0;)
+      if (seen.insert(slot[i] * S + span_idx[i]).second) keep.push_back(i);
+  }
+  n = (uint32_t)keep.size();
   const size_t o_grid = 0, o_sid = align_up_sz((size_t)n * sizeof(uint4), 16), bytes = o_sid + (size_t)n * 4;
   std::vector<uint8_t> blob(bytes);
   uint4* hg = reinterpret_cast<uint4*>(blob.data() + o_grid);
   uint32_t* hs = reinterpret_cast<uint32_t*>(blob.data() + o_sid);
-  for (uint32_t i = 0; i < n; ++i) {
-    hg[i] = make_uint4(grid_thw[3ull * i], grid_thw[3ull * i + 1], grid_thw[3ull * i + 2], 0);
-    hs[i] = slot[i] * S + span_idx[i];
+  for (uint32_t k = 0; k < n; ++k) {
+    const uint32_t i = keep[k];
+    hg[k] = make_uint4(grid_thw[3ull * i], grid_thw[3ull * i + 1], grid_thw[3ull * i + 2], 0);
+    hs[k] = slot[i] * S + span_idx[i];
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   {

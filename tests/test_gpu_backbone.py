@@ -150,6 +150,7 @@ def test_grid_errors_and_lifetime_match_oracle():
         ([7], [0], [[1, 1, n0]]),            # slot out of range
         ([0], [0], [[65536, 65536, 1]]),     # product wraps 32 bits: still rejected
         ([], [], np.zeros((0, 3))),          # empty call
+        ([0, 1, 0], [0, 0, 0], [[1, n0, 1], [1, 1, int(w.spans_of(1)[1][0])], [n0, 1, 1]]),   # a span named twice: the last item stays
     ]
     for slots, spans, grids in calls:
         assert r.pool.set_span_grids(slots, spans, grids, gh.cuda_stream()) == op.set_span_grids(slots, spans, grids)

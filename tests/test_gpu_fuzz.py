@@ -34,7 +34,7 @@ def test_random_call_sequences_agree_with_oracle(seed, ring_order, page_bytes, h
     table = workloads.embed_table(w, device="cuda")
     table_h = bits16(table)
     keep, plans = [], []
-    n_calls = {"register": 0, "write": 0, "free": 0, "plan": 0, "gather": 0}
+    n_calls = {"register": 0, "write": 0, "free": 0, "plan": 0, "gather": 0, "grids": 0, "padded": 0, "grad": 0}
     n_ok = dict(n_calls)
 
     def check_state():
@@ -50,7 +50,7 @@ def test_random_call_sequences_agree_with_oracle(seed, ring_order, page_bytes, h
         return [s for s, wr in state.items() if len(wr) == int(w.n_spans[s])]
 
     for step in range(260):
-        op = rng.choice(["register", "write", "write", "free", "plan", "gather"])
+        op = rng.choice(["register", "write", "write", "free", "plan", "gather", "grids", "padded", "grad"])
         n_calls[op] += 1
         sloppy = rng.random() < 0.2     # one call in five is built without looking at the model
         if op == "register":
@@ -115,12 +115,70 @@ def test_random_call_sequences_agree_with_oracle(seed, ring_order, page_bytes, h
                 assert ga["n_mb"] == oa["n_mb"]
                 for key in PLAN_KEYS:
                     assert np.array_equal(ga[key], oa[key]), (step, key)
-                plans.append((gp, op_, len(slots)))
+                plans.append((gp, op_, len(slots), cfg["budget_L"]))
                 plans[:] = plans[-4:]
+        elif op == "grids":
+            if sloppy or not state:
+                k = int(rng.integers(1, 4))
+                slots = rng.integers(0, w.n_samples + 1, size=k)
+                spans = rng.integers(0, 5, size=k)
+                grids = rng.integers(0, 40, size=(k, 3))
+            else:
+                slots = rng.choice(list(state.keys()), size=int(rng.integers(1, 4)))
+                spans = [int(rng.integers(0, int(w.n_spans[s_]))) for s_ in slots]
+                grids = []
+                for s_, j_ in zip(slots, spans):
+                    n_tok = int(w.spans_of(int(s_))[1][j_])
+                    d = [x for x in range(1, 65) if n_tok % x == 0]
+                    wdt = int(rng.choice(d))
+                    t_ = int(rng.choice([x for x in (1, 2, 3) if (n_tok // wdt) % x == 0]))
+                    grids.append([t_, n_tok // wdt // t_, wdt])
+            g, o = pool.set_span_grids(slots, spans, grids, cuda_stream()), opool.set_span_grids(slots, spans, grids)
+        elif op in ("padded", "grad"):
+            if not plans:
+                n_calls[op] -= 1
+                continue
+            gp, op_, n, budget = plans[int(rng.integers(0, len(plans)))]
+            n_mb, total, _ = op_.summary()
+            lo = int(rng.integers(0, n_mb + 1))
+            hi = int(rng.integers(0, n_mb + 2))
+            padded_layout = op == "padded" or bool(rng.random() < 0.5)
+            rows = max(1, (max(hi - lo, 0) * budget) if padded_layout else int(total))
+            if rows * w.hidden > (96 << 20):   # keep the buffers of one call below a few hundred MB
+                n_calls[op] -= 1
+                continue
+            if op == "padded":
+                out = torch.full((rows, w.hidden), -1, dtype=torch.int16, device="cuda")
+                cu = torch.full((n + 2 * n_mb + 2,), -7, dtype=torch.int32, device="cuda")
+                pos3 = torch.full((3, rows), -7, dtype=torch.int32, device="cuda")
+                ids_, lab = (torch.full((rows,), -7, dtype=torch.int32, device="cuda") for _ in range(2))
+                msk = torch.full((rows,), 7, dtype=torch.uint8, device="cuda")
+                g = pool.gather_padded(gp, lo, hi, table.data_ptr(), w.vocab, -1, out.data_ptr(), cu.data_ptr(), pos3.data_ptr(),
+                                       ids_.data_ptr(), lab.data_ptr(), msk.data_ptr(), cuda_stream())
+                eo = dict(out=np.full((rows, w.hidden), 0xFFFF, np.uint16), cu=np.full(n + 2 * n_mb + 2, -7, np.int32),
+                          pos3=np.full((3, rows), -7, np.int32), ids=np.full(rows, -7, np.int32), labels=np.full(rows, -7, np.int32),
+                          mask=np.full(rows, 7, np.uint8))
+                o = opool.gather_padded(op_, lo, hi, table_h, -1, eo["out"], eo["cu"], eo["pos3"], eo["ids"], eo["labels"], eo["mask"])
+                if g == 0 and o == 0:
+                    torch.cuda.synchronize()
+                    if hi > lo:   # an empty range writes nothing; the layouts of the poison differ ([3, rows] with rows = 1)
+                        got = dict(out=out.cpu().numpy().view(np.uint16), cu=cu.cpu().numpy(), pos3=pos3.cpu().numpy(),
+                                   ids=ids_.cpu().numpy(), labels=lab.cpu().numpy(), mask=msk.cpu().numpy())
+                        for key in got:
+                            assert np.array_equal(got[key], eo[key]), (step, key)
+            else:
+                grad = workloads.grad_values(w, 0, rows, device="cuda")
+                gt = torch.zeros((w.vocab, w.hidden), dtype=torch.float32, device="cuda")
+                g = pool.embed_grad(gp, lo, hi, padded_layout, grad.data_ptr(), gt.data_ptr(), w.vocab, cuda_stream())
+                et = np.zeros((w.vocab, w.hidden), np.float32)
+                o = opool.embed_grad(op_, lo, hi, padded_layout, bits16(grad), et)
+                if g == 0 and o == 0:
+                    torch.cuda.synchronize()
+                    assert np.array_equal(gt.cpu().numpy().view(np.uint32), et.view(np.uint32)), step
         else:
             if not plans:
                 continue
-            gp, op_, n = plans[int(rng.integers(0, len(plans)))]
+            gp, op_, n, _budget = plans[int(rng.integers(0, len(plans)))]
             n_mb, total, _ = op_.summary()
             lo = int(rng.integers(0, n_mb + 1))
             hi = int(rng.integers(0, n_mb + 2))
