@@ -133,6 +133,65 @@ def oracle_setup(name, n_samples, all_hbm):
     return w, step
 
 
+def time_oracle_gather_threads(name, n_samples, all_hbm, reps=2):
+    """The oracle's assembly alone, as it stands, once on one core and once with the microbatches split over all
+    cores this process may use (one thread per contiguous range of microbatches; ctypes releases the GIL)."""
+    import concurrent.futures
+    import torch
+    import workloads
+    from harness import bits16, bits32, pool_config_fields, plan_config_fields, register_args, write_args
+    from oracle import OraclePool, PlanConfig, PoolConfig
+    w = workloads.make_workload(name, n_samples=n_samples, all_hbm=all_hbm)
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    conv = bits16 if w.src_dtype == 0 else bits32
+    table = bits16(workloads.embed_table(w, device=dev))
+    pool = OraclePool(PoolConfig(**pool_config_fields(w)))
+    assert pool.rc == 0
+    for call in w.write_calls:
+        samples = sorted({s for s, _ in call}, key=[s for s, _ in call].index)
+        assert pool.register_samples(*register_args(w, samples)) == 0
+        srcs = [conv(workloads.span_values(w, s, j, device=dev)) for s, j in call]
+        assert pool.write_embeddings(*write_args(w, call), srcs, w.src_dtype) == 0
+    rc, plan = pool.plan_microbatches(np.asarray(w.plan_order, dtype=np.uint32), PlanConfig(**plan_config_fields(w)))
+    assert rc == 0
+    a = plan.arrays()
+    n_mb = int(a["n_mb"])
+    cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1)
+    tok = np.concatenate([[0], np.cumsum(a["mb_tokens"].astype(np.int64))])
+
+    def ranges(parts):
+        cuts = sorted({int(np.searchsorted(tok, tok[-1] * k / parts)) for k in range(parts + 1)} | {0, n_mb})
+        return [(b, e) for b, e in zip(cuts[:-1], cuts[1:]) if e > b]
+
+    def run(parts):
+        bufs = []
+        for b, e in ranges(parts):
+            rows = int(tok[e] - tok[b])
+            n_s = int(a["mb_sample_off"][e] - a["mb_sample_off"][b])
+            bufs.append((b, e, np.empty((rows, w.hidden), np.uint16), np.empty(n_s + (e - b), np.int32), np.empty(rows, np.int32)))
+        best = None
+        for _ in range(reps):
+            t0 = time.perf_counter()
+            if len(bufs) == 1:
+                b, e, o, c, p_ = bufs[0]
+                assert pool.gather_packed(plan, b, e, table, o, c, p_) == 0
+            else:
+                with concurrent.futures.ThreadPoolExecutor(len(bufs)) as ex:
+                    rcs = list(ex.map(lambda t: pool.gather_packed(plan, t[0], t[1], table, t[2], t[3], t[4]), bufs))
+                assert all(r == 0 for r in rcs)
+            dt = time.perf_counter() - t0
+            best = dt if best is None else min(best, dt)
+        return best, len(bufs)
+
+    gb = w.total_tokens * 4 * w.hidden
+    t1, _ = run(1)
+    tn, used = run(min(cores, n_mb))
+    plan.destroy()
+    pool.destroy()
+    return {"gather_1_core_gbs": gb / t1 / 1e9, "gather_all_cores_gbs": gb / tn / 1e9, "gather_threads": used,
+            "cores_available": cores}
+
+
 def time_oracle(name, n_samples, all_hbm, steps, warmup):
     w, step = oracle_setup(name, n_samples, all_hbm)
     for _ in range(warmup):
@@ -662,6 +721,7 @@ def run_ours(args):
             n = min(CPU_SAMPLE, w.n_samples)
             r = time_oracle(args.workload, n, args.all_hbm, 4, 1)   # about 15 s of CPU work on this workload
             line["cpu_baseline"] = {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")}
+            line["cpu_baseline"]["assembly_only"] = time_oracle_gather_threads(args.workload, n, args.all_hbm)
         print(json.dumps(line))
     if dist:
         dist.barrier()
