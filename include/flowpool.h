@@ -318,7 +318,7 @@ int32_t pool_take_ready(ft_pool* pool, uint64_t min_tokens, uint32_t max_samples
  *                     three base addresses at which this device reaches the peer's HBM slab, host slab and text
  *                     frames.  INVALID_ARG: malformed blob, another GVA space, own rank, missing or misaligned
  *                     base; SLOT_IN_USE: that rank was imported before.  Init-time: allocates, synchronises.
- * pool_export_samples descriptors of READY samples (lengths, spans, page GVAs, text-page GVAs) into a host buffer
+ * pool_export_samples descriptors of READY samples (lengths, spans with their token grids, page GVAs, text-page GVAs) into a host buffer
  *                     -- the "lightweight metadata" a consumer needs; no embedding bytes.  Synchronises `stream`.
  *                     UNKNOWN_SAMPLE / NOT_READY / INVALID_ARG (repeated slot) per sample in order; buf = NULL
  *                     queries the size.

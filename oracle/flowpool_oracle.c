@@ -944,7 +944,7 @@ int32_t oracle_pool_export_samples(oracle_pool* p, const uint32_t* slot, uint32_
       if (slot[j] == slot[i]) return OR_ERR_INVALID_ARG;
     if (s->state != SLOT_READY) return OR_ERR_NOT_READY;
     words += 3 + s->n_text_pages;
-    for (uint32_t j = 0; j < s->n_spans; ++j) words += 3 + s->spans[j].n_pages;
+    for (uint32_t j = 0; j < s->n_spans; ++j) words += 6 + s->spans[j].n_pages; /* pos, tokens, pages, grid T H W */
   }
   if (bytes) *bytes = 8 * words;
   if (!buf) return OR_OK;
@@ -956,6 +956,7 @@ int32_t oracle_pool_export_samples(oracle_pool* p, const uint32_t* slot, uint32_
     *w++ = s->seq_len; *w++ = s->n_spans; *w++ = s->n_text_pages;
     for (uint32_t j = 0; j < s->n_spans; ++j) {
       *w++ = s->spans[j].pos_start; *w++ = s->spans[j].n_tokens; *w++ = s->spans[j].n_pages;
+      *w++ = s->spans[j].grid[0]; *w++ = s->spans[j].grid[1]; *w++ = s->spans[j].grid[2];
       for (uint32_t o = 0; o < s->spans[j].n_pages; ++o) *w++ = s->spans[j].pages[o];
     }
     for (uint32_t k = 0; k < s->n_text_pages; ++k) *w++ = s->text_pages[k];
@@ -985,10 +986,15 @@ int32_t oracle_pool_import_samples(oracle_pool* p, const uint32_t* local_slot, u
     if (seq_len == 0 || ntp != (seq_len + TEXT_PAGE_IDS - 1) / TEXT_PAGE_IDS) return OR_ERR_INVALID_ARG;
     if (seq_len > p->c.max_seq_len || n_spans > p->c.max_spans_per_sample) return OR_ERR_CAPACITY;
     for (uint64_t j = 0; j < n_spans; ++j) {
-      if (r + 3 > end) return OR_ERR_INVALID_ARG;
+      if (r + 6 > end) return OR_ERR_INVALID_ARG;
       uint64_t np = r[2];
       if (np > (uint64_t)((p->c.max_pages_per_span + 63) / 64) * 64) return OR_ERR_CAPACITY;
-      r += 3 + np;
+      /* the span's token grid travels with it: none (all zero), or extents whose product is the token count */
+      if (r[3] | r[4] | r[5]) {
+        if (!r[3] || !r[4] || !r[5] || r[3] > r[1] || r[4] > r[1] || r[5] > r[1]) return OR_ERR_INVALID_ARG;
+        if (r[3] * r[4] > r[1] || r[3] * r[4] * r[5] != r[1]) return OR_ERR_INVALID_ARG;
+      }
+      r += 6 + np;
     }
     r += ntp;
     if (r > end) return OR_ERR_INVALID_ARG;
@@ -1005,7 +1011,8 @@ int32_t oracle_pool_import_samples(oracle_pool* p, const uint32_t* local_slot, u
     s->spans = (or_span*)calloc(s->n_spans + 1, sizeof(or_span));
     for (uint32_t j = 0; j < s->n_spans; ++j) {
       s->spans[j].pos_start = (uint32_t)r[0]; s->spans[j].n_tokens = (uint32_t)r[1]; s->spans[j].n_pages = (uint32_t)r[2];
-      r += 3;
+      s->spans[j].grid[0] = (uint32_t)r[3]; s->spans[j].grid[1] = (uint32_t)r[4]; s->spans[j].grid[2] = (uint32_t)r[5];
+      r += 6;
       s->spans[j].pages = (uint64_t*)malloc(8 * (s->spans[j].n_pages + 1));
       for (uint32_t o = 0; o < s->spans[j].n_pages; ++o) s->spans[j].pages[o] = *r++;
     }

@@ -16,6 +16,7 @@
 //                    one list (row, id) for the rest
 //   k_embed_grad_hot one CTA per (frequent id, 256-column slice): streams the listed rows, adds in list order
 #include <algorithm>
+#include <cstring>
 #include <unordered_set>
 #include <vector>
 
@@ -593,6 +594,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_set_span_grids(ft
   c.span_id = reinterpret_cast<const uint32_t*>(static_cast<uint8_t*>(d) + o_sid);
   k_set_grids<<<(n + 255) / 256, 256, 0, st>>>(p->view, c);
   FT_CUDA(cudaGetLastError());
+  for (uint32_t k = 0; k < n; ++k) memcpy(p->spans[hs[k]].grid, &hg[k], 12);  // host mirror (exported with the sample)
   p->gpu_launches += 1;
   return end_producer(p, st);
 }

@@ -220,6 +220,7 @@ struct ft_slot_mirror {
 };
 struct ft_span_mirror {
   uint32_t pos = 0, tokens = 0, npages = 0;
+  uint32_t grid[3] = {0, 0, 0};  // token grid (T, H, W) as last set; all zero = none
   bool written = false;
 };
 

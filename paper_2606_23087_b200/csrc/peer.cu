@@ -69,6 +69,7 @@ struct ImportCall {
   const uint32_t *page_off, *blk_off, *tp_off;               // prefix sums made on the host
   const uint64_t* gva;                                       // page GVAs then text-page GVAs
   uint32_t* head;                                            // [1] block ring head before the pops
+  const uint4* span_grid;                                    // per span: token grid (T, H, W, 0), zero = none
 };
 
 __global__ void k_import_pop(PoolView v, ImportCall c, uint32_t total_blocks) {
@@ -89,7 +90,7 @@ __global__ void __launch_bounds__(256) k_import_fill(PoolView v, ImportCall c, u
     for (uint32_t j = 0; j < c.n_spans_of[t]; ++j) {
       const uint32_t sid = slot * v.spans_per_sample + j, g = c.span_begin[t] + j;
       v.sp_pos[sid] = c.span_pos[g]; v.sp_tokens[sid] = c.span_tok[g]; v.sp_npages[sid] = c.span_npages[g];
-      v.sp_grid[sid] = make_uint4(0, 0, 0, 0);
+      v.sp_grid[sid] = c.span_grid[g];
     }
   }
   if (t < total_pages) {
@@ -208,7 +209,7 @@ FT_API int32_t pool_export_samples(ft_pool* p, const uint32_t* slot, uint32_t n,
     total_spans += s.n_spans;
     total_text += s.n_text_pages;
   }
-  const uint64_t need = sizeof(SampleHeader) + 12ull * n + 12ull * total_spans + 8ull * (total_pages + total_text);
+  const uint64_t need = sizeof(SampleHeader) + 12ull * n + 24ull * total_spans + 8ull * (total_pages + total_text);
   if (bytes) *bytes = need;
   if (!buf) return FT_OK;  // size query
   if (cap < need) return FT_ERR_CAPACITY;
@@ -220,7 +221,7 @@ FT_API int32_t pool_export_samples(ft_pool* p, const uint32_t* slot, uint32_t n,
   memcpy(out, &h, sizeof(h));
   uint32_t* ps = reinterpret_cast<uint32_t*>(out + sizeof(h));
   uint32_t* pp = ps + 3ull * n;
-  uint64_t* pg = reinterpret_cast<uint64_t*>(pp + 3ull * total_spans);
+  uint64_t* pg = reinterpret_cast<uint64_t*>(pp + 6ull * total_spans);
   // descriptors for the list kernel
   std::vector<uint32_t> span_id, page_off(1, 0), tp_off(1, 0);
   for (uint32_t i = 0; i < n; ++i) {
@@ -229,6 +230,7 @@ FT_API int32_t pool_export_samples(ft_pool* p, const uint32_t* slot, uint32_t n,
     for (uint32_t j = 0; j < s.n_spans; ++j) {
       const ft_span_mirror& m = p->spans[(uint64_t)slot[i] * S + j];
       *pp++ = m.pos; *pp++ = m.tokens; *pp++ = m.npages;
+      *pp++ = m.grid[0]; *pp++ = m.grid[1]; *pp++ = m.grid[2];  // the span's token grid travels with it
       span_id.push_back(slot[i] * S + j);
       page_off.push_back(page_off.back() + m.npages);
     }
@@ -269,14 +271,14 @@ FT_API int32_t pool_import_samples(ft_pool* p, const uint32_t* local_slot, uint3
   SampleHeader h;
   memcpy(&h, buf, sizeof(h));
   if (h.magic != kSampleMagic || h.n != n) return FT_ERR_INVALID_ARG;
-  if (bytes != sizeof(SampleHeader) + 12ull * n + 12ull * h.total_spans + 8ull * (h.total_pages + h.total_text_pages)) return FT_ERR_INVALID_ARG;
+  if (bytes != sizeof(SampleHeader) + 12ull * n + 24ull * h.total_spans + 8ull * (h.total_pages + h.total_text_pages)) return FT_ERR_INVALID_ARG;
   const ft_pool_config& c = p->cfg;
   if (h.src_rank >= c.world_size || !p->peer_imported[h.src_rank]) return FT_ERR_INVALID_ARG;  // mapping first
   if (n == 0) return FT_OK;
   const uint8_t* in = static_cast<const uint8_t*>(buf);
   const uint32_t* ps = reinterpret_cast<const uint32_t*>(in + sizeof(h));
   const uint32_t* pp = ps + 3ull * n;
-  const uint64_t* pg = reinterpret_cast<const uint64_t*>(pp + 3ull * h.total_spans);
+  const uint64_t* pg = reinterpret_cast<const uint64_t*>(pp + 6ull * h.total_spans);
   const uint32_t S = c.max_spans_per_sample, TPS = p->view.text_pages_per_sample, MB = p->view.blocks_per_span;
   std::vector<uint8_t> seen(c.max_samples, 0);
   uint64_t spans = 0, pages = 0, text = 0, blocks = 0;
@@ -289,8 +291,13 @@ FT_API int32_t pool_import_samples(ft_pool* p, const uint32_t* local_slot, uint3
     if (seq_len > c.max_seq_len || nsp > S || ntp > TPS) return FT_ERR_CAPACITY;
     if (spans + nsp > h.total_spans) return FT_ERR_INVALID_ARG;
     for (uint32_t j = 0; j < nsp; ++j) {
-      const uint32_t np = pp[3 * (spans + j) + 2];
+      const uint32_t* rec = pp + 6 * (spans + j);
+      const uint32_t np = rec[2];
       if ((np + kListBlock - 1) / kListBlock > MB) return FT_ERR_CAPACITY;
+      if (rec[3] | rec[4] | rec[5]) {  // a token grid: extents whose product is the token count
+        const uint64_t tokens = rec[1], th = (uint64_t)rec[3] * rec[4];
+        if (!rec[3] || !rec[4] || !rec[5] || th > tokens || th * rec[5] != tokens) return FT_ERR_INVALID_ARG;
+      }
       pages += np; blocks += (np + kListBlock - 1) / kListBlock;
     }
     spans += nsp; text += ntp;
@@ -302,12 +309,14 @@ FT_API int32_t pool_import_samples(ft_pool* p, const uint32_t* local_slot, uint3
   // upload: per-sample arrays, per-span arrays, prefix sums, GVAs
   const uint32_t ns = (uint32_t)spans;
   std::vector<uint32_t> seq(n), nsp(n), sbeg(n + 1, 0), pos(ns), tok(ns), npg(ns), poff(ns + 1, 0), boff(ns + 1, 0), tpoff(n + 1, 0);
+  std::vector<uint4> grid(ns);
   for (uint32_t i = 0, g = 0; i < n; ++i) {
     seq[i] = ps[3 * i]; nsp[i] = ps[3 * i + 1];
     sbeg[i + 1] = sbeg[i] + nsp[i];
     tpoff[i + 1] = tpoff[i] + ps[3 * i + 2];
     for (uint32_t j = 0; j < nsp[i]; ++j, ++g) {
-      pos[g] = pp[3 * g]; tok[g] = pp[3 * g + 1]; npg[g] = pp[3 * g + 2];
+      pos[g] = pp[6 * g]; tok[g] = pp[6 * g + 1]; npg[g] = pp[6 * g + 2];
+      grid[g] = make_uint4(pp[6 * g + 3], pp[6 * g + 4], pp[6 * g + 5], 0);
       poff[g + 1] = poff[g] + npg[g];
       boff[g + 1] = boff[g] + (npg[g] + kListBlock - 1) / kListBlock;
     }
@@ -318,6 +327,7 @@ FT_API int32_t pool_import_samples(ft_pool* p, const uint32_t* local_slot, uint3
   const size_t o_slot = take(4ull * n), o_seq = take(4ull * n), o_nsp = take(4ull * n), o_sbeg = take(4ull * (n + 1));
   const size_t o_pos = take(4ull * ns), o_tok = take(4ull * ns), o_npg = take(4ull * ns);
   const size_t o_poff = take(4ull * (ns + 1)), o_boff = take(4ull * (ns + 1)), o_tpoff = take(4ull * (n + 1));
+  const size_t o_grid = take(16ull * ns);
   const size_t blob_bytes = align_up_sz(off, 256), o_head = blob_bytes, total_bytes = o_head + 16;
   std::vector<uint8_t> blob(blob_bytes, 0);
   memcpy(blob.data() + o_gva, pg, 8 * (pages + text));
@@ -325,6 +335,7 @@ FT_API int32_t pool_import_samples(ft_pool* p, const uint32_t* local_slot, uint3
   memcpy(blob.data() + o_seq, seq.data(), 4ull * n);
   memcpy(blob.data() + o_nsp, nsp.data(), 4ull * n);
   memcpy(blob.data() + o_sbeg, sbeg.data(), 4ull * (n + 1));
+  if (ns) memcpy(blob.data() + o_grid, grid.data(), 16ull * ns);
   if (ns) { memcpy(blob.data() + o_pos, pos.data(), 4ull * ns); memcpy(blob.data() + o_tok, tok.data(), 4ull * ns); memcpy(blob.data() + o_npg, npg.data(), 4ull * ns); }
   memcpy(blob.data() + o_poff, poff.data(), 4ull * (ns + 1));
   memcpy(blob.data() + o_boff, boff.data(), 4ull * (ns + 1));
@@ -336,7 +347,7 @@ FT_API int32_t pool_import_samples(ft_pool* p, const uint32_t* local_slot, uint3
   uint8_t* db = static_cast<uint8_t*>(d);
   auto U = [&](size_t o) { return reinterpret_cast<uint32_t*>(db + o); };
   ImportCall ic{ns, n, U(o_slot), U(o_seq), U(o_nsp), U(o_sbeg), U(o_pos), U(o_tok), U(o_npg), U(o_poff), U(o_boff), U(o_tpoff),
-                reinterpret_cast<uint64_t*>(db + o_gva), U(o_head)};
+                reinterpret_cast<uint64_t*>(db + o_gva), U(o_head), reinterpret_cast<const uint4*>(db + o_grid)};
   k_import_pop<<<1, 1, 0, st>>>(p->view, ic, (uint32_t)blocks);
   const uint64_t items = std::max<uint64_t>(pages + text, n);
   k_import_fill<<<(unsigned)((items + 255) / 256), 256, 0, st>>>(p->view, ic, (uint32_t)pages, (uint32_t)text);
@@ -351,6 +362,7 @@ FT_API int32_t pool_import_samples(ft_pool* p, const uint32_t* local_slot, uint3
     for (uint32_t j = 0; j < nsp[i]; ++j, ++g) {
       ft_span_mirror& m = p->spans[(uint64_t)local_slot[i] * S + j];
       m.pos = pos[g]; m.tokens = tok[g]; m.npages = npg[g]; m.written = true;
+      m.grid[0] = grid[g].x; m.grid[1] = grid[g].y; m.grid[2] = grid[g].z;
     }
     p->live_samples++; p->live_spans += nsp[i];
   }

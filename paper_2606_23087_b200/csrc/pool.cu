@@ -835,6 +835,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_register_samples(
     for (uint32_t j = 0; j < n_spans[i]; ++j, ++sp) {
       ft_span_mirror& m = p->spans[(uint64_t)slot[i] * c.max_spans_per_sample + j];
       m.pos = span_pos[sp]; m.tokens = span_tokens[sp]; m.npages = 0; m.written = false;
+      m.grid[0] = m.grid[1] = m.grid[2] = 0;
     }
     p->live_samples++; p->live_spans += n_spans[i];
   }

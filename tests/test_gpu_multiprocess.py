@@ -47,6 +47,10 @@ def test_consumer_reads_producer_pages_in_place(name, kw):
         assert g[rank].write_embeddings(*write_args(w, call), [t.data_ptr() for t in srcs], w.src_dtype, cuda_stream()) == 0
         host = [bits16(t) if w.src_dtype == 0 else t.view(torch.int32).cpu().numpy().view(np.uint32) for t in srcs]
         assert o[rank].write_embeddings(*write_args(w, call), host, w.src_dtype) == 0
+        gi = [(s, j, workloads.span_grid(w, s, j)) for s, j in call]
+        gi = [t for t in gi if t[2] is not None]
+        ga_ = ([s for s, _, _ in gi], [j for _, j, _ in gi], [t for _, _, t in gi])
+        assert g[rank].set_span_grids(*ga_, cuda_stream()) == o[rank].set_span_grids(*ga_) == 0
 
     fill(1, remote)
     fill(0, local)
@@ -102,6 +106,43 @@ def test_consumer_reads_producer_pages_in_place(name, kw):
     got = out.cpu().numpy().view(np.uint16)
     assert np.array_equal(got, oout) and not np.any(np.all(got == 0xFFFF, axis=1))
     assert np.array_equal(cu.cpu().numpy(), ocu) and np.array_equal(pos.cpu().numpy(), opos)
+    assert g[0].status() == o[0].status() == (0, 0)
+    # backbone-side outputs over the same mixed microbatches: the imported spans' token grids came with the descriptors
+    L = w.budget_L
+    rows = n_mb * L
+    p_out = torch.full((rows, w.hidden), -1, dtype=torch.int16, device="cuda")
+    p_cu = torch.full((len(order) + 2 * n_mb,), -7, dtype=torch.int32, device="cuda")
+    p_pos3 = torch.full((3, rows), -7, dtype=torch.int32, device="cuda")
+    p_ids, p_lab = (torch.full((rows,), -7, dtype=torch.int32, device="cuda") for _ in range(2))
+    p_msk = torch.full((rows,), 7, dtype=torch.uint8, device="cuda")
+    assert g[0].gather_padded(gp, 0, n_mb, table.data_ptr(), w.vocab, -1, p_out.data_ptr(), p_cu.data_ptr(), p_pos3.data_ptr(),
+                              p_ids.data_ptr(), p_lab.data_ptr(), p_msk.data_ptr(), cuda_stream()) == 0
+    e = dict(out=np.full((rows, w.hidden), 0xFFFF, np.uint16), cu=np.full(len(order) + 2 * n_mb, -7, np.int32),
+             pos3=np.full((3, rows), -7, np.int32), ids=np.full(rows, -7, np.int32), labels=np.full(rows, -7, np.int32),
+             mask=np.full(rows, 7, np.uint8))
+    assert o[0].gather_padded(op, 0, n_mb, bits16(table), -1, e["out"], e["cu"], e["pos3"], e["ids"], e["labels"], e["mask"]) == 0
+    torch.cuda.synchronize()
+    for key, t in (("out", p_out), ("cu", p_cu), ("pos3", p_pos3), ("ids", p_ids), ("labels", p_lab), ("mask", p_msk)):
+        got_k = t.cpu().numpy()
+        assert np.array_equal(got_k.view(np.uint16) if key == "out" else got_k, e[key]), key
+    # an imported gridded span shows in the positions (the three components differ somewhere inside an imported sample)
+    row = 0
+    imported_rows = []
+    for j in range(n_mb):
+        row = j * L
+        for slot in oa["mb_samples"][oa["mb_sample_off"][j]:oa["mb_sample_off"][j + 1]]:
+            ln = int(w.seq_len[remote[loc.index(int(slot))]]) if int(slot) in loc else int(w.seq_len[int(slot)])
+            if int(slot) in loc:
+                imported_rows.append((row, row + ln))
+            row += ln
+    assert any(np.any(e["pos3"][0, a:b] != e["pos3"][2, a:b]) for a, b in imported_rows)
+    grad = workloads.grad_values(w, 0, total, device="cuda")
+    gt = torch.zeros((w.vocab, w.hidden), dtype=torch.float32, device="cuda")
+    assert g[0].embed_grad(gp, 0, n_mb, False, grad.data_ptr(), gt.data_ptr(), w.vocab, cuda_stream()) == 0
+    et = np.zeros((w.vocab, w.hidden), np.float32)
+    assert o[0].embed_grad(op, 0, n_mb, False, bits16(grad), et) == 0
+    torch.cuda.synchronize()
+    assert np.array_equal(gt.cpu().numpy().view(np.uint32), et.view(np.uint32))
     assert g[0].status() == o[0].status() == (0, 0)
     # freeing imports returns nothing to the consumer's rings, and the plan dies with them
     assert g[0].free(loc, cuda_stream()) == o[0].free(loc) == 0

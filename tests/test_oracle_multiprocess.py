@@ -21,6 +21,19 @@ def fill(pool, w, samples):
     assert pool.register_samples(*register_args(w, samples)) == 0
     call = [(s, j) for s in samples for j in range(int(w.n_spans[s]))]
     assert pool.write_embeddings(*write_args(w, call), [host_span(w, s, j) for s, j in call], w.src_dtype) == 0
+    grids = [(s, j, workloads.span_grid(w, s, j)) for s, j in call]
+    grids = [t for t in grids if t[2] is not None]
+    assert pool.set_span_grids([s for s, _, _ in grids], [j for _, j, _ in grids], [g for _, _, g in grids]) == 0
+
+
+def padded_all(pool, plan, w, table, n_slots):
+    n_mb = plan.summary()[0]
+    rows = n_mb * w.budget_L
+    o = dict(out=np.full((rows, w.hidden), 0xFFFF, np.uint16), cu=np.full(n_slots + 2 * n_mb, -7, np.int32),
+             pos3=np.full((3, rows), -7, np.int32), ids=np.full(rows, -7, np.int32), labels=np.full(rows, -7, np.int32),
+             mask=np.full(rows, 7, np.uint8))
+    assert pool.gather_padded(plan, 0, n_mb, table, -1, o["out"], o["cu"], o["pos3"], o["ids"], o["labels"], o["mask"]) == 0
+    return o
 
 
 def gather_all(pool, slots, w, table):
@@ -105,6 +118,16 @@ def test_consumer_assembles_what_the_producer_would():
     a, b = plan.arrays(), plan_ref.arrays()
     for k in ("mb_sample_off", "mb_tokens", "mb_cost", "mb_rank", "sample_mb"):
         assert np.array_equal(a[k], b[k])
+    # the spans' token grids travel with the descriptors: positions, labels and the table gradient are the single process's
+    po, pr = padded_all(cons, plan, w, table, len(order_cons)), padded_all(ref, plan_ref, w, table, len(order_ref))
+    for k in po:
+        assert np.array_equal(po[k], pr[k]), k
+    assert np.any(po["pos3"][0] != po["pos3"][2])
+    grad = bits16(workloads.grad_values(w, 0, out.shape[0]))
+    t_c, t_r = np.zeros((w.vocab, w.hidden), np.float32), np.zeros((w.vocab, w.hidden), np.float32)
+    assert cons.embed_grad(plan, 0, plan.summary()[0], False, grad, t_c) == 0
+    assert ref.embed_grad(plan_ref, 0, plan_ref.summary()[0], False, grad, t_r) == 0
+    assert np.array_equal(t_c.view(np.uint32), t_r.view(np.uint32)) and np.any(t_c != 0)
     # imported page lists are the producer's
     for loc, rem in zip([10, 11, 12, 13, 14], remote):
         for j in range(int(w.n_spans[rem])):
