@@ -876,6 +876,46 @@ int32_t oracle_pool_gather_packed(oracle_pool* p, const oracle_plan* pl, uint32_
   return OR_OK;
 }
 
+/* The microbatches named in mb_list, in list order (Algorithm 1 deals microbatches to ranks, lines 15-27: a rank
+ * consumes its own list, which is not a contiguous range).  Outputs are the concatenation of what
+ * oracle_pool_gather_packed writes for each [j, j+1).  An index may repeat. */
+int32_t oracle_pool_gather_list(oracle_pool* p, const oracle_plan* pl, const uint32_t* mb_list, uint32_t n_list,
+                                const void* embed_table, uint32_t vocab, void* out_embeds,
+                                int32_t* out_cu_seqlens, int32_t* out_position_ids) {
+  if (!p || !pl || (n_list && !mb_list)) return OR_ERR_INVALID_ARG;
+  p->call_seq++;
+  for (uint32_t i = 0; i < n_list; ++i)
+    if (mb_list[i] >= pl->n_mb) return OR_ERR_INVALID_ARG;
+  for (uint32_t t = 0; t < pl->n; ++t) {
+    or_sample* s = &p->samples[pl->slots[t]];
+    if (s->state != SLOT_READY || s->generation != pl->slot_generation[t]) return OR_ERR_NOT_READY;
+  }
+  if (n_list == 0) return OR_OK;
+  if (!embed_table || !out_embeds || !out_cu_seqlens || !out_position_ids) return OR_ERR_INVALID_ARG;
+  const uint64_t row_bytes = 2ull * p->c.hidden;
+  const uint64_t call = p->call_seq;
+  uint64_t row = 0, cu_w = 0;
+  for (uint32_t i = 0; i < n_list; ++i) {
+    const uint32_t j = mb_list[i];
+    /* one microbatch through the packed assembly; asynchronous errors keep this call's number and report the row
+     * index in the list's output */
+    const uint64_t key_before = p->status_key;
+    p->status_key = UINT64_MAX;
+    int32_t rc = oracle_pool_gather_packed(p, pl, j, j + 1, embed_table, vocab, (uint8_t*)out_embeds + row * row_bytes,
+                                           out_cu_seqlens + cu_w, out_position_ids + row);
+    p->call_seq = call;
+    if (p->status_key != UINT64_MAX) {
+      const uint64_t code = (p->status_key >> 32) & 0xFF, detail = (p->status_key & 0xFFFFFFFFull) + row;
+      p->status_key = (call << 40) | (code << 32) | detail;
+    }
+    if (key_before < p->status_key) p->status_key = key_before;
+    if (rc != OR_OK) return rc;
+    row += pl->mb_tokens[j];
+    cu_w += (uint64_t)(pl->mb_sample_off[j + 1] - pl->mb_sample_off[j]) + 1;
+  }
+  return OR_OK;
+}
+
 /* ------------------------------------------------------------------------
  * More than one process (Sec. 3.2): each process exports its memory mapping,
  * the others update their page tables; samples cross processes as descriptors

@@ -187,6 +187,12 @@ class OraclePool:
         return lib().oracle_pool_gather_packed(self.h, plan.h, C.c_uint32(mb_begin), C.c_uint32(mb_end), _p(table),
                                                C.c_uint32(table.shape[0]), _p(out), _p(cu), _p(pos))
 
+    def gather_list(self, plan, mb_list, table, out, cu, pos):
+        """The microbatches of mb_list, in list order (outputs as gather_packed, concatenated)."""
+        mb_list = _u32(mb_list)
+        return lib().oracle_pool_gather_list(self.h, plan.h, _p(mb_list), C.c_uint32(len(mb_list)), _p(table),
+                                             C.c_uint32(table.shape[0]), _p(out), _p(cu), _p(pos))
+
     def set_span_grids(self, slots, span_idx, grids):
         """grids: [n, 3] (T, H, W) per named span."""
         slots, span_idx = _u32(slots), _u32(span_idx)

@@ -230,3 +230,56 @@ def test_table_gradient_integer_case_matches_add_at():
             np.add.at(exp, ids[text], gv[row:row + len(ids)][text])
             row += len(ids)
     assert np.allclose(full, exp, rtol=1e-5, atol=1e-5)
+
+
+def test_list_assembly_is_the_concatenation_of_single_microbatch_assemblies():
+    """A rank consumes the microbatches dealt to it (Algorithm 1, lines 15-27), not a contiguous range."""
+    w = workloads.make_workload("image_mix_7b", n_samples=40, hidden=56, page_bytes=4096)
+    w.budget_L = int(w.seq_len.max())   # several microbatches
+    res = run_oracle(w, keep_pool=True)
+    pool, plan, a = res["pool"], res["plan_handle"], res["plan"]
+    n_mb, H = int(a["n_mb"]), w.hidden
+    assert n_mb >= 6
+    tok = a["mb_tokens"].astype(np.int64)
+    row_off = np.concatenate([[0], np.cumsum(tok)])
+    cu_off = np.concatenate([[0], np.cumsum(np.diff(a["mb_sample_off"].astype(np.int64)) + 1)])
+
+    def by_list(lst):
+        rows = int(tok[lst].sum()) if len(lst) else 0
+        n_cu = int(sum(cu_off[j + 1] - cu_off[j] for j in lst))
+        out = np.full((max(rows, 1), H), 0xFFFF, np.uint16)
+        cu = np.full(max(n_cu, 1), -7, np.int32)
+        pos = np.full(max(rows, 1), -7, np.int32)
+        assert pool.gather_list(plan, lst, res["table"], out, cu, pos) == 0
+        return out[:rows], cu[:n_cu], pos[:rows]
+
+    # the identity list is the full-range assembly
+    out, cu, pos = by_list(list(range(n_mb)))
+    assert np.array_equal(out, res["out"]) and np.array_equal(cu, res["cu_seqlens"]) and np.array_equal(pos, res["position_ids"])
+    # every rank's list, a reversed list and a list with a repeat: slices of the full-range assembly, in list order
+    lists = [list(a["rank_mbs"][a["rank_mb_off"][r]:a["rank_mb_off"][r + 1]]) for r in range(w.n_ranks_N)]
+    lists += [list(range(n_mb))[::-1], [2, 2, 0]]
+    assert sorted(j for l in lists[:w.n_ranks_N] for j in l) == list(range(n_mb))
+    for lst in lists:
+        lst = [int(j) for j in lst]
+        out, cu, pos = by_list(lst)
+        exp_out = np.concatenate([res["out"][row_off[j]:row_off[j + 1]] for j in lst]) if lst else np.zeros((0, H), np.uint16)
+        exp_cu = np.concatenate([res["cu_seqlens"][cu_off[j]:cu_off[j + 1]] for j in lst]) if lst else np.zeros(0, np.int32)
+        exp_pos = np.concatenate([res["position_ids"][row_off[j]:row_off[j + 1]] for j in lst]) if lst else np.zeros(0, np.int32)
+        assert np.array_equal(out, exp_out) and np.array_equal(cu, exp_cu) and np.array_equal(pos, exp_pos)
+    one = np.zeros((1, H), np.uint16); c1 = np.zeros(1, np.int32)
+    assert pool.gather_list(plan, [n_mb], res["table"], one, c1, c1) == -1      # no such microbatch
+    assert pool.gather_list(plan, [], res["table"], one, c1, c1) == 0
+    # an id outside the table: reported with the row index in the list's output
+    small = res["table"][:100]
+    lst = [3, 1]
+    rows = int(tok[lst].sum())
+    out = np.full((rows, H), 0xFFFF, np.uint16); cu = np.zeros(64, np.int32); pos = np.zeros(rows, np.int32)
+    assert pool.gather_list(plan, lst, small, out, cu, pos) == 0
+    code, detail = pool.status()
+    ids3 = np.concatenate([workloads.input_ids(w, int(s)) for s in a["mb_samples"][a["mb_sample_off"][3]:a["mb_sample_off"][4]]])
+    first_bad = int(np.nonzero((ids3 != w.placeholder_id) & (ids3 >= 100))[0][0])
+    assert (code, detail) == (-9, first_bad)
+    assert pool.free([int(a["mb_samples"][0])]) == 0
+    assert pool.gather_list(plan, [0], res["table"], out, cu, pos) == -5        # the plan died with its sample
+    plan.destroy(); pool.destroy()
