@@ -601,6 +601,26 @@ def backbone_side(job, reps=3):
 
     ms_packed = timed(packed_all)
     ms_padded = timed(padded_all)
+    # every rank's share of the zig-zag deal: one list call per rank, against one range call per microbatch
+    rank_lists = [[int(j) for j in a["rank_mbs"][a["rank_mb_off"][k]:a["rank_mb_off"][k + 1]]] for k in range(w.n_ranks_N)]
+    mb_rows = np.concatenate([[0], np.cumsum(a["mb_tokens"].astype(np.int64))])
+
+    def by_rank_lists():
+        base = 0
+        for lst in rank_lists:
+            if lst:
+                job.check(pool.gather_list(plan, lst, job.table.data_ptr(), w.vocab, job.out[base:].data_ptr(), job.cu.data_ptr(),
+                                           job.pos.data_ptr(), st), "pool_gather_list")
+            base += int(sum(mb_rows[j + 1] - mb_rows[j] for j in lst))
+
+    def by_microbatch():
+        for j in range(n_mb):
+            job.check(pool.gather_packed(plan, j, j + 1, job.table.data_ptr(), w.vocab, job.out[int(mb_rows[j]):].data_ptr(),
+                                         job.cu.data_ptr(), job.pos.data_ptr(), st), "pool_gather_packed")
+
+    ms_rank_lists = timed(by_rank_lists)
+    ms_per_mb = timed(by_microbatch)
+    gather_bytes = w.total_tokens * 4 * H
     pad_rows = n_mb * L - w.total_tokens
     padded_bytes = w.total_tokens * 4 * H + pad_rows * 2 * H + n_mb * L * 21   # rows read+written, zero rows, 21 index bytes per row
     # table gradient: the assembled rows stand in for the gradient (bf16 values of unit scale), packed layout
@@ -624,6 +644,9 @@ def backbone_side(job, reps=3):
     torch.cuda.synchronize()
     return {
         "gather_packed_ms": ms_packed,
+        "gather_rank_lists": {"ms": ms_rank_lists, "calls": len(rank_lists), "gbs": gather_bytes / ms_rank_lists / 1e6,
+                              "per_microbatch_range_calls_ms": ms_per_mb, "per_microbatch_calls": n_mb,
+                              "per_microbatch_gbs": gather_bytes / ms_per_mb / 1e6},
         "gather_padded": {"ms": ms_padded, "calls": -(-n_mb // per_call), "padding_rows": int(pad_rows), "algorithmic_bytes": int(padded_bytes),
                           "gbs": padded_bytes / ms_padded / 1e6, "frac_of_measured_peak": padded_bytes / ms_padded / 1e6 / peak,
                           "outputs": "embeds, cu_seqlens, 3-component positions, ids, labels, loss mask"},

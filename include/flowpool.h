@@ -278,6 +278,19 @@ int32_t pool_gather_packed(ft_pool* pool, const ft_plan* plan, uint32_t mb_begin
                            int32_t* out_cu_seqlens, int32_t* out_position_ids, void* stream);
 
 /*
+ * pool_gather_list -- pool_gather_packed for a list of microbatches instead of a range (Algorithm 1 deals
+ * microbatches to ranks, lines 15-27: a rank's share, `rank_mbs` of plan_arrays, is not contiguous).  Outputs are
+ * the concatenation, in list order, of what pool_gather_packed writes for each [j, j+1): rows, n_j + 1
+ * cu_seqlens entries per listed microbatch, position ids.  One launch per tier for the whole list.
+ *   mb_list host [n_list]; an index may repeat.
+ * Errors: index >= n_mb INVALID_ARG; otherwise as pool_gather_packed (asynchronous errors: detail = row index in
+ * this call's output).  Asynchronous.
+ */
+int32_t pool_gather_list(ft_pool* pool, const ft_plan* plan, const uint32_t* mb_list, uint32_t n_list,
+                         const void* embed_table, uint32_t vocab, void* out_embeds, int32_t* out_cu_seqlens,
+                         int32_t* out_position_ids, void* stream);
+
+/*
  * pool_free -- release samples: their pages go back to the free-ring tail
  * (samples in argument order, spans by index, pages by ordinal), their text
  * pages and slots are recycled.  Plans holding a freed sample become invalid.

@@ -25,7 +25,7 @@ STATUS = {
 EXPORTS = (
     "pool_create", "pool_register_samples", "pool_write_embeddings", "pool_write_embeddings_noalloc",
     "pool_plan_microbatches", "plan_summary",
-    "plan_arrays", "plan_destroy", "pool_gather_packed", "pool_set_span_grids", "pool_gather_padded", "pool_embed_grad", "pool_free", "pool_status", "pool_stats",
+    "plan_arrays", "plan_destroy", "pool_gather_packed", "pool_gather_list", "pool_set_span_grids", "pool_gather_padded", "pool_embed_grad", "pool_free", "pool_status", "pool_stats",
     "pool_ready_count", "pool_take_ready", "pool_backing", "pool_export_mapping", "pool_import_mapping", "pool_export_samples", "pool_import_samples",
     "pool_profile_enable", "pool_profile_read", "pool_debug_span_pages", "pool_debug_ring", "pool_debug_translate", "pool_destroy", "flowpool_last_cuda_error",
 )
@@ -92,6 +92,7 @@ def lib():
             "plan_arrays": [P] * 13,
             "plan_destroy": [P],
             "pool_gather_packed": [P, P, u32, u32, P, u32, P, P, P, P],
+            "pool_gather_list": [P, P, P, u32, P, u32, P, P, P, P],
             "pool_set_span_grids": [P, u32, P, P, P, P],
             "pool_gather_padded": [P, P, u32, u32, P, u32, i32, P, P, P, P, P, P, P],
             "pool_embed_grad": [P, P, u32, u32, u32, P, P, u32, P],
@@ -208,6 +209,12 @@ class Pool:
                       pos_ptr: int, stream: int = 0):
         return lib().pool_gather_packed(self.h, plan.h, mb_begin, mb_end, table_ptr or None, vocab, out_ptr or None,
                                         cu_ptr or None, pos_ptr or None, stream or None)
+
+    def gather_list(self, plan: Plan, mb_list, table_ptr: int, vocab: int, out_ptr: int, cu_ptr: int, pos_ptr: int,
+                    stream: int = 0):
+        mb_list = _u32(mb_list)
+        return lib().pool_gather_list(self.h, plan.h, _p(mb_list), len(mb_list), table_ptr or None, vocab, out_ptr or None,
+                                      cu_ptr or None, pos_ptr or None, stream or None)
 
     def set_span_grids(self, slots, span_idx, grids, stream: int = 0):
         slots, span_idx = _u32(slots), _u32(span_idx)

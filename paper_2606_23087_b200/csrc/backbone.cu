@@ -621,7 +621,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_gather_padded(ft_
     if (rc0 != FT_OK) return rc0;
   }
   {
-    const int32_t rc1 = gather_launch(p, pl, mb_begin, mb_end, embed_table, vocab, out_embeds, nullptr, nullptr, lay.L, st);
+    const int32_t rc1 = gather_launch(p, pl, mb_begin, mb_end, embed_table, vocab, out_embeds, nullptr, nullptr, lay.L, st, nullptr, 0, 0, 0);
     if (rc1 != FT_OK) return rc1;
   }
   const PlanView pv = make_plan_view(pl);

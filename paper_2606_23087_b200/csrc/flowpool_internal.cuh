@@ -295,8 +295,10 @@ namespace ft {
 // with the pool's device current
 int32_t gather_device_setup(ft_pool* p);
 int32_t plan_device_setup(ft_pool* p);
+// (d_list: device array of the list layout's entries, or nullptr for the range [mb_begin, mb_end))
 int32_t gather_launch(ft_pool* p, const ft_plan* pl, uint32_t mb_begin, uint32_t mb_end, const void* embed_table,
-                      uint32_t vocab, void* out_embeds, int32_t* out_cu, int32_t* out_pos, uint32_t pad_L, cudaStream_t st);
+                      uint32_t vocab, void* out_embeds, int32_t* out_cu, int32_t* out_pos, uint32_t pad_L, cudaStream_t st,
+                      const void* d_list, uint32_t n_list, uint64_t list_tiles, uint64_t list_rows);
 __global__ void k_page_table_init(uint64_t* pte, const uint32_t* bind, uint64_t n, uint64_t base, uint64_t frame_bytes,
                                   uint64_t flags);
 // uploads `bytes` from `src` (pageable) to the front of the pool's device scratch, asynchronously,

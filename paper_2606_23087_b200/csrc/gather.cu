@@ -8,6 +8,8 @@
 // kernel is launched twice, once per tier, so host-link reads never stall HBM reads.
 #include <algorithm>
 #include <cstdlib>
+#include <type_traits>
+#include <vector>
 
 #include "bulk_copy.cuh"
 #include "flowpool_internal.cuh"
@@ -25,7 +27,16 @@ struct RowDesc {
   uint32_t off0;          // byte offset of the row inside its first page (0 for a text row)
   uint32_t shift;         // log2(page bytes); 31 for a text row (one segment)
   uint32_t nseg;          // 0 = nothing to copy
-  uint32_t dst_shift;     // rows to add to the packed output row (padded layout), else 0
+  uint32_t out_row;       // output row of this row (range, padded or list layout)
+};
+
+// One listed microbatch (list layout): its plan rows, where its tiles start in the claim order, where its output starts.
+struct ListEntry {
+  uint64_t row_lo, row_hi;  // plan-global rows
+  uint64_t tile0;           // claim index of its first tile
+  uint64_t out_row0;        // first output row
+  uint32_t q_lo, q_hi;      // plan positions of its samples
+  uint32_t cu0, pad;        // first cu_seqlens entry
 };
 
 struct GatherArgs {
@@ -40,9 +51,12 @@ struct GatherArgs {
   uint32_t write_index;  // this launch writes cu_seqlens / position ids
   uint32_t pad_L;        // 0: packed rows; else every microbatch starts at a multiple of pad_L rows (padded layout)
   unsigned long long* tile_counter;  // device, zero at launch
+  const ListEntry* list;             // list layout: the microbatches to assemble, in output order (else nullptr)
+  uint32_t n_list;
+  uint64_t list_tiles;               // tiles over all entries
 };
 
-template <int MODE, int U>
+template <int MODE, int U, bool LIST>
 __global__ void __launch_bounds__(kGatherThreads) k_gather(PoolView v, PlanView pl, GatherArgs a) {
   __shared__ RowDesc desc[kTileRows];
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -50,35 +64,57 @@ __global__ void __launch_bounds__(kGatherThreads) k_gather(PoolView v, PlanView 
   const uint32_t row_vecs = v.row_bytes >> 4;
 
   __shared__ uint64_t next_tile;
+  __shared__ uint32_t cur_entry;
   for (;;) {
     // tiles are claimed in order from a device counter (zeroed by the host before the launch): the CTAs in
     // flight always cover one compact window of the output, and uneven tiles balance themselves
-    if (threadIdx.x == 0) next_tile = tile_lo + atomicAdd(a.tile_counter, 1ull);
+    if (threadIdx.x == 0) {
+      const uint64_t c = atomicAdd(a.tile_counter, 1ull);
+      if (LIST) {
+        // list layout: the entry holding claim c (last entry whose first tile is <= c), then its plan tile
+        uint32_t lo = 0, hi = a.n_list;
+        while (hi - lo > 1) {
+          const uint32_t mid = (lo + hi) >> 1;
+          if (a.list[mid].tile0 <= c) lo = mid; else hi = mid;
+        }
+        cur_entry = lo;
+        next_tile = c < a.list_tiles ? a.list[lo].row_lo / kTileRows + (c - a.list[lo].tile0) : ~0ull;
+      } else {
+        next_tile = tile_lo + c;
+      }
+    }
     __syncthreads();
     const uint64_t tile = next_tile;
-    if (tile >= tile_hi) break;
+    if (LIST ? tile == ~0ull : tile >= tile_hi) break;
     if (warp == 0) {
       const uint64_t row = tile * kTileRows + lane;
       RowDesc d;
-      d.nseg = 0; d.off0 = 0; d.shift = 31; d.dst_shift = 0;
-      if (row >= a.row_lo && row < a.row_hi) {
+      d.nseg = 0; d.off0 = 0; d.shift = 31; d.out_row = 0;
+      // the rows this tile may touch: the call's range, or the listed microbatch it belongs to
+      uint64_t row_lo = a.row_lo, row_hi = a.row_hi, out0 = 0, cu0 = 0;
+      uint32_t q_lo = a.q_lo;
+      if (LIST) {
+        const ListEntry en = a.list[cur_entry];
+        row_lo = en.row_lo; row_hi = en.row_hi; out0 = en.out_row0; cu0 = en.cu0; q_lo = en.q_lo;
+      }
+      if (row >= row_lo && row < row_hi) {
         // plan position of the sample holding this row: the tile's first sample, then a short walk
         uint32_t q = pl.tile_first_sample[tile];
-        if (q < a.q_lo) q = a.q_lo;
+        if (q < q_lo) q = q_lo;
         while (row >= pl.sample_row_off[q + 1]) ++q;
         const uint32_t p = (uint32_t)(row - pl.sample_row_off[q]);
         const uint32_t slot = pl.mb_samples[q];
-        uint64_t out_row = row - a.row_lo;
-        if (a.pad_L) {  // padded layout: microbatch j of the range starts at row (j - mb_begin) * L
+        uint64_t out_row = out0 + (row - row_lo);
+        if (!LIST && a.pad_L) {  // padded layout: microbatch j of the range starts at row (j - mb_begin) * L
           const uint32_t j = pl.plan_sample_mb[q];
-          d.dst_shift = (uint32_t)((uint64_t)(j - a.mb_begin) * a.pad_L - (pl.mb_row_off[j] - a.row_lo));
-          out_row += d.dst_shift;
+          out_row += (uint64_t)(j - a.mb_begin) * a.pad_L - (pl.mb_row_off[j] - a.row_lo);
         }
+        d.out_row = (uint32_t)out_row;
         if (a.write_index) {
           a.pos_ids[out_row] = (int32_t)p;
           if (p == 0) {  // cu_seqlens: every sample writes its start; the last of a microbatch also the end
             const uint32_t j = pl.plan_sample_mb[q];
-            const uint64_t e = (uint64_t)(q - a.q_lo) + (j - a.mb_begin);
+            const uint64_t e = LIST ? cu0 + (q - q_lo) : (uint64_t)(q - a.q_lo) + (j - a.mb_begin);
             a.cu[e] = (int32_t)(pl.sample_row_off[q] - pl.mb_row_off[j]);
             if (q + 1 == pl.mb_sample_off[j + 1]) a.cu[e + 1] = (int32_t)(pl.sample_row_off[q + 1] - pl.mb_row_off[j]);
           }
@@ -134,7 +170,7 @@ __global__ void __launch_bounds__(kGatherThreads) k_gather(PoolView v, PlanView 
       const uint32_t nseg = desc[r].nseg;
       if (nseg == 0) continue;
       const uint32_t off0 = desc[r].off0, shift = desc[r].shift, mask = (1u << shift) - 1;
-      uint4* dst = reinterpret_cast<uint4*>(a.out + (tile * kTileRows + r - a.row_lo + desc[r].dst_shift) * v.row_bytes);
+      uint4* dst = reinterpret_cast<uint4*>(a.out + (uint64_t)desc[r].out_row * v.row_bytes);
       auto src_of = [&](uint32_t x, bool* take) -> const uint4* {
         const uint32_t ab = off0 + (x << 4);
         const uint64_t pte = desc[r].seg[ab >> shift];
@@ -177,33 +213,43 @@ __global__ void __launch_bounds__(32) k_gather_host_bulk(PoolView v, PlanView pl
   BulkRing ring;
   ring.init(smem, bars, dst_q, len_q);
   uint64_t item = 0;
-  for (uint32_t q = a.q_lo; q < a.q_hi; ++q) {
-    const uint32_t slot = pl.mb_samples[q], ns = v.s_n_spans[slot];
-    uint64_t row0 = pl.sample_row_off[q] - a.row_lo;
-    if (a.pad_L) {
-      const uint32_t mb = pl.plan_sample_mb[q];
-      row0 += (uint64_t)(mb - a.mb_begin) * a.pad_L - (pl.mb_row_off[mb] - a.row_lo);
+  // the samples to assemble: the call's range, or the samples of each listed microbatch in turn
+  const uint32_t n_parts = a.list ? a.n_list : 1;
+  for (uint32_t part = 0; part < n_parts; ++part) {
+    uint32_t q_lo = a.q_lo, q_hi = a.q_hi;
+    uint64_t part_row_lo = a.row_lo, part_out0 = 0;
+    if (a.list) {
+      const ListEntry en = a.list[part];
+      q_lo = en.q_lo; q_hi = en.q_hi; part_row_lo = en.row_lo; part_out0 = en.out_row0;
     }
-    for (uint32_t j = 0; j < ns; ++j) {
-      const uint32_t sid = slot * v.spans_per_sample + j;
-      const uint32_t npages = v.sp_npages[sid];
-      const uint64_t nbytes = (uint64_t)v.sp_tokens[sid] * v.row_bytes;
-      uint8_t* dst_base = a.out + (row0 + v.sp_pos[sid]) * v.row_bytes;
-      for (uint32_t g = 0; g < npages; g += 32, ++item) {
-        if (item % gridDim.x != blockIdx.x) continue;
-        const uint32_t o = g + lane;
-        uint64_t pte = 0, off;
-        if (o < npages) pte = translate(v, span_page_gva(v, sid, o), &off);
-        const bool host = (pte & kPteValid) && (pte & kPteHost);
-        const uint32_t mask = __ballot_sync(0xFFFFFFFFu, host);
-        for (uint32_t m = mask; m; m &= m - 1) {
-          const int l = __ffs(m) - 1;
-          const uint64_t p_l = __shfl_sync(0xFFFFFFFFu, pte, l);
-          const uint64_t b0 = (uint64_t)(g + l) << v.page_shift;
-          const uint64_t len = min(v.page_bytes, nbytes - b0);
-          const uint8_t* src = reinterpret_cast<const uint8_t*>(p_l & ~kPteFlagMask);
-          for (uint64_t x = 0; x < len; x += kBulkStageBytes)
-            ring.push(src + x, dst_base + b0 + x, (uint32_t)min((uint64_t)kBulkStageBytes, len - x));
+    for (uint32_t q = q_lo; q < q_hi; ++q) {
+      const uint32_t slot = pl.mb_samples[q], ns = v.s_n_spans[slot];
+      uint64_t row0 = part_out0 + (pl.sample_row_off[q] - part_row_lo);
+      if (!a.list && a.pad_L) {
+        const uint32_t mb = pl.plan_sample_mb[q];
+        row0 += (uint64_t)(mb - a.mb_begin) * a.pad_L - (pl.mb_row_off[mb] - a.row_lo);
+      }
+      for (uint32_t j = 0; j < ns; ++j) {
+        const uint32_t sid = slot * v.spans_per_sample + j;
+        const uint32_t npages = v.sp_npages[sid];
+        const uint64_t nbytes = (uint64_t)v.sp_tokens[sid] * v.row_bytes;
+        uint8_t* dst_base = a.out + (row0 + v.sp_pos[sid]) * v.row_bytes;
+        for (uint32_t g = 0; g < npages; g += 32, ++item) {
+          if (item % gridDim.x != blockIdx.x) continue;
+          const uint32_t o = g + lane;
+          uint64_t pte = 0, off;
+          if (o < npages) pte = translate(v, span_page_gva(v, sid, o), &off);
+          const bool host = (pte & kPteValid) && (pte & kPteHost);
+          const uint32_t mask = __ballot_sync(0xFFFFFFFFu, host);
+          for (uint32_t m = mask; m; m &= m - 1) {
+            const int l = __ffs(m) - 1;
+            const uint64_t p_l = __shfl_sync(0xFFFFFFFFu, pte, l);
+            const uint64_t b0 = (uint64_t)(g + l) << v.page_shift;
+            const uint64_t len = min(v.page_bytes, nbytes - b0);
+            const uint8_t* src = reinterpret_cast<const uint8_t*>(p_l & ~kPteFlagMask);
+            for (uint64_t x = 0; x < len; x += kBulkStageBytes)
+              ring.push(src + x, dst_base + b0 + x, (uint32_t)min((uint64_t)kBulkStageBytes, len - x));
+          }
         }
       }
     }
@@ -218,8 +264,10 @@ namespace ft {
 int32_t gather_device_setup(ft_pool* p) {
   FT_CUDA(cudaFuncSetAttribute(k_gather_host_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBulkSmemBytes));
   auto occ = [](auto kernel) { int v = 0; return cudaOccupancyMaxActiveBlocksPerMultiprocessor(&v, kernel, kGatherThreads, 0) == cudaSuccess && v > 0 ? v : 1; };
-  p->occ_gather[kTierAll][0] = occ(k_gather<kTierAll, 4>); p->occ_gather[kTierAll][1] = occ(k_gather<kTierAll, 8>);
-  p->occ_gather[kTierDeviceOnly][0] = occ(k_gather<kTierDeviceOnly, 4>); p->occ_gather[kTierDeviceOnly][1] = occ(k_gather<kTierDeviceOnly, 8>);
+  p->occ_gather[kTierAll][0] = std::min(occ(k_gather<kTierAll, 4, false>), occ(k_gather<kTierAll, 4, true>));
+  p->occ_gather[kTierAll][1] = std::min(occ(k_gather<kTierAll, 8, false>), occ(k_gather<kTierAll, 8, true>));
+  p->occ_gather[kTierDeviceOnly][0] = std::min(occ(k_gather<kTierDeviceOnly, 4, false>), occ(k_gather<kTierDeviceOnly, 4, true>));
+  p->occ_gather[kTierDeviceOnly][1] = std::min(occ(k_gather<kTierDeviceOnly, 8, false>), occ(k_gather<kTierDeviceOnly, 8, true>));
   return FT_OK;
 }
 }  // namespace ft
@@ -229,31 +277,45 @@ namespace ft {
 // pad_L = 0: packed rows, cu_seqlens and position ids written; pad_L = L: rows land in the padded layout and
 // the index outputs are left to the caller.  Arguments are validated by the caller.
 int32_t gather_launch(ft_pool* p, const ft_plan* pl, uint32_t mb_begin, uint32_t mb_end, const void* embed_table,
-                      uint32_t vocab, void* out_embeds, int32_t* out_cu, int32_t* out_pos, uint32_t pad_L, cudaStream_t st) {
+                      uint32_t vocab, void* out_embeds, int32_t* out_cu, int32_t* out_pos, uint32_t pad_L, cudaStream_t st,
+                      const void* d_list, uint32_t n_list, uint64_t list_tiles, uint64_t list_rows) {
+  if (p->view.row_bytes > (kMaxSeg - 1) * 4096) return FT_ERR_CAPACITY;
   const PlanView pv = make_plan_view(pl);
+  const bool listed = d_list != nullptr;
   GatherArgs a;
   a.q_lo = pl->h_mb_sample_off[mb_begin]; a.q_hi = pl->h_mb_sample_off[mb_end]; a.mb_begin = mb_begin;
   a.row_lo = pl->h_mb_row_off[mb_begin]; a.row_hi = pl->h_mb_row_off[mb_end];
   a.table = static_cast<const uint8_t*>(embed_table); a.vocab = vocab;
   a.out = static_cast<uint8_t*>(out_embeds); a.cu = out_cu; a.pos_ids = out_pos;
   a.call_seq = p->call_seq; a.write_index = pad_L == 0; a.pad_L = pad_L;
+  a.list = static_cast<const ListEntry*>(d_list); a.n_list = n_list; a.list_tiles = list_tiles;
+  const uint64_t n_tiles = listed ? list_tiles : (a.row_hi + kTileRows - 1) / kTileRows - a.row_lo / kTileRows;
+  const uint64_t n_rows = listed ? list_rows : a.row_hi - a.row_lo;
+  if (n_rows >> 32) return FT_ERR_CAPACITY;  // output row indices are 32-bit inside the kernel
   a.tile_counter = p->view.status + 1;  // scratch word next to the status word
   FT_CUDA(cudaMemsetAsync(a.tile_counter, 0, 8, st));
-  const uint64_t n_tiles = (a.row_hi + kTileRows - 1) / kTileRows - a.row_lo / kTileRows;
   // the grid-stride tile loop assumes every CTA runs from the start: never launch more than fit at once
   auto launch = [&](auto kernel, int mode, uint64_t want_per_sm, const GatherArgs& args, cudaStream_t s) {
     const uint64_t resident = (uint64_t)std::max(1, p->occ_gather[mode][p->gather_unroll == 8 ? 1 : 0]);
     const uint64_t ctas = (uint64_t)p->sm_count * std::min<uint64_t>(want_per_sm, resident);
     kernel<<<(unsigned)std::min<uint64_t>(n_tiles, ctas), kGatherThreads, 0, s>>>(p->view, pv, args);
   };
+  auto launch_mode = [&](auto mode_tag, const GatherArgs& args, uint64_t want_per_sm) {
+    constexpr int M = decltype(mode_tag)::value;
+    const bool u8 = p->gather_unroll == 8;
+    if (listed) {
+      if (u8) launch(k_gather<M, 8, true>, M, want_per_sm, args, st); else launch(k_gather<M, 4, true>, M, want_per_sm, args, st);
+    } else {
+      if (u8) launch(k_gather<M, 8, false>, M, want_per_sm, args, st); else launch(k_gather<M, 4, false>, M, want_per_sm, args, st);
+    }
+  };
   const uint64_t per_sm = (p->cfg.hbm_pages == 0 && p->cfg.world_size == 1) ? 1 : (uint64_t)p->dev_ctas_per_sm;
-  const bool u8 = p->gather_unroll == 8;
   // one launch when only one tier can be a source (own and imported bindings); otherwise one launch per tier
   const bool host_sources = p->cfg.host_pages != 0 || p->peer_host_frames;
   const bool only_host = p->cfg.hbm_pages == 0 && !(p->cfg.world_size > 1);
   if (!host_sources || only_host) {
     prof_begin(p, only_host ? FT_K_GATHER_HOST : FT_K_GATHER_DEVICE, st);
-    if (u8) launch(k_gather<kTierAll, 8>, kTierAll, per_sm, a, st); else launch(k_gather<kTierAll, 4>, kTierAll, per_sm, a, st);
+    launch_mode(std::integral_constant<int, kTierAll>{}, a, per_sm);
     prof_end(p, st);
     p->gpu_launches += 1;
   } else {
@@ -266,13 +328,13 @@ int32_t gather_launch(ft_pool* p, const ft_plan* pl, uint32_t mb_begin, uint32_t
     prof_end(p, p->side_stream[1]);
     FT_CUDA(cudaEventRecord(p->join_ev[1], p->side_stream[1]));
     prof_begin(p, FT_K_GATHER_DEVICE, st);
-    if (u8) launch(k_gather<kTierDeviceOnly, 8>, kTierDeviceOnly, per_sm, a, st); else launch(k_gather<kTierDeviceOnly, 4>, kTierDeviceOnly, per_sm, a, st);
+    launch_mode(std::integral_constant<int, kTierDeviceOnly>{}, a, per_sm);
     prof_end(p, st);
     FT_CUDA(cudaStreamWaitEvent(st, p->join_ev[1], 0));
     p->gpu_launches += 2;
   }
   FT_CUDA(cudaGetLastError());
-  p->bytes_gathered += (a.row_hi - a.row_lo) * 2ull * p->view.row_bytes;
+  p->bytes_gathered += n_rows * 2ull * p->view.row_bytes;
   return FT_OK;
 }
 }  // namespace ft
@@ -303,8 +365,58 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_gather_packed(ft_
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   {
-    const int32_t rc1 = gather_launch(p, pl, mb_begin, mb_end, embed_table, vocab, out_embeds, out_cu, out_pos, 0, st);
+    const int32_t rc1 = gather_launch(p, pl, mb_begin, mb_end, embed_table, vocab, out_embeds, out_cu, out_pos, 0, st, nullptr, 0, 0, 0);
     if (rc1 != FT_OK) return rc1;
+  }
+  const_cast<ft_plan*>(pl)->last_stream = st;
+  return end_consumer(p, st);
+}
+
+extern "C" __attribute__((visibility("default"))) int32_t pool_gather_list(ft_pool* p, const ft_plan* pl, const uint32_t* mb_list, uint32_t n_list,
+                                                                           const void* embed_table, uint32_t vocab, void* out_embeds, int32_t* out_cu,
+                                                                           int32_t* out_pos, void* stream) {
+  if (!p || !pl || pl->pool != p || (n_list && !mb_list)) return FT_ERR_INVALID_ARG;
+  p->call_seq++;
+  for (uint32_t i = 0; i < n_list; ++i)
+    if (mb_list[i] >= pl->n_mb) return FT_ERR_INVALID_ARG;
+  if (pl->free_epoch != p->free_epoch || (pl->cfg.flags & FT_PLAN_ALLOW_UNWRITTEN)) {
+    for (uint32_t t = 0; t < pl->n; ++t) {
+      const ft_slot_mirror& s = p->slots[pl->slots[t]];
+      if (s.state != FT_SLOT_READY || s.generation != pl->slot_generation[t]) return FT_ERR_NOT_READY;
+    }
+  }
+  if (n_list == 0) return FT_OK;
+  if (!embed_table || !out_embeds || !out_cu || !out_pos) return FT_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(out_embeds) & 15 || reinterpret_cast<uintptr_t>(embed_table) & 15) return FT_ERR_INVALID_ARG;
+  if (p->view.row_bytes > (kMaxSeg - 1) * 4096) return FT_ERR_CAPACITY;
+  // one entry per listed microbatch: its plan rows, and where its tiles, output rows and cu_seqlens entries start
+  std::vector<ListEntry> entries(n_list);
+  uint64_t tiles = 0, rows = 0, cu = 0;
+  for (uint32_t i = 0; i < n_list; ++i) {
+    const uint32_t j = mb_list[i];
+    ListEntry& en = entries[i];
+    en.row_lo = pl->h_mb_row_off[j]; en.row_hi = pl->h_mb_row_off[j + 1];
+    en.q_lo = pl->h_mb_sample_off[j]; en.q_hi = pl->h_mb_sample_off[j + 1];
+    en.tile0 = tiles; en.out_row0 = rows; en.cu0 = (uint32_t)cu; en.pad = 0;
+    tiles += (en.row_hi + kTileRows - 1) / kTileRows - en.row_lo / kTileRows;
+    rows += en.row_hi - en.row_lo;
+    cu += (uint64_t)(en.q_hi - en.q_lo) + 1;
+  }
+  if ((rows >> 32) || (cu >> 32)) return FT_ERR_CAPACITY;  // output row indices are 32-bit inside the kernels
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  {
+    const int32_t rc0 = begin_consumer(p, st);
+    if (rc0 != FT_OK) return rc0;
+  }
+  void* d = nullptr;
+  const size_t bytes = entries.size() * sizeof(ListEntry);
+  {
+    const int32_t rc1 = stage_upload(p, 1, entries.data(), bytes, bytes, st, &d);
+    if (rc1 != FT_OK) return rc1;
+  }
+  {
+    const int32_t rc2 = gather_launch(p, pl, 0, pl->n_mb, embed_table, vocab, out_embeds, out_cu, out_pos, 0, st, d, n_list, tiles, rows);
+    if (rc2 != FT_OK) return rc2;
   }
   const_cast<ft_plan*>(pl)->last_stream = st;
   return end_consumer(p, st);

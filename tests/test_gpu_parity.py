@@ -450,3 +450,67 @@ def test_plan_variants_match_oracle(flags):
     assert np.array_equal(out.cpu().numpy().view(np.uint16), oout)
     assert np.array_equal(cu.cpu().numpy(), ocu) and np.array_equal(pos.cpu().numpy(), opos)
     pool.destroy(); opool.destroy()
+
+
+@pytest.mark.parametrize("name,kw", [
+    ("image_mix_7b", dict(n_samples=40, hidden=56, page_bytes=4096)),    # host tier, many small microbatches
+    ("image_mix_7b", dict(n_samples=14)),                                # 2 MiB pages, both tiers
+    ("video_heavy", dict(n_samples=6)),
+])
+def test_rank_lists_match_oracle(name, kw):
+    """A rank assembles the microbatches dealt to it (Algorithm 1, lines 15-27) in one call."""
+    gh = _gpu()
+    w = workloads.make_workload(name, **kw)
+    w.budget_L = int(w.seq_len.max())          # several microbatches
+    r = gh.CudaRun(w)
+    r.run_schedule()
+    rc, plan = r.plan()
+    assert rc == 0
+    a = plan.arrays()
+    n_mb = int(a["n_mb"])
+    assert n_mb >= 3
+    table = workloads.embed_table(w, device="cuda")
+    pool = OraclePool(PoolConfig(**pool_config_fields(w)))
+    for call in w.write_calls:
+        samples = sorted({s for s, _ in call}, key=[s for s, _ in call].index)
+        assert pool.register_samples(*register_args(w, samples)) == 0
+        assert pool.write_embeddings(*write_args(w, call), [gh.host_bits(r.srcs[c]) for c in call], w.src_dtype) == 0
+    rc, oplan = pool.plan_microbatches(np.asarray(w.plan_order, dtype=np.uint32), PlanConfig(**plan_config_fields(w)))
+    assert rc == 0 and np.array_equal(oplan.arrays()["rank_mbs"], a["rank_mbs"])
+    tok = a["mb_tokens"].astype(np.int64)
+    n_s = np.diff(a["mb_sample_off"].astype(np.int64))
+    lists = [[int(j) for j in a["rank_mbs"][a["rank_mb_off"][k]:a["rank_mb_off"][k + 1]]] for k in range(w.n_ranks_N)]
+    lists += [list(range(n_mb))[::-1], [1, 1, 0], [n_mb - 1]]
+    for lst in lists:
+        rows, n_cu = int(tok[lst].sum()) if lst else 0, int((n_s[lst] + 1).sum()) if lst else 0
+        out = torch.full((max(rows, 1), w.hidden), -1, dtype=torch.int16, device="cuda")
+        cu = torch.full((max(n_cu, 1),), -7, dtype=torch.int32, device="cuda")
+        pos = torch.full((max(rows, 1),), -7, dtype=torch.int32, device="cuda")
+        g = r.pool.gather_list(plan, lst, table.data_ptr(), w.vocab, out.data_ptr(), cu.data_ptr(), pos.data_ptr(), gh.cuda_stream())
+        oout = np.full((max(rows, 1), w.hidden), 0xFFFF, np.uint16)
+        ocu = np.full(max(n_cu, 1), -7, np.int32)
+        opos = np.full(max(rows, 1), -7, np.int32)
+        o = pool.gather_list(oplan, lst, bits16(table), oout, ocu, opos)
+        assert g == o == 0
+        torch.cuda.synchronize()
+        assert np.array_equal(out.cpu().numpy().view(np.uint16), oout), lst
+        assert np.array_equal(cu.cpu().numpy(), ocu) and np.array_equal(pos.cpu().numpy(), opos), lst
+    # errors: no such microbatch; ids outside a short table (detail = row in the list's output); dead plan
+    args = (table.data_ptr(), w.vocab, out.data_ptr(), cu.data_ptr(), pos.data_ptr(), gh.cuda_stream())
+    assert r.pool.gather_list(plan, [0, n_mb], *args) == pool.gather_list(oplan, [0, n_mb], bits16(table), oout, ocu, opos) == -1
+    lst = [2, 0]
+    rows = int(tok[lst].sum())
+    out = torch.full((rows, w.hidden), -1, dtype=torch.int16, device="cuda")
+    cu = torch.zeros((int((n_s[lst] + 1).sum()),), dtype=torch.int32, device="cuda")
+    pos = torch.zeros((rows,), dtype=torch.int32, device="cuda")
+    assert r.pool.gather_list(plan, lst, table.data_ptr(), 100, out.data_ptr(), cu.data_ptr(), pos.data_ptr(), gh.cuda_stream()) == 0
+    oout = np.full((rows, w.hidden), 0xFFFF, np.uint16)
+    assert pool.gather_list(oplan, lst, bits16(table)[:100], oout, np.zeros(len(cu), np.int32), np.zeros(rows, np.int32)) == 0
+    st_g, st_o = r.pool.status(), pool.status()
+    assert st_g == st_o and st_g[0] == -9
+    assert np.array_equal(out.cpu().numpy().view(np.uint16), oout)          # skipped rows stay untouched on both sides
+    first = int(a["mb_samples"][0])
+    assert r.pool.free([first], gh.cuda_stream()) == pool.free([first]) == 0
+    assert r.pool.gather_list(plan, [0], *args) == pool.gather_list(oplan, [0], bits16(table), oout, ocu, opos) == -5
+    oplan.destroy(); pool.destroy()
+    r.close()
