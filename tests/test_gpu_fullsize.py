@@ -85,6 +85,33 @@ def test_full_size_plan_and_sampled_rows(name, kw):
             pass
     # no row left at poison anywhere (checked on the device)
     assert not bool((out == -1).all(dim=1).any().item())
+    # every rank's share of the deal in one list call each: the same rows, cu_seqlens and positions as the
+    # slices of the range assembly checked above
+    from gpu_harness import cuda_stream
+    mb_rows = np.concatenate([[0], np.cumsum(exp["mb_tokens"].astype(np.int64))])
+    mb_cu = np.concatenate([[0], np.cumsum(np.diff(exp["mb_sample_off"].astype(np.int64)) + 1)])
+    cu_h, pos_h = cu.cpu().numpy(), pos.cpu().numpy()
+    cap = int(max(sum(mb_rows[j + 1] - mb_rows[j] for j in exp["rank_mbs"][exp["rank_mb_off"][k]:exp["rank_mb_off"][k + 1]])
+                  for k in range(w.n_ranks_N)))
+    l_out = torch.empty((cap, w.hidden), dtype=torch.int16, device="cuda")
+    l_cu = torch.empty((len(cu_h),), dtype=torch.int32, device="cuda")
+    l_pos = torch.empty((cap,), dtype=torch.int32, device="cuda")
+    for k in range(w.n_ranks_N):
+        lst = [int(j) for j in exp["rank_mbs"][exp["rank_mb_off"][k]:exp["rank_mb_off"][k + 1]]]
+        if not lst:
+            continue
+        l_out.fill_(-1)
+        assert run.pool.gather_list(plan, lst, run.table.data_ptr(), w.vocab, l_out.data_ptr(), l_cu.data_ptr(), l_pos.data_ptr(),
+                                    cuda_stream()) == 0
+        torch.cuda.synchronize()
+        base = c_base = 0
+        for j in lst:
+            n_r, n_c = int(mb_rows[j + 1] - mb_rows[j]), int(mb_cu[j + 1] - mb_cu[j])
+            assert torch.equal(l_out[base:base + n_r], out[int(mb_rows[j]):int(mb_rows[j + 1])])
+            assert np.array_equal(l_pos[base:base + n_r].cpu().numpy(), pos_h[mb_rows[j]:mb_rows[j + 1]])
+            assert np.array_equal(l_cu[c_base:c_base + n_c].cpu().numpy(), cu_h[mb_cu[j]:mb_cu[j + 1]])
+            base += n_r; c_base += n_c
+    assert run.pool.status() == (0, 0)
     oplan.destroy()
     run.close()
 

@@ -34,7 +34,7 @@ def test_random_call_sequences_agree_with_oracle(seed, ring_order, page_bytes, h
     table = workloads.embed_table(w, device="cuda")
     table_h = bits16(table)
     keep, plans = [], []
-    n_calls = {"register": 0, "write": 0, "free": 0, "plan": 0, "gather": 0, "grids": 0, "padded": 0, "grad": 0}
+    n_calls = {"register": 0, "write": 0, "free": 0, "plan": 0, "gather": 0, "glist": 0, "grids": 0, "padded": 0, "grad": 0}
     n_ok = dict(n_calls)
 
     def check_state():
@@ -50,7 +50,7 @@ def test_random_call_sequences_agree_with_oracle(seed, ring_order, page_bytes, h
         return [s for s, wr in state.items() if len(wr) == int(w.n_spans[s])]
 
     for step in range(260):
-        op = rng.choice(["register", "write", "write", "free", "plan", "gather", "grids", "padded", "grad"])
+        op = rng.choice(["register", "write", "write", "free", "plan", "gather", "glist", "grids", "padded", "grad"])
         n_calls[op] += 1
         sloppy = rng.random() < 0.2     # one call in five is built without looking at the model
         if op == "register":
@@ -117,6 +117,29 @@ def test_random_call_sequences_agree_with_oracle(seed, ring_order, page_bytes, h
                     assert np.array_equal(ga[key], oa[key]), (step, key)
                 plans.append((gp, op_, len(slots), cfg["budget_L"]))
                 plans[:] = plans[-4:]
+        elif op == "glist":
+            if not plans:
+                n_calls[op] -= 1
+                continue
+            gp, op_, n, _budget = plans[int(rng.integers(0, len(plans)))]
+            n_mb, total, _ = op_.summary()
+            oa_ = op_.arrays()
+            lst = [int(x) for x in rng.integers(0, n_mb + (1 if sloppy else 0), size=int(rng.integers(0, 6)))] if n_mb or sloppy else []
+            ok_l = [j for j in lst if j < n_mb]
+            rows = max(1, int(sum(int(oa_["mb_tokens"][j]) for j in ok_l)))
+            n_cu = max(1, int(sum(int(oa_["mb_sample_off"][j + 1] - oa_["mb_sample_off"][j]) + 1 for j in ok_l)))
+            out = torch.full((rows, w.hidden), -1, dtype=torch.int16, device="cuda")
+            cu = torch.full((n_cu,), -7, dtype=torch.int32, device="cuda")
+            pos = torch.full((rows,), -7, dtype=torch.int32, device="cuda")
+            g = pool.gather_list(gp, lst, table.data_ptr(), w.vocab, out.data_ptr(), cu.data_ptr(), pos.data_ptr(), cuda_stream())
+            oout = np.full((rows, w.hidden), 0xFFFF, np.uint16)
+            ocu = np.full(n_cu, -7, np.int32)
+            opos = np.full(rows, -7, np.int32)
+            o = opool.gather_list(op_, lst, table_h, oout, ocu, opos)
+            if g == 0 and o == 0:
+                torch.cuda.synchronize()
+                assert np.array_equal(out.cpu().numpy().view(np.uint16), oout), step
+                assert np.array_equal(cu.cpu().numpy(), ocu) and np.array_equal(pos.cpu().numpy(), opos), step
         elif op == "grids":
             if sloppy or not state:
                 k = int(rng.integers(1, 4))
