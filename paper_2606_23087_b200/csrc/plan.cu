@@ -58,144 +58,151 @@ __global__ void __launch_bounds__(256) k_pack_order(const uint32_t* __restrict__
 }
 
 // Residual bitmap: bit r of level 0 is set when some open microbatch has residual r; bit i of level k+1 is set
-// when word i of level k is non-zero.  Four levels of 32-ary words cover residuals below 2^20.
-struct FitLevels {
-  uint32_t *b0, *b1, *b2, *b3;
-  uint32_t w0, w1, w2, w3;
+// when word i of level k is non-zero.  Four levels of 32-ary words cover residuals below 2^20.  The levels live in
+// the kernel's shared memory and are addressed by word offsets from its base; every level carries one zero word
+// of padding behind its last word, so the query needs no bounds checks.
+struct FitOff {
+  uint32_t b0, b1, b2, b3;  // word offsets of the levels
 };
 
 // smallest set index >= l, or kNone: the best-fit query (the segment-tree descent of Algorithm 1, 32-ary)
-__device__ __forceinline__ uint32_t fit_find(const FitLevels& f, uint32_t l) {
+__device__ __forceinline__ uint32_t fit_find(const uint32_t* sm, const FitOff f, uint32_t l) {
   uint32_t w = l >> 5;
-  uint32_t m = w < f.w0 ? f.b0[w] & (0xFFFFFFFFu << (l & 31)) : 0;
+  uint32_t m = sm[f.b0 + w] & (0xFFFFFFFFu << (l & 31));
   if (m) return (w << 5) + __ffs(m) - 1;
-  uint32_t i1 = w + 1;
+  const uint32_t i1 = w + 1;
   w = i1 >> 5;
-  m = w < f.w1 ? f.b1[w] & (0xFFFFFFFFu << (i1 & 31)) : 0;
+  m = sm[f.b1 + w] & (0xFFFFFFFFu << (i1 & 31));
   if (m) {
     const uint32_t p0 = (w << 5) + __ffs(m) - 1;
-    return (p0 << 5) + __ffs(f.b0[p0]) - 1;
+    return (p0 << 5) + __ffs(sm[f.b0 + p0]) - 1;
   }
-  uint32_t i2 = w + 1;
+  const uint32_t i2 = w + 1;
   w = i2 >> 5;
-  m = w < f.w2 ? f.b2[w] & (0xFFFFFFFFu << (i2 & 31)) : 0;
+  m = sm[f.b2 + w] & (0xFFFFFFFFu << (i2 & 31));
   if (m) {
     const uint32_t p1 = (w << 5) + __ffs(m) - 1;
-    const uint32_t p0 = (p1 << 5) + __ffs(f.b1[p1]) - 1;
-    return (p0 << 5) + __ffs(f.b0[p0]) - 1;
+    const uint32_t p0 = (p1 << 5) + __ffs(sm[f.b1 + p1]) - 1;
+    return (p0 << 5) + __ffs(sm[f.b0 + p0]) - 1;
   }
-  uint32_t i3 = w + 1;
+  const uint32_t i3 = w + 1;
   w = i3 >> 5;
-  m = w < f.w3 ? f.b3[w] & (0xFFFFFFFFu << (i3 & 31)) : 0;
+  m = sm[f.b3 + w] & (0xFFFFFFFFu << (i3 & 31));
   if (m) {
     const uint32_t p2 = (w << 5) + __ffs(m) - 1;
-    const uint32_t p1 = (p2 << 5) + __ffs(f.b2[p2]) - 1;
-    const uint32_t p0 = (p1 << 5) + __ffs(f.b1[p1]) - 1;
-    return (p0 << 5) + __ffs(f.b0[p0]) - 1;
+    const uint32_t p1 = (p2 << 5) + __ffs(sm[f.b2 + p2]) - 1;
+    const uint32_t p0 = (p1 << 5) + __ffs(sm[f.b1 + p1]) - 1;
+    return (p0 << 5) + __ffs(sm[f.b0 + p0]) - 1;
   }
   return kNone;
 }
-__device__ __forceinline__ void fit_set(const FitLevels& f, uint32_t r) {
-  uint32_t old = f.b0[r >> 5];
-  f.b0[r >> 5] = old | (1u << (r & 31));
+__device__ __forceinline__ void fit_set(uint32_t* sm, const FitOff f, uint32_t r) {
+  uint32_t old = sm[f.b0 + (r >> 5)];
+  sm[f.b0 + (r >> 5)] = old | (1u << (r & 31));
   if (old) return;
-  r >>= 5; old = f.b1[r >> 5]; f.b1[r >> 5] = old | (1u << (r & 31));
+  r >>= 5; old = sm[f.b1 + (r >> 5)]; sm[f.b1 + (r >> 5)] = old | (1u << (r & 31));
   if (old) return;
-  r >>= 5; old = f.b2[r >> 5]; f.b2[r >> 5] = old | (1u << (r & 31));
+  r >>= 5; old = sm[f.b2 + (r >> 5)]; sm[f.b2 + (r >> 5)] = old | (1u << (r & 31));
   if (old) return;
-  r >>= 5; f.b3[r >> 5] |= 1u << (r & 31);
+  r >>= 5; sm[f.b3 + (r >> 5)] |= 1u << (r & 31);
 }
-__device__ __forceinline__ void fit_clear(const FitLevels& f, uint32_t r) {
-  uint32_t nw = f.b0[r >> 5] & ~(1u << (r & 31));
-  f.b0[r >> 5] = nw;
+__device__ __forceinline__ void fit_clear(uint32_t* sm, const FitOff f, uint32_t r) {
+  uint32_t nw = sm[f.b0 + (r >> 5)] & ~(1u << (r & 31));
+  sm[f.b0 + (r >> 5)] = nw;
   if (nw) return;
-  r >>= 5; nw = f.b1[r >> 5] & ~(1u << (r & 31)); f.b1[r >> 5] = nw;
+  r >>= 5; nw = sm[f.b1 + (r >> 5)] & ~(1u << (r & 31)); sm[f.b1 + (r >> 5)] = nw;
   if (nw) return;
-  r >>= 5; nw = f.b2[r >> 5] & ~(1u << (r & 31)); f.b2[r >> 5] = nw;
+  r >>= 5; nw = sm[f.b2 + (r >> 5)] & ~(1u << (r & 31)); sm[f.b2 + (r >> 5)] = nw;
   if (nw) return;
-  r >>= 5; f.b3[r >> 5] &= ~(1u << (r & 31));
+  r >>= 5; sm[f.b3 + (r >> 5)] &= ~(1u << (r & 31));
 }
 
 // One block.  Thread 0 walks the samples in order (the dependency chain of online best fit); the other
 // threads stage lengths in and results out, coalesced, and initialise / flush the tables.
 // HEAD_SMEM: the per-residual stack heads live in shared memory (budgets up to about 32 K), else in global.
-template <bool HEAD_SMEM>
+// RECS_SMEM: every microbatch record fits in shared memory (else those past rec_smem_cap live in global).
+template <bool HEAD_SMEM, bool RECS_SMEM>
 __global__ void __launch_bounds__(1024) k_bestfit(const uint32_t* __restrict__ len, uint32_t n, uint32_t L,
                                                   uint32_t* __restrict__ head_g, MbRec* __restrict__ recs_g,
                                                   uint32_t rec_smem_cap, uint32_t* sample_mb, uint32_t* sample_rank,
                                                   uint32_t* mb_residual, uint32_t* mb_tokens, uint32_t* mb_lmax,
                                                   uint32_t* mb_count, uint32_t* scalars) {
-  extern __shared__ uint32_t sm[];
-  FitLevels f;
-  uint32_t* p = sm;
-  f.w0 = (L + 1 + 31) / 32; f.b0 = p; p += f.w0;
-  f.w1 = (f.w0 + 31) / 32;  f.b1 = p; p += f.w1;
-  f.w2 = (f.w1 + 31) / 32;  f.b2 = p; p += f.w2;
-  f.w3 = (f.w2 + 31) / 32;  f.b3 = p; p += f.w3;
-  const uint32_t total_words = (uint32_t)(p - sm);
-  uint32_t* c_len = p; p += kFitChunk;
-  uint32_t* c_mb = p; p += kFitChunk;
-  uint32_t* c_rank = p; p += kFitChunk;
-  uint32_t* head_s = p;
-  if (HEAD_SMEM) p += L + 1;
-  p += (4 - ((p - sm) & 3)) & 3;  // 16-byte align the records
-  MbRec* recs_s = reinterpret_cast<MbRec*>(p);
+  extern __shared__ __align__(16) uint32_t sm[];
+  FitOff f;
+  uint32_t o = 0;
+  const uint32_t w0 = (L + 1 + 31) / 32, w1 = (w0 + 31) / 32, w2 = (w1 + 31) / 32, w3 = (w2 + 31) / 32;
+  f.b0 = o; o += w0 + 1;
+  f.b1 = o; o += w1 + 1;
+  f.b2 = o; o += w2 + 1;
+  f.b3 = o; o += w3 + 1;
+  const uint32_t total_words = o;
+  const uint32_t o_len = o; o += kFitChunk;
+  const uint32_t o_mb = o; o += kFitChunk;
+  const uint32_t o_rank = o; o += kFitChunk;
+  const uint32_t o_head = o;
+  if (HEAD_SMEM) o += L + 1;
+  o = (o + 3) & ~3u;  // 16-byte align the records
+  uint4* recs_s = reinterpret_cast<uint4*>(sm + o);
+  uint4* recs_gv = reinterpret_cast<uint4*>(recs_g);
 
   for (uint32_t i = threadIdx.x; i < total_words; i += blockDim.x) sm[i] = 0;
-  if (HEAD_SMEM) { for (uint32_t i = threadIdx.x; i <= L; i += blockDim.x) head_s[i] = kNone; }
+  if (HEAD_SMEM) { for (uint32_t i = threadIdx.x; i <= L; i += blockDim.x) sm[o_head + i] = kNone; }
   else { for (uint32_t i = threadIdx.x; i <= L; i += blockDim.x) head_g[i] = kNone; }
   __shared__ uint32_t s_nmb;
   if (threadIdx.x == 0) s_nmb = 0;
   __syncthreads();
 
-  auto head_ld = [&](uint32_t r) -> uint32_t { return HEAD_SMEM ? head_s[r] : head_g[r]; };
-  auto head_st = [&](uint32_t r, uint32_t v) { if (HEAD_SMEM) head_s[r] = v; else head_g[r] = v; };
+  auto head_ld = [&](uint32_t r) -> uint32_t { return HEAD_SMEM ? sm[o_head + r] : head_g[r]; };
+  auto head_st = [&](uint32_t r, uint32_t v) { if (HEAD_SMEM) sm[o_head + r] = v; else head_g[r] = v; };
+  // a record: x = residual, y = lmax, z = count, w = next (the MbRec layout)
+  auto rec_ld = [&](uint32_t j) -> uint4 { return (RECS_SMEM || j < rec_smem_cap) ? recs_s[j] : recs_gv[j]; };
+  auto rec_st = [&](uint32_t j, uint4 v) { if (RECS_SMEM || j < rec_smem_cap) recs_s[j] = v; else recs_gv[j] = v; };
 
   for (uint32_t base = 0; base < n; base += kFitChunk) {
     const uint32_t cnt = min(kFitChunk, n - base);
-    for (uint32_t i = threadIdx.x; i < cnt; i += blockDim.x) c_len[i] = len[base + i];
+    for (uint32_t i = threadIdx.x; i < cnt; i += blockDim.x) sm[o_len + i] = len[base + i];
     __syncthreads();
     if (threadIdx.x == 0) {
       uint32_t n_mb = s_nmb;
       for (uint32_t i = 0; i < cnt; ++i) {
-        const uint32_t l = c_len[i];
-        const uint32_t r = fit_find(f, l);  // the smallest residual >= l among open microbatches
+        const uint32_t l = sm[o_len + i];
+        const uint32_t r = fit_find(sm, f, l);  // the smallest residual >= l among open microbatches
         uint32_t j;
-        MbRec rec;
+        uint4 rec;
         if (r != kNone) {
           j = head_ld(r);  // most recently changed microbatch with that residual
-          if (j < rec_smem_cap) rec = recs_s[j]; else rec = recs_g[j];
-          head_st(r, rec.next);
-          if (rec.next == kNone) fit_clear(f, r);
-          rec.residual = r - l;
-          rec.lmax = max(rec.lmax, l);
-          rec.count++;
+          rec = rec_ld(j);
+          head_st(r, rec.w);
+          if (rec.w == kNone) fit_clear(sm, f, r);
+          rec.x = r - l;
+          rec.y = max(rec.y, l);
+          rec.z++;
         } else {
           j = n_mb++;
-          rec.residual = L - l; rec.lmax = l; rec.count = 1;
+          rec.x = L - l; rec.y = l; rec.z = 1;
         }
         // a residual of 0 can never be chosen again (l >= 1): it needs no stack entry
-        if (rec.residual) {
-          rec.next = head_ld(rec.residual);
-          head_st(rec.residual, j);
-          if (rec.next == kNone) fit_set(f, rec.residual);
+        if (rec.x) {
+          rec.w = head_ld(rec.x);
+          head_st(rec.x, j);
+          if (rec.w == kNone) fit_set(sm, f, rec.x);
         } else {
-          rec.next = kNone;
+          rec.w = kNone;
         }
-        if (j < rec_smem_cap) recs_s[j] = rec; else recs_g[j] = rec;
-        c_mb[i] = j;
-        c_rank[i] = rec.count - 1;
+        rec_st(j, rec);
+        sm[o_mb + i] = j;
+        sm[o_rank + i] = rec.z - 1;
       }
       s_nmb = n_mb;
     }
     __syncthreads();
-    for (uint32_t i = threadIdx.x; i < cnt; i += blockDim.x) { sample_mb[base + i] = c_mb[i]; sample_rank[base + i] = c_rank[i]; }
+    for (uint32_t i = threadIdx.x; i < cnt; i += blockDim.x) { sample_mb[base + i] = sm[o_mb + i]; sample_rank[base + i] = sm[o_rank + i]; }
     __syncthreads();
   }
   const uint32_t n_mb = s_nmb;
   for (uint32_t j = threadIdx.x; j < n_mb; j += blockDim.x) {
-    const MbRec rec = j < rec_smem_cap ? recs_s[j] : recs_g[j];
-    mb_residual[j] = rec.residual; mb_tokens[j] = L - rec.residual; mb_lmax[j] = rec.lmax; mb_count[j] = rec.count;
+    const uint4 rec = rec_ld(j);
+    mb_residual[j] = rec.x; mb_tokens[j] = L - rec.x; mb_lmax[j] = rec.y; mb_count[j] = rec.z;
   }
   if (threadIdx.x == 0) scalars[SC_NMB] = n_mb;
 }
@@ -357,8 +364,10 @@ static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; 
 namespace ft {
 constexpr size_t kBestfitSmemLimit = 227 * 1024 - 64;
 int32_t plan_device_setup(ft_pool* p) {
-  FT_CUDA(cudaFuncSetAttribute(k_bestfit<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBestfitSmemLimit));
-  FT_CUDA(cudaFuncSetAttribute(k_bestfit<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBestfitSmemLimit));
+  FT_CUDA(cudaFuncSetAttribute(k_bestfit<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBestfitSmemLimit));
+  FT_CUDA(cudaFuncSetAttribute(k_bestfit<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBestfitSmemLimit));
+  FT_CUDA(cudaFuncSetAttribute(k_bestfit<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBestfitSmemLimit));
+  FT_CUDA(cudaFuncSetAttribute(k_bestfit<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBestfitSmemLimit));
   // keep freed plan blocks cached in the device's default memory pool instead of returning them to the driver
   cudaMemPool_t mp;
   uint64_t keep = ~0ull;
@@ -470,7 +479,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_plan_microbatches
 
   // shared memory plan of k_bestfit: bitmaps, staging chunk, then the stack heads and records if they fit
   size_t words = 0;
-  { uint32_t w = (L + 1 + 31) / 32; for (int l = 0; l < 4; ++l) { words += w; w = (w + 31) / 32; } }
+  { uint32_t w = (L + 1 + 31) / 32; for (int l = 0; l < 4; ++l) { words += w + 1; w = (w + 31) / 32; } }  // one pad word per level
   const size_t fixed = (words + 3 * (size_t)kFitChunk) * 4 + 16;
   const size_t limit = kBestfitSmemLimit;
   const size_t head_bytes = ((size_t)L + 1) * 4;
@@ -481,12 +490,13 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_plan_microbatches
   const uint32_t f_sort = (cfg->flags & FT_PLAN_SORT_DECREASING) != 0, f_sumsq = (cfg->flags & FT_PLAN_COST_SUMSQ) != 0;
   const uint32_t f_carry = (cfg->flags & FT_PLAN_ZIGZAG_CARRY) != 0;
   k_pack_order<<<gb, 256, 0, st>>>(pl->d_len, n, f_sort, d_pk_t, d_pk_len);
-  if (head_in_smem)
-    k_bestfit<true><<<1, 1024, used, st>>>(d_pk_len, n, L, d_head, d_recs, rec_cap, d_pk_mb, pl->d_sample_rank,
-                                           pl->d_mb_residual, pl->d_mb_tokens, pl->d_mb_lmax, pl->d_mb_count, pl->d_scalars);
-  else
-    k_bestfit<false><<<1, 1024, used, st>>>(d_pk_len, n, L, d_head, d_recs, rec_cap, d_pk_mb, pl->d_sample_rank,
-                                            pl->d_mb_residual, pl->d_mb_tokens, pl->d_mb_lmax, pl->d_mb_count, pl->d_scalars);
+  {
+    const bool all_recs = rec_cap >= n;
+    auto fit = head_in_smem ? (all_recs ? k_bestfit<true, true> : k_bestfit<true, false>)
+                            : (all_recs ? k_bestfit<false, true> : k_bestfit<false, false>);
+    fit<<<1, 1024, used, st>>>(d_pk_len, n, L, d_head, d_recs, rec_cap, d_pk_mb, pl->d_sample_rank, pl->d_mb_residual,
+                               pl->d_mb_tokens, pl->d_mb_lmax, pl->d_mb_count, pl->d_scalars);
+  }
   k_mb_finalize<<<1, 1024, 0, st>>>(pl->d_mb_tokens, pl->d_mb_count, pl->d_mb_sample_off, pl->d_mb_row_off, pl->d_scalars);
   k_plan_scatter<<<gb, 256, 0, st>>>(pl->d_slots, d_pk_t, d_pk_len, d_pk_mb, pl->d_sample_rank, pl->d_mb_sample_off, n,
                                      pl->d_mb_samples, pl->d_plan_len, pl->d_plan_sample_mb, pl->d_sample_mb);
