@@ -334,26 +334,28 @@ struct HotArgs {
 // one CTA: the first kMaxHot ids (in ascending id order) with at least `threshold` rows; they are then numbered by
 // descending row count (ties by id), so the longest lists are started first; and where each list starts
 __global__ void __launch_bounds__(1024) k_hot_select(HotArgs a) {
-  __shared__ uint32_t s_base;
   __shared__ int32_t s_ids[kMaxHot];
   __shared__ uint32_t s_cnt[kMaxHot], s_sorted[kMaxHot];
   static_assert(kMaxHot <= 1024, "one thread per frequent id below");
-  if (threadIdx.x == 0) s_base = 0;
-  __syncthreads();
-  for (uint32_t v0 = 0; v0 < a.vocab; v0 += blockDim.x) {
-    const uint32_t v = v0 + threadIdx.x;
-    const uint32_t base = s_base;
-    const uint32_t c = (base < kMaxHot && v < a.vocab) ? a.id_count[v] : 0;
-    const bool hot = c >= a.threshold && c > 0;
-    uint64_t tot;
-    const uint32_t idx = base + (uint32_t)block_exclusive_scan(hot ? 1 : 0, &tot);
-    if (hot && idx < kMaxHot) { s_ids[idx] = (int32_t)v; s_cnt[idx] = c; }
-    if (v < a.vocab) a.hot_index[v] = -1;
-    __syncthreads();
-    if (threadIdx.x == 0) s_base = min(kMaxHot, base + (uint32_t)tot);
-    __syncthreads();
+  // thread t looks at the ids [t * per, (t + 1) * per): one scan over the threads' counts keeps id order
+  const uint32_t per = (a.vocab + blockDim.x - 1) / blockDim.x;
+  const uint32_t v0 = threadIdx.x * per, v1 = min(a.vocab, v0 + per);
+  uint32_t mine = 0;
+  for (uint32_t v = v0; v < v1; ++v) {
+    const uint32_t c = a.id_count[v];
+    mine += c >= a.threshold && c > 0;
+    a.hot_index[v] = -1;
   }
-  const uint32_t n = s_base;
+  uint64_t tot;
+  uint32_t idx = (uint32_t)block_exclusive_scan(mine, &tot);
+  if (mine && idx < kMaxHot) {
+    for (uint32_t v = v0; v < v1 && idx < kMaxHot; ++v) {
+      const uint32_t c = a.id_count[v];
+      if (c >= a.threshold && c > 0) { s_ids[idx] = (int32_t)v; s_cnt[idx] = c; ++idx; }
+    }
+  }
+  __syncthreads();
+  const uint32_t n = min((uint32_t)tot, kMaxHot);
   const uint32_t i = threadIdx.x;
   if (i < n) {
     uint32_t rank = 0;
