@@ -263,3 +263,88 @@ def test_full_size_backbone_side(name, id_skew):
         assert np.array_equal(gt[v].cpu().numpy().view(np.uint32), acc.view(np.uint32)), v
     assert run.pool.status() == (0, 0)
     run.close()
+
+
+@pytest.mark.parametrize("page_bytes", [2 << 20, 4096])
+def test_full_size_fragmentation_sweep(page_bytes):
+    """Config 5 as bench.py runs it: a stream of 65 536 samples flows through a 64 GiB all-HBM pool (10 write/free
+    cycles, final admit), then the residents are planned and assembled in ranges.  The plan is compared array by
+    array with the oracle's Algorithm 1 on the residents' lengths; position ids and cu_seqlens in full with what the
+    plan determines; sampled rows of every range with rows the generator gives one by one."""
+    if not torch.cuda.is_available():
+        pytest.fail("a CUDA device is required for -m gpu tests")
+    from gpu_harness import cuda_stream
+    from harness import pool_config_fields, register_args, write_args
+    from paper_2606_23087_b200 import binding as fp
+    free_b, _ = torch.cuda.mem_get_info()
+    pool_bytes = (64 << 30) if free_b >= (90 << 30) else (32 << 30)
+    w = workloads.make_workload("frag_sweep", n_samples=65536, page_bytes=page_bytes, pool_bytes=pool_bytes)
+    ops, residents = workloads.admit_free_schedule(w, cycles=10)
+    pool = fp.Pool(fp.PoolConfig(**pool_config_fields(w)))
+    assert pool.rc == 0
+    st = cuda_stream()
+    for kind, samples in ops:
+        if kind == "free":
+            assert pool.free(samples, st) == 0
+            continue
+        for i in range(0, len(samples), 256):
+            part = samples[i:i + 256]
+            reg = register_args(w, part)
+            ids = torch.from_numpy(reg[5]).cuda()
+            srcs = [workloads.span_values(w, s, 0, device="cuda") for s in part]
+            assert pool.register_samples(*reg[:5], ids.data_ptr(), st) == 0
+            assert pool.write_embeddings(*write_args(w, [(s, 0) for s in part]), [t.data_ptr() for t in srcs], 0, st) == 0
+            torch.cuda.synchronize()
+    assert pool.status() == (0, 0)
+    order = np.asarray(residents, dtype=np.uint32)
+    cfg = plan_config_fields(w)
+    rc, plan = pool.plan_microbatches(order, fp.PlanConfig(**cfg), st)
+    assert rc == 0
+    got = plan.arrays()
+    rc, oplan = plan_from_lengths(w.seq_len[order], PlanConfig(**cfg), slots=order)
+    assert rc == 0
+    exp = oplan.arrays()
+    for k in PLAN_KEYS:
+        assert np.array_equal(got[k], exp[k]), k
+    n_mb, total, _ = plan.summary()
+    assert (n_mb, total) == oplan.summary()[:2] and len(residents) > 8000
+    table = workloads.embed_table(w, device="cuda")
+    buf_rows = min(total, 1 << 20)
+    out = torch.empty((buf_rows, w.hidden), dtype=torch.int16, device="cuda")
+    cu = torch.empty((len(residents) + n_mb + 8,), dtype=torch.int32, device="cuda")
+    pos = torch.empty((buf_rows,), dtype=torch.int32, device="cuda")
+    lens = w.seq_len[exp["mb_samples"]].astype(np.int64)
+    row_off = np.concatenate([[0], np.cumsum(lens)])
+    mb_row = np.concatenate([[0], np.cumsum(exp["mb_tokens"].astype(np.int64))])
+    ranges, b, rows = [], 0, 0
+    for j in range(n_mb):
+        t = int(exp["mb_tokens"][j])
+        if rows + t > buf_rows:
+            ranges.append((b, j)); b, rows = j, 0
+        rows += t
+    ranges.append((b, n_mb))
+    rng = np.random.default_rng(17)
+    for lo, hi in ranges:
+        out.fill_(-1)
+        assert pool.gather_packed(plan, lo, hi, table.data_ptr(), w.vocab, out.data_ptr(), cu.data_ptr(), pos.data_ptr(), st) == 0
+        torch.cuda.synchronize()
+        q0, q1 = int(exp["mb_sample_off"][lo]), int(exp["mb_sample_off"][hi])
+        n_rows = int(mb_row[hi] - mb_row[lo])
+        exp_pos = np.concatenate([np.arange(l, dtype=np.int32) for l in lens[q0:q1]])
+        assert np.array_equal(pos[:n_rows].cpu().numpy(), exp_pos)
+        exp_cu = np.concatenate([np.concatenate([[0], np.cumsum(lens[int(exp["mb_sample_off"][j]):int(exp["mb_sample_off"][j + 1])])])
+                                 for j in range(lo, hi)]).astype(np.int32)
+        assert np.array_equal(cu[:len(exp_cu)].cpu().numpy(), exp_cu)
+        assert not bool((out[:n_rows] == -1).all(dim=1).any().item())
+        picks = []
+        for q in rng.choice(np.arange(q0, q1), size=min(6, q1 - q0), replace=False):
+            s = int(exp["mb_samples"][q])
+            sp, tk = w.spans_of(s)
+            for p in {0, int(lens[q]) - 1, int(sp[0]), int(sp[0]) + int(tk[0]) - 1, int(rng.integers(0, lens[q]))}:
+                picks.append((int(row_off[q] - mb_row[lo]) + p, s, p))
+        got_rows = out[torch.tensor([r for r, _, _ in picks], device="cuda")].cpu().numpy().view(np.uint16)
+        for i, (_, s, p) in enumerate(picks):
+            assert np.array_equal(got_rows[i], expected_row(w, s, p)), (lo, hi, s, p)
+    assert pool.status() == (0, 0)
+    plan.destroy(); oplan.destroy()
+    pool.destroy()
