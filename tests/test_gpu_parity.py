@@ -514,3 +514,41 @@ def test_rank_lists_match_oracle(name, kw):
     assert r.pool.gather_list(plan, [0], *args) == pool.gather_list(oplan, [0], bits16(table), oout, ocu, opos) == -5
     oplan.destroy(); pool.destroy()
     r.close()
+
+
+def test_library_limits_at_their_edges():
+    """The largest row the assembly accepts (hidden 18432 over 4 KiB pages: a row touches up to 10 pages), one
+    column more (CAPACITY, nothing written), the largest budget the planner accepts (2^20 - 1) and one more."""
+    gh = _gpu()
+    fp = gh.fp
+    w = workloads.make_workload("tiny", n_samples=3, hidden=18432, page_bytes=4096)
+    got = gh.run_cuda(w)
+    exp = oracle_from_device_sources(w, got["srcs"], got["table"])
+    assert_same(got, exp)
+    w2 = workloads.make_workload("tiny", n_samples=2, hidden=18440, page_bytes=4096)
+    r = gh.CudaRun(w2)
+    r.run_schedule()
+    rc, plan = r.plan()
+    assert rc == 0
+    rc, out, cu, pos = r.gather_all(table=torch.zeros((w2.vocab, w2.hidden), dtype=torch.bfloat16, device="cuda"))
+    assert rc == -11 and bool((out == -1).all().item())
+    lst_rc = r.pool.gather_list(plan, [0], r.table.data_ptr(), w2.vocab, out.data_ptr(), cu.data_ptr(), pos.data_ptr(), gh.cuda_stream())
+    assert lst_rc == -11
+    r.close()
+    # planner budgets
+    w3 = workloads.make_workload("tiny", n_samples=8, hidden=64, page_bytes=4096)
+    r = gh.CudaRun(w3)
+    r.run_schedule()
+    lens = w3.seq_len[w3.plan_order]
+    for L, want in (((1 << 20) - 1, 0), (1 << 20, -11)):
+        cfg = dict(coef_A=3, coef_B=1, budget_L=L, n_buckets_K=2, n_ranks_N=3, flags=0)
+        rc, gp = r.pool.plan_microbatches(np.asarray(w3.plan_order, np.uint32), fp.PlanConfig(**cfg), gh.cuda_stream())
+        assert rc == want
+        if rc == 0:
+            rc2, op = plan_from_lengths(lens, PlanConfig(**cfg), slots=w3.plan_order)
+            ga, oa = gp.arrays(), op.arrays()
+            for k in PLAN_KEYS:
+                assert np.array_equal(ga[k], oa[k]), k
+            assert ga["n_mb"] == 1
+            gp.destroy(); op.destroy()
+    r.close()
