@@ -521,17 +521,6 @@ __global__ void __launch_bounds__(kHotThreads) k_embed_grad_hot(HotArgs a, uint3
   async_wait_pending<0>();
 }
 
-// a plan dies with any of its samples (freed, or never completed under ALLOW_UNWRITTEN)
-static int32_t plan_alive(const ft_pool* p, const ft_plan* pl) {
-  if (pl->free_epoch != p->free_epoch || (pl->cfg.flags & FT_PLAN_ALLOW_UNWRITTEN)) {
-    for (uint32_t t = 0; t < pl->n; ++t) {
-      const ft_slot_mirror& s = p->slots[pl->slots[t]];
-      if (s.state != FT_SLOT_READY || s.generation != pl->slot_generation[t]) return FT_ERR_NOT_READY;
-    }
-  }
-  return FT_OK;
-}
-
 static LayoutArgs layout_of(const ft_plan* pl, uint32_t mb_begin, uint32_t mb_end, bool padded) {
   LayoutArgs a;
   a.mb_begin = mb_begin; a.mb_end = mb_end;

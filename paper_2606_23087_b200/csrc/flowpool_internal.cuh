@@ -201,6 +201,9 @@ inline PlanView make_plan_view(const ft_plan* pl) {
   pv.mb_row_off = pl->d_mb_row_off; pv.tile_first_sample = pl->d_tile_first_sample;
   return pv;
 }
+// A plan dies with any of its samples (freed, or never completed under ALLOW_UNWRITTEN): FT_OK while every sample
+// of the plan is READY in the generation the plan was made for, else FT_ERR_NOT_READY.
+inline int32_t plan_alive(const ft_pool* p, const ft_plan* pl);
 int32_t cuda_fail(cudaError_t e, const char* what);
 #define FT_CUDA(call)                                          \
   do {                                                         \
@@ -350,6 +353,15 @@ inline int32_t begin_free(ft_pool* p, cudaStream_t st) {
 inline int32_t end_producer(ft_pool* p, cudaStream_t st) {
   FT_CUDA(cudaEventRecord(p->ev_producer, st));
   p->have_producer_ev = true; p->last_producer_stream = st;
+  return FT_OK;
+}
+inline int32_t plan_alive(const ft_pool* p, const ft_plan* pl) {
+  if (pl->free_epoch != p->free_epoch || (pl->cfg.flags & FT_PLAN_ALLOW_UNWRITTEN)) {
+    for (uint32_t t = 0; t < pl->n; ++t) {
+      const ft_slot_mirror& s = p->slots[pl->slots[t]];
+      if (s.state != FT_SLOT_READY || s.generation != pl->slot_generation[t]) return FT_ERR_NOT_READY;
+    }
+  }
   return FT_OK;
 }
 }  // namespace ft

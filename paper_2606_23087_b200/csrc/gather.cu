@@ -347,12 +347,9 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_gather_packed(ft_
   if (!p || !pl || pl->pool != p) return FT_ERR_INVALID_ARG;
   p->call_seq++;
   if (mb_begin > mb_end || mb_end > pl->n_mb) return FT_ERR_INVALID_ARG;
-  // a plan dies with any of its samples (freed, or never completed under ALLOW_UNWRITTEN)
-  if (pl->free_epoch != p->free_epoch || (pl->cfg.flags & FT_PLAN_ALLOW_UNWRITTEN)) {
-    for (uint32_t t = 0; t < pl->n; ++t) {
-      const ft_slot_mirror& s = p->slots[pl->slots[t]];
-      if (s.state != FT_SLOT_READY || s.generation != pl->slot_generation[t]) return FT_ERR_NOT_READY;
-    }
+  {
+    const int32_t alive = plan_alive(p, pl);
+    if (alive != FT_OK) return alive;
   }
   if (mb_begin == mb_end) return FT_OK;
   if (!embed_table || !out_embeds || !out_cu || !out_pos) return FT_ERR_INVALID_ARG;
@@ -379,11 +376,9 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_gather_list(ft_po
   p->call_seq++;
   for (uint32_t i = 0; i < n_list; ++i)
     if (mb_list[i] >= pl->n_mb) return FT_ERR_INVALID_ARG;
-  if (pl->free_epoch != p->free_epoch || (pl->cfg.flags & FT_PLAN_ALLOW_UNWRITTEN)) {
-    for (uint32_t t = 0; t < pl->n; ++t) {
-      const ft_slot_mirror& s = p->slots[pl->slots[t]];
-      if (s.state != FT_SLOT_READY || s.generation != pl->slot_generation[t]) return FT_ERR_NOT_READY;
-    }
+  {
+    const int32_t alive = plan_alive(p, pl);
+    if (alive != FT_OK) return alive;
   }
   if (n_list == 0) return FT_OK;
   if (!embed_table || !out_embeds || !out_cu || !out_pos) return FT_ERR_INVALID_ARG;
