@@ -343,6 +343,23 @@ int32_t pool_take_ready(ft_pool* pool, uint64_t min_tokens, uint32_t max_samples
  *                     CAPACITY: a sample exceeds this pool's limits or the list blocks run out.  Asynchronous.
  */
 int32_t pool_backing(ft_pool* pool, void** hbm_base, void** host_base_device, void** text_base);
+
+/*
+ * Peers in other processes of the same node.  pool_ipc_export fills shareable handles (CUDA IPC) of the HBM slab
+ * and the text frames this pool allocated (INVALID_ARG for a caller-owned HBM slab: share that yourself);
+ * pool_ipc_open, called in the consumer's process, maps them and returns the base addresses to hand to
+ * pool_import_mapping; pool_ipc_close unmaps them (after the imported samples were freed).  The handle bytes travel
+ * by any host channel, next to the mapping blob.  Host-tier pages of another process are reached through a
+ * pointer the caller provides (shared host memory registered with the device); these calls do not cover them.
+ */
+#define FT_IPC_HANDLE_BYTES 64
+typedef struct {
+  uint8_t hbm[FT_IPC_HANDLE_BYTES], text[FT_IPC_HANDLE_BYTES];
+  uint32_t has_hbm, has_text;
+} ft_ipc_handles;
+int32_t pool_ipc_export(ft_pool* pool, ft_ipc_handles* out);
+int32_t pool_ipc_open(const ft_ipc_handles* in, void** hbm_base, void** text_base);
+int32_t pool_ipc_close(void* hbm_base, void* text_base);
 int32_t pool_export_mapping(ft_pool* pool, void* buf /* host */, uint64_t cap, uint64_t* bytes);
 int32_t pool_import_mapping(ft_pool* pool, const void* buf /* host */, uint64_t bytes, void* peer_hbm_base,
                             void* peer_host_base, void* peer_text_base);

@@ -26,7 +26,7 @@ EXPORTS = (
     "pool_create", "pool_register_samples", "pool_write_embeddings", "pool_write_embeddings_noalloc",
     "pool_plan_microbatches", "plan_summary",
     "plan_arrays", "plan_destroy", "pool_gather_packed", "pool_gather_list", "pool_set_span_grids", "pool_gather_padded", "pool_embed_grad", "pool_free", "pool_status", "pool_stats",
-    "pool_ready_count", "pool_take_ready", "pool_backing", "pool_export_mapping", "pool_import_mapping", "pool_export_samples", "pool_import_samples",
+    "pool_ready_count", "pool_take_ready", "pool_backing", "pool_ipc_export", "pool_ipc_open", "pool_ipc_close", "pool_export_mapping", "pool_import_mapping", "pool_export_samples", "pool_import_samples",
     "pool_profile_enable", "pool_profile_read", "pool_debug_span_pages", "pool_debug_ring", "pool_debug_translate", "pool_destroy", "flowpool_last_cuda_error",
 )
 
@@ -71,6 +71,21 @@ class KernelTime(C.Structure):
 
 KERNEL_CLASSES = ("gather_device", "gather_host", "scatter_device", "scatter_host", "embed_grad")
 
+IPC_HANDLES_BYTES = 2 * 64 + 8   # ft_ipc_handles
+
+
+def ipc_open(handles: bytes):
+    """Maps a peer process's slabs into this process: (rc, hbm_base, text_base)."""
+    buf = (C.c_uint8 * IPC_HANDLES_BYTES).from_buffer_copy(handles)
+    a, b = C.c_void_p(), C.c_void_p()
+    rc = lib().pool_ipc_open(buf, C.byref(a), C.byref(b))
+    return rc, a.value or 0, b.value or 0
+
+
+def ipc_close(hbm_base: int, text_base: int):
+    return lib().pool_ipc_close(hbm_base or None, text_base or None)
+
+
 _lib = None
 
 
@@ -106,6 +121,9 @@ def lib():
             "pool_import_mapping": [P, P, u64, P, P, P],
             "pool_export_samples": [P, P, u32, P, u64, P, P],
             "pool_import_samples": [P, P, u32, P, u64, P],
+            "pool_ipc_export": [P, P],
+            "pool_ipc_open": [P, P, P],
+            "pool_ipc_close": [P, P],
             "pool_profile_enable": [P, i32],
             "pool_profile_read": [P, P],
             "pool_debug_span_pages": [P, u32, u32, P, u32, P],
@@ -270,6 +288,12 @@ class Pool:
         if rc:
             raise FlowpoolError(rc, "pool_backing")
         return a.value or 0, b.value or 0, c.value or 0
+
+    def ipc_export(self):
+        """Shareable handles (bytes) of this pool's HBM slab and text frames, for a consumer in another process."""
+        buf = (C.c_uint8 * IPC_HANDLES_BYTES)()
+        rc = lib().pool_ipc_export(self.h, buf)
+        return rc, bytes(buf)
 
     def export_mapping(self):
         n = C.c_uint64()

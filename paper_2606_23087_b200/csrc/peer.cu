@@ -124,6 +124,54 @@ FT_API int32_t pool_backing(ft_pool* p, void** hbm_base, void** host_base_device
   return FT_OK;
 }
 
+// Shareable handles of this pool's device slabs for a consumer in another process on the same node (Sec. 3.2:
+// every process can address every other process's segment).  Only slabs the library allocated itself have a handle
+// of their own; a caller-owned HBM slab is the caller's to share.
+FT_API int32_t pool_ipc_export(ft_pool* p, ft_ipc_handles* out) {
+  if (!p || !out) return FT_ERR_INVALID_ARG;
+  static_assert(sizeof(cudaIpcMemHandle_t) == FT_IPC_HANDLE_BYTES, "handle size");
+  memset(out, 0, sizeof(*out));
+  if (p->cfg.hbm_pages) {
+    if (!p->own_hbm) return FT_ERR_INVALID_ARG;
+    cudaIpcMemHandle_t h;
+    FT_CUDA(cudaIpcGetMemHandle(&h, p->hbm_base));
+    memcpy(out->hbm, &h, sizeof(h));
+    out->has_hbm = 1;
+  }
+  cudaIpcMemHandle_t t;
+  FT_CUDA(cudaIpcGetMemHandle(&t, p->d_text));
+  memcpy(out->text, &t, sizeof(t));
+  out->has_text = 1;
+  return FT_OK;
+}
+
+// Maps a peer process's slabs into this process: the base addresses pool_import_mapping wants.
+FT_API int32_t pool_ipc_open(const ft_ipc_handles* in, void** hbm_base, void** text_base) {
+  if (!in || !hbm_base || !text_base) return FT_ERR_INVALID_ARG;
+  *hbm_base = nullptr; *text_base = nullptr;
+  if (in->has_hbm) {
+    cudaIpcMemHandle_t h;
+    memcpy(&h, in->hbm, sizeof(h));
+    FT_CUDA(cudaIpcOpenMemHandle(hbm_base, h, cudaIpcMemLazyEnablePeerAccess));
+  }
+  if (in->has_text) {
+    cudaIpcMemHandle_t t;
+    memcpy(&t, in->text, sizeof(t));
+    const cudaError_t e = cudaIpcOpenMemHandle(text_base, t, cudaIpcMemLazyEnablePeerAccess);
+    if (e != cudaSuccess) {
+      if (*hbm_base) { cudaIpcCloseMemHandle(*hbm_base); *hbm_base = nullptr; }
+      return cuda_fail(e, "cudaIpcOpenMemHandle(text)");
+    }
+  }
+  return FT_OK;
+}
+
+FT_API int32_t pool_ipc_close(void* hbm_base, void* text_base) {
+  if (hbm_base) FT_CUDA(cudaIpcCloseMemHandle(hbm_base));
+  if (text_base) FT_CUDA(cudaIpcCloseMemHandle(text_base));
+  return FT_OK;
+}
+
 FT_API int32_t pool_export_mapping(ft_pool* p, void* buf, uint64_t cap, uint64_t* bytes) {
   if (!p) return FT_ERR_INVALID_ARG;
   const uint64_t need = sizeof(MapHeader) + 4 * (p->cfg.hbm_pages + p->cfg.host_pages);
