@@ -276,6 +276,9 @@ def test_full_size_fragmentation_sweep(page_bytes):
     from gpu_harness import cuda_stream
     from harness import pool_config_fields, register_args, write_args
     from paper_2606_23087_b200 import binding as fp
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()          # blocks cached by earlier tests of this process are not in use
     free_b, _ = torch.cuda.mem_get_info()
     pool_bytes = (64 << 30) if free_b >= (90 << 30) else (32 << 30)
     w = workloads.make_workload("frag_sweep", n_samples=65536, page_bytes=page_bytes, pool_bytes=pool_bytes)
@@ -307,7 +310,7 @@ def test_full_size_fragmentation_sweep(page_bytes):
     for k in PLAN_KEYS:
         assert np.array_equal(got[k], exp[k]), k
     n_mb, total, _ = plan.summary()
-    assert (n_mb, total) == oplan.summary()[:2] and len(residents) > 8000
+    assert (n_mb, total) == oplan.summary()[:2] and len(residents) > (8000 if pool_bytes == (64 << 30) else 4000)
     table = workloads.embed_table(w, device="cuda")
     buf_rows = min(total, 1 << 20)
     out = torch.empty((buf_rows, w.hidden), dtype=torch.int16, device="cuda")
