@@ -417,7 +417,7 @@ int32_t pool_gather_padded(ft_pool* pool, const ft_plan* plan, uint32_t mb_begin
  *   grad_out    device bf16 [rows, H], 16-byte aligned
  *   grad_table  device fp32 [vocab, H], 16-byte aligned, accumulated in place
  * Errors: as pool_gather_packed; asynchronous: id outside [0, vocab) BAD_TOKEN_ID (row skipped).  Allocates
- * stream-ordered scratch for the call (about 16 bytes per row plus 8 bytes per table row).  Ids that own many
+ * stream-ordered scratch for the call (about 24 bytes per row plus 8 bytes per table row).  Ids that own many
  * rows are added by a separate kernel on the pool's second consumer-side stream; the call returns with `stream`
  * ordered after both.
  */
