@@ -276,9 +276,12 @@ struct ft_pool {
   int sm_count = 148;
   int occ_scatter[3][2] = {};   // resident CTAs/SM of k_scatter<tier mode, f32>, from the occupancy API
   int occ_gather[3][2] = {};    // resident CTAs/SM of k_gather<tier mode, U = 4 | 8>
-  int host_ctas = 8;            // grid of the host-tier copy kernels: few SMs, so that long-latency host-link
-                                // accesses do not clog the memory pipelines of the SMs that stream HBM
-                                // (FLOWPOOL_HOST_CTAS overrides)
+  int host_ctas = 6;            // grid of the host-tier bulk-copy kernels: few SMs, so that long-latency host-link
+                                // accesses do not clog the memory pipelines of the SMs that stream HBM; 6 rather
+                                // than 8 because a write and a read kernel running together (two streams) share
+                                // the link better with fewer requests in flight (FLOWPOOL_HOST_CTAS overrides)
+  int host_store_ctas = 8;      // grid of the vector-store scatter into host frames (fp32 sources, host-only pools;
+                                // FLOWPOOL_HOST_STORE_CTAS overrides)
   int chunk_shift = 16;         // log2 of k_scatter's work unit in bytes of a span's image (14..21)
   int scatter_group = 0;        // chunks per round-robin group of k_scatter; 0 = the measured default
   int scatter_ctas_per_sm = 0;  // resident CTAs per SM of the device-tier scatter kernel; 0 = the measured default

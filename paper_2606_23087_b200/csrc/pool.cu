@@ -602,8 +602,9 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_create(const ft_p
   } while (0)
   CK(cudaGetDevice(&p->device));
   CK(cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, p->device));
-  p->host_ctas = 8;
+  p->host_ctas = 6;
   if (const char* e = getenv("FLOWPOOL_HOST_CTAS")) { int v = atoi(e); if (v > 0) p->host_ctas = v; }
+  if (const char* e = getenv("FLOWPOOL_HOST_STORE_CTAS")) { int v = atoi(e); if (v > 0) p->host_store_ctas = v; }
   // A warp's region is 1/8 of a chunk and must hold at least one 2 KiB batch.
   if (const char* e = getenv("FLOWPOOL_CHUNK_SHIFT")) { int v = atoi(e); if (v >= 14 && v <= 21) p->chunk_shift = v; }
   if (const char* e = getenv("FLOWPOOL_SCATTER_GROUP")) { int v = atoi(e); if (v > 0) p->scatter_group = v; }
@@ -916,7 +917,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings(
   auto launch = [&](int mode, cudaStream_t s) {
     const bool host_class = mode == kTierHostOnly || (mode == kTierAll && c.hbm_pages == 0);
     prof_begin(p, host_class ? FT_K_SCATTER_HOST : FT_K_SCATTER_DEVICE, s);
-    launch_scatter_any(p, mode, f32, w, total_chunks, host_class ? (uint64_t)p->host_ctas : ~0ull, s);
+    launch_scatter_any(p, mode, f32, w, total_chunks, host_class ? (uint64_t)p->host_store_ctas : ~0ull, s);
     prof_end(p, s);
     p->gpu_launches++;
   };
@@ -931,7 +932,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings(
     // bf16 source: bulk-async copies through shared memory.  fp32 source: the cast needs the values in
     // registers, and stores to host memory are posted (no latency to hide), so a few vector-store CTAs do it
     if (f32) {
-      launch_scatter<kTierHostOnly, true>(p, w, total_chunks, (uint64_t)p->host_ctas, p->side_stream[0]);
+      launch_scatter<kTierHostOnly, true>(p, w, total_chunks, (uint64_t)p->host_store_ctas, p->side_stream[0]);
     } else {
       k_scatter_host_bulk<<<(unsigned)p->host_ctas, 32, kBulkSmemBytes, p->side_stream[0]>>>(p->view, w, p->call_seq);
     }
@@ -1278,7 +1279,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings_
   const bool f32 = src_dtype == FT_F32;
   auto launch = [&](int mode, cudaStream_t s) {
     const bool host_class = mode == kTierAll && c.hbm_pages == 0;
-    launch_scatter_any(p, mode, f32, w, total_chunks, host_class ? (uint64_t)p->host_ctas : ~0ull, s);
+    launch_scatter_any(p, mode, f32, w, total_chunks, host_class ? (uint64_t)p->host_store_ctas : ~0ull, s);
     p->gpu_launches++;
   };
   if (c.host_pages == 0 || c.hbm_pages == 0) {
@@ -1287,7 +1288,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings_
     FT_CUDA(cudaEventRecord(p->fork_ev[0], st));
     FT_CUDA(cudaStreamWaitEvent(p->side_stream[0], p->fork_ev[0], 0));
     if (f32) {
-      launch_scatter<kTierHostOnly, true>(p, w, total_chunks, (uint64_t)p->host_ctas, p->side_stream[0]);
+      launch_scatter<kTierHostOnly, true>(p, w, total_chunks, (uint64_t)p->host_store_ctas, p->side_stream[0]);
     } else {
       k_scatter_host_bulk<<<(unsigned)p->host_ctas, 32, kBulkSmemBytes, p->side_stream[0]>>>(p->view, w, p->call_seq);
     }
