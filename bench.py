@@ -1021,6 +1021,136 @@ def run_streaming(args, all_hbm, batches=6, warm=2):
 # ---------------------------------------------------------------------------------------------
 # two processes of one GVA space, emulated on one GPU: producer pool (rank 1) -> consumer pool (rank 0)
 # ---------------------------------------------------------------------------------------------
+def _peer_producer_process(args_dict, to_parent, from_parent):
+    """The producer of --via-peer --two-processes: owns rank 1's pool in a process of its own."""
+    import torch
+    import workloads
+    from harness import pool_config_fields, register_args, write_args
+    from paper_2606_23087_b200 import binding as fp
+    try:
+        torch.cuda.set_device(0)
+        st = torch.cuda.current_stream().cuda_stream
+        w = workloads.make_workload(args_dict["workload"], n_samples=args_dict["samples"], all_hbm=True)
+        f = pool_config_fields(w, max_samples=w.n_samples)
+        f.update(world_size=2, rank=1)
+        prod = fp.Pool(fp.PoolConfig(**f))
+        assert prod.rc == 0
+        calls = []
+        for call in w.write_calls:
+            samples = sorted({s for s, _ in call}, key=[s for s, _ in call].index)
+            reg = register_args(w, samples)
+            calls.append((reg[:5], torch.from_numpy(reg[5]).cuda(), write_args(w, call),
+                          [workloads.span_values(w, s, j, device="cuda") for s, j in call]))
+        order = np.asarray(w.plan_order, dtype=np.uint32)
+        rc, mblob = prod.export_mapping()
+        rc2, handles = prod.ipc_export()
+        assert rc == 0 and rc2 == 0
+        to_parent.put(("mapping", mblob.tobytes(), handles))
+        while True:
+            cmd = from_parent.get(timeout=600)
+            if cmd == "write":
+                for reg, ids, wr, srcs in calls:
+                    assert prod.register_samples(*reg, ids.data_ptr(), st) == 0
+                    assert prod.write_embeddings(*wr, [t.data_ptr() for t in srcs], w.src_dtype, st) == 0
+                rc, sblob = prod.export_samples(order, st)    # synchronises the stream: the pages are written
+                assert rc == 0
+                to_parent.put(("samples", sblob.tobytes()))
+            elif cmd == "free":
+                assert prod.free(order, st) == 0
+                torch.cuda.synchronize()
+                to_parent.put(("freed",))
+            else:
+                break
+        assert prod.status() == (0, 0)
+        prod.destroy()
+        to_parent.put(("bye",))
+    except BaseException as e:
+        to_parent.put(("error", repr(e)))
+        raise
+
+
+def run_peer_two_processes(args):
+    """--via-peer with the producer in a process of its own: its slabs reach the consumer through CUDA IPC handles,
+    its mapping and its samples' descriptors through a host queue.  All pages in HBM (host-tier slabs are not shared
+    by these calls).  One GPU: the two processes' segments are in the same HBM."""
+    import multiprocessing as mp
+    import torch
+    import workloads
+    from harness import pool_config_fields, plan_config_fields
+    from paper_2606_23087_b200 import binding as fp
+    torch.cuda.set_device(0)
+    st = torch.cuda.current_stream().cuda_stream
+    w = workloads.make_workload(args.workload, n_samples=args.samples, all_hbm=True)
+    n = w.n_samples
+    ctx = mp.get_context("spawn")
+    to_child, from_child = ctx.Queue(), ctx.Queue()
+    child = ctx.Process(target=_peer_producer_process, args=({"workload": args.workload, "samples": args.samples}, from_child, to_child),
+                        daemon=True)
+    child.start()
+    try:
+        f = pool_config_fields(w, max_samples=n)
+        f.update(world_size=2, rank=0, hbm_pages=64, host_pages=0, max_imported_pages=w.hbm_pages + w.host_pages)
+        cons = fp.Pool(fp.PoolConfig(**f))
+        assert cons.rc == 0
+        msg = from_child.get(timeout=600)
+        assert msg[0] == "mapping", msg
+        rc, hbm, text = fp.ipc_open(msg[2])
+        assert rc == 0 and cons.import_mapping(np.frombuffer(msg[1], np.uint8), hbm, 0, text) == 0
+        table = workloads.embed_table(w, device="cuda")
+        out = torch.empty((w.total_tokens, w.hidden), dtype=torch.bfloat16, device="cuda")
+        cu = torch.empty((2 * n + 8,), dtype=torch.int32, device="cuda")
+        pos = torch.empty((w.total_tokens,), dtype=torch.int32, device="cuda")
+        order = np.asarray(w.plan_order, dtype=np.uint32)
+        pcfg = fp.PlanConfig(**plan_config_fields(w))
+        cons.profile_enable(True)
+        n_mb, blob_bytes, xfer_ms = 0, 0, []
+        for it in range(args.warmup + args.steps):
+            to_child.put("write")
+            msg = from_child.get(timeout=600)
+            assert msg[0] == "samples", msg
+            t0 = time.perf_counter()
+            sblob = np.frombuffer(msg[1], np.uint8)
+            assert cons.import_samples(order, sblob, st) == 0
+            torch.cuda.synchronize()
+            xfer_ms.append((time.perf_counter() - t0) * 1e3)
+            rc, plan = cons.plan_microbatches(order, pcfg, st)
+            assert rc == 0
+            n_mb = plan.summary()[0]
+            if it == args.warmup:
+                cons.profile_read()
+            assert cons.gather_packed(plan, 0, n_mb, table.data_ptr(), w.vocab, out.data_ptr(), cu.data_ptr(), pos.data_ptr(), st) == 0
+            assert cons.free(order, st) == 0
+            plan.destroy()
+            torch.cuda.synchronize()
+            to_child.put("free")
+            assert from_child.get(timeout=600)[0] == "freed"
+            blob_bytes = len(sblob)
+        prof = cons.profile_read()
+        assert cons.status() == (0, 0)
+        # spot-check a few rows against the generator: text rows of the first sample
+        ids0 = workloads.input_ids(w, int(order[0]))
+        row = int(np.nonzero(ids0 != w.placeholder_id)[0][0])
+        ok = bool(torch.equal(out[row], table[int(ids0[row])]))
+        cons.destroy()
+        assert fp.ipc_close(hbm, text) == 0
+        to_child.put("quit")
+        assert from_child.get(timeout=600)[0] == "bye"
+        child.join(timeout=60)
+    finally:
+        if child.is_alive():
+            child.kill()   # this very process object
+    g_ms = prof["gather_device"]["ms"] / args.steps
+    peak, _ = measured_peak()
+    gbs = 2 * w.total_tokens * w.row_bytes / g_ms / 1e6
+    args.all_hbm = True
+    label = workload_label(args)
+    print(json.dumps({"metric": "packed-microbatch assembly GB/s, consumer process reading a producer process's pages (CUDA IPC, one GPU)",
+                      "value": gbs, "unit": "GB/s", "n_gpus": 1, "higher_is_better": True, "dtype": "u8", "data": "synthetic",
+                      "config": {"workload": label, "processes": 2, "note": "both segments in the same HBM"},
+                      "gather_device_ms": g_ms, "frac_of_measured_peak": gbs / peak, "descriptor_import_ms": float(np.median(xfer_ms[args.warmup:])),
+                      "descriptor_blob_bytes": blob_bytes, "microbatches": n_mb, "sampled_row_matches": ok}))
+
+
 def run_peer(args):
     """The producer writes the batch into its own segment; the consumer imports its mapping (once) and, per step,
     the samples' descriptors, plans, and assembles every microbatch by reading the producer's pages in place.
@@ -1114,6 +1244,7 @@ def main():
     ap.add_argument("--cycles", type=int, default=10, help="frag_sweep: write/free cycles")
     ap.add_argument("--id-skew", default="uniform", choices=["uniform", "zipf"], help="distribution of the text-token ids")
     ap.add_argument("--backbone-only", action="store_true", help="only the backbone-side outputs (padded assembly, table gradient) on an all-HBM pool")
+    ap.add_argument("--two-processes", action="store_true", help="with --via-peer: the producer pool lives in a process of its own (CUDA IPC)")
     ap.add_argument("--via-peer", action="store_true", help="producer and consumer are two processes' pools of one GVA space")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -1123,6 +1254,8 @@ def main():
         run_sweep(args)
     elif args.backbone_only:
         run_backbone_only(args)
+    elif args.via_peer and args.two_processes:
+        run_peer_two_processes(args)
     elif args.via_peer:
         run_peer(args)
     else:
