@@ -1151,6 +1151,143 @@ def run_peer_two_processes(args):
                       "descriptor_blob_bytes": blob_bytes, "microbatches": n_mb, "sampled_row_matches": ok}))
 
 
+def run_exchange(args):
+    """The paper's own setting (Sec. 3.2, 3.4) with one process per rank: every rank writes its batch into its own
+    segment; mappings and slab handles are exchanged once, the samples' descriptors every step; every rank plans ALL
+    samples (Algorithm 1 is deterministic, so the plans agree) and assembles only the microbatches dealt to it,
+    reading the other ranks' pages in place (peer loads over NVLink when the ranks own different GPUs).  All pages
+    in HBM.  Launch under torchrun; FLOWPOOL_BENCH_BACKEND=gloo runs several ranks on one GPU (their kernels never
+    wait on one another), which is how this mode is exercised where only one GPU is at hand."""
+    import torch
+    import torch.distributed as dist
+    import workloads
+    from harness import pool_config_fields, plan_config_fields, register_args, write_args
+    from paper_2606_23087_b200 import binding as fp
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0")) % max(1, torch.cuda.device_count())
+    torch.cuda.set_device(local)
+    backend = os.environ.get("FLOWPOOL_BENCH_BACKEND", "nccl")
+    if backend == "nccl":
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    else:
+        dist.init_process_group(backend)
+    st = torch.cuda.current_stream().cuda_stream
+    w = workloads.make_workload(args.workload, n_samples=args.samples, all_hbm=True)
+    n = w.n_samples
+    f = pool_config_fields(w, max_samples=world * n)
+    f.update(world_size=world, rank=rank, bind_seed=100 + rank, ring_seed=200 + rank,
+             max_imported_pages=(world - 1) * (w.hbm_pages + w.host_pages), max_text_tokens=world * w.total_text_tokens_capacity)
+    pool = fp.Pool(fp.PoolConfig(**f))
+    assert pool.rc == 0, pool.rc
+    # once: everybody's mapping and slab handles
+    rc1, mblob = pool.export_mapping()
+    rc2, handles = pool.ipc_export()
+    assert rc1 == 0 and rc2 == 0
+    everyone = [None] * world
+    dist.all_gather_object(everyone, (mblob.tobytes(), handles))
+    opened = []
+    for r, (mb, hd) in enumerate(everyone):
+        if r == rank:
+            continue
+        rc, hbm, text = fp.ipc_open(hd)
+        assert rc == 0, rc
+        opened.append((hbm, text))
+        assert pool.import_mapping(np.frombuffer(mb, np.uint8), hbm, 0, text) == 0
+    # own batch: global sample g = rank * n + s lives in slot g on every rank
+    calls = []
+    for call in w.write_calls:
+        samples = sorted({s for s, _ in call}, key=[s for s, _ in call].index)
+        reg = register_args(w, samples)
+        slots = (np.asarray(reg[0], np.uint32) + rank * n).astype(np.uint32)
+        wr = write_args(w, call)
+        calls.append(((slots,) + tuple(reg[1:5]), torch.from_numpy(reg[5]).cuda(),
+                      ((np.asarray(wr[0], np.uint32) + rank * n).astype(np.uint32),) + tuple(wr[1:]),
+                      [workloads.span_values(w, s, j, device="cuda") for s, j in call]))
+    own = (np.asarray(w.plan_order, np.uint32) + rank * n).astype(np.uint32)
+    order = np.concatenate([(np.asarray(w.plan_order, np.uint32) + r * n) for r in range(world)]).astype(np.uint32)
+    pc = plan_config_fields(w)
+    pc["n_ranks_N"] = world
+    pcfg = fp.PlanConfig(**pc)
+    table = workloads.embed_table(w, device="cuda")
+    cap_rows = int(w.total_tokens * 1.5) + w.budget_L
+    out = torch.empty((cap_rows, w.hidden), dtype=torch.bfloat16, device="cuda")
+    cu = torch.empty((2 * world * n + 8,), dtype=torch.int32, device="cuda")
+    pos = torch.empty((cap_rows,), dtype=torch.int32, device="cuda")
+    step_ms, my_rows, n_mb = [], 0, 0
+    for it in range(args.warmup + args.steps):
+        dist.barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for reg, ids, wr, srcs in calls:
+            assert pool.register_samples(*reg, ids.data_ptr(), st) == 0
+            assert pool.write_embeddings(*wr, [t.data_ptr() for t in srcs], w.src_dtype, st) == 0
+        rc, sblob = pool.export_samples(own, st)          # synchronises: this rank's pages are written
+        assert rc == 0
+        blobs = [None] * world
+        dist.all_gather_object(blobs, sblob.tobytes())    # the per-round exchange of "lightweight metadata"
+        for r in range(world):
+            if r != rank:
+                theirs = (np.asarray(w.plan_order, np.uint32) + r * n).astype(np.uint32)
+                assert pool.import_samples(theirs, np.frombuffer(blobs[r], np.uint8), st) == 0
+        rc, plan = pool.plan_microbatches(order, pcfg, st)
+        assert rc == 0
+        pa = plan.arrays()
+        n_mb = int(pa["n_mb"])
+        mine = [int(j) for j in pa["rank_mbs"][pa["rank_mb_off"][rank]:pa["rank_mb_off"][rank + 1]]]
+        my_rows = int(pa["mb_tokens"][mine].sum()) if mine else 0
+        assert my_rows <= cap_rows
+        if mine:
+            assert pool.gather_list(plan, mine, table.data_ptr(), w.vocab, out.data_ptr(), cu.data_ptr(), pos.data_ptr(), st) == 0
+        e1.record()
+        torch.cuda.synchronize()
+        if mine and it == 0:
+            # spot check against the generator: first and last row of the first sample of this rank's share
+            q0 = int(pa["mb_sample_off"][mine[0]])
+            g = int(pa["mb_samples"][q0])
+            s_local = g % n                                  # every rank generated the same workload
+            ids_s = workloads.input_ids(w, s_local)
+            sp_pos, sp_tok = w.spans_of(s_local)
+            for p_ in (0, len(ids_s) - 1):
+                in_span = [j for j in range(len(sp_pos)) if int(sp_pos[j]) <= p_ < int(sp_pos[j]) + int(sp_tok[j])]
+                if in_span:
+                    j = in_span[0]
+                    want = workloads.span_values(w, s_local, j, device="cuda", rows=(p_ - int(sp_pos[j]), p_ - int(sp_pos[j]) + 1))[0]
+                else:
+                    want = table[int(ids_s[p_])]
+                assert torch.equal(out[p_].view(torch.int16), want.to(torch.bfloat16).view(torch.int16)), (rank, g, p_)
+        for r in range(world):
+            if r != rank:
+                assert pool.free((np.asarray(w.plan_order, np.uint32) + r * n).astype(np.uint32), st) == 0
+        plan.destroy()
+        torch.cuda.synchronize()
+        dist.barrier()                                    # nobody reads this rank's pages any more
+        assert pool.free(own, st) == 0
+        torch.cuda.synchronize()
+        if it >= args.warmup:
+            step_ms.append(e0.elapsed_time(e1))
+    assert pool.status() == (0, 0)
+    ms = float(np.median(step_ms))
+    t = torch.tensor([ms, float(my_rows)], dtype=torch.float64, device="cuda" if backend == "nccl" else "cpu")
+    mx = t.clone(); dist.all_reduce(mx, op=dist.ReduceOp.MAX)
+    sm = t.clone(); dist.all_reduce(sm, op=dist.ReduceOp.SUM)
+    ms_max, rows_all = float(mx[0]), float(sm[1])
+    wb, _ = algorithmic_bytes(w)
+    moved = world * wb + rows_all * 4 * w.hidden
+    pool.destroy()
+    for hbm, text in opened:
+        fp.ipc_close(hbm, text)
+    if rank == 0:
+        print(json.dumps({"metric": METRIC + ", ranks exchanging descriptors and reading each other's pages in place", "value": moved / ms_max / 1e6,
+                          "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_max,
+                          "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+                          "config": {"workload": workload_label(args), "ranks": world, "gpus_used": min(world, torch.cuda.device_count()),
+                                     "backend": backend, "microbatches": n_mb, "packed_tokens_all_ranks": int(rows_all)},
+                          "tokens_per_s": rows_all / ms_max * 1e3}))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
 def run_peer(args):
     """The producer writes the batch into its own segment; the consumer imports its mapping (once) and, per step,
     the samples' descriptors, plans, and assembles every microbatch by reading the producer's pages in place.
@@ -1244,6 +1381,7 @@ def main():
     ap.add_argument("--cycles", type=int, default=10, help="frag_sweep: write/free cycles")
     ap.add_argument("--id-skew", default="uniform", choices=["uniform", "zipf"], help="distribution of the text-token ids")
     ap.add_argument("--backbone-only", action="store_true", help="only the backbone-side outputs (padded assembly, table gradient) on an all-HBM pool")
+    ap.add_argument("--exchange", action="store_true", help="under torchrun: every rank writes its batch, all plan everything, each assembles its own share from everybody's pages")
     ap.add_argument("--two-processes", action="store_true", help="with --via-peer: the producer pool lives in a process of its own (CUDA IPC)")
     ap.add_argument("--via-peer", action="store_true", help="producer and consumer are two processes' pools of one GVA space")
     args = ap.parse_args()
@@ -1254,6 +1392,9 @@ def main():
         run_sweep(args)
     elif args.backbone_only:
         run_backbone_only(args)
+    elif args.exchange:
+        args.all_hbm = True
+        run_exchange(args)
     elif args.via_peer and args.two_processes:
         run_peer_two_processes(args)
     elif args.via_peer:
