@@ -2,7 +2,7 @@
 // of shared-memory stages: global -> shared (completion on an mbarrier), then shared -> global (bulk groups).
 // One thread keeps `kDepth` loads in flight, so a handful of single-warp CTAs saturate a long-latency link
 // (mapped pinned host memory) without tying up the load/store pipelines of the SMs that stream HBM.
-// No cluster multicast anywhere.  Every wait is bounded.
+// Every copy lands in the issuing CTA only.  Every wait is bounded.
 #pragma once
 #include <stdint.h>
 
