@@ -346,6 +346,8 @@ def max_over_ranks(ms, dist, device="cuda"):
     if dist is None:
         return ms
     import torch
+    if dist.get_backend() != "nccl":
+        device = "cpu"
     t = torch.tensor([ms], dtype=torch.float64, device=device)
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     return float(t.item())
@@ -702,11 +704,17 @@ def run_ours(args):
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
+    backend = os.environ.get("FLOWPOOL_BENCH_BACKEND", "nccl")   # gloo: several ranks may share a GPU (checks of this script)
+    if backend != "nccl":
+        local %= max(1, torch.cuda.device_count())
     torch.cuda.set_device(local)
     dist = None
     if world > 1 or "TORCHELASTIC_RUN_ID" in os.environ:   # under torchrun, also at one rank: same code path at every N
         import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        if backend == "nccl":
+            dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        else:
+            dist.init_process_group(backend)
     sampler = ClockSampler(local)
     job = DeviceJob(args, args.all_hbm)
     w = job.w
