@@ -1,9 +1,13 @@
-"""Parity at the benchmark's full size (the 7B image-mix batch, 80 % HBM / 20 % pinned host, as bench.py
-launches it).  The oracle cannot hold this pool in seconds, so: the plan is compared array by array with the
-oracle's Algorithm 1 on the same lengths; cu_seqlens and position ids are compared in full with what the plan
-arrays determine; and sampled output rows are compared with rows the oracle side computes one by one from the
-generator (vision rows: the span's source row, through the oracle's cast when the source is fp32; text rows:
-the table row of the generated id)."""
+"""Parity at the sizes the five configurations name, in the launch configuration bench.py times.
+
+The plan is compared array by array with the oracle's Algorithm 1 on the same lengths; cu_seqlens and position
+ids are compared in full with what the plan arrays determine; and EVERY assembled row is compared, on the device,
+with the row the consumer semantics fix (Sec. 3.1-3.2: a placeholder position reads the span's row through its
+GVA, any other position the table row of its id), rebuilt sample by sample from the seeded generator with plain
+tensor indexing -- no library call on that side.  Where the host has the memory for it, the oracle itself also
+runs once at full size and its whole output is compared.  Sampled rows are still checked one by one against rows
+the oracle side computes (for fp32 sources through the oracle's own cast)."""
+import gc
 import numpy as np
 import pytest
 import torch
@@ -13,6 +17,77 @@ from harness import bits16, bits32, plan_config_fields
 from oracle import PlanConfig, f32_to_bf16_rne, plan_from_lengths
 
 pytestmark = pytest.mark.gpu
+
+def rne_bf16_bits(x_f32):
+    """bf16 bit patterns (int16 tensor) of an fp32 tensor under the write path's rule, in integer arithmetic on
+    the device: round to nearest even on the bit pattern, denormals kept, every NaN -> sign | 0x7FC0.  A test-side
+    restatement used only to cover 100 % of rows at sizes the oracle cannot hold; test_cast_restatement_equals_oracle
+    ties it to the oracle's cast."""
+    u = x_f32.contiguous().view(torch.int32).to(torch.int64) & 0xFFFFFFFF
+    nan = (u & 0x7FFFFFFF) > 0x7F800000
+    r = (u + 0x7FFF + ((u >> 16) & 1)) >> 16
+    r = torch.where(nan, ((u >> 16) & 0x8000) | 0x7FC0, r) & 0xFFFF
+    return torch.where(r >= 0x8000, r - 0x10000, r).to(torch.int16)
+
+
+def expected_sample_rows(w, s, table_i16):
+    """int16 [seq_len, H] on the device: what the assembly of sample s must contain, from the generator alone."""
+    ids = torch.from_numpy(workloads.input_ids(w, s).astype(np.int64)).cuda()
+    exp = table_i16[ids]                       # text rows (rows at placeholder positions are overwritten below)
+    pos, tok = w.spans_of(s)
+    for j in range(len(pos)):
+        v = workloads.span_values(w, s, j, device="cuda")
+        v = v.view(torch.int16) if w.src_dtype == 0 else rne_bf16_bits(v)
+        exp[int(pos[j]):int(pos[j]) + int(tok[j])] = v
+    return exp
+
+
+def assert_every_row(w, out_i16, samples, row_offsets, table_i16):
+    """Compares all rows of `out_i16` that belong to the listed samples (sample k starts at row_offsets[k])."""
+    bad = []
+    for k, s in enumerate(samples):
+        exp = expected_sample_rows(w, int(s), table_i16)
+        r0 = int(row_offsets[k])
+        if not torch.equal(out_i16[r0:r0 + exp.shape[0]], exp):
+            bad.append(int(s))
+    assert not bad, f"{len(bad)} samples differ, first {bad[:5]}"
+    return len(samples)
+
+
+def host_mem_available():
+    try:
+        for line in open("/proc/meminfo"):
+            if line.startswith("MemAvailable:"):
+                return int(line.split()[1]) * 1024
+    except OSError:
+        pass
+    return 0
+
+
+def oracle_full_output(w, srcs_dev, table_dev):
+    """The oracle itself on the whole workload (host copies of the very tensors the device read):
+    (plan arrays, out uint16 [rows, H], cu, pos)."""
+    from harness import pool_config_fields, register_args, write_args
+    from gpu_harness import host_bits
+    from oracle import OraclePool, PoolConfig
+    pool = OraclePool(PoolConfig(**pool_config_fields(w)))
+    assert pool.rc == 0
+    for call in w.write_calls:
+        samples = sorted({s for s, _ in call}, key=[s for s, _ in call].index)
+        assert pool.register_samples(*register_args(w, samples)) == 0
+        assert pool.write_embeddings(*write_args(w, call), [host_bits(srcs_dev[c]) for c in call], w.src_dtype) == 0
+    rc, plan = pool.plan_microbatches(np.asarray(w.plan_order, dtype=np.uint32), PlanConfig(**plan_config_fields(w)))
+    assert rc == 0
+    n_mb, total, _ = plan.summary()
+    out = np.full((total, w.hidden), 0xFFFF, dtype=np.uint16)
+    cu = np.full(len(w.plan_order) + n_mb, -1, dtype=np.int32)
+    pos = np.full(total, -1, dtype=np.int32)
+    assert pool.gather_packed(plan, 0, n_mb, bits16(table_dev), out, cu, pos) == 0
+    assert pool.status() == (0, 0)
+    plan.destroy()
+    pool.destroy()
+    return out, cu, pos
+
 
 PLAN_KEYS = ("mb_sample_off", "mb_samples", "mb_tokens", "mb_lmax", "mb_residual", "mb_cost", "mb_bucket", "mb_rank",
              "rank_mb_off", "rank_mbs", "sample_cost", "sample_mb")
@@ -32,6 +107,41 @@ def expected_row(w, s, p):
     return bits16(workloads.embed_table(w, "cpu", rows=(i, i + 1))).ravel()
 
 
+FULL_ORACLE = {}
+
+
+def test_cast_restatement_equals_oracle():
+    """The integer restatement of the cast that the full-coverage compare uses for fp32 sources, against the oracle:
+    a whole sample of the host-tier-stress workload (special bit patterns included) written and assembled by the
+    oracle, and every special pattern through the oracle's scalar cast."""
+    if not torch.cuda.is_available():
+        pytest.fail("a CUDA device is required for -m gpu tests")
+    from harness import host_span, pool_config_fields
+    from oracle import OraclePool, PoolConfig
+    spec = workloads.special_f32_bits()
+    t = torch.from_numpy(spec.view(np.int32).copy()).cuda().view(torch.float32)
+    assert np.array_equal(rne_bf16_bits(t).cpu().numpy().view(np.uint16),
+                          np.array([f32_to_bf16_rne(int(b)) for b in spec], dtype=np.uint16))
+    w = workloads.make_workload("host_tier_stress", n_samples=3)
+    table = workloads.embed_table(w, device="cuda")
+    for s in (0, 2):
+        f = pool_config_fields(w, max_samples=1)
+        f.update(hbm_pages=w.pages_of_span(int(w.spans_of(s)[1][0])) + 1, host_pages=0)
+        pool = OraclePool(PoolConfig(**f))
+        assert pool.rc == 0
+        pos, tok = w.spans_of(s)
+        assert pool.register_samples([0], [int(w.seq_len[s])], [1], pos, tok, workloads.input_ids(w, s)) == 0
+        assert pool.write_embeddings([0], [0], tok, [host_span(w, s, 0)], 1) == 0
+        rc, plan = pool.plan_microbatches([0], PlanConfig(**plan_config_fields(w)))
+        assert rc == 0
+        n = int(w.seq_len[s])
+        out = np.zeros((n, w.hidden), np.uint16)
+        assert pool.gather_packed(plan, 0, 1, bits16(table), out, np.zeros(2, np.int32), np.zeros(n, np.int32)) == 0
+        exp = expected_sample_rows(w, s, table.view(torch.int16)).cpu().numpy().view(np.uint16)
+        assert np.array_equal(out, exp)
+        plan.destroy(); pool.destroy()
+
+
 @pytest.mark.parametrize("name,kw", [("image_mix_7b", {}), ("video_heavy", {}), ("host_tier_stress", {})])
 def test_full_size_plan_and_sampled_rows(name, kw):
     if not torch.cuda.is_available():
@@ -42,7 +152,7 @@ def test_full_size_plan_and_sampled_rows(name, kw):
     for call in w.write_calls:
         samples = sorted({s for s, _ in call}, key=[s for s, _ in call].index)
         assert run.register(samples) == 0
-        assert run.write(call, keep_src=False) == 0
+        assert run.write(call, keep_src=True) == 0
     rc, plan = run.plan()
     assert rc == 0
     got = plan.arrays()
@@ -85,6 +195,23 @@ def test_full_size_plan_and_sampled_rows(name, kw):
             pass
     # no row left at poison anywhere (checked on the device)
     assert not bool((out == -1).all(dim=1).any().item())
+    # EVERY row of the assembly against the generator (device-side compare, sample by sample)
+    table_i16 = run.table.view(torch.int16)
+    assert assert_every_row(w, out, exp["mb_samples"], row_off[:-1], table_i16) == w.n_samples
+    assert int(row_off[-1]) == out.shape[0]
+    # the oracle itself at full size, whole output, where the host can hold its pool, the sources and the result
+    src_bytes = sum(t.numel() * t.element_size() for t in run.srcs.values())
+    need = src_bytes + (w.hbm_pages + w.host_pages) * w.page_bytes + 2 * out.numel() * 2 + (4 << 30)
+    FULL_ORACLE[name] = False
+    if w.src_dtype == 0 and host_mem_available() >= int(1.25 * need):
+        o_out, o_cu, o_pos = oracle_full_output(w, run.srcs, run.table)
+        assert np.array_equal(o_cu, cu.cpu().numpy()) and np.array_equal(o_pos, pos.cpu().numpy())
+        step = 1 << 18
+        for r in range(0, out.shape[0], step):
+            assert np.array_equal(out[r:r + step].cpu().numpy().view(np.uint16), o_out[r:r + step]), r
+        del o_out
+        FULL_ORACLE[name] = True
+    print(f"full-size {name}: all {out.shape[0]} rows equal the generator's; whole-output oracle run: {FULL_ORACLE[name]}")
     # every rank's share of the deal in one list call each: the same rows, cu_seqlens and positions as the
     # slices of the range assembly checked above
     from gpu_harness import cuda_stream
@@ -327,6 +454,8 @@ def test_full_size_fragmentation_sweep(page_bytes):
         rows += t
     ranges.append((b, n_mb))
     rng = np.random.default_rng(17)
+    table_i16 = table.view(torch.int16)
+    covered = 0
     for lo, hi in ranges:
         out.fill_(-1)
         assert pool.gather_packed(plan, lo, hi, table.data_ptr(), w.vocab, out.data_ptr(), cu.data_ptr(), pos.data_ptr(), st) == 0
@@ -339,6 +468,8 @@ def test_full_size_fragmentation_sweep(page_bytes):
                                  for j in range(lo, hi)]).astype(np.int32)
         assert np.array_equal(cu[:len(exp_cu)].cpu().numpy(), exp_cu)
         assert not bool((out[:n_rows] == -1).all(dim=1).any().item())
+        # every row of the range against the generator
+        covered += assert_every_row(w, out, exp["mb_samples"][q0:q1], row_off[q0:q1] - mb_row[lo], table_i16)
         picks = []
         for q in rng.choice(np.arange(q0, q1), size=min(6, q1 - q0), replace=False):
             s = int(exp["mb_samples"][q])
@@ -348,6 +479,7 @@ def test_full_size_fragmentation_sweep(page_bytes):
         got_rows = out[torch.tensor([r for r, _, _ in picks], device="cuda")].cpu().numpy().view(np.uint16)
         for i, (_, s, p) in enumerate(picks):
             assert np.array_equal(got_rows[i], expected_row(w, s, p)), (lo, hi, s, p)
+    assert covered == len(residents)
     assert pool.status() == (0, 0)
     plan.destroy(); oplan.destroy()
     pool.destroy()
