@@ -250,6 +250,7 @@ class DeviceJob:
         self.pool = fp.Pool(fp.PoolConfig(**pool_config_fields(w)))
         if self.pool.rc != 0:
             raise fp.FlowpoolError(self.pool.rc, "pool_create")
+        apply_tuning(self.pool, args)
         self.table = workloads.embed_table(w, device="cuda")
         self.calls = []
         for call in w.write_calls:
@@ -318,6 +319,15 @@ class DeviceJob:
     def close(self):
         self.torch.cuda.synchronize()
         self.pool.destroy()
+
+
+def apply_tuning(pool, args):
+    """--tuning key=value,...: launch-geometry knobs of the library (pool_set_tuning), for sweeps."""
+    spec = getattr(args, "tuning", None)
+    if spec:
+        rc = pool.set_tuning(**{k: int(v) for k, v in (kv.split("=") for kv in spec.split(","))})
+        if rc != 0:
+            raise SystemExit(f"pool_set_tuning({spec}) -> {rc}")
 
 
 def measure_host_link(torch, nbytes=1 << 30, reps=5):
@@ -397,6 +407,7 @@ def timed_steps(job, steps, warmup, dist):
     prof = job.pool.profile_read()
     job.pool.profile_enable(False)
     launches = job.pool.stats()["gpu_launches"] - launches0
+    job.plan_ms_in_step = float(np.median(job.plan_ms)) if job.plan_ms else None
     if dist:
         ms = max_over_ranks(ms, dist)
         dist.barrier()
@@ -757,7 +768,7 @@ def run_ours(args):
                        "l2": ("L2 flushed between steps (512 MiB scrub outside the timed regions)" if job.fits_l2()
                               else "inputs larger than L2 (no flush needed)"), "parallelism": f"dp{world} (independent batches)"},
             "tokens_per_s": world * w.total_tokens / ms * 1e3,
-            "gpu_launches": launches, "kernels": kern, "phase_ms": phases, "host_link_memcpy": link, "roofline": roofline, "clocks": clocks,
+            "gpu_launches": launches, "kernels": kern, "phase_ms": phases, "plan_call_host_ms_in_step": job.plan_ms_in_step, "host_link_memcpy": link, "roofline": roofline, "clocks": clocks,
         }
     # end to end through host buffers, on the same pool as the headline number
     if rank == 0:
@@ -1387,6 +1398,7 @@ def main():
     ap.add_argument("--page-bytes", type=int, default=2 << 20, help="frag_sweep: page size")
     ap.add_argument("--pool-gib", type=float, default=64.0, help="frag_sweep: pool capacity")
     ap.add_argument("--cycles", type=int, default=10, help="frag_sweep: write/free cycles")
+    ap.add_argument("--tuning", default=None, help="library launch-geometry knobs, e.g. dev_ctas_per_sm=4,host_ctas=6")
     ap.add_argument("--id-skew", default="uniform", choices=["uniform", "zipf"], help="distribution of the text-token ids")
     ap.add_argument("--backbone-only", action="store_true", help="only the backbone-side outputs (padded assembly, table gradient) on an all-HBM pool")
     ap.add_argument("--exchange", action="store_true", help="under torchrun: every rank writes its batch, all plan everything, each assembles its own share from everybody's pages")

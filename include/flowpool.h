@@ -12,15 +12,26 @@
  *  - Every call returns an int32 status: FT_OK or a negative FT_ERR_* code.
  *    Nothing throws, aborts or traps.
  *  - "host" / "device" in a parameter comment says where the pointer lives.
- *    Host arrays are read before the call returns.  Device work is enqueued on
- *    the caller's stream (`stream` = a cudaStream_t passed as void*; NULL = the
- *    legacy default stream); ordering between calls is stream order.
+ *    Host arrays are read before the call returns.  `stream` is a cudaStream_t
+ *    passed as void* (NULL = the legacy default stream).  Kernels that read or
+ *    write the caller's data (token ids, embedding sources, the table, outputs)
+ *    run on that stream, in stream order.  Kernels that only touch the pool's
+ *    own tables, rings and page lists (registration scan, page allocation, the
+ *    packing plan, free, import/export lists, span grids) run on a metadata
+ *    stream the pool owns, in call order; the library links the two with
+ *    events, so that every call still sees the effects of every earlier call
+ *    of the pool, and whatever the caller enqueues on `stream` after a call
+ *    comes after that call.  The gain: the page allocation of producer call
+ *    i+1 is worked out while the copy of call i is streaming (the producer
+ *    "immediately proceeds", Sec. 3.1).
  *  - Two streams per pool are supported: a producer side (register, write, import, free) and a consumer side
  *    (plan, export, gather) may be issued, from one host thread, on two different streams so that the encoder's
  *    scatter of the next batch overlaps the backbone's assembly of the current one (the decoupled
- *    producer-consumer flow of Sec. 3.1).  The library orders the sides itself: a consumer-side call waits for
- *    the producer-side calls issued before it, and pool_free waits for the consumer-side calls issued before it;
- *    the sides use separate scratch and separate side streams for host-tier traffic.
+ *    producer-consumer flow of Sec. 3.1).  The library orders the sides itself: a consumer-side copy waits for
+ *    the producer-side copies issued before it, and pool_free waits for the copies of both sides issued before it;
+ *    the sides use separate call contexts and separate side streams for host-tier traffic.
+ *  - A call may block the host briefly when the caller runs more than 8 calls of one side ahead of the device
+ *    (the per-call descriptor staging is a ring of 16 pinned buffers per side).
  *  - One caller thread per pool.  The caller owns every buffer it passes in
  *    (backing memory, sources, table, outputs); the library owns its metadata
  *    and anything it allocated itself.
@@ -300,8 +311,9 @@ int32_t pool_gather_list(ft_pool* pool, const ft_plan* plan, const uint32_t* mb_
  */
 int32_t pool_free(ft_pool* pool, const uint32_t* sample_slot, uint32_t n, void* stream);
 
-/* First asynchronous error since the last call (smallest call, then smallest
- * detail), then cleared.  Synchronises the device. */
+/* First asynchronous error since the last call of pool_status (smallest call, then smallest code, then smallest
+ * detail), then cleared.  Synchronises the device.  Calls are numbered from the last read, on 28 bits: read the
+ * status at least once every 2^28 calls of the pool (a training run that checks it once per step never comes close). */
 int32_t pool_status(ft_pool* pool, int32_t* first_device_error, uint64_t* detail);
 
 int32_t pool_stats(ft_pool* pool, ft_pool_stats* out);
@@ -439,6 +451,31 @@ typedef struct {
 int32_t pool_profile_enable(ft_pool* pool, int32_t on);
 int32_t pool_profile_read(ft_pool* pool, ft_kernel_time* out /* host [FT_K_COUNT] */);
 
+/*
+ * Launch geometry of the data kernels.  The paper has no counterpart: these are this library's knobs, all of them
+ * in this one struct (nothing is read from the environment).  pool_get_tuning returns the values in force;
+ * pool_set_tuning replaces them (0 in a field = that field's built-in default, the optimum measured on a B200);
+ * out-of-range values INVALID_ARG and nothing changes.  Call it between other calls of the pool; it synchronises
+ * the device.  None of the knobs changes any result.
+ *   dev_ctas_per_sm      resident CTAs per SM of the HBM-tier gather kernel (default 4; 1..8)
+ *   scatter_ctas_per_sm  resident CTAs per SM of the HBM-tier scatter kernel (default 4; 1..8)
+ *   scatter_group        chunks a scatter CTA claims at a time (default 1)
+ *   chunk_shift          log2 of the scatter's work unit in bytes of a span's image (default 16; 14..21)
+ *   host_ctas            grid of the host-tier bulk-copy kernels (default 6): few SMs, so that long-latency host-link
+ *                        accesses do not clog the memory pipelines of the SMs that stream HBM
+ *   host_store_ctas      grid of the vector-store scatter into host frames (fp32 sources, host-only pools; default 8)
+ *   gather_unroll        16-byte vectors per lane in flight in the gather kernel (4 or 8; default 4)
+ *   grad_ctas_per_sm     CTAs per SM of the table-gradient kernel (default 6; 1..8)
+ *   grad_hot_threshold   rows from which an id takes the frequent-id gradient kernel (default rows / (8 x grid), >= 64)
+ */
+typedef struct {
+  uint32_t dev_ctas_per_sm, scatter_ctas_per_sm, scatter_group, chunk_shift;
+  uint32_t host_ctas, host_store_ctas, gather_unroll, grad_ctas_per_sm, grad_hot_threshold;
+  uint32_t reserved[7];
+} ft_tuning;
+int32_t pool_get_tuning(ft_pool* pool, ft_tuning* out);
+int32_t pool_set_tuning(ft_pool* pool, const ft_tuning* in);
+
 /* Page GVAs of one span, by ordinal (for parity checks).  Synchronises. */
 int32_t pool_debug_span_pages(ft_pool* pool, uint32_t slot, uint32_t span, uint64_t* gva_out,
                               uint32_t cap, uint32_t* n);
@@ -455,7 +492,8 @@ int32_t pool_debug_translate(ft_pool* pool, const uint64_t* gva, uint32_t n, uin
 /* Tear down: frees everything the library allocated.  Synchronises. */
 int32_t pool_destroy(ft_pool* pool);
 
-/* Last CUDA error string seen by this library in this process (static storage). */
+/* Last CUDA error string seen by this library on the calling thread (thread-local storage: with one caller
+ * thread per pool, that is the pool's own last error). */
 const char* flowpool_last_cuda_error(void);
 
 #ifdef __cplusplus

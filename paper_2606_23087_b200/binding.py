@@ -27,7 +27,7 @@ EXPORTS = (
     "pool_plan_microbatches", "plan_summary",
     "plan_arrays", "plan_destroy", "pool_gather_packed", "pool_gather_list", "pool_set_span_grids", "pool_gather_padded", "pool_embed_grad", "pool_free", "pool_status", "pool_stats",
     "pool_ready_count", "pool_take_ready", "pool_backing", "pool_ipc_export", "pool_ipc_open", "pool_ipc_close", "pool_export_mapping", "pool_import_mapping", "pool_export_samples", "pool_import_samples",
-    "pool_profile_enable", "pool_profile_read", "pool_debug_span_pages", "pool_debug_ring", "pool_debug_translate", "pool_destroy", "flowpool_last_cuda_error",
+    "pool_get_tuning", "pool_set_tuning", "pool_profile_enable", "pool_profile_read", "pool_debug_span_pages", "pool_debug_ring", "pool_debug_translate", "pool_destroy", "flowpool_last_cuda_error",
 )
 
 
@@ -63,6 +63,14 @@ class PoolStats(C.Structure):
     _fields_ = [(k, C.c_uint64) for k in (
         "pages_total", "pages_free", "hbm_pages", "host_pages", "text_pages_total", "text_pages_free",
         "live_samples", "live_spans", "bytes_written", "bytes_gathered", "gpu_launches")]
+
+
+TUNING_FIELDS = ("dev_ctas_per_sm", "scatter_ctas_per_sm", "scatter_group", "chunk_shift", "host_ctas", "host_store_ctas",
+                 "gather_unroll", "grad_ctas_per_sm", "grad_hot_threshold")
+
+
+class Tuning(C.Structure):
+    _fields_ = [(k, C.c_uint32) for k in TUNING_FIELDS] + [("reserved", C.c_uint32 * 7)]
 
 
 class KernelTime(C.Structure):
@@ -124,6 +132,8 @@ def lib():
             "pool_ipc_export": [P, P],
             "pool_ipc_open": [P, P, P],
             "pool_ipc_close": [P, P],
+            "pool_get_tuning": [P, P],
+            "pool_set_tuning": [P, P],
             "pool_profile_enable": [P, i32],
             "pool_profile_read": [P, P],
             "pool_debug_span_pages": [P, u32, u32, P, u32, P],
@@ -323,6 +333,22 @@ class Pool:
         local_slots = _u32(local_slots)
         blob = np.ascontiguousarray(blob, dtype=np.uint8)
         return lib().pool_import_samples(self.h, _p(local_slots), len(local_slots), _p(blob), len(blob), stream or None)
+
+    def get_tuning(self):
+        t = Tuning()
+        rc = lib().pool_get_tuning(self.h, C.byref(t))
+        if rc:
+            raise FlowpoolError(rc, "pool_get_tuning")
+        return {k: getattr(t, k) for k in TUNING_FIELDS}
+
+    def set_tuning(self, **fields):
+        """pool_set_tuning: the named knobs, every other one at its default."""
+        t = Tuning()
+        for k, v in fields.items():
+            if k not in TUNING_FIELDS:
+                raise KeyError(k)
+            setattr(t, k, int(v))
+        return lib().pool_set_tuning(self.h, C.byref(t))
 
     def profile_enable(self, on=True):
         return lib().pool_profile_enable(self.h, 1 if on else 0)

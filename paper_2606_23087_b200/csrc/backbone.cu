@@ -563,30 +563,31 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_set_span_grids(ft
   }
   n = (uint32_t)keep.size();
   const size_t o_grid = 0, o_sid = align_up_sz((size_t)n * sizeof(uint4), 16), bytes = o_sid + (size_t)n * 4;
-  std::vector<uint8_t> blob(bytes);
-  uint4* hg = reinterpret_cast<uint4*>(blob.data() + o_grid);
-  uint32_t* hs = reinterpret_cast<uint32_t*>(blob.data() + o_sid);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  ft_call_ctx* cx = nullptr;
+  int32_t rc = ctx_acquire(p, 0, bytes, bytes, &cx);
+  if (rc != FT_OK) return rc;
+  uint4* hg = reinterpret_cast<uint4*>(static_cast<uint8_t*>(cx->h) + o_grid);
+  uint32_t* hs = reinterpret_cast<uint32_t*>(static_cast<uint8_t*>(cx->h) + o_sid);
   for (uint32_t k = 0; k < n; ++k) {
     const uint32_t i = keep[k];
     hg[k] = make_uint4(grid_thw[3ull * i], grid_thw[3ull * i + 1], grid_thw[3ull * i + 2], 0);
     hs[k] = slot[i] * S + span_idx[i];
   }
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
-  {
-    const int32_t rc0 = begin_free(p, st);  // assemblies issued on another stream read the grids first
-    if (rc0 != FT_OK) return rc0;
-  }
-  void* d = nullptr;
-  const int32_t rc = stage_upload(p, 0, blob.data(), bytes, bytes, st, &d);
-  if (rc != FT_OK) return rc;
+  for (uint32_t k = 0; k < n; ++k) memcpy(p->spans[hs[k]].grid, &hg[k], 12);  // host mirror (exported with the sample)
+  if ((rc = ctx_upload(p, cx, bytes)) != FT_OK) return rc;
+  // assemblies already in flight on a caller's stream read the grids as they were: the metadata stream waits for them
+  if ((rc = meta_after_data(p)) != FT_OK) return rc;
+  if ((rc = meta_after(p, st)) != FT_OK) return rc;
   GridCall c;
   c.n = n;
-  c.grid = reinterpret_cast<const uint4*>(static_cast<uint8_t*>(d) + o_grid);
-  c.span_id = reinterpret_cast<const uint32_t*>(static_cast<uint8_t*>(d) + o_sid);
-  k_set_grids<<<(n + 255) / 256, 256, 0, st>>>(p->view, c);
+  c.grid = reinterpret_cast<const uint4*>(static_cast<uint8_t*>(cx->d) + o_grid);
+  c.span_id = reinterpret_cast<const uint32_t*>(static_cast<uint8_t*>(cx->d) + o_sid);
+  k_set_grids<<<(n + 255) / 256, 256, 0, p->meta>>>(p->view, c);
   FT_CUDA(cudaGetLastError());
-  for (uint32_t k = 0; k < n; ++k) memcpy(p->spans[hs[k]].grid, &hg[k], 12);  // host mirror (exported with the sample)
+  if ((rc = ctx_release(p, cx, p->meta)) != FT_OK) return rc;
   p->gpu_launches += 1;
+  if ((rc = meta_to(p, st)) != FT_OK) return rc;
   return end_producer(p, st);
 }
 
@@ -612,14 +613,18 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_gather_padded(ft_
     if (rc0 != FT_OK) return rc0;
   }
   {
-    const int32_t rc1 = gather_launch(p, pl, mb_begin, mb_end, embed_table, vocab, out_embeds, nullptr, nullptr, lay.L, st, nullptr, 0, 0, 0);
+    ft_call_ctx* cx = nullptr;
+    int32_t rc1 = ctx_acquire(p, 1, 0, 0, &cx, false, st);  // for its claim counter
     if (rc1 != FT_OK) return rc1;
+    rc1 = gather_launch(p, pl, mb_begin, mb_end, embed_table, vocab, out_embeds, nullptr, nullptr, lay.L, st, nullptr, 0, 0, 0, cx->counters);
+    if (rc1 != FT_OK) return rc1;
+    if ((rc1 = ctx_release(p, cx, st)) != FT_OK) return rc1;
   }
   const PlanView pv = make_plan_view(pl);
   k_pad_zero<<<(unsigned)p->sm_count * 8, 256, 0, st>>>(pv, lay, p->view.row_bytes, static_cast<uint8_t*>(out_embeds));
   IndexArgs ia;
   ia.lay = lay; ia.pad_id = pad_id; ia.cu = out_cu; ia.pos3 = out_pos3; ia.ids = out_ids; ia.labels = out_labels;
-  ia.mask = out_mask; ia.call_seq = p->call_seq;
+  ia.mask = out_mask; ia.call_seq = status_seq(p);
   k_backbone_index<<<(unsigned)((lay.rows + 255) / 256), 256, 0, st>>>(p->view, pv, ia);
   FT_CUDA(cudaGetLastError());
   p->gpu_launches += 2;
@@ -665,7 +670,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_embed_grad(ft_poo
   FT_CUDA(cudaMallocAsync(reinterpret_cast<void**>(&d), off, st));
   RowIdArgs ra;
   ra.lay = lay; ra.vocab = vocab; ra.row_id = reinterpret_cast<int32_t*>(d + o_row);
-  ra.id_count = reinterpret_cast<uint32_t*>(d + o_cnt); ra.call_seq = p->call_seq;
+  ra.id_count = reinterpret_cast<uint32_t*>(d + o_cnt); ra.call_seq = status_seq(p);
   HotArgs ha;
   ha.rows = lay.rows; ha.vocab = vocab; ha.n_blocks = n_blocks;
   // an id is frequent when its rows alone are an eighth of an average CTA's share of the layout's rows

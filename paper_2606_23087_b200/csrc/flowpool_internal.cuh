@@ -70,10 +70,26 @@ struct PoolView {
   unsigned long long* status;  // first asynchronous error key; ~0 = none
 };
 
-// key = call_seq << 40 | (-code) << 32 | detail ; the smallest key is reported
-__device__ __forceinline__ void note_error(const PoolView& v, uint64_t call_seq, int32_t code, uint32_t detail) {
-  unsigned long long key = (call_seq << 40) | ((unsigned long long)(uint32_t)(-code) << 32) | detail;
+// key = seq << 36 | (-code) << 32 | detail ; the smallest key is reported.  seq = calls since the status word was
+// last read (28 bits: pool_status restarts the count), so the order of the keys is the order of the calls.
+constexpr uint64_t kStatusSeqMask = (1ull << 28) - 1;
+__device__ __forceinline__ void note_error(const PoolView& v, uint64_t seq, int32_t code, uint32_t detail) {
+  unsigned long long key = ((seq & kStatusSeqMask) << 36) | ((unsigned long long)((uint32_t)(-code) & 15u) << 32) | detail;
   atomicMin(v.status, key);
+}
+
+// Work counters of the persistent data kernels.  A kernel claims its work units in order with atomicAdd(claim) and,
+// when a CTA runs out of work, reports with atomicAdd(done): the last CTA of the grid puts both words back to zero,
+// so a counter pair is zero whenever no kernel is using it and no launch needs a memset in front of it.
+struct ClaimCounter {
+  unsigned long long claim, done;
+};
+__device__ __forceinline__ void claim_release(ClaimCounter* c) {  // one thread per CTA, after its last claim
+  __threadfence();
+  if (atomicAdd(&c->done, 1ull) == (unsigned long long)gridDim.x * gridDim.y - 1) {
+    c->claim = 0; c->done = 0;
+    __threadfence();
+  }
 }
 
 __device__ __forceinline__ uint64_t page_gva(const PoolView& v, uint32_t global_page) {
@@ -220,23 +236,28 @@ struct ft_slot_mirror {
   bool remote = false;  // imported from a peer: pages and text pages are not ours to recycle
   uint32_t seq_len = 0, n_spans = 0, spans_written = 0, n_text_pages = 0;
   uint64_t generation = 0;
+  uint64_t named = 0;   // call_seq of the call that last listed this slot (duplicate detection inside one call)
 };
 struct ft_span_mirror {
   uint32_t pos = 0, tokens = 0, npages = 0;
   uint32_t grid[3] = {0, 0, 0};  // token grid (T, H, W) as last set; all zero = none
   bool written = false;
+  uint64_t named = 0;   // call_seq of the write call that last named this span
 };
 
-// Pinned staging for per-call descriptor uploads: a small ring of buffers, each guarded by an
-// event, so a call never rewrites host memory that an earlier asynchronous copy may still read.
-struct ft_staging {
-  static constexpr int kBufs = 8;
-  void* h[kBufs] = {};
-  size_t cap[kBufs] = {};
-  cudaEvent_t ev[kBufs] = {};
-  bool busy[kBufs] = {};
-  int next = 0;
+// Per-call context: the descriptors of one ABI call travel host -> device through one of a small ring of these.
+// `h` is pinned staging the call fills on the host; `d` is device scratch that receives the upload and the call's scan
+// outputs; `counters` are two claim counters in the pool's metadata block (main and side stream of the call).  Two
+// events guard reuse: the host waits for `ev_up` before it rewrites `h`; the metadata stream waits for `ev_done`
+// (recorded behind the last kernel of the call that reads `d` or the counters) before it rewrites `d`.
+struct ft_call_ctx {
+  void* h = nullptr;   size_t hcap = 0;
+  void* d = nullptr;   size_t dcap = 0;
+  cudaEvent_t ev_up = nullptr, ev_done = nullptr;
+  bool busy_up = false, busy_done = false;
+  ft::ClaimCounter* counters = nullptr;  // [2], device
 };
+constexpr int kCallCtx = 16;
 
 struct ft_pool {
   ft_pool_config cfg;
@@ -253,16 +274,34 @@ struct ft_pool {
   void* hbm_base = nullptr;    bool own_hbm = false;
   void* host_base = nullptr;   bool own_host = false;  // host pointer
   void* host_dev = nullptr;                            // the same memory as the device sees it
-  // per-call descriptors and scan outputs: one arena per side, so that a producer call and a consumer call issued on
-  // different streams never share scratch (0 = register/write/import/free, 1 = plan/export)
-  void* d_scratch[2] = {nullptr, nullptr};   size_t scratch_cap[2] = {0, 0};
+  // per-call descriptors and scan outputs (see ft_call_ctx): one ring per side (0 = register, write, import, free,
+  // span grids; 1 = plan, export, assemblies), so that a context of a long-running assembly is never the one a producer
+  // call has to wait for
+  ft_call_ctx ctx[2][kCallCtx];
+  int ctx_next[2] = {0, 0};
+  // The metadata stream.  Every kernel that only touches the pool's tables, rings and page lists (registration scan,
+  // page allocation, the packing plan, free, import/export lists, span grids) runs here, in call order; the kernels
+  // that move data (token ids, scatter, gather) run on the caller's stream behind an event of this one.  The
+  // metadata of producer call i+1 is thus worked out while the scatter of call i streams, and the plan is made
+  // while the last scatters run.
+  cudaStream_t meta = nullptr;
+  cudaEvent_t ev_meta = nullptr;      // re-recorded on `meta` whenever a caller's stream has to wait for it
+  cudaEvent_t ev_in = nullptr;        // re-recorded on a caller's stream when `meta` has to wait for that stream
+  cudaEvent_t ev_noalloc = nullptr;   // behind the last reader of the fixed no-allocation scratch
+  bool have_noalloc_ev = false;
+  uint64_t meta_seq = 0;              // metadata batches enqueued so far
+  cudaStream_t synced_stream[2] = {nullptr, nullptr};  // the caller streams that waited for `meta` last ...
+  uint64_t synced_seq[2] = {~0ull, ~0ull};             // ... and the batch count they waited for
+  uint64_t status_base = 0;           // call_seq at the last pool_status read
+  std::vector<uint8_t> noalloc_blob;  // host staging of pool_write_embeddings_noalloc, made at pool_create
+  void* plan_pinned = nullptr;        // pinned landing zone of the plan's summary read-back
+  size_t plan_pinned_cap = 0;
   std::vector<uint32_t> bind_hbm, bind_host;           // vpn -> frame of this process's binding (exported to peers)
   void* d_text_base() const { return d_text; }
   std::vector<void*> peer_allocs;                      // imported peers' page-table arrays
   std::vector<uint8_t> peer_imported;                  // [world_size]
   bool peer_host_frames = false;                       // some imported peer binds host-tier pages
   std::vector<std::array<uint64_t, 3>> peer_bases;     // [world_size] slab addresses (HBM, host, text) as seen here
-  ft_staging staging;
   // host-tier traffic runs beside the HBM kernels on a side stream: one per side (0 producer, 1 consumer), so that
   // host-tier writes and host-tier reads of concurrent calls can use both directions of the link at once
   cudaStream_t side_stream[2] = {nullptr, nullptr};
@@ -279,9 +318,8 @@ struct ft_pool {
   int host_ctas = 6;            // grid of the host-tier bulk-copy kernels: few SMs, so that long-latency host-link
                                 // accesses do not clog the memory pipelines of the SMs that stream HBM; 6 rather
                                 // than 8 because a write and a read kernel running together (two streams) share
-                                // the link better with fewer requests in flight (FLOWPOOL_HOST_CTAS overrides)
-  int host_store_ctas = 8;      // grid of the vector-store scatter into host frames (fp32 sources, host-only pools;
-                                // FLOWPOOL_HOST_STORE_CTAS overrides)
+                                // the link better with fewer requests in flight
+  int host_store_ctas = 8;      // grid of the vector-store scatter into host frames (fp32 sources, host-only pools)
   int chunk_shift = 16;         // log2 of k_scatter's work unit in bytes of a span's image (14..21)
   int scatter_group = 0;        // chunks per round-robin group of k_scatter; 0 = the measured default
   int scatter_ctas_per_sm = 0;  // resident CTAs per SM of the device-tier scatter kernel; 0 = the measured default
@@ -304,7 +342,7 @@ int32_t plan_device_setup(ft_pool* p);
 // (d_list: device array of the list layout's entries, or nullptr for the range [mb_begin, mb_end))
 int32_t gather_launch(ft_pool* p, const ft_plan* pl, uint32_t mb_begin, uint32_t mb_end, const void* embed_table,
                       uint32_t vocab, void* out_embeds, int32_t* out_cu, int32_t* out_pos, uint32_t pad_L, cudaStream_t st,
-                      const void* d_list, uint32_t n_list, uint64_t list_tiles, uint64_t list_rows);
+                      const void* d_list, uint32_t n_list, uint64_t list_tiles, uint64_t list_rows, ClaimCounter* counter);
 __global__ void k_page_table_init(uint64_t* pte, const uint32_t* bind, uint64_t n, uint64_t base, uint64_t frame_bytes,
                                   uint64_t flags);
 // uploads `bytes` from `src` (pageable) to the front of the pool's device scratch, asynchronously,
@@ -322,8 +360,39 @@ inline void prof_end(ft_pool* p, cudaStream_t st) {
   cudaEventRecord(p->prof.back().e1, st);
 }
 size_t align_up_sz(size_t x, size_t a);
-// (arena: 0 = producer-side calls, 1 = consumer-side calls)
-int32_t stage_upload(ft_pool* p, int arena, const void* src, size_t bytes, size_t total_bytes, cudaStream_t st, void** d_out);
+// Threads of a one-block scan kernel over n items: no more warps than there are items, so that the block fits on an
+// SM beside the resident CTAs of a copy kernel (the metadata of one call is worked out while another call streams).
+inline unsigned scan_threads(uint64_t n) { return (unsigned)(n >= 1024 ? 1024 : (n < 32 ? 32 : (n + 31) / 32 * 32)); }
+// Takes the next call context: afterwards `h` holds at least `blob_bytes` of pinned staging the caller may fill, `d`
+// at least `total_bytes` of device scratch no earlier kernel still reads (the metadata stream has been told to wait
+// for the previous user; with on_meta = false it is `first_user` that waits, for a call that uploads nothing and
+// only needs the context's counters on that stream).
+// (side: 0 = producer-side calls, 1 = consumer-side calls)
+int32_t ctx_acquire(ft_pool* p, int side, size_t blob_bytes, size_t total_bytes, ft_call_ctx** out, bool on_meta = true,
+                    cudaStream_t first_user = nullptr);
+// h[0, bytes) -> d[0, bytes) on the metadata stream
+int32_t ctx_upload(ft_pool* p, ft_call_ctx* c, size_t bytes);
+// `last` is the stream of the call's last kernel that reads the context
+int32_t ctx_release(ft_pool* p, ft_call_ctx* c, cudaStream_t last);
+// sequence number for asynchronous error keys of the current call
+inline uint64_t status_seq(const ft_pool* p) { return (p->call_seq - p->status_base) & kStatusSeqMask; }
+// `st` waits for everything enqueued on the metadata stream so far (skipped when it already has)
+inline int32_t meta_to(ft_pool* p, cudaStream_t st) {
+  for (int i = 0; i < 2; ++i)
+    if (p->synced_stream[i] == st && p->synced_seq[i] == p->meta_seq) return FT_OK;
+  FT_CUDA(cudaEventRecord(p->ev_meta, p->meta));
+  FT_CUDA(cudaStreamWaitEvent(st, p->ev_meta, 0));
+  int slot = p->synced_stream[0] == st && p->synced_seq[0] != ~0ull ? 0 : (p->synced_stream[1] == st && p->synced_seq[1] != ~0ull ? 1 : -1);
+  if (slot < 0) slot = p->synced_seq[0] == ~0ull ? 0 : (p->synced_seq[1] == ~0ull ? 1 : (p->synced_seq[0] <= p->synced_seq[1] ? 0 : 1));
+  p->synced_stream[slot] = st; p->synced_seq[slot] = p->meta_seq;
+  return FT_OK;
+}
+// the metadata stream waits for everything enqueued on `st` so far
+inline int32_t meta_after(ft_pool* p, cudaStream_t st) {
+  FT_CUDA(cudaEventRecord(p->ev_in, st));
+  FT_CUDA(cudaStreamWaitEvent(p->meta, p->ev_in, 0));
+  return FT_OK;
+}
 
 // appends a sample that just became READY; entries of samples freed since are dropped whenever the queue has grown
 // past four entries per slot, so a caller that never takes from it cannot make it grow without bound
@@ -337,20 +406,26 @@ inline void ready_push(ft_pool* p, uint32_t slot) {
   p->ready_fifo.emplace_back(slot, p->slots[slot].generation);
 }
 
-// Cross-stream ordering (the producer side and the consumer side of a pool may be driven from two streams):
-// a consumer-side call waits for the producer-side calls issued before it; pool_free waits for the consumer-side
-// calls issued before it.  Same-stream use costs one event record per call and no wait.
+// Cross-stream ordering.  Data kernels run on the callers' streams (a producer side and a consumer side, possibly two
+// streams), metadata kernels on the pool's metadata stream:
+//  * a consumer-side data kernel waits for the producer-side data kernels issued before it (another stream's only)
+//    and for the metadata enqueued so far;
+//  * a metadata kernel that changes what data kernels already in flight may read (free, span grids) waits for the
+//    latest producer-side and consumer-side data kernels;
+//  * metadata kernels among themselves are ordered by the metadata stream.
 inline int32_t begin_consumer(ft_pool* p, cudaStream_t st) {
   if (p->have_producer_ev && p->last_producer_stream != st) FT_CUDA(cudaStreamWaitEvent(st, p->ev_producer, 0));
-  return FT_OK;
+  return meta_to(p, st);
 }
 inline int32_t end_consumer(ft_pool* p, cudaStream_t st) {
   FT_CUDA(cudaEventRecord(p->ev_consumer, st));
   p->have_consumer_ev = true; p->last_consumer_stream = st;
   return FT_OK;
 }
-inline int32_t begin_free(ft_pool* p, cudaStream_t st) {
-  if (p->have_consumer_ev && p->last_consumer_stream != st) FT_CUDA(cudaStreamWaitEvent(st, p->ev_consumer, 0));
+// before metadata kernels that retire or change state data kernels in flight may still read
+inline int32_t meta_after_data(ft_pool* p) {
+  if (p->have_consumer_ev) FT_CUDA(cudaStreamWaitEvent(p->meta, p->ev_consumer, 0));
+  if (p->have_producer_ev) FT_CUDA(cudaStreamWaitEvent(p->meta, p->ev_producer, 0));
   return FT_OK;
 }
 inline int32_t end_producer(ft_pool* p, cudaStream_t st) {

@@ -1,13 +1,15 @@
 // The consumer: GVA translation and packed-microbatch assembly (Sec. 3.1-3.2).
 //
-// k_gather: output rows are cut into tiles of 32 consecutive rows.  For each tile one warp resolves the
-// 32 row sources, one lane per row (plan position -> slot -> token id from the text page; a placeholder
-// position -> span -> page ordinal -> page GVA from the span's two-level list -> page-table entry), and
-// leaves the frame addresses in shared memory; then every warp of the CTA streams rows with 16-byte
-// vectors.  Rows that straddle pages carry one address per page touched.  With a two-tier pool the
-// kernel is launched twice, once per tier, so host-link reads never stall HBM reads.
+// k_gather: output rows are cut into units of up to 32 consecutive rows, claimed in order from a device counter.
+// Each CTA has one resolver warp and eight streaming warps.  The resolver works one unit ahead: while the streaming
+// warps copy unit t with 16-byte vectors, it claims unit t+1 and resolves its row sources, one lane per row (plan
+// position -> slot -> token id from the text page; a placeholder position -> span -> page ordinal -> page GVA from
+// the span's two-level list -> page-table entry), leaving the frame addresses in the other half of a double buffer
+// in shared memory.  Rows that straddle pages carry one address per page touched.  With a two-tier pool the kernel
+// is launched once per tier, so host-link reads never stall HBM reads.
 #include <algorithm>
 #include <cstdlib>
+#include <cstring>
 #include <type_traits>
 #include <vector>
 
@@ -18,7 +20,8 @@ namespace ft {
 
 constexpr int kTileRows = 32;
 constexpr int kMaxSeg = 10;  // pages one row can touch: row_bytes <= 32 KiB over 4 KiB pages, plus a straddle
-constexpr int kGatherThreads = 256;
+constexpr int kStreamWarps = 8;                          // warps that copy rows
+constexpr int kGatherThreads = 32 * (kStreamWarps + 1);  // + the resolver warp
 
 enum { kTierAll = 0, kTierDeviceOnly = 1, kTierHostOnly = 2 };
 
@@ -50,7 +53,8 @@ struct GatherArgs {
   uint64_t call_seq;
   uint32_t write_index;  // this launch writes cu_seqlens / position ids
   uint32_t pad_L;        // 0: packed rows; else every microbatch starts at a multiple of pad_L rows (padded layout)
-  unsigned long long* tile_counter;  // device, zero at launch
+  uint32_t sub_shift;    // a claim covers 32 >> sub_shift rows (short ranges are cut finer, so that every SM has work)
+  ClaimCounter* tile_counter;  // device, zero at rest
   const ListEntry* list;             // list layout: the microbatches to assemble, in output order (else nullptr)
   uint32_t n_list;
   uint64_t list_tiles;               // tiles over all entries
@@ -58,145 +62,160 @@ struct GatherArgs {
 
 template <int MODE, int U, bool LIST>
 __global__ void __launch_bounds__(kGatherThreads) k_gather(PoolView v, PlanView pl, GatherArgs a) {
-  __shared__ RowDesc desc[kTileRows];
+  __shared__ RowDesc desc[2][kTileRows];
+  __shared__ uint32_t valid[2];
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const uint64_t tile_lo = a.row_lo / kTileRows, tile_hi = (a.row_hi + kTileRows - 1) / kTileRows;
   const uint32_t row_vecs = v.row_bytes >> 4;
+  const uint32_t R = kTileRows >> a.sub_shift, sub_mask = (1u << a.sub_shift) - 1;
+  const bool resolver = warp == kStreamWarps;
 
-  __shared__ uint64_t next_tile;
-  __shared__ uint32_t cur_entry;
-  for (;;) {
-    // tiles are claimed in order from a device counter (zeroed by the host before the launch): the CTAs in
-    // flight always cover one compact window of the output, and uneven tiles balance themselves
-    if (threadIdx.x == 0) {
-      const uint64_t c = atomicAdd(a.tile_counter, 1ull);
-      if (LIST) {
-        // list layout: the entry holding claim c (last entry whose first tile is <= c), then its plan tile
-        uint32_t lo = 0, hi = a.n_list;
-        while (hi - lo > 1) {
-          const uint32_t mid = (lo + hi) >> 1;
-          if (a.list[mid].tile0 <= c) lo = mid; else hi = mid;
-        }
-        cur_entry = lo;
-        next_tile = c < a.list_tiles ? a.list[lo].row_lo / kTileRows + (c - a.list[lo].tile0) : ~0ull;
-      } else {
-        next_tile = tile_lo + c;
+  // Resolver warp: claims the next unit (units are claimed in order, so the CTAs in flight always cover one compact
+  // window of the output and uneven units balance themselves) and resolves its rows into desc[buf].
+  auto resolve = [&](uint32_t buf) {
+    unsigned long long c = 0;
+    if (lane == 0) c = atomicAdd(&a.tile_counter->claim, 1ull);
+    c = __shfl_sync(0xFFFFFFFFu, c, 0);
+    const uint64_t ct = c >> a.sub_shift;  // claim index in whole 32-row tiles
+    uint64_t tile = ~0ull;
+    uint32_t entry = 0;
+    if (LIST) {
+      // list layout: the entry holding the claim (last entry whose first tile is <= ct), then its plan tile
+      uint32_t lo = 0, hi = a.n_list;
+      while (hi - lo > 1) {
+        const uint32_t mid = (lo + hi) >> 1;
+        if (a.list[mid].tile0 <= ct) lo = mid; else hi = mid;
       }
+      entry = lo;
+      if (ct < a.list_tiles) tile = a.list[lo].row_lo / kTileRows + (ct - a.list[lo].tile0);
+    } else if (tile_lo + ct < tile_hi) {
+      tile = tile_lo + ct;
     }
-    __syncthreads();
-    const uint64_t tile = next_tile;
-    if (LIST ? tile == ~0ull : tile >= tile_hi) break;
-    if (warp == 0) {
-      const uint64_t row = tile * kTileRows + lane;
-      RowDesc d;
-      d.nseg = 0; d.off0 = 0; d.shift = 31; d.out_row = 0;
-      // the rows this tile may touch: the call's range, or the listed microbatch it belongs to
-      uint64_t row_lo = a.row_lo, row_hi = a.row_hi, out0 = 0, cu0 = 0;
-      uint32_t q_lo = a.q_lo;
-      if (LIST) {
-        const ListEntry en = a.list[cur_entry];
-        row_lo = en.row_lo; row_hi = en.row_hi; out0 = en.out_row0; cu0 = en.cu0; q_lo = en.q_lo;
+    if (tile == ~0ull) {  // past the end: this CTA is done claiming
+      if (lane == 0) { valid[buf] = 0; claim_release(a.tile_counter); }
+      return;
+    }
+    if (lane == 0) valid[buf] = 1;
+    if (lane >= R) return;
+    const uint64_t row = tile * kTileRows + (uint64_t)((uint32_t)c & sub_mask) * R + lane;
+    RowDesc d;
+    d.nseg = 0; d.off0 = 0; d.shift = 31; d.out_row = 0;
+    // the rows this unit may touch: the call's range, or the listed microbatch it belongs to
+    uint64_t row_lo = a.row_lo, row_hi = a.row_hi, out0 = 0, cu0 = 0;
+    uint32_t q_lo = a.q_lo;
+    if (LIST) {
+      const ListEntry en = a.list[entry];
+      row_lo = en.row_lo; row_hi = en.row_hi; out0 = en.out_row0; cu0 = en.cu0; q_lo = en.q_lo;
+    }
+    if (row >= row_lo && row < row_hi) {
+      // plan position of the sample holding this row: the tile's first sample, then a short walk
+      uint32_t q = pl.tile_first_sample[tile];
+      if (q < q_lo) q = q_lo;
+      while (row >= pl.sample_row_off[q + 1]) ++q;
+      const uint32_t p = (uint32_t)(row - pl.sample_row_off[q]);
+      const uint32_t slot = pl.mb_samples[q];
+      uint64_t out_row = out0 + (row - row_lo);
+      if (!LIST && a.pad_L) {  // padded layout: microbatch j of the range starts at row (j - mb_begin) * L
+        const uint32_t j = pl.plan_sample_mb[q];
+        out_row += (uint64_t)(j - a.mb_begin) * a.pad_L - (pl.mb_row_off[j] - a.row_lo);
       }
-      if (row >= row_lo && row < row_hi) {
-        // plan position of the sample holding this row: the tile's first sample, then a short walk
-        uint32_t q = pl.tile_first_sample[tile];
-        if (q < q_lo) q = q_lo;
-        while (row >= pl.sample_row_off[q + 1]) ++q;
-        const uint32_t p = (uint32_t)(row - pl.sample_row_off[q]);
-        const uint32_t slot = pl.mb_samples[q];
-        uint64_t out_row = out0 + (row - row_lo);
-        if (!LIST && a.pad_L) {  // padded layout: microbatch j of the range starts at row (j - mb_begin) * L
+      d.out_row = (uint32_t)out_row;
+      if (a.write_index) {
+        a.pos_ids[out_row] = (int32_t)p;
+        if (p == 0) {  // cu_seqlens: every sample writes its start; the last of a microbatch also the end
           const uint32_t j = pl.plan_sample_mb[q];
-          out_row += (uint64_t)(j - a.mb_begin) * a.pad_L - (pl.mb_row_off[j] - a.row_lo);
+          const uint64_t e = LIST ? cu0 + (q - q_lo) : (uint64_t)(q - a.q_lo) + (j - a.mb_begin);
+          a.cu[e] = (int32_t)(pl.sample_row_off[q] - pl.mb_row_off[j]);
+          if (q + 1 == pl.mb_sample_off[j + 1]) a.cu[e + 1] = (int32_t)(pl.sample_row_off[q + 1] - pl.mb_row_off[j]);
         }
-        d.out_row = (uint32_t)out_row;
-        if (a.write_index) {
-          a.pos_ids[out_row] = (int32_t)p;
-          if (p == 0) {  // cu_seqlens: every sample writes its start; the last of a microbatch also the end
-            const uint32_t j = pl.plan_sample_mb[q];
-            const uint64_t e = LIST ? cu0 + (q - q_lo) : (uint64_t)(q - a.q_lo) + (j - a.mb_begin);
-            a.cu[e] = (int32_t)(pl.sample_row_off[q] - pl.mb_row_off[j]);
-            if (q + 1 == pl.mb_sample_off[j + 1]) a.cu[e + 1] = (int32_t)(pl.sample_row_off[q + 1] - pl.mb_row_off[j]);
-          }
-        }
-        // Is position p inside a placeholder run?  The span table decides (last span with pos_start <= p).
-        const uint32_t sbase = slot * v.spans_per_sample, ns = v.s_n_spans[slot];
-        uint32_t lo = 0, hi = ns;
-        while (lo < hi) {
-          const uint32_t mid = (lo + hi) >> 1;
-          if (v.sp_pos[sbase + mid] <= p) lo = mid + 1; else hi = mid;
-        }
-        const uint32_t sid = sbase + lo - 1;
-        const bool in_run = lo > 0 && p < v.sp_pos[sid] + v.sp_tokens[sid];
-        if (!in_run) {
-          // token id, through the text page, then the embedding-table row
-          const uint64_t tp_gva = v.s_text_pages[(uint64_t)slot * v.text_pages_per_sample + p / kTextPageIds];
-          uint64_t off;
-          const uint64_t tpte = translate(v, tp_gva, &off);
-          int32_t id = -1;
-          const bool text_ok = (tpte & kPteValid) && (tpte & kPteText);  // e.g. a peer's page whose mapping was never imported
-          if (text_ok) id = reinterpret_cast<const int32_t*>(tpte & ~kPteFlagMask)[p % kTextPageIds];
-          if (!text_ok) {
-            note_error(v, a.call_seq, FT_ERR_BAD_GVA, (uint32_t)out_row);
-          } else if (id < 0 || (uint32_t)id >= a.vocab) {
-            note_error(v, a.call_seq, FT_ERR_BAD_TOKEN_ID, (uint32_t)out_row);
-          } else {
-            // a table row is one segment in device memory: the low address bits ride in off0
-            const uint64_t addr = reinterpret_cast<uint64_t>(a.table + (uint64_t)id * v.row_bytes);
-            d.seg[0] = addr & ~kPteFlagMask;
-            d.off0 = (uint32_t)(addr & kPteFlagMask);
-            d.nseg = 1;
-          }
+      }
+      // Is position p inside a placeholder run?  The span table decides (last span with pos_start <= p).
+      const uint32_t sbase = slot * v.spans_per_sample, ns = v.s_n_spans[slot];
+      uint32_t lo = 0, hi = ns;
+      while (lo < hi) {
+        const uint32_t mid = (lo + hi) >> 1;
+        if (v.sp_pos[sbase + mid] <= p) lo = mid + 1; else hi = mid;
+      }
+      const uint32_t sid = sbase + lo - 1;
+      const bool in_run = lo > 0 && p < v.sp_pos[sid] + v.sp_tokens[sid];
+      if (!in_run) {
+        // token id, through the text page, then the embedding-table row
+        const uint64_t tp_gva = v.s_text_pages[(uint64_t)slot * v.text_pages_per_sample + p / kTextPageIds];
+        uint64_t off;
+        const uint64_t tpte = translate(v, tp_gva, &off);
+        int32_t id = -1;
+        const bool text_ok = (tpte & kPteValid) && (tpte & kPteText);  // e.g. a peer's page whose mapping was never imported
+        if (text_ok) id = reinterpret_cast<const int32_t*>(tpte & ~kPteFlagMask)[p % kTextPageIds];
+        if (!text_ok) {
+          note_error(v, a.call_seq, FT_ERR_BAD_GVA, (uint32_t)out_row);
+        } else if (id < 0 || (uint32_t)id >= a.vocab) {
+          note_error(v, a.call_seq, FT_ERR_BAD_TOKEN_ID, (uint32_t)out_row);
         } else {
-          const uint64_t b = (uint64_t)(p - v.sp_pos[sid]) * v.row_bytes;  // byte offset inside the span image
-          const uint32_t o0 = (uint32_t)(b >> v.page_shift);
-          d.off0 = (uint32_t)(b & (v.page_bytes - 1));
-          d.shift = v.page_shift;
-          const uint32_t nseg = ((d.off0 + v.row_bytes - 1) >> v.page_shift) + 1;
-          bool ok = nseg <= kMaxSeg;
-          for (uint32_t s = 0; ok && s < nseg; ++s) {
-            uint64_t poff;
-            const uint64_t pte = translate(v, span_page_gva(v, sid, o0 + s), &poff);
-            ok = (pte & kPteValid) && !(pte & kPteText);
-            d.seg[s] = pte;
-          }
-          if (ok) d.nseg = nseg; else note_error(v, a.call_seq, FT_ERR_BAD_GVA, (uint32_t)out_row);
+          // a table row is one segment in device memory: the low address bits ride in off0
+          const uint64_t addr = reinterpret_cast<uint64_t>(a.table + (uint64_t)id * v.row_bytes);
+          d.seg[0] = addr & ~kPteFlagMask;
+          d.off0 = (uint32_t)(addr & kPteFlagMask);
+          d.nseg = 1;
         }
-      }
-      desc[lane] = d;
-    }
-    __syncthreads();
-    for (uint32_t r = warp; r < kTileRows; r += kGatherThreads / 32) {
-      const uint32_t nseg = desc[r].nseg;
-      if (nseg == 0) continue;
-      const uint32_t off0 = desc[r].off0, shift = desc[r].shift, mask = (1u << shift) - 1;
-      uint4* dst = reinterpret_cast<uint4*>(a.out + (uint64_t)desc[r].out_row * v.row_bytes);
-      auto src_of = [&](uint32_t x, bool* take) -> const uint4* {
-        const uint32_t ab = off0 + (x << 4);
-        const uint64_t pte = desc[r].seg[ab >> shift];
-        const bool host = (pte & kPteHost) != 0;
-        *take = MODE == kTierAll || (MODE == kTierHostOnly) == host;
-        return reinterpret_cast<const uint4*>((pte & ~kPteFlagMask) + (ab & mask));
-      };
-      // U vectors per lane in flight before the first store
-      for (uint32_t x0 = lane; x0 < row_vecs; x0 += 32 * U) {
-        uint4 val[U];
-        bool take[U];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-          const uint32_t x = x0 + 32 * u;
-          take[u] = false;
-          if (x < row_vecs) {
-            const uint4* s = src_of(x, &take[u]);
-            if (take[u]) val[u] = __ldcs(s);
-          }
+      } else {
+        const uint64_t b = (uint64_t)(p - v.sp_pos[sid]) * v.row_bytes;  // byte offset inside the span image
+        const uint32_t o0 = (uint32_t)(b >> v.page_shift);
+        d.off0 = (uint32_t)(b & (v.page_bytes - 1));
+        d.shift = v.page_shift;
+        const uint32_t nseg = ((d.off0 + v.row_bytes - 1) >> v.page_shift) + 1;
+        bool ok = nseg <= kMaxSeg;
+        for (uint32_t s = 0; ok && s < nseg; ++s) {
+          uint64_t poff;
+          const uint64_t pte = translate(v, span_page_gva(v, sid, o0 + s), &poff);
+          ok = (pte & kPteValid) && !(pte & kPteText);
+          d.seg[s] = pte;
         }
-#pragma unroll
-        for (int u = 0; u < U; ++u)
-          if (take[u]) __stcs(dst + x0 + 32 * u, val[u]);
+        if (ok) d.nseg = nseg; else note_error(v, a.call_seq, FT_ERR_BAD_GVA, (uint32_t)out_row);
       }
     }
-    __syncthreads();
+    desc[buf][lane] = d;
+  };
+
+  if (resolver) resolve(0);
+  __syncthreads();
+  for (uint32_t buf = 0;; buf ^= 1) {
+    if (!valid[buf]) break;
+    if (resolver) {
+      resolve(buf ^ 1);  // one unit ahead of the copy
+    } else {
+      for (uint32_t r = warp; r < R; r += kStreamWarps) {
+        const RowDesc& dr = desc[buf][r];
+        const uint32_t nseg = dr.nseg;
+        if (nseg == 0) continue;
+        const uint32_t off0 = dr.off0, shift = dr.shift, mask = (1u << shift) - 1;
+        uint4* dst = reinterpret_cast<uint4*>(a.out + (uint64_t)dr.out_row * v.row_bytes);
+        auto src_of = [&](uint32_t x, bool* take) -> const uint4* {
+          const uint32_t ab = off0 + (x << 4);
+          const uint64_t pte = dr.seg[ab >> shift];
+          const bool host = (pte & kPteHost) != 0;
+          *take = MODE == kTierAll || (MODE == kTierHostOnly) == host;
+          return reinterpret_cast<const uint4*>((pte & ~kPteFlagMask) + (ab & mask));
+        };
+        // U vectors per lane in flight before the first store
+        for (uint32_t x0 = lane; x0 < row_vecs; x0 += 32 * U) {
+          uint4 val[U];
+          bool take[U];
+#pragma unroll
+          for (int u = 0; u < U; ++u) {
+            const uint32_t x = x0 + 32 * u;
+            take[u] = false;
+            if (x < row_vecs) {
+              const uint4* s = src_of(x, &take[u]);
+              if (take[u]) val[u] = __ldcs(s);
+            }
+          }
+#pragma unroll
+          for (int u = 0; u < U; ++u)
+            if (take[u]) __stcs(dst + x0 + 32 * u, val[u]);
+        }
+      }
+    }
+    __syncthreads();  // desc[buf ^ 1] is complete, desc[buf] is free
   }
 }
 
@@ -278,7 +297,7 @@ namespace ft {
 // the index outputs are left to the caller.  Arguments are validated by the caller.
 int32_t gather_launch(ft_pool* p, const ft_plan* pl, uint32_t mb_begin, uint32_t mb_end, const void* embed_table,
                       uint32_t vocab, void* out_embeds, int32_t* out_cu, int32_t* out_pos, uint32_t pad_L, cudaStream_t st,
-                      const void* d_list, uint32_t n_list, uint64_t list_tiles, uint64_t list_rows) {
+                      const void* d_list, uint32_t n_list, uint64_t list_tiles, uint64_t list_rows, ClaimCounter* counter) {
   if (p->view.row_bytes > (kMaxSeg - 1) * 4096) return FT_ERR_CAPACITY;
   const PlanView pv = make_plan_view(pl);
   const bool listed = d_list != nullptr;
@@ -287,18 +306,23 @@ int32_t gather_launch(ft_pool* p, const ft_plan* pl, uint32_t mb_begin, uint32_t
   a.row_lo = pl->h_mb_row_off[mb_begin]; a.row_hi = pl->h_mb_row_off[mb_end];
   a.table = static_cast<const uint8_t*>(embed_table); a.vocab = vocab;
   a.out = static_cast<uint8_t*>(out_embeds); a.cu = out_cu; a.pos_ids = out_pos;
-  a.call_seq = p->call_seq; a.write_index = pad_L == 0; a.pad_L = pad_L;
+  a.call_seq = status_seq(p); a.write_index = pad_L == 0; a.pad_L = pad_L;
   a.list = static_cast<const ListEntry*>(d_list); a.n_list = n_list; a.list_tiles = list_tiles;
   const uint64_t n_tiles = listed ? list_tiles : (a.row_hi + kTileRows - 1) / kTileRows - a.row_lo / kTileRows;
   const uint64_t n_rows = listed ? list_rows : a.row_hi - a.row_lo;
   if (n_rows >> 32) return FT_ERR_CAPACITY;  // output row indices are 32-bit inside the kernel
-  a.tile_counter = p->view.status + 1;  // scratch word next to the status word
-  FT_CUDA(cudaMemsetAsync(a.tile_counter, 0, 8, st));
-  // the grid-stride tile loop assumes every CTA runs from the start: never launch more than fit at once
+  a.tile_counter = counter;
+  // never launch more CTAs than fit at once (every CTA claims until the units run out); a short range is cut into
+  // finer units, down to 4 rows, until there are about two per CTA
+  const uint64_t per_sm_cap = (p->cfg.hbm_pages == 0 && p->cfg.world_size == 1) ? 1 : (uint64_t)p->dev_ctas_per_sm;
+  const uint64_t full_grid = (uint64_t)p->sm_count * per_sm_cap;
+  a.sub_shift = 0;
+  while (a.sub_shift < 3 && (n_tiles << a.sub_shift) < 2 * full_grid) ++a.sub_shift;
+  const uint64_t n_units = n_tiles << a.sub_shift;
   auto launch = [&](auto kernel, int mode, uint64_t want_per_sm, const GatherArgs& args, cudaStream_t s) {
     const uint64_t resident = (uint64_t)std::max(1, p->occ_gather[mode][p->gather_unroll == 8 ? 1 : 0]);
     const uint64_t ctas = (uint64_t)p->sm_count * std::min<uint64_t>(want_per_sm, resident);
-    kernel<<<(unsigned)std::min<uint64_t>(n_tiles, ctas), kGatherThreads, 0, s>>>(p->view, pv, args);
+    kernel<<<(unsigned)std::min<uint64_t>(n_units, ctas), kGatherThreads, 0, s>>>(p->view, pv, args);
   };
   auto launch_mode = [&](auto mode_tag, const GatherArgs& args, uint64_t want_per_sm) {
     constexpr int M = decltype(mode_tag)::value;
@@ -309,7 +333,7 @@ int32_t gather_launch(ft_pool* p, const ft_plan* pl, uint32_t mb_begin, uint32_t
       if (u8) launch(k_gather<M, 8, false>, M, want_per_sm, args, st); else launch(k_gather<M, 4, false>, M, want_per_sm, args, st);
     }
   };
-  const uint64_t per_sm = (p->cfg.hbm_pages == 0 && p->cfg.world_size == 1) ? 1 : (uint64_t)p->dev_ctas_per_sm;
+  const uint64_t per_sm = per_sm_cap;
   // one launch when only one tier can be a source (own and imported bindings); otherwise one launch per tier
   const bool host_sources = p->cfg.host_pages != 0 || p->peer_host_frames;
   const bool only_host = p->cfg.hbm_pages == 0 && !(p->cfg.world_size > 1);
@@ -361,8 +385,17 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_gather_packed(ft_
     if (rc0 != FT_OK) return rc0;
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  ft_call_ctx* cx = nullptr;
   {
-    const int32_t rc1 = gather_launch(p, pl, mb_begin, mb_end, embed_table, vocab, out_embeds, out_cu, out_pos, 0, st, nullptr, 0, 0, 0);
+    const int32_t rc1 = ctx_acquire(p, 1, 0, 0, &cx, false, st);  // for its claim counter
+    if (rc1 != FT_OK) return rc1;
+  }
+  {
+    const int32_t rc1 = gather_launch(p, pl, mb_begin, mb_end, embed_table, vocab, out_embeds, out_cu, out_pos, 0, st, nullptr, 0, 0, 0, cx->counters);
+    if (rc1 != FT_OK) return rc1;
+  }
+  {
+    const int32_t rc1 = ctx_release(p, cx, st);
     if (rc1 != FT_OK) return rc1;
   }
   const_cast<ft_plan*>(pl)->last_stream = st;
@@ -399,19 +432,25 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_gather_list(ft_po
   }
   if ((rows >> 32) || (cu >> 32)) return FT_ERR_CAPACITY;  // output row indices are 32-bit inside the kernels
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t bytes = entries.size() * sizeof(ListEntry);
+  ft_call_ctx* cx = nullptr;
+  {
+    int32_t rc1 = ctx_acquire(p, 1, bytes, bytes, &cx);
+    if (rc1 != FT_OK) return rc1;
+    memcpy(cx->h, entries.data(), bytes);
+    if ((rc1 = ctx_upload(p, cx, bytes)) != FT_OK) return rc1;  // on the metadata stream; begin_consumer orders `st` behind it
+  }
   {
     const int32_t rc0 = begin_consumer(p, st);
     if (rc0 != FT_OK) return rc0;
   }
-  void* d = nullptr;
-  const size_t bytes = entries.size() * sizeof(ListEntry);
   {
-    const int32_t rc1 = stage_upload(p, 1, entries.data(), bytes, bytes, st, &d);
-    if (rc1 != FT_OK) return rc1;
+    const int32_t rc2 = gather_launch(p, pl, 0, pl->n_mb, embed_table, vocab, out_embeds, out_cu, out_pos, 0, st, cx->d, n_list, tiles, rows, cx->counters);
+    if (rc2 != FT_OK) return rc2;
   }
   {
-    const int32_t rc2 = gather_launch(p, pl, 0, pl->n_mb, embed_table, vocab, out_embeds, out_cu, out_pos, 0, st, d, n_list, tiles, rows);
-    if (rc2 != FT_OK) return rc2;
+    const int32_t rc3 = ctx_release(p, cx, st);
+    if (rc3 != FT_OK) return rc3;
   }
   const_cast<ft_plan*>(pl)->last_stream = st;
   return end_consumer(p, st);

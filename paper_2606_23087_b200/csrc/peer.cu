@@ -289,27 +289,32 @@ FT_API int32_t pool_export_samples(ft_pool* p, const uint32_t* slot, uint32_t n,
   const size_t o_sid = 0, o_poff = (size_t)ns * 4, o_slot = o_poff + (size_t)(ns + 1) * 4, o_tpoff = o_slot + (size_t)n * 4;
   const size_t blob_bytes = align_up_sz(o_tpoff + (size_t)(n + 1) * 4, 256);
   const size_t o_out = blob_bytes, total_bytes = o_out + 8 * (total_pages + total_text);
-  std::vector<uint8_t> blob(blob_bytes, 0);
-  if (ns) memcpy(blob.data() + o_sid, span_id.data(), (size_t)ns * 4);
-  memcpy(blob.data() + o_poff, page_off.data(), (size_t)(ns + 1) * 4);
-  memcpy(blob.data() + o_slot, slot, (size_t)n * 4);
-  memcpy(blob.data() + o_tpoff, tp_off.data(), (size_t)(n + 1) * 4);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  void* d = nullptr;
-  int32_t rc = begin_consumer(p, st);  // the lists may still be being written on another stream
+  ft_call_ctx* cx = nullptr;
+  int32_t rc = ctx_acquire(p, 1, blob_bytes, total_bytes, &cx);
   if (rc != FT_OK) return rc;
-  rc = stage_upload(p, 1, blob.data(), blob_bytes, total_bytes, st, &d);
-  if (rc != FT_OK) return rc;
-  uint8_t* db = static_cast<uint8_t*>(d);
+  uint8_t* hb = static_cast<uint8_t*>(cx->h);
+  if (ns) memcpy(hb + o_sid, span_id.data(), (size_t)ns * 4);
+  memcpy(hb + o_poff, page_off.data(), (size_t)(ns + 1) * 4);
+  memcpy(hb + o_slot, slot, (size_t)n * 4);
+  memcpy(hb + o_tpoff, tp_off.data(), (size_t)(n + 1) * 4);
+  if ((rc = ctx_upload(p, cx, blob_bytes)) != FT_OK) return rc;
+  uint8_t* db = static_cast<uint8_t*>(cx->d);
   ListCall lc{ns, n, reinterpret_cast<uint32_t*>(db + o_sid), reinterpret_cast<uint32_t*>(db + o_poff),
               reinterpret_cast<uint32_t*>(db + o_slot), reinterpret_cast<uint32_t*>(db + o_tpoff)};
   const uint64_t items = total_pages + total_text;
-  k_export_lists<<<(unsigned)((items + 255) / 256), 256, 0, st>>>(p->view, lc, (uint32_t)total_pages, (uint32_t)total_text,
-                                                                   reinterpret_cast<uint64_t*>(db + o_out));
+  // the page lists are metadata: the list kernel runs on the metadata stream, behind the allocations that wrote them
+  k_export_lists<<<(unsigned)((items + 255) / 256), 256, 0, p->meta>>>(p->view, lc, (uint32_t)total_pages, (uint32_t)total_text,
+                                                                       reinterpret_cast<uint64_t*>(db + o_out));
   p->gpu_launches++;
-  FT_CUDA(cudaMemcpyAsync(pg, db + o_out, 8 * items, cudaMemcpyDeviceToHost, st));
+  FT_CUDA(cudaMemcpyAsync(pg, db + o_out, 8 * items, cudaMemcpyDeviceToHost, p->meta));
+  if ((rc = ctx_release(p, cx, p->meta)) != FT_OK) return rc;
+  FT_CUDA(cudaStreamSynchronize(p->meta));
+  // a consumer will read the pages themselves as soon as it holds the descriptors: the copies that fill them (on
+  // the producer side's stream and on `stream`) are complete when this call returns
+  if (p->have_producer_ev) FT_CUDA(cudaEventSynchronize(p->ev_producer));
   FT_CUDA(cudaStreamSynchronize(st));
-  return end_consumer(p, st);
+  return FT_OK;
 }
 
 FT_API int32_t pool_import_samples(ft_pool* p, const uint32_t* local_slot, uint32_t n, const void* buf, uint64_t bytes,
@@ -377,29 +382,31 @@ FT_API int32_t pool_import_samples(ft_pool* p, const uint32_t* local_slot, uint3
   const size_t o_poff = take(4ull * (ns + 1)), o_boff = take(4ull * (ns + 1)), o_tpoff = take(4ull * (n + 1));
   const size_t o_grid = take(16ull * ns);
   const size_t blob_bytes = align_up_sz(off, 256), o_head = blob_bytes, total_bytes = o_head + 16;
-  std::vector<uint8_t> blob(blob_bytes, 0);
-  memcpy(blob.data() + o_gva, pg, 8 * (pages + text));
-  memcpy(blob.data() + o_slot, local_slot, 4ull * n);
-  memcpy(blob.data() + o_seq, seq.data(), 4ull * n);
-  memcpy(blob.data() + o_nsp, nsp.data(), 4ull * n);
-  memcpy(blob.data() + o_sbeg, sbeg.data(), 4ull * (n + 1));
-  if (ns) memcpy(blob.data() + o_grid, grid.data(), 16ull * ns);
-  if (ns) { memcpy(blob.data() + o_pos, pos.data(), 4ull * ns); memcpy(blob.data() + o_tok, tok.data(), 4ull * ns); memcpy(blob.data() + o_npg, npg.data(), 4ull * ns); }
-  memcpy(blob.data() + o_poff, poff.data(), 4ull * (ns + 1));
-  memcpy(blob.data() + o_boff, boff.data(), 4ull * (ns + 1));
-  memcpy(blob.data() + o_tpoff, tpoff.data(), 4ull * (n + 1));
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  void* d = nullptr;
-  int32_t rc = stage_upload(p, 0, blob.data(), blob_bytes, total_bytes, st, &d);
+  ft_call_ctx* cx = nullptr;
+  int32_t rc = ctx_acquire(p, 0, blob_bytes, total_bytes, &cx);
   if (rc != FT_OK) return rc;
-  uint8_t* db = static_cast<uint8_t*>(d);
+  uint8_t* hb = static_cast<uint8_t*>(cx->h);
+  memcpy(hb + o_gva, pg, 8 * (pages + text));
+  memcpy(hb + o_slot, local_slot, 4ull * n);
+  memcpy(hb + o_seq, seq.data(), 4ull * n);
+  memcpy(hb + o_nsp, nsp.data(), 4ull * n);
+  memcpy(hb + o_sbeg, sbeg.data(), 4ull * (n + 1));
+  if (ns) memcpy(hb + o_grid, grid.data(), 16ull * ns);
+  if (ns) { memcpy(hb + o_pos, pos.data(), 4ull * ns); memcpy(hb + o_tok, tok.data(), 4ull * ns); memcpy(hb + o_npg, npg.data(), 4ull * ns); }
+  memcpy(hb + o_poff, poff.data(), 4ull * (ns + 1));
+  memcpy(hb + o_boff, boff.data(), 4ull * (ns + 1));
+  memcpy(hb + o_tpoff, tpoff.data(), 4ull * (n + 1));
+  if ((rc = ctx_upload(p, cx, blob_bytes)) != FT_OK) return rc;
+  uint8_t* db = static_cast<uint8_t*>(cx->d);
   auto U = [&](size_t o) { return reinterpret_cast<uint32_t*>(db + o); };
   ImportCall ic{ns, n, U(o_slot), U(o_seq), U(o_nsp), U(o_sbeg), U(o_pos), U(o_tok), U(o_npg), U(o_poff), U(o_boff), U(o_tpoff),
                 reinterpret_cast<uint64_t*>(db + o_gva), U(o_head), reinterpret_cast<const uint4*>(db + o_grid)};
-  k_import_pop<<<1, 1, 0, st>>>(p->view, ic, (uint32_t)blocks);
+  k_import_pop<<<1, 1, 0, p->meta>>>(p->view, ic, (uint32_t)blocks);
   const uint64_t items = std::max<uint64_t>(pages + text, n);
-  k_import_fill<<<(unsigned)((items + 255) / 256), 256, 0, st>>>(p->view, ic, (uint32_t)pages, (uint32_t)text);
+  k_import_fill<<<(unsigned)((items + 255) / 256), 256, 0, p->meta>>>(p->view, ic, (uint32_t)pages, (uint32_t)text);
   FT_CUDA(cudaGetLastError());
+  if ((rc = ctx_release(p, cx, p->meta)) != FT_OK) return rc;
   p->gpu_launches += 2;
 
   for (uint32_t i = 0, g = 0; i < n; ++i) {
@@ -415,5 +422,6 @@ FT_API int32_t pool_import_samples(ft_pool* p, const uint32_t* local_slot, uint3
     p->live_samples++; p->live_spans += nsp[i];
   }
   p->free_blocks -= blocks;
+  if ((rc = meta_to(p, st)) != FT_OK) return rc;  // what the caller queues on `stream` next sees the imported samples
   return end_producer(p, st);
 }

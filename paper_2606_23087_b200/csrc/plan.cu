@@ -423,7 +423,11 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_plan_microbatches
     *out = pl;
     return FT_OK;
   }
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // The plan reads the pool's tables only (lengths and states), never embedding bytes or token ids: all of its
+  // kernels run on the metadata stream, so a plan requested right after the last producer call is made while that
+  // call's copy is still streaming on the caller's stream.
+  (void)stream;
+  cudaStream_t st = p->meta;
   const uint64_t n_tiles = (total_tokens + 31) / 32 + 1;
 
   // one device block for every plan array
@@ -464,14 +468,16 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_plan_microbatches
     cudaError_t e__ = (call);                                                               \
     if (e__ != cudaSuccess) { rc = ft::cuda_fail(e__, #call); plan_destroy(pl); return rc; } \
   } while (0)
-  // the sample table may still be being written on another stream
-  rc = begin_consumer(p, st);
+  // the slot list goes up through a call context (scratch front), then into the plan
+  ft_call_ctx* cx = nullptr;
+  rc = ctx_acquire(p, 1, (size_t)n * 4, (size_t)n * 4, &cx);
   if (rc != FT_OK) { plan_destroy(pl); return rc; }
-  // the slot list goes up through the pool's staging ring (scratch front), then into the plan
-  void* d_up = nullptr;
-  rc = stage_upload(p, 1, slot, (size_t)n * 4, (size_t)n * 4, st, &d_up);
+  memcpy(cx->h, slot, (size_t)n * 4);
+  rc = ctx_upload(p, cx, (size_t)n * 4);
   if (rc != FT_OK) { plan_destroy(pl); return rc; }
-  CK(cudaMemcpyAsync(pl->d_slots, d_up, (size_t)n * 4, cudaMemcpyDeviceToDevice, st));
+  CK(cudaMemcpyAsync(pl->d_slots, cx->d, (size_t)n * 4, cudaMemcpyDeviceToDevice, st));
+  rc = ctx_release(p, cx, st);
+  if (rc != FT_OK) { plan_destroy(pl); return rc; }
   CK(cudaMemsetAsync(pl->d_rank_cnt, 0, (size_t)N * 4, st));
 
   const unsigned gb = (n + 255) / 256;
@@ -480,6 +486,10 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_plan_microbatches
   // shared memory plan of k_bestfit: bitmaps, staging chunk, then the stack heads and records if they fit
   size_t words = 0;
   { uint32_t w = (L + 1 + 31) / 32; for (int l = 0; l < 4; ++l) { words += w + 1; w = (w + 31) / 32; } }  // one pad word per level
+  // (The packing kernel wants most of an SM's storage as shared memory, so it cannot start on an SM that still holds
+  // CTAs of a copy kernel with their small shared-memory split; keeping its tables in global memory instead lets it
+  // run beside the copies, but every dependent access then pays the loaded memory system's latency: 4.5 ms instead
+  // of 0.25 ms for 512 samples.  It therefore keeps its tables in shared memory and runs when an SM is free.)
   const size_t fixed = (words + 3 * (size_t)kFitChunk) * 4 + 16;
   const size_t limit = kBestfitSmemLimit;
   const size_t head_bytes = ((size_t)L + 1) * 4;
@@ -494,37 +504,47 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_plan_microbatches
     const bool all_recs = rec_cap >= n;
     auto fit = head_in_smem ? (all_recs ? k_bestfit<true, true> : k_bestfit<true, false>)
                             : (all_recs ? k_bestfit<false, true> : k_bestfit<false, false>);
-    fit<<<1, 1024, used, st>>>(d_pk_len, n, L, d_head, d_recs, rec_cap, d_pk_mb, pl->d_sample_rank, pl->d_mb_residual,
+    fit<<<1, n > 8192 ? 1024 : 256, used, st>>>(d_pk_len, n, L, d_head, d_recs, rec_cap, d_pk_mb, pl->d_sample_rank, pl->d_mb_residual,
                                pl->d_mb_tokens, pl->d_mb_lmax, pl->d_mb_count, pl->d_scalars);
   }
-  k_mb_finalize<<<1, 1024, 0, st>>>(pl->d_mb_tokens, pl->d_mb_count, pl->d_mb_sample_off, pl->d_mb_row_off, pl->d_scalars);
+  k_mb_finalize<<<1, scan_threads(n), 0, st>>>(pl->d_mb_tokens, pl->d_mb_count, pl->d_mb_sample_off, pl->d_mb_row_off, pl->d_scalars);
   k_plan_scatter<<<gb, 256, 0, st>>>(pl->d_slots, d_pk_t, d_pk_len, d_pk_mb, pl->d_sample_rank, pl->d_mb_sample_off, n,
                                      pl->d_mb_samples, pl->d_plan_len, pl->d_plan_sample_mb, pl->d_sample_mb);
   k_mb_cost<<<gb, 256, 0, st>>>(cfg->coef_A, cfg->coef_B, f_sumsq, pl->d_mb_tokens, pl->d_mb_lmax, pl->d_mb_sample_off,
                                 pl->d_plan_len, pl->d_mb_cost, pl->d_scalars);
-  k_row_offsets<<<1, 1024, 0, st>>>(pl->d_plan_len, n, pl->d_sample_row_off);
+  k_row_offsets<<<1, scan_threads(n), 0, st>>>(pl->d_plan_len, n, pl->d_sample_row_off);
   k_tiles<<<gb, 256, 0, st>>>(pl->d_sample_row_off, n, pl->d_tile_first_sample);
   k_bucket<<<gb, 256, 0, st>>>(pl->d_mb_cost, K, (cfg->flags & FT_PLAN_AUTO_K) ? N : 0u, pl->d_scalars, pl->d_mb_bucket);
   k_sort_deal<<<gb, 256, 0, st>>>(pl->d_mb_cost, pl->d_mb_bucket, N, f_carry, pl->d_scalars, pl->d_mb_pos, pl->d_mb_rank);
   k_rank_index<<<gb, 256, 0, st>>>(pl->d_mb_pos, pl->d_mb_rank, pl->d_scalars, d_mb_idx, pl->d_rank_cnt);
-  k_rank_scan<<<1, 1024, 0, st>>>(pl->d_rank_cnt, N, pl->d_rank_mb_off);
+  k_rank_scan<<<1, scan_threads(N), 0, st>>>(pl->d_rank_cnt, N, pl->d_rank_mb_off);
   k_rank_lists<<<gb, 256, 0, st>>>(pl->d_mb_rank, d_mb_idx, pl->d_rank_mb_off, pl->d_scalars, pl->d_rank_mbs);
   CK(cudaGetLastError());
   p->gpu_launches += 13;
 
-  uint32_t sc[SC_COUNT];
-  CK(cudaMemcpyAsync(sc, pl->d_scalars, sizeof(sc), cudaMemcpyDeviceToHost, st));
+  // the summary and the two offset arrays the host sizes assemblies with come back in one go (n + 1 entries bound
+  // n_mb + 1), into a pinned landing zone, behind one synchronisation of the metadata stream
+  const size_t rb_sc = 0, rb_so = align_up(sizeof(uint32_t) * SC_COUNT, 16), rb_ro = align_up(rb_so + n1 * 4, 16), rb_bytes = rb_ro + n1 * 8;
+  if (p->plan_pinned_cap < rb_bytes) {
+    if (p->plan_pinned) CK(cudaFreeHost(p->plan_pinned));
+    p->plan_pinned = nullptr; p->plan_pinned_cap = 0;
+    size_t cap = 1 << 16;
+    while (cap < rb_bytes) cap <<= 1;
+    CK(cudaHostAlloc(&p->plan_pinned, cap, cudaHostAllocDefault));
+    p->plan_pinned_cap = cap;
+  }
+  uint8_t* rb = static_cast<uint8_t*>(p->plan_pinned);
+  CK(cudaMemcpyAsync(rb + rb_sc, pl->d_scalars, sizeof(uint32_t) * SC_COUNT, cudaMemcpyDeviceToHost, st));
+  CK(cudaMemcpyAsync(rb + rb_so, pl->d_mb_sample_off, n1 * 4, cudaMemcpyDeviceToHost, st));
+  CK(cudaMemcpyAsync(rb + rb_ro, pl->d_mb_row_off, n1 * 8, cudaMemcpyDeviceToHost, st));
   CK(cudaStreamSynchronize(st));
+  const uint32_t* sc = reinterpret_cast<const uint32_t*>(rb + rb_sc);
   pl->n_mb = sc[SC_NMB];
   pl->max_mb_tokens = sc[SC_MAXTOK];
   pl->total_tokens = (uint64_t)sc[SC_TOTAL_LO] | ((uint64_t)sc[SC_TOTAL_HI] << 32);
-  pl->h_mb_sample_off.resize((size_t)pl->n_mb + 1);
-  pl->h_mb_row_off.resize((size_t)pl->n_mb + 1);
-  CK(cudaMemcpy(pl->h_mb_sample_off.data(), pl->d_mb_sample_off, ((size_t)pl->n_mb + 1) * 4, cudaMemcpyDeviceToHost));
-  CK(cudaMemcpy(pl->h_mb_row_off.data(), pl->d_mb_row_off, ((size_t)pl->n_mb + 1) * 8, cudaMemcpyDeviceToHost));
+  pl->h_mb_sample_off.assign(reinterpret_cast<const uint32_t*>(rb + rb_so), reinterpret_cast<const uint32_t*>(rb + rb_so) + pl->n_mb + 1);
+  pl->h_mb_row_off.assign(reinterpret_cast<const uint64_t*>(rb + rb_ro), reinterpret_cast<const uint64_t*>(rb + rb_ro) + pl->n_mb + 1);
 #undef CK
-  rc = end_consumer(p, st);
-  if (rc != FT_OK) { plan_destroy(pl); return rc; }
   *out = pl;
   return FT_OK;
 }

@@ -20,7 +20,8 @@
 
 namespace ft {
 
-static char g_last_error[512] = "";
+// one caller thread per pool, so a per-thread string is per pool as far as any caller can tell
+static thread_local char g_last_error[512] = "";
 
 int32_t cuda_fail(cudaError_t e, const char* what) {
   snprintf(g_last_error, sizeof(g_last_error), "%s: %s", what, cudaGetErrorString(e));
@@ -43,33 +44,46 @@ static void seeded_shuffle(std::vector<uint32_t>& a, uint64_t seed) {
   }
 }
 
-int32_t stage_upload(ft_pool* p, int arena, const void* src, size_t bytes, size_t total_bytes, cudaStream_t st, void** d_out) {
-  ft_staging& s = p->staging;
-  const int i = s.next;
-  s.next = (i + 1) % ft_staging::kBufs;
-  if (s.busy[i]) { FT_CUDA(cudaEventSynchronize(s.ev[i])); s.busy[i] = false; }
-  if (!s.ev[i]) FT_CUDA(cudaEventCreateWithFlags(&s.ev[i], cudaEventDisableTiming));
-  if (s.cap[i] < bytes) {
-    if (s.h[i]) FT_CUDA(cudaFreeHost(s.h[i]));
+int32_t ctx_acquire(ft_pool* p, int side, size_t blob_bytes, size_t total_bytes, ft_call_ctx** out, bool on_meta, cudaStream_t first_user) {
+  ft_call_ctx& c = p->ctx[side][p->ctx_next[side]];
+  p->ctx_next[side] = (p->ctx_next[side] + 1) % kCallCtx;
+  if (c.busy_up) { FT_CUDA(cudaEventSynchronize(c.ev_up)); c.busy_up = false; }  // the upload that last read `h` is over
+  if (c.hcap < blob_bytes) {
+    if (c.h) FT_CUDA(cudaFreeHost(c.h));
     size_t cap = 1 << 16;
-    while (cap < bytes) cap <<= 1;
-    s.h[i] = nullptr; s.cap[i] = 0;
-    FT_CUDA(cudaHostAlloc(&s.h[i], cap, cudaHostAllocDefault));
-    s.cap[i] = cap;
+    while (cap < blob_bytes) cap <<= 1;
+    c.h = nullptr; c.hcap = 0;
+    FT_CUDA(cudaHostAlloc(&c.h, cap, cudaHostAllocDefault));
+    c.hcap = cap;
   }
-  memcpy(s.h[i], src, bytes);
-  if (p->scratch_cap[arena] < total_bytes) {
-    if (p->d_scratch[arena]) FT_CUDA(cudaFree(p->d_scratch[arena]));  // synchronises: no kernel still reads the old scratch
+  if (c.dcap < total_bytes) {
+    if (c.busy_done) { FT_CUDA(cudaEventSynchronize(c.ev_done)); c.busy_done = false; }  // nobody reads the old scratch
+    if (c.d) FT_CUDA(cudaFree(c.d));
     size_t cap = 1 << 20;
     while (cap < total_bytes) cap <<= 1;
-    p->d_scratch[arena] = nullptr; p->scratch_cap[arena] = 0;
-    FT_CUDA(cudaMalloc(&p->d_scratch[arena], cap));
-    p->scratch_cap[arena] = cap;
+    c.d = nullptr; c.dcap = 0;
+    FT_CUDA(cudaMalloc(&c.d, cap));
+    c.dcap = cap;
   }
-  FT_CUDA(cudaMemcpyAsync(p->d_scratch[arena], s.h[i], bytes, cudaMemcpyHostToDevice, st));
-  FT_CUDA(cudaEventRecord(s.ev[i], st));
-  s.busy[i] = true;
-  *d_out = p->d_scratch[arena];
+  if (c.busy_done) { FT_CUDA(cudaStreamWaitEvent(on_meta ? p->meta : first_user, c.ev_done, 0)); c.busy_done = false; }
+  *out = &c;
+  return FT_OK;
+}
+
+int32_t ctx_upload(ft_pool* p, ft_call_ctx* c, size_t bytes) {
+  p->meta_seq++;
+  if (bytes) {
+    FT_CUDA(cudaMemcpyAsync(c->d, c->h, bytes, cudaMemcpyHostToDevice, p->meta));
+    FT_CUDA(cudaEventRecord(c->ev_up, p->meta));
+    c->busy_up = true;
+  }
+  return FT_OK;
+}
+
+int32_t ctx_release(ft_pool* p, ft_call_ctx* c, cudaStream_t last) {
+  (void)p;
+  FT_CUDA(cudaEventRecord(c->ev_done, last));
+  c->busy_done = true;
   return FT_OK;
 }
 
@@ -214,7 +228,6 @@ __global__ void __launch_bounds__(1024) k_alloc_scan(PoolView v, WriteCall c) {
   }
   if (threadIdx.x == 0) {
     c.page_off[c.n] = (uint32_t)cp; c.blk_off[c.n] = (uint32_t)cb; c.chunk_off[c.n] = cc;
-    v.status[2] = 0; v.status[3] = 0;  // k_scatter's claim counters (main and side stream) start at zero
     RingState s = *v.ring_state;
     c.heads[0] = s.head;
     s.head = (uint32_t)((s.head + cp) % v.ring_cap); s.count -= (uint32_t)cp;
@@ -267,10 +280,10 @@ enum { kTierAll = 0, kTierDeviceOnly = 1, kTierHostOnly = 2 };
 
 template <int MODE, bool F32>
 __global__ void __launch_bounds__(256, F32 ? 4 : 6) k_scatter(PoolView v, WriteCall c, uint64_t total_chunks, uint64_t per_cta,
-                                                              unsigned long long* group_counter) {
+                                                              ClaimCounter* group_counter) {
   // Work unit = a chunk of 2^chunk_shift bytes of one span's image (the page size does not cap it).  Groups of
-  // per_cta consecutive chunks are claimed in order from a device counter (zeroed before the launch), so at
-  // any moment the grid streams one compact window of the call's bytes.  Inside a chunk warp w owns the w-th eighth and walks it in 2 KiB
+  // per_cta consecutive chunks are claimed in order from a device counter (zero at rest: the grid's last CTA puts
+  // it back), so at any moment the grid streams one compact window of the call's bytes.  Inside a chunk warp w owns the w-th eighth and walks it in 2 KiB
   // batches (four 512-byte lines per lane in flight); a batch never straddles a page (pages are >= 4 KiB and
   // batches 2 KiB-aligned), and each warp resolves its batch's frame through the span's page list and the
   // page table, once per page.
@@ -280,10 +293,13 @@ __global__ void __launch_bounds__(256, F32 ? 4 : 6) k_scatter(PoolView v, WriteC
   __shared__ uint64_t next_group;
   for (;;) {
     __syncthreads();  // everyone has read the previous claim
-    if (threadIdx.x == 0) next_group = atomicAdd(group_counter, 1ull);
+    if (threadIdx.x == 0) next_group = atomicAdd(&group_counter->claim, 1ull);
     __syncthreads();
     const uint64_t c0 = next_group * per_cta;
-    if (c0 >= total_chunks) break;
+    if (c0 >= total_chunks) {
+      if (threadIdx.x == 0) claim_release(group_counter);
+      break;
+    }
     const uint64_t c1 = min(total_chunks, c0 + per_cta);
     uint32_t q;
     if (c.chunk_span) {
@@ -358,10 +374,10 @@ __global__ void __launch_bounds__(256, F32 ? 4 : 6) k_scatter(PoolView v, WriteC
 // launches k_scatter<MODE, F32> on a grid of at most `max_ctas` CTAs, never more than fit on the GPU at once
 // (the round-robin deal assumes every CTA runs from the start)
 template <int MODE, bool F32>
-static void launch_scatter(ft_pool* p, const WriteCall& w, uint64_t total_chunks, uint64_t max_ctas, cudaStream_t s) {
-  // one claim counter per stream the library launches on: main (word 2) and side (word 3) of the status block
-  // (k_alloc_scan, which precedes every scatter launch of the call, zeroes them)
-  unsigned long long* counter = p->view.status + (s == p->side_stream[0] ? 3 : 2);
+static void launch_scatter(ft_pool* p, const WriteCall& w, uint64_t total_chunks, uint64_t max_ctas, cudaStream_t s,
+                           ClaimCounter* counters) {
+  // one claim counter per stream the call launches on: main ([0]) and side ([1])
+  ClaimCounter* counter = counters + (s == p->side_stream[0] ? 1 : 0);
   const int per_sm = std::max(1, p->occ_scatter[MODE][F32 ? 1 : 0]);
   // HBM streams best with a bounded amount of loads in flight per SM; more resident warps only deepen the DRAM
   // queues (measured optimum: 4 CTAs/SM, one chunk per claim)
@@ -373,10 +389,10 @@ static void launch_scatter(ft_pool* p, const WriteCall& w, uint64_t total_chunks
 }
 
 static void launch_scatter_any(ft_pool* p, int mode, bool f32, const WriteCall& w, uint64_t total_chunks, uint64_t max_ctas,
-                               cudaStream_t s) {
-  if (mode == kTierAll) { if (f32) launch_scatter<kTierAll, true>(p, w, total_chunks, max_ctas, s); else launch_scatter<kTierAll, false>(p, w, total_chunks, max_ctas, s); }
-  else if (mode == kTierDeviceOnly) { if (f32) launch_scatter<kTierDeviceOnly, true>(p, w, total_chunks, max_ctas, s); else launch_scatter<kTierDeviceOnly, false>(p, w, total_chunks, max_ctas, s); }
-  else { if (f32) launch_scatter<kTierHostOnly, true>(p, w, total_chunks, max_ctas, s); else launch_scatter<kTierHostOnly, false>(p, w, total_chunks, max_ctas, s); }
+                               cudaStream_t s, ClaimCounter* cc) {
+  if (mode == kTierAll) { if (f32) launch_scatter<kTierAll, true>(p, w, total_chunks, max_ctas, s, cc); else launch_scatter<kTierAll, false>(p, w, total_chunks, max_ctas, s, cc); }
+  else if (mode == kTierDeviceOnly) { if (f32) launch_scatter<kTierDeviceOnly, true>(p, w, total_chunks, max_ctas, s, cc); else launch_scatter<kTierDeviceOnly, false>(p, w, total_chunks, max_ctas, s, cc); }
+  else { if (f32) launch_scatter<kTierHostOnly, true>(p, w, total_chunks, max_ctas, s, cc); else launch_scatter<kTierHostOnly, false>(p, w, total_chunks, max_ctas, s, cc); }
 }
 
 // Host-tier pages of a producer call (bf16 source), page by page: source bytes -> shared -> host frame with
@@ -416,6 +432,41 @@ __global__ void __launch_bounds__(32) k_scatter_host_bulk(PoolView v, WriteCall 
   }
   ring.drain();
   if (ring.lost && lane == 0) note_error(v, call_seq, FT_ERR_TIMEOUT, blockIdx.x);
+}
+
+// The byte copy of a producer call, shared by pool_write_embeddings and its no-allocation variant: HBM-bound chunks on
+// the caller's stream, host-bound chunks beside them on the producer side's second stream.
+static int32_t launch_write_copies(ft_pool* p, const WriteCall& w, uint64_t total_chunks, bool f32, cudaStream_t st, ClaimCounter* cc,
+                                   bool profile) {
+  const ft_pool_config& c = p->cfg;
+  auto launch = [&](int mode, cudaStream_t s) {
+    const bool host_class = mode == kTierHostOnly || (mode == kTierAll && c.hbm_pages == 0);
+    if (profile) prof_begin(p, host_class ? FT_K_SCATTER_HOST : FT_K_SCATTER_DEVICE, s);
+    launch_scatter_any(p, mode, f32, w, total_chunks, host_class ? (uint64_t)p->host_store_ctas : ~0ull, s, cc);
+    if (profile) prof_end(p, s);
+    p->gpu_launches++;
+  };
+  if (c.host_pages == 0 || c.hbm_pages == 0) {
+    launch(kTierAll, st);
+  } else {
+    FT_CUDA(cudaEventRecord(p->fork_ev[0], st));
+    FT_CUDA(cudaStreamWaitEvent(p->side_stream[0], p->fork_ev[0], 0));
+    if (profile) prof_begin(p, FT_K_SCATTER_HOST, p->side_stream[0]);
+    // bf16 source: bulk-async copies through shared memory.  fp32 source: the cast needs the values in
+    // registers, and stores to host memory are posted (no latency to hide), so a few vector-store CTAs do it
+    if (f32) {
+      launch_scatter<kTierHostOnly, true>(p, w, total_chunks, (uint64_t)p->host_store_ctas, p->side_stream[0], cc);
+    } else {
+      k_scatter_host_bulk<<<(unsigned)p->host_ctas, 32, kBulkSmemBytes, p->side_stream[0]>>>(p->view, w, status_seq(p));
+    }
+    if (profile) prof_end(p, p->side_stream[0]);
+    p->gpu_launches++;
+    FT_CUDA(cudaEventRecord(p->join_ev[0], p->side_stream[0]));
+    launch(kTierDeviceOnly, st);
+    FT_CUDA(cudaStreamWaitEvent(st, p->join_ev[0], 0));
+  }
+  FT_CUDA(cudaGetLastError());
+  return FT_OK;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -545,11 +596,18 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_destroy(ft_pool* 
   if (!p) return FT_ERR_INVALID_ARG;
   cudaSetDevice(p->device);
   cudaDeviceSynchronize();
-  for (int i = 0; i < ft_staging::kBufs; ++i) {
-    if (p->staging.h[i]) cudaFreeHost(p->staging.h[i]);
-    if (p->staging.ev[i]) cudaEventDestroy(p->staging.ev[i]);
+  for (ft_call_ctx* ring : {p->ctx[0], p->ctx[1]}) for (int i = 0; i < kCallCtx; ++i) {
+    ft_call_ctx& c = ring[i];
+    if (c.h) cudaFreeHost(c.h);
+    if (c.d) cudaFree(c.d);
+    if (c.ev_up) cudaEventDestroy(c.ev_up);
+    if (c.ev_done) cudaEventDestroy(c.ev_done);
   }
-  for (int a = 0; a < 2; ++a) if (p->d_scratch[a]) cudaFree(p->d_scratch[a]);
+  if (p->plan_pinned) cudaFreeHost(p->plan_pinned);
+  if (p->meta) cudaStreamDestroy(p->meta);
+  if (p->ev_meta) cudaEventDestroy(p->ev_meta);
+  if (p->ev_in) cudaEventDestroy(p->ev_in);
+  if (p->ev_noalloc) cudaEventDestroy(p->ev_noalloc);
   for (void* a : p->peer_allocs) cudaFree(a);
   if (p->d_meta) cudaFree(p->d_meta);
   if (p->d_text) cudaFree(p->d_text);
@@ -602,17 +660,6 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_create(const ft_p
   } while (0)
   CK(cudaGetDevice(&p->device));
   CK(cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, p->device));
-  p->host_ctas = 6;
-  if (const char* e = getenv("FLOWPOOL_HOST_CTAS")) { int v = atoi(e); if (v > 0) p->host_ctas = v; }
-  if (const char* e = getenv("FLOWPOOL_HOST_STORE_CTAS")) { int v = atoi(e); if (v > 0) p->host_store_ctas = v; }
-  // A warp's region is 1/8 of a chunk and must hold at least one 2 KiB batch.
-  if (const char* e = getenv("FLOWPOOL_CHUNK_SHIFT")) { int v = atoi(e); if (v >= 14 && v <= 21) p->chunk_shift = v; }
-  if (const char* e = getenv("FLOWPOOL_SCATTER_GROUP")) { int v = atoi(e); if (v > 0) p->scatter_group = v; }
-  if (const char* e = getenv("FLOWPOOL_SCATTER_CTAS_PER_SM")) { int v = atoi(e); if (v > 0) p->scatter_ctas_per_sm = v; }
-  if (const char* e = getenv("FLOWPOOL_GRAD_HOT_THRESHOLD")) { int v = atoi(e); if (v > 0) p->grad_hot_threshold = v; }
-  if (const char* e = getenv("FLOWPOOL_GRAD_CTAS_PER_SM")) { int v = atoi(e); if (v > 0 && v <= 8) p->grad_ctas_per_sm = v; }
-  if (const char* e = getenv("FLOWPOOL_GATHER_U")) { int v = atoi(e); if (v == 4 || v == 8) p->gather_unroll = v; }
-  if (const char* e = getenv("FLOWPOOL_DEV_CTAS_PER_SM")) { int v = atoi(e); if (v > 0) p->dev_ctas_per_sm = v; }
   for (int a = 0; a < 2; ++a) {
     CK(cudaStreamCreateWithFlags(&p->side_stream[a], cudaStreamNonBlocking));
     CK(cudaEventCreateWithFlags(&p->fork_ev[a], cudaEventDisableTiming));
@@ -620,6 +667,15 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_create(const ft_p
   }
   CK(cudaEventCreateWithFlags(&p->ev_producer, cudaEventDisableTiming));
   CK(cudaEventCreateWithFlags(&p->ev_consumer, cudaEventDisableTiming));
+  CK(cudaStreamCreateWithFlags(&p->meta, cudaStreamNonBlocking));
+  CK(cudaEventCreateWithFlags(&p->ev_meta, cudaEventDisableTiming));
+  CK(cudaEventCreateWithFlags(&p->ev_in, cudaEventDisableTiming));
+  CK(cudaEventCreateWithFlags(&p->ev_noalloc, cudaEventDisableTiming));
+  for (int side = 0; side < 2; ++side) for (int i = 0; i < kCallCtx; ++i) {
+    CK(cudaEventCreateWithFlags(&p->ctx[side][i].ev_up, cudaEventDisableTiming));
+    CK(cudaEventCreateWithFlags(&p->ctx[side][i].ev_done, cudaEventDisableTiming));
+  }
+  p->noalloc_blob.resize(16 * (size_t)FT_NOALLOC_MAX_SPANS + 256);
   // per-device kernel set-up: shared-memory opt-ins and occupancy of the data kernels
   CK(cudaFuncSetAttribute(k_scatter_host_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBulkSmemBytes));
   {
@@ -659,7 +715,8 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_create(const ft_p
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
   const size_t o_pte_hbm = take(c.hbm_pages * 8), o_pte_host = take(c.host_pages * 8), o_pte_text = take(n_text * 8);
   const size_t o_ring = take(P * 4), o_tring = take(n_text * 4), o_bring = take(NB * 4);
-  const size_t o_states = take(3 * sizeof(RingState)), o_status = take(32);  // status word, the gather's tile counter, the scatter's claim counters
+  // status word, then two claim counters per call context (zero at rest)
+  const size_t o_states = take(3 * sizeof(RingState)), o_status = take(64 + (size_t)2 * kCallCtx * 2 * sizeof(ClaimCounter));
   const size_t o_seq = take((size_t)c.max_samples * 4), o_nsp = take((size_t)c.max_samples * 4);
   const size_t o_stp = take((size_t)c.max_samples * TPS * 8), o_sfl = take((size_t)c.max_samples * 4);
   const size_t o_peers = take((size_t)c.world_size * sizeof(PeerTables));
@@ -690,6 +747,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_create(const ft_p
   RingState* st = reinterpret_cast<RingState*>(m + o_states);
   v.ring_state = st; v.tring_state = st + 1; v.bring_state = st + 2;
   v.status = reinterpret_cast<unsigned long long*>(m + o_status);
+  for (int i = 0; i < 2 * kCallCtx; ++i) p->ctx[i / kCallCtx][i % kCallCtx].counters = reinterpret_cast<ClaimCounter*>(m + o_status + 64) + 2 * i;
   v.s_seq_len = reinterpret_cast<uint32_t*>(m + o_seq); v.s_n_spans = reinterpret_cast<uint32_t*>(m + o_nsp);
   v.s_text_pages = reinterpret_cast<uint64_t*>(m + o_stp);
   v.s_flags = reinterpret_cast<uint32_t*>(m + o_sfl);
@@ -790,23 +848,24 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_register_samples(
   const size_t blob_bytes = align_up(o_tok + total_spans * 4, 256);
   const size_t o_tpoff = blob_bytes, o_head = align_up(o_tpoff + (size_t)(n + 1) * 4, 16);
   const size_t total_bytes = o_head + 16;
-  std::vector<uint8_t> blob(blob_bytes, 0);
-  uint64_t* ids_off = reinterpret_cast<uint64_t*>(blob.data() + o_idsoff);
-  uint32_t* sb = reinterpret_cast<uint32_t*>(blob.data() + o_sb);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  ft_call_ctx* cx = nullptr;
+  int32_t rc = ctx_acquire(p, 0, blob_bytes, total_bytes, &cx);
+  if (rc != FT_OK) return rc;
+  uint8_t* hb = static_cast<uint8_t*>(cx->h);
+  uint64_t* ids_off = reinterpret_cast<uint64_t*>(hb + o_idsoff);
+  uint32_t* sb = reinterpret_cast<uint32_t*>(hb + o_sb);
   ids_off[0] = 0; sb[0] = 0;
   for (uint32_t i = 0; i < n; ++i) { ids_off[i + 1] = ids_off[i] + seq_len[i]; sb[i + 1] = sb[i] + n_spans[i]; }
-  memcpy(blob.data() + o_slot, slot, (size_t)n * 4);
-  memcpy(blob.data() + o_len, seq_len, (size_t)n * 4);
-  memcpy(blob.data() + o_nsp, n_spans, (size_t)n * 4);
+  memcpy(hb + o_slot, slot, (size_t)n * 4);
+  memcpy(hb + o_len, seq_len, (size_t)n * 4);
+  memcpy(hb + o_nsp, n_spans, (size_t)n * 4);
   if (total_spans) {
-    memcpy(blob.data() + o_pos, span_pos, total_spans * 4);
-    memcpy(blob.data() + o_tok, span_tokens, total_spans * 4);
+    memcpy(hb + o_pos, span_pos, total_spans * 4);
+    memcpy(hb + o_tok, span_tokens, total_spans * 4);
   }
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
-  void* d = nullptr;
-  int32_t rc = stage_upload(p, 0, blob.data(), blob_bytes, total_bytes, st, &d);
-  if (rc != FT_OK) return rc;
-  uint8_t* db = static_cast<uint8_t*>(d);
+  if ((rc = ctx_upload(p, cx, blob_bytes)) != FT_OK) return rc;
+  uint8_t* db = static_cast<uint8_t*>(cx->d);
   RegisterCall rcall;
   rcall.n = n;
   rcall.ids_off = reinterpret_cast<uint64_t*>(db + o_idsoff);
@@ -819,10 +878,13 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_register_samples(
   rcall.ids = input_ids;
   rcall.tp_off = reinterpret_cast<uint32_t*>(db + o_tpoff);
   rcall.head = reinterpret_cast<uint32_t*>(db + o_head);
-  rcall.call_seq = p->call_seq;
-  k_register_scan<<<1, 1024, 0, st>>>(p->view, rcall);
+  rcall.call_seq = status_seq(p);
+  // tables and the text-page pops on the metadata stream; the ids themselves (the caller's data) on the caller's
+  k_register_scan<<<1, scan_threads(n), 0, p->meta>>>(p->view, rcall);
+  if ((rc = meta_to(p, st)) != FT_OK) return rc;
   k_register_ids<<<(unsigned)text_need, 256, 0, st>>>(p->view, rcall);
   FT_CUDA(cudaGetLastError());
+  if ((rc = ctx_release(p, cx, st)) != FT_OK) return rc;
   p->gpu_launches += 2;
 
   // host mirror
@@ -844,6 +906,53 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_register_samples(
   return end_producer(p, st);
 }
 
+namespace ft {
+// Argument and state checks of a producer write, shared by both entry points (same codes, same order).  On success
+// the call's totals are in `t` and, when `b_*` are given, the descriptors in the caller's staging arrays.
+struct WriteTotals {
+  uint64_t need = 0, need_blocks = 0, total_chunks = 0, bytes_total = 0;
+};
+static int32_t check_write(ft_pool* p, uint32_t n, const uint32_t* slot, const uint32_t* span_idx, const uint32_t* n_tokens,
+                           const void* const* src, WriteTotals* t) {
+  const ft_pool_config& c = p->cfg;
+  const uint32_t S = c.max_spans_per_sample;
+  const uint32_t chunk_shift = (uint32_t)p->chunk_shift;
+  for (uint32_t q = 0; q < n; ++q) {
+    if (slot[q] >= c.max_samples) return FT_ERR_INVALID_ARG;
+    const ft_slot_mirror& s = p->slots[slot[q]];
+    if (s.state == FT_SLOT_FREE) return FT_ERR_UNKNOWN_SAMPLE;
+    if (span_idx[q] >= s.n_spans) return FT_ERR_INVALID_ARG;
+    ft_span_mirror& m = p->spans[(uint64_t)slot[q] * S + span_idx[q]];
+    if (n_tokens[q] != m.tokens) return FT_ERR_INVALID_ARG;
+    if (!src[q] || (reinterpret_cast<uintptr_t>(src[q]) & 15)) return FT_ERR_INVALID_ARG;
+    if (m.written || m.named == p->call_seq) return FT_ERR_ALREADY_WRITTEN;  // written before, or named twice in this call
+    m.named = p->call_seq;
+    const uint64_t k = pages_for_tokens(p, n_tokens[q]);
+    t->need += k; t->need_blocks += (k + kListBlock - 1) / kListBlock;
+    const uint64_t bytes = (uint64_t)n_tokens[q] * p->view.row_bytes;
+    t->total_chunks += (bytes + (1ull << chunk_shift) - 1) >> chunk_shift;
+    t->bytes_total += bytes;
+  }
+  if (t->need > p->free_pages) return FT_ERR_POOL_EXHAUSTED;
+  if (t->need_blocks > p->free_blocks) return FT_ERR_CAPACITY;
+  if (t->need > 0xFFFFFFFFull) return FT_ERR_INVALID_ARG;
+  return FT_OK;
+}
+
+static void mirror_write(ft_pool* p, uint32_t n, const uint32_t* slot, const uint32_t* span_idx, const uint32_t* n_tokens,
+                         const WriteTotals& t, bool f32) {
+  const uint32_t S = p->cfg.max_spans_per_sample;
+  for (uint32_t q = 0; q < n; ++q) {
+    ft_slot_mirror& s = p->slots[slot[q]];
+    ft_span_mirror& m = p->spans[(uint64_t)slot[q] * S + span_idx[q]];
+    m.written = true; m.npages = (uint32_t)pages_for_tokens(p, n_tokens[q]);
+    if (++s.spans_written == s.n_spans) { s.state = FT_SLOT_READY; ready_push(p, slot[q]); }
+  }
+  p->free_pages -= t.need; p->free_blocks -= t.need_blocks;
+  p->bytes_written += t.bytes_total * (f32 ? 3 : 2);
+}
+}  // namespace ft
+
 extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings(ft_pool* p, uint32_t n, const uint32_t* slot, const uint32_t* span_idx,
                                          const uint32_t* n_tokens, const void* const* src, uint32_t src_dtype,
                                          void* stream) {
@@ -852,34 +961,11 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings(
   if (src_dtype != FT_BF16 && src_dtype != FT_F32) return FT_ERR_INVALID_ARG;
   if (n == 0) return FT_OK;
   if (!slot || !span_idx || !n_tokens || !src) return FT_ERR_INVALID_ARG;
-  const ft_pool_config& c = p->cfg;
-  const uint32_t S = c.max_spans_per_sample;
-  uint64_t need = 0, need_blocks = 0, total_chunks = 0, bytes_total = 0;
-  const uint32_t chunk_shift = (uint32_t)p->chunk_shift;
-  std::vector<uint32_t> span_id(n);
-  {
-    std::unordered_set<uint32_t> named;
-    named.reserve(n * 2);
-    for (uint32_t q = 0; q < n; ++q) {
-      if (slot[q] >= c.max_samples) return FT_ERR_INVALID_ARG;
-      const ft_slot_mirror& s = p->slots[slot[q]];
-      if (s.state == FT_SLOT_FREE) return FT_ERR_UNKNOWN_SAMPLE;
-      if (span_idx[q] >= s.n_spans) return FT_ERR_INVALID_ARG;
-      const ft_span_mirror& m = p->spans[(uint64_t)slot[q] * S + span_idx[q]];
-      if (n_tokens[q] != m.tokens) return FT_ERR_INVALID_ARG;
-      if (!src[q] || (reinterpret_cast<uintptr_t>(src[q]) & 15)) return FT_ERR_INVALID_ARG;
-      span_id[q] = slot[q] * S + span_idx[q];
-      if (m.written || !named.insert(span_id[q]).second) return FT_ERR_ALREADY_WRITTEN;
-      const uint64_t k = pages_for_tokens(p, n_tokens[q]);
-      need += k; need_blocks += (k + kListBlock - 1) / kListBlock;
-      const uint64_t bytes = (uint64_t)n_tokens[q] * p->view.row_bytes;
-      total_chunks += (bytes + (1ull << chunk_shift) - 1) >> chunk_shift;
-      bytes_total += bytes;
-    }
-  }
-  if (need > p->free_pages) return FT_ERR_POOL_EXHAUSTED;
-  if (need_blocks > p->free_blocks) return FT_ERR_CAPACITY;
-  if (need > 0xFFFFFFFFull) return FT_ERR_INVALID_ARG;
+  const uint32_t S = p->cfg.max_spans_per_sample;
+  WriteTotals t;
+  int32_t rc = check_write(p, n, slot, span_idx, n_tokens, src, &t);
+  if (rc != FT_OK) return rc;
+  const uint64_t need = t.need, total_chunks = t.total_chunks;
 
   // blob: [src u64 n][span_id n][n_tokens n] ; outputs: page_off, blk_off (n+1), chunk_off u64 (n+1), heads
   const size_t o_src = 0, o_sid = (size_t)n * 8, o_ntk = o_sid + (size_t)n * 4;
@@ -888,15 +974,17 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings(
   const size_t o_boff = o_poff + (size_t)(n + 1) * 4, o_heads = align_up(o_boff + (size_t)(n + 1) * 4, 16);
   const size_t o_cspan = o_heads + 16;
   const size_t total_bytes = o_cspan + total_chunks * 4;
-  std::vector<uint8_t> blob(blob_bytes, 0);
-  for (uint32_t q = 0; q < n; ++q) reinterpret_cast<uint64_t*>(blob.data())[q] = reinterpret_cast<uint64_t>(src[q]);
-  memcpy(blob.data() + o_sid, span_id.data(), (size_t)n * 4);
-  memcpy(blob.data() + o_ntk, n_tokens, (size_t)n * 4);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  void* d = nullptr;
-  int32_t rc = stage_upload(p, 0, blob.data(), blob_bytes, total_bytes, st, &d);
-  if (rc != FT_OK) return rc;
-  uint8_t* db = static_cast<uint8_t*>(d);
+  ft_call_ctx* cx = nullptr;
+  if ((rc = ctx_acquire(p, 0, blob_bytes, total_bytes, &cx)) != FT_OK) return rc;
+  uint8_t* hb = static_cast<uint8_t*>(cx->h);
+  for (uint32_t q = 0; q < n; ++q) {
+    reinterpret_cast<uint64_t*>(hb + o_src)[q] = reinterpret_cast<uint64_t>(src[q]);
+    reinterpret_cast<uint32_t*>(hb + o_sid)[q] = slot[q] * S + span_idx[q];
+  }
+  memcpy(hb + o_ntk, n_tokens, (size_t)n * 4);
+  if ((rc = ctx_upload(p, cx, blob_bytes)) != FT_OK) return rc;
+  uint8_t* db = static_cast<uint8_t*>(cx->d);
   WriteCall w;
   w.n = n;
   w.src = reinterpret_cast<uint64_t*>(db + o_src);
@@ -907,51 +995,16 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings(
   w.blk_off = reinterpret_cast<uint32_t*>(db + o_boff);
   w.heads = reinterpret_cast<uint32_t*>(db + o_heads);
   w.chunk_span = reinterpret_cast<uint32_t*>(db + o_cspan);
-  w.chunk_shift = chunk_shift;
-  k_alloc_scan<<<1, 1024, 0, st>>>(p->view, w);
-  k_alloc_fill<<<(unsigned)((std::max<uint64_t>(need, total_chunks) + 255) / 256), 256, 0, st>>>(p->view, w, (uint32_t)need, total_chunks);
+  w.chunk_shift = (uint32_t)p->chunk_shift;
+  // page allocation on the metadata stream (it overlaps the copy of the call before), the copy on the caller's
+  k_alloc_scan<<<1, scan_threads(n), 0, p->meta>>>(p->view, w);
+  k_alloc_fill<<<(unsigned)((std::max<uint64_t>(need, total_chunks) + 255) / 256), 256, 0, p->meta>>>(p->view, w, (uint32_t)need, total_chunks);
   p->gpu_launches += 2;
-
-  // the byte copy: HBM-bound chunks on the caller's stream, host-bound chunks beside them
+  if ((rc = meta_to(p, st)) != FT_OK) return rc;
   const bool f32 = src_dtype == FT_F32;
-  auto launch = [&](int mode, cudaStream_t s) {
-    const bool host_class = mode == kTierHostOnly || (mode == kTierAll && c.hbm_pages == 0);
-    prof_begin(p, host_class ? FT_K_SCATTER_HOST : FT_K_SCATTER_DEVICE, s);
-    launch_scatter_any(p, mode, f32, w, total_chunks, host_class ? (uint64_t)p->host_store_ctas : ~0ull, s);
-    prof_end(p, s);
-    p->gpu_launches++;
-  };
-  if (c.host_pages == 0) {
-    launch(kTierAll, st);
-  } else if (c.hbm_pages == 0) {
-    launch(kTierAll, st);
-  } else {
-    FT_CUDA(cudaEventRecord(p->fork_ev[0], st));
-    FT_CUDA(cudaStreamWaitEvent(p->side_stream[0], p->fork_ev[0], 0));
-    prof_begin(p, FT_K_SCATTER_HOST, p->side_stream[0]);
-    // bf16 source: bulk-async copies through shared memory.  fp32 source: the cast needs the values in
-    // registers, and stores to host memory are posted (no latency to hide), so a few vector-store CTAs do it
-    if (f32) {
-      launch_scatter<kTierHostOnly, true>(p, w, total_chunks, (uint64_t)p->host_store_ctas, p->side_stream[0]);
-    } else {
-      k_scatter_host_bulk<<<(unsigned)p->host_ctas, 32, kBulkSmemBytes, p->side_stream[0]>>>(p->view, w, p->call_seq);
-    }
-    prof_end(p, p->side_stream[0]);
-    p->gpu_launches++;
-    FT_CUDA(cudaEventRecord(p->join_ev[0], p->side_stream[0]));
-    launch(kTierDeviceOnly, st);
-    FT_CUDA(cudaStreamWaitEvent(st, p->join_ev[0], 0));
-  }
-  FT_CUDA(cudaGetLastError());
-
-  for (uint32_t q = 0; q < n; ++q) {
-    ft_slot_mirror& s = p->slots[slot[q]];
-    ft_span_mirror& m = p->spans[span_id[q]];
-    m.written = true; m.npages = (uint32_t)pages_for_tokens(p, n_tokens[q]);
-    if (++s.spans_written == s.n_spans) { s.state = FT_SLOT_READY; ready_push(p, slot[q]); }
-  }
-  p->free_pages -= need; p->free_blocks -= need_blocks;
-  p->bytes_written += bytes_total * (f32 ? 3 : 2);
+  if ((rc = launch_write_copies(p, w, total_chunks, f32, st, cx->counters, true)) != FT_OK) return rc;
+  if ((rc = ctx_release(p, cx, st)) != FT_OK) return rc;
+  mirror_write(p, n, slot, span_idx, n_tokens, t, f32);
   return end_producer(p, st);
 }
 
@@ -962,39 +1015,44 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_free(ft_pool* p, 
   if (!slot) return FT_ERR_INVALID_ARG;
   const ft_pool_config& c = p->cfg;
   const uint32_t S = c.max_spans_per_sample;
-  std::vector<uint8_t> seen(c.max_samples, 0);
   for (uint32_t i = 0; i < n; ++i) {
     if (slot[i] >= c.max_samples) return FT_ERR_INVALID_ARG;
-    if (p->slots[slot[i]].state == FT_SLOT_FREE || seen[slot[i]]) return FT_ERR_UNKNOWN_SAMPLE;
-    seen[slot[i]] = 1;
+    ft_slot_mirror& sm = p->slots[slot[i]];
+    if (sm.state == FT_SLOT_FREE || sm.named == p->call_seq) return FT_ERR_UNKNOWN_SAMPLE;  // free, or listed twice
+    sm.named = p->call_seq;
   }
-  std::vector<uint32_t> span_ids;
-  uint64_t pages = 0, blocks = 0, text = 0;
+  uint64_t pages = 0, blocks = 0, text = 0, ns64 = 0;
   for (uint32_t i = 0; i < n; ++i) {
     const ft_slot_mirror& s = p->slots[slot[i]];
-    for (uint32_t j = 0; j < s.n_spans; ++j) {
-      const ft_span_mirror& m = p->spans[(uint64_t)slot[i] * S + j];
-      if (!m.written) continue;
-      span_ids.push_back(slot[i] * S + j);
-      blocks += (m.npages + kListBlock - 1) / kListBlock;
-      if (!s.remote) pages += m.npages;  // an imported sample's pages belong to the peer that wrote them
-    }
-    if (!s.remote) text += s.n_text_pages;
+    for (uint32_t j = 0; j < s.n_spans; ++j) ns64 += p->spans[(uint64_t)slot[i] * S + j].written ? 1 : 0;
   }
-  const uint32_t ns = (uint32_t)span_ids.size();
+  const uint32_t ns = (uint32_t)ns64;
   const size_t o_sid = 0, o_slot = (size_t)ns * 4;
   const size_t blob_bytes = align_up(o_slot + (size_t)n * 4, 256);
   const size_t o_poff = blob_bytes, o_boff = o_poff + (size_t)(ns + 1) * 4, o_toff = o_boff + (size_t)(ns + 1) * 4;
   const size_t o_tails = align_up(o_toff + (size_t)(n + 1) * 4, 16);
   const size_t total_bytes = o_tails + 16;
-  std::vector<uint8_t> blob(blob_bytes, 0);
-  if (ns) memcpy(blob.data() + o_sid, span_ids.data(), (size_t)ns * 4);
-  memcpy(blob.data() + o_slot, slot, (size_t)n * 4);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  void* d = nullptr;
-  int32_t rc = stage_upload(p, 0, blob.data(), blob_bytes, total_bytes, st, &d);
+  ft_call_ctx* cx = nullptr;
+  int32_t rc = ctx_acquire(p, 0, blob_bytes, total_bytes, &cx);
   if (rc != FT_OK) return rc;
-  uint8_t* db = static_cast<uint8_t*>(d);
+  uint8_t* hb = static_cast<uint8_t*>(cx->h);
+  uint32_t* h_sid = reinterpret_cast<uint32_t*>(hb + o_sid);
+  uint32_t k = 0;
+  for (uint32_t i = 0; i < n; ++i) {
+    const ft_slot_mirror& s = p->slots[slot[i]];
+    for (uint32_t j = 0; j < s.n_spans; ++j) {
+      const ft_span_mirror& m = p->spans[(uint64_t)slot[i] * S + j];
+      if (!m.written) continue;
+      h_sid[k++] = slot[i] * S + j;
+      blocks += (m.npages + kListBlock - 1) / kListBlock;
+      if (!s.remote) pages += m.npages;  // an imported sample's pages belong to the peer that wrote them
+    }
+    if (!s.remote) text += s.n_text_pages;
+  }
+  memcpy(hb + o_slot, slot, (size_t)n * 4);
+  if ((rc = ctx_upload(p, cx, blob_bytes)) != FT_OK) return rc;
+  uint8_t* db = static_cast<uint8_t*>(cx->d);
   FreeCall f;
   f.n_spans = ns; f.n_samples = n;
   f.span_id = reinterpret_cast<uint32_t*>(db + o_sid);
@@ -1003,12 +1061,16 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_free(ft_pool* p, 
   f.blk_off = reinterpret_cast<uint32_t*>(db + o_boff);
   f.tp_off = reinterpret_cast<uint32_t*>(db + o_toff);
   f.tails = reinterpret_cast<uint32_t*>(db + o_tails);
-  if ((rc = begin_free(p, st)) != FT_OK) return rc;  // a gather issued earlier on another stream may still read these pages
-  k_free_scan<<<1, 1024, 0, st>>>(p->view, f);
+  // copies and assemblies still in flight (on the callers' streams) read these samples' tables and pages: the
+  // metadata stream waits for the latest of each side, and for what the caller queued on `st` before this call
+  if ((rc = meta_after_data(p)) != FT_OK) return rc;
+  if ((rc = meta_after(p, st)) != FT_OK) return rc;
+  k_free_scan<<<1, scan_threads(std::max(n, ns)), 0, p->meta>>>(p->view, f);
   const uint64_t items = pages + blocks + text;
-  if (items) k_free_fill<<<(unsigned)((items + 255) / 256), 256, 0, st>>>(p->view, f, (uint32_t)pages, (uint32_t)blocks, (uint32_t)text);
-  k_free_clear<<<(std::max(n, ns) + 255) / 256, 256, 0, st>>>(p->view, f);
+  if (items) k_free_fill<<<(unsigned)((items + 255) / 256), 256, 0, p->meta>>>(p->view, f, (uint32_t)pages, (uint32_t)blocks, (uint32_t)text);
+  k_free_clear<<<(std::max(n, ns) + 255) / 256, 256, 0, p->meta>>>(p->view, f);
   FT_CUDA(cudaGetLastError());
+  if ((rc = ctx_release(p, cx, p->meta)) != FT_OK) return rc;
   p->gpu_launches += items ? 3 : 2;
 
   for (uint32_t i = 0; i < n; ++i) {
@@ -1021,6 +1083,8 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_free(ft_pool* p, 
   }
   p->free_pages += pages; p->free_blocks += blocks; p->free_text_pages += text;
   p->free_epoch++;
+  // what the caller queues on `st` next comes after the release
+  if ((rc = meta_to(p, st)) != FT_OK) return rc;
   return end_producer(p, st);
 }
 
@@ -1069,8 +1133,9 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_status(ft_pool* p
   FT_CUDA(cudaDeviceSynchronize());
   unsigned long long key = 0;
   FT_CUDA(cudaMemcpy(&key, p->view.status, 8, cudaMemcpyDeviceToHost));
+  p->status_base = p->call_seq;  // error keys count calls from here on
   if (key == ~0ull) { if (code) *code = 0; if (detail) *detail = 0; return FT_OK; }
-  if (code) *code = -(int32_t)((key >> 32) & 0xFF);
+  if (code) *code = -(int32_t)((key >> 32) & 0xF);
   if (detail) *detail = key & 0xFFFFFFFFull;
   FT_CUDA(cudaMemset(p->view.status, 0xFF, 8));
   return FT_OK;
@@ -1085,6 +1150,39 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_stats(ft_pool* p,
   out->live_samples = p->live_samples; out->live_spans = p->live_spans;
   out->bytes_written = p->bytes_written; out->bytes_gathered = p->bytes_gathered;
   out->gpu_launches = p->gpu_launches;
+  return FT_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int32_t pool_get_tuning(ft_pool* p, ft_tuning* out) {
+  if (!p || !out) return FT_ERR_INVALID_ARG;
+  memset(out, 0, sizeof(*out));
+  out->dev_ctas_per_sm = (uint32_t)p->dev_ctas_per_sm;
+  out->scatter_ctas_per_sm = (uint32_t)(p->scatter_ctas_per_sm > 0 ? p->scatter_ctas_per_sm : 4);
+  out->scatter_group = (uint32_t)(p->scatter_group > 0 ? p->scatter_group : 1);
+  out->chunk_shift = (uint32_t)p->chunk_shift;
+  out->host_ctas = (uint32_t)p->host_ctas; out->host_store_ctas = (uint32_t)p->host_store_ctas;
+  out->gather_unroll = (uint32_t)p->gather_unroll;
+  out->grad_ctas_per_sm = (uint32_t)p->grad_ctas_per_sm; out->grad_hot_threshold = (uint32_t)p->grad_hot_threshold;
+  return FT_OK;
+}
+
+extern "C" __attribute__((visibility("default"))) int32_t pool_set_tuning(ft_pool* p, const ft_tuning* in) {
+  if (!p || !in) return FT_ERR_INVALID_ARG;
+  const ft_tuning& t = *in;
+  if (t.dev_ctas_per_sm > 8 || t.scatter_ctas_per_sm > 8 || t.grad_ctas_per_sm > 8) return FT_ERR_INVALID_ARG;
+  if (t.chunk_shift && (t.chunk_shift < 14 || t.chunk_shift > 21)) return FT_ERR_INVALID_ARG;  // a warp's eighth holds a 2 KiB batch
+  if (t.gather_unroll && t.gather_unroll != 4 && t.gather_unroll != 8) return FT_ERR_INVALID_ARG;
+  if (t.host_ctas > 1024 || t.host_store_ctas > 1024 || t.scatter_group > (1u << 20)) return FT_ERR_INVALID_ARG;
+  FT_CUDA(cudaDeviceSynchronize());  // no kernel of an earlier call is still being sized by the old values
+  p->dev_ctas_per_sm = t.dev_ctas_per_sm ? (int)t.dev_ctas_per_sm : 4;
+  p->scatter_ctas_per_sm = (int)t.scatter_ctas_per_sm;
+  p->scatter_group = (int)t.scatter_group;
+  p->chunk_shift = t.chunk_shift ? (int)t.chunk_shift : 16;
+  p->host_ctas = t.host_ctas ? (int)t.host_ctas : 6;
+  p->host_store_ctas = t.host_store_ctas ? (int)t.host_store_ctas : 8;
+  p->gather_unroll = t.gather_unroll ? (int)t.gather_unroll : 4;
+  p->grad_ctas_per_sm = t.grad_ctas_per_sm ? (int)t.grad_ctas_per_sm : 6;
+  p->grad_hot_threshold = (int)t.grad_hot_threshold;
   return FT_OK;
 }
 
@@ -1209,58 +1307,32 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings_
   int cur = -1;
   FT_CUDA(cudaGetDevice(&cur));
   if (cur != p->device) return FT_ERR_INVALID_ARG;
-  const ft_pool_config& c = p->cfg;
-  const uint32_t S = c.max_spans_per_sample;
-  const uint32_t chunk_shift = (uint32_t)p->chunk_shift;
-  uint64_t need = 0, need_blocks = 0, total_chunks = 0, bytes_total = 0;
+  const uint32_t S = p->cfg.max_spans_per_sample;
+  WriteTotals t;
+  int32_t rc = check_write(p, n, slot, span_idx, n_tokens, src, &t);
+  if (rc != FT_OK) return rc;
 
-  // descriptor blob on the stack: [src u64 n][span_id n][n_tokens n]; duplicate check in a fixed hash table
-  constexpr size_t kBlobMax = 16 * (size_t)FT_NOALLOC_MAX_SPANS + 256;
-  alignas(16) uint8_t blob[kBlobMax];
-  constexpr uint32_t kTab = 4 * FT_NOALLOC_MAX_SPANS;  // open addressing, load <= 1/4
-  uint32_t table[kTab];
-  memset(table, 0xFF, sizeof(table));
+  // descriptor blob [src u64 n][span_id n][n_tokens n] in the host buffer pool_create made for this purpose
   const size_t o_src = 0, o_sid = (size_t)n * 8, o_ntk = o_sid + (size_t)n * 4;
   const size_t blob_bytes = align_up(o_ntk + (size_t)n * 4, 256);
-  uint64_t* b_src = reinterpret_cast<uint64_t*>(blob + o_src);
-  uint32_t* b_sid = reinterpret_cast<uint32_t*>(blob + o_sid);
-  uint32_t* b_ntk = reinterpret_cast<uint32_t*>(blob + o_ntk);
+  uint8_t* blob = p->noalloc_blob.data();
   for (uint32_t q = 0; q < n; ++q) {
-    if (slot[q] >= c.max_samples) return FT_ERR_INVALID_ARG;
-    const ft_slot_mirror& s = p->slots[slot[q]];
-    if (s.state == FT_SLOT_FREE) return FT_ERR_UNKNOWN_SAMPLE;
-    if (span_idx[q] >= s.n_spans) return FT_ERR_INVALID_ARG;
-    const ft_span_mirror& m = p->spans[(uint64_t)slot[q] * S + span_idx[q]];
-    if (n_tokens[q] != m.tokens) return FT_ERR_INVALID_ARG;
-    if (!src[q] || (reinterpret_cast<uintptr_t>(src[q]) & 15)) return FT_ERR_INVALID_ARG;
-    const uint32_t sid = slot[q] * S + span_idx[q];
-    if (m.written) return FT_ERR_ALREADY_WRITTEN;
-    uint32_t h = (sid * 2654435761u) % kTab;
-    while (table[h] != 0xFFFFFFFFu) {
-      if (table[h] == sid) return FT_ERR_ALREADY_WRITTEN;  // named twice in this call
-      h = (h + 1) % kTab;
-    }
-    table[h] = sid;
-    b_src[q] = reinterpret_cast<uint64_t>(src[q]); b_sid[q] = sid; b_ntk[q] = n_tokens[q];
-    const uint64_t k = pages_for_tokens(p, n_tokens[q]);
-    need += k; need_blocks += (k + kListBlock - 1) / kListBlock;
-    const uint64_t bytes = (uint64_t)n_tokens[q] * p->view.row_bytes;
-    total_chunks += (bytes + (1ull << chunk_shift) - 1) >> chunk_shift;
-    bytes_total += bytes;
+    reinterpret_cast<uint64_t*>(blob + o_src)[q] = reinterpret_cast<uint64_t>(src[q]);
+    reinterpret_cast<uint32_t*>(blob + o_sid)[q] = slot[q] * S + span_idx[q];
   }
-  if (need > p->free_pages) return FT_ERR_POOL_EXHAUSTED;
-  if (need_blocks > p->free_blocks) return FT_ERR_CAPACITY;
-  if (need > 0xFFFFFFFFull) return FT_ERR_INVALID_ARG;
-
+  memcpy(blob + o_ntk, n_tokens, (size_t)n * 4);
   const size_t o_choff = blob_bytes, o_poff = align_up(o_choff + (size_t)(n + 1) * 8, 16);
   const size_t o_boff = o_poff + (size_t)(n + 1) * 4, o_heads = align_up(o_boff + (size_t)(n + 1) * 4, 16);
-  if (o_heads + 16 > FT_NOALLOC_SCRATCH_BYTES) return FT_ERR_CAPACITY;
+  constexpr size_t o_counters = FT_NOALLOC_SCRATCH_BYTES - 2 * sizeof(ClaimCounter);  // the array's last 32 bytes
+  if (o_heads + 16 > o_counters) return FT_ERR_CAPACITY;
   uint8_t* db = nullptr;
-  int32_t rc = noalloc_scratch(p->device, &db);
-  if (rc != FT_OK) return rc;
+  if ((rc = noalloc_scratch(p->device, &db)) != FT_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  // pageable source: the call returns once the bytes have been taken, so the stack buffer may die after it
-  FT_CUDA(cudaMemcpyAsync(db, blob, blob_bytes, cudaMemcpyHostToDevice, st));
+  // the array still serves the previous no-allocation write of this pool until that call's copy has finished
+  if (p->have_noalloc_ev) FT_CUDA(cudaStreamWaitEvent(p->meta, p->ev_noalloc, 0));
+  // pageable source: cudaMemcpyAsync returns once the bytes have been taken, so the buffer is free again after it
+  p->meta_seq++;
+  FT_CUDA(cudaMemcpyAsync(db, blob, blob_bytes, cudaMemcpyHostToDevice, p->meta));
   WriteCall w;
   w.n = n;
   w.src = reinterpret_cast<uint64_t*>(db + o_src);
@@ -1271,41 +1343,16 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings_
   w.blk_off = reinterpret_cast<uint32_t*>(db + o_boff);
   w.heads = reinterpret_cast<uint32_t*>(db + o_heads);
   w.chunk_span = nullptr;  // the fixed scratch has no room for a per-chunk table: k_scatter searches chunk_off
-  w.chunk_shift = chunk_shift;
-  k_alloc_scan<<<1, 1024, 0, st>>>(p->view, w);
-  k_alloc_fill<<<(unsigned)((need + 255) / 256), 256, 0, st>>>(p->view, w, (uint32_t)need, 0);
+  w.chunk_shift = (uint32_t)p->chunk_shift;
+  k_alloc_scan<<<1, scan_threads(n), 0, p->meta>>>(p->view, w);
+  k_alloc_fill<<<(unsigned)((t.need + 255) / 256), 256, 0, p->meta>>>(p->view, w, (uint32_t)t.need, 0);
   p->gpu_launches += 2;
-
+  if ((rc = meta_to(p, st)) != FT_OK) return rc;
   const bool f32 = src_dtype == FT_F32;
-  auto launch = [&](int mode, cudaStream_t s) {
-    const bool host_class = mode == kTierAll && c.hbm_pages == 0;
-    launch_scatter_any(p, mode, f32, w, total_chunks, host_class ? (uint64_t)p->host_store_ctas : ~0ull, s);
-    p->gpu_launches++;
-  };
-  if (c.host_pages == 0 || c.hbm_pages == 0) {
-    launch(kTierAll, st);
-  } else {
-    FT_CUDA(cudaEventRecord(p->fork_ev[0], st));
-    FT_CUDA(cudaStreamWaitEvent(p->side_stream[0], p->fork_ev[0], 0));
-    if (f32) {
-      launch_scatter<kTierHostOnly, true>(p, w, total_chunks, (uint64_t)p->host_store_ctas, p->side_stream[0]);
-    } else {
-      k_scatter_host_bulk<<<(unsigned)p->host_ctas, 32, kBulkSmemBytes, p->side_stream[0]>>>(p->view, w, p->call_seq);
-    }
-    p->gpu_launches++;
-    FT_CUDA(cudaEventRecord(p->join_ev[0], p->side_stream[0]));
-    launch(kTierDeviceOnly, st);
-    FT_CUDA(cudaStreamWaitEvent(st, p->join_ev[0], 0));
-  }
-  FT_CUDA(cudaGetLastError());
-
-  for (uint32_t q = 0; q < n; ++q) {
-    ft_slot_mirror& s = p->slots[slot[q]];
-    ft_span_mirror& m = p->spans[b_sid[q]];
-    m.written = true; m.npages = (uint32_t)pages_for_tokens(p, n_tokens[q]);
-    if (++s.spans_written == s.n_spans) { s.state = FT_SLOT_READY; ready_push(p, slot[q]); }
-  }
-  p->free_pages -= need; p->free_blocks -= need_blocks;
-  p->bytes_written += bytes_total * (f32 ? 3 : 2);
+  // the claim counters of the copy kernels sit at the end of the array; they are zero whenever no kernel uses them
+  if ((rc = launch_write_copies(p, w, t.total_chunks, f32, st, reinterpret_cast<ClaimCounter*>(db + o_counters), true)) != FT_OK) return rc;
+  FT_CUDA(cudaEventRecord(p->ev_noalloc, st));
+  p->have_noalloc_ev = true;
+  mirror_write(p, n, slot, span_idx, n_tokens, t, f32);
   return end_producer(p, st);
 }
