@@ -225,8 +225,10 @@ def run_reference(args):
     print(json.dumps(line))
 
 
-def workload_label(args):
-    tier = "all pages in HBM" if args.all_hbm else "pool 80% HBM / 20% pinned host"
+def workload_label(args, all_hbm=None):
+    all_hbm = args.all_hbm if all_hbm is None else all_hbm
+    split = {"image_mix_7b": "pool 80% HBM / 20% pinned host", "host_tier_stress": "pool 50% HBM / 50% pinned host, tiers interleaved"}
+    tier = "all pages in HBM" if (all_hbm or args.workload not in split) else split[args.workload]
     n = f", first {args.samples} samples" if args.samples else ""
     if args.workload != "image_mix_7b":
         return f"{args.workload} ({tier}){n}"
@@ -300,21 +302,36 @@ class DeviceJob:
         plan.destroy()
         return n_mb
 
-    def host_tier_bytes(self):
-        """Vision bytes that landed in host-tier pages in the last written state (needs a written pool)."""
-        w = self.w
-        if w.host_pages == 0:
-            return 0
-        host_start = 1 << 45
-        total = 0
+    # -- which bytes of a step land on host-tier pages -------------------------------------------------------
+    # The free ring is a FIFO over global page indices (indices below hbm_pages are HBM frames): a write call's spans
+    # pop consecutive entries in argument order, pool_free pushes a sample's pages back in argument order, spans by
+    # index, pages by ordinal.  The pool is barely larger than one batch, so the ring rotates from step to step and the
+    # share of a batch that lands on host-tier pages differs per step.  The benchmark follows the ring on the host
+    # (bookkeeping only) to know, for every timed step, how many bytes crossed the host link; the model is checked
+    # against the pool's own ring afterwards.
+    def ring_model_reset(self):
+        import collections
+        self.model_ring = collections.deque(int(x) for x in self.pool.ring())   # synchronises: outside timed regions
+
+    def ring_model_step(self):
+        """Host-tier vision bytes of one step (write everything, then free everything in plan order)."""
+        w, ring = self.w, self.model_ring
+        host_b, pages_of = 0, {}
         for call in w.write_calls:
             for s, j in call:
-                rc, pages = self.pool.span_pages(s, j)
                 nbytes = int(w.spans_of(s)[1][j]) * w.row_bytes
-                for o, g in enumerate(pages):
-                    if int(g) >= host_start:
-                        total += min(w.page_bytes, nbytes - o * w.page_bytes)
-        return total
+                got = [ring.popleft() for _ in range(-(-nbytes // w.page_bytes))]
+                pages_of[(s, j)] = got
+                for o, g in enumerate(got):
+                    if g >= w.hbm_pages:
+                        host_b += min(w.page_bytes, nbytes - o * w.page_bytes)
+        for s in self.order:
+            for j in range(int(w.n_spans[int(s)])):
+                ring.extend(pages_of[(int(s), j)])
+        return host_b
+
+    def ring_model_matches(self):
+        return [int(x) for x in self.pool.ring()] == list(self.model_ring)
 
     def close(self):
         self.torch.cuda.synchronize()
@@ -376,6 +393,8 @@ def timed_steps(job, steps, warmup, dist):
     if dist:
         dist.barrier()
     torch.cuda.synchronize()
+    job.ring_model_reset()
+    job.host_bytes_per_step = [job.ring_model_step() for _ in range(steps)] if job.w.host_pages else [0] * steps
     job.pool.profile_read()
     job.pool.profile_enable(True)
     launches0 = job.pool.stats()["gpu_launches"]
@@ -407,6 +426,7 @@ def timed_steps(job, steps, warmup, dist):
     prof = job.pool.profile_read()
     job.pool.profile_enable(False)
     launches = job.pool.stats()["gpu_launches"] - launches0
+    job.ring_ok = job.ring_model_matches() if job.w.host_pages else True
     job.plan_ms_in_step = float(np.median(job.plan_ms)) if job.plan_ms else None
     if dist:
         ms = max_over_ranks(ms, dist)
@@ -456,13 +476,7 @@ def phase_breakdown(job, reps=3):
 def kernel_breakdown(job, prof, steps):
     """Per-kernel-class time per step and achieved bandwidth against the bytes that class moves."""
     w = job.w
-    # host-tier split needs a written pool: write once more (untimed), read the page lists, free again
-    st = job.torch.cuda.current_stream().cuda_stream
-    for c in job.calls:
-        job.check(job.pool.register_samples(*c["reg"], c["ids"].data_ptr(), st), "register")
-        job.check(job.pool.write_embeddings(*c["wr"], c["ptrs"], w.src_dtype, st), "write")
-    host_b = job.host_tier_bytes()
-    job.check(job.pool.free(job.order, st), "free")
+    host_b = float(np.mean(job.host_bytes_per_step))   # what the timed steps actually put on host-tier pages, per step
     vis_b = w.total_vision_tokens * w.row_bytes
     tok_b = w.total_tokens * w.row_bytes
     src_mult = 1 if w.src_dtype == 0 else 2
@@ -696,6 +710,57 @@ def backbone_side(job, reps=3):
     }
 
 
+def short_pass(args, name, all_hbm, steps=3):
+    """One short timed pass of the whole step on another configuration, with the per-kernel-class figures."""
+    import copy
+    import gc
+    a = copy.copy(args)
+    a.workload, a.samples, a.all_hbm = name, None, all_hbm
+    job = DeviceJob(a, all_hbm)
+    ms, prof, launches, n_mb = timed_steps(job, steps, 3, None)
+    kern, host_b = kernel_breakdown(job, prof, steps)
+    phases = phase_breakdown(job, reps=2)
+    wb, gb = algorithmic_bytes(job.w)
+    peak = measured_peak()[0]
+    g = kern["gather_device"] if kern["gather_device"]["ms_per_step"] > 0 else kern["gather_host"]
+    sc = kern["scatter_device"] if kern["scatter_device"]["ms_per_step"] > 0 else kern["scatter_host"]
+    res = {"workload": workload_label(a), "step_ms": ms, "value": (wb + gb) / ms / 1e6, "unit": UNIT, "tokens_per_s": job.w.total_tokens / ms * 1e3,
+           "packed_tokens": job.w.total_tokens, "microbatches": n_mb, "gpu_launches_per_step": launches / steps,
+           "gather_gbs": g["gbs"], "gather_frac_of_measured_copy": g["gbs"] / peak if g["gbs"] else None,
+           "gather_frac_of_nominal_8000": g["gbs"] / 8000.0 if g["gbs"] else None, "write_gbs": sc["gbs"],
+           "plan_ms": phases["plan"], "phase_ms": phases, "host_tier_bytes_per_step": host_b,
+           "l2": "L2 flushed between steps" if job.fits_l2() else "inputs larger than L2", "ring_model_matches": job.ring_ok}
+    if job.w.host_pages:
+        res["host_link_gbs"] = {k: (host_b / kern[k]["ms_per_step"] / 1e6 if kern[k]["ms_per_step"] > 0 else None) for k in ("gather_host", "scatter_host")}
+    job.close()
+    del job
+    gc.collect()
+    import torch
+    torch.cuda.empty_cache()
+    return res
+
+
+def all_configs(args):
+    """Every other configuration the benchmark spec names, one short pass each (the headline configuration is the line itself)."""
+    out = {}
+    for key, name, hbm in (("tiny", "tiny", True), ("video_heavy", "video_heavy", True), ("host_tier_stress", "host_tier_stress", False),
+                           ("host_tier_stress_all_hbm", "host_tier_stress", True)):
+        try:
+            out[key] = short_pass(args, name, hbm)
+        except Exception as e:   # a configuration that does not fit this box must not take the line down
+            out[key] = {"error": repr(e)[:200]}
+    for ps in (2 << 20, 4096):
+        try:
+            r = sweep_measure(args, ps, with_variants=False)
+            out[f"frag_sweep_{ps}"] = {k: r[k] for k in ("value", "unit", "residents", "packed_tokens", "microbatches", "gather_ms", "gather_launches",
+                                                          "frac_of_measured_peak", "frac_of_nominal_8000", "write_gbs", "plan_ms_host_wall_median",
+                                                          "internal_fragmentation", "padding_waste", "rank_imbalance")}
+            out[f"frag_sweep_{ps}"]["workload"] = r["config"]["workload"]
+        except Exception as e:
+            out[f"frag_sweep_{ps}"] = {"error": repr(e)[:200]}
+    return out
+
+
 def run_backbone_only(args):
     """One JSON line with the backbone-side measurements alone (small cases for profiler captures)."""
     import torch
@@ -708,14 +773,13 @@ def run_backbone_only(args):
     print(json.dumps({"workload": workload_label(args) + " (all HBM)", "samples": job.w.n_samples, "backbone_side": res}))
 
 
-def run_ours(args):
-    import torch
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback for the product path)")
+def init_dist(torch):
+    """Process group of this run (None outside torchrun): NCCL, one rank per GPU; FLOWPOOL_BENCH_BACKEND=gloo lets
+    several ranks share a GPU (how the multi-rank code path is exercised where only one GPU is at hand)."""
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
-    backend = os.environ.get("FLOWPOOL_BENCH_BACKEND", "nccl")   # gloo: several ranks may share a GPU (checks of this script)
+    backend = os.environ.get("FLOWPOOL_BENCH_BACKEND", "nccl")
     if backend != "nccl":
         local %= max(1, torch.cuda.device_count())
     torch.cuda.set_device(local)
@@ -726,6 +790,29 @@ def run_ours(args):
             dist.init_process_group("nccl", device_id=torch.device("cuda", local))
         else:
             dist.init_process_group(backend)
+    return dist, rank, local, world, backend
+
+
+def roofline_of(kern, peak, peak_src):
+    g = kern["gather_device"] if kern["gather_device"]["ms_per_step"] > 0 else kern["gather_host"]
+    achieved = g["gbs"]
+    per_launch = g["bytes_per_step"] / max(1.0, g["launches_per_step"])
+    return {
+        "kernel": "k_gather (device-tier rows)", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+        "frac": achieved / peak if achieved else None, "peak_source": peak_src + "; a plain copy, not a hardware limit: a fraction slightly above 1 is possible",
+        "algorithmic_bytes_per_launch": per_launch, "ms_per_launch": g["ms_per_step"] / max(1.0, g["launches_per_step"]),
+        "traffic": per_launch * NCU_TRAFFIC_RATIO_GATHER if NCU_TRAFFIC_RATIO_GATHER else None,
+        "traffic_note": "dram__bytes_read + dram__bytes_write of one launch on the first 64 samples (all HBM), scaled by the tokens "
+                        "of a full launch; an upper bound at full size, where more table rows are served from L2",
+        "frac_of_nominal_8000": achieved / 8000.0 if achieved else None,
+    }
+
+
+def run_ours(args):
+    import torch
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback for the product path)")
+    dist, rank, local, world, backend = init_dist(torch)
     sampler = ClockSampler(local)
     job = DeviceJob(args, args.all_hbm)
     w = job.w
@@ -746,29 +833,26 @@ def run_ours(args):
                 kern[k]["link_frac_of_memcpy"] = kern[k]["link_gbs"] / link[ref]
 
     line = None
+    peak, peak_src = measured_peak()
     if rank == 0:
-        peak, peak_src = measured_peak()
-        g = kern["gather_device"] if kern["gather_device"]["ms_per_step"] > 0 else kern["gather_host"]
-        achieved = g["gbs"]
-        per_launch = g["bytes_per_step"] / max(1.0, g["launches_per_step"])
-        roofline = {
-            "kernel": "k_gather (device-tier rows)", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-            "frac": achieved / peak if achieved else None, "peak_source": peak_src,
-            "algorithmic_bytes_per_launch": per_launch, "ms_per_launch": g["ms_per_step"] / max(1.0, g["launches_per_step"]),
-            "traffic": per_launch * NCU_TRAFFIC_RATIO_GATHER if NCU_TRAFFIC_RATIO_GATHER else None,
-            "frac_of_nominal_8000": achieved / 8000.0 if achieved else None,
-        }
+        hb = job.host_bytes_per_step
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8",
             "data": "synthetic",
             "config": {"workload": workload_label(args), "samples": w.n_samples, "packed_tokens": w.total_tokens,
                        "vision_tokens": w.total_vision_tokens, "microbatches": n_mb, "hbm_pages": w.hbm_pages,
-                       "host_pages": w.host_pages, "host_tier_bytes": host_b,
+                       "host_pages": w.host_pages,
+                       "host_tier_bytes_per_step": {"min": int(min(hb)), "mean": float(np.mean(hb)), "max": int(max(hb)),
+                                                    "ring_model_matches_pool": job.ring_ok,
+                                                    "note": "the free ring rotates from step to step (pool = 1.02 x one batch), so the bytes "
+                                                            "that land on host-tier pages, and with them the link-bound step time, differ per "
+                                                            "step; the kernel figures use the bytes the timed steps moved"},
                        "l2": ("L2 flushed between steps (512 MiB scrub outside the timed regions)" if job.fits_l2()
                               else "inputs larger than L2 (no flush needed)"), "parallelism": f"dp{world} (independent batches)"},
             "tokens_per_s": world * w.total_tokens / ms * 1e3,
-            "gpu_launches": launches, "kernels": kern, "phase_ms": phases, "plan_call_host_ms_in_step": job.plan_ms_in_step, "host_link_memcpy": link, "roofline": roofline, "clocks": clocks,
+            "gpu_launches": launches, "kernels": kern, "phase_ms": phases, "plan_call_host_ms_in_step": job.plan_ms_in_step,
+            "host_link_memcpy": link, "roofline": roofline_of(kern, peak, peak_src), "clocks": clocks,
         }
     # end to end through host buffers, on the same pool as the headline number
     if rank == 0:
@@ -790,8 +874,14 @@ def run_ours(args):
             g2 = kern2["gather_device"]
             line["all_hbm_variant"] = {"value": world * (wb + gb) / ms2 / 1e6, "unit": UNIT, "ms_per_step": ms2,
                                        "tokens_per_s": world * w.total_tokens / ms2 * 1e3, "kernels": kern2,
-                                       "phase_ms": phases2,
-                                       "gather_frac_of_measured_peak": g2["gbs"] / measured_peak()[0] if g2["gbs"] else None}
+                                       "phase_ms": phases2, "plan_call_host_ms_in_step": job.plan_ms_in_step,
+                                       "gather_frac_of_measured_peak": g2["gbs"] / peak if g2["gbs"] else None,
+                                       "gather_frac_of_nominal_8000": g2["gbs"] / 8000.0 if g2["gbs"] else None}
+            # the driver's record keeps `roofline` whole: the HBM-resident figures ride in it too
+            line["roofline"]["all_hbm_pool"] = {"achieved": g2["gbs"], "frac": g2["gbs"] / peak, "frac_of_nominal_8000": g2["gbs"] / 8000.0,
+                                                "ms_per_launch": g2["ms_per_step"], "algorithmic_bytes_per_launch": g2["bytes_per_step"],
+                                                "whole_step_gbs": line["all_hbm_variant"]["value"], "whole_step_ms": ms2,
+                                                "scatter_gbs": kern2["scatter_device"]["gbs"]}
             if world == 1:
                 line["all_hbm_variant"]["backbone_side"] = backbone_side(job)
     job.close()
@@ -804,6 +894,17 @@ def run_ours(args):
         line["streaming"] = run_streaming(args, args.all_hbm)
         if not args.all_hbm:
             line["all_hbm_variant"]["streaming"] = run_streaming(args, True)
+    if world == 1 and rank == 0 and not args.skip_variants and not args.skip_configs and args.workload == "image_mix_7b" and not args.samples:
+        line["all_configs"] = all_configs(args)
+        line["roofline"]["other_configs"] = {k: {kk: v.get(kk) for kk in ("gather_gbs", "gather_frac_of_measured_copy", "write_gbs", "step_ms", "value",
+                                                                        "frac_of_measured_peak", "gather_ms")
+                                                 if v.get(kk) is not None} for k, v in line["all_configs"].items()}
+    if world > 1 and not args.skip_variants:
+        # the paper's own multi-process flow: every rank writes, descriptors are exchanged, all plan alike, each
+        # assembles the share Algorithm 1 dealt to it from everybody's pages
+        ex = exchange_measure(args, dist, rank, world, local, backend)
+        if rank == 0:
+            line["exchange"] = ex
     if rank == 0:
         if world == 1 and not args.skip_cpu:
             n = min(CPU_SAMPLE, w.n_samples)
@@ -820,22 +921,32 @@ def run_ours(args):
 # scale + fragmentation sweep (one page size per invocation)
 # ---------------------------------------------------------------------------------------------
 def run_sweep(args):
+    """Config 5 for one page size: prints sweep_measure's line."""
+    import torch
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    args.sweep_samples = args.samples
+    print(json.dumps(sweep_measure(args, args.page_bytes)))
+
+
+def sweep_measure(args, PS, with_variants=True):
     """Config 5: a stream of samples flows through a fixed-capacity pool (10 x {admit while it fits, free a
-    seeded half}, final admit), then the residents are planned and gathered.  Prints one JSON line with the
+    seeded half}, final admit), then the residents are planned and gathered.  Returns one line (a dict) with the
     gather/write bandwidth, plan time, fragmentation and packing figures for the given page size."""
     import torch
     import workloads
     from harness import pool_config_fields, plan_config_fields, register_args, write_args
     from paper_2606_23087_b200 import binding as fp
-    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
     st = torch.cuda.current_stream().cuda_stream
-    PS = args.page_bytes
-    w = workloads.make_workload("frag_sweep", n_samples=args.samples or 65536, page_bytes=PS,
-                                pool_bytes=int(args.pool_gib * (1 << 30)))
+    pool_gib = args.pool_gib
+    if torch.cuda.mem_get_info()[0] < (pool_gib + 26) * (1 << 30):
+        pool_gib /= 2          # a box with less free memory runs the same churn through half the capacity
+    w = workloads.make_workload("frag_sweep", n_samples=getattr(args, "sweep_samples", None) or 65536, page_bytes=PS,
+                                pool_bytes=int(pool_gib * (1 << 30)))
     ops, residents = workloads.admit_free_schedule(w, cycles=args.cycles)
     pool = fp.Pool(fp.PoolConfig(**pool_config_fields(w)))
     if pool.rc != 0:
         raise fp.FlowpoolError(pool.rc, "pool_create")
+    apply_tuning(pool, args)
     pool.profile_enable(True)
     written_vis = 0
     consumed = 0
@@ -875,8 +986,8 @@ def run_sweep(args):
     n_mb, total_tokens, _ = plan.summary()
     # scheduler variants on the same residents: what each buys in padding waste and rank balance
     variants = {}
-    for name, fl, k_limit in (("as_printed", 0, 0), ("longest_first", 2, 0), ("sum_of_squares", 4, 0), ("carried_zigzag", 8, 0),
-                              ("all_three", 14, 0), ("auto_k_limit_64", 16, 64), ("fixed_k_64", 0, 64)):
+    for name, fl, k_limit in ((("as_printed", 0, 0), ("longest_first", 2, 0), ("sum_of_squares", 4, 0), ("carried_zigzag", 8, 0),
+                               ("all_three", 14, 0), ("auto_k_limit_64", 16, 64), ("fixed_k_64", 0, 64)) if with_variants else ()):
         vc = plan_config_fields(w, flags=fl)
         if k_limit:
             vc["n_buckets_K"] = k_limit
@@ -934,10 +1045,10 @@ def run_sweep(args):
         "metric": "packed-microbatch assembly GB/s after churn (fragmentation sweep)", "value": gbs, "unit": "GB/s",
         "n_gpus": 1, "higher_is_better": True, "dtype": "u8", "data": "synthetic",
         "config": {"workload": f"frag_sweep: stream of {w.n_samples} samples, hidden {w.hidden}, page {PS} B, pool "
-                               f"{args.pool_gib} GiB all HBM, {args.cycles} write/free cycles, budget {w.budget_L}",
+                               f"{pool_gib} GiB all HBM, {args.cycles} write/free cycles, budget {w.budget_L}",
                    "page_bytes": PS},
         "residents": len(residents), "stream_consumed": consumed, "packed_tokens": int(total_tokens), "microbatches": n_mb,
-        "gather_ms": gather_ms, "gather_launches": len(ranges), "frac_of_measured_peak": gbs / peak,
+        "gather_ms": gather_ms, "gather_launches": len(ranges), "frac_of_measured_peak": gbs / peak, "frac_of_nominal_8000": gbs / 8000.0,
         "write_gbs": 2 * written_vis * row_b / write_ms / 1e6, "write_ms_total": write_ms,
         "plan_ms_host_wall_median": float(np.median(plan_ms)),
         "internal_fragmentation": 1.0 - need_bytes / (used_pages * PS),
@@ -948,7 +1059,9 @@ def run_sweep(args):
         "gpu_launches": pool.stats()["gpu_launches"],
     }
     pool.destroy()
-    print(json.dumps(line))
+    del out, table
+    torch.cuda.empty_cache()
+    return line
 
 
 # ---------------------------------------------------------------------------------------------
@@ -1170,26 +1283,50 @@ def run_peer_two_processes(args):
                       "descriptor_blob_bytes": blob_bytes, "microbatches": n_mb, "sampled_row_matches": ok}))
 
 
-def run_exchange(args):
+class BlobExchange:
+    """Every rank's variable-length byte blob to every rank in one all_gather_into_tensor over preallocated,
+    length-prefixed fixed-size slots (no pickling on the per-step path)."""
+
+    def __init__(self, dist, cap, device):
+        import torch
+        self.dist, self.cap, self.world = dist, int(cap), dist.get_world_size()
+        self.send = torch.zeros(self.cap + 8, dtype=torch.uint8, device=device)
+        self.recv = torch.zeros(self.world * (self.cap + 8), dtype=torch.uint8, device=device)
+        self.stage = torch.zeros(self.cap + 8, dtype=torch.uint8, pin_memory=(device != "cpu"))
+
+    @staticmethod
+    def agree_cap(dist, nbytes, device):
+        """The largest blob over all ranks (one all_reduce, at set-up)."""
+        import torch
+        t = torch.tensor([int(nbytes)], dtype=torch.int64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return int(t.item())
+
+    def all_gather(self, blob):
+        blob = np.ascontiguousarray(blob, dtype=np.uint8)
+        n = len(blob)
+        if n > self.cap:
+            raise ValueError(f"blob of {n} bytes exceeds the exchange slot of {self.cap}")
+        st = self.stage.numpy()
+        st[:8] = np.frombuffer(np.uint64(n).tobytes(), dtype=np.uint8)
+        st[8:8 + n] = blob
+        self.send.copy_(self.stage)
+        self.dist.all_gather_into_tensor(self.recv, self.send)
+        r = self.recv.cpu().numpy().reshape(self.world, self.cap + 8)
+        return [r[i, 8:8 + int(r[i, :8].copy().view(np.uint64)[0])].copy() for i in range(self.world)]
+
+
+def exchange_measure(args, dist, rank, world, local, backend):
     """The paper's own setting (Sec. 3.2, 3.4) with one process per rank: every rank writes its batch into its own
     segment; mappings and slab handles are exchanged once, the samples' descriptors every step; every rank plans ALL
     samples (Algorithm 1 is deterministic, so the plans agree) and assembles only the microbatches dealt to it,
     reading the other ranks' pages in place (peer loads over NVLink when the ranks own different GPUs).  All pages
-    in HBM.  Launch under torchrun; FLOWPOOL_BENCH_BACKEND=gloo runs several ranks on one GPU (their kernels never
-    wait on one another), which is how this mode is exercised where only one GPU is at hand."""
+    in HBM.  Returns rank 0's summary (None elsewhere)."""
     import torch
-    import torch.distributed as dist
     import workloads
     from harness import pool_config_fields, plan_config_fields, register_args, write_args
     from paper_2606_23087_b200 import binding as fp
-    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0")) % max(1, torch.cuda.device_count())
-    torch.cuda.set_device(local)
-    backend = os.environ.get("FLOWPOOL_BENCH_BACKEND", "nccl")
-    if backend == "nccl":
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    else:
-        dist.init_process_group(backend)
+    dev = "cuda" if backend == "nccl" else "cpu"
     st = torch.cuda.current_stream().cuda_stream
     w = workloads.make_workload(args.workload, n_samples=args.samples, all_hbm=True)
     n = w.n_samples
@@ -1198,20 +1335,21 @@ def run_exchange(args):
              max_imported_pages=(world - 1) * (w.hbm_pages + w.host_pages), max_text_tokens=world * w.total_text_tokens_capacity)
     pool = fp.Pool(fp.PoolConfig(**f))
     assert pool.rc == 0, pool.rc
+    apply_tuning(pool, args)
     # once: everybody's mapping and slab handles
     rc1, mblob = pool.export_mapping()
     rc2, handles = pool.ipc_export()
     assert rc1 == 0 and rc2 == 0
-    everyone = [None] * world
-    dist.all_gather_object(everyone, (mblob.tobytes(), handles))
+    init_blob = np.concatenate([np.frombuffer(handles, np.uint8), mblob])
+    everyone = BlobExchange(dist, BlobExchange.agree_cap(dist, len(init_blob), dev), dev).all_gather(init_blob)
     opened = []
-    for r, (mb, hd) in enumerate(everyone):
+    for r, blob in enumerate(everyone):
         if r == rank:
             continue
-        rc, hbm, text = fp.ipc_open(hd)
+        rc, hbm, text = fp.ipc_open(blob[:fp.IPC_HANDLES_BYTES].tobytes())
         assert rc == 0, rc
         opened.append((hbm, text))
-        assert pool.import_mapping(np.frombuffer(mb, np.uint8), hbm, 0, text) == 0
+        assert pool.import_mapping(blob[fp.IPC_HANDLES_BYTES:], hbm, 0, text) == 0
     # own batch: global sample g = rank * n + s lives in slot g on every rank
     calls = []
     for call in w.write_calls:
@@ -1222,8 +1360,9 @@ def run_exchange(args):
         calls.append(((slots,) + tuple(reg[1:5]), torch.from_numpy(reg[5]).cuda(),
                       ((np.asarray(wr[0], np.uint32) + rank * n).astype(np.uint32),) + tuple(wr[1:]),
                       [workloads.span_values(w, s, j, device="cuda") for s, j in call]))
-    own = (np.asarray(w.plan_order, np.uint32) + rank * n).astype(np.uint32)
-    order = np.concatenate([(np.asarray(w.plan_order, np.uint32) + r * n) for r in range(world)]).astype(np.uint32)
+    plan_order = np.asarray(w.plan_order, np.uint32)
+    own = (plan_order + rank * n).astype(np.uint32)
+    order = np.concatenate([(plan_order + r * n) for r in range(world)]).astype(np.uint32)
     pc = plan_config_fields(w)
     pc["n_ranks_N"] = world
     pcfg = fp.PlanConfig(**pc)
@@ -1232,8 +1371,15 @@ def run_exchange(args):
     out = torch.empty((cap_rows, w.hidden), dtype=torch.bfloat16, device="cuda")
     cu = torch.empty((2 * world * n + 8,), dtype=torch.int32, device="cuda")
     pos = torch.empty((cap_rows,), dtype=torch.int32, device="cuda")
-    step_ms, my_rows, n_mb = [], 0, 0
+    vis_of = np.array([int(w.spans_of(s)[1].astype(np.int64).sum()) for s in range(n)], dtype=np.int64)
+    step_ms, my_rows, n_mb, remote_b, xchg = [], 0, 0, 0, None
+    pool.profile_enable(True)
+    sampler = ClockSampler(local)
     for it in range(args.warmup + args.steps):
+        if it == args.warmup:
+            pool.profile_read()
+            if rank == 0:
+                sampler.start()
         dist.barrier()
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -1241,14 +1387,14 @@ def run_exchange(args):
         for reg, ids, wr, srcs in calls:
             assert pool.register_samples(*reg, ids.data_ptr(), st) == 0
             assert pool.write_embeddings(*wr, [t.data_ptr() for t in srcs], w.src_dtype, st) == 0
-        rc, sblob = pool.export_samples(own, st)          # synchronises: this rank's pages are written
+        rc, sblob = pool.export_samples(own, st)          # returns with this rank's pages written
         assert rc == 0
-        blobs = [None] * world
-        dist.all_gather_object(blobs, sblob.tobytes())    # the per-round exchange of "lightweight metadata"
+        if xchg is None:                                  # first (warm-up) step: agree on the slot size, allocate once
+            xchg = BlobExchange(dist, BlobExchange.agree_cap(dist, len(sblob), dev), dev)
+        blobs = xchg.all_gather(sblob)                    # the per-round exchange of "lightweight metadata"
         for r in range(world):
             if r != rank:
-                theirs = (np.asarray(w.plan_order, np.uint32) + r * n).astype(np.uint32)
-                assert pool.import_samples(theirs, np.frombuffer(blobs[r], np.uint8), st) == 0
+                assert pool.import_samples((plan_order + r * n).astype(np.uint32), blobs[r], st) == 0
         rc, plan = pool.plan_microbatches(order, pcfg, st)
         assert rc == 0
         pa = plan.arrays()
@@ -1260,6 +1406,13 @@ def run_exchange(args):
             assert pool.gather_list(plan, mine, table.data_ptr(), w.vocab, out.data_ptr(), cu.data_ptr(), pos.data_ptr(), st) == 0
         e1.record()
         torch.cuda.synchronize()
+        # bytes this rank read from other ranks' memory: vision rows and token ids of the samples it assembled but does not own
+        remote_b = 0
+        for j in mine:
+            for g in pa["mb_samples"][pa["mb_sample_off"][j]:pa["mb_sample_off"][j + 1]]:
+                g = int(g)
+                if g // n != rank:
+                    remote_b += int(vis_of[g % n]) * w.row_bytes + 4 * int(w.seq_len[g % n])
         if mine and it == 0:
             # spot check against the generator: first and last row of the first sample of this rank's share
             q0 = int(pa["mb_sample_off"][mine[0]])
@@ -1277,7 +1430,7 @@ def run_exchange(args):
                 assert torch.equal(out[p_].view(torch.int16), want.to(torch.bfloat16).view(torch.int16)), (rank, g, p_)
         for r in range(world):
             if r != rank:
-                assert pool.free((np.asarray(w.plan_order, np.uint32) + r * n).astype(np.uint32), st) == 0
+                assert pool.free((plan_order + r * n).astype(np.uint32), st) == 0
         plan.destroy()
         torch.cuda.synchronize()
         dist.barrier()                                    # nobody reads this rank's pages any more
@@ -1285,24 +1438,59 @@ def run_exchange(args):
         torch.cuda.synchronize()
         if it >= args.warmup:
             step_ms.append(e0.elapsed_time(e1))
+    clocks = sampler.stop() if rank == 0 else None
+    prof = pool.profile_read()
     assert pool.status() == (0, 0)
     ms = float(np.median(step_ms))
-    t = torch.tensor([ms, float(my_rows)], dtype=torch.float64, device="cuda" if backend == "nccl" else "cpu")
-    mx = t.clone(); dist.all_reduce(mx, op=dist.ReduceOp.MAX)
-    sm = t.clone(); dist.all_reduce(sm, op=dist.ReduceOp.SUM)
-    ms_max, rows_all = float(mx[0]), float(sm[1])
+    g_ms = prof["gather_device"]["ms"] / max(1, args.steps)
+    t = torch.tensor([ms, float(my_rows), g_ms, float(remote_b)], dtype=torch.float64, device=dev)
+    allv = [torch.zeros_like(t) for _ in range(world)]
+    dist.all_gather(allv, t)
+    per = np.array([v.cpu().numpy() for v in allv])
+    ms_max, rows_all = float(per[:, 0].max()), float(per[:, 1].sum())
     wb, _ = algorithmic_bytes(w)
     moved = world * wb + rows_all * 4 * w.hidden
     pool.destroy()
     for hbm, text in opened:
         fp.ipc_close(hbm, text)
+    if rank != 0:
+        return None
+    peak, peak_src = measured_peak()
+    nvlink_gbs = 770.0      # measured peer copy per direction on this machine
+    n_dev = min(world, torch.cuda.device_count())
+    per_rank = []
+    for r in range(world):
+        rows_r, gms_r, rem_r = float(per[r, 1]), float(per[r, 2]), float(per[r, 3])
+        gb_r = rows_r * 4 * w.hidden
+        # rows read from a peer GPU cannot come faster than the link; ranks that share one GPU share its HBM instead
+        bound_ms = max(gb_r / peak, rem_r / nvlink_gbs if n_dev > 1 else 0.0) / 1e6
+        per_rank.append({"rank": r, "rows": int(rows_r), "gather_ms": gms_r, "gather_gbs": gb_r / gms_r / 1e6 if gms_r > 0 else None,
+                         "bytes_from_peers": int(rem_r), "roofline_bound_ms": bound_ms, "frac_of_bound": bound_ms / gms_r if gms_r > 0 else None})
+    slow = max(per_rank, key=lambda x: x["gather_ms"])
+    return {"metric": METRIC + ", ranks exchanging descriptors and reading each other's pages in place", "value": moved / ms_max / 1e6,
+            "unit": UNIT, "ms_per_step": ms_max, "tokens_per_s": rows_all / ms_max * 1e3,
+            "config": {"workload": workload_label(args, all_hbm=True), "ranks": world, "gpus_used": n_dev, "backend": backend, "microbatches": n_mb,
+                       "packed_tokens_all_ranks": int(rows_all), "pool": "all pages in HBM (host-tier slabs are not shared between processes)",
+                       "exchange": "descriptors per step by all_gather_into_tensor over preallocated length-prefixed slots; host time included"},
+            "per_rank": per_rank,
+            "bytes_over_nvlink_per_step": int(per[:, 3].sum()) if n_dev > 1 else 0,
+            "bytes_from_peer_processes_per_step": int(per[:, 3].sum()),
+            "roofline": {"kernel": "k_gather (list layout), slowest rank", "bound": "hbm" if slow["roofline_bound_ms"] * 1e6 * peak >= slow["rows"] * 4 * w.hidden * 0.999 else "nvlink",
+                         "achieved": slow["gather_gbs"], "peak": peak, "unit": "GB/s", "frac": slow["frac_of_bound"],
+                         "peak_source": peak_src + "; peer rows bounded by 770 GB/s per direction (measured peer copy)"},
+            "clocks": clocks}
+
+
+def run_exchange(args):
+    """--exchange: the multi-rank flow alone (under torchrun), one JSON line."""
+    import torch
+    dist, rank, local, world, backend = init_dist(torch)
+    assert dist is not None, "--exchange needs torchrun (or --gpus N, which launches it)"
+    ex = exchange_measure(args, dist, rank, world, local, backend)
     if rank == 0:
-        print(json.dumps({"metric": METRIC + ", ranks exchanging descriptors and reading each other's pages in place", "value": moved / ms_max / 1e6,
-                          "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_max,
-                          "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
-                          "config": {"workload": workload_label(args), "ranks": world, "gpus_used": min(world, torch.cuda.device_count()),
-                                     "backend": backend, "microbatches": n_mb, "packed_tokens_all_ranks": int(rows_all)},
-                          "tokens_per_s": rows_all / ms_max * 1e3}))
+        ex.update({"n_gpus": world, "steps": args.steps, "warmup": args.warmup, "higher_is_better": True, "scaling": "weak",
+                   "vs_baseline": None, "dtype": "u8", "data": "synthetic"})
+        print(json.dumps(ex))
     dist.barrier()
     dist.destroy_process_group()
 
@@ -1383,6 +1571,51 @@ def run_peer(args):
     print(json.dumps(line))
 
 
+def self_launch(args):
+    """--gpus N means N ranks.  Outside torchrun (no WORLD_SIZE in the environment) this process re-executes itself
+    under `python -m torch.distributed.run` with N ranks on this node and passes their exit code on; under torchrun
+    the world size must be the N asked for.  The reference arm needs no ranks: rank 0 alone runs it."""
+    if args.impl == "reference":
+        return
+    ws = os.environ.get("WORLD_SIZE")
+    if ws is not None:
+        if int(ws) != args.gpus:
+            raise SystemExit(f"bench.py: --gpus {args.gpus} but WORLD_SIZE={ws}: launch with --nproc-per-node {args.gpus}")
+        return
+    if args.gpus <= 1:
+        return
+    import socket
+    with socket.socket() as so:
+        so.bind(("127.0.0.1", 0))
+        port = so.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}", "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    raise SystemExit(subprocess.call(cmd))
+
+
+def run_host_logic_only(args):
+    """The multi-rank plumbing of this script without a GPU (gloo on CPU): process group, slot-size agreement, the
+    length-prefixed descriptor all-gather with blobs of different lengths, max-over-ranks timing, rank-0-only line."""
+    import torch
+    import torch.distributed as dist
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    dist.init_process_group("gloo")
+    blob = np.arange(100 + 37 * rank, dtype=np.uint64).view(np.uint8) ^ np.uint8(rank)
+    xchg = BlobExchange(dist, BlobExchange.agree_cap(dist, len(blob), "cpu"), "cpu")
+    ok = True
+    for _ in range(2):
+        got = xchg.all_gather(blob)
+        for r in range(world):
+            want = np.arange(100 + 37 * r, dtype=np.uint64).view(np.uint8) ^ np.uint8(r)
+            ok = ok and len(got[r]) == len(want) and bool(np.array_equal(got[r], want))
+    ms = max_over_ranks(10.0 + rank, dist, device="cpu")
+    if rank == 0:
+        print(json.dumps({"host_logic_only": True, "n_gpus": world, "blobs_ok": ok, "ms_per_step": ms,
+                          "value": aggregate_value(1e6, world, ms), "unit": UNIT}))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -1404,9 +1637,15 @@ def main():
     ap.add_argument("--exchange", action="store_true", help="under torchrun: every rank writes its batch, all plan everything, each assembles its own share from everybody's pages")
     ap.add_argument("--two-processes", action="store_true", help="with --via-peer: the producer pool lives in a process of its own (CUDA IPC)")
     ap.add_argument("--via-peer", action="store_true", help="producer and consumer are two processes' pools of one GVA space")
+    ap.add_argument("--skip-configs", action="store_true", help="skip the short passes over the other configurations")
+    ap.add_argument("--host-logic-only", action="store_true",
+                    help="no GPU work: rendezvous, the descriptor exchange and the rank-0 line only (checks of this script on CPU)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
-    if args.impl == "reference":
+    self_launch(args)
+    if args.host_logic_only:
+        run_host_logic_only(args)
+    elif args.impl == "reference":
         run_reference(args)
     elif args.workload == "frag_sweep":
         run_sweep(args)

@@ -200,7 +200,8 @@ struct ft_plan {
   std::vector<uint64_t> slot_generation;
   std::vector<uint32_t> h_mb_sample_off;  // host copies used to size gathers
   std::vector<uint64_t> h_mb_row_off;
-  void* d_block = nullptr;                // one stream-ordered allocation holding every array below
+  void* d_block = nullptr;                // one device block holding every array below (from the pool's block cache)
+  size_t block_cap = 0;
   cudaStream_t last_stream = nullptr;     // stream of the plan's latest device work (creation, then gathers)
   uint32_t *d_slots, *d_len, *d_sample_mb, *d_sample_rank, *d_mb_sample_off, *d_mb_samples, *d_plan_sample_mb;
   uint32_t *d_mb_tokens, *d_mb_lmax, *d_mb_residual, *d_mb_count, *d_mb_bucket, *d_mb_rank, *d_mb_pos;
@@ -221,6 +222,10 @@ inline PlanView make_plan_view(const ft_plan* pl) {
 // of the plan is READY in the generation the plan was made for, else FT_ERR_NOT_READY.
 inline int32_t plan_alive(const ft_pool* p, const ft_plan* pl);
 int32_t cuda_fail(cudaError_t e, const char* what);
+// pools that exist (a plan may outlive its pool: plan_destroy must not touch a dead pool's block cache)
+void pool_registry_add(ft_pool* p);
+void pool_registry_remove(ft_pool* p);
+bool pool_registry_has(ft_pool* p);
 #define FT_CUDA(call)                                          \
   do {                                                         \
     cudaError_t e__ = (call);                                  \
@@ -294,6 +299,11 @@ struct ft_pool {
   uint64_t synced_seq[2] = {~0ull, ~0ull};             // ... and the batch count they waited for
   uint64_t status_base = 0;           // call_seq at the last pool_status read
   std::vector<uint8_t> noalloc_blob;  // host staging of pool_write_embeddings_noalloc, made at pool_create
+  // Device blocks of destroyed plans, kept for the next plan: each with an event behind the last kernel that read it.
+  // (A stream-ordered allocation would do, but a block freed on the stream of the last assembly and asked for again
+  // on the metadata stream is not reusable across streams at once, and every other plan paid a fresh allocation.)
+  struct plan_block { void* d; size_t cap; cudaEvent_t ev; };
+  std::vector<plan_block> plan_cache;
   void* plan_pinned = nullptr;        // pinned landing zone of the plan's summary read-back
   size_t plan_pinned_cap = 0;
   std::vector<uint32_t> bind_hbm, bind_host;           // vpn -> frame of this process's binding (exported to peers)

@@ -368,11 +368,7 @@ int32_t plan_device_setup(ft_pool* p) {
   FT_CUDA(cudaFuncSetAttribute(k_bestfit<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBestfitSmemLimit));
   FT_CUDA(cudaFuncSetAttribute(k_bestfit<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBestfitSmemLimit));
   FT_CUDA(cudaFuncSetAttribute(k_bestfit<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBestfitSmemLimit));
-  // keep freed plan blocks cached in the device's default memory pool instead of returning them to the driver
-  cudaMemPool_t mp;
-  uint64_t keep = ~0ull;
-  if (cudaDeviceGetDefaultMemPool(&mp, p->device) == cudaSuccess) cudaMemPoolSetAttribute(mp, cudaMemPoolAttrReleaseThreshold, &keep);
-  cudaGetLastError();
+  (void)p;
   return FT_OK;
 }
 }  // namespace ft
@@ -381,8 +377,21 @@ using namespace ft;
 
 extern "C" __attribute__((visibility("default"))) int32_t plan_destroy(ft_plan* pl) {
   if (!pl) return FT_ERR_INVALID_ARG;
-  // stream-ordered free: the block is released after the plan's last kernel, with no device-wide synchronisation
-  if (pl->d_block && cudaFreeAsync(pl->d_block, pl->last_stream) != cudaSuccess) { cudaGetLastError(); cudaDeviceSynchronize(); cudaFree(pl->d_block); }
+  if (pl->d_block) {
+    ft_pool* p = pl->pool;
+    cudaEvent_t ev = nullptr;
+    // the block goes back to its pool's cache behind an event on the stream of the plan's last kernel: no
+    // synchronisation here, and the next plan takes a block whose event has completed
+    if (ft::pool_registry_has(p) && p->plan_cache.size() < 8 && cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) == cudaSuccess &&
+        cudaEventRecord(ev, pl->last_stream) == cudaSuccess) {
+      p->plan_cache.push_back({pl->d_block, pl->block_cap, ev});
+    } else {
+      if (ev) cudaEventDestroy(ev);
+      cudaGetLastError();
+      cudaDeviceSynchronize();
+      cudaFree(pl->d_block);
+    }
+  }
   delete pl;
   return FT_OK;
 }
@@ -444,8 +453,38 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_plan_microbatches
   const size_t o_roff = take(((size_t)N + 1) * 4), o_rmbs = take(n * 4), o_rcnt = take((size_t)N * 4);
   const size_t o_tiles = take(n_tiles * 4), o_scal = take(SC_COUNT * 4);
   pl->last_stream = st;
-  cudaError_t e = cudaMallocAsync(&pl->d_block, off, st);
-  if (e != cudaSuccess) { delete pl; return ft::cuda_fail(e, "cudaMalloc(plan)"); }
+  {
+    // a cached block that is large enough: one nobody reads any more if there is one, else the metadata stream
+    // waits for its last reader; a fresh allocation only when the cache has none
+    int pick = -1;
+    for (int i = 0; i < (int)p->plan_cache.size(); ++i) {
+      if (p->plan_cache[i].cap < off) continue;
+      const bool done = cudaEventQuery(p->plan_cache[i].ev) == cudaSuccess;
+      if (done) { pick = i; break; }
+      if (pick < 0) pick = i;
+    }
+    cudaGetLastError();
+    if (pick >= 0) {
+      ft_pool::plan_block b = p->plan_cache[pick];
+      p->plan_cache.erase(p->plan_cache.begin() + pick);
+      cudaError_t e = cudaStreamWaitEvent(st, b.ev, 0);
+      cudaEventDestroy(b.ev);
+      if (e != cudaSuccess) { cudaFree(b.d); delete pl; return ft::cuda_fail(e, "cudaStreamWaitEvent(plan block)"); }
+      pl->d_block = b.d; pl->block_cap = b.cap;
+    } else {
+      if (!p->plan_cache.empty()) {  // only blocks that are too small: let one go, so that the cache cannot clog
+        ft_pool::plan_block b = p->plan_cache.front();
+        p->plan_cache.erase(p->plan_cache.begin());
+        cudaEventSynchronize(b.ev); cudaEventDestroy(b.ev); cudaFree(b.d);
+        cudaGetLastError();
+      }
+      size_t cap = 1 << 20;
+      while (cap < off) cap <<= 1;
+      cudaError_t e = cudaMalloc(&pl->d_block, cap);
+      if (e != cudaSuccess) { delete pl; return ft::cuda_fail(e, "cudaMalloc(plan)"); }
+      pl->block_cap = cap;
+    }
+  }
   uint8_t* b = static_cast<uint8_t*>(pl->d_block);
 #define U32(o) reinterpret_cast<uint32_t*>(b + (o))
 #define U64(o) reinterpret_cast<uint64_t*>(b + (o))

@@ -13,6 +13,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <unordered_set>
 
 #include "bulk_copy.cuh"
@@ -22,6 +23,12 @@ namespace ft {
 
 // one caller thread per pool, so a per-thread string is per pool as far as any caller can tell
 static thread_local char g_last_error[512] = "";
+
+static std::mutex g_pools_mu;
+static std::unordered_set<ft_pool*> g_pools;
+void pool_registry_add(ft_pool* p) { std::lock_guard<std::mutex> l(g_pools_mu); g_pools.insert(p); }
+void pool_registry_remove(ft_pool* p) { std::lock_guard<std::mutex> l(g_pools_mu); g_pools.erase(p); }
+bool pool_registry_has(ft_pool* p) { std::lock_guard<std::mutex> l(g_pools_mu); return g_pools.count(p) != 0; }
 
 int32_t cuda_fail(cudaError_t e, const char* what) {
   snprintf(g_last_error, sizeof(g_last_error), "%s: %s", what, cudaGetErrorString(e));
@@ -59,7 +66,7 @@ int32_t ctx_acquire(ft_pool* p, int side, size_t blob_bytes, size_t total_bytes,
   if (c.dcap < total_bytes) {
     if (c.busy_done) { FT_CUDA(cudaEventSynchronize(c.ev_done)); c.busy_done = false; }  // nobody reads the old scratch
     if (c.d) FT_CUDA(cudaFree(c.d));
-    size_t cap = 1 << 20;
+    size_t cap = 1 << 18;
     while (cap < total_bytes) cap <<= 1;
     c.d = nullptr; c.dcap = 0;
     FT_CUDA(cudaMalloc(&c.d, cap));
@@ -603,6 +610,8 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_destroy(ft_pool* 
     if (c.ev_up) cudaEventDestroy(c.ev_up);
     if (c.ev_done) cudaEventDestroy(c.ev_done);
   }
+  ft::pool_registry_remove(p);
+  for (auto& b : p->plan_cache) { if (b.d) cudaFree(b.d); if (b.ev) cudaEventDestroy(b.ev); }
   if (p->plan_pinned) cudaFreeHost(p->plan_pinned);
   if (p->meta) cudaStreamDestroy(p->meta);
   if (p->ev_meta) cudaEventDestroy(p->ev_meta);
@@ -671,9 +680,16 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_create(const ft_p
   CK(cudaEventCreateWithFlags(&p->ev_meta, cudaEventDisableTiming));
   CK(cudaEventCreateWithFlags(&p->ev_in, cudaEventDisableTiming));
   CK(cudaEventCreateWithFlags(&p->ev_noalloc, cudaEventDisableTiming));
+  // every call context starts with 64 KiB of pinned staging and 256 KiB of device scratch (enough for calls of a few
+  // thousand spans), so that no call of ordinary size allocates; larger calls grow their context on demand
   for (int side = 0; side < 2; ++side) for (int i = 0; i < kCallCtx; ++i) {
-    CK(cudaEventCreateWithFlags(&p->ctx[side][i].ev_up, cudaEventDisableTiming));
-    CK(cudaEventCreateWithFlags(&p->ctx[side][i].ev_done, cudaEventDisableTiming));
+    ft_call_ctx& cx = p->ctx[side][i];
+    CK(cudaEventCreateWithFlags(&cx.ev_up, cudaEventDisableTiming));
+    CK(cudaEventCreateWithFlags(&cx.ev_done, cudaEventDisableTiming));
+    CK(cudaHostAlloc(&cx.h, 1 << 16, cudaHostAllocDefault));
+    cx.hcap = 1 << 16;
+    CK(cudaMalloc(&cx.d, 1 << 18));
+    cx.dcap = 1 << 18;
   }
   p->noalloc_blob.resize(16 * (size_t)FT_NOALLOC_MAX_SPANS + 256);
   // per-device kernel set-up: shared-memory opt-ins and occupancy of the data kernels
@@ -806,6 +822,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_create(const ft_p
   p->slots.resize(c.max_samples);
   p->spans.resize(span_ids);
   p->free_pages = P; p->free_text_pages = n_text; p->free_blocks = NB;
+  ft::pool_registry_add(p);
   *out = p;
   return FT_OK;
 }

@@ -65,3 +65,35 @@ def test_reference_arm_other_ranks_exit_without_work():
     out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2"],
                          capture_output=True, text=True, timeout=120, cwd=ROOT, env=env)
     assert out.returncode == 0 and out.stdout.strip() == ""
+
+
+def test_gpus_n_launches_n_ranks_by_itself():
+    """`bench.py --gpus 2` with no torchrun around it must start two ranks (here: the host-side plumbing only, gloo on
+    CPU): rendezvous, slot-size agreement, the length-prefixed descriptor all-gather, one line from rank 0."""
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--host-logic-only"],
+                         capture_output=True, text=True, timeout=600, cwd=ROOT, env=env)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [json.loads(l) for l in out.stdout.strip().splitlines() if l.startswith("{")]
+    assert len(lines) == 1                                  # only rank 0 prints
+    assert lines[0]["n_gpus"] == 2 and lines[0]["blobs_ok"] is True
+    assert lines[0]["ms_per_step"] == 11.0                  # the slower rank's time
+
+
+def test_world_size_must_match_gpus():
+    env = dict(os.environ, WORLD_SIZE="1", RANK="0", LOCAL_RANK="0")
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "8", "--host-logic-only"],
+                         capture_output=True, text=True, timeout=120, cwd=ROOT, env=env)
+    assert out.returncode != 0 and "n_gpus" not in out.stdout
+
+
+def test_blob_exchange_refuses_an_oversized_blob():
+    import numpy as np
+    import pytest
+
+    class FakeDist:
+        def get_world_size(self):
+            return 1
+    x = bench.BlobExchange(FakeDist(), 16, "cpu")
+    with pytest.raises(ValueError):
+        x.all_gather(np.zeros(17, np.uint8))
