@@ -1086,6 +1086,7 @@ def run_streaming(args, all_hbm, batches=6, warm=2):
     pool = fp.Pool(fp.PoolConfig(**f))
     if pool.rc != 0:
         raise fp.FlowpoolError(pool.rc, "pool_create")
+    apply_tuning(pool, args)
     prod, cons = torch.cuda.Stream(), torch.cuda.Stream()
     table = workloads.embed_table(w, device="cuda")
     calls = []
@@ -1129,6 +1130,8 @@ def run_streaming(args, all_hbm, batches=6, warm=2):
     for k in range(total):
         if k == warm:
             torch.cuda.synchronize()
+            pool.profile_read()
+            pool.profile_enable(True)
             t0 = time.perf_counter()
         slots, plan = assemble(k)
         produce(k + 1)
@@ -1136,6 +1139,9 @@ def run_streaming(args, all_hbm, batches=6, warm=2):
         plan.destroy()
     torch.cuda.synchronize()
     ms = (time.perf_counter() - t0) * 1e3 / batches
+    prof = pool.profile_read()
+    pool.profile_enable(False)
+    kernel_ms = {k: v["ms"] / batches for k, v in prof.items() if v["launches"]}
     # drain the batch that was produced but never consumed
     rc, slots, _ = pool.take_ready(1, n)
     if rc == 0 and len(slots):
@@ -1146,7 +1152,8 @@ def run_streaming(args, all_hbm, batches=6, warm=2):
     del calls, outs, table
     torch.cuda.empty_cache()
     return {"ms_per_batch": ms, "value": (wb + gb) / ms / 1e6, "unit": UNIT, "tokens_per_s": w.total_tokens / ms * 1e3,
-            "batches": batches, "pool": "two batches resident, same tier split, tiers interleaved in the free ring",
+            "batches": batches, "kernel_ms_per_batch": kernel_ms,
+            "pool": "two batches resident, same tier split, tiers interleaved in the free ring",
             "note": "host wall clock over steady-state batches; producer and consumer on two streams"}
 
 
@@ -1637,6 +1644,7 @@ def main():
     ap.add_argument("--exchange", action="store_true", help="under torchrun: every rank writes its batch, all plan everything, each assembles its own share from everybody's pages")
     ap.add_argument("--two-processes", action="store_true", help="with --via-peer: the producer pool lives in a process of its own (CUDA IPC)")
     ap.add_argument("--via-peer", action="store_true", help="producer and consumer are two processes' pools of one GVA space")
+    ap.add_argument("--streaming-only", action="store_true", help="only the two-stream producer/consumer measurement")
     ap.add_argument("--skip-configs", action="store_true", help="skip the short passes over the other configurations")
     ap.add_argument("--host-logic-only", action="store_true",
                     help="no GPU work: rendezvous, the descriptor exchange and the rank-0 line only (checks of this script on CPU)")
@@ -1651,6 +1659,10 @@ def main():
         run_sweep(args)
     elif args.backbone_only:
         run_backbone_only(args)
+    elif args.streaming_only:
+        import torch
+        torch.cuda.set_device(0)
+        print(json.dumps({"streaming": run_streaming(args, args.all_hbm), "workload": workload_label(args)}))
     elif args.exchange:
         args.all_hbm = True
         run_exchange(args)

@@ -311,6 +311,15 @@ int32_t pool_gather_list(ft_pool* pool, const ft_plan* plan, const uint32_t* mb_
  */
 int32_t pool_free(ft_pool* pool, const uint32_t* sample_slot, uint32_t n, void* stream);
 
+/*
+ * FT_ERR_TIMEOUT is the one asynchronous error that is not about the caller's data.  The host-tier kernels move pages
+ * with bulk-asynchronous copies and wait for each staged load on an mbarrier; that wait, the library's only device-side
+ * spin, gives up after 2 s of wall clock (a host link that has stopped answering).  The CTA then issues no further
+ * copy, waits once more -- again at most 2 s -- for the loads it had already issued, and returns; detail = CTA index
+ * (low 16 bits) | loads that had still not arrived when it returned (high 16 bits; 0 means that none can land later).
+ * The bytes of that call are incomplete and the pool's state is no longer trustworthy: after FT_ERR_TIMEOUT the only
+ * call a pool still supports is pool_destroy.
+ */
 /* First asynchronous error since the last call of pool_status (smallest call, then smallest code, then smallest
  * detail), then cleared.  Synchronises the device.  Calls are numbered from the last read, on 28 bits: read the
  * status at least once every 2^28 calls of the pool (a training run that checks it once per step never comes close). */
@@ -341,7 +350,9 @@ int32_t pool_take_ready(ft_pool* pool, uint64_t min_tokens, uint32_t max_samples
  *                     buf = NULL queries the size.  CAPACITY if cap is too small.
  * pool_import_mapping installs a peer's binding: builds that process's page-table arrays from the blob and the
  *                     three base addresses at which this device reaches the peer's HBM slab, host slab and text
- *                     frames.  INVALID_ARG: malformed blob, another GVA space, own rank, missing or misaligned
+ *                     frames.  HBM frames of a slab that lives on another GPU are flagged remote (the transport is
+ *                     chosen by where source and destination are, Sec. 3.2): assemblies read them with a separate,
+ *                     small bulk-copy launch beside the one that streams local HBM.  INVALID_ARG: malformed blob, another GVA space, own rank, missing or misaligned
  *                     base; SLOT_IN_USE: that rank was imported before.  Init-time: allocates, synchronises.
  * pool_export_samples descriptors of READY samples (lengths, spans with their token grids, page GVAs, text-page GVAs) into a host buffer
  *                     -- the "lightweight metadata" a consumer needs; no embedding bytes.  Synchronises `stream`.
@@ -443,7 +454,7 @@ int32_t pool_embed_grad(ft_pool* pool, const ft_plan* plan, uint32_t mb_begin, u
  * since the last read, and clears them.  Classes: a single-tier pool's kernels count under its tier.
  */
 enum { FT_K_GATHER_DEVICE = 0, FT_K_GATHER_HOST = 1, FT_K_SCATTER_DEVICE = 2, FT_K_SCATTER_HOST = 3, FT_K_EMBED_GRAD = 4,
-       FT_K_COUNT = 5 };
+       FT_K_GATHER_REMOTE = 5, FT_K_COUNT = 6 };
 typedef struct {
   double ms;
   uint64_t launches;
@@ -467,11 +478,17 @@ int32_t pool_profile_read(ft_pool* pool, ft_kernel_time* out /* host [FT_K_COUNT
  *   gather_unroll        16-byte vectors per lane in flight in the gather kernel (4 or 8; default 4)
  *   grad_ctas_per_sm     CTAs per SM of the table-gradient kernel (default 6; 1..8)
  *   grad_hot_threshold   rows from which an id takes the frequent-id gradient kernel (default rows / (8 x grid), >= 64)
+ *   remote_ctas          grid of the bulk-copy gather that reads frames in ANOTHER GPU's HBM (default 16): like the
+ *                        host tier, peer frames are long-latency sources and get a small grid of their own, so that the
+ *                        SMs that stream local HBM keep their memory pipelines; to be tuned where a second GPU exists
+ *   peers_remote         1: pool_import_mapping flags every peer's HBM frames as remote even when they are on this
+ *                        device (exercises the remote path on one GPU); 0: only frames of another device are remote
  */
 typedef struct {
   uint32_t dev_ctas_per_sm, scatter_ctas_per_sm, scatter_group, chunk_shift;
   uint32_t host_ctas, host_store_ctas, gather_unroll, grad_ctas_per_sm, grad_hot_threshold;
-  uint32_t reserved[7];
+  uint32_t remote_ctas, peers_remote;
+  uint32_t reserved[5];
 } ft_tuning;
 int32_t pool_get_tuning(ft_pool* pool, ft_tuning* out);
 int32_t pool_set_tuning(ft_pool* pool, const ft_tuning* in);

@@ -66,18 +66,18 @@ class PoolStats(C.Structure):
 
 
 TUNING_FIELDS = ("dev_ctas_per_sm", "scatter_ctas_per_sm", "scatter_group", "chunk_shift", "host_ctas", "host_store_ctas",
-                 "gather_unroll", "grad_ctas_per_sm", "grad_hot_threshold")
+                 "gather_unroll", "grad_ctas_per_sm", "grad_hot_threshold", "remote_ctas", "peers_remote")
 
 
 class Tuning(C.Structure):
-    _fields_ = [(k, C.c_uint32) for k in TUNING_FIELDS] + [("reserved", C.c_uint32 * 7)]
+    _fields_ = [(k, C.c_uint32) for k in TUNING_FIELDS] + [("reserved", C.c_uint32 * 5)]
 
 
 class KernelTime(C.Structure):
     _fields_ = [("ms", C.c_double), ("launches", C.c_uint64)]
 
 
-KERNEL_CLASSES = ("gather_device", "gather_host", "scatter_device", "scatter_host", "embed_grad")
+KERNEL_CLASSES = ("gather_device", "gather_host", "scatter_device", "scatter_host", "embed_grad", "gather_remote")
 
 IPC_HANDLES_BYTES = 2 * 64 + 8   # ft_ipc_handles
 

@@ -3,6 +3,12 @@
 // One thread keeps `kDepth` loads in flight, so a handful of single-warp CTAs saturate a long-latency link
 // (mapped pinned host memory) without tying up the load/store pipelines of the SMs that stream HBM.
 // Every copy lands in the issuing CTA only.  Every wait is bounded.
+//
+// Giving up.  A staged load that has not arrived after kBulkWaitLimitNs is declared lost: the ring issues no further
+// load or store, and before the CTA returns drain() waits once more, again bounded, for every load it had already
+// issued, so that none of them can land later in shared memory that by then belongs to another CTA; `stranded`
+// counts the loads that had still not arrived when that second wait ran out as well (the kernel reports it in the
+// error detail).  Stores already issued are waited for with the hardware's group wait.
 #pragma once
 #include <stdint.h>
 
@@ -57,11 +63,12 @@ struct BulkRing {
   uint64_t* dst_q;   // kBulkStages pending destinations (shared memory)
   uint32_t* len_q;   // kBulkStages pending staged lengths
   uint64_t issued, retired;
+  uint32_t stranded;  // loads still not arrived when a CTA that gave up returned
   bool lost;
 
   __device__ void init(uint8_t* stage_, uint64_t* bar_, uint64_t* dst_q_, uint32_t* len_q_) {
     stage = stage_; bar = bar_; dst_q = dst_q_; len_q = len_q_;
-    issued = retired = 0; lost = false;
+    issued = retired = 0; lost = false; stranded = 0;
     if ((threadIdx.x & 31) == 0) {
       for (int i = 0; i < kBulkStages; ++i) mbar_init(&bar[i], 1);
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -110,6 +117,22 @@ struct BulkRing {
   }
   __device__ void drain() {
     while (!lost && retired < issued) retire_one();
+    if (lost) {
+      // gave up: the loads issued before that are still owed to this CTA's shared memory; wait for them, bounded
+      uint32_t left = 0;
+      if ((threadIdx.x & 31) == 0) {
+        const uint64_t t0 = global_timer_ns();
+        for (uint64_t k = retired - 1; k < issued; ++k) {  // retired - 1 is the load whose wait ran out
+          const int st = (int)(k % kBulkStages);
+          const uint32_t parity = (uint32_t)((k / kBulkStages) & 1);
+          bool here = mbar_try_wait(&bar[st], parity);
+          uint32_t spins = 0;
+          while (!here && !((++spins & 1023u) == 0 && global_timer_ns() - t0 > kBulkWaitLimitNs)) here = mbar_try_wait(&bar[st], parity);
+          if (!here) ++left;
+        }
+      }
+      stranded = __shfl_sync(0xFFFFFFFFu, left, 0);
+    }
     if ((threadIdx.x & 31) == 0) bulk_wait_all<0>();
     __syncwarp();
   }

@@ -15,7 +15,7 @@ namespace ft {
 constexpr uint32_t kTextPageIds = 1024;       // ids per 4 KiB text page
 constexpr uint32_t kListBlock = 64;           // page GVAs per list block (two-level span page lists)
 constexpr uint32_t kNone = 0xFFFFFFFFu;
-constexpr uint64_t kPteValid = 1, kPteHost = 2, kPteText = 4, kPteFlagMask = 0xFF;
+constexpr uint64_t kPteValid = 1, kPteHost = 2, kPteText = 4, kPteRemote = 8, kPteFlagMask = 0xFF;  // Remote: HBM of another GPU
 
 struct RingState {
   uint32_t head;   // index of the oldest free entry
@@ -311,11 +311,13 @@ struct ft_pool {
   std::vector<void*> peer_allocs;                      // imported peers' page-table arrays
   std::vector<uint8_t> peer_imported;                  // [world_size]
   bool peer_host_frames = false;                       // some imported peer binds host-tier pages
+  bool peer_remote_frames = false;                     // some imported peer's HBM frames live on another GPU
   std::vector<std::array<uint64_t, 3>> peer_bases;     // [world_size] slab addresses (HBM, host, text) as seen here
   // host-tier traffic runs beside the HBM kernels on a side stream: one per side (0 producer, 1 consumer), so that
   // host-tier writes and host-tier reads of concurrent calls can use both directions of the link at once
-  cudaStream_t side_stream[2] = {nullptr, nullptr};
-  cudaEvent_t fork_ev[2] = {nullptr, nullptr}, join_ev[2] = {nullptr, nullptr};
+  // (index 2: the consumer side's stream for frames in another GPU's HBM, read over NVLink)
+  cudaStream_t side_stream[3] = {nullptr, nullptr, nullptr};
+  cudaEvent_t fork_ev[3] = {nullptr, nullptr, nullptr}, join_ev[3] = {nullptr, nullptr, nullptr};
   // cross-stream ordering when the producer side and the consumer side are driven from different streams
   cudaEvent_t ev_producer = nullptr, ev_consumer = nullptr;  // end of the latest producer-side / consumer-side call
   cudaStream_t last_producer_stream = nullptr, last_consumer_stream = nullptr;
@@ -329,6 +331,9 @@ struct ft_pool {
                                 // accesses do not clog the memory pipelines of the SMs that stream HBM; 6 rather
                                 // than 8 because a write and a read kernel running together (two streams) share
                                 // the link better with fewer requests in flight
+  int remote_ctas = 16;         // grid of the bulk-copy gather from another GPU's HBM (about 128 KiB in flight per CTA;
+                                // 770 GB/s x a few microseconds of NVLink latency wants 1.5 MB and more in flight)
+  int peers_remote = 0;         // 1: flag every imported peer's HBM frames as remote, whatever device they are on
   int host_store_ctas = 8;      // grid of the vector-store scatter into host frames (fp32 sources, host-only pools)
   int chunk_shift = 16;         // log2 of k_scatter's work unit in bytes of a span's image (14..21)
   int scatter_group = 0;        // chunks per round-robin group of k_scatter; 0 = the measured default

@@ -192,8 +192,8 @@ __global__ void __launch_bounds__(kGatherThreads) k_gather(PoolView v, PlanView 
         auto src_of = [&](uint32_t x, bool* take) -> const uint4* {
           const uint32_t ab = off0 + (x << 4);
           const uint64_t pte = dr.seg[ab >> shift];
-          const bool host = (pte & kPteHost) != 0;
-          *take = MODE == kTierAll || (MODE == kTierHostOnly) == host;
+          const bool far = (pte & (kPteHost | kPteRemote)) != 0;  // host-tier frame, or a frame in another GPU's HBM
+          *take = MODE == kTierAll || !far;                     // (far frames have launches of their own)
           return reinterpret_cast<const uint4*>((pte & ~kPteFlagMask) + (ab & mask));
         };
         // U vectors per lane in flight before the first store
@@ -223,7 +223,7 @@ __global__ void __launch_bounds__(kGatherThreads) k_gather(PoolView v, PlanView 
 // contiguous byte range of the output: each host-tier page becomes a few bulk copies host frame -> shared ->
 // output, read in place over the mapped pointer.  One warp per CTA: the lanes translate 32 page ordinals at a
 // time (page list -> GVA -> page-table entry), lane 0 drives the copy ring.  A handful of CTAs saturate the link.
-__global__ void __launch_bounds__(32) k_gather_host_bulk(PoolView v, PlanView pl, GatherArgs a) {
+__global__ void __launch_bounds__(32) k_gather_host_bulk(PoolView v, PlanView pl, GatherArgs a, uint64_t want) {
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ uint64_t bars[kBulkStages];
   __shared__ uint64_t dst_q[kBulkStages];
@@ -258,8 +258,8 @@ __global__ void __launch_bounds__(32) k_gather_host_bulk(PoolView v, PlanView pl
           const uint32_t o = g + lane;
           uint64_t pte = 0, off;
           if (o < npages) pte = translate(v, span_page_gva(v, sid, o), &off);
-          const bool host = (pte & kPteValid) && (pte & kPteHost);
-          const uint32_t mask = __ballot_sync(0xFFFFFFFFu, host);
+          const bool mine = (pte & kPteValid) && (pte & want);  // want: kPteHost, or kPteRemote (a peer GPU's HBM)
+          const uint32_t mask = __ballot_sync(0xFFFFFFFFu, mine);
           for (uint32_t m = mask; m; m &= m - 1) {
             const int l = __ffs(m) - 1;
             const uint64_t p_l = __shfl_sync(0xFFFFFFFFu, pte, l);
@@ -274,7 +274,7 @@ __global__ void __launch_bounds__(32) k_gather_host_bulk(PoolView v, PlanView pl
     }
   }
   ring.drain();
-  if (ring.lost && lane == 0) note_error(v, a.call_seq, FT_ERR_TIMEOUT, blockIdx.x);
+  if (ring.lost && lane == 0) note_error(v, a.call_seq, FT_ERR_TIMEOUT, (blockIdx.x & 0xFFFFu) | (min(ring.stranded, 0xFFFFu) << 16));
 }
 
 }  // namespace ft
@@ -340,28 +340,44 @@ int32_t gather_launch(ft_pool* p, const ft_plan* pl, uint32_t mb_begin, uint32_t
     }
   };
   const uint64_t per_sm = per_sm_cap;
-  // one launch when only one tier can be a source (own and imported bindings); otherwise one launch per tier
+  // one launch when only one kind of frame can be a source (own and imported bindings); otherwise one launch per
+  // kind: local HBM by vector streams from every SM, host-tier frames and frames in another GPU's HBM each by a
+  // few bulk-copy CTAs on a stream of their own (plain bulk copies, each CTA fetching its own bytes)
   const bool host_sources = p->cfg.host_pages != 0 || p->peer_host_frames;
+  const bool remote_sources = p->peer_remote_frames;
   const bool only_host = p->cfg.hbm_pages == 0 && !(p->cfg.world_size > 1);
-  if (!host_sources || only_host) {
+  if ((!host_sources && !remote_sources) || only_host) {
     prof_begin(p, only_host ? FT_K_GATHER_HOST : FT_K_GATHER_DEVICE, st);
     launch_mode(std::integral_constant<int, kTierAll>{}, a, per_sm);
     prof_end(p, st);
     p->gpu_launches += 1;
   } else {
-    FT_CUDA(cudaEventRecord(p->fork_ev[1], st));
-    FT_CUDA(cudaStreamWaitEvent(p->side_stream[1], p->fork_ev[1], 0));
     GatherArgs ah = a;
     ah.write_index = 0;
-    prof_begin(p, FT_K_GATHER_HOST, p->side_stream[1]);
-    k_gather_host_bulk<<<(unsigned)p->host_ctas, 32, kBulkSmemBytes, p->side_stream[1]>>>(p->view, pv, ah);
-    prof_end(p, p->side_stream[1]);
-    FT_CUDA(cudaEventRecord(p->join_ev[1], p->side_stream[1]));
+    if (host_sources) {
+      FT_CUDA(cudaEventRecord(p->fork_ev[1], st));
+      FT_CUDA(cudaStreamWaitEvent(p->side_stream[1], p->fork_ev[1], 0));
+      prof_begin(p, FT_K_GATHER_HOST, p->side_stream[1]);
+      k_gather_host_bulk<<<(unsigned)p->host_ctas, 32, kBulkSmemBytes, p->side_stream[1]>>>(p->view, pv, ah, kPteHost);
+      prof_end(p, p->side_stream[1]);
+      FT_CUDA(cudaEventRecord(p->join_ev[1], p->side_stream[1]));
+      p->gpu_launches += 1;
+    }
+    if (remote_sources) {
+      FT_CUDA(cudaEventRecord(p->fork_ev[2], st));
+      FT_CUDA(cudaStreamWaitEvent(p->side_stream[2], p->fork_ev[2], 0));
+      prof_begin(p, FT_K_GATHER_REMOTE, p->side_stream[2]);
+      k_gather_host_bulk<<<(unsigned)p->remote_ctas, 32, kBulkSmemBytes, p->side_stream[2]>>>(p->view, pv, ah, kPteRemote);
+      prof_end(p, p->side_stream[2]);
+      FT_CUDA(cudaEventRecord(p->join_ev[2], p->side_stream[2]));
+      p->gpu_launches += 1;
+    }
     prof_begin(p, FT_K_GATHER_DEVICE, st);
     launch_mode(std::integral_constant<int, kTierDeviceOnly>{}, a, per_sm);
     prof_end(p, st);
-    FT_CUDA(cudaStreamWaitEvent(st, p->join_ev[1], 0));
-    p->gpu_launches += 2;
+    if (host_sources) FT_CUDA(cudaStreamWaitEvent(st, p->join_ev[1], 0));
+    if (remote_sources) FT_CUDA(cudaStreamWaitEvent(st, p->join_ev[2], 0));
+    p->gpu_launches += 1;
   }
   FT_CUDA(cudaGetLastError());
   p->bytes_gathered += n_rows * 2ull * p->view.row_bytes;

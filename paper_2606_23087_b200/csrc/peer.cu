@@ -222,7 +222,14 @@ FT_API int32_t pool_import_mapping(ft_pool* p, const void* buf, uint64_t bytes, 
   uint64_t* pte_hbm = d_pte;
   uint64_t* pte_host = d_pte + h.hbm_pages;
   uint64_t* pte_text = pte_host + h.host_pages;
-  if (h.hbm_pages) k_page_table_init<<<blocks(h.hbm_pages), 256>>>(pte_hbm, d_bind, h.hbm_pages, reinterpret_cast<uint64_t>(peer_hbm_base), h.page_bytes, kPteValid);
+  // where the peer's HBM slab lives: frames of another device are remote (read over NVLink by a launch of their own)
+  bool remote = p->peers_remote != 0;
+  if (h.hbm_pages && !remote) {
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, peer_hbm_base) == cudaSuccess && at.type == cudaMemoryTypeDevice && at.device != p->device) remote = true;
+    cudaGetLastError();
+  }
+  if (h.hbm_pages) k_page_table_init<<<blocks(h.hbm_pages), 256>>>(pte_hbm, d_bind, h.hbm_pages, reinterpret_cast<uint64_t>(peer_hbm_base), h.page_bytes, kPteValid | (remote ? kPteRemote : 0));
   if (h.host_pages) k_page_table_init<<<blocks(h.host_pages), 256>>>(pte_host, d_bind + h.hbm_pages, h.host_pages, reinterpret_cast<uint64_t>(peer_host_base), h.page_bytes, kPteValid | kPteHost);
   if (h.text_pages) k_page_table_init<<<blocks(h.text_pages), 256>>>(pte_text, nullptr, h.text_pages, reinterpret_cast<uint64_t>(peer_text_base), FT_TEXT_PAGE_BYTES, kPteValid | kPteText);
   p->gpu_launches += 3;
@@ -235,6 +242,7 @@ FT_API int32_t pool_import_mapping(ft_pool* p, const void* buf, uint64_t bytes, 
   p->peer_allocs.push_back(d_pte);
   p->peer_imported[h.rank] = 1;
   if (h.host_pages) p->peer_host_frames = true;
+  if (h.hbm_pages && remote) p->peer_remote_frames = true;
   p->peer_bases[h.rank] = {reinterpret_cast<uint64_t>(peer_hbm_base), reinterpret_cast<uint64_t>(peer_host_base), reinterpret_cast<uint64_t>(peer_text_base)};
   return FT_OK;
 }

@@ -64,13 +64,19 @@ int32_t ctx_acquire(ft_pool* p, int side, size_t blob_bytes, size_t total_bytes,
     c.hcap = cap;
   }
   if (c.dcap < total_bytes) {
-    if (c.busy_done) { FT_CUDA(cudaEventSynchronize(c.ev_done)); c.busy_done = false; }  // nobody reads the old scratch
-    if (c.d) FT_CUDA(cudaFree(c.d));
+    // a call larger than any before it on this side: every context of the side grows now (allocating synchronises
+    // the device; once for all of them instead of once per context as the ring comes round)
     size_t cap = 1 << 18;
     while (cap < total_bytes) cap <<= 1;
-    c.d = nullptr; c.dcap = 0;
-    FT_CUDA(cudaMalloc(&c.d, cap));
-    c.dcap = cap;
+    for (int i = 0; i < kCallCtx; ++i) {
+      ft_call_ctx& g = p->ctx[side][i];
+      if (g.dcap >= cap) continue;
+      if (g.busy_done) { FT_CUDA(cudaEventSynchronize(g.ev_done)); g.busy_done = false; }  // nobody reads the old scratch
+      if (g.d) FT_CUDA(cudaFree(g.d));
+      g.d = nullptr; g.dcap = 0;
+      FT_CUDA(cudaMalloc(&g.d, cap));
+      g.dcap = cap;
+    }
   }
   if (c.busy_done) { FT_CUDA(cudaStreamWaitEvent(on_meta ? p->meta : first_user, c.ev_done, 0)); c.busy_done = false; }
   *out = &c;
@@ -438,7 +444,7 @@ __global__ void __launch_bounds__(32) k_scatter_host_bulk(PoolView v, WriteCall 
     }
   }
   ring.drain();
-  if (ring.lost && lane == 0) note_error(v, call_seq, FT_ERR_TIMEOUT, blockIdx.x);
+  if (ring.lost && lane == 0) note_error(v, call_seq, FT_ERR_TIMEOUT, (blockIdx.x & 0xFFFFu) | (min(ring.stranded, 0xFFFFu) << 16));
 }
 
 // The byte copy of a producer call, shared by pool_write_embeddings and its no-allocation variant: HBM-bound chunks on
@@ -622,7 +628,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_destroy(ft_pool* 
   if (p->d_text) cudaFree(p->d_text);
   if (p->own_hbm && p->hbm_base) cudaFree(p->hbm_base);
   if (p->own_host && p->host_base) cudaFreeHost(p->host_base);
-  for (int a = 0; a < 2; ++a) {
+  for (int a = 0; a < 3; ++a) {
     if (p->side_stream[a]) cudaStreamDestroy(p->side_stream[a]);
     if (p->fork_ev[a]) cudaEventDestroy(p->fork_ev[a]);
     if (p->join_ev[a]) cudaEventDestroy(p->join_ev[a]);
@@ -669,7 +675,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_create(const ft_p
   } while (0)
   CK(cudaGetDevice(&p->device));
   CK(cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, p->device));
-  for (int a = 0; a < 2; ++a) {
+  for (int a = 0; a < 3; ++a) {
     CK(cudaStreamCreateWithFlags(&p->side_stream[a], cudaStreamNonBlocking));
     CK(cudaEventCreateWithFlags(&p->fork_ev[a], cudaEventDisableTiming));
     CK(cudaEventCreateWithFlags(&p->join_ev[a], cudaEventDisableTiming));
@@ -1180,6 +1186,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_get_tuning(ft_poo
   out->host_ctas = (uint32_t)p->host_ctas; out->host_store_ctas = (uint32_t)p->host_store_ctas;
   out->gather_unroll = (uint32_t)p->gather_unroll;
   out->grad_ctas_per_sm = (uint32_t)p->grad_ctas_per_sm; out->grad_hot_threshold = (uint32_t)p->grad_hot_threshold;
+  out->remote_ctas = (uint32_t)p->remote_ctas; out->peers_remote = (uint32_t)p->peers_remote;
   return FT_OK;
 }
 
@@ -1189,7 +1196,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_set_tuning(ft_poo
   if (t.dev_ctas_per_sm > 8 || t.scatter_ctas_per_sm > 8 || t.grad_ctas_per_sm > 8) return FT_ERR_INVALID_ARG;
   if (t.chunk_shift && (t.chunk_shift < 14 || t.chunk_shift > 21)) return FT_ERR_INVALID_ARG;  // a warp's eighth holds a 2 KiB batch
   if (t.gather_unroll && t.gather_unroll != 4 && t.gather_unroll != 8) return FT_ERR_INVALID_ARG;
-  if (t.host_ctas > 1024 || t.host_store_ctas > 1024 || t.scatter_group > (1u << 20)) return FT_ERR_INVALID_ARG;
+  if (t.host_ctas > 1024 || t.host_store_ctas > 1024 || t.remote_ctas > 1024 || t.scatter_group > (1u << 20) || t.peers_remote > 1) return FT_ERR_INVALID_ARG;
   FT_CUDA(cudaDeviceSynchronize());  // no kernel of an earlier call is still being sized by the old values
   p->dev_ctas_per_sm = t.dev_ctas_per_sm ? (int)t.dev_ctas_per_sm : 4;
   p->scatter_ctas_per_sm = (int)t.scatter_ctas_per_sm;
@@ -1200,6 +1207,8 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_set_tuning(ft_poo
   p->gather_unroll = t.gather_unroll ? (int)t.gather_unroll : 4;
   p->grad_ctas_per_sm = t.grad_ctas_per_sm ? (int)t.grad_ctas_per_sm : 6;
   p->grad_hot_threshold = (int)t.grad_hot_threshold;
+  p->remote_ctas = t.remote_ctas ? (int)t.remote_ctas : 16;
+  p->peers_remote = (int)t.peers_remote;
   return FT_OK;
 }
 

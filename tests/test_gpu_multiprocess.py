@@ -13,12 +13,15 @@ from oracle import OraclePool, PlanConfig, PoolConfig
 pytestmark = pytest.mark.gpu
 
 
+@pytest.mark.parametrize("peers_remote", [0, 1])
 @pytest.mark.parametrize("name,kw", [
     ("image_mix_7b", dict(n_samples=10, hidden=56, page_bytes=4096)),
     ("image_mix_7b", dict(n_samples=12, hidden=3584)),                    # 2 MiB pages, both tiers on both sides
     ("host_tier_stress", dict(n_samples=4, hidden=1024, page_bytes=65536)),
 ])
-def test_consumer_reads_producer_pages_in_place(name, kw):
+def test_consumer_reads_producer_pages_in_place(name, kw, peers_remote):
+    """peers_remote = 1: the consumer treats the producer's HBM frames as another GPU's (they get the separate
+    bulk-copy launch that frames behind NVLink get), which must not change a byte."""
     if not torch.cuda.is_available():
         pytest.fail("a CUDA device is required for -m gpu tests")
     from gpu_harness import cuda_stream
@@ -36,6 +39,8 @@ def test_consumer_reads_producer_pages_in_place(name, kw):
     g = {r: fp.Pool(fp.PoolConfig(**cfg(r))) for r in (0, 1)}
     o = {r: OraclePool(PoolConfig(**cfg(r))) for r in (0, 1)}
     assert all(p.rc == 0 for p in g.values()) and all(p.rc == 0 for p in o.values())
+    assert g[0].set_tuning(peers_remote=peers_remote, remote_ctas=3) == 0 and g[0].get_tuning()["peers_remote"] == peers_remote
+    g[0].profile_enable(True)
     keep = []
 
     def fill(rank, samples):
@@ -107,6 +112,8 @@ def test_consumer_reads_producer_pages_in_place(name, kw):
     assert np.array_equal(got, oout) and not np.any(np.all(got == 0xFFFF, axis=1))
     assert np.array_equal(cu.cpu().numpy(), ocu) and np.array_equal(pos.cpu().numpy(), opos)
     assert g[0].status() == o[0].status() == (0, 0)
+    prof = g[0].profile_read()
+    assert (prof["gather_remote"]["launches"] > 0) == bool(peers_remote) and prof["gather_device"]["launches"] > 0
     # backbone-side outputs over the same mixed microbatches: the imported spans' token grids came with the descriptors
     L = w.budget_L
     rows = n_mb * L
