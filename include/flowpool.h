@@ -211,11 +211,14 @@ int32_t pool_write_embeddings(ft_pool* pool, uint32_t n_spans, const uint32_t* s
  *   - the device current at the call must be the pool's device, else FT_ERR_INVALID_ARG.
  * The first call on each device looks up the array's device address once (cudaGetSymbolAddress); make
  * that first call before any stream capture begins.  All calls, from every pool on the device, share
- * the one array: it still holds the previous call's descriptors when the next call starts, nothing in
- * it needs to start at zero (each call overwrites all it reads), and two calls whose kernels may overlap
- * on the GPU (different streams without an ordering between them) race on it -- keep no-alloc writes on
- * one stream, or order them with events.  The descriptors are copied from pageable host memory with
- * cudaMemcpyAsync, which returns only after the host data has been taken.
+ * the one array: it still holds the previous call's descriptors when the next call starts, and nothing in
+ * it needs to start at zero except the two claim counters of the copy kernels in its last 32 bytes, which
+ * the kernels themselves put back to zero when they finish.  A pool orders its own no-alloc writes (the
+ * next one waits, on the GPU, for the copy of the one before); calls of DIFFERENT pools whose kernels may
+ * overlap on the GPU race on the array -- give them one stream, or order them with events.
+ * Host side: the descriptors are assembled in a buffer pool_create made for this purpose (the call needs
+ * no more than a few hundred bytes of the caller's stack) and go up by cudaMemcpyAsync from that pageable
+ * buffer, which returns only after the host data has been taken: the call blocks the host for that copy.
  */
 #define FT_NOALLOC_MAX_SPANS 4096u
 #define FT_NOALLOC_SCRATCH_BYTES (256u + 32u * (FT_NOALLOC_MAX_SPANS + 8u))

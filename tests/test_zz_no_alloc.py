@@ -6,14 +6,16 @@ implicit synchronisation).  The no-alloc entry point keeps its per-call scratch 
 instead.  This test writes the same embeddings through both entry points into two pools of identical
 configuration, on two producer calls in a row (the second call finds the first call's descriptors still in
 the shared array), and requires identical page lists and bit-identical assembled output -- the same
-bit-exact bar as every other GPU test here.  The file name sorts last so that pytest collects it last.
+bit-exact bar as every other GPU test here -- and the same again against the CPU oracle.  A second case fills
+the fixed array to its limit: 4096 one-token spans in one call on an all-HBM pool with 4 KiB pages.  The file
+name sorts last so that pytest collects it last.
 """
 import numpy as np
 import pytest
 import torch
 
 import workloads
-from harness import plan_config_fields, pool_config_fields, register_args, write_args
+from harness import plan_config_fields, pool_config_fields, register_args, run_oracle, write_args
 
 pytestmark = pytest.mark.gpu
 
@@ -73,6 +75,42 @@ def test_noalloc_write_matches_regular_write(name, kw):
         assert np.array_equal(a, b)                  # bit-exact, as everywhere in this suite
     assert got[4] == ref[4] == (0, 0) and got[5] == ref[5]
     assert not np.any(np.all(got[1] == -1, axis=1))
+    _assert_equals_oracle(w, got)
+
+
+def _assert_equals_oracle(w, got):
+    """The same call sequence through the CPU oracle: page lists, rows, cu_seqlens, position ids."""
+    exp = run_oracle(w)
+    assert all(rc == 0 for rc in exp["rc"]) and exp["status"] == (0, 0)
+    for k, pages in exp["span_pages"].items():
+        assert np.array_equal(got[0][k], pages), k
+    assert np.array_equal(got[1].view(np.uint16), exp["out"])
+    assert np.array_equal(got[2], exp["cu_seqlens"]) and np.array_equal(got[3], exp["position_ids"])
+
+
+def test_noalloc_at_its_span_limit_on_an_all_hbm_pool():
+    """FT_NOALLOC_MAX_SPANS spans in ONE call: the fixed array is used up to its last descriptor slot, the copy
+    kernel finds each chunk's span by search (the array has no room for a per-chunk table), and with every page in
+    HBM the whole call is one launch.  1024 samples x 4 one-token spans, hidden 64, 4 KiB pages (one page per span)."""
+    if not torch.cuda.is_available():
+        pytest.fail("a CUDA device is required for -m gpu tests")
+    from paper_2606_23087_b200 import binding as fp
+    from workloads.gen import _assemble
+    n = fp.FT_NOALLOC_MAX_SPANS // 4
+    w = _assemble("span_limit", 7, 64, 4096, np.full(n, 8), [[1, 1, 1, 1]] * n, budget_L=4096)
+    w.hbm_pages, w.host_pages = 4 * n + 16, 0
+    order = list(range(n))
+    w.write_calls = [[(s, j) for s in order for j in range(4)]]
+    w.plan_order = order
+    assert len(w.write_calls[0]) == fp.FT_NOALLOC_MAX_SPANS
+    ref = _run(w, use_noalloc=False)
+    got = _run(w, use_noalloc=True)
+    for k in ref[0]:
+        assert np.array_equal(got[0][k], ref[0][k]), k
+    for a, b in zip(got[1:4], ref[1:4]):
+        assert np.array_equal(a, b)
+    assert got[4] == ref[4] == (0, 0) and got[5] == ref[5] == 16
+    _assert_equals_oracle(w, got)
 
 
 def test_noalloc_rejects_oversized_calls():
