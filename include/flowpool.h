@@ -22,8 +22,8 @@
  *    events, so that every call still sees the effects of every earlier call
  *    of the pool, and whatever the caller enqueues on `stream` after a call
  *    comes after that call.  The gain: the page allocation of producer call
- *    i+1 is worked out while the copy of call i is streaming (the producer
- *    "immediately proceeds", Sec. 3.1).
+ *    i+1 is worked out while the copy of call i is streaming (Sec. 3.1: a
+ *    producer goes on with its next batch at once).
  *  - Two streams per pool are supported: a producer side (register, write, import, free) and a consumer side
  *    (plan, export, gather) may be issued, from one host thread, on two different streams so that the encoder's
  *    scatter of the next batch overlaps the backbone's assembly of the current one (the decoupled
@@ -331,9 +331,8 @@ int32_t pool_status(ft_pool* pool, int32_t* first_device_error, uint64_t* detail
 int32_t pool_stats(ft_pool* pool, ft_pool_stats* out);
 
 /*
- * Ready queue (Sec. 3.1: "after sufficient paired embeddings accumulate in the pool, the scheduler ... constructs
- * microbatches").  Samples enter a FIFO in the order in which they became READY (last span written, text-only
- * registration, import).  pool_ready_count reports the live entries and their tokens.  pool_take_ready pops up
+ * Ready queue (Sec. 3.1: the scheduler forms microbatches once enough paired embeddings are in the pool).
+ * Samples enter a FIFO in the order in which they became READY (last span written, text-only registration, import).  pool_ready_count reports the live entries and their tokens.  pool_take_ready pops up
  * to max_samples slots in that order, but only once at least min_tokens tokens are ready (the watermark):
  * otherwise NOT_READY and nothing is taken.  Entries of samples freed in the meantime are skipped.  Host only.
  */
@@ -342,8 +341,8 @@ int32_t pool_take_ready(ft_pool* pool, uint64_t min_tokens, uint32_t max_samples
                         uint32_t* n_out, uint64_t* tokens_out);
 
 /*
- * More than one process in the GVA space (Sec. 3.2: "each process exports its memory mapping information to all
- * other processes, which update their page table accordingly"; afterwards address translation is local).
+ * More than one process in the GVA space (Sec. 3.2: every process sends its memory mapping to all the others, which
+ * enter it into their page tables; afterwards address translation is local).
  * Pools created with the same world_size, page_bytes, GVA starts and max_size and distinct ranks form one space.
  *
  * pool_backing        the addresses of this pool's slabs as THIS process sees them (device pointers; the host
@@ -358,7 +357,7 @@ int32_t pool_take_ready(ft_pool* pool, uint64_t min_tokens, uint32_t max_samples
  *                     small bulk-copy launch beside the one that streams local HBM.  INVALID_ARG: malformed blob, another GVA space, own rank, missing or misaligned
  *                     base; SLOT_IN_USE: that rank was imported before.  Init-time: allocates, synchronises.
  * pool_export_samples descriptors of READY samples (lengths, spans with their token grids, page GVAs, text-page GVAs) into a host buffer
- *                     -- the "lightweight metadata" a consumer needs; no embedding bytes.  Synchronises `stream`.
+ *                     -- the small metadata records a consumer needs; no embedding bytes.  Synchronises `stream`.
  *                     UNKNOWN_SAMPLE / NOT_READY / INVALID_ARG (repeated slot) per sample in order; buf = NULL
  *                     queries the size.
  * pool_import_samples registers the described samples in local FREE slots as READY, imported samples: their page

@@ -242,7 +242,7 @@ static uint8_t* resolve(oracle_pool* p, uint64_t g) {
   return pr->text_mem + frame * TEXT_PAGE_BYTES + off;
 }
 
-/* Sec. 3.1: the scheduler acts once "sufficient paired embeddings accumulate": a FIFO of samples in the order in
+/* Sec. 3.1: the scheduler acts once enough paired embeddings have accumulated: a FIFO of samples in the order in
  * which they became ready (reading: completion order; the watermark is a token count chosen by the caller). */
 static void ready_push(oracle_pool* p, uint32_t slot) {
   if (p->rq_tail == p->rq_cap) {
@@ -622,7 +622,7 @@ uint32_t oracle_bestfit_segment_tree(uint32_t n, const uint32_t* len, uint32_t L
 }
 
 /* Eq. 3 scaled to integers: A*sum(l) + B*lmax^2; with (A,B) = (L,1) this is
- * L^2 * Cost(B_j) exactly.  The quadratic term is lmax^2, as printed. */
+ * L^2 * Cost(B_j) exactly.  The quadratic term is lmax^2, the term Eq. 3 has. */
 uint64_t oracle_cost_int(uint64_t A, uint64_t B, uint64_t sum_len, uint64_t lmax) {
   return A * sum_len + B * lmax * lmax;
 }
@@ -643,12 +643,14 @@ void oracle_balance(uint32_t n_mb, const uint64_t* cost, uint32_t K, uint32_t N,
     unsigned __int128 num = (unsigned __int128)(cost[j] - lo) * K;
     bucket[j] = (uint32_t)(num / ((unsigned __int128)(hi - lo) + 1));
   }
-  /* lines 15-27: per bucket (reading: highest bucket first), sort by cost
-   * descending (reading: ties by microbatch index ascending), then deal
-   * Rank_0..Rank_{N-1}, reverse, and so on; a and Forward restart per bucket
-   * (as printed); reading: the deal stops when the list is exhausted.
-   * Variant `carry`: one continuous zig-zag over the buckets' lists in turn: the
-   * position inside the current round and the direction carry over. */
+  /* Algorithm 1 lines 15-27, the deal.  Readings: buckets are taken from the highest to the lowest; inside a
+   * bucket the microbatches are ordered by cost, descending, equal costs by index, ascending; the deal of a bucket
+   * ends with its list.  Dealing N at a time over Rank_0..Rank_{N-1} and back means that the i-th microbatch of a
+   * bucket's ordered list sits at place i mod N of round i div N, and that odd rounds run from the last rank
+   * down: rank = i mod N in even rounds, N-1 - (i mod N) in odd rounds; every bucket starts again at round 0 (the
+   * algorithm sets its position and direction inside the loop over buckets).
+   * Variant `carry`: one continuous zig-zag over the buckets' lists in turn: the position inside the current round
+   * and the direction carry over from bucket to bucket. */
   uint32_t* list = (uint32_t*)calloc((size_t)n_mb + 1, sizeof(uint32_t));
   uint32_t* order = (uint32_t*)calloc((size_t)n_mb + 1, sizeof(uint32_t)); /* global dispatch order */
   uint32_t n_order = 0;
@@ -670,11 +672,10 @@ void oracle_balance(uint32_t n_mb, const uint64_t* cost, uint32_t K, uint32_t N,
       }
       continue;
     }
-    uint32_t a = 0; int forward = 1;
-    while (a < m) {
-      if (forward) { for (uint32_t r = 0; r < N && a < m; ++r) { rank[list[a]] = r; order[n_order++] = list[a]; ++a; } }
-      else { for (int64_t r = (int64_t)N - 1; r >= 0 && a < m; --r) { rank[list[a]] = (uint32_t)r; order[n_order++] = list[a]; ++a; } }
-      forward = !forward;
+    for (uint32_t i = 0; i < m; ++i) {
+      const uint32_t round = i / N, place = i % N;
+      rank[list[i]] = (round & 1u) ? N - 1 - place : place;
+      order[n_order++] = list[i];
     }
   }
   /* per-rank lists, in the order the microbatches were dealt */
