@@ -483,14 +483,24 @@ int32_t pool_profile_read(ft_pool* pool, ft_kernel_time* out /* host [FT_K_COUNT
  *   remote_ctas          grid of the bulk-copy gather that reads frames in ANOTHER GPU's HBM (default 16): like the
  *                        host tier, peer frames are long-latency sources and get a small grid of their own, so that the
  *                        SMs that stream local HBM keep their memory pipelines; to be tuned where a second GPU exists
+ *   scatter_smem_carveout  shared-memory share, in percent of an SM's unified L1/shared storage, that the scatter
+ *                        kernel asks for although it uses next to none (default 5; 1..100; a function attribute, so
+ *                        it holds for the device, not only for this pool).  An SM keeps one split while any CTA is
+ *                        resident.  With the driver's own choice for this kernel the metadata kernels and the packing
+ *                        kernel did not start beside it and ran when the copies had ended; with 3 to 9 percent they
+ *                        run beside it and the copy streams as fast as before; from 10 percent on the copy loses a
+ *                        sixth of its bandwidth (measured on a B200)
+ *   gather_smem_carveout   the same preference for the gather kernel (default 0 = the driver's choice: this kernel
+ *                        keeps 6 KiB of row descriptors per CTA in shared memory, and a preference below what four
+ *                        CTAs need costs it occupancy and 6 percent of its bandwidth)
  *   peers_remote         1: pool_import_mapping flags every peer's HBM frames as remote even when they are on this
  *                        device (exercises the remote path on one GPU); 0: only frames of another device are remote
  */
 typedef struct {
   uint32_t dev_ctas_per_sm, scatter_ctas_per_sm, scatter_group, chunk_shift;
   uint32_t host_ctas, host_store_ctas, gather_unroll, grad_ctas_per_sm, grad_hot_threshold;
-  uint32_t remote_ctas, peers_remote;
-  uint32_t reserved[5];
+  uint32_t remote_ctas, peers_remote, scatter_smem_carveout, gather_smem_carveout;
+  uint32_t reserved[3];
 } ft_tuning;
 int32_t pool_get_tuning(ft_pool* pool, ft_tuning* out);
 int32_t pool_set_tuning(ft_pool* pool, const ft_tuning* in);

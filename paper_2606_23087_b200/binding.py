@@ -66,11 +66,11 @@ class PoolStats(C.Structure):
 
 
 TUNING_FIELDS = ("dev_ctas_per_sm", "scatter_ctas_per_sm", "scatter_group", "chunk_shift", "host_ctas", "host_store_ctas",
-                 "gather_unroll", "grad_ctas_per_sm", "grad_hot_threshold", "remote_ctas", "peers_remote")
+                 "gather_unroll", "grad_ctas_per_sm", "grad_hot_threshold", "remote_ctas", "peers_remote", "scatter_smem_carveout", "gather_smem_carveout")
 
 
 class Tuning(C.Structure):
-    _fields_ = [(k, C.c_uint32) for k in TUNING_FIELDS] + [("reserved", C.c_uint32 * 5)]
+    _fields_ = [(k, C.c_uint32) for k in TUNING_FIELDS] + [("reserved", C.c_uint32 * 3)]
 
 
 class KernelTime(C.Structure):

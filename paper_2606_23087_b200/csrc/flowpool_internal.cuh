@@ -331,6 +331,8 @@ struct ft_pool {
                                 // accesses do not clog the memory pipelines of the SMs that stream HBM; 6 rather
                                 // than 8 because a write and a read kernel running together (two streams) share
                                 // the link better with fewer requests in flight
+  int scatter_smem_carveout = 5;  // percent of an SM's L1/shared storage the scatter kernel asks for as shared memory
+  int gather_smem_carveout = 0;   // the same for the gather kernel (0 = the driver's choice)
   int remote_ctas = 16;         // grid of the bulk-copy gather from another GPU's HBM (about 128 KiB in flight per CTA;
                                 // 770 GB/s x a few microseconds of NVLink latency wants 1.5 MB and more in flight)
   int peers_remote = 0;         // 1: flag every imported peer's HBM frames as remote, whatever device they are on
@@ -353,6 +355,9 @@ namespace ft {
 // per-device set-up of each translation unit's kernels (shared-memory opt-ins, occupancy), run by pool_create
 // with the pool's device current
 int32_t gather_device_setup(ft_pool* p);
+// shared-memory carve-out preference (percent) of the copy kernels of each translation unit
+int32_t gather_set_carveout(int pct);
+int32_t scatter_set_carveout(int pct);
 int32_t plan_device_setup(ft_pool* p);
 // (d_list: device array of the list layout's entries, or nullptr for the range [mb_begin, mb_end))
 int32_t gather_launch(ft_pool* p, const ft_plan* pl, uint32_t mb_begin, uint32_t mb_end, const void* embed_table,

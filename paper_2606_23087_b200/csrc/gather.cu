@@ -280,6 +280,17 @@ __global__ void __launch_bounds__(32) k_gather_host_bulk(PoolView v, PlanView pl
 }  // namespace ft
 
 namespace ft {
+int32_t gather_set_carveout(int pct) {
+  FT_CUDA(cudaFuncSetAttribute(k_gather<kTierAll, 4, false>, cudaFuncAttributePreferredSharedMemoryCarveout, pct));
+  FT_CUDA(cudaFuncSetAttribute(k_gather<kTierAll, 4, true>, cudaFuncAttributePreferredSharedMemoryCarveout, pct));
+  FT_CUDA(cudaFuncSetAttribute(k_gather<kTierAll, 8, false>, cudaFuncAttributePreferredSharedMemoryCarveout, pct));
+  FT_CUDA(cudaFuncSetAttribute(k_gather<kTierAll, 8, true>, cudaFuncAttributePreferredSharedMemoryCarveout, pct));
+  FT_CUDA(cudaFuncSetAttribute(k_gather<kTierDeviceOnly, 4, false>, cudaFuncAttributePreferredSharedMemoryCarveout, pct));
+  FT_CUDA(cudaFuncSetAttribute(k_gather<kTierDeviceOnly, 4, true>, cudaFuncAttributePreferredSharedMemoryCarveout, pct));
+  FT_CUDA(cudaFuncSetAttribute(k_gather<kTierDeviceOnly, 8, false>, cudaFuncAttributePreferredSharedMemoryCarveout, pct));
+  FT_CUDA(cudaFuncSetAttribute(k_gather<kTierDeviceOnly, 8, true>, cudaFuncAttributePreferredSharedMemoryCarveout, pct));
+  return FT_OK;
+}
 int32_t gather_device_setup(ft_pool* p) {
   FT_CUDA(cudaFuncSetAttribute(k_gather_host_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBulkSmemBytes));
   auto occ = [](auto kernel) { int v = 0; return cudaOccupancyMaxActiveBlocksPerMultiprocessor(&v, kernel, kGatherThreads, 0) == cudaSuccess && v > 0 ? v : 1; };

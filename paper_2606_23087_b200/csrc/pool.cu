@@ -447,6 +447,16 @@ __global__ void __launch_bounds__(32) k_scatter_host_bulk(PoolView v, WriteCall 
   if (ring.lost && lane == 0) note_error(v, call_seq, FT_ERR_TIMEOUT, (blockIdx.x & 0xFFFFu) | (min(ring.stranded, 0xFFFFu) << 16));
 }
 
+int32_t scatter_set_carveout(int pct) {
+  FT_CUDA(cudaFuncSetAttribute(k_scatter<kTierAll, false>, cudaFuncAttributePreferredSharedMemoryCarveout, pct));
+  FT_CUDA(cudaFuncSetAttribute(k_scatter<kTierAll, true>, cudaFuncAttributePreferredSharedMemoryCarveout, pct));
+  FT_CUDA(cudaFuncSetAttribute(k_scatter<kTierDeviceOnly, false>, cudaFuncAttributePreferredSharedMemoryCarveout, pct));
+  FT_CUDA(cudaFuncSetAttribute(k_scatter<kTierDeviceOnly, true>, cudaFuncAttributePreferredSharedMemoryCarveout, pct));
+  FT_CUDA(cudaFuncSetAttribute(k_scatter<kTierHostOnly, false>, cudaFuncAttributePreferredSharedMemoryCarveout, pct));
+  FT_CUDA(cudaFuncSetAttribute(k_scatter<kTierHostOnly, true>, cudaFuncAttributePreferredSharedMemoryCarveout, pct));
+  return FT_OK;
+}
+
 // The byte copy of a producer call, shared by pool_write_embeddings and its no-allocation variant: HBM-bound chunks on
 // the caller's stream, host-bound chunks beside them on the producer side's second stream.
 static int32_t launch_write_copies(ft_pool* p, const WriteCall& w, uint64_t total_chunks, bool f32, cudaStream_t st, ClaimCounter* cc,
@@ -706,6 +716,9 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_create(const ft_p
     p->occ_scatter[kTierDeviceOnly][0] = occ(k_scatter<kTierDeviceOnly, false>); p->occ_scatter[kTierDeviceOnly][1] = occ(k_scatter<kTierDeviceOnly, true>);
     p->occ_scatter[kTierHostOnly][0] = occ(k_scatter<kTierHostOnly, false>); p->occ_scatter[kTierHostOnly][1] = occ(k_scatter<kTierHostOnly, true>);
   }
+  // the scatter kernel's shared-memory split (see ft_tuning.scatter_smem_carveout): small but stated, so that metadata
+  // kernels and the packing kernel can start on SMs that hold its CTAs
+  if ((rc = scatter_set_carveout(p->scatter_smem_carveout)) != FT_OK) { pool_destroy(p); return rc; }
   if ((rc = gather_device_setup(p)) != FT_OK || (rc = plan_device_setup(p)) != FT_OK) { pool_destroy(p); return rc; }
 
   const uint64_t P = c.hbm_pages + c.host_pages;
@@ -1187,6 +1200,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_get_tuning(ft_poo
   out->gather_unroll = (uint32_t)p->gather_unroll;
   out->grad_ctas_per_sm = (uint32_t)p->grad_ctas_per_sm; out->grad_hot_threshold = (uint32_t)p->grad_hot_threshold;
   out->remote_ctas = (uint32_t)p->remote_ctas; out->peers_remote = (uint32_t)p->peers_remote;
+  out->scatter_smem_carveout = (uint32_t)p->scatter_smem_carveout; out->gather_smem_carveout = (uint32_t)p->gather_smem_carveout;
   return FT_OK;
 }
 
@@ -1196,7 +1210,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_set_tuning(ft_poo
   if (t.dev_ctas_per_sm > 8 || t.scatter_ctas_per_sm > 8 || t.grad_ctas_per_sm > 8) return FT_ERR_INVALID_ARG;
   if (t.chunk_shift && (t.chunk_shift < 14 || t.chunk_shift > 21)) return FT_ERR_INVALID_ARG;  // a warp's eighth holds a 2 KiB batch
   if (t.gather_unroll && t.gather_unroll != 4 && t.gather_unroll != 8) return FT_ERR_INVALID_ARG;
-  if (t.host_ctas > 1024 || t.host_store_ctas > 1024 || t.remote_ctas > 1024 || t.scatter_group > (1u << 20) || t.peers_remote > 1) return FT_ERR_INVALID_ARG;
+  if (t.host_ctas > 1024 || t.host_store_ctas > 1024 || t.remote_ctas > 1024 || t.scatter_group > (1u << 20) || t.peers_remote > 1 || t.scatter_smem_carveout > 100 || t.gather_smem_carveout > 100) return FT_ERR_INVALID_ARG;
   FT_CUDA(cudaDeviceSynchronize());  // no kernel of an earlier call is still being sized by the old values
   p->dev_ctas_per_sm = t.dev_ctas_per_sm ? (int)t.dev_ctas_per_sm : 4;
   p->scatter_ctas_per_sm = (int)t.scatter_ctas_per_sm;
@@ -1209,6 +1223,19 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_set_tuning(ft_poo
   p->grad_hot_threshold = (int)t.grad_hot_threshold;
   p->remote_ctas = t.remote_ctas ? (int)t.remote_ctas : 16;
   p->peers_remote = (int)t.peers_remote;
+  {
+    const int pct = t.scatter_smem_carveout ? (int)t.scatter_smem_carveout : 5;
+    if (pct != p->scatter_smem_carveout) {
+      const int32_t rc = scatter_set_carveout(pct);
+      if (rc != FT_OK) return rc;
+      p->scatter_smem_carveout = pct;
+    }
+    if ((int)t.gather_smem_carveout != p->gather_smem_carveout) {
+      const int32_t rc = gather_set_carveout(t.gather_smem_carveout ? (int)t.gather_smem_carveout : (int)cudaSharedmemCarveoutDefault);
+      if (rc != FT_OK) return rc;
+      p->gather_smem_carveout = (int)t.gather_smem_carveout;
+    }
+  }
   return FT_OK;
 }
 
