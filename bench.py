@@ -1109,22 +1109,27 @@ def run_streaming(args, all_hbm, batches=6, warm=2):
             rc = pool.write_embeddings(wr[0] + off, wr[1], wr[2], ptrs, w.src_dtype, prod.cuda_stream)
             assert rc == 0, rc
 
-    def assemble(k):
+    def make_plan():
         rc, slots, _ = pool.take_ready(w.total_tokens, n)      # watermark: one whole batch is ready
         assert rc == 0 and len(slots) == n, (rc, len(slots))
         rc, plan = pool.plan_microbatches(slots, pcfg, cons.cuda_stream)
         assert rc == 0, rc
+        return slots, plan
+
+    def assemble(k, plan):
         n_mb = plan.summary()[0]
         rc = pool.gather_packed(plan, 0, n_mb, table.data_ptr(), w.vocab, outs[k % 2].data_ptr(), cu.data_ptr(), pos.data_ptr(),
                                 cons.cuda_stream)
         assert rc == 0, rc
-        return slots, plan
 
-    # Issue order per round: assemble batch k (consumer stream), then write batch k+1 (producer stream), then free
-    # batch k (producer stream; the library makes it wait for the gather).  The consumer waits only for producer
-    # calls issued before it, so the write of k+1 and the assembly of k run side by side.
+    # Issue order per round: assemble batch k (consumer stream); write batch k+1 (producer stream); plan batch k+1 as
+    # soon as its write calls are queued (the plan needs the metadata only, which the metadata stream has ready long
+    # before the copies end); free batch k (the library makes it wait for the assembly).  The consumer waits only for
+    # producer calls issued before it, so the write of k+1 and the assembly of k run side by side, and no round
+    # starts by waiting for a plan.
     torch.cuda.synchronize()
     produce(0)
+    slots, plan = make_plan()
     t0 = None
     total = warm + batches
     for k in range(total):
@@ -1133,19 +1138,20 @@ def run_streaming(args, all_hbm, batches=6, warm=2):
             pool.profile_read()
             pool.profile_enable(True)
             t0 = time.perf_counter()
-        slots, plan = assemble(k)
+        assemble(k, plan)
         produce(k + 1)
+        next_slots, next_plan = make_plan()
         assert pool.free(slots, prod.cuda_stream) == 0
         plan.destroy()
+        slots, plan = next_slots, next_plan
     torch.cuda.synchronize()
     ms = (time.perf_counter() - t0) * 1e3 / batches
     prof = pool.profile_read()
     pool.profile_enable(False)
     kernel_ms = {k: v["ms"] / batches for k, v in prof.items() if v["launches"]}
-    # drain the batch that was produced but never consumed
-    rc, slots, _ = pool.take_ready(1, n)
-    if rc == 0 and len(slots):
-        pool.free(slots, prod.cuda_stream)
+    # drain the batch that was produced and planned but never consumed
+    plan.destroy()
+    pool.free(slots, prod.cuda_stream)
     assert pool.status() == (0, 0)
     wb, gb = algorithmic_bytes(w)
     pool.destroy()
