@@ -348,10 +348,14 @@ def apply_tuning(pool, args):
 
 
 def measure_host_link(torch, nbytes=1 << 30, reps=5):
-    """Host-link reference rates: plain cudaMemcpyAsync between pinned host memory and the device, best of reps."""
+    """Host-link reference rates: plain cudaMemcpyAsync between pinned host memory and the device, best of reps, one
+    direction at a time, and one copy each way at the same time on two streams (what the copy engines get when the
+    link is used in both directions at once)."""
     try:
         h = torch.empty(nbytes, dtype=torch.uint8, pin_memory=True)
         d = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+        h2 = torch.empty(nbytes, dtype=torch.uint8, pin_memory=True)
+        d2 = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
     except RuntimeError:
         return None
     res = {}
@@ -365,6 +369,20 @@ def measure_host_link(torch, nbytes=1 << 30, reps=5):
             torch.cuda.synchronize()
             best = max(best, nbytes / e0.elapsed_time(e1) / 1e6)
         res[name] = best
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    best = None
+    for _ in range(reps):
+        torch.cuda.synchronize()
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+        with torch.cuda.stream(s1):
+            ev[0].record(); d.copy_(h, non_blocking=True); ev[1].record()
+        with torch.cuda.stream(s2):
+            ev[2].record(); h2.copy_(d2, non_blocking=True); ev[3].record()
+        torch.cuda.synchronize()
+        a, b = nbytes / ev[0].elapsed_time(ev[1]) / 1e6, nbytes / ev[2].elapsed_time(ev[3]) / 1e6
+        if best is None or a + b > best[0] + best[1]:
+            best = (a, b)
+    res["both_ways_h2d_gbs"], res["both_ways_d2h_gbs"] = best
     return res
 
 

@@ -23,7 +23,7 @@ def host_bits(t):
 class CudaRun:
     """register -> write -> plan -> gather over a workload, keeping device buffers alive."""
 
-    def __init__(self, w, caller_owned_memory=False, max_samples=None):
+    def __init__(self, w, caller_owned_memory=False, max_samples=None, tuning=None):
         self.w = w
         self.keep = []
         f = pool_config_fields(w, max_samples=max_samples)
@@ -34,6 +34,8 @@ class CudaRun:
                 hbm_ptr = (self.hbm.data_ptr() + 255) // 256 * 256
         self.pool = fp.Pool(fp.PoolConfig(**f), hbm_base=hbm_ptr, host_base=host_ptr)
         assert self.pool.rc == 0, fp.STATUS.get(self.pool.rc)
+        if tuning:
+            assert self.pool.set_tuning(**tuning) == 0
         self.rc = []
         self.srcs = {}
 
@@ -95,8 +97,8 @@ class CudaRun:
         self.pool.destroy()
 
 
-def run_cuda(w, caller_owned_memory=False):
-    r = CudaRun(w, caller_owned_memory)
+def run_cuda(w, caller_owned_memory=False, tuning=None):
+    r = CudaRun(w, caller_owned_memory, tuning=tuning)
     r.run_schedule()
     rc, plan = r.plan()
     assert rc == 0, fp.STATUS.get(rc)

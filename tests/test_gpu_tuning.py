@@ -1,0 +1,83 @@
+"""The launch-geometry knobs (pool_set_tuning) change how the copy kernels are launched, never what they compute:
+the same two-tier workloads, written and assembled under unusual settings, must equal the oracle bit for bit."""
+import json
+import os
+import subprocess
+import sys
+
+import numpy as np
+import pytest
+import torch
+
+import workloads
+from test_gpu_parity import assert_same, oracle_from_device_sources
+
+pytestmark = pytest.mark.gpu
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+TUNINGS = [
+    dict(dev_ctas_per_sm=1, scatter_ctas_per_sm=1, gather_unroll=8),
+    dict(dev_ctas_per_sm=8, scatter_ctas_per_sm=8, scatter_group=5, chunk_shift=14),
+    dict(chunk_shift=21, host_ctas=1, host_store_ctas=1, scatter_smem_carveout=30, gather_smem_carveout=30),
+    dict(host_ctas=13, host_store_ctas=17, scatter_group=2, chunk_shift=18),
+]
+
+
+@pytest.mark.parametrize("tuning", TUNINGS)
+@pytest.mark.parametrize("name,kw", [
+    ("image_mix_7b", dict(n_samples=10, hidden=512, page_bytes=65536)),      # both tiers, rows straddle pages
+    ("host_tier_stress", dict(n_samples=4, hidden=1024, page_bytes=16384)),  # fp32 source, tiers interleaved
+])
+def test_results_do_not_depend_on_the_launch_geometry(name, kw, tuning):
+    if not torch.cuda.is_available():
+        pytest.fail("a CUDA device is required for -m gpu tests")
+    from gpu_harness import run_cuda
+    w = workloads.make_workload(name, **kw)
+    got = run_cuda(w, tuning=tuning)
+    exp = oracle_from_device_sources(w, got["srcs"], got["table"])
+    assert_same(got, exp)
+    assert not np.any(np.all(got["out"] == 0xFFFF, axis=1))
+
+
+def test_tuning_round_trip_and_range_checks():
+    if not torch.cuda.is_available():
+        pytest.fail("a CUDA device is required for -m gpu tests")
+    from harness import pool_config_fields
+    from paper_2606_23087_b200 import binding as fp
+    w = workloads.make_workload("tiny")
+    pool = fp.Pool(fp.PoolConfig(**pool_config_fields(w)))
+    assert pool.rc == 0
+    d = pool.get_tuning()
+    assert (d["dev_ctas_per_sm"], d["scatter_ctas_per_sm"], d["chunk_shift"], d["host_ctas"], d["gather_unroll"]) == (4, 4, 16, 6, 4)
+    assert d["scatter_smem_carveout"] == 5 and d["gather_smem_carveout"] == 0 and d["remote_ctas"] == 16
+    for bad in (dict(chunk_shift=13), dict(chunk_shift=22), dict(gather_unroll=6), dict(dev_ctas_per_sm=9), dict(peers_remote=2),
+                dict(scatter_smem_carveout=101)):
+        assert pool.set_tuning(**bad) == -1 and pool.get_tuning() == d          # INVALID_ARG, nothing changed
+    assert pool.set_tuning(host_ctas=3, chunk_shift=17) == 0
+    t = pool.get_tuning()
+    assert t["host_ctas"] == 3 and t["chunk_shift"] == 17 and t["dev_ctas_per_sm"] == 4   # unnamed knobs go back to their defaults
+    assert pool.set_tuning() == 0 and pool.get_tuning() == d
+    pool.destroy()
+
+
+def test_bench_gpus_2_runs_the_exchange_flow_with_two_ranks_on_this_gpu():
+    """`bench.py --gpus 2` launches two ranks by itself; with the gloo backend both may share this GPU (their kernels
+    never wait on one another: the ranks meet only in host-side collectives).  One line, from rank 0, with the
+    independent-batches value and the exchange flow (every rank writes, all plan alike, each assembles its share from
+    everybody's pages) beside it."""
+    if not torch.cuda.is_available():
+        pytest.fail("a CUDA device is required for -m gpu tests")
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    env["FLOWPOOL_BENCH_BACKEND"] = "gloo"
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--samples", "48", "--steps", "1", "--warmup", "3",
+                          "--skip-e2e", "--skip-cpu"], capture_output=True, text=True, timeout=900, cwd=ROOT, env=env)
+    assert out.returncode == 0, out.stderr[-3000:]
+    lines = [json.loads(l) for l in out.stdout.strip().splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    line = lines[0]
+    assert line["n_gpus"] == 2 and line["value"] > 0 and line["scaling"] == "weak"
+    ex = line["exchange"]
+    assert ex["config"]["ranks"] == 2 and len(ex["per_rank"]) == 2 and ex["value"] > 0
+    assert sum(r["rows"] for r in ex["per_rank"]) == ex["config"]["packed_tokens_all_ranks"]
+    assert all(r["bytes_from_peers"] > 0 and r["gather_gbs"] > 0 for r in ex["per_rank"])
+    assert ex["bytes_over_nvlink_per_step"] == 0            # both ranks on one GPU here
