@@ -81,3 +81,55 @@ def test_bench_gpus_2_runs_the_exchange_flow_with_two_ranks_on_this_gpu():
     assert sum(r["rows"] for r in ex["per_rank"]) == ex["config"]["packed_tokens_all_ranks"]
     assert all(r["bytes_from_peers"] > 0 and r["gather_gbs"] > 0 for r in ex["per_rank"])
     assert ex["bytes_over_nvlink_per_step"] == 0            # both ranks on one GPU here
+
+
+def test_a_call_larger_than_the_preallocated_contexts_grows_them():
+    """20 000 one-token spans in ONE register call and ONE write call: their descriptors (320 KB) exceed both the
+    pinned staging (64 KiB) and the device scratch (256 KiB) every call context starts with, so the contexts grow in
+    the middle of the run; page lists and every assembled byte must still equal the oracle's."""
+    if not torch.cuda.is_available():
+        pytest.fail("a CUDA device is required for -m gpu tests")
+    from gpu_harness import run_cuda
+    from workloads.gen import _assemble
+    n = 5000
+    w = _assemble("many_spans", 9, 64, 4096, np.full(n, 6), [[1, 1, 1, 1]] * n, budget_L=2048)
+    w.hbm_pages, w.host_pages = 3 * n, n + 32          # both tiers
+    order = list(range(n))
+    w.write_calls = [[(s, j) for s in order for j in range(4)]]
+    w.plan_order = order
+    got = run_cuda(w)
+    exp = oracle_from_device_sources(w, got["srcs"], got["table"])
+    assert_same(got, exp)
+    assert not np.any(np.all(got["out"] == 0xFFFF, axis=1))
+
+
+def test_a_plan_may_outlive_its_pool_and_plans_may_pile_up():
+    """Plan blocks come from a per-pool cache: a dozen plans alive at once, destroyed in another order, and one
+    destroyed after its pool is gone."""
+    if not torch.cuda.is_available():
+        pytest.fail("a CUDA device is required for -m gpu tests")
+    from gpu_harness import CudaRun
+    w = workloads.make_workload("tiny")
+    run = CudaRun(w)
+    run.run_schedule()
+    plans = []
+    for _ in range(12):
+        rc, plan = run.plan()
+        assert rc == 0
+        plans.append(plan)
+    ref = plans[0].arrays()
+    for p in plans[1:]:
+        a = p.arrays()
+        assert all(np.array_equal(a[k], ref[k]) for k in ref)
+    for p in plans[3:] + plans[1:3]:
+        p.destroy()
+    rc, plan = run.plan()                     # takes a cached block
+    assert rc == 0
+    rc, out, cu, pos = run.gather_all()
+    assert rc == 0 and run.pool.status() == (0, 0)
+    plan.destroy()
+    run.plan_handle = None
+    last = plans[0]
+    torch.cuda.synchronize()
+    run.pool.destroy()
+    last.destroy()                            # its pool no longer exists: the block is freed directly
