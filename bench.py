@@ -1004,7 +1004,7 @@ def sweep_measure(args, PS, with_variants=True):
     n_mb, total_tokens, _ = plan.summary()
     # scheduler variants on the same residents: what each buys in padding waste and rank balance
     variants = {}
-    for name, fl, k_limit in ((("as_printed", 0, 0), ("longest_first", 2, 0), ("sum_of_squares", 4, 0), ("carried_zigzag", 8, 0),
+    for name, fl, k_limit in ((("default", 0, 0), ("longest_first", 2, 0), ("sum_of_squares", 4, 0), ("carried_zigzag", 8, 0),
                                ("all_three", 14, 0), ("auto_k_limit_64", 16, 64), ("fixed_k_64", 0, 64)) if with_variants else ()):
         vc = plan_config_fields(w, flags=fl)
         if k_limit:
