@@ -295,8 +295,7 @@ struct ft_pool {
   cudaEvent_t ev_noalloc = nullptr;   // behind the last reader of the fixed no-allocation scratch
   bool have_noalloc_ev = false;
   uint64_t meta_seq = 0;              // metadata batches enqueued so far
-  cudaStream_t synced_stream[2] = {nullptr, nullptr};  // the caller streams that waited for `meta` last ...
-  uint64_t synced_seq[2] = {~0ull, ~0ull};             // ... and the batch count they waited for
+  uint64_t ev_meta_seq = ~0ull;       // the batch count `ev_meta` was last recorded behind
   uint64_t status_base = 0;           // call_seq at the last pool_status read
   std::vector<uint8_t> noalloc_blob;  // host staging of pool_write_embeddings_noalloc, made at pool_create
   // Device blocks of destroyed plans, kept for the next plan: each with an event behind the last kernel that read it.
@@ -320,7 +319,6 @@ struct ft_pool {
   cudaEvent_t fork_ev[3] = {nullptr, nullptr, nullptr}, join_ev[3] = {nullptr, nullptr, nullptr};
   // cross-stream ordering when the producer side and the consumer side are driven from different streams
   cudaEvent_t ev_producer = nullptr, ev_consumer = nullptr;  // end of the latest producer-side / consumer-side call
-  cudaStream_t last_producer_stream = nullptr, last_consumer_stream = nullptr;
   bool have_producer_ev = false, have_consumer_ev = false;
   // samples in the order in which they became READY (slot, generation), for pool_take_ready
   std::deque<std::pair<uint32_t, uint64_t>> ready_fifo;
@@ -396,15 +394,19 @@ int32_t ctx_upload(ft_pool* p, ft_call_ctx* c, size_t bytes);
 int32_t ctx_release(ft_pool* p, ft_call_ctx* c, cudaStream_t last);
 // sequence number for asynchronous error keys of the current call
 inline uint64_t status_seq(const ft_pool* p) { return (p->call_seq - p->status_base) & kStatusSeqMask; }
-// `st` waits for everything enqueued on the metadata stream so far (skipped when it already has)
+// `st` waits for everything enqueued on the metadata stream so far.  One event serves every stream that asks while no
+// new metadata work is enqueued; once it has completed nobody needs to wait at all.  (No decision rests on the identity
+// of a stream handle: a destroyed stream's handle may come back for a new stream.)
 inline int32_t meta_to(ft_pool* p, cudaStream_t st) {
-  for (int i = 0; i < 2; ++i)
-    if (p->synced_stream[i] == st && p->synced_seq[i] == p->meta_seq) return FT_OK;
-  FT_CUDA(cudaEventRecord(p->ev_meta, p->meta));
+  if (p->ev_meta_seq != p->meta_seq) {
+    FT_CUDA(cudaEventRecord(p->ev_meta, p->meta));
+    p->ev_meta_seq = p->meta_seq;
+  } else {
+    const cudaError_t q = cudaEventQuery(p->ev_meta);
+    if (q == cudaSuccess) return FT_OK;
+    if (q != cudaErrorNotReady) return cuda_fail(q, "cudaEventQuery(ev_meta)");
+  }
   FT_CUDA(cudaStreamWaitEvent(st, p->ev_meta, 0));
-  int slot = p->synced_stream[0] == st && p->synced_seq[0] != ~0ull ? 0 : (p->synced_stream[1] == st && p->synced_seq[1] != ~0ull ? 1 : -1);
-  if (slot < 0) slot = p->synced_seq[0] == ~0ull ? 0 : (p->synced_seq[1] == ~0ull ? 1 : (p->synced_seq[0] <= p->synced_seq[1] ? 0 : 1));
-  p->synced_stream[slot] = st; p->synced_seq[slot] = p->meta_seq;
   return FT_OK;
 }
 // the metadata stream waits for everything enqueued on `st` so far
@@ -428,18 +430,22 @@ inline void ready_push(ft_pool* p, uint32_t slot) {
 
 // Cross-stream ordering.  Data kernels run on the callers' streams (a producer side and a consumer side, possibly two
 // streams), metadata kernels on the pool's metadata stream:
-//  * a consumer-side data kernel waits for the producer-side data kernels issued before it (another stream's only)
+//  * a consumer-side data kernel waits for the producer-side data kernels issued before it
 //    and for the metadata enqueued so far;
 //  * a metadata kernel that changes what data kernels already in flight may read (free, span grids) waits for the
 //    latest producer-side and consumer-side data kernels;
 //  * metadata kernels among themselves are ordered by the metadata stream.
 inline int32_t begin_consumer(ft_pool* p, cudaStream_t st) {
-  if (p->have_producer_ev && p->last_producer_stream != st) FT_CUDA(cudaStreamWaitEvent(st, p->ev_producer, 0));
+  // (a wait for an event of the same stream costs nothing on the device; a completed event needs no wait)
+  if (p->have_producer_ev && cudaEventQuery(p->ev_producer) != cudaSuccess) {
+    cudaGetLastError();
+    FT_CUDA(cudaStreamWaitEvent(st, p->ev_producer, 0));
+  }
   return meta_to(p, st);
 }
 inline int32_t end_consumer(ft_pool* p, cudaStream_t st) {
   FT_CUDA(cudaEventRecord(p->ev_consumer, st));
-  p->have_consumer_ev = true; p->last_consumer_stream = st;
+  p->have_consumer_ev = true;
   return FT_OK;
 }
 // before metadata kernels that retire or change state data kernels in flight may still read
@@ -450,7 +456,7 @@ inline int32_t meta_after_data(ft_pool* p) {
 }
 inline int32_t end_producer(ft_pool* p, cudaStream_t st) {
   FT_CUDA(cudaEventRecord(p->ev_producer, st));
-  p->have_producer_ev = true; p->last_producer_stream = st;
+  p->have_producer_ev = true;
   return FT_OK;
 }
 inline int32_t plan_alive(const ft_pool* p, const ft_plan* pl) {
