@@ -317,11 +317,12 @@ int32_t pool_free(ft_pool* pool, const uint32_t* sample_slot, uint32_t n, void* 
 /*
  * FT_ERR_TIMEOUT is the one asynchronous error that is not about the caller's data.  The host-tier kernels move pages
  * with bulk-asynchronous copies and wait for each staged load on an mbarrier; that wait, the library's only device-side
- * spin, gives up after 2 s of wall clock (a host link that has stopped answering).  The CTA then issues no further
- * copy, waits once more -- again at most 2 s -- for the loads it had already issued, and returns; detail = CTA index
- * (low 16 bits) | loads that had still not arrived when it returned (high 16 bits; 0 means that none can land later).
- * The bytes of that call are incomplete and the pool's state is no longer trustworthy: after FT_ERR_TIMEOUT the only
- * call a pool still supports is pool_destroy.
+ * spin, gives up after 2 s of wall clock (a host link that has stopped answering; ft_tuning.bulk_wait_limit_us).  The
+ * CTA then issues no further copy, waits once more -- again at most that long -- for the loads it had already issued,
+ * and returns; detail = CTA index (low 16 bits) | loads that had still not arrived when it returned (high 16 bits; 0
+ * means that none can land later).  The bytes of that call are incomplete and the pool's state is no longer
+ * trustworthy: after FT_ERR_TIMEOUT the only call a pool still supports is pool_destroy.  (Under the test hook
+ * ft_tuning.bulk_timeout_test nothing was lost: the call's output is incomplete, the pool is intact.)
  */
 /* First asynchronous error since the last call of pool_status (smallest call, then smallest code, then smallest
  * detail), then cleared.  Synchronises the device.  Calls are numbered from the last read, on 28 bits: read the
@@ -469,7 +470,7 @@ int32_t pool_profile_read(ft_pool* pool, ft_kernel_time* out /* host [FT_K_COUNT
  * in this one struct (nothing is read from the environment).  pool_get_tuning returns the values in force;
  * pool_set_tuning replaces them (0 in a field = that field's built-in default, the optimum measured on a B200);
  * out-of-range values INVALID_ARG and nothing changes.  Call it between other calls of the pool; it synchronises
- * the device.  None of the knobs changes any result.
+ * the device.  None of the knobs changes any result (bulk_timeout_test, a test hook, excepted).
  *   dev_ctas_per_sm      resident CTAs per SM of the HBM-tier gather kernel (default 4; 1..8)
  *   scatter_ctas_per_sm  resident CTAs per SM of the HBM-tier scatter kernel (default 4; 1..8)
  *   scatter_group        chunks a scatter CTA claims at a time (default 1)
@@ -495,12 +496,23 @@ int32_t pool_profile_read(ft_pool* pool, ft_kernel_time* out /* host [FT_K_COUNT
  *                        CTAs need costs it occupancy and 6 percent of its bandwidth)
  *   peers_remote         1: pool_import_mapping flags every peer's HBM frames as remote even when they are on this
  *                        device (exercises the remote path on one GPU); 0: only frames of another device are remote
+ *   bulk_wait_limit_us   bound, in microseconds, of every wait of the bulk-copy kernels for a staged load (default
+ *                        2 000 000; 100..10 000 000).  A load not seen within it is declared lost and the call
+ *                        reports FT_ERR_TIMEOUT through the status word (see FT_ERR_TIMEOUT above)
+ *   bulk_timeout_test    test hook for that path, 0 in use.  1: every staged load announces 16 bytes more to its
+ *                        completion barrier than it requests, so that no load is ever SEEN complete although all of
+ *                        them arrive: each bulk-copy CTA runs its first wait to the limit, gives up, waits once more
+ *                        (bounded) for the loads it had issued, and returns; the call stores nothing from those
+ *                        frames and reports FT_ERR_TIMEOUT.  Nothing faults and nothing spins beyond twice the
+ *                        limit; accepted only with bulk_wait_limit_us set to at most 100 000.  This is the one knob
+ *                        that changes results
  */
 typedef struct {
   uint32_t dev_ctas_per_sm, scatter_ctas_per_sm, scatter_group, chunk_shift;
   uint32_t host_ctas, host_store_ctas, gather_unroll, grad_ctas_per_sm, grad_hot_threshold;
   uint32_t remote_ctas, peers_remote, scatter_smem_carveout, gather_smem_carveout;
-  uint32_t reserved[3];
+  uint32_t bulk_wait_limit_us, bulk_timeout_test;
+  uint32_t reserved[1];
 } ft_tuning;
 int32_t pool_get_tuning(ft_pool* pool, ft_tuning* out);
 int32_t pool_set_tuning(ft_pool* pool, const ft_tuning* in);

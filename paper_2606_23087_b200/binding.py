@@ -66,11 +66,12 @@ class PoolStats(C.Structure):
 
 
 TUNING_FIELDS = ("dev_ctas_per_sm", "scatter_ctas_per_sm", "scatter_group", "chunk_shift", "host_ctas", "host_store_ctas",
-                 "gather_unroll", "grad_ctas_per_sm", "grad_hot_threshold", "remote_ctas", "peers_remote", "scatter_smem_carveout", "gather_smem_carveout")
+                 "gather_unroll", "grad_ctas_per_sm", "grad_hot_threshold", "remote_ctas", "peers_remote", "scatter_smem_carveout", "gather_smem_carveout",
+                 "bulk_wait_limit_us", "bulk_timeout_test")
 
 
 class Tuning(C.Structure):
-    _fields_ = [(k, C.c_uint32) for k in TUNING_FIELDS] + [("reserved", C.c_uint32 * 3)]
+    _fields_ = [(k, C.c_uint32) for k in TUNING_FIELDS] + [("reserved", C.c_uint32 * 1)]
 
 
 class KernelTime(C.Structure):

@@ -4,8 +4,8 @@
 // (mapped pinned host memory) without tying up the load/store pipelines of the SMs that stream HBM.
 // Every copy lands in the issuing CTA only.  Every wait is bounded.
 //
-// Giving up.  A staged load that has not arrived after kBulkWaitLimitNs is declared lost: the ring issues no further
-// load or store, and before the CTA returns drain() waits once more, again bounded, for every load it had already
+// Giving up.  A staged load that has not arrived after the wait limit (2 s unless the pool's tuning says otherwise)
+// is declared lost: the ring issues no further load or store, and before the CTA returns drain() waits once more, again bounded, for every load it had already
 // issued, so that none of them can land later in shared memory that by then belongs to another CTA; `stranded`
 // counts the loads that had still not arrived when that second wait ran out as well (the kernel reports it in the
 // error detail).  Stores already issued are waited for with the hardware's group wait.
@@ -46,7 +46,7 @@ __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.a
 constexpr int kBulkStages = 12;            // ring size
 constexpr int kBulkDepth = 8;              // loads in flight
 constexpr uint32_t kBulkStageBytes = 16384;
-constexpr uint64_t kBulkWaitLimitNs = 2000000000ull;  // a staged load not seen after 2 s is declared lost
+constexpr uint64_t kBulkWaitLimitNs = 2000000000ull;  // default: a staged load not seen after 2 s is declared lost
 __device__ __forceinline__ uint64_t global_timer_ns() {
   uint64_t t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -63,11 +63,14 @@ struct BulkRing {
   uint64_t* dst_q;   // kBulkStages pending destinations (shared memory)
   uint32_t* len_q;   // kBulkStages pending staged lengths
   uint64_t issued, retired;
+  uint64_t limit_ns;  // bound of every wait
+  uint32_t tx_slack;  // bytes announced to the barrier beyond the load's size (0; 16 under the timeout test)
   uint32_t stranded;  // loads still not arrived when a CTA that gave up returned
   bool lost;
 
-  __device__ void init(uint8_t* stage_, uint64_t* bar_, uint64_t* dst_q_, uint32_t* len_q_) {
+  __device__ void init(uint8_t* stage_, uint64_t* bar_, uint64_t* dst_q_, uint32_t* len_q_, uint64_t limit_ns_, uint32_t tx_slack_) {
     stage = stage_; bar = bar_; dst_q = dst_q_; len_q = len_q_;
+    limit_ns = limit_ns_; tx_slack = tx_slack_;
     issued = retired = 0; lost = false; stranded = 0;
     if ((threadIdx.x & 31) == 0) {
       for (int i = 0; i < kBulkStages; ++i) mbar_init(&bar[i], 1);
@@ -87,7 +90,7 @@ struct BulkRing {
       const uint64_t t0 = global_timer_ns();
       uint32_t spins = 0;
       while (!mbar_try_wait(&bar[st], parity)) {
-        if ((++spins & 1023u) == 0 && global_timer_ns() - t0 > kBulkWaitLimitNs) { bad = 1; break; }
+        if ((++spins & 1023u) == 0 && global_timer_ns() - t0 > limit_ns) { bad = 1; break; }
       }
     }
     bad = __shfl_sync(0xFFFFFFFFu, bad, 0);
@@ -109,7 +112,7 @@ struct BulkRing {
       bulk_wait_read<kBulkStages - kBulkDepth>();
       dst_q[st] = reinterpret_cast<uint64_t>(dst);
       len_q[st] = bytes;
-      mbar_expect_tx(&bar[st], bytes);
+      mbar_expect_tx(&bar[st], bytes + tx_slack);
       bulk_g2s(stage + (size_t)st * kBulkStageBytes, src, bytes, &bar[st]);
     }
     __syncwarp();
@@ -127,7 +130,7 @@ struct BulkRing {
           const uint32_t parity = (uint32_t)((k / kBulkStages) & 1);
           bool here = mbar_try_wait(&bar[st], parity);
           uint32_t spins = 0;
-          while (!here && !((++spins & 1023u) == 0 && global_timer_ns() - t0 > kBulkWaitLimitNs)) here = mbar_try_wait(&bar[st], parity);
+          while (!here && !((++spins & 1023u) == 0 && global_timer_ns() - t0 > limit_ns)) here = mbar_try_wait(&bar[st], parity);
           if (!here) ++left;
         }
       }

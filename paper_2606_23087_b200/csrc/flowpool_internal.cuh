@@ -68,6 +68,10 @@ struct PoolView {
   uint64_t* list_blocks;   // [bring_cap][kListBlock] page GVAs
   uint4* sp_grid;          // token grid (T, H, W, 0) of a span; all zero = none given
   unsigned long long* status;  // first asynchronous error key; ~0 = none
+  // the bulk-copy rings' bounded waits: limit per wait, and bytes a staged load announces beyond what it requests
+  // (0 in use; 16 only under the timeout test, whose loads are therefore never seen complete)
+  uint64_t bulk_wait_ns;
+  uint32_t bulk_tx_slack;
 };
 
 // key = seq << 36 | (-code) << 32 | detail ; the smallest key is reported.  seq = calls since the status word was

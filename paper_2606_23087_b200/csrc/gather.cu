@@ -230,7 +230,7 @@ __global__ void __launch_bounds__(32) k_gather_host_bulk(PoolView v, PlanView pl
   __shared__ uint32_t len_q[kBulkStages];
   const uint32_t lane = threadIdx.x;
   BulkRing ring;
-  ring.init(smem, bars, dst_q, len_q);
+  ring.init(smem, bars, dst_q, len_q, v.bulk_wait_ns, v.bulk_tx_slack);
   uint64_t item = 0;
   // the samples to assemble: the call's range, or the samples of each listed microbatch in turn
   const uint32_t n_parts = a.list ? a.n_list : 1;

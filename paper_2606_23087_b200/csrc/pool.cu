@@ -418,7 +418,7 @@ __global__ void __launch_bounds__(32) k_scatter_host_bulk(PoolView v, WriteCall 
   __shared__ uint32_t len_q[kBulkStages];
   const uint32_t lane = threadIdx.x;
   BulkRing ring;
-  ring.init(smem, bars, dst_q, len_q);
+  ring.init(smem, bars, dst_q, len_q, v.bulk_wait_ns, v.bulk_tx_slack);
   uint64_t item = 0;
   for (uint32_t q = 0; q < c.n; ++q) {
     const uint32_t sid = c.span_id[q];
@@ -782,6 +782,8 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_create(const ft_p
   RingState* st = reinterpret_cast<RingState*>(m + o_states);
   v.ring_state = st; v.tring_state = st + 1; v.bring_state = st + 2;
   v.status = reinterpret_cast<unsigned long long*>(m + o_status);
+  v.bulk_wait_ns = kBulkWaitLimitNs;
+  v.bulk_tx_slack = 0;
   for (int i = 0; i < 2 * kCallCtx; ++i) p->ctx[i / kCallCtx][i % kCallCtx].counters = reinterpret_cast<ClaimCounter*>(m + o_status + 64) + 2 * i;
   v.s_seq_len = reinterpret_cast<uint32_t*>(m + o_seq); v.s_n_spans = reinterpret_cast<uint32_t*>(m + o_nsp);
   v.s_text_pages = reinterpret_cast<uint64_t*>(m + o_stp);
@@ -1201,6 +1203,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_get_tuning(ft_poo
   out->grad_ctas_per_sm = (uint32_t)p->grad_ctas_per_sm; out->grad_hot_threshold = (uint32_t)p->grad_hot_threshold;
   out->remote_ctas = (uint32_t)p->remote_ctas; out->peers_remote = (uint32_t)p->peers_remote;
   out->scatter_smem_carveout = (uint32_t)p->scatter_smem_carveout; out->gather_smem_carveout = (uint32_t)p->gather_smem_carveout;
+  out->bulk_wait_limit_us = (uint32_t)(p->view.bulk_wait_ns / 1000); out->bulk_timeout_test = p->view.bulk_tx_slack ? 1u : 0u;
   return FT_OK;
 }
 
@@ -1211,7 +1214,11 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_set_tuning(ft_poo
   if (t.chunk_shift && (t.chunk_shift < 14 || t.chunk_shift > 21)) return FT_ERR_INVALID_ARG;  // a warp's eighth holds a 2 KiB batch
   if (t.gather_unroll && t.gather_unroll != 4 && t.gather_unroll != 8) return FT_ERR_INVALID_ARG;
   if (t.host_ctas > 1024 || t.host_store_ctas > 1024 || t.remote_ctas > 1024 || t.scatter_group > (1u << 20) || t.peers_remote > 1 || t.scatter_smem_carveout > 100 || t.gather_smem_carveout > 100) return FT_ERR_INVALID_ARG;
+  if (t.bulk_wait_limit_us && (t.bulk_wait_limit_us < 100 || t.bulk_wait_limit_us > 10000000)) return FT_ERR_INVALID_ARG;
+  if (t.bulk_timeout_test > 1 || (t.bulk_timeout_test && (t.bulk_wait_limit_us == 0 || t.bulk_wait_limit_us > 100000))) return FT_ERR_INVALID_ARG;
   FT_CUDA(cudaDeviceSynchronize());  // no kernel of an earlier call is still being sized by the old values
+  p->view.bulk_wait_ns = t.bulk_wait_limit_us ? (uint64_t)t.bulk_wait_limit_us * 1000 : kBulkWaitLimitNs;
+  p->view.bulk_tx_slack = t.bulk_timeout_test ? 16u : 0u;
   p->dev_ctas_per_sm = t.dev_ctas_per_sm ? (int)t.dev_ctas_per_sm : 4;
   p->scatter_ctas_per_sm = (int)t.scatter_ctas_per_sm;
   p->scatter_group = (int)t.scatter_group;

@@ -60,6 +60,56 @@ def test_tuning_round_trip_and_range_checks():
     pool.destroy()
 
 
+def test_a_bulk_wait_that_runs_out_reports_timeout_and_leaves_the_context_usable():
+    """The one device-side wait of the library (a bulk-copy CTA waiting for a staged load) is made to run out without
+    any fault: under the `bulk_timeout_test` hook every load announces 16 bytes more than it requests, so no load is
+    ever seen complete although all of them arrive.  Each host-tier CTA waits 2 ms, gives up, waits once more for the
+    loads it had issued, and returns; the call reports FT_ERR_TIMEOUT with the loads it counted as not arrived, stores
+    nothing from host frames, and the CUDA context and the pool stay usable: with the hook off, the same plan
+    assembles bit-exactly."""
+    if not torch.cuda.is_available():
+        pytest.fail("a CUDA device is required for -m gpu tests")
+    from gpu_harness import CudaRun, bits16, host_bits
+    from paper_2606_23087_b200 import binding as fp
+    w = workloads.make_workload("image_mix_7b", n_samples=10, hidden=512, page_bytes=65536)
+    r = CudaRun(w)
+    r.run_schedule()
+    assert w.host_pages > 0
+    rc, plan = r.plan()
+    assert rc == 0
+    # the hook is refused without a short limit
+    assert r.pool.set_tuning(bulk_timeout_test=1) == -1 and r.pool.set_tuning(bulk_timeout_test=1, bulk_wait_limit_us=200000) == -1
+    assert r.pool.set_tuning(bulk_wait_limit_us=50) == -1
+    assert r.pool.set_tuning(bulk_timeout_test=1, bulk_wait_limit_us=2000) == 0
+    rc, out, cu, pos = r.gather_all()
+    assert rc == 0                                           # the error is asynchronous
+    code, detail = r.pool.status()
+    assert code == -13, fp.STATUS.get(code)                  # FT_ERR_TIMEOUT
+    assert (detail >> 16) & 0xFFFF >= 1                      # loads counted as not arrived when the CTA returned
+    assert (detail & 0xFFFF) < r.pool.get_tuning()["host_ctas"]
+    poisoned = np.all(out.cpu().numpy().view(np.uint16) == 0xFFFF, axis=1)
+    assert poisoned.any()                                    # rows that live on host frames were not stored
+    assert r.pool.status() == (0, 0)                         # reading clears it
+    # a producer call under the hook: same report from the host-tier scatter (into a second pool, to keep this one's data)
+    r2 = CudaRun(w, tuning=dict(bulk_timeout_test=1, bulk_wait_limit_us=2000))
+    r2.run_schedule()
+    torch.cuda.synchronize()
+    assert all(c == 0 for c in r2.rc) and r2.pool.status()[0] == -13
+    r2.close()
+    # hook off: the first pool, its plan and the context still work, bit for bit
+    assert r.pool.set_tuning() == 0 and r.pool.get_tuning()["bulk_timeout_test"] == 0
+    assert r.pool.get_tuning()["bulk_wait_limit_us"] == 2000000
+    rc, out, cu, pos = r.gather_all()
+    got = dict(plan=plan.arrays(), rc=r.rc, out=out.cpu().numpy().view(np.uint16), cu_seqlens=cu.cpu().numpy(),
+               position_ids=pos.cpu().numpy(), status=r.pool.status(), table=bits16(r.table),
+               span_pages={(s, j): r.pool.span_pages(s, j)[1] for call in w.write_calls for s, j in call},
+               srcs={c: host_bits(t) for c, t in r.srcs.items()}, stats=r.pool.stats())
+    exp = oracle_from_device_sources(w, got["srcs"], got["table"])
+    got["rc"] = [c for c in got["rc"]][:len(exp["rc"])]
+    assert_same(got, exp)
+    r.close()
+
+
 def test_bench_gpus_2_runs_the_exchange_flow_with_two_ranks_on_this_gpu():
     """`bench.py --gpus 2` launches two ranks by itself; with the gloo backend both may share this GPU (their kernels
     never wait on one another: the ranks meet only in host-side collectives).  One line, from rank 0, with the
