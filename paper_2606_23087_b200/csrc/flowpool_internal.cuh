@@ -188,6 +188,7 @@ struct PlanView {
   const uint32_t* mb_sample_off;     // [n_mb+1]
   const uint64_t* mb_row_off;        // [n_mb+1]
   const uint32_t* tile_first_sample; // [ceil(rows/32)] plan position of the sample holding row 32*T
+  const uint64_t* row_src;           // [rows] row words (kind | position | token id or span id), or nullptr
 };
 
 }  // namespace ft
@@ -211,6 +212,7 @@ struct ft_plan {
   uint32_t *d_mb_tokens, *d_mb_lmax, *d_mb_residual, *d_mb_count, *d_mb_bucket, *d_mb_rank, *d_mb_pos;
   uint32_t *d_rank_mb_off, *d_rank_mbs, *d_rank_cnt, *d_tile_first_sample, *d_scalars;
   uint64_t *d_sample_cost, *d_mb_cost, *d_sample_row_off, *d_mb_row_off, *d_plan_len;
+  uint64_t* d_row_src = nullptr;          // row words of the assembly (plans of written samples only)
 };
 
 namespace ft {
@@ -220,6 +222,7 @@ inline PlanView make_plan_view(const ft_plan* pl) {
   pv.mb_samples = pl->d_mb_samples; pv.plan_sample_mb = pl->d_plan_sample_mb;
   pv.sample_row_off = pl->d_sample_row_off; pv.mb_sample_off = pl->d_mb_sample_off;
   pv.mb_row_off = pl->d_mb_row_off; pv.tile_first_sample = pl->d_tile_first_sample;
+  pv.row_src = pl->d_row_src;
   return pv;
 }
 // A plan dies with any of its samples (freed, or never completed under ALLOW_UNWRITTEN): FT_OK while every sample
@@ -296,6 +299,8 @@ struct ft_pool {
   cudaStream_t meta = nullptr;
   cudaEvent_t ev_meta = nullptr;      // re-recorded on `meta` whenever a caller's stream has to wait for it
   cudaEvent_t ev_in = nullptr;        // re-recorded on a caller's stream when `meta` has to wait for that stream
+  cudaEvent_t ev_ids = nullptr;       // behind the latest copy of token ids into text pages (a caller's stream)
+  bool have_ids_ev = false;
   cudaEvent_t ev_noalloc = nullptr;   // behind the last reader of the fixed no-allocation scratch
   bool have_noalloc_ev = false;
   uint64_t meta_seq = 0;              // metadata batches enqueued so far
@@ -359,6 +364,8 @@ namespace ft {
 int32_t gather_device_setup(ft_pool* p);
 // shared-memory carve-out preference (percent) of the copy kernels of each translation unit
 int32_t gather_set_carveout(int pct);
+// fills the plan's row words (metadata stream, behind the latest copy of token ids)
+int32_t plan_rows_launch(ft_pool* p, ft_plan* pl);
 int32_t scatter_set_carveout(int pct);
 int32_t plan_device_setup(ft_pool* p);
 // (d_list: device array of the list layout's entries, or nullptr for the range [mb_begin, mb_end))

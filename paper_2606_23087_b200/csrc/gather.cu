@@ -7,6 +7,13 @@
 // the span's two-level list -> page-table entry), leaving the frame addresses in the other half of a double buffer
 // in shared memory.  Rows that straddle pages carry one address per page touched.  With a two-tier pool the kernel
 // is launched once per tier, so host-link reads never stall HBM reads.
+//
+// Row table.  A plan of written samples carries one 64-bit word per output row, made once when the plan is made
+// (k_plan_rows): position in the sample plus the token id (text row) or the span (placeholder row).  With it the
+// resolver's chain of dependent loads is claim -> row word -> table row (text) or -> page list -> page-table entry
+// (vision) instead of eight to ten steps; it matters where a CTA resolves its first unit with nothing to overlap it
+// (short ranges: one microbatch per call, the tiny configuration).  The table holds no address and no page: a row
+// whose word says "unresolved" (0) takes the long way, so results and errors are the same with and without it.
 #include <algorithm>
 #include <cstdlib>
 #include <cstring>
@@ -24,6 +31,9 @@ constexpr int kStreamWarps = 8;                          // warps that copy rows
 constexpr int kGatherThreads = 32 * (kStreamWarps + 1);  // + the resolver warp
 
 enum { kTierAll = 0, kTierDeviceOnly = 1, kTierHostOnly = 2 };
+
+// row word: kind (2 bits: 0 unresolved, 1 text, 2 placeholder) | position in the sample (30 bits) | token id or span id
+constexpr uint64_t kRowText = 1ull << 62, kRowVision = 2ull << 62;
 
 struct RowDesc {
   uint64_t seg[kMaxSeg];  // page-table entries (frame address | flags) of the pages the row touches
@@ -71,11 +81,33 @@ __global__ void __launch_bounds__(kGatherThreads) k_gather(PoolView v, PlanView 
   const bool resolver = warp == kStreamWarps;
 
   // Resolver warp: claims the next unit (units are claimed in order, so the CTAs in flight always cover one compact
-  // window of the output and uneven units balance themselves) and resolves its rows into desc[buf].
+  // window of the output and uneven units balance themselves; a CTA's first unit is its block index, which saves one
+  // round trip to the counter) and resolves its rows into desc[buf].
+  const bool use_rows = pl.row_src != nullptr && a.pad_L == 0;
+  bool first_claim = true;
+  // cu_seqlens of a sample whose first row was resolved through the row table: written after the unit is published
+  uint64_t pend_row = ~0ull, pend_cu0 = 0;
+  uint32_t pend_q_lo = 0, pend_tile_q = 0;
+  auto finish_index = [&]() {
+    if (pend_row == ~0ull) return;
+    uint32_t q = pend_tile_q;
+    if (q < pend_q_lo) q = pend_q_lo;
+    while (pend_row >= pl.sample_row_off[q + 1]) ++q;
+    const uint32_t j = pl.plan_sample_mb[q];
+    const uint64_t e = LIST ? pend_cu0 + (q - pend_q_lo) : (uint64_t)(q - a.q_lo) + (j - a.mb_begin);
+    a.cu[e] = (int32_t)(pl.sample_row_off[q] - pl.mb_row_off[j]);
+    if (q + 1 == pl.mb_sample_off[j + 1]) a.cu[e + 1] = (int32_t)(pl.sample_row_off[q + 1] - pl.mb_row_off[j]);
+    pend_row = ~0ull;
+  };
   auto resolve = [&](uint32_t buf) {
     unsigned long long c = 0;
-    if (lane == 0) c = atomicAdd(&a.tile_counter->claim, 1ull);
-    c = __shfl_sync(0xFFFFFFFFu, c, 0);
+    if (first_claim) {
+      c = blockIdx.x;
+      first_claim = false;
+    } else {
+      if (lane == 0) c = gridDim.x + atomicAdd(&a.tile_counter->claim, 1ull);
+      c = __shfl_sync(0xFFFFFFFFu, c, 0);
+    }
     const uint64_t ct = c >> a.sub_shift;  // claim index in whole 32-row tiles
     uint64_t tile = ~0ull;
     uint32_t entry = 0;
@@ -108,44 +140,60 @@ __global__ void __launch_bounds__(kGatherThreads) k_gather(PoolView v, PlanView 
       row_lo = en.row_lo; row_hi = en.row_hi; out0 = en.out_row0; cu0 = en.cu0; q_lo = en.q_lo;
     }
     if (row >= row_lo && row < row_hi) {
-      // plan position of the sample holding this row: the tile's first sample, then a short walk
-      uint32_t q = pl.tile_first_sample[tile];
-      if (q < q_lo) q = q_lo;
-      while (row >= pl.sample_row_off[q + 1]) ++q;
-      const uint32_t p = (uint32_t)(row - pl.sample_row_off[q]);
-      const uint32_t slot = pl.mb_samples[q];
+      const uint64_t word = use_rows ? pl.row_src[row] : 0ull;
+      uint32_t p, sid = 0;
       uint64_t out_row = out0 + (row - row_lo);
-      if (!LIST && a.pad_L) {  // padded layout: microbatch j of the range starts at row (j - mb_begin) * L
-        const uint32_t j = pl.plan_sample_mb[q];
-        out_row += (uint64_t)(j - a.mb_begin) * a.pad_L - (pl.mb_row_off[j] - a.row_lo);
-      }
-      d.out_row = (uint32_t)out_row;
-      if (a.write_index) {
-        a.pos_ids[out_row] = (int32_t)p;
-        if (p == 0) {  // cu_seqlens: every sample writes its start; the last of a microbatch also the end
+      int kind = (int)(word >> 62);  // 0: the long way
+      int32_t id = -1;
+      bool text_ok = true;
+      if (kind) {
+        p = (uint32_t)(word >> 32) & 0x3FFFFFFFu;
+        if (kind == 1) id = (int32_t)(uint32_t)word; else sid = (uint32_t)word;
+        if (a.write_index) {
+          a.pos_ids[out_row] = (int32_t)p;
+          if (p == 0) { pend_row = row; pend_cu0 = cu0; pend_q_lo = q_lo; pend_tile_q = pl.tile_first_sample[tile]; }
+        }
+      } else {
+        // plan position of the sample holding this row: the tile's first sample, then a short walk
+        uint32_t q = pl.tile_first_sample[tile];
+        if (q < q_lo) q = q_lo;
+        while (row >= pl.sample_row_off[q + 1]) ++q;
+        p = (uint32_t)(row - pl.sample_row_off[q]);
+        const uint32_t slot = pl.mb_samples[q];
+        if (!LIST && a.pad_L) {  // padded layout: microbatch j of the range starts at row (j - mb_begin) * L
           const uint32_t j = pl.plan_sample_mb[q];
-          const uint64_t e = LIST ? cu0 + (q - q_lo) : (uint64_t)(q - a.q_lo) + (j - a.mb_begin);
-          a.cu[e] = (int32_t)(pl.sample_row_off[q] - pl.mb_row_off[j]);
-          if (q + 1 == pl.mb_sample_off[j + 1]) a.cu[e + 1] = (int32_t)(pl.sample_row_off[q + 1] - pl.mb_row_off[j]);
+          out_row += (uint64_t)(j - a.mb_begin) * a.pad_L - (pl.mb_row_off[j] - a.row_lo);
+        }
+        if (a.write_index) {
+          a.pos_ids[out_row] = (int32_t)p;
+          if (p == 0) {  // cu_seqlens: every sample writes its start; the last of a microbatch also the end
+            const uint32_t j = pl.plan_sample_mb[q];
+            const uint64_t e = LIST ? cu0 + (q - q_lo) : (uint64_t)(q - a.q_lo) + (j - a.mb_begin);
+            a.cu[e] = (int32_t)(pl.sample_row_off[q] - pl.mb_row_off[j]);
+            if (q + 1 == pl.mb_sample_off[j + 1]) a.cu[e + 1] = (int32_t)(pl.sample_row_off[q + 1] - pl.mb_row_off[j]);
+          }
+        }
+        // Is position p inside a placeholder run?  The span table decides (last span with pos_start <= p).
+        const uint32_t sbase = slot * v.spans_per_sample, ns = v.s_n_spans[slot];
+        uint32_t lo = 0, hi = ns;
+        while (lo < hi) {
+          const uint32_t mid = (lo + hi) >> 1;
+          if (v.sp_pos[sbase + mid] <= p) lo = mid + 1; else hi = mid;
+        }
+        sid = sbase + lo - 1;
+        const bool in_run = lo > 0 && p < v.sp_pos[sid] + v.sp_tokens[sid];
+        kind = in_run ? 2 : 1;
+        if (!in_run) {
+          // token id, through the text page
+          const uint64_t tp_gva = v.s_text_pages[(uint64_t)slot * v.text_pages_per_sample + p / kTextPageIds];
+          uint64_t off;
+          const uint64_t tpte = translate(v, tp_gva, &off);
+          text_ok = (tpte & kPteValid) && (tpte & kPteText);  // e.g. a peer's page whose mapping was never imported
+          if (text_ok) id = reinterpret_cast<const int32_t*>(tpte & ~kPteFlagMask)[p % kTextPageIds];
         }
       }
-      // Is position p inside a placeholder run?  The span table decides (last span with pos_start <= p).
-      const uint32_t sbase = slot * v.spans_per_sample, ns = v.s_n_spans[slot];
-      uint32_t lo = 0, hi = ns;
-      while (lo < hi) {
-        const uint32_t mid = (lo + hi) >> 1;
-        if (v.sp_pos[sbase + mid] <= p) lo = mid + 1; else hi = mid;
-      }
-      const uint32_t sid = sbase + lo - 1;
-      const bool in_run = lo > 0 && p < v.sp_pos[sid] + v.sp_tokens[sid];
-      if (!in_run) {
-        // token id, through the text page, then the embedding-table row
-        const uint64_t tp_gva = v.s_text_pages[(uint64_t)slot * v.text_pages_per_sample + p / kTextPageIds];
-        uint64_t off;
-        const uint64_t tpte = translate(v, tp_gva, &off);
-        int32_t id = -1;
-        const bool text_ok = (tpte & kPteValid) && (tpte & kPteText);  // e.g. a peer's page whose mapping was never imported
-        if (text_ok) id = reinterpret_cast<const int32_t*>(tpte & ~kPteFlagMask)[p % kTextPageIds];
+      d.out_row = (uint32_t)out_row;
+      if (kind == 1) {
         if (!text_ok) {
           note_error(v, a.call_seq, FT_ERR_BAD_GVA, (uint32_t)out_row);
         } else if (id < 0 || (uint32_t)id >= a.vocab) {
@@ -181,6 +229,7 @@ __global__ void __launch_bounds__(kGatherThreads) k_gather(PoolView v, PlanView 
   for (uint32_t buf = 0;; buf ^= 1) {
     if (!valid[buf]) break;
     if (resolver) {
+      finish_index();    // what the unit just published still owes to cu_seqlens
       resolve(buf ^ 1);  // one unit ahead of the copy
     } else {
       for (uint32_t r = warp; r < R; r += kStreamWarps) {
@@ -217,6 +266,49 @@ __global__ void __launch_bounds__(kGatherThreads) k_gather(PoolView v, PlanView 
     }
     __syncthreads();  // desc[buf ^ 1] is complete, desc[buf] is free
   }
+}
+
+// The plan's row words: one thread per output row walks the same tables the resolver's long way walks (plan position,
+// span table, text page) and leaves what it found.  Rows whose text page cannot be translated stay unresolved (0).
+__global__ void __launch_bounds__(256) k_plan_rows(PoolView v, PlanView pl, uint64_t rows, uint64_t* __restrict__ row_src) {
+  for (uint64_t row = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; row < rows; row += (uint64_t)gridDim.x * blockDim.x) {
+    uint32_t q = pl.tile_first_sample[row / kTileRows];
+    while (row >= pl.sample_row_off[q + 1]) ++q;
+    const uint32_t p = (uint32_t)(row - pl.sample_row_off[q]);
+    const uint32_t slot = pl.mb_samples[q];
+    const uint32_t sbase = slot * v.spans_per_sample, ns = v.s_n_spans[slot];
+    uint32_t lo = 0, hi = ns;
+    while (lo < hi) {
+      const uint32_t mid = (lo + hi) >> 1;
+      if (v.sp_pos[sbase + mid] <= p) lo = mid + 1; else hi = mid;
+    }
+    const uint32_t sid = sbase + lo - 1;
+    uint64_t word = 0;
+    if (lo > 0 && p < v.sp_pos[sid] + v.sp_tokens[sid]) {
+      word = kRowVision | ((uint64_t)p << 32) | sid;
+    } else {
+      const uint64_t tp_gva = v.s_text_pages[(uint64_t)slot * v.text_pages_per_sample + p / kTextPageIds];
+      uint64_t off;
+      const uint64_t tpte = translate(v, tp_gva, &off);
+      if ((tpte & kPteValid) && (tpte & kPteText)) {
+        const int32_t id = reinterpret_cast<const int32_t*>(tpte & ~kPteFlagMask)[p % kTextPageIds];
+        word = kRowText | ((uint64_t)p << 32) | (uint32_t)id;
+      }
+    }
+    row_src[row] = word;
+  }
+}
+
+int32_t plan_rows_launch(ft_pool* p, ft_plan* pl) {
+  if (!pl->d_row_src || pl->total_tokens == 0) return FT_OK;
+  if (p->have_ids_ev) FT_CUDA(cudaStreamWaitEvent(p->meta, p->ev_ids, 0));  // the ids are a caller's data, copied on its stream
+  const uint64_t rows = pl->total_tokens;
+  const unsigned grid = (unsigned)std::min<uint64_t>((rows + 255) / 256, (uint64_t)p->sm_count * 16);
+  k_plan_rows<<<grid, 256, 0, p->meta>>>(p->view, make_plan_view(pl), rows, pl->d_row_src);
+  FT_CUDA(cudaGetLastError());
+  ++p->meta_seq;
+  ++p->gpu_launches;
+  return FT_OK;
 }
 
 // Host-tier vision data, page by page.  A span's rows are consecutive output rows, so a page of the span is one

@@ -432,9 +432,10 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_plan_microbatches
     *out = pl;
     return FT_OK;
   }
-  // The plan reads the pool's tables only (lengths and states), never embedding bytes or token ids: all of its
-  // kernels run on the metadata stream, so a plan requested right after the last producer call is made while that
-  // call's copy is still streaming on the caller's stream.
+  // The plan reads the pool's tables only (lengths and states), never embedding bytes: all of its kernels run on the
+  // metadata stream, so a plan requested right after the last producer call is made while that call's copy is still
+  // streaming on the caller's stream.  (The row words, filled after the summary has come back, read token ids: that
+  // one kernel waits for the latest registration's copy of ids, which precedes the producer call's copy.)
   (void)stream;
   cudaStream_t st = p->meta;
   const uint64_t n_tiles = (total_tokens + 31) / 32 + 1;
@@ -452,6 +453,9 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_plan_microbatches
   const size_t o_bkt = take(n * 4), o_rank = take(n * 4), o_pos = take(n * 4), o_idx = take(n * 4);
   const size_t o_roff = take(((size_t)N + 1) * 4), o_rmbs = take(n * 4), o_rcnt = take((size_t)N * 4);
   const size_t o_tiles = take(n_tiles * 4), o_scal = take(SC_COUNT * 4);
+  // row words of the assembly: only where every sample is written (a metadata-only plan is not assembled from)
+  const bool with_rows = !(cfg->flags & FT_PLAN_ALLOW_UNWRITTEN);
+  const size_t o_rows = with_rows ? take((size_t)total_tokens * 8) : 0;
   pl->last_stream = st;
   {
     // a cached block that is large enough: one nobody reads any more if there is one, else the metadata stream
@@ -496,6 +500,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_plan_microbatches
   pl->d_mb_bucket = U32(o_bkt); pl->d_mb_rank = U32(o_rank); pl->d_mb_pos = U32(o_pos);
   pl->d_rank_mb_off = U32(o_roff); pl->d_rank_mbs = U32(o_rmbs); pl->d_rank_cnt = U32(o_rcnt);
   pl->d_tile_first_sample = U32(o_tiles); pl->d_scalars = U32(o_scal);
+  pl->d_row_src = with_rows ? U64(o_rows) : nullptr;
   uint32_t* d_mb_idx = U32(o_idx);
   uint32_t *d_pk_t = U32(o_pkt), *d_pk_len = U32(o_pklen), *d_pk_mb = U32(o_pkmb);
   MbRec* d_recs = reinterpret_cast<MbRec*>(b + o_recs);
@@ -583,6 +588,10 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_plan_microbatches
   pl->total_tokens = (uint64_t)sc[SC_TOTAL_LO] | ((uint64_t)sc[SC_TOTAL_HI] << 32);
   pl->h_mb_sample_off.assign(reinterpret_cast<const uint32_t*>(rb + rb_so), reinterpret_cast<const uint32_t*>(rb + rb_so) + pl->n_mb + 1);
   pl->h_mb_row_off.assign(reinterpret_cast<const uint64_t*>(rb + rb_ro), reinterpret_cast<const uint64_t*>(rb + rb_ro) + pl->n_mb + 1);
+  // the row words are filled behind the caller's back: the plan is complete for the host, assemblies wait for the
+  // metadata stream anyway
+  rc = plan_rows_launch(p, pl);
+  if (rc != FT_OK) { plan_destroy(pl); return rc; }
 #undef CK
   *out = pl;
   return FT_OK;

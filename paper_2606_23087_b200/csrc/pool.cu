@@ -632,6 +632,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_destroy(ft_pool* 
   if (p->meta) cudaStreamDestroy(p->meta);
   if (p->ev_meta) cudaEventDestroy(p->ev_meta);
   if (p->ev_in) cudaEventDestroy(p->ev_in);
+  if (p->ev_ids) cudaEventDestroy(p->ev_ids);
   if (p->ev_noalloc) cudaEventDestroy(p->ev_noalloc);
   for (void* a : p->peer_allocs) cudaFree(a);
   if (p->d_meta) cudaFree(p->d_meta);
@@ -695,6 +696,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_create(const ft_p
   CK(cudaStreamCreateWithFlags(&p->meta, cudaStreamNonBlocking));
   CK(cudaEventCreateWithFlags(&p->ev_meta, cudaEventDisableTiming));
   CK(cudaEventCreateWithFlags(&p->ev_in, cudaEventDisableTiming));
+  CK(cudaEventCreateWithFlags(&p->ev_ids, cudaEventDisableTiming));
   CK(cudaEventCreateWithFlags(&p->ev_noalloc, cudaEventDisableTiming));
   // every call context starts with 64 KiB of pinned staging and 256 KiB of device scratch (enough for calls of a few
   // thousand spans), so that no call of ordinary size allocates; larger calls grow their context on demand
@@ -922,6 +924,8 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_register_samples(
   if ((rc = meta_to(p, st)) != FT_OK) return rc;
   k_register_ids<<<(unsigned)text_need, 256, 0, st>>>(p->view, rcall);
   FT_CUDA(cudaGetLastError());
+  FT_CUDA(cudaEventRecord(p->ev_ids, st));
+  p->have_ids_ev = true;
   if ((rc = ctx_release(p, cx, st)) != FT_OK) return rc;
   p->gpu_launches += 2;
 
