@@ -281,11 +281,19 @@ __global__ void __launch_bounds__(1024) k_row_offsets(const uint64_t* plan_len, 
   if (threadIdx.x == 0) sample_row_off[n] = carry;
 }
 
-__global__ void k_tiles(const uint64_t* sample_row_off, uint32_t n, uint32_t* tile_first_sample) {
-  const uint32_t q = blockIdx.x * blockDim.x + threadIdx.x;
-  if (q >= n) return;
-  const uint64_t t0 = (sample_row_off[q] + 31) / 32, t1 = (sample_row_off[q + 1] + 31) / 32;
-  for (uint64_t t = t0; t < t1; ++t) tile_first_sample[t] = q;  // rows 32t lies inside sample q
+// one thread per 32-row tile: the plan position of the sample holding the tile's first row (last q with
+// sample_row_off[q] <= 32 t; samples are never empty)
+__global__ void k_tiles(const uint64_t* sample_row_off, uint32_t n, uint64_t n_tiles, uint32_t* tile_first_sample) {
+  const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= n_tiles) return;
+  const uint64_t row = t * 32;
+  if (row >= sample_row_off[n]) return;  // the spare entry past the last row
+  uint32_t lo = 0, hi = n;
+  while (hi - lo > 1) {
+    const uint32_t mid = (lo + hi) >> 1;
+    if (sample_row_off[mid] <= row) lo = mid; else hi = mid;
+  }
+  tile_first_sample[t] = lo;
 }
 
 // auto_N != 0 (variant): K is only the upper limit; one bucket per full zig-zag round trip of 2N microbatches.
@@ -557,7 +565,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_plan_microbatches
   k_mb_cost<<<gb, 256, 0, st>>>(cfg->coef_A, cfg->coef_B, f_sumsq, pl->d_mb_tokens, pl->d_mb_lmax, pl->d_mb_sample_off,
                                 pl->d_plan_len, pl->d_mb_cost, pl->d_scalars);
   k_row_offsets<<<1, scan_threads(n), 0, st>>>(pl->d_plan_len, n, pl->d_sample_row_off);
-  k_tiles<<<gb, 256, 0, st>>>(pl->d_sample_row_off, n, pl->d_tile_first_sample);
+  k_tiles<<<(unsigned)((n_tiles + 255) / 256), 256, 0, st>>>(pl->d_sample_row_off, n, n_tiles, pl->d_tile_first_sample);
   k_bucket<<<gb, 256, 0, st>>>(pl->d_mb_cost, K, (cfg->flags & FT_PLAN_AUTO_K) ? N : 0u, pl->d_scalars, pl->d_mb_bucket);
   k_sort_deal<<<gb, 256, 0, st>>>(pl->d_mb_cost, pl->d_mb_bucket, N, f_carry, pl->d_scalars, pl->d_mb_pos, pl->d_mb_rank);
   k_rank_index<<<gb, 256, 0, st>>>(pl->d_mb_pos, pl->d_mb_rank, pl->d_scalars, d_mb_idx, pl->d_rank_cnt);

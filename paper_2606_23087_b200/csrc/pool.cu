@@ -128,6 +128,8 @@ struct RegisterCall {
   const int32_t* ids;                                     // device, concatenated
   uint32_t* tp_off;                                       // [n+1] out: exclusive scan of text pages
   uint32_t* head;                                         // [1]   out: text ring head before the pops
+  uint32_t* pg_sample;                                    // [text pages of the call] out: call-local sample of each page
+  uint64_t* pg_dst;                                       // [text pages of the call] out: frame address of each page
   uint64_t call_seq;
 };
 
@@ -154,36 +156,39 @@ __global__ void __launch_bounds__(1024) k_register_scan(PoolView v, RegisterCall
     if (i < c.n) c.tp_off[i] = (uint32_t)(carry + ex);
     carry += total;
   }
+  __shared__ uint32_t sh_head;
   if (threadIdx.x == 0) {
     c.tp_off[c.n] = (uint32_t)carry;
     RingState s = *v.tring_state;
     c.head[0] = s.head;
+    sh_head = s.head;
     s.head = (uint32_t)((s.head + carry) % v.tring_cap);
     s.count -= (uint32_t)carry;
     *v.tring_state = s;
   }
-}
-
-// one block per (sample, text page): pops the page, stores up to 1024 ids, validates the runs
-__global__ void __launch_bounds__(256) k_register_ids(PoolView v, RegisterCall c) {
-  __shared__ uint32_t sh_i;
-  const uint32_t b = blockIdx.x;
-  if (threadIdx.x == 0) {
+  __syncthreads();
+  // every text page of the call: which sample it serves and where it lives, so that the copy of the ids (on the
+  // caller's stream, between its data kernels) starts from one small record instead of a search and three lookups
+  for (uint32_t b = threadIdx.x; b < (uint32_t)carry; b += blockDim.x) {
     uint32_t lo = 0, hi = c.n;  // largest i with tp_off[i] <= b
     while (hi - lo > 1) {
       uint32_t mid = (lo + hi) >> 1;
       if (c.tp_off[mid] <= b) lo = mid; else hi = mid;
     }
-    sh_i = lo;
+    const uint32_t tp = v.tring[(sh_head + b) % v.tring_cap];
+    const uint64_t tp_gva = v.text_gva_base + (uint64_t)tp * FT_TEXT_PAGE_BYTES;
+    v.s_text_pages[(uint64_t)c.slot[lo] * v.text_pages_per_sample + (b - c.tp_off[lo])] = tp_gva;
+    uint64_t off;
+    c.pg_sample[b] = lo;
+    c.pg_dst[b] = translate(v, tp_gva, &off) & ~kPteFlagMask;
   }
-  __syncthreads();
-  const uint32_t i = sh_i, k = b - c.tp_off[i], slot = c.slot[i];
-  const uint32_t tp = v.tring[(c.head[0] + b) % v.tring_cap];
-  const uint64_t tp_gva = v.text_gva_base + (uint64_t)tp * FT_TEXT_PAGE_BYTES;
-  if (threadIdx.x == 0) v.s_text_pages[(uint64_t)slot * v.text_pages_per_sample + k] = tp_gva;
-  uint64_t off;
-  const uint64_t pte = translate(v, tp_gva, &off);
-  int32_t* dst = reinterpret_cast<int32_t*>(pte & ~kPteFlagMask);
+}
+
+// one block per (sample, text page): stores up to 1024 ids, validates the runs
+__global__ void __launch_bounds__(256) k_register_ids(PoolView v, RegisterCall c) {
+  const uint32_t b = blockIdx.x;
+  const uint32_t i = c.pg_sample[b], k = b - c.tp_off[i], slot = c.slot[i];
+  int32_t* dst = reinterpret_cast<int32_t*>(c.pg_dst[b]);
   const uint32_t len = c.seq_len[i], p0 = k * kTextPageIds;
   const uint32_t cnt = min(kTextPageIds, len - p0);
   const uint32_t sb = c.span_begin[i], ns = c.n_spans[i];
@@ -887,7 +892,8 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_register_samples(
   const size_t o_pos = o_sb + (size_t)(n + 1) * 4, o_tok = o_pos + total_spans * 4;
   const size_t blob_bytes = align_up(o_tok + total_spans * 4, 256);
   const size_t o_tpoff = blob_bytes, o_head = align_up(o_tpoff + (size_t)(n + 1) * 4, 16);
-  const size_t total_bytes = o_head + 16;
+  const size_t o_pgdst = o_head + 16, o_pgs = o_pgdst + (size_t)text_need * 8;
+  const size_t total_bytes = o_pgs + (size_t)text_need * 4;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   ft_call_ctx* cx = nullptr;
   int32_t rc = ctx_acquire(p, 0, blob_bytes, total_bytes, &cx);
@@ -918,6 +924,8 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_register_samples(
   rcall.ids = input_ids;
   rcall.tp_off = reinterpret_cast<uint32_t*>(db + o_tpoff);
   rcall.head = reinterpret_cast<uint32_t*>(db + o_head);
+  rcall.pg_dst = reinterpret_cast<uint64_t*>(db + o_pgdst);
+  rcall.pg_sample = reinterpret_cast<uint32_t*>(db + o_pgs);
   rcall.call_seq = status_seq(p);
   // tables and the text-page pops on the metadata stream; the ids themselves (the caller's data) on the caller's
   k_register_scan<<<1, scan_threads(n), 0, p->meta>>>(p->view, rcall);

@@ -391,7 +391,8 @@ def test_planner_scale_matches_oracle():
     pool.destroy()
 
 
-@pytest.mark.parametrize("flags", [2, 4, 8, 16, 2 | 4 | 8 | 16])
+# (flag 1 = ALLOW_UNWRITTEN: such a plan carries no row words, so its assembly resolves every row the long way)
+@pytest.mark.parametrize("flags", [2, 4, 8, 16, 2 | 4 | 8 | 16, 1, 1 | 2])
 def test_plan_variants_match_oracle(flags):
     """Scheduler variants (longest-first packing, sum-of-squares cost, carried zig-zag): every plan array equals
     the oracle's, on 6000 descriptors (metadata only) and on a written batch whose gather follows the new order."""
