@@ -207,6 +207,136 @@ __global__ void __launch_bounds__(1024) k_bestfit(const uint32_t* __restrict__ l
   if (threadIdx.x == 0) scalars[SC_NMB] = n_mb;
 }
 
+// Online best fit with a whole warp, for plans with few microbatches.  The open microbatches' residuals and stamps
+// (the sample that changed them last) live in shared memory; every lane looks at a 32nd of them and three warp
+// reductions pick the smallest residual >= l, then the latest stamp among those (stamps are distinct, so exactly one
+// lane holds the winner).  A step of the chain costs a few hundred cycles instead of the thousand of the bitmap
+// descent with its per-residual stacks, and the kernel needs 16 bytes of shared memory per microbatch, so it also
+// fits on an SM whose shared-memory split was chosen for the copy kernels.  `cap` bounds the microbatch count: any-fit
+// packing leaves at most one microbatch half empty, so n_mb <= 2 sum(l) / L + 1.
+constexpr uint32_t kWarpFitChunk = 256;
+constexpr uint32_t kWarpFitMaxCap = 2048;
+__global__ void __launch_bounds__(256) k_bestfit_warp(const uint32_t* __restrict__ len, uint32_t n, uint32_t L, uint32_t cap,
+                                                      uint32_t* sample_mb, uint32_t* sample_rank, uint32_t* mb_residual,
+                                                      uint32_t* mb_tokens, uint32_t* mb_lmax, uint32_t* mb_count, uint32_t* scalars) {
+  extern __shared__ __align__(16) uint32_t sm[];
+  uint32_t *P = sm, *stamp = P + cap, *lmax = stamp + cap, *cnt = lmax + cap;
+  uint32_t *s_len = cnt + cap, *s_mb = s_len + kWarpFitChunk, *s_rank = s_mb + kWarpFitChunk;
+  __shared__ uint32_t s_nmb;
+  const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (threadIdx.x == 0) s_nmb = 0;
+  for (uint32_t base = 0; base < n; base += kWarpFitChunk) {
+    const uint32_t c = min(kWarpFitChunk, n - base);
+    for (uint32_t i = threadIdx.x; i < c; i += blockDim.x) s_len[i] = len[base + i];
+    __syncthreads();
+    if (warp == 0) {
+      uint32_t n_mb = s_nmb;
+      for (uint32_t i = 0; i < c; ++i) {
+        const uint32_t l = s_len[i];
+        uint32_t bp = 0xFFFFFFFFu, bs = 0, bj = 0;  // this lane's best: smallest residual >= l, then the latest stamp
+        for (uint32_t j = lane; j < n_mb; j += 32) {
+          const uint32_t p = P[j], st = stamp[j];
+          if (p >= l && (p < bp || (p == bp && st > bs))) { bp = p; bs = st; bj = j; }
+        }
+        const uint32_t mp = __reduce_min_sync(0xFFFFFFFFu, bp);
+        if (mp != 0xFFFFFFFFu) {
+          const uint32_t mine = bp == mp ? bs + 1 : 0;  // + 1: sample 0's stamp counts too
+          const uint32_t ms = __reduce_max_sync(0xFFFFFFFFu, mine);
+          const uint32_t who = __ffs(__ballot_sync(0xFFFFFFFFu, mine == ms)) - 1;
+          const uint32_t j = __shfl_sync(0xFFFFFFFFu, bj, who);
+          if (lane == 0) {
+            P[j] = mp - l; stamp[j] = base + i;
+            lmax[j] = max(lmax[j], l);
+            const uint32_t k = cnt[j];
+            cnt[j] = k + 1;
+            s_mb[i] = j; s_rank[i] = k;
+          }
+        } else {
+          const uint32_t j = n_mb;
+          if (lane == 0 && j < cap) { P[j] = L - l; stamp[j] = base + i; lmax[j] = l; cnt[j] = 1; }
+          if (lane == 0) { s_mb[i] = j; s_rank[i] = 0; }
+          if (j < cap) ++n_mb;  // (the bound guarantees it)
+        }
+        __syncwarp();
+      }
+      if (lane == 0) s_nmb = n_mb;
+    }
+    __syncthreads();
+    for (uint32_t i = threadIdx.x; i < c; i += blockDim.x) { sample_mb[base + i] = s_mb[i]; sample_rank[base + i] = s_rank[i]; }
+    __syncthreads();
+  }
+  const uint32_t n_mb = s_nmb;
+  for (uint32_t j = threadIdx.x; j < n_mb; j += blockDim.x) {
+    mb_residual[j] = P[j]; mb_tokens[j] = L - P[j]; mb_lmax[j] = lmax[j]; mb_count[j] = cnt[j];
+  }
+  if (threadIdx.x == 0) scalars[SC_NMB] = n_mb;
+}
+
+// The same with the open microbatches in registers, for plans of at most 32 R microbatches (microbatch j lives in
+// slot j / 32 of lane j % 32): a step of the chain is R comparisons per lane and two warp reductions, with no memory
+// access on the chain at all.
+template <int R>
+__global__ void __launch_bounds__(256) k_bestfit_regs(const uint32_t* __restrict__ len, uint32_t n, uint32_t L,
+                                                      uint32_t* sample_mb, uint32_t* sample_rank, uint32_t* mb_residual,
+                                                      uint32_t* mb_tokens, uint32_t* mb_lmax, uint32_t* mb_count, uint32_t* scalars) {
+  __shared__ uint32_t s_len[kWarpFitChunk], s_mb[kWarpFitChunk], s_rank[kWarpFitChunk];
+  const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t P[R], St[R], Lm[R], Cn[R];  // residual (0 = not open or full: never chosen, l >= 1), stamp, lmax, count
+#pragma unroll
+  for (int s = 0; s < R; ++s) { P[s] = 0; St[s] = 0; Lm[s] = 0; Cn[s] = 0; }
+  uint32_t n_mb = 0;
+  for (uint32_t base = 0; base < n; base += kWarpFitChunk) {
+    const uint32_t c = min(kWarpFitChunk, n - base);
+    for (uint32_t i = threadIdx.x; i < c; i += blockDim.x) s_len[i] = len[base + i];
+    __syncthreads();
+    if (warp == 0) {
+      for (uint32_t i = 0; i < c; ++i) {
+        const uint32_t l = s_len[i];
+        uint32_t bp = 0xFFFFFFFFu, bs = 0;
+        int bslot = 0;
+#pragma unroll
+        for (int s = 0; s < R; ++s) {
+          const bool better = P[s] >= l && (P[s] < bp || (P[s] == bp && St[s] > bs));
+          if (better) { bp = P[s]; bs = St[s]; bslot = s; }
+        }
+        const uint32_t mp = __reduce_min_sync(0xFFFFFFFFu, bp);
+        if (mp != 0xFFFFFFFFu) {
+          const uint32_t mine = bp == mp ? bs + 1 : 0;  // + 1: sample 0's stamp counts too
+          const uint32_t ms = __reduce_max_sync(0xFFFFFFFFu, mine);
+          if (mine == ms) {  // stamps are distinct: one lane
+            uint32_t k = 0;
+#pragma unroll
+            for (int s = 0; s < R; ++s)
+              if (s == bslot) { P[s] = mp - l; St[s] = base + i; Lm[s] = max(Lm[s], l); k = Cn[s]; Cn[s] = k + 1; }
+            s_mb[i] = lane + 32u * (uint32_t)bslot;
+            s_rank[i] = k;
+          }
+        } else {
+          if (lane == (n_mb & 31u)) {
+            const int slot = (int)(n_mb >> 5);
+#pragma unroll
+            for (int s = 0; s < R; ++s)
+              if (s == slot) { P[s] = L - l; St[s] = base + i; Lm[s] = l; Cn[s] = 1; }
+            s_mb[i] = n_mb; s_rank[i] = 0;
+          }
+          ++n_mb;
+        }
+      }
+    }
+    __syncthreads();
+    for (uint32_t i = threadIdx.x; i < c; i += blockDim.x) { sample_mb[base + i] = s_mb[i]; sample_rank[base + i] = s_rank[i]; }
+    __syncthreads();
+  }
+  if (warp == 0) {
+#pragma unroll
+    for (int s = 0; s < R; ++s) {
+      const uint32_t j = lane + 32u * (uint32_t)s;
+      if (j < n_mb) { mb_residual[j] = P[s]; mb_tokens[j] = L - P[s]; mb_lmax[j] = Lm[s]; mb_count[j] = Cn[s]; }
+    }
+    if (lane == 0) scalars[SC_NMB] = n_mb;
+  }
+}
+
 __global__ void __launch_bounds__(1024) k_mb_finalize(const uint32_t* mb_tokens, const uint32_t* mb_count,
                                                       uint32_t* mb_sample_off, uint64_t* mb_row_off, uint32_t* scalars) {
   __shared__ uint32_t s_max;
@@ -552,7 +682,19 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_plan_microbatches
   const uint32_t f_sort = (cfg->flags & FT_PLAN_SORT_DECREASING) != 0, f_sumsq = (cfg->flags & FT_PLAN_COST_SUMSQ) != 0;
   const uint32_t f_carry = (cfg->flags & FT_PLAN_ZIGZAG_CARRY) != 0;
   k_pack_order<<<gb, 256, 0, st>>>(pl->d_len, n, f_sort, d_pk_t, d_pk_len);
-  {
+  // few microbatches (n_mb <= 2 sum(l)/L + 1 for any-fit packing): the warp-wide kernel; else the bitmap descent
+  const uint64_t mb_bound = std::min<uint64_t>(n, 2 * total_tokens / L + 1);
+  if (mb_bound <= 128) {
+    k_bestfit_regs<4><<<1, 256, 0, st>>>(d_pk_len, n, L, d_pk_mb, pl->d_sample_rank, pl->d_mb_residual, pl->d_mb_tokens, pl->d_mb_lmax,
+                                         pl->d_mb_count, pl->d_scalars);
+  } else if (mb_bound <= 256) {
+    k_bestfit_regs<8><<<1, 256, 0, st>>>(d_pk_len, n, L, d_pk_mb, pl->d_sample_rank, pl->d_mb_residual, pl->d_mb_tokens, pl->d_mb_lmax,
+                                         pl->d_mb_count, pl->d_scalars);
+  } else if (mb_bound <= kWarpFitMaxCap) {
+    const uint32_t cap = (uint32_t)align_up((size_t)mb_bound, 64);
+    k_bestfit_warp<<<1, 256, ((size_t)4 * cap + 3 * kWarpFitChunk) * 4, st>>>(d_pk_len, n, L, cap, d_pk_mb, pl->d_sample_rank, pl->d_mb_residual,
+                                                                          pl->d_mb_tokens, pl->d_mb_lmax, pl->d_mb_count, pl->d_scalars);
+  } else {
     const bool all_recs = rec_cap >= n;
     auto fit = head_in_smem ? (all_recs ? k_bestfit<true, true> : k_bestfit<true, false>)
                             : (all_recs ? k_bestfit<false, true> : k_bestfit<false, false>);

@@ -391,6 +391,37 @@ def test_planner_scale_matches_oracle():
     pool.destroy()
 
 
+@pytest.mark.parametrize("n", [150, 300, 2000, 6000])
+def test_best_fit_ties_match_oracle_in_every_packing_kernel(n):
+    """Lengths from a handful of values, budget 1000: equal residuals all the time, so the tie-break (the microbatch
+    changed most recently) decides most placements.  The sample counts put the bound on the microbatch count
+    (2 sum(l)/L + 1) into the range of each of the four packing kernels: registers (up to 128 and up to 256 microbatches),
+    shared-memory scan (up to 2048), bitmap descent with per-residual stacks (beyond)."""
+    gh = _gpu()
+    from paper_2606_23087_b200 import binding as fp
+    rng = np.random.default_rng(n)
+    seq_len = rng.choice(np.array([100, 200, 250, 300, 400, 500], dtype=np.uint32), size=n).astype(np.uint32)
+    pool = fp.Pool(fp.PoolConfig(page_bytes=4096, hbm_pages=16, host_pages=0, hidden=64, max_samples=n, max_spans_per_sample=1,
+                                 max_pages_per_span=1, max_seq_len=1000, max_text_tokens=1024 * n, placeholder_id=7, world_size=1))
+    assert pool.rc == 0
+    d_ids = torch.zeros(int(seq_len.sum()), dtype=torch.int32, device="cuda")
+    z = np.zeros(0, np.uint32)
+    assert pool.register_samples(list(range(n)), seq_len, np.zeros(n, np.uint32), z, z, d_ids.data_ptr(), gh.cuda_stream()) == 0
+    order = [int(x) for x in rng.permutation(n)]
+    for flags in (0, 2):
+        cfg = dict(coef_A=1000, coef_B=1, budget_L=1000, n_buckets_K=4, n_ranks_N=8, flags=flags)
+        rc, gp = pool.plan_microbatches(order, fp.PlanConfig(**cfg), gh.cuda_stream())
+        rc2, op = plan_from_lengths(seq_len[order], PlanConfig(**cfg), slots=order)
+        assert rc == rc2 == 0
+        ga, oa = gp.arrays(), op.arrays()
+        assert ga["n_mb"] == oa["n_mb"]
+        for k in PLAN_KEYS:
+            assert np.array_equal(ga[k], oa[k]), (k, n, flags)
+        gp.destroy(); op.destroy()
+    assert pool.status() == (0, 0)
+    pool.destroy()
+
+
 # (flag 1 = ALLOW_UNWRITTEN: such a plan carries no row words, so its assembly resolves every row the long way)
 @pytest.mark.parametrize("flags", [2, 4, 8, 16, 2 | 4 | 8 | 16, 1, 1 | 2])
 def test_plan_variants_match_oracle(flags):
@@ -410,7 +441,7 @@ def test_plan_variants_match_oracle(flags):
     d_ids = torch.from_numpy(ids).cuda()
     assert pool.register_samples(list(range(w.n_samples)), seq_len, n_spans, w.span_pos, w.span_tokens, d_ids.data_ptr(), gh.cuda_stream()) == 0
     order = [int(x) for x in np.random.default_rng(flags).permutation(w.n_samples)]
-    for K, N, L in ((4, 8, 32768), (1, 3, 18000), (7, 5, 131072)):
+    for K, N, L in ((4, 8, 32768), (1, 3, 18000), (7, 5, 131072), (3, 4, 65536)):   # (each budget takes another packing kernel)
         cfg = dict(coef_A=L, coef_B=1, budget_L=L, n_buckets_K=K, n_ranks_N=N, flags=flags | 1)
         rc, gp = pool.plan_microbatches(order, fp.PlanConfig(**cfg), gh.cuda_stream())
         rc2, op = plan_from_lengths(seq_len[order], PlanConfig(**cfg), slots=order)
