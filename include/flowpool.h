@@ -474,7 +474,10 @@ int32_t pool_profile_read(ft_pool* pool, ft_kernel_time* out /* host [FT_K_COUNT
  *   dev_ctas_per_sm      resident CTAs per SM of the HBM-tier gather kernel (default 4; 1..8)
  *   scatter_ctas_per_sm  resident CTAs per SM of the HBM-tier scatter kernel (default 4; 1..8)
  *   scatter_group        chunks a scatter CTA claims at a time (default 1)
- *   chunk_shift          log2 of the scatter's work unit in bytes of a span's image (default 16; 14..21)
+ *   chunk_shift          log2 of the scatter's work unit in bytes of a span's image (14..21).  Default 0 = chosen per
+ *                        call: 16 KiB chunks while the call has at most 2^17 of them, else 32 KiB, else 64 KiB (small
+ *                        chunks shorten the last wave of a launch; each chunk has a 24-byte record in the call's
+ *                        scratch where pages are at least a chunk long)
  *   host_ctas            grid of the host-tier bulk-copy kernels (default 6): few SMs, so that long-latency host-link
  *                        accesses do not clog the memory pipelines of the SMs that stream HBM
  *   host_store_ctas      grid of the vector-store scatter into host frames (fp32 sources, host-only pools; default 8)

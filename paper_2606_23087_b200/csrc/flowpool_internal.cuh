@@ -344,7 +344,7 @@ struct ft_pool {
                                 // 770 GB/s x a few microseconds of NVLink latency wants 1.5 MB and more in flight)
   int peers_remote = 0;         // 1: flag every imported peer's HBM frames as remote, whatever device they are on
   int host_store_ctas = 8;      // grid of the vector-store scatter into host frames (fp32 sources, host-only pools)
-  int chunk_shift = 16;         // log2 of k_scatter's work unit in bytes of a span's image (14..21)
+  int chunk_shift = 0;          // log2 of k_scatter's work unit in bytes of a span's image (14..21); 0 = chosen per call
   int scatter_group = 0;        // chunks per round-robin group of k_scatter; 0 = the measured default
   int scatter_ctas_per_sm = 0;  // resident CTAs per SM of the device-tier scatter kernel; 0 = the measured default
   bool grad_attr_set = false;   // k_embed_grad_hot's shared-memory opt-in done

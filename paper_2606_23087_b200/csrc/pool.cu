@@ -212,6 +212,14 @@ __global__ void __launch_bounds__(256) k_register_ids(PoolView v, RegisterCall c
 // ------------------------------------------------------------------------------------------
 // K3: page allocation
 // ------------------------------------------------------------------------------------------
+// A scatter work unit resolved ahead of the copy (chunks never straddle a page when the page is at least a chunk).
+struct ChunkDesc {
+  uint64_t src;       // the span's source
+  uint64_t dst;       // frame address + offset of the chunk inside its page | page-table flags (low 4 bits)
+  uint32_t ch_local;  // index of the chunk inside the span's image
+  uint32_t len;       // bytes of the image in this chunk
+};
+
 struct WriteCall {
   uint32_t n;
   const uint64_t* src;       // [n] device pointers
@@ -221,6 +229,7 @@ struct WriteCall {
   uint32_t* blk_off;         // [n+1] out
   uint64_t* chunk_off;       // [n+1] out
   uint32_t* chunk_span;      // [total chunks] out: call-local span index of each chunk; NULL = search chunk_off
+  struct ChunkDesc* chunk_desc;  // [total chunks] out: where each chunk comes from and goes to (pages >= chunk), or NULL
   uint32_t* heads;           // [2]   out: page ring head, block ring head before the pops
   uint32_t chunk_shift;      // scatter work unit = 2^chunk_shift bytes of a span's image
 };
@@ -267,6 +276,19 @@ __global__ void __launch_bounds__(256) k_alloc_fill(PoolView v, WriteCall c, uin
       if (c.chunk_off[mid] <= tc) lo = mid; else hi = mid;
     }
     c.chunk_span[tc] = lo;
+    if (c.chunk_desc) {
+      const uint32_t ch_local = (uint32_t)(tc - c.chunk_off[lo]);
+      const uint64_t B0 = (uint64_t)ch_local << c.chunk_shift, bytes_q = (uint64_t)c.n_tokens[lo] * v.row_bytes;
+      const uint32_t g = v.ring[(c.heads[0] + c.page_off[lo] + (uint32_t)(B0 >> v.page_shift)) % v.ring_cap];
+      uint64_t off;
+      const uint64_t pte = translate(v, page_gva(v, g), &off);
+      ChunkDesc d;
+      d.src = c.src[lo];
+      d.dst = ((pte & ~kPteFlagMask) + (B0 & (v.page_bytes - 1))) | (pte & kPteFlagMask);
+      d.ch_local = ch_local;
+      d.len = (uint32_t)min((uint64_t)1 << c.chunk_shift, bytes_q - B0);
+      c.chunk_desc[tc] = d;
+    }
   }
   if (tc >= total_pages) return;
   const uint32_t t = (uint32_t)tc;
@@ -296,7 +318,37 @@ __device__ __forceinline__ uint32_t pack2(uint32_t a, uint32_t b) { return rne_b
 
 enum { kTierAll = 0, kTierDeviceOnly = 1, kTierHostOnly = 2 };
 
-template <int MODE, bool F32>
+// One warp moves up to 2 KiB of a span's image (nv 16-byte vectors, <= 128) from byte offset B of the source image
+// (an fp32 source holds two vectors per bf16 vector) to d: four 512-byte lines per lane in flight.
+template <bool F32>
+__device__ __forceinline__ void copy_batch(const uint8_t* src_q, uint64_t B, uint4* d, uint32_t nv, uint32_t lane) {
+  const bool t0 = lane < nv, t1 = lane + 32 < nv, t2 = lane + 64 < nv, t3 = lane + 96 < nv;
+  if (!F32) {
+    const uint4* s = reinterpret_cast<const uint4*>(src_q + B);
+    uint4 a0, a1, a2, a3;
+    if (t0) a0 = __ldcs(s + lane);
+    if (t1) a1 = __ldcs(s + lane + 32);
+    if (t2) a2 = __ldcs(s + lane + 64);
+    if (t3) a3 = __ldcs(s + lane + 96);
+    if (t0) __stcs(d + lane, a0);
+    if (t1) __stcs(d + lane + 32, a1);
+    if (t2) __stcs(d + lane + 64, a2);
+    if (t3) __stcs(d + lane + 96, a3);
+  } else {
+    const uint4* s = reinterpret_cast<const uint4*>(src_q + 2 * B);  // two fp32 vectors per bf16 vector
+    uint4 a0, a1, a2, a3, e0, e1, e2, e3;
+    if (t0) { a0 = __ldcs(s + 2 * lane); e0 = __ldcs(s + 2 * lane + 1); }
+    if (t1) { a1 = __ldcs(s + 2 * (lane + 32)); e1 = __ldcs(s + 2 * (lane + 32) + 1); }
+    if (t2) { a2 = __ldcs(s + 2 * (lane + 64)); e2 = __ldcs(s + 2 * (lane + 64) + 1); }
+    if (t3) { a3 = __ldcs(s + 2 * (lane + 96)); e3 = __ldcs(s + 2 * (lane + 96) + 1); }
+    if (t0) __stcs(d + lane, make_uint4(pack2(a0.x, a0.y), pack2(a0.z, a0.w), pack2(e0.x, e0.y), pack2(e0.z, e0.w)));
+    if (t1) __stcs(d + lane + 32, make_uint4(pack2(a1.x, a1.y), pack2(a1.z, a1.w), pack2(e1.x, e1.y), pack2(e1.z, e1.w)));
+    if (t2) __stcs(d + lane + 64, make_uint4(pack2(a2.x, a2.y), pack2(a2.z, a2.w), pack2(e2.x, e2.y), pack2(e2.z, e2.w)));
+    if (t3) __stcs(d + lane + 96, make_uint4(pack2(a3.x, a3.y), pack2(a3.z, a3.w), pack2(e3.x, e3.y), pack2(e3.z, e3.w)));
+  }
+}
+
+template <int MODE, bool F32, bool DESC>
 __global__ void __launch_bounds__(256, F32 ? 4 : 6) k_scatter(PoolView v, WriteCall c, uint64_t total_chunks, uint64_t per_cta,
                                                               ClaimCounter* group_counter) {
   // Work unit = a chunk of 2^chunk_shift bytes of one span's image (the page size does not cap it).  Groups of
@@ -308,17 +360,39 @@ __global__ void __launch_bounds__(256, F32 ? 4 : 6) k_scatter(PoolView v, WriteC
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const uint64_t CH = 1ull << c.chunk_shift;
   const uint32_t region = (uint32_t)(CH >> 3);  // bytes per warp and chunk
-  __shared__ uint64_t next_group;
-  for (;;) {
-    __syncthreads();  // everyone has read the previous claim
-    if (threadIdx.x == 0) next_group = atomicAdd(&group_counter->claim, 1ull);
-    __syncthreads();
-    const uint64_t c0 = next_group * per_cta;
+  // A CTA's first group is its block index; every later one comes from the counter, claimed while the current group
+  // is being copied (the answer is needed only when the group is done).
+  __shared__ uint64_t next_group[2];
+  uint64_t grp = blockIdx.x;
+  for (uint32_t it = 0;; ++it) {
+    const uint64_t c0 = grp * per_cta;
     if (c0 >= total_chunks) {
       if (threadIdx.x == 0) claim_release(group_counter);
       break;
     }
+    unsigned long long nxt = 0;
+    if (DESC && threadIdx.x == 0) nxt = gridDim.x + atomicAdd(&group_counter->claim, 1ull);
     const uint64_t c1 = min(total_chunks, c0 + per_cta);
+    if (DESC) {
+      // resolved chunks: one record, then the bytes
+      for (uint64_t ch = c0; ch < c1; ++ch) {
+        const ChunkDesc d = c.chunk_desc[ch];
+        const bool host = (d.dst & kPteHost) != 0;
+        if ((MODE == kTierDeviceOnly && host) || (MODE == kTierHostOnly && !host)) continue;
+        const uint64_t B0 = (uint64_t)d.ch_local << c.chunk_shift;
+        const uint8_t* src_q = reinterpret_cast<const uint8_t*>(d.src);
+        uint8_t* dst0 = reinterpret_cast<uint8_t*>(d.dst & ~kPteFlagMask);
+        for (uint32_t b = 0; b < region; b += 2048) {
+          const uint32_t Bl = warp * region + b;  // offset inside the chunk
+          if (Bl >= d.len) break;
+          copy_batch<F32>(src_q, B0 + Bl, reinterpret_cast<uint4*>(dst0 + Bl), (min(2048u, d.len - Bl)) >> 4, lane);
+        }
+      }
+      if (threadIdx.x == 0) next_group[it & 1] = nxt;
+      __syncthreads();
+      grp = next_group[it & 1];
+      continue;
+    }
     uint32_t q;
     if (c.chunk_span) {
       q = c.chunk_span[c0];
@@ -358,33 +432,13 @@ __global__ void __launch_bounds__(256, F32 ? 4 : 6) k_scatter(PoolView v, WriteC
         const bool host = (pte & kPteHost) != 0;
         if ((MODE == kTierDeviceOnly && host) || (MODE == kTierHostOnly && !host)) continue;
         uint4* d = reinterpret_cast<uint4*>((pte & ~kPteFlagMask) + (B & (v.page_bytes - 1)));
-        const uint32_t nv = (uint32_t)(min((uint64_t)2048, bytes_q - B) >> 4);  // vectors in this batch (<= 128)
-        const bool t0 = lane < nv, t1 = lane + 32 < nv, t2 = lane + 64 < nv, t3 = lane + 96 < nv;
-        if (!F32) {
-          const uint4* s = reinterpret_cast<const uint4*>(src_q + B);
-          uint4 a0, a1, a2, a3;
-          if (t0) a0 = __ldcs(s + lane);
-          if (t1) a1 = __ldcs(s + lane + 32);
-          if (t2) a2 = __ldcs(s + lane + 64);
-          if (t3) a3 = __ldcs(s + lane + 96);
-          if (t0) __stcs(d + lane, a0);
-          if (t1) __stcs(d + lane + 32, a1);
-          if (t2) __stcs(d + lane + 64, a2);
-          if (t3) __stcs(d + lane + 96, a3);
-        } else {
-          const uint4* s = reinterpret_cast<const uint4*>(src_q + 2 * B);  // two fp32 vectors per bf16 vector
-          uint4 a0, a1, a2, a3, e0, e1, e2, e3;
-          if (t0) { a0 = __ldcs(s + 2 * lane); e0 = __ldcs(s + 2 * lane + 1); }
-          if (t1) { a1 = __ldcs(s + 2 * (lane + 32)); e1 = __ldcs(s + 2 * (lane + 32) + 1); }
-          if (t2) { a2 = __ldcs(s + 2 * (lane + 64)); e2 = __ldcs(s + 2 * (lane + 64) + 1); }
-          if (t3) { a3 = __ldcs(s + 2 * (lane + 96)); e3 = __ldcs(s + 2 * (lane + 96) + 1); }
-          if (t0) __stcs(d + lane, make_uint4(pack2(a0.x, a0.y), pack2(a0.z, a0.w), pack2(e0.x, e0.y), pack2(e0.z, e0.w)));
-          if (t1) __stcs(d + lane + 32, make_uint4(pack2(a1.x, a1.y), pack2(a1.z, a1.w), pack2(e1.x, e1.y), pack2(e1.z, e1.w)));
-          if (t2) __stcs(d + lane + 64, make_uint4(pack2(a2.x, a2.y), pack2(a2.z, a2.w), pack2(e2.x, e2.y), pack2(e2.z, e2.w)));
-          if (t3) __stcs(d + lane + 96, make_uint4(pack2(a3.x, a3.y), pack2(a3.z, a3.w), pack2(e3.x, e3.y), pack2(e3.z, e3.w)));
-        }
+        copy_batch<F32>(src_q, B, d, (uint32_t)(min((uint64_t)2048, bytes_q - B) >> 4), lane);
       }
     }
+    if (threadIdx.x == 0) nxt = gridDim.x + atomicAdd(&group_counter->claim, 1ull);
+    if (threadIdx.x == 0) next_group[it & 1] = nxt;
+    __syncthreads();
+    grp = next_group[it & 1];
   }
 }
 
@@ -403,7 +457,8 @@ static void launch_scatter(ft_pool* p, const WriteCall& w, uint64_t total_chunks
   uint64_t grid = std::min<uint64_t>(max_ctas, (uint64_t)p->sm_count * std::min(per_sm, want));
   const uint64_t per = p->scatter_group > 0 ? (uint64_t)p->scatter_group : 1;
   grid = std::max<uint64_t>(1, std::min<uint64_t>(grid, (total_chunks + per - 1) / per));
-  k_scatter<MODE, F32><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per, counter);
+  if (w.chunk_desc) k_scatter<MODE, F32, true><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per, counter);
+  else k_scatter<MODE, F32, false><<<(unsigned)grid, 256, 0, s>>>(p->view, w, total_chunks, per, counter);
 }
 
 static void launch_scatter_any(ft_pool* p, int mode, bool f32, const WriteCall& w, uint64_t total_chunks, uint64_t max_ctas,
@@ -453,12 +508,18 @@ __global__ void __launch_bounds__(32) k_scatter_host_bulk(PoolView v, WriteCall 
 }
 
 int32_t scatter_set_carveout(int pct) {
-  FT_CUDA(cudaFuncSetAttribute(k_scatter<kTierAll, false>, cudaFuncAttributePreferredSharedMemoryCarveout, pct));
-  FT_CUDA(cudaFuncSetAttribute(k_scatter<kTierAll, true>, cudaFuncAttributePreferredSharedMemoryCarveout, pct));
-  FT_CUDA(cudaFuncSetAttribute(k_scatter<kTierDeviceOnly, false>, cudaFuncAttributePreferredSharedMemoryCarveout, pct));
-  FT_CUDA(cudaFuncSetAttribute(k_scatter<kTierDeviceOnly, true>, cudaFuncAttributePreferredSharedMemoryCarveout, pct));
-  FT_CUDA(cudaFuncSetAttribute(k_scatter<kTierHostOnly, false>, cudaFuncAttributePreferredSharedMemoryCarveout, pct));
-  FT_CUDA(cudaFuncSetAttribute(k_scatter<kTierHostOnly, true>, cudaFuncAttributePreferredSharedMemoryCarveout, pct));
+  FT_CUDA(cudaFuncSetAttribute(k_scatter<kTierAll, false, false>, cudaFuncAttributePreferredSharedMemoryCarveout, pct));
+  FT_CUDA(cudaFuncSetAttribute(k_scatter<kTierAll, false, true>, cudaFuncAttributePreferredSharedMemoryCarveout, pct));
+  FT_CUDA(cudaFuncSetAttribute(k_scatter<kTierAll, true, false>, cudaFuncAttributePreferredSharedMemoryCarveout, pct));
+  FT_CUDA(cudaFuncSetAttribute(k_scatter<kTierAll, true, true>, cudaFuncAttributePreferredSharedMemoryCarveout, pct));
+  FT_CUDA(cudaFuncSetAttribute(k_scatter<kTierDeviceOnly, false, false>, cudaFuncAttributePreferredSharedMemoryCarveout, pct));
+  FT_CUDA(cudaFuncSetAttribute(k_scatter<kTierDeviceOnly, false, true>, cudaFuncAttributePreferredSharedMemoryCarveout, pct));
+  FT_CUDA(cudaFuncSetAttribute(k_scatter<kTierDeviceOnly, true, false>, cudaFuncAttributePreferredSharedMemoryCarveout, pct));
+  FT_CUDA(cudaFuncSetAttribute(k_scatter<kTierDeviceOnly, true, true>, cudaFuncAttributePreferredSharedMemoryCarveout, pct));
+  FT_CUDA(cudaFuncSetAttribute(k_scatter<kTierHostOnly, false, false>, cudaFuncAttributePreferredSharedMemoryCarveout, pct));
+  FT_CUDA(cudaFuncSetAttribute(k_scatter<kTierHostOnly, false, true>, cudaFuncAttributePreferredSharedMemoryCarveout, pct));
+  FT_CUDA(cudaFuncSetAttribute(k_scatter<kTierHostOnly, true, false>, cudaFuncAttributePreferredSharedMemoryCarveout, pct));
+  FT_CUDA(cudaFuncSetAttribute(k_scatter<kTierHostOnly, true, true>, cudaFuncAttributePreferredSharedMemoryCarveout, pct));
   return FT_OK;
 }
 
@@ -719,9 +780,9 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_create(const ft_p
   CK(cudaFuncSetAttribute(k_scatter_host_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBulkSmemBytes));
   {
     auto occ = [](auto kernel) { int v = 0; return cudaOccupancyMaxActiveBlocksPerMultiprocessor(&v, kernel, 256, 0) == cudaSuccess && v > 0 ? v : 1; };
-    p->occ_scatter[kTierAll][0] = occ(k_scatter<kTierAll, false>); p->occ_scatter[kTierAll][1] = occ(k_scatter<kTierAll, true>);
-    p->occ_scatter[kTierDeviceOnly][0] = occ(k_scatter<kTierDeviceOnly, false>); p->occ_scatter[kTierDeviceOnly][1] = occ(k_scatter<kTierDeviceOnly, true>);
-    p->occ_scatter[kTierHostOnly][0] = occ(k_scatter<kTierHostOnly, false>); p->occ_scatter[kTierHostOnly][1] = occ(k_scatter<kTierHostOnly, true>);
+    p->occ_scatter[kTierAll][0] = std::min(occ(k_scatter<kTierAll, false, false>), occ(k_scatter<kTierAll, false, true>)); p->occ_scatter[kTierAll][1] = std::min(occ(k_scatter<kTierAll, true, false>), occ(k_scatter<kTierAll, true, true>));
+    p->occ_scatter[kTierDeviceOnly][0] = std::min(occ(k_scatter<kTierDeviceOnly, false, false>), occ(k_scatter<kTierDeviceOnly, false, true>)); p->occ_scatter[kTierDeviceOnly][1] = std::min(occ(k_scatter<kTierDeviceOnly, true, false>), occ(k_scatter<kTierDeviceOnly, true, true>));
+    p->occ_scatter[kTierHostOnly][0] = std::min(occ(k_scatter<kTierHostOnly, false, false>), occ(k_scatter<kTierHostOnly, false, true>)); p->occ_scatter[kTierHostOnly][1] = std::min(occ(k_scatter<kTierHostOnly, true, false>), occ(k_scatter<kTierHostOnly, true, true>));
   }
   // the scatter kernel's shared-memory split (see ft_tuning.scatter_smem_carveout): small but stated, so that metadata
   // kernels and the packing kernel can start on SMs that hold its CTAs
@@ -961,12 +1022,23 @@ namespace ft {
 // the call's totals are in `t` and, when `b_*` are given, the descriptors in the caller's staging arrays.
 struct WriteTotals {
   uint64_t need = 0, need_blocks = 0, total_chunks = 0, bytes_total = 0;
+  uint32_t chunk_shift = 16;  // the copy's work unit for this call
 };
+// The copy's work unit when the tuning leaves it open: the smaller the chunk, the shorter the kernel's last wave (a
+// producer call of 0.7 GB streams at 6.3 TB/s with 64 KiB chunks and at 6.5 TB/s with 16 KiB chunks), as long as the
+// per-chunk records stay a small table; `fine` = the caller can hold such records.
+static uint32_t auto_chunk_shift(const uint64_t chunks_at[3], bool fine) {
+  if (fine)
+    for (int i = 0; i < 2; ++i)
+      if (chunks_at[i] <= (1u << 17)) return 14 + i;
+  return 16;
+}
 static int32_t check_write(ft_pool* p, uint32_t n, const uint32_t* slot, const uint32_t* span_idx, const uint32_t* n_tokens,
-                           const void* const* src, WriteTotals* t) {
+                           const void* const* src, WriteTotals* t, bool fine_chunks) {
   const ft_pool_config& c = p->cfg;
   const uint32_t S = c.max_spans_per_sample;
-  const uint32_t chunk_shift = (uint32_t)p->chunk_shift;
+  uint64_t chunks_at[3] = {0, 0, 0};  // with 16, 32 and 64 KiB chunks
+  uint64_t chunks_fixed = 0;
   for (uint32_t q = 0; q < n; ++q) {
     if (slot[q] >= c.max_samples) return FT_ERR_INVALID_ARG;
     const ft_slot_mirror& s = p->slots[slot[q]];
@@ -980,8 +1052,15 @@ static int32_t check_write(ft_pool* p, uint32_t n, const uint32_t* slot, const u
     const uint64_t k = pages_for_tokens(p, n_tokens[q]);
     t->need += k; t->need_blocks += (k + kListBlock - 1) / kListBlock;
     const uint64_t bytes = (uint64_t)n_tokens[q] * p->view.row_bytes;
-    t->total_chunks += (bytes + (1ull << chunk_shift) - 1) >> chunk_shift;
+    for (int i = 0; i < 3; ++i) chunks_at[i] += (bytes + (1ull << (14 + i)) - 1) >> (14 + i);
+    if (p->chunk_shift) chunks_fixed += (bytes + (1ull << p->chunk_shift) - 1) >> p->chunk_shift;
     t->bytes_total += bytes;
+  }
+  if (p->chunk_shift) {
+    t->chunk_shift = (uint32_t)p->chunk_shift; t->total_chunks = chunks_fixed;
+  } else {
+    t->chunk_shift = auto_chunk_shift(chunks_at, fine_chunks && c.page_bytes >= (1u << 14));
+    t->total_chunks = chunks_at[t->chunk_shift - 14];
   }
   if (t->need > p->free_pages) return FT_ERR_POOL_EXHAUSTED;
   if (t->need_blocks > p->free_blocks) return FT_ERR_CAPACITY;
@@ -1013,7 +1092,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings(
   if (!slot || !span_idx || !n_tokens || !src) return FT_ERR_INVALID_ARG;
   const uint32_t S = p->cfg.max_spans_per_sample;
   WriteTotals t;
-  int32_t rc = check_write(p, n, slot, span_idx, n_tokens, src, &t);
+  int32_t rc = check_write(p, n, slot, span_idx, n_tokens, src, &t, true);
   if (rc != FT_OK) return rc;
   const uint64_t need = t.need, total_chunks = t.total_chunks;
 
@@ -1023,7 +1102,10 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings(
   const size_t o_choff = blob_bytes, o_poff = align_up(o_choff + (size_t)(n + 1) * 8, 16);
   const size_t o_boff = o_poff + (size_t)(n + 1) * 4, o_heads = align_up(o_boff + (size_t)(n + 1) * 4, 16);
   const size_t o_cspan = o_heads + 16;
-  const size_t total_bytes = o_cspan + total_chunks * 4;
+  // chunk records for the copy kernel where a chunk cannot straddle a page (pages at least a chunk long)
+  const bool with_desc = p->cfg.page_bytes >= (1ull << t.chunk_shift);
+  const size_t o_cdesc = align_up(o_cspan + total_chunks * 4, 16);
+  const size_t total_bytes = o_cdesc + (with_desc ? total_chunks * sizeof(ChunkDesc) : 0);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   ft_call_ctx* cx = nullptr;
   if ((rc = ctx_acquire(p, 0, blob_bytes, total_bytes, &cx)) != FT_OK) return rc;
@@ -1045,7 +1127,8 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings(
   w.blk_off = reinterpret_cast<uint32_t*>(db + o_boff);
   w.heads = reinterpret_cast<uint32_t*>(db + o_heads);
   w.chunk_span = reinterpret_cast<uint32_t*>(db + o_cspan);
-  w.chunk_shift = (uint32_t)p->chunk_shift;
+  w.chunk_desc = with_desc ? reinterpret_cast<ChunkDesc*>(db + o_cdesc) : nullptr;
+  w.chunk_shift = t.chunk_shift;
   // page allocation on the metadata stream (it overlaps the copy of the call before), the copy on the caller's
   k_alloc_scan<<<1, scan_threads(n), 0, p->meta>>>(p->view, w);
   k_alloc_fill<<<(unsigned)((std::max<uint64_t>(need, total_chunks) + 255) / 256), 256, 0, p->meta>>>(p->view, w, (uint32_t)need, total_chunks);
@@ -1234,7 +1317,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_set_tuning(ft_poo
   p->dev_ctas_per_sm = t.dev_ctas_per_sm ? (int)t.dev_ctas_per_sm : 4;
   p->scatter_ctas_per_sm = (int)t.scatter_ctas_per_sm;
   p->scatter_group = (int)t.scatter_group;
-  p->chunk_shift = t.chunk_shift ? (int)t.chunk_shift : 16;
+  p->chunk_shift = (int)t.chunk_shift;
   p->host_ctas = t.host_ctas ? (int)t.host_ctas : 6;
   p->host_store_ctas = t.host_store_ctas ? (int)t.host_store_ctas : 8;
   p->gather_unroll = t.gather_unroll ? (int)t.gather_unroll : 4;
@@ -1381,7 +1464,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings_
   if (cur != p->device) return FT_ERR_INVALID_ARG;
   const uint32_t S = p->cfg.max_spans_per_sample;
   WriteTotals t;
-  int32_t rc = check_write(p, n, slot, span_idx, n_tokens, src, &t);
+  int32_t rc = check_write(p, n, slot, span_idx, n_tokens, src, &t, false);  // (no room for per-chunk records here)
   if (rc != FT_OK) return rc;
 
   // descriptor blob [src u64 n][span_id n][n_tokens n] in the host buffer pool_create made for this purpose
@@ -1414,8 +1497,9 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings_
   w.page_off = reinterpret_cast<uint32_t*>(db + o_poff);
   w.blk_off = reinterpret_cast<uint32_t*>(db + o_boff);
   w.heads = reinterpret_cast<uint32_t*>(db + o_heads);
-  w.chunk_span = nullptr;  // the fixed scratch has no room for a per-chunk table: k_scatter searches chunk_off
-  w.chunk_shift = (uint32_t)p->chunk_shift;
+  w.chunk_span = nullptr;  // the fixed scratch has no room for per-chunk tables: k_scatter searches chunk_off
+  w.chunk_desc = nullptr;
+  w.chunk_shift = t.chunk_shift;
   k_alloc_scan<<<1, scan_threads(n), 0, p->meta>>>(p->view, w);
   k_alloc_fill<<<(unsigned)((t.need + 255) / 256), 256, 0, p->meta>>>(p->view, w, (uint32_t)t.need, 0);
   p->gpu_launches += 2;

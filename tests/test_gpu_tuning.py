@@ -48,7 +48,7 @@ def test_tuning_round_trip_and_range_checks():
     pool = fp.Pool(fp.PoolConfig(**pool_config_fields(w)))
     assert pool.rc == 0
     d = pool.get_tuning()
-    assert (d["dev_ctas_per_sm"], d["scatter_ctas_per_sm"], d["chunk_shift"], d["host_ctas"], d["gather_unroll"]) == (4, 4, 16, 6, 4)
+    assert (d["dev_ctas_per_sm"], d["scatter_ctas_per_sm"], d["chunk_shift"], d["host_ctas"], d["gather_unroll"]) == (4, 4, 0, 6, 4)   # chunk_shift 0: chosen per call
     assert d["scatter_smem_carveout"] == 5 and d["gather_smem_carveout"] == 0 and d["remote_ctas"] == 16
     for bad in (dict(chunk_shift=13), dict(chunk_shift=22), dict(gather_unroll=6), dict(dev_ctas_per_sm=9), dict(peers_remote=2),
                 dict(scatter_smem_carveout=101)):
