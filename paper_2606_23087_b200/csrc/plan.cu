@@ -207,20 +207,37 @@ __global__ void __launch_bounds__(1024) k_bestfit(const uint32_t* __restrict__ l
   if (threadIdx.x == 0) scalars[SC_NMB] = n_mb;
 }
 
-// Online best fit with a whole warp, for plans with few microbatches.  The open microbatches' residuals and stamps
-// (the sample that changed them last) live in shared memory; every lane looks at a 32nd of them and three warp
-// reductions pick the smallest residual >= l, then the latest stamp among those (stamps are distinct, so exactly one
-// lane holds the winner).  A step of the chain costs a few hundred cycles instead of the thousand of the bitmap
-// descent with its per-residual stacks, and the kernel needs 16 bytes of shared memory per microbatch, so it also
-// fits on an SM whose shared-memory split was chosen for the copy kernels.  `cap` bounds the microbatch count: any-fit
-// packing leaves at most one microbatch half empty, so n_mb <= 2 sum(l) / L + 1.
+// Online best fit with a whole warp, for plans with few microbatches.  Every open microbatch has a 64-bit key,
+// residual << 32 | ~stamp (stamp = the sample that changed it last): the smallest key among those whose residual is
+// >= l is the smallest such residual and, among equal residuals, the most recently changed microbatch: the
+// tie-break of the packing rule.  Stamps are distinct, so keys are.  Every lane looks at a 32nd of the keys and two
+// warp reductions (high word, then low word among the lanes that hold the winning high word) find the winner.
+// A step of the chain costs a few hundred cycles instead of the thousand of the bitmap descent with its per-residual
+// stacks, and the kernels need little or no shared memory, so they also start on an SM whose shared-memory split was
+// chosen for the copy kernels.  The caller bounds the microbatch count: any-fit packing leaves at most one microbatch
+// half empty, so n_mb <= 2 sum(l) / L + 1.
 constexpr uint32_t kWarpFitChunk = 256;
-constexpr uint32_t kWarpFitMaxCap = 2048;
+constexpr uint32_t kWarpFitMaxCap = 1024;
+constexpr unsigned long long kNoKey = ~0ull;
+__device__ __forceinline__ unsigned long long fit_key(uint32_t residual, uint32_t stamp) {
+  return ((unsigned long long)residual << 32) | (0xFFFFFFFFu - stamp);
+}
+// the smallest key of the warp (kNoKey if no lane has one)
+__device__ __forceinline__ unsigned long long warp_min_key(unsigned long long k) {
+  const uint32_t hi = (uint32_t)(k >> 32), lo = (uint32_t)k;
+  const uint32_t mh = __reduce_min_sync(0xFFFFFFFFu, hi);
+  const uint32_t ml = __reduce_min_sync(0xFFFFFFFFu, hi == mh ? lo : 0xFFFFFFFFu);
+  return ((unsigned long long)mh << 32) | ml;
+}
+
+// Keys in shared memory (8 bytes per microbatch, + 8 for lmax and count): up to kWarpFitMaxCap microbatches.
 __global__ void __launch_bounds__(256) k_bestfit_warp(const uint32_t* __restrict__ len, uint32_t n, uint32_t L, uint32_t cap,
                                                       uint32_t* sample_mb, uint32_t* sample_rank, uint32_t* mb_residual,
                                                       uint32_t* mb_tokens, uint32_t* mb_lmax, uint32_t* mb_count, uint32_t* scalars) {
-  extern __shared__ __align__(16) uint32_t sm[];
-  uint32_t *P = sm, *stamp = P + cap, *lmax = stamp + cap, *cnt = lmax + cap;
+  extern __shared__ __align__(16) unsigned long long smk[];
+  unsigned long long* key = smk;                                 // [cap]; kNoKey = not open
+  uint32_t* lmax = reinterpret_cast<uint32_t*>(key + cap);       // [cap]
+  uint32_t* cnt = lmax + cap;                                    // [cap]
   uint32_t *s_len = cnt + cap, *s_mb = s_len + kWarpFitChunk, *s_rank = s_mb + kWarpFitChunk;
   __shared__ uint32_t s_nmb;
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -233,29 +250,35 @@ __global__ void __launch_bounds__(256) k_bestfit_warp(const uint32_t* __restrict
       uint32_t n_mb = s_nmb;
       for (uint32_t i = 0; i < c; ++i) {
         const uint32_t l = s_len[i];
-        uint32_t bp = 0xFFFFFFFFu, bs = 0, bj = 0;  // this lane's best: smallest residual >= l, then the latest stamp
-        for (uint32_t j = lane; j < n_mb; j += 32) {
-          const uint32_t p = P[j], st = stamp[j];
-          if (p >= l && (p < bp || (p == bp && st > bs))) { bp = p; bs = st; bj = j; }
+        const unsigned long long floor_key = (unsigned long long)l << 32;  // keys below it have a residual < l
+        unsigned long long best = kNoKey;
+        uint32_t bj = 0;
+        for (uint32_t j0 = 0; j0 < n_mb; j0 += 128) {  // four independent loads per lane and round
+          unsigned long long k[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const uint32_t j = j0 + 32 * u + lane;
+            k[u] = j < n_mb ? key[j] : kNoKey;
+          }
+#pragma unroll
+          for (int u = 0; u < 4; ++u)
+            if (k[u] >= floor_key && k[u] < best) { best = k[u]; bj = j0 + 32 * u + lane; }
         }
-        const uint32_t mp = __reduce_min_sync(0xFFFFFFFFu, bp);
-        if (mp != 0xFFFFFFFFu) {
-          const uint32_t mine = bp == mp ? bs + 1 : 0;  // + 1: sample 0's stamp counts too
-          const uint32_t ms = __reduce_max_sync(0xFFFFFFFFu, mine);
-          const uint32_t who = __ffs(__ballot_sync(0xFFFFFFFFu, mine == ms)) - 1;
-          const uint32_t j = __shfl_sync(0xFFFFFFFFu, bj, who);
-          if (lane == 0) {
-            P[j] = mp - l; stamp[j] = base + i;
-            lmax[j] = max(lmax[j], l);
-            const uint32_t k = cnt[j];
-            cnt[j] = k + 1;
-            s_mb[i] = j; s_rank[i] = k;
+        const unsigned long long win = warp_min_key(best);
+        if (win != kNoKey) {
+          if (best == win) {  // keys are distinct: one lane
+            key[bj] = fit_key((uint32_t)(win >> 32) - l, base + i);
+            lmax[bj] = max(lmax[bj], l);
+            const uint32_t k0 = cnt[bj];
+            cnt[bj] = k0 + 1;
+            s_mb[i] = bj; s_rank[i] = k0;
           }
         } else {
-          const uint32_t j = n_mb;
-          if (lane == 0 && j < cap) { P[j] = L - l; stamp[j] = base + i; lmax[j] = l; cnt[j] = 1; }
-          if (lane == 0) { s_mb[i] = j; s_rank[i] = 0; }
-          if (j < cap) ++n_mb;  // (the bound guarantees it)
+          if (lane == 0) {
+            if (n_mb < cap) { key[n_mb] = fit_key(L - l, base + i); lmax[n_mb] = l; cnt[n_mb] = 1; }
+            s_mb[i] = n_mb; s_rank[i] = 0;
+          }
+          if (n_mb < cap) ++n_mb;  // (the bound guarantees it)
         }
         __syncwarp();
       }
@@ -267,56 +290,61 @@ __global__ void __launch_bounds__(256) k_bestfit_warp(const uint32_t* __restrict
   }
   const uint32_t n_mb = s_nmb;
   for (uint32_t j = threadIdx.x; j < n_mb; j += blockDim.x) {
-    mb_residual[j] = P[j]; mb_tokens[j] = L - P[j]; mb_lmax[j] = lmax[j]; mb_count[j] = cnt[j];
+    const uint32_t r = (uint32_t)(key[j] >> 32);
+    mb_residual[j] = r; mb_tokens[j] = L - r; mb_lmax[j] = lmax[j]; mb_count[j] = cnt[j];
   }
   if (threadIdx.x == 0) scalars[SC_NMB] = n_mb;
 }
 
-// The same with the open microbatches in registers, for plans of at most 32 R microbatches (microbatch j lives in
-// slot j / 32 of lane j % 32): a step of the chain is R comparisons per lane and two warp reductions, with no memory
-// access on the chain at all.
+// The same with the keys in registers, for plans of at most 32 R microbatches (microbatch j lives in slot j / 32 of
+// lane j % 32): no memory access on the chain at all.
 template <int R>
 __global__ void __launch_bounds__(256) k_bestfit_regs(const uint32_t* __restrict__ len, uint32_t n, uint32_t L,
                                                       uint32_t* sample_mb, uint32_t* sample_rank, uint32_t* mb_residual,
                                                       uint32_t* mb_tokens, uint32_t* mb_lmax, uint32_t* mb_count, uint32_t* scalars) {
-  __shared__ uint32_t s_len[kWarpFitChunk], s_mb[kWarpFitChunk], s_rank[kWarpFitChunk];
+  __shared__ uint32_t s_len[kWarpFitChunk + 1], s_mb[kWarpFitChunk], s_rank[kWarpFitChunk];
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  uint32_t P[R], St[R], Lm[R], Cn[R];  // residual (0 = not open or full: never chosen, l >= 1), stamp, lmax, count
+  unsigned long long K[R];  // kNoKey = not open (a full microbatch has residual 0 and is never >= l)
+  uint32_t Lm[R], Cn[R];
 #pragma unroll
-  for (int s = 0; s < R; ++s) { P[s] = 0; St[s] = 0; Lm[s] = 0; Cn[s] = 0; }
+  for (int s = 0; s < R; ++s) { K[s] = kNoKey; Lm[s] = 0; Cn[s] = 0; }
   uint32_t n_mb = 0;
   for (uint32_t base = 0; base < n; base += kWarpFitChunk) {
     const uint32_t c = min(kWarpFitChunk, n - base);
     for (uint32_t i = threadIdx.x; i < c; i += blockDim.x) s_len[i] = len[base + i];
+    if (threadIdx.x == 0) s_len[c] = 0;
     __syncthreads();
     if (warp == 0) {
+      uint32_t l_next = s_len[0];
       for (uint32_t i = 0; i < c; ++i) {
-        const uint32_t l = s_len[i];
-        uint32_t bp = 0xFFFFFFFFu, bs = 0;
-        int bslot = 0;
+        const uint32_t l = l_next;
+        l_next = s_len[i + 1];  // off the chain
+        const unsigned long long floor_key = (unsigned long long)l << 32;
+        unsigned long long cand[R];
 #pragma unroll
-        for (int s = 0; s < R; ++s) {
-          const bool better = P[s] >= l && (P[s] < bp || (P[s] == bp && St[s] > bs));
-          if (better) { bp = P[s]; bs = St[s]; bslot = s; }
-        }
-        const uint32_t mp = __reduce_min_sync(0xFFFFFFFFu, bp);
-        if (mp != 0xFFFFFFFFu) {
-          const uint32_t mine = bp == mp ? bs + 1 : 0;  // + 1: sample 0's stamp counts too
-          const uint32_t ms = __reduce_max_sync(0xFFFFFFFFu, mine);
-          if (mine == ms) {  // stamps are distinct: one lane
-            uint32_t k = 0;
+        for (int s = 0; s < R; ++s) cand[s] = (K[s] >= floor_key && K[s] != kNoKey) ? K[s] : kNoKey;
+#pragma unroll
+        for (int w = 1; w < R; w <<= 1)  // pairwise minimum
+#pragma unroll
+          for (int s = 0; s + w < R; s += 2 * w) cand[s] = min(cand[s], cand[s + w]);
+        const unsigned long long best = cand[0];
+        const unsigned long long win = warp_min_key(best);
+        if (win != kNoKey) {
+          if (best == win) {  // keys are distinct: one lane, one slot
+            const unsigned long long upd = fit_key((uint32_t)(win >> 32) - l, base + i);
+            uint32_t k0 = 0, slot = 0;
 #pragma unroll
             for (int s = 0; s < R; ++s)
-              if (s == bslot) { P[s] = mp - l; St[s] = base + i; Lm[s] = max(Lm[s], l); k = Cn[s]; Cn[s] = k + 1; }
-            s_mb[i] = lane + 32u * (uint32_t)bslot;
-            s_rank[i] = k;
+              if (K[s] == win) { K[s] = upd; Lm[s] = max(Lm[s], l); k0 = Cn[s]; Cn[s] = k0 + 1; slot = s; }
+            s_mb[i] = lane + 32u * slot;
+            s_rank[i] = k0;
           }
         } else {
           if (lane == (n_mb & 31u)) {
             const int slot = (int)(n_mb >> 5);
 #pragma unroll
             for (int s = 0; s < R; ++s)
-              if (s == slot) { P[s] = L - l; St[s] = base + i; Lm[s] = l; Cn[s] = 1; }
+              if (s == slot) { K[s] = fit_key(L - l, base + i); Lm[s] = l; Cn[s] = 1; }
             s_mb[i] = n_mb; s_rank[i] = 0;
           }
           ++n_mb;
@@ -331,7 +359,10 @@ __global__ void __launch_bounds__(256) k_bestfit_regs(const uint32_t* __restrict
 #pragma unroll
     for (int s = 0; s < R; ++s) {
       const uint32_t j = lane + 32u * (uint32_t)s;
-      if (j < n_mb) { mb_residual[j] = P[s]; mb_tokens[j] = L - P[s]; mb_lmax[j] = Lm[s]; mb_count[j] = Cn[s]; }
+      if (j < n_mb) {
+        const uint32_t r = (uint32_t)(K[s] >> 32);
+        mb_residual[j] = r; mb_tokens[j] = L - r; mb_lmax[j] = Lm[s]; mb_count[j] = Cn[s];
+      }
     }
     if (lane == 0) scalars[SC_NMB] = n_mb;
   }
