@@ -2,10 +2,10 @@
 //
 // Kernels in this file
 //   k_page_table_init  PTEs from the vpn->frame binding (Sec. 3.2: page tables map GVA -> physical)
-//   k_register_scan    per-sample text-page counts -> exclusive scan, sample + span tables
+//   k_register_scan    per-sample text-page counts -> exclusive scan, sample + span tables, text-page pops and records
 //   k_register_ids     token ids into text pages, placeholder-run validation
 //   k_alloc_scan       pages/list blocks/chunks per span -> exclusive scans, ring pops
-//   k_alloc_fill       span page lists (two-level) from consecutive ring entries
+//   k_alloc_fill       span page lists (two-level) from consecutive ring entries; chunk records for k_scatter
 //   k_scatter          the producer byte copy into pages, optional fused fp32->bf16 RNE cast
 //   k_scatter_host_bulk  bf16 sources into host-tier pages by bulk-async copies
 //   k_free_scan/_fill  pages, list blocks and text pages back to the ring tails
@@ -305,9 +305,10 @@ __global__ void __launch_bounds__(256) k_alloc_fill(PoolView v, WriteCall c, uin
 }
 
 // ------------------------------------------------------------------------------------------
-// K4: producer scatter.  Work unit = one chunk of destination bytes inside one page; each CTA owns a
-// contiguous chunk range (one search at its start, then a walk), resolves the destination frame through
-// the span's page list and the page table once per page, and moves 16-byte vectors.
+// K4: producer scatter.  Work unit = one chunk of a span's image.  Where pages are at least a chunk long the chunk
+// is one record (source, destination frame + offset, length) that k_alloc_fill prepared; else the CTA finds the
+// chunk's span by table or search and each warp resolves its destination frame through the span's page list and
+// the page table once per page.  16-byte vectors either way.
 // ------------------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t rne_bf16(uint32_t u) {
   // IEEE round-to-nearest-even on the bit pattern; NaN -> sign | 0x7FC0; denormals kept
@@ -443,8 +444,7 @@ __global__ void __launch_bounds__(256, F32 ? 4 : 6) k_scatter(PoolView v, WriteC
 }
 
 
-// launches k_scatter<MODE, F32> on a grid of at most `max_ctas` CTAs, never more than fit on the GPU at once
-// (the round-robin deal assumes every CTA runs from the start)
+// launches k_scatter<MODE, F32, records> on a grid of at most `max_ctas` CTAs, never more than fit on the GPU at once
 template <int MODE, bool F32>
 static void launch_scatter(ft_pool* p, const WriteCall& w, uint64_t total_chunks, uint64_t max_ctas, cudaStream_t s,
                            ClaimCounter* counters) {
