@@ -231,6 +231,33 @@ def test_bestfit_invariants_and_brute_force_optimum():
         plan.destroy()
 
 
+def test_any_fit_bound_on_the_microbatch_count():
+    """Best fit opens a microbatch only when the sample fits none that is open, so at most one microbatch ends at most
+    half full: n_mb <= 2 sum(l) / L + 1 (integer division).  The device sizes its packing tables by this bound; here it
+    is checked on the oracle, for both packing orders and for length mixes that make it tight."""
+    rng = np.random.default_rng(7)
+    for trial in range(300):
+        n = int(rng.integers(1, 500))
+        L = int(rng.integers(2, 2000))
+        kind = trial % 4
+        if kind == 0:
+            lengths = rng.integers(1, L + 1, size=n)
+        elif kind == 1:
+            lengths = np.full(n, L // 2 + 1)                     # every sample alone: n_mb = n, just above half full
+        elif kind == 2:
+            lengths = rng.choice([1, max(1, L // 2), L], size=n)
+        else:
+            lengths = rng.integers(1, max(2, L // 8), size=n)
+        for flags in (0, 2):                                     # caller's order, longest first
+            cfg = plan_cfg(L)
+            cfg.flags = flags
+            rc, plan = plan_from_lengths(lengths, cfg)
+            assert rc == 0
+            n_mb = plan.arrays()["n_mb"]
+            assert n_mb <= 2 * int(lengths.sum()) // L + 1, (trial, n, L, n_mb)
+            plan.destroy()
+
+
 def test_linear_scan_equals_literal_segment_tree():
     rng = np.random.default_rng(2)
     for trial in range(200):
