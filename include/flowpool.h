@@ -499,6 +499,16 @@ int32_t pool_profile_read(ft_pool* pool, ft_kernel_time* out /* host [FT_K_COUNT
  *                        CTAs need costs it occupancy and 6 percent of its bandwidth)
  *   peers_remote         1: pool_import_mapping flags every peer's HBM frames as remote even when they are on this
  *                        device (exercises the remote path on one GPU); 0: only frames of another device are remote
+ *   host_copy_engine     who moves host-tier pages of bf16 writes and of assemblies.  0 (default): the bulk-copy
+ *                        kernels.  1: the copy engines: one cudaMemcpyAsync per run of pages that are contiguous in a
+ *                        span's image and in the host slab, issued from the host's own copy of the page lists (fp32
+ *                        sources, imported samples and plans made under the other setting still take the kernels).
+ *                        Measured on a B200 host: single 2 MiB pages move as fast either way (50 GB/s), runs of 8 MiB
+ *                        and more reach the link's rate (54-55 GB/s against 46-51), which a pool with an identity
+ *                        binding gets (config 2: 717 against 645 GB/s for the whole step).  The price: a copy
+ *                        engine serves its queue in order, so these copies wait behind any bulk copy the application
+ *                        has queued in the same direction, and the application's behind them; the kernels share
+ *                        the link but no queue.  Hence off by default
  *   bulk_wait_limit_us   bound, in microseconds, of every wait of the bulk-copy kernels for a staged load (default
  *                        2 000 000; 100..10 000 000).  A load not seen within it is declared lost and the call
  *                        reports FT_ERR_TIMEOUT through the status word (see FT_ERR_TIMEOUT above)
@@ -515,7 +525,7 @@ typedef struct {
   uint32_t host_ctas, host_store_ctas, gather_unroll, grad_ctas_per_sm, grad_hot_threshold;
   uint32_t remote_ctas, peers_remote, scatter_smem_carveout, gather_smem_carveout;
   uint32_t bulk_wait_limit_us, bulk_timeout_test;
-  uint32_t reserved[1];
+  uint32_t host_copy_engine;
 } ft_tuning;
 int32_t pool_get_tuning(ft_pool* pool, ft_tuning* out);
 int32_t pool_set_tuning(ft_pool* pool, const ft_tuning* in);

@@ -67,11 +67,11 @@ class PoolStats(C.Structure):
 
 TUNING_FIELDS = ("dev_ctas_per_sm", "scatter_ctas_per_sm", "scatter_group", "chunk_shift", "host_ctas", "host_store_ctas",
                  "gather_unroll", "grad_ctas_per_sm", "grad_hot_threshold", "remote_ctas", "peers_remote", "scatter_smem_carveout", "gather_smem_carveout",
-                 "bulk_wait_limit_us", "bulk_timeout_test")
+                 "bulk_wait_limit_us", "bulk_timeout_test", "host_copy_engine")
 
 
 class Tuning(C.Structure):
-    _fields_ = [(k, C.c_uint32) for k in TUNING_FIELDS] + [("reserved", C.c_uint32 * 1)]
+    _fields_ = [(k, C.c_uint32) for k in TUNING_FIELDS]
 
 
 class KernelTime(C.Structure):

@@ -213,6 +213,19 @@ struct ft_plan {
   uint32_t *d_rank_mb_off, *d_rank_mbs, *d_rank_cnt, *d_tile_first_sample, *d_scalars;
   uint64_t *d_sample_cost, *d_mb_cost, *d_sample_row_off, *d_mb_row_off, *d_plan_len;
   uint64_t* d_row_src = nullptr;          // row words of the assembly (plans of written samples only)
+  // Host-tier pages of the plan's own samples as copy-engine work: one entry per run of pages that follow one another
+  // in a span's image and in the host slab, grouped by microbatch (entries of microbatch j: [mb_copy_off[j],
+  // mb_copy_off[j+1])).  Made with the plan where the pool sends its host tier through the copy engine and no sample
+  // of the plan is imported; a plan dies with the first free of one of its samples, so the pages cannot change.
+  struct HostCopy {
+    uint64_t row0;     // plan-global row of the span's first row
+    uint64_t img_off;  // byte offset of the run in the span's image
+    const void* src;   // host address of the run
+    uint64_t len;
+  };
+  std::vector<HostCopy> host_copies;
+  std::vector<uint32_t> mb_copy_off;
+  bool host_copies_valid = false;
 };
 
 namespace ft {
@@ -255,6 +268,7 @@ struct ft_span_mirror {
   uint32_t grid[3] = {0, 0, 0};  // token grid (T, H, W) as last set; all zero = none
   bool written = false;
   uint64_t named = 0;   // call_seq of the write call that last named this span
+  std::vector<uint32_t> pages;  // global page index by ordinal (own written spans; the host's copy of the page list)
 };
 
 // Per-call context: the descriptors of one ABI call travel host -> device through one of a small ring of these.
@@ -263,7 +277,7 @@ struct ft_span_mirror {
 // events guard reuse: the host waits for `ev_up` before it rewrites `h`; the metadata stream waits for `ev_done`
 // (recorded behind the last kernel of the call that reads `d` or the counters) before it rewrites `d`.
 struct ft_call_ctx {
-  void* h = nullptr;   size_t hcap = 0;
+  void* h = nullptr;   size_t hcap = 0;   void* hd = nullptr;  // `h` as the device sees it (mapped pinned memory)
   void* d = nullptr;   size_t dcap = 0;
   cudaEvent_t ev_up = nullptr, ev_done = nullptr;
   bool busy_up = false, busy_done = false;
@@ -312,9 +326,16 @@ struct ft_pool {
   // on the metadata stream is not reusable across streams at once, and every other plan paid a fresh allocation.)
   struct plan_block { void* d; size_t cap; cudaEvent_t ev; };
   std::vector<plan_block> plan_cache;
-  void* plan_pinned = nullptr;        // pinned landing zone of the plan's summary read-back
+  void* plan_pinned = nullptr;        // pinned landing zone of the plan's summary read-back (mapped: a kernel stores into it)
+  void* plan_pinned_dev = nullptr;
   size_t plan_pinned_cap = 0;
   std::vector<uint32_t> bind_hbm, bind_host;           // vpn -> frame of this process's binding (exported to peers)
+  // The host's copy of the FIFO page ring: pops and pushes are deterministic (calls in order, spans in argument order,
+  // pages by ordinal), so the host can follow them and knows every span's pages without asking the device.  It serves
+  // the copy-engine path of the host tier; the device's ring stays the one the kernels read.
+  std::vector<uint32_t> h_ring;
+  uint64_t h_ring_head = 0, h_ring_count = 0;
+  int host_dma = 0;             // 1: host-tier pages of bf16 writes and of assemblies go through the copy engines
   void* d_text_base() const { return d_text; }
   std::vector<void*> peer_allocs;                      // imported peers' page-table arrays
   std::vector<uint8_t> peer_imported;                  // [world_size]
@@ -364,6 +385,9 @@ namespace ft {
 int32_t gather_device_setup(ft_pool* p);
 // shared-memory carve-out preference (percent) of the copy kernels of each translation unit
 int32_t gather_set_carveout(int pct);
+// n 32-bit words device <-> mapped host memory by a small kernel on `st` (not by a copy engine: see ctx_upload)
+int32_t copy_words(void* dst, const void* src, size_t n_words, cudaStream_t st);
+bool host_tier_by_copy_engine(const ft_pool* p);
 // fills the plan's row words (metadata stream, behind the latest copy of token ids)
 int32_t plan_rows_launch(ft_pool* p, ft_plan* pl);
 int32_t scatter_set_carveout(int pct);
@@ -371,7 +395,8 @@ int32_t plan_device_setup(ft_pool* p);
 // (d_list: device array of the list layout's entries, or nullptr for the range [mb_begin, mb_end))
 int32_t gather_launch(ft_pool* p, const ft_plan* pl, uint32_t mb_begin, uint32_t mb_end, const void* embed_table,
                       uint32_t vocab, void* out_embeds, int32_t* out_cu, int32_t* out_pos, uint32_t pad_L, cudaStream_t st,
-                      const void* d_list, uint32_t n_list, uint64_t list_tiles, uint64_t list_rows, ClaimCounter* counter);
+                      const void* d_list, uint32_t n_list, uint64_t list_tiles, uint64_t list_rows, ClaimCounter* counter,
+                      const uint32_t* h_mb_list = nullptr);
 __global__ void k_page_table_init(uint64_t* pte, const uint32_t* bind, uint64_t n, uint64_t base, uint64_t frame_bytes,
                                   uint64_t flags);
 // uploads `bytes` from `src` (pageable) to the front of the pool's device scratch, asynchronously,

@@ -400,7 +400,8 @@ namespace ft {
 // the index outputs are left to the caller.  Arguments are validated by the caller.
 int32_t gather_launch(ft_pool* p, const ft_plan* pl, uint32_t mb_begin, uint32_t mb_end, const void* embed_table,
                       uint32_t vocab, void* out_embeds, int32_t* out_cu, int32_t* out_pos, uint32_t pad_L, cudaStream_t st,
-                      const void* d_list, uint32_t n_list, uint64_t list_tiles, uint64_t list_rows, ClaimCounter* counter) {
+                      const void* d_list, uint32_t n_list, uint64_t list_tiles, uint64_t list_rows, ClaimCounter* counter,
+                      const uint32_t* h_mb_list) {
   if (p->view.row_bytes > (kMaxSeg - 1) * 4096) return FT_ERR_CAPACITY;
   const PlanView pv = make_plan_view(pl);
   const bool listed = d_list != nullptr;
@@ -462,10 +463,38 @@ int32_t gather_launch(ft_pool* p, const ft_plan* pl, uint32_t mb_begin, uint32_t
       FT_CUDA(cudaEventRecord(p->fork_ev[1], st));
       FT_CUDA(cudaStreamWaitEvent(p->side_stream[1], p->fork_ev[1], 0));
       prof_begin(p, FT_K_GATHER_HOST, p->side_stream[1]);
-      k_gather_host_bulk<<<(unsigned)p->host_ctas, 32, kBulkSmemBytes, p->side_stream[1]>>>(p->view, pv, ah, kPteHost);
+      if (host_tier_by_copy_engine(p) && pl->host_copies_valid && !p->peer_host_frames && (!listed || h_mb_list)) {
+        // the host tier through the copy engine: every run of host pages of the microbatches asked for is one
+        // contiguous byte range of the output (a span's rows are consecutive output rows)
+        const uint64_t rb = p->view.row_bytes;
+        auto issue = [&](uint32_t j, uint64_t out_row0) -> int32_t {  // out_row0: output row of the microbatch's first row
+          for (uint32_t e = pl->mb_copy_off[j]; e < pl->mb_copy_off[j + 1]; ++e) {
+            const ft_plan::HostCopy& hc = pl->host_copies[e];
+            uint8_t* dst = a.out + (out_row0 + (hc.row0 - pl->h_mb_row_off[j])) * rb + hc.img_off;
+            FT_CUDA(cudaMemcpyAsync(dst, hc.src, hc.len, cudaMemcpyHostToDevice, p->side_stream[1]));
+          }
+          return FT_OK;
+        };
+        uint64_t out_row0 = 0;
+        if (listed) {
+          for (uint32_t i = 0; i < n_list; ++i) {
+            const uint32_t j = h_mb_list[i];
+            const int32_t rcj = issue(j, out_row0);
+            if (rcj != FT_OK) return rcj;
+            out_row0 += pl->h_mb_row_off[j + 1] - pl->h_mb_row_off[j];
+          }
+        } else {
+          for (uint32_t j = mb_begin; j < mb_end; ++j) {
+            const int32_t rcj = issue(j, pad_L ? (uint64_t)(j - mb_begin) * pad_L : pl->h_mb_row_off[j] - a.row_lo);
+            if (rcj != FT_OK) return rcj;
+          }
+        }
+      } else {
+        k_gather_host_bulk<<<(unsigned)p->host_ctas, 32, kBulkSmemBytes, p->side_stream[1]>>>(p->view, pv, ah, kPteHost);
+        p->gpu_launches += 1;
+      }
       prof_end(p, p->side_stream[1]);
       FT_CUDA(cudaEventRecord(p->join_ev[1], p->side_stream[1]));
-      p->gpu_launches += 1;
     }
     if (remote_sources) {
       FT_CUDA(cudaEventRecord(p->fork_ev[2], st));
@@ -571,7 +600,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_gather_list(ft_po
     if (rc0 != FT_OK) return rc0;
   }
   {
-    const int32_t rc2 = gather_launch(p, pl, 0, pl->n_mb, embed_table, vocab, out_embeds, out_cu, out_pos, 0, st, cx->d, n_list, tiles, rows, cx->counters);
+    const int32_t rc2 = gather_launch(p, pl, 0, pl->n_mb, embed_table, vocab, out_embeds, out_cu, out_pos, 0, st, cx->d, n_list, tiles, rows, cx->counters, mb_list);
     if (rc2 != FT_OK) return rc2;
   }
   {

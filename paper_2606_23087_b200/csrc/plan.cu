@@ -688,7 +688,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_plan_microbatches
   memcpy(cx->h, slot, (size_t)n * 4);
   rc = ctx_upload(p, cx, (size_t)n * 4);
   if (rc != FT_OK) { plan_destroy(pl); return rc; }
-  CK(cudaMemcpyAsync(pl->d_slots, cx->d, (size_t)n * 4, cudaMemcpyDeviceToDevice, st));
+  if ((rc = copy_words(pl->d_slots, cx->d, n, st)) != FT_OK) { plan_destroy(pl); return rc; }
   rc = ctx_release(p, cx, st);
   if (rc != FT_OK) { plan_destroy(pl); return rc; }
   CK(cudaMemsetAsync(pl->d_rank_cnt, 0, (size_t)N * 4, st));
@@ -749,19 +749,26 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_plan_microbatches
 
   // the summary and the two offset arrays the host sizes assemblies with come back in one go (n + 1 entries bound
   // n_mb + 1), into a pinned landing zone, behind one synchronisation of the metadata stream
-  const size_t rb_sc = 0, rb_so = align_up(sizeof(uint32_t) * SC_COUNT, 16), rb_ro = align_up(rb_so + n1 * 4, 16), rb_bytes = rb_ro + n1 * 8;
+  const bool want_copies = with_rows && host_tier_by_copy_engine(p) && p->cfg.host_pages != 0;
+  const size_t rb_sc = 0, rb_so = align_up(sizeof(uint32_t) * SC_COUNT, 16), rb_ro = align_up(rb_so + n1 * 4, 16);
+  const size_t rb_ms = align_up(rb_ro + n1 * 8, 16), rb_bytes = rb_ms + (want_copies ? (size_t)n * 4 : 0);
   if (p->plan_pinned_cap < rb_bytes) {
     if (p->plan_pinned) CK(cudaFreeHost(p->plan_pinned));
     p->plan_pinned = nullptr; p->plan_pinned_cap = 0;
     size_t cap = 1 << 16;
     while (cap < rb_bytes) cap <<= 1;
-    CK(cudaHostAlloc(&p->plan_pinned, cap, cudaHostAllocDefault));
+    CK(cudaHostAlloc(&p->plan_pinned, cap, cudaHostAllocMapped));
+    CK(cudaHostGetDevicePointer(&p->plan_pinned_dev, p->plan_pinned, 0));
     p->plan_pinned_cap = cap;
   }
   uint8_t* rb = static_cast<uint8_t*>(p->plan_pinned);
-  CK(cudaMemcpyAsync(rb + rb_sc, pl->d_scalars, sizeof(uint32_t) * SC_COUNT, cudaMemcpyDeviceToHost, st));
-  CK(cudaMemcpyAsync(rb + rb_so, pl->d_mb_sample_off, n1 * 4, cudaMemcpyDeviceToHost, st));
-  CK(cudaMemcpyAsync(rb + rb_ro, pl->d_mb_row_off, n1 * 8, cudaMemcpyDeviceToHost, st));
+  {
+    uint8_t* rbd = static_cast<uint8_t*>(p->plan_pinned_dev);  // the landing zone as the device sees it
+    if ((rc = copy_words(rbd + rb_sc, pl->d_scalars, SC_COUNT, st)) != FT_OK) { plan_destroy(pl); return rc; }
+    if ((rc = copy_words(rbd + rb_so, pl->d_mb_sample_off, n1, st)) != FT_OK) { plan_destroy(pl); return rc; }
+    if ((rc = copy_words(rbd + rb_ro, pl->d_mb_row_off, n1 * 2, st)) != FT_OK) { plan_destroy(pl); return rc; }
+    if (want_copies && (rc = copy_words(rbd + rb_ms, pl->d_mb_samples, n, st)) != FT_OK) { plan_destroy(pl); return rc; }
+  }
   CK(cudaStreamSynchronize(st));
   const uint32_t* sc = reinterpret_cast<const uint32_t*>(rb + rb_sc);
   pl->n_mb = sc[SC_NMB];
@@ -769,6 +776,39 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_plan_microbatches
   pl->total_tokens = (uint64_t)sc[SC_TOTAL_LO] | ((uint64_t)sc[SC_TOTAL_HI] << 32);
   pl->h_mb_sample_off.assign(reinterpret_cast<const uint32_t*>(rb + rb_so), reinterpret_cast<const uint32_t*>(rb + rb_so) + pl->n_mb + 1);
   pl->h_mb_row_off.assign(reinterpret_cast<const uint64_t*>(rb + rb_ro), reinterpret_cast<const uint64_t*>(rb + rb_ro) + pl->n_mb + 1);
+  if (want_copies) {
+    // the plan's host-tier pages as copy-engine work, from the host's page lists, in plan order
+    const uint32_t* order = reinterpret_cast<const uint32_t*>(rb + rb_ms);
+    const uint64_t PS = p->cfg.page_bytes, hbm = p->cfg.hbm_pages;
+    const uint32_t S = p->cfg.max_spans_per_sample;
+    const uint8_t* base = static_cast<const uint8_t*>(p->host_base);
+    pl->mb_copy_off.assign(pl->n_mb + 1, 0);
+    bool ok = true;
+    uint64_t row = 0;
+    for (uint32_t j = 0; j < pl->n_mb && ok; ++j) {
+      for (uint32_t q = pl->h_mb_sample_off[j]; q < pl->h_mb_sample_off[j + 1]; ++q) {
+        const uint32_t slot_q = order[q];
+        const ft_slot_mirror& sm = p->slots[slot_q];
+        if (sm.remote) { ok = false; break; }  // an imported sample: its pages are a peer's, the kernels read them
+        for (uint32_t js = 0; js < sm.n_spans; ++js) {
+          const ft_span_mirror& m = p->spans[(uint64_t)slot_q * S + js];
+          const uint64_t bytes = (uint64_t)m.tokens * p->view.row_bytes;
+          for (uint32_t k = 0; k < (uint32_t)m.pages.size();) {
+            if (m.pages[k] < hbm) { ++k; continue; }
+            const uint64_t frame = p->bind_host[m.pages[k] - hbm];
+            uint32_t k1 = k + 1;
+            while (k1 < m.pages.size() && m.pages[k1] >= hbm && p->bind_host[m.pages[k1] - hbm] == frame + (k1 - k)) ++k1;
+            const uint64_t off = (uint64_t)k * PS;
+            pl->host_copies.push_back({row + m.pos, off, base + frame * PS, std::min<uint64_t>(bytes, (uint64_t)k1 * PS) - off});
+            k = k1;
+          }
+        }
+        row += sm.seq_len;
+      }
+      pl->mb_copy_off[j + 1] = (uint32_t)pl->host_copies.size();
+    }
+    pl->host_copies_valid = ok;
+  }
   // the row words are filled behind the caller's back: the plan is complete for the host, assemblies wait for the
   // metadata stream anyway
   rc = plan_rows_launch(p, pl);

@@ -60,7 +60,8 @@ int32_t ctx_acquire(ft_pool* p, int side, size_t blob_bytes, size_t total_bytes,
     size_t cap = 1 << 16;
     while (cap < blob_bytes) cap <<= 1;
     c.h = nullptr; c.hcap = 0;
-    FT_CUDA(cudaHostAlloc(&c.h, cap, cudaHostAllocDefault));
+    FT_CUDA(cudaHostAlloc(&c.h, cap, cudaHostAllocMapped));
+    FT_CUDA(cudaHostGetDevicePointer(&c.hd, c.h, 0));
     c.hcap = cap;
   }
   if (c.dcap < total_bytes) {
@@ -83,10 +84,26 @@ int32_t ctx_acquire(ft_pool* p, int side, size_t blob_bytes, size_t total_bytes,
   return FT_OK;
 }
 
+// The library's own small transfers (a call's descriptors up, a plan's summary down) are made by a kernel that reads or
+// writes mapped pinned memory, not by cudaMemcpyAsync: the copy engines serve their queues in order, so a descriptor
+// upload behind an application's bulk host-to-device copy (or a plan's summary behind a bulk copy-out) would wait for
+// all of it, and every call of the pool with it.
+__global__ void k_copy_words(uint32_t* __restrict__ dst, const uint32_t* __restrict__ src, size_t n) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) dst[i] = src[i];
+}
+int32_t copy_words(void* dst, const void* src, size_t n_words, cudaStream_t st) {
+  if (n_words == 0) return FT_OK;
+  const unsigned grid = (unsigned)std::min<size_t>((n_words + 255) / 256, 64);
+  k_copy_words<<<grid, 256, 0, st>>>(static_cast<uint32_t*>(dst), static_cast<const uint32_t*>(src), n_words);
+  FT_CUDA(cudaGetLastError());
+  return FT_OK;
+}
+
 int32_t ctx_upload(ft_pool* p, ft_call_ctx* c, size_t bytes) {
   p->meta_seq++;
   if (bytes) {
-    FT_CUDA(cudaMemcpyAsync(c->d, c->h, bytes, cudaMemcpyHostToDevice, p->meta));
+    const int32_t rc = copy_words(c->d, c->hd, (bytes + 3) / 4, p->meta);
+    if (rc != FT_OK) return rc;
     FT_CUDA(cudaEventRecord(c->ev_up, p->meta));
     c->busy_up = true;
   }
@@ -525,8 +542,40 @@ int32_t scatter_set_carveout(int pct) {
 
 // The byte copy of a producer call, shared by pool_write_embeddings and its no-allocation variant: HBM-bound chunks on
 // the caller's stream, host-bound chunks beside them on the producer side's second stream.
+// The caller's arguments of a producer write, for the copy-engine path (which works from the host's page lists).
+struct WriteArgs {
+  uint32_t n;
+  const uint32_t *slot, *span_idx, *n_tokens;
+  const void* const* src;
+};
+bool host_tier_by_copy_engine(const ft_pool* p) {
+  return p->host_dma == 1;
+}
+// bf16 sources into host-tier pages through the copy engine: one copy per run of pages that follow one another both
+// in the span's image and in the host slab.  The pages come from the host's copy of the page lists (mirror_write ran).
+static int32_t dma_write_host_pages(ft_pool* p, const WriteArgs& a, cudaStream_t s) {
+  const uint64_t PS = p->cfg.page_bytes, hbm = p->cfg.hbm_pages;
+  const uint32_t S = p->cfg.max_spans_per_sample;
+  uint8_t* base = static_cast<uint8_t*>(p->host_base);
+  for (uint32_t q = 0; q < a.n; ++q) {
+    const ft_span_mirror& m = p->spans[(uint64_t)a.slot[q] * S + a.span_idx[q]];
+    const uint64_t bytes = (uint64_t)a.n_tokens[q] * p->view.row_bytes;
+    const uint8_t* src = static_cast<const uint8_t*>(a.src[q]);
+    for (uint32_t k = 0; k < m.npages;) {
+      if (m.pages[k] < hbm) { ++k; continue; }
+      const uint64_t frame = p->bind_host[m.pages[k] - hbm];
+      uint32_t k1 = k + 1;
+      while (k1 < m.npages && m.pages[k1] >= hbm && p->bind_host[m.pages[k1] - hbm] == frame + (k1 - k)) ++k1;
+      const uint64_t off = (uint64_t)k * PS, len = std::min<uint64_t>(bytes, (uint64_t)k1 * PS) - off;
+      FT_CUDA(cudaMemcpyAsync(base + frame * PS, src + off, len, cudaMemcpyDeviceToHost, s));
+      k = k1;
+    }
+  }
+  return FT_OK;
+}
+
 static int32_t launch_write_copies(ft_pool* p, const WriteCall& w, uint64_t total_chunks, bool f32, cudaStream_t st, ClaimCounter* cc,
-                                   bool profile) {
+                                   bool profile, const WriteArgs& args) {
   const ft_pool_config& c = p->cfg;
   auto launch = [&](int mode, cudaStream_t s) {
     const bool host_class = mode == kTierHostOnly || (mode == kTierAll && c.hbm_pages == 0);
@@ -545,11 +594,15 @@ static int32_t launch_write_copies(ft_pool* p, const WriteCall& w, uint64_t tota
     // registers, and stores to host memory are posted (no latency to hide), so a few vector-store CTAs do it
     if (f32) {
       launch_scatter<kTierHostOnly, true>(p, w, total_chunks, (uint64_t)p->host_store_ctas, p->side_stream[0], cc);
+      p->gpu_launches++;
+    } else if (host_tier_by_copy_engine(p)) {
+      const int32_t rc = dma_write_host_pages(p, args, p->side_stream[0]);
+      if (rc != FT_OK) return rc;
     } else {
       k_scatter_host_bulk<<<(unsigned)p->host_ctas, 32, kBulkSmemBytes, p->side_stream[0]>>>(p->view, w, status_seq(p));
+      p->gpu_launches++;
     }
     if (profile) prof_end(p, p->side_stream[0]);
-    p->gpu_launches++;
     FT_CUDA(cudaEventRecord(p->join_ev[0], p->side_stream[0]));
     launch(kTierDeviceOnly, st);
     FT_CUDA(cudaStreamWaitEvent(st, p->join_ev[0], 0));
@@ -770,7 +823,8 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_create(const ft_p
     ft_call_ctx& cx = p->ctx[side][i];
     CK(cudaEventCreateWithFlags(&cx.ev_up, cudaEventDisableTiming));
     CK(cudaEventCreateWithFlags(&cx.ev_done, cudaEventDisableTiming));
-    CK(cudaHostAlloc(&cx.h, 1 << 16, cudaHostAllocDefault));
+    CK(cudaHostAlloc(&cx.h, 1 << 16, cudaHostAllocMapped));
+    CK(cudaHostGetDevicePointer(&cx.hd, cx.h, 0));
     cx.hcap = 1 << 16;
     CK(cudaMalloc(&cx.d, 1 << 18));
     cx.dcap = 1 << 18;
@@ -906,6 +960,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_create(const ft_p
   CK(cudaDeviceSynchronize());
   CK(cudaFree(d_tmp));
   p->bind_hbm = bind_h; p->bind_host = bind_d;
+  p->h_ring = ring; p->h_ring_head = 0; p->h_ring_count = P;
   p->gpu_launches += 5;
 #undef CK
   p->slots.resize(c.max_samples);
@@ -1075,6 +1130,12 @@ static void mirror_write(ft_pool* p, uint32_t n, const uint32_t* slot, const uin
     ft_slot_mirror& s = p->slots[slot[q]];
     ft_span_mirror& m = p->spans[(uint64_t)slot[q] * S + span_idx[q]];
     m.written = true; m.npages = (uint32_t)pages_for_tokens(p, n_tokens[q]);
+    m.pages.resize(m.npages);  // the ring's next entries, as k_alloc_fill takes them
+    for (uint32_t k = 0; k < m.npages; ++k) {
+      m.pages[k] = p->h_ring[p->h_ring_head];
+      p->h_ring_head = (p->h_ring_head + 1) % p->h_ring.size();
+    }
+    p->h_ring_count -= m.npages;
     if (++s.spans_written == s.n_spans) { s.state = FT_SLOT_READY; ready_push(p, slot[q]); }
   }
   p->free_pages -= t.need; p->free_blocks -= t.need_blocks;
@@ -1135,9 +1196,9 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings(
   p->gpu_launches += 2;
   if ((rc = meta_to(p, st)) != FT_OK) return rc;
   const bool f32 = src_dtype == FT_F32;
-  if ((rc = launch_write_copies(p, w, total_chunks, f32, st, cx->counters, true)) != FT_OK) return rc;
+  mirror_write(p, n, slot, span_idx, n_tokens, t, f32);  // (the copy-engine path reads the page lists it leaves)
+  if ((rc = launch_write_copies(p, w, total_chunks, f32, st, cx->counters, true, WriteArgs{n, slot, span_idx, n_tokens, src})) != FT_OK) return rc;
   if ((rc = ctx_release(p, cx, st)) != FT_OK) return rc;
-  mirror_write(p, n, slot, span_idx, n_tokens, t, f32);
   return end_producer(p, st);
 }
 
@@ -1208,6 +1269,12 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_free(ft_pool* p, 
 
   for (uint32_t i = 0; i < n; ++i) {
     ft_slot_mirror& s = p->slots[slot[i]];
+    if (!s.remote)  // the pages go to the ring's tail as k_free_fill pushes them: spans by index, pages by ordinal
+      for (uint32_t j = 0; j < s.n_spans; ++j)
+        for (uint32_t g : p->spans[(uint64_t)slot[i] * S + j].pages) {
+          p->h_ring[(p->h_ring_head + p->h_ring_count) % p->h_ring.size()] = g;
+          ++p->h_ring_count;
+        }
     for (uint32_t j = 0; j < s.n_spans; ++j) p->spans[(uint64_t)slot[i] * S + j] = ft_span_mirror();
     p->live_samples--; p->live_spans -= s.n_spans;
     const uint64_t gen = s.generation + 1;
@@ -1299,6 +1366,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_get_tuning(ft_poo
   out->remote_ctas = (uint32_t)p->remote_ctas; out->peers_remote = (uint32_t)p->peers_remote;
   out->scatter_smem_carveout = (uint32_t)p->scatter_smem_carveout; out->gather_smem_carveout = (uint32_t)p->gather_smem_carveout;
   out->bulk_wait_limit_us = (uint32_t)(p->view.bulk_wait_ns / 1000); out->bulk_timeout_test = p->view.bulk_tx_slack ? 1u : 0u;
+  out->host_copy_engine = (uint32_t)p->host_dma;
   return FT_OK;
 }
 
@@ -1309,11 +1377,13 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_set_tuning(ft_poo
   if (t.chunk_shift && (t.chunk_shift < 14 || t.chunk_shift > 21)) return FT_ERR_INVALID_ARG;  // a warp's eighth holds a 2 KiB batch
   if (t.gather_unroll && t.gather_unroll != 4 && t.gather_unroll != 8) return FT_ERR_INVALID_ARG;
   if (t.host_ctas > 1024 || t.host_store_ctas > 1024 || t.remote_ctas > 1024 || t.scatter_group > (1u << 20) || t.peers_remote > 1 || t.scatter_smem_carveout > 100 || t.gather_smem_carveout > 100) return FT_ERR_INVALID_ARG;
+  if (t.host_copy_engine > 1) return FT_ERR_INVALID_ARG;
   if (t.bulk_wait_limit_us && (t.bulk_wait_limit_us < 100 || t.bulk_wait_limit_us > 10000000)) return FT_ERR_INVALID_ARG;
   if (t.bulk_timeout_test > 1 || (t.bulk_timeout_test && (t.bulk_wait_limit_us == 0 || t.bulk_wait_limit_us > 100000))) return FT_ERR_INVALID_ARG;
   FT_CUDA(cudaDeviceSynchronize());  // no kernel of an earlier call is still being sized by the old values
   p->view.bulk_wait_ns = t.bulk_wait_limit_us ? (uint64_t)t.bulk_wait_limit_us * 1000 : kBulkWaitLimitNs;
   p->view.bulk_tx_slack = t.bulk_timeout_test ? 16u : 0u;
+  p->host_dma = (int)t.host_copy_engine;
   p->dev_ctas_per_sm = t.dev_ctas_per_sm ? (int)t.dev_ctas_per_sm : 4;
   p->scatter_ctas_per_sm = (int)t.scatter_ctas_per_sm;
   p->scatter_group = (int)t.scatter_group;
@@ -1506,9 +1576,10 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_write_embeddings_
   if ((rc = meta_to(p, st)) != FT_OK) return rc;
   const bool f32 = src_dtype == FT_F32;
   // the claim counters of the copy kernels sit at the end of the array; they are zero whenever no kernel uses them
-  if ((rc = launch_write_copies(p, w, t.total_chunks, f32, st, reinterpret_cast<ClaimCounter*>(db + o_counters), true)) != FT_OK) return rc;
+  mirror_write(p, n, slot, span_idx, n_tokens, t, f32);
+  if ((rc = launch_write_copies(p, w, t.total_chunks, f32, st, reinterpret_cast<ClaimCounter*>(db + o_counters), true,
+                                WriteArgs{n, slot, span_idx, n_tokens, src})) != FT_OK) return rc;
   FT_CUDA(cudaEventRecord(p->ev_noalloc, st));
   p->have_noalloc_ev = true;
-  mirror_write(p, n, slot, span_idx, n_tokens, t, f32);
   return end_producer(p, st);
 }

@@ -15,8 +15,11 @@ PLAN_KEYS = ("mb_sample_off", "mb_samples", "mb_tokens", "mb_lmax", "mb_residual
              "rank_mb_off", "rank_mbs", "sample_cost", "sample_mb")
 
 
-@pytest.mark.parametrize("seed,ring_order,page_bytes,hidden", [(0, 0, 4096, 64), (1, 1, 4096, 56), (2, 1, 16384, 1024)])
-def test_random_call_sequences_agree_with_oracle(seed, ring_order, page_bytes, hidden):
+# (copy_engine = 1: host-tier pages of writes and assemblies go through the copy engines, from the host's own copy of
+# the page ring, which the churn of this test has to keep in step with the device's)
+@pytest.mark.parametrize("seed,ring_order,page_bytes,hidden,copy_engine", [
+    (0, 0, 4096, 64, 0), (1, 1, 4096, 56, 0), (2, 1, 16384, 1024, 0), (3, 1, 4096, 64, 1), (4, 0, 16384, 1024, 1)])
+def test_random_call_sequences_agree_with_oracle(seed, ring_order, page_bytes, hidden, copy_engine):
     if not torch.cuda.is_available():
         pytest.fail("a CUDA device is required for -m gpu tests")
     from gpu_harness import cuda_stream
@@ -31,6 +34,7 @@ def test_random_call_sequences_agree_with_oracle(seed, ring_order, page_bytes, h
     f["max_text_tokens"] = w.total_text_tokens_capacity // 2
     opool, pool = OraclePool(PoolConfig(**f)), fp.Pool(fp.PoolConfig(**f))
     assert pool.rc == 0 and opool.rc == 0
+    assert pool.set_tuning(host_copy_engine=copy_engine) == 0
     table = workloads.embed_table(w, device="cuda")
     table_h = bits16(table)
     keep, plans = [], []

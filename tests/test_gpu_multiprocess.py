@@ -39,7 +39,10 @@ def test_consumer_reads_producer_pages_in_place(name, kw, peers_remote):
     g = {r: fp.Pool(fp.PoolConfig(**cfg(r))) for r in (0, 1)}
     o = {r: OraclePool(PoolConfig(**cfg(r))) for r in (0, 1)}
     assert all(p.rc == 0 for p in g.values()) and all(p.rc == 0 for p in o.values())
-    assert g[0].set_tuning(peers_remote=peers_remote, remote_ctas=3) == 0 and g[0].get_tuning()["peers_remote"] == peers_remote
+    # (with peers_remote = 1 both pools also send their own host tier through the copy engines; a plan that holds an
+    # imported sample still assembles with the kernels)
+    assert g[0].set_tuning(peers_remote=peers_remote, remote_ctas=3, host_copy_engine=peers_remote) == 0 and g[0].get_tuning()["peers_remote"] == peers_remote
+    assert g[1].set_tuning(host_copy_engine=peers_remote) == 0
     g[0].profile_enable(True)
     keep = []
 

@@ -14,11 +14,12 @@ from oracle import OraclePool, PlanConfig, PoolConfig
 pytestmark = pytest.mark.gpu
 
 
+@pytest.mark.parametrize("copy_engine", [0, 1])   # 1: the host tier through the copy engines, both directions at once
 @pytest.mark.parametrize("name,kw,group", [
     ("image_mix_7b", dict(n_samples=48, hidden=512, page_bytes=65536), 8),
     ("host_tier_stress", dict(n_samples=12, hidden=1024, page_bytes=65536), 3),
 ])
-def test_overlapped_write_and_gather_match_sequential_oracle(name, kw, group):
+def test_overlapped_write_and_gather_match_sequential_oracle(name, kw, group, copy_engine):
     if not torch.cuda.is_available():
         pytest.fail("a CUDA device is required for -m gpu tests")
     from paper_2606_23087_b200 import binding as fp
@@ -29,6 +30,7 @@ def test_overlapped_write_and_gather_match_sequential_oracle(name, kw, group):
     f["hbm_pages"], f["host_pages"] = (cap + 1) // 2, cap // 2
     pool, opool = fp.Pool(fp.PoolConfig(**f)), OraclePool(PoolConfig(**f))
     assert pool.rc == 0 and opool.rc == 0
+    assert pool.set_tuning(host_copy_engine=copy_engine) == 0
     prod, cons = torch.cuda.Stream(), torch.cuda.Stream()
     table = workloads.embed_table(w, device="cuda")
     table_h = bits16(table)

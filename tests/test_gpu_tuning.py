@@ -20,6 +20,8 @@ TUNINGS = [
     dict(dev_ctas_per_sm=8, scatter_ctas_per_sm=8, scatter_group=5, chunk_shift=14),
     dict(chunk_shift=21, host_ctas=1, host_store_ctas=1, scatter_smem_carveout=30, gather_smem_carveout=30),
     dict(host_ctas=13, host_store_ctas=17, scatter_group=2, chunk_shift=18),
+    dict(host_copy_engine=1),                      # host-tier pages by cudaMemcpyAsync runs instead of the bulk-copy kernels
+    dict(host_copy_engine=1, chunk_shift=14, dev_ctas_per_sm=2),
 ]
 
 
@@ -51,7 +53,7 @@ def test_tuning_round_trip_and_range_checks():
     assert (d["dev_ctas_per_sm"], d["scatter_ctas_per_sm"], d["chunk_shift"], d["host_ctas"], d["gather_unroll"]) == (4, 4, 0, 6, 4)   # chunk_shift 0: chosen per call
     assert d["scatter_smem_carveout"] == 5 and d["gather_smem_carveout"] == 0 and d["remote_ctas"] == 16
     for bad in (dict(chunk_shift=13), dict(chunk_shift=22), dict(gather_unroll=6), dict(dev_ctas_per_sm=9), dict(peers_remote=2),
-                dict(scatter_smem_carveout=101)):
+                dict(scatter_smem_carveout=101), dict(host_copy_engine=3)):
         assert pool.set_tuning(**bad) == -1 and pool.get_tuning() == d          # INVALID_ARG, nothing changed
     assert pool.set_tuning(host_ctas=3, chunk_shift=17) == 0
     t = pool.get_tuning()
