@@ -268,7 +268,8 @@ struct ft_span_mirror {
   uint32_t grid[3] = {0, 0, 0};  // token grid (T, H, W) as last set; all zero = none
   bool written = false;
   uint64_t named = 0;   // call_seq of the write call that last named this span
-  std::vector<uint32_t> pages;  // global page index by ordinal (own written spans; the host's copy of the page list)
+  // the host's copy of the page list of an own written span: a chain through ft_pool::h_page_next (no allocation per write)
+  uint32_t first_page = 0xFFFFFFFFu, owned_pages = 0;
 };
 
 // Per-call context: the descriptors of one ABI call travel host -> device through one of a small ring of these.
@@ -335,6 +336,7 @@ struct ft_pool {
   // the copy-engine path of the host tier; the device's ring stays the one the kernels read.
   std::vector<uint32_t> h_ring;
   uint64_t h_ring_head = 0, h_ring_count = 0;
+  std::vector<uint32_t> h_page_next;  // [pages] the page that follows in the same span's list
   int host_dma = 0;             // 1: host-tier pages of bf16 writes and of assemblies go through the copy engines
   void* d_text_base() const { return d_text; }
   std::vector<void*> peer_allocs;                      // imported peers' page-table arrays
@@ -494,6 +496,22 @@ inline int32_t end_producer(ft_pool* p, cudaStream_t st) {
   FT_CUDA(cudaEventRecord(p->ev_producer, st));
   p->have_producer_ev = true;
   return FT_OK;
+}
+// The host-tier runs of an own span, from the host's copy of its page list: maximal sequences of pages that follow one
+// another in the span's image and in the host slab.  fn(byte offset in the image, first frame, bytes).
+template <class F>
+inline void for_each_host_run(const ft_pool* p, const ft_span_mirror& m, uint64_t image_bytes, F&& fn) {
+  const uint64_t PS = p->cfg.page_bytes, hbm = p->cfg.hbm_pages;
+  uint32_t g = m.first_page;
+  for (uint32_t k = 0; k < m.owned_pages;) {
+    if (g < hbm) { g = p->h_page_next[g]; ++k; continue; }
+    const uint64_t frame = p->bind_host[g - hbm];
+    uint32_t k1 = k + 1, g1 = p->h_page_next[g];
+    while (k1 < m.owned_pages && g1 >= hbm && p->bind_host[g1 - hbm] == frame + (k1 - k)) { g1 = p->h_page_next[g1]; ++k1; }
+    const uint64_t off = (uint64_t)k * PS;
+    fn(off, frame, (image_bytes < (uint64_t)k1 * PS ? image_bytes : (uint64_t)k1 * PS) - off);
+    k = k1; g = g1;
+  }
 }
 inline int32_t plan_alive(const ft_pool* p, const ft_plan* pl) {
   if (pl->free_epoch != p->free_epoch || (pl->cfg.flags & FT_PLAN_ALLOW_UNWRITTEN)) {

@@ -779,7 +779,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_plan_microbatches
   if (want_copies) {
     // the plan's host-tier pages as copy-engine work, from the host's page lists, in plan order
     const uint32_t* order = reinterpret_cast<const uint32_t*>(rb + rb_ms);
-    const uint64_t PS = p->cfg.page_bytes, hbm = p->cfg.hbm_pages;
+    const uint64_t PS = p->cfg.page_bytes;
     const uint32_t S = p->cfg.max_spans_per_sample;
     const uint8_t* base = static_cast<const uint8_t*>(p->host_base);
     pl->mb_copy_off.assign(pl->n_mb + 1, 0);
@@ -792,16 +792,9 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_plan_microbatches
         if (sm.remote) { ok = false; break; }  // an imported sample: its pages are a peer's, the kernels read them
         for (uint32_t js = 0; js < sm.n_spans; ++js) {
           const ft_span_mirror& m = p->spans[(uint64_t)slot_q * S + js];
-          const uint64_t bytes = (uint64_t)m.tokens * p->view.row_bytes;
-          for (uint32_t k = 0; k < (uint32_t)m.pages.size();) {
-            if (m.pages[k] < hbm) { ++k; continue; }
-            const uint64_t frame = p->bind_host[m.pages[k] - hbm];
-            uint32_t k1 = k + 1;
-            while (k1 < m.pages.size() && m.pages[k1] >= hbm && p->bind_host[m.pages[k1] - hbm] == frame + (k1 - k)) ++k1;
-            const uint64_t off = (uint64_t)k * PS;
-            pl->host_copies.push_back({row + m.pos, off, base + frame * PS, std::min<uint64_t>(bytes, (uint64_t)k1 * PS) - off});
-            k = k1;
-          }
+          for_each_host_run(p, m, (uint64_t)m.tokens * p->view.row_bytes, [&](uint64_t off, uint64_t frame, uint64_t len) {
+            pl->host_copies.push_back({row + m.pos, off, base + frame * PS, len});
+          });
         }
         row += sm.seq_len;
       }

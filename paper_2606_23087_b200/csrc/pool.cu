@@ -554,23 +554,18 @@ bool host_tier_by_copy_engine(const ft_pool* p) {
 // bf16 sources into host-tier pages through the copy engine: one copy per run of pages that follow one another both
 // in the span's image and in the host slab.  The pages come from the host's copy of the page lists (mirror_write ran).
 static int32_t dma_write_host_pages(ft_pool* p, const WriteArgs& a, cudaStream_t s) {
-  const uint64_t PS = p->cfg.page_bytes, hbm = p->cfg.hbm_pages;
+  const uint64_t PS = p->cfg.page_bytes;
   const uint32_t S = p->cfg.max_spans_per_sample;
   uint8_t* base = static_cast<uint8_t*>(p->host_base);
+  cudaError_t err = cudaSuccess;
   for (uint32_t q = 0; q < a.n; ++q) {
     const ft_span_mirror& m = p->spans[(uint64_t)a.slot[q] * S + a.span_idx[q]];
-    const uint64_t bytes = (uint64_t)a.n_tokens[q] * p->view.row_bytes;
     const uint8_t* src = static_cast<const uint8_t*>(a.src[q]);
-    for (uint32_t k = 0; k < m.npages;) {
-      if (m.pages[k] < hbm) { ++k; continue; }
-      const uint64_t frame = p->bind_host[m.pages[k] - hbm];
-      uint32_t k1 = k + 1;
-      while (k1 < m.npages && m.pages[k1] >= hbm && p->bind_host[m.pages[k1] - hbm] == frame + (k1 - k)) ++k1;
-      const uint64_t off = (uint64_t)k * PS, len = std::min<uint64_t>(bytes, (uint64_t)k1 * PS) - off;
-      FT_CUDA(cudaMemcpyAsync(base + frame * PS, src + off, len, cudaMemcpyDeviceToHost, s));
-      k = k1;
-    }
+    for_each_host_run(p, m, (uint64_t)a.n_tokens[q] * p->view.row_bytes, [&](uint64_t off, uint64_t frame, uint64_t len) {
+      if (err == cudaSuccess) err = cudaMemcpyAsync(base + frame * PS, src + off, len, cudaMemcpyDeviceToHost, s);
+    });
   }
+  if (err != cudaSuccess) return cuda_fail(err, "cudaMemcpyAsync(host-tier pages)");
   return FT_OK;
 }
 
@@ -961,6 +956,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_create(const ft_p
   CK(cudaFree(d_tmp));
   p->bind_hbm = bind_h; p->bind_host = bind_d;
   p->h_ring = ring; p->h_ring_head = 0; p->h_ring_count = P;
+  p->h_page_next.assign(P, kNone);
   p->gpu_launches += 5;
 #undef CK
   p->slots.resize(c.max_samples);
@@ -1130,11 +1126,14 @@ static void mirror_write(ft_pool* p, uint32_t n, const uint32_t* slot, const uin
     ft_slot_mirror& s = p->slots[slot[q]];
     ft_span_mirror& m = p->spans[(uint64_t)slot[q] * S + span_idx[q]];
     m.written = true; m.npages = (uint32_t)pages_for_tokens(p, n_tokens[q]);
-    m.pages.resize(m.npages);  // the ring's next entries, as k_alloc_fill takes them
+    uint32_t prev = kNone;  // the ring's next entries, as k_alloc_fill takes them, chained in order
     for (uint32_t k = 0; k < m.npages; ++k) {
-      m.pages[k] = p->h_ring[p->h_ring_head];
+      const uint32_t g = p->h_ring[p->h_ring_head];
       p->h_ring_head = (p->h_ring_head + 1) % p->h_ring.size();
+      if (prev == kNone) m.first_page = g; else p->h_page_next[prev] = g;
+      prev = g;
     }
+    m.owned_pages = m.npages;
     p->h_ring_count -= m.npages;
     if (++s.spans_written == s.n_spans) { s.state = FT_SLOT_READY; ready_push(p, slot[q]); }
   }
@@ -1271,10 +1270,15 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_free(ft_pool* p, 
     ft_slot_mirror& s = p->slots[slot[i]];
     if (!s.remote)  // the pages go to the ring's tail as k_free_fill pushes them: spans by index, pages by ordinal
       for (uint32_t j = 0; j < s.n_spans; ++j)
-        for (uint32_t g : p->spans[(uint64_t)slot[i] * S + j].pages) {
+      {
+        const ft_span_mirror& m = p->spans[(uint64_t)slot[i] * S + j];
+        uint32_t g = m.first_page;
+        for (uint32_t k = 0; k < m.owned_pages; ++k) {
           p->h_ring[(p->h_ring_head + p->h_ring_count) % p->h_ring.size()] = g;
           ++p->h_ring_count;
+          g = p->h_page_next[g];
         }
+      }
     for (uint32_t j = 0; j < s.n_spans; ++j) p->spans[(uint64_t)slot[i] * S + j] = ft_span_mirror();
     p->live_samples--; p->live_spans -= s.n_spans;
     const uint64_t gen = s.generation + 1;
