@@ -768,6 +768,7 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_plan_microbatches
     if ((rc = copy_words(rbd + rb_so, pl->d_mb_sample_off, n1, st)) != FT_OK) { plan_destroy(pl); return rc; }
     if ((rc = copy_words(rbd + rb_ro, pl->d_mb_row_off, n1 * 2, st)) != FT_OK) { plan_destroy(pl); return rc; }
     if (want_copies && (rc = copy_words(rbd + rb_ms, pl->d_mb_samples, n, st)) != FT_OK) { plan_destroy(pl); return rc; }
+    p->gpu_launches += want_copies ? 5 : 4;  // these and the copy of the slot list into the plan
   }
   CK(cudaStreamSynchronize(st));
   const uint32_t* sc = reinterpret_cast<const uint32_t*>(rb + rb_sc);

@@ -104,6 +104,7 @@ int32_t ctx_upload(ft_pool* p, ft_call_ctx* c, size_t bytes) {
   if (bytes) {
     const int32_t rc = copy_words(c->d, c->hd, (bytes + 3) / 4, p->meta);
     if (rc != FT_OK) return rc;
+    p->gpu_launches++;
     FT_CUDA(cudaEventRecord(c->ev_up, p->meta));
     c->busy_up = true;
   }
