@@ -41,6 +41,26 @@ def test_results_do_not_depend_on_the_launch_geometry(name, kw, tuning):
     assert not np.any(np.all(got["out"] == 0xFFFF, axis=1))
 
 
+@pytest.mark.parametrize("name,kw", [
+    ("image_mix_7b", dict(n_samples=10, hidden=512, page_bytes=16384)),     # spans of several pages each
+    ("image_mix_7b", dict(n_samples=6)),                                     # 2 MiB pages, 7 KiB rows
+])
+def test_copy_engine_runs_over_contiguous_host_frames(name, kw):
+    """With an identity binding and the sorted ring, the host-tier pages of a span are consecutive frames, so the
+    copy-engine path merges them into one copy per run (with the permuted binding of the other cases every run is
+    one page).  Written and assembled that way, the result must equal the oracle bit for bit."""
+    if not torch.cuda.is_available():
+        pytest.fail("a CUDA device is required for -m gpu tests")
+    from gpu_harness import run_cuda
+    w = workloads.make_workload(name, **kw)
+    w.bind_order = 0
+    assert w.ring_order == 0 and w.host_pages > 0
+    got = run_cuda(w, tuning=dict(host_copy_engine=1))
+    exp = oracle_from_device_sources(w, got["srcs"], got["table"])
+    assert_same(got, exp)
+    assert not np.any(np.all(got["out"] == 0xFFFF, axis=1))
+
+
 def test_tuning_round_trip_and_range_checks():
     if not torch.cuda.is_available():
         pytest.fail("a CUDA device is required for -m gpu tests")
