@@ -248,6 +248,8 @@ class DeviceJob:
         from paper_2606_23087_b200 import binding as fp
         self.torch, self.fp = torch, fp
         w = workloads.make_workload(args.workload, n_samples=args.samples, all_hbm=all_hbm, id_skew=getattr(args, "id_skew", "uniform"))
+        if getattr(args, "bind_order", "workload") == "identity":
+            w.bind_order = 0      # virtual page k lives in frame k: a span's consecutive pages are contiguous in the slab
         self.w = w
         self.pool = fp.Pool(fp.PoolConfig(**pool_config_fields(w)))
         if self.pool.rc != 0:
@@ -888,6 +890,7 @@ def run_ours(args):
             "config": {"workload": workload_label(args), "samples": w.n_samples, "packed_tokens": w.total_tokens,
                        "vision_tokens": w.total_vision_tokens, "microbatches": n_mb, "hbm_pages": w.hbm_pages,
                        "host_pages": w.host_pages,
+                       "bind_order": "identity" if w.bind_order == 0 else "seeded permutation", "tuning": args.tuning,
                        "host_tier_bytes_per_step": {"min": int(min(hb)), "mean": float(np.mean(hb)), "max": int(max(hb)),
                                                     "ring_model_matches_pool": job.ring_ok,
                                                     "note": "the free ring rotates from step to step (pool = 1.02 x one batch), so the bytes "
@@ -1691,6 +1694,8 @@ def main():
     ap.add_argument("--cycles", type=int, default=10, help="frag_sweep: write/free cycles")
     ap.add_argument("--tuning", default=None, help="library launch-geometry knobs, e.g. dev_ctas_per_sm=4,host_ctas=6")
     ap.add_argument("--id-skew", default="uniform", choices=["uniform", "zipf"], help="distribution of the text-token ids")
+    ap.add_argument("--bind-order", default="workload", choices=["workload", "identity"],
+                    help="vpn -> frame binding of the main pool: the workload's (a seeded permutation) or the identity")
     ap.add_argument("--backbone-only", action="store_true", help="only the backbone-side outputs (padded assembly, table gradient) on an all-HBM pool")
     ap.add_argument("--exchange", action="store_true", help="under torchrun: every rank writes its batch, all plan everything, each assembles its own share from everybody's pages")
     ap.add_argument("--two-processes", action="store_true", help="with --via-peer: the producer pool lives in a process of its own (CUDA IPC)")
