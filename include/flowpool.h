@@ -471,7 +471,9 @@ int32_t pool_profile_read(ft_pool* pool, ft_kernel_time* out /* host [FT_K_COUNT
  * pool_set_tuning replaces them (0 in a field = that field's built-in default, the optimum measured on a B200);
  * out-of-range values INVALID_ARG and nothing changes.  Call it between other calls of the pool; it synchronises
  * the device.  None of the knobs changes any result (bulk_timeout_test, a test hook, excepted).
- *   dev_ctas_per_sm      resident CTAs per SM of the HBM-tier gather kernel (default 4; 1..8)
+ *   dev_ctas_per_sm      resident CTAs per SM of the HBM-tier gather kernel (1..8).  Default 0 = chosen per launch
+ *                        together with gather_unroll: 4 CTAs x 4 vectors for a range of one wave or rows under 4 KiB,
+ *                        2 CTAs x 8 vectors for longer ranges
  *   scatter_ctas_per_sm  resident CTAs per SM of the HBM-tier scatter kernel (default 4; 1..8)
  *   scatter_group        chunks a scatter CTA claims at a time (default 1)
  *   chunk_shift          log2 of the scatter's work unit in bytes of a span's image (14..21).  Default 0 = chosen per
@@ -481,7 +483,7 @@ int32_t pool_profile_read(ft_pool* pool, ft_kernel_time* out /* host [FT_K_COUNT
  *   host_ctas            grid of the host-tier bulk-copy kernels (default 6): few SMs, so that long-latency host-link
  *                        accesses do not clog the memory pipelines of the SMs that stream HBM
  *   host_store_ctas      grid of the vector-store scatter into host frames (fp32 sources, host-only pools; default 8)
- *   gather_unroll        16-byte vectors per lane in flight in the gather kernel (4 or 8; default 4)
+ *   gather_unroll        16-byte vectors per lane in flight in the gather kernel (4 or 8; default 0 = see above)
  *   grad_ctas_per_sm     CTAs per SM of the table-gradient kernel (default 6; 1..8)
  *   grad_hot_threshold   rows from which an id takes the frequent-id gradient kernel (default rows / (8 x grid), >= 64)
  *   remote_ctas          grid of the bulk-copy gather that reads frames in ANOTHER GPU's HBM (default 16): like the

@@ -373,8 +373,8 @@ struct ft_pool {
   bool grad_attr_set = false;   // k_embed_grad_hot's shared-memory opt-in done
   int grad_hot_threshold = 0;   // rows from which an id takes k_embed_grad_hot; 0 = rows / (8 x grid), at least 64
   int grad_ctas_per_sm = 6;     // CTAs per SM of k_embed_grad (each owns the table rows v with v % grid == its index)
-  int gather_unroll = 4;        // 16-byte vectors per lane in flight in k_gather (4 or 8)
-  int dev_ctas_per_sm = 4;      // resident CTAs per SM of the device-tier gather kernel (measured optimum 3-5)
+  int gather_unroll = 0;        // 16-byte vectors per lane in flight in k_gather (4 or 8); 0 = chosen per launch
+  int dev_ctas_per_sm = 0;      // resident CTAs per SM of the device-tier gather kernel; 0 = chosen per launch
   // optional kernel timing (pool_profile_*)
   bool profiling = false;
   struct prof_rec { int kind; cudaEvent_t e0, e1; };

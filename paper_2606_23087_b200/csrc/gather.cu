@@ -421,7 +421,16 @@ int32_t gather_launch(ft_pool* p, const ft_plan* pl, uint32_t mb_begin, uint32_t
   // CTA: the latency floor).  Any longer range is cut into units of 8 or 16 rows (one or two rows per copy warp) as
   // long as a unit still streams 48 KiB and more, so that the resolver keeps ahead of the copy: finer units balance
   // the CTAs of an SM and shorten the last wave (6.80 against 6.68 TB/s on a 2.6 M-row range with 7 KiB rows).
-  const uint64_t per_sm_cap = (p->cfg.hbm_pages == 0 && p->cfg.world_size == 1) ? 1 : (uint64_t)p->dev_ctas_per_sm;
+  // Launch geometry when the tuning leaves it open: a range of one wave keeps 4 CTAs per SM with 4 vectors per lane
+  // in flight (more, smaller units: the latency floor); a longer range of rows of 4 KiB and more streams a little
+  // better from 2 CTAs per SM with 8 vectors per lane (the same bytes in flight per SM from half the warps: 6.85
+  // against 6.80 TB/s on the long range, 6.26 against 6.15 for one call per microbatch).
+  // (Beside a bulk-copy launch for host or remote frames the device-tier launch keeps 4 x 4: 6.70 against 6.57 TB/s.)
+  const bool one_launch = !(p->cfg.host_pages != 0 || p->peer_host_frames || p->peer_remote_frames);
+  const bool long_range = one_launch && n_tiles > (uint64_t)p->sm_count * 4 && p->view.row_bytes >= 4096;
+  const int want_ctas = p->dev_ctas_per_sm ? p->dev_ctas_per_sm : (long_range ? 2 : 4);
+  const int unroll = p->gather_unroll ? p->gather_unroll : (long_range ? 8 : 4);
+  const uint64_t per_sm_cap = (p->cfg.hbm_pages == 0 && p->cfg.world_size == 1) ? 1 : (uint64_t)want_ctas;
   const uint64_t full_grid = (uint64_t)p->sm_count * per_sm_cap;
   a.sub_shift = 0;
   if (n_tiles <= full_grid) {
@@ -431,13 +440,13 @@ int32_t gather_launch(ft_pool* p, const ft_plan* pl, uint32_t mb_begin, uint32_t
   }
   const uint64_t n_units = n_tiles << a.sub_shift;
   auto launch = [&](auto kernel, int mode, uint64_t want_per_sm, const GatherArgs& args, cudaStream_t s) {
-    const uint64_t resident = (uint64_t)std::max(1, p->occ_gather[mode][p->gather_unroll == 8 ? 1 : 0]);
+    const uint64_t resident = (uint64_t)std::max(1, p->occ_gather[mode][unroll == 8 ? 1 : 0]);
     const uint64_t ctas = (uint64_t)p->sm_count * std::min<uint64_t>(want_per_sm, resident);
     kernel<<<(unsigned)std::min<uint64_t>(n_units, ctas), kGatherThreads, 0, s>>>(p->view, pv, args);
   };
   auto launch_mode = [&](auto mode_tag, const GatherArgs& args, uint64_t want_per_sm) {
     constexpr int M = decltype(mode_tag)::value;
-    const bool u8 = p->gather_unroll == 8;
+    const bool u8 = unroll == 8;
     if (listed) {
       if (u8) launch(k_gather<M, 8, true>, M, want_per_sm, args, st); else launch(k_gather<M, 4, true>, M, want_per_sm, args, st);
     } else {

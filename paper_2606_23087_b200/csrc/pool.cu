@@ -1389,13 +1389,13 @@ extern "C" __attribute__((visibility("default"))) int32_t pool_set_tuning(ft_poo
   p->view.bulk_wait_ns = t.bulk_wait_limit_us ? (uint64_t)t.bulk_wait_limit_us * 1000 : kBulkWaitLimitNs;
   p->view.bulk_tx_slack = t.bulk_timeout_test ? 16u : 0u;
   p->host_dma = (int)t.host_copy_engine;
-  p->dev_ctas_per_sm = t.dev_ctas_per_sm ? (int)t.dev_ctas_per_sm : 4;
+  p->dev_ctas_per_sm = (int)t.dev_ctas_per_sm;
   p->scatter_ctas_per_sm = (int)t.scatter_ctas_per_sm;
   p->scatter_group = (int)t.scatter_group;
   p->chunk_shift = (int)t.chunk_shift;
   p->host_ctas = t.host_ctas ? (int)t.host_ctas : 6;
   p->host_store_ctas = t.host_store_ctas ? (int)t.host_store_ctas : 8;
-  p->gather_unroll = t.gather_unroll ? (int)t.gather_unroll : 4;
+  p->gather_unroll = (int)t.gather_unroll;
   p->grad_ctas_per_sm = t.grad_ctas_per_sm ? (int)t.grad_ctas_per_sm : 6;
   p->grad_hot_threshold = (int)t.grad_hot_threshold;
   p->remote_ctas = t.remote_ctas ? (int)t.remote_ctas : 16;

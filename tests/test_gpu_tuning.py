@@ -70,14 +70,14 @@ def test_tuning_round_trip_and_range_checks():
     pool = fp.Pool(fp.PoolConfig(**pool_config_fields(w)))
     assert pool.rc == 0
     d = pool.get_tuning()
-    assert (d["dev_ctas_per_sm"], d["scatter_ctas_per_sm"], d["chunk_shift"], d["host_ctas"], d["gather_unroll"]) == (4, 4, 0, 6, 4)   # chunk_shift 0: chosen per call
+    assert (d["dev_ctas_per_sm"], d["scatter_ctas_per_sm"], d["chunk_shift"], d["host_ctas"], d["gather_unroll"]) == (0, 4, 0, 6, 0)   # 0: chosen per call or per launch
     assert d["scatter_smem_carveout"] == 5 and d["gather_smem_carveout"] == 0 and d["remote_ctas"] == 16
     for bad in (dict(chunk_shift=13), dict(chunk_shift=22), dict(gather_unroll=6), dict(dev_ctas_per_sm=9), dict(peers_remote=2),
                 dict(scatter_smem_carveout=101), dict(host_copy_engine=3)):
         assert pool.set_tuning(**bad) == -1 and pool.get_tuning() == d          # INVALID_ARG, nothing changed
     assert pool.set_tuning(host_ctas=3, chunk_shift=17) == 0
     t = pool.get_tuning()
-    assert t["host_ctas"] == 3 and t["chunk_shift"] == 17 and t["dev_ctas_per_sm"] == 4   # unnamed knobs go back to their defaults
+    assert t["host_ctas"] == 3 and t["chunk_shift"] == 17 and t["dev_ctas_per_sm"] == 0   # unnamed knobs go back to their defaults
     assert pool.set_tuning() == 0 and pool.get_tuning() == d
     pool.destroy()
 
